@@ -1,0 +1,348 @@
+/*
+ * CPU oracle for the fused residual-add + RMSNorm operator.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain, obviously-correct
+ * statement of what the operator computes.  It is used by the tests, by the
+ * smoke check and by the CPU-baseline leg of the benchmark.  The product (the
+ * CUDA library) never links, imports or calls it, and it shares no code,
+ * header, table or helper with the CUDA path.
+ *
+ * What is computed, per token row t (rows are independent):
+ *
+ *   s_j   = fl32(x_j) + fl32(r_j)            one IEEE binary32 addition (RNE)
+ *   r'_j  = RNE_dtype(s_j)                   written to r_out, bit-exact contract
+ *   ms    = (1/H) * sum_j s_j^2              fp64, plain left-to-right
+ *   y_j   = RNE_dtype( s_j * w_j / sqrt(ms + eps) )   fp64, ONE final rounding
+ *
+ * The operator is the `fused_add_rmsnorm` kernel named in the paper's
+ * "Kernels" paragraph (Experimental Setup); the paper prints no formula, so the
+ * formula above is the standard residual-add + RMSNorm definition with eps
+ * inside the square root and a division by H (no mean subtraction).  The
+ * correctness criterion it serves is the paper's "Correctness" paragraph
+ * (max over the test set of d(S~(x), S(x)) <= eps_tol, element-wise).
+ *
+ * Readings taken where the definition leaves a choice:
+ *   - the normalisation uses the UN-ROUNDED fp32 sum s_j; the switch
+ *     `norm_from_rounded` selects the other reading (r'_j decoded back) so a
+ *     test can bound the difference;
+ *   - eps arrives as a binary32 scalar and is widened exactly to fp64;
+ *   - y is rounded directly from fp64 to the output type (gradual underflow,
+ *     overflow to infinity), not through binary32.
+ *
+ * Pins (tests/test_oracle_*.py): closed forms (constant row, one-hot row,
+ * x = -r, +-1 row, power-of-two scale invariance), exact rational brute force
+ * on tiny shapes, exhaustive codec checks over all 65 536 16-bit patterns
+ * against a library conversion and against an exact-fraction bracket search,
+ * and a float64 library evaluation of the same formula.  No function here is
+ * "parity unpinned".
+ *
+ * Plain C99 + pthreads (threads only split independent rows).  Build:
+ *   gcc -O2 -fno-fast-math -ffp-contract=off -shared -fPIC -pthread \
+ *       add_rmsnorm_oracle.c -o libadd_rmsnorm_oracle.so -lm
+ */
+#include <math.h>
+#include <pthread.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+enum { ORACLE_BF16 = 0, ORACLE_FP16 = 1, ORACLE_FP32 = 2 };
+
+/* ---- number formats ------------------------------------------------------ */
+
+typedef struct {
+    int ebits; /* exponent field width */
+    int mbits; /* stored significand bits */
+} fmt16;
+
+static const fmt16 FMT_BF16 = {8, 7};
+static const fmt16 FMT_FP16 = {5, 10};
+
+/* Exact value of a 16-bit floating-point pattern, as a double. */
+static double decode16(uint16_t bits, fmt16 f)
+{
+    const int emax_field = (1 << f.ebits) - 1;
+    const int bias = (1 << (f.ebits - 1)) - 1;
+    const int sign = bits >> 15;
+    const int e = (bits >> f.mbits) & emax_field;
+    const int m = bits & ((1 << f.mbits) - 1);
+    double v;
+    if (e == emax_field)
+        v = m ? NAN : INFINITY;
+    else if (e == 0)
+        v = ldexp((double)m, 1 - bias - f.mbits); /* zero and subnormals */
+    else
+        v = ldexp((double)(m | (1 << f.mbits)), e - bias - f.mbits);
+    return sign ? -v : v;
+}
+
+/*
+ * Round a double to the nearest value of a 16-bit format, ties to even, with
+ * gradual underflow and overflow to infinity.  One rounding, done on integers:
+ * the value is scaled by an exact power of two so that one unit of the target
+ * format's last place becomes 1, then rounded to an integer.
+ */
+static uint16_t encode16(double d, fmt16 f)
+{
+    const int emax_field = (1 << f.ebits) - 1;
+    const int bias = (1 << (f.ebits - 1)) - 1;
+    const uint32_t inf_bits = (uint32_t)emax_field << f.mbits;
+    const uint16_t sign = signbit(d) ? 0x8000u : 0u;
+    if (isnan(d))
+        return (uint16_t)(sign | inf_bits | (1u << (f.mbits - 1)));
+    double a = fabs(d);
+    if (isinf(a))
+        return (uint16_t)(sign | inf_bits);
+    if (a == 0.0)
+        return sign;
+
+    int e2;
+    (void)frexp(a, &e2);       /* a = m * 2^e2 with m in [0.5, 1) */
+    const int E = e2 - 1;      /* a in [2^E, 2^(E+1)) */
+    const int emin = 1 - bias; /* smallest normal exponent */
+    const int q = (E < emin ? emin : E) - f.mbits; /* exponent of one ulp */
+    const double scaled = ldexp(a, -q);            /* exact */
+    const double lo = floor(scaled);
+    const double rem = scaled - lo; /* exact, in [0, 1) */
+    uint64_t n = (uint64_t)lo;
+    if (rem > 0.5 || (rem == 0.5 && (n & 1u)))
+        n += 1;
+
+    uint32_t bits;
+    if (E < emin)
+        bits = (uint32_t)n; /* subnormal; n == 2^mbits is the smallest normal */
+    else if (E + bias >= emax_field)
+        bits = inf_bits;
+    else
+        bits = ((uint32_t)(E + bias) << f.mbits) + (uint32_t)(n - (1ull << f.mbits));
+    if (bits > inf_bits)
+        bits = inf_bits;
+    return (uint16_t)(sign | bits);
+}
+
+/* ---- exported codec entry points (used by the pins) ---------------------- */
+
+void oracle_decode16(const uint16_t* bits, double* out, int64_t n, int dtype)
+{
+    const fmt16 f = dtype == ORACLE_BF16 ? FMT_BF16 : FMT_FP16;
+    for (int64_t i = 0; i < n; ++i) out[i] = decode16(bits[i], f);
+}
+
+void oracle_encode16_from_f64(const double* v, uint16_t* out, int64_t n, int dtype)
+{
+    const fmt16 f = dtype == ORACLE_BF16 ? FMT_BF16 : FMT_FP16;
+    for (int64_t i = 0; i < n; ++i) out[i] = encode16(v[i], f);
+}
+
+/* binary32 -> 16-bit: a binary32 value is exactly a double, so one rounding. */
+void oracle_encode16_from_f32(const float* v, uint16_t* out, int64_t n, int dtype)
+{
+    const fmt16 f = dtype == ORACLE_BF16 ? FMT_BF16 : FMT_FP16;
+    for (int64_t i = 0; i < n; ++i) out[i] = encode16((double)v[i], f);
+}
+
+/* ---- the operator ---------------------------------------------------------- */
+
+typedef struct {
+    const void *x, *r, *w;
+    void *y, *r_out;
+    int64_t row_begin, row_end, hidden;
+    double eps;
+    int dtype, norm_from_rounded;
+    int status;
+} row_job;
+
+static void run_rows(row_job* job)
+{
+    const int64_t H = job->hidden;
+    double* s = (double*)malloc((size_t)H * sizeof(double));
+    if (!s) {
+        job->status = 2;
+        return;
+    }
+    for (int64_t t = job->row_begin; t < job->row_end; ++t) {
+        const int64_t base = t * H;
+        double acc = 0.0;
+        /* residual add in binary32, then the bit-exact rounded residual. */
+        for (int64_t j = 0; j < H; ++j) {
+            float xf, rf;
+            if (job->dtype == ORACLE_FP32) {
+                xf = ((const float*)job->x)[base + j];
+                rf = ((const float*)job->r)[base + j];
+            } else {
+                const fmt16 f = job->dtype == ORACLE_BF16 ? FMT_BF16 : FMT_FP16;
+                xf = (float)decode16(((const uint16_t*)job->x)[base + j], f);
+                rf = (float)decode16(((const uint16_t*)job->r)[base + j], f);
+            }
+            const float s32 = xf + rf; /* one binary32 addition, RNE */
+            double used = (double)s32;
+            if (job->dtype == ORACLE_FP32) {
+                ((float*)job->r_out)[base + j] = s32;
+            } else {
+                const fmt16 f = job->dtype == ORACLE_BF16 ? FMT_BF16 : FMT_FP16;
+                const uint16_t rb = encode16((double)s32, f);
+                ((uint16_t*)job->r_out)[base + j] = rb;
+                if (job->norm_from_rounded)
+                    used = decode16(rb, f);
+            }
+            s[j] = used;
+            acc += used * used; /* fp64, left to right */
+        }
+        const double ms = acc / (double)H;
+        const double denom = sqrt(ms + job->eps);
+        for (int64_t j = 0; j < H; ++j) {
+            double wj;
+            if (job->dtype == ORACLE_FP32) {
+                wj = (double)((const float*)job->w)[j];
+            } else {
+                const fmt16 f = job->dtype == ORACLE_BF16 ? FMT_BF16 : FMT_FP16;
+                wj = decode16(((const uint16_t*)job->w)[j], f);
+            }
+            const double y64 = s[j] * wj / denom;
+            if (job->dtype == ORACLE_FP32) {
+                ((float*)job->y)[base + j] = (float)y64; /* RNE to binary32 */
+            } else {
+                const fmt16 f = job->dtype == ORACLE_BF16 ? FMT_BF16 : FMT_FP16;
+                ((uint16_t*)job->y)[base + j] = encode16(y64, f);
+            }
+        }
+    }
+    free(s);
+    job->status = 0;
+}
+
+static void* thread_main(void* arg)
+{
+    run_rows((row_job*)arg);
+    return NULL;
+}
+
+/*
+ * x, r, y, r_out: [n_tokens, hidden] row-major, contiguous; w: [hidden].
+ * All buffers are host memory of element type `dtype`.  y and r_out must not
+ * alias the inputs here (the oracle is not an in-place routine).
+ * n_threads <= 1 runs in the calling thread; otherwise rows are split into
+ * contiguous blocks, one per thread.  Returns 0, or 1 for a bad argument,
+ * 2 for an allocation failure.
+ */
+int oracle_add_rmsnorm(const void* x, const void* r, const void* w, void* y, void* r_out,
+                       int64_t n_tokens, int64_t hidden, float eps, int dtype,
+                       int norm_from_rounded, int n_threads)
+{
+    if (n_tokens < 0 || hidden <= 0 || dtype < 0 || dtype > 2) return 1;
+    if (n_tokens == 0) return 0;
+    if (!x || !r || !w || !y || !r_out) return 1;
+    if (n_threads < 1) n_threads = 1;
+    if ((int64_t)n_threads > n_tokens) n_threads = (int)n_tokens;
+
+    row_job proto;
+    memset(&proto, 0, sizeof(proto));
+    proto.x = x; proto.r = r; proto.w = w; proto.y = y; proto.r_out = r_out;
+    proto.hidden = hidden;
+    proto.eps = (double)eps; /* exact widening of the binary32 scalar */
+    proto.dtype = dtype;
+    proto.norm_from_rounded = norm_from_rounded;
+
+    if (n_threads == 1) {
+        proto.row_begin = 0;
+        proto.row_end = n_tokens;
+        run_rows(&proto);
+        return proto.status;
+    }
+
+    row_job* jobs = (row_job*)malloc((size_t)n_threads * sizeof(row_job));
+    pthread_t* tids = (pthread_t*)malloc((size_t)n_threads * sizeof(pthread_t));
+    if (!jobs || !tids) {
+        free(jobs);
+        free(tids);
+        return 2;
+    }
+    int status = 0;
+    for (int k = 0; k < n_threads; ++k) {
+        jobs[k] = proto;
+        jobs[k].row_begin = n_tokens * k / n_threads;
+        jobs[k].row_end = n_tokens * (k + 1) / n_threads;
+        if (pthread_create(&tids[k], NULL, thread_main, &jobs[k]) != 0) {
+            run_rows(&jobs[k]); /* fall back to running this block here */
+            tids[k] = 0;
+        }
+    }
+    for (int k = 0; k < n_threads; ++k) {
+        if (tids[k]) pthread_join(tids[k], NULL);
+        if (jobs[k].status) status = jobs[k].status;
+    }
+    free(jobs);
+    free(tids);
+    return status;
+}
+
+/* ---- comparison metrics d(.,.) --------------------------------------------- */
+
+/* Position of a 16-bit pattern on a line where adjacent representable values
+ * are one apart and +0 and -0 coincide. */
+static int32_t lattice16(uint16_t b)
+{
+    const int32_t mag = b & 0x7FFF;
+    return (b & 0x8000u) ? -mag : mag;
+}
+
+static int is_nan16(uint16_t b, fmt16 f)
+{
+    const int emax_field = (1 << f.ebits) - 1;
+    return ((b >> f.mbits) & emax_field) == emax_field && (b & ((1 << f.mbits) - 1));
+}
+
+/*
+ * Distance in units of the last place between two arrays of 16-bit values.
+ * Writes the maximum distance and how many elements exceed `tol_ulp`.
+ * NaN matches NaN (distance 0); NaN against a number counts as 65535.
+ */
+void oracle_ulp_compare16(const uint16_t* got, const uint16_t* ref, int64_t n, int dtype,
+                          int32_t tol_ulp, int32_t* max_ulp, int64_t* n_bad)
+{
+    const fmt16 f = dtype == ORACLE_BF16 ? FMT_BF16 : FMT_FP16;
+    int32_t worst = 0;
+    int64_t bad = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        int32_t d;
+        const int gn = is_nan16(got[i], f), rn = is_nan16(ref[i], f);
+        if (gn || rn)
+            d = (gn && rn) ? 0 : 65535;
+        else {
+            d = lattice16(got[i]) - lattice16(ref[i]);
+            if (d < 0) d = -d;
+        }
+        if (d > worst) worst = d;
+        if (d > tol_ulp) ++bad;
+    }
+    *max_ulp = worst;
+    *n_bad = bad;
+}
+
+/*
+ * binary32 outputs: relative error |got - ref| / max(|ref|, floor); writes the
+ * maximum and how many elements exceed `tol_rel`.  NaN matches NaN.
+ */
+void oracle_rel_compare32(const float* got, const float* ref, int64_t n, double tol_rel,
+                          double abs_floor, double* max_rel, int64_t* n_bad)
+{
+    double worst = 0.0;
+    int64_t bad = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        const double g = (double)got[i], q = (double)ref[i];
+        double e;
+        if (isnan(g) || isnan(q))
+            e = (isnan(g) && isnan(q)) ? 0.0 : INFINITY;
+        else if (g == q)
+            e = 0.0;
+        else {
+            double den = fabs(q);
+            if (den < abs_floor) den = abs_floor;
+            e = fabs(g - q) / den;
+        }
+        if (e > worst) worst = e;
+        if (e > tol_rel) ++bad;
+    }
+    *max_rel = worst;
+    *n_bad = bad;
+}

@@ -1,0 +1,166 @@
+"""Seeded synthetic inputs for the fused residual-add + RMSNorm workloads.
+
+This module only draws random numbers and converts them to the storage type.
+It holds none of the operator's arithmetic, so both the CPU oracle's tests and
+the CUDA path's tests feed from it without sharing anything else.
+
+Generator.  Counter-based Philox-4x64 (numpy's ``Philox`` bit generator).  The
+key is ``(seed, tensor_id)`` and the third counter word is the index of a block
+of ``ROWS_PER_BLOCK`` rows, so any row block can be regenerated on its own:
+the first rows of a tensor do not depend on how many rows follow, and a sample
+of rows of a very large workload can be re-drawn for a row-by-row check.
+
+Distributions.  ``x`` and ``r``: N(0, sigma) element-wise; with probability
+``outlier_p`` an element is *replaced* by a draw from N(0, outlier_sigma).
+``w``: N(w_mean, w_sigma).  The second argument of every normal is a standard
+deviation.  Values are drawn in float32 and converted to the storage dtype by
+``torch.Tensor.to`` (round to nearest even).
+
+The workload table mirrors the shapes of the paper's Experimental Setup
+("Kernels": hidden sizes typical of LLaMA-class models, fp32 and fp16/bf16) as
+five named configurations; no dataset is involved.
+"""
+from __future__ import annotations
+
+from concurrent.futures import ThreadPoolExecutor
+from dataclasses import dataclass, field
+
+import numpy as np
+import torch
+
+ROWS_PER_BLOCK = 64
+TENSOR_X, TENSOR_R, TENSOR_W = 0, 1, 2
+
+TORCH_DTYPES = {"bf16": torch.bfloat16, "fp16": torch.float16, "fp32": torch.float32}
+DTYPE_CODES = {"bf16": 0, "fp16": 1, "fp32": 2}
+DTYPE_BYTES = {"bf16": 2, "fp16": 2, "fp32": 4}
+
+
+@dataclass(frozen=True)
+class Dist:
+    sigma: float = 1.0
+    outlier_p: float = 0.0
+    outlier_sigma: float = 50.0
+    w_mean: float = 1.0
+    w_sigma: float = 0.1
+
+
+@dataclass(frozen=True)
+class Workload:
+    name: str
+    dtype: str
+    n_tokens: int
+    hidden: int
+    seed: int
+    dist: Dist = field(default_factory=Dist)
+    eps: float = 1e-6
+
+    @property
+    def elements(self) -> int:
+        return self.n_tokens * self.hidden
+
+    @property
+    def algorithmic_bytes(self) -> int:
+        """Bytes the operator must move: read x, read r, write r', write y, w once."""
+        b = DTYPE_BYTES[self.dtype]
+        return 4 * b * self.elements + b * self.hidden
+
+    @property
+    def nominal_bytes(self) -> int:
+        """Three reads and two writes per element (w counted as a full stream)."""
+        return 5 * DTYPE_BYTES[self.dtype] * self.elements
+
+
+_PREFILL_DIST = Dist(sigma=2.0, outlier_p=0.01, outlier_sigma=50.0)
+
+
+def workloads() -> dict[str, Workload]:
+    """The five benchmark configurations, keyed by name."""
+    out: dict[str, Workload] = {}
+
+    def add(wl: Workload):
+        out[wl.name] = wl
+
+    add(Workload("c1_bf16_128x4096", "bf16", 128, 4096, seed=0))
+    for t in (1, 4, 16, 64, 256):
+        add(Workload(f"c2_decode_bf16_{t}x4096", "bf16", t, 4096, seed=1))
+    add(Workload("c3_prefill_bf16_16384x8192", "bf16", 16384, 8192, seed=2, dist=_PREFILL_DIST))
+    for h in (5120, 7168, 6152):
+        add(Workload(f"c4_fp16_8192x{h}", "fp16", 8192, h, seed=3))
+    add(Workload("c4x_fp16_8192x6148", "fp16", 8192, 6148, seed=3))
+    add(Workload("c5_fp32_32768x12288", "fp32", 32768, 12288, seed=4))
+    return out
+
+
+# Shapes (m, n) listed in the paper's Experimental Setup for its two row-wise kernels.
+PAPER_SHAPES_FP32 = [(128, 4096), (256, 4096), (1024, 4096), (2048, 8192), (128, 11008),
+                     (256, 13824), (512, 14336), (1024, 8192)]
+PAPER_SHAPES_16BIT = [(16, 4096), (32, 5120), (32, 8192), (16, 12288), (64, 8192)]
+
+
+def _rng(seed: int, tensor_id: int, block: int) -> np.random.Generator:
+    return np.random.Generator(np.random.Philox(key=[seed, tensor_id], counter=[0, 0, block, 0]))
+
+
+def _block_f32(seed: int, tensor_id: int, block: int, hidden: int, dist: Dist) -> np.ndarray:
+    g = _rng(seed, tensor_id, block)
+    n = ROWS_PER_BLOCK * hidden
+    v = g.standard_normal(n, dtype=np.float32)
+    v *= np.float32(dist.sigma)
+    if dist.outlier_p > 0.0:
+        u = g.random(n, dtype=np.float32)
+        o = g.standard_normal(n, dtype=np.float32)
+        o *= np.float32(dist.outlier_sigma)
+        np.copyto(v, o, where=u < np.float32(dist.outlier_p))
+    return v.reshape(ROWS_PER_BLOCK, hidden)
+
+
+def make_rows(tensor_id: int, row_begin: int, row_end: int, hidden: int, dtype: str, seed: int,
+              dist: Dist = Dist(), threads: int = 8) -> torch.Tensor:
+    """Rows [row_begin, row_end) of tensor ``x`` (tensor_id 0) or ``r`` (1) as a CPU tensor."""
+    if row_end <= row_begin:
+        return torch.empty((0, hidden), dtype=TORCH_DTYPES[dtype])
+    b0, b1 = row_begin // ROWS_PER_BLOCK, (row_end - 1) // ROWS_PER_BLOCK + 1
+    out = torch.empty(((b1 - b0) * ROWS_PER_BLOCK, hidden), dtype=TORCH_DTYPES[dtype])
+
+    def fill(b: int):
+        blk = torch.from_numpy(_block_f32(seed, tensor_id, b, hidden, dist))
+        lo = (b - b0) * ROWS_PER_BLOCK
+        out[lo:lo + ROWS_PER_BLOCK].copy_(blk)  # dtype conversion, round to nearest even
+
+    if b1 - b0 > 1 and threads > 1:
+        with ThreadPoolExecutor(max_workers=threads) as pool:
+            list(pool.map(fill, range(b0, b1)))
+    else:
+        for b in range(b0, b1):
+            fill(b)
+    lo = row_begin - b0 * ROWS_PER_BLOCK
+    return out[lo:lo + (row_end - row_begin)]
+
+
+def make_weight(hidden: int, dtype: str, seed: int, dist: Dist = Dist()) -> torch.Tensor:
+    g = _rng(seed, TENSOR_W, 0)
+    v = g.standard_normal(hidden, dtype=np.float32)
+    v = v * np.float32(dist.w_sigma) + np.float32(dist.w_mean)
+    return torch.from_numpy(v).to(TORCH_DTYPES[dtype])
+
+
+def make_inputs(n_tokens: int, hidden: int, dtype: str, seed: int, dist: Dist = Dist(),
+                threads: int = 8):
+    """(x, r, w) as contiguous CPU tensors of the storage dtype."""
+    x = make_rows(TENSOR_X, 0, n_tokens, hidden, dtype, seed, dist, threads).contiguous()
+    r = make_rows(TENSOR_R, 0, n_tokens, hidden, dtype, seed, dist, threads).contiguous()
+    w = make_weight(hidden, dtype, seed, dist)
+    return x, r, w
+
+
+def make_workload_inputs(wl: Workload, threads: int = 8):
+    return make_inputs(wl.n_tokens, wl.hidden, wl.dtype, wl.seed, wl.dist, threads)
+
+
+def sample_rows(wl: Workload, rows, threads: int = 1):
+    """Regenerate the given rows of a workload: (x_rows, r_rows, w), each row drawn on its own."""
+    xs = [make_rows(TENSOR_X, t, t + 1, wl.hidden, wl.dtype, wl.seed, wl.dist, threads) for t in rows]
+    rs = [make_rows(TENSOR_R, t, t + 1, wl.hidden, wl.dtype, wl.seed, wl.dist, threads) for t in rows]
+    w = make_weight(wl.hidden, wl.dtype, wl.seed, wl.dist)
+    return torch.cat(xs).contiguous(), torch.cat(rs).contiguous(), w

@@ -1,0 +1,108 @@
+"""The pins must be able to fail: plant one mistake at a time in a copy of the oracle's C source
+(on the CPU), build it, and check that the core pins reject it while the real source passes."""
+import math
+import os
+import subprocess
+
+import numpy as np
+import pytest
+import torch
+
+import refnum
+
+MUTATIONS = {
+    "divide_by_h_minus_1": ("acc / (double)H", "acc / (double)(H - 1)"),
+    "eps_outside_sqrt": ("sqrt(ms + job->eps)", "(sqrt(ms) + job->eps)"),
+    "weight_dropped": ("s[j] * wj / denom", "s[j] / denom"),
+    "residual_dropped": ("const float s32 = xf + rf;", "const float s32 = xf;"),
+    "residual_sign": ("const float s32 = xf + rf;", "const float s32 = xf - rf;"),
+    "sum_not_squared": ("acc += used * used;", "acc += used;"),
+    "ties_away_from_zero": ("(rem == 0.5 && (n & 1u))", "(rem == 0.5)"),
+    "truncating_encode": ("if (rem > 0.5 ||", "if (rem > 2.0 ||"),
+    "weight_indexed_by_row": ("wj = decode16(((const uint16_t*)job->w)[j], f);",
+                              "wj = decode16(((const uint16_t*)job->w)[t % H], f);"),
+    "output_row_ignored": ("((uint16_t*)job->y)[base + j] = encode16(y64, f);",
+                           "((uint16_t*)job->y)[j] = encode16(y64, f);"),
+    "add_in_double_then_round_direct": ("const uint16_t rb = encode16((double)s32, f);",
+                                        "const uint16_t rb = encode16((double)xf * 1.0000001 + (double)rf, f);"),
+    "rounded_residual_in_norm": ("if (job->norm_from_rounded)", "if (1)"),
+    "subnormal_flush": ("bits = (uint32_t)n; /* subnormal", "bits = 0; /* subnormal"),
+}
+
+
+def _core_pins(o) -> bool:
+    """A condensed set of the pins (bf16 and fp16), True when all hold."""
+    bf, hf = torch.bfloat16, torch.float16
+    try:
+        for dtype, td in ((0, bf), (1, hf)):
+            H = 37
+            c, eps = 1.5, 0.25
+            w = torch.linspace(-2, 2, H, dtype=torch.float64).to(td)
+            x = torch.full((3, H), c / 2, dtype=td)
+            y, ro = o.add_rmsnorm(x, x, w, eps)
+            want = refnum.round_array(np.repeat((w.double().numpy() * c / math.sqrt(c * c + eps))[None], 3, 0), dtype)
+            if not np.array_equal(y.view(torch.int16).numpy().view(np.uint16), want):
+                return False
+            # one-hot row: the mean divides by H
+            xo = torch.zeros(1, 24, dtype=td); xo[0, 5] = 3.0
+            wo = torch.linspace(0.5, 1.5, 24, dtype=torch.float64).to(td)
+            y, _ = o.add_rmsnorm(xo, torch.zeros_like(xo), wo, eps)
+            want = np.zeros(24); want[5] = float(wo[5]) * 3.0 / math.sqrt(9.0 / 24 + eps)
+            if not np.array_equal(y.view(torch.int16).numpy().view(np.uint16)[0], refnum.round_array(want, dtype)):
+                return False
+            # library evaluation, ragged shape, two readings of the residual
+            g = np.random.Generator(np.random.Philox(key=[41, dtype]))
+            x = torch.from_numpy(g.standard_normal((5, 300)) * np.exp(g.uniform(-12, 3, (5, 300)))).to(td)
+            r = torch.from_numpy(g.standard_normal((5, 300)) * np.exp(g.uniform(-12, 3, (5, 300)))).to(td)
+            w = torch.from_numpy(1 + 0.3 * g.standard_normal(300)).to(td)
+            y, ro = o.add_rmsnorm(x, r, w, 1e-6)
+            s32 = x.float() + r.float()
+            if not torch.equal(ro, s32.to(td)):
+                return False
+            s = s32.double()
+            y64 = s * torch.rsqrt(s.pow(2).mean(-1, keepdim=True) + float(np.float32(1e-6))) * w.double()
+            got = y.view(torch.int16).numpy().view(np.uint16)
+            if np.count_nonzero(got != refnum.round_array(y64.numpy(), dtype)) > 1:
+                return False
+            # ties and subnormals of the codec
+            vals, bits = refnum.finite_table(dtype)
+            mid = (vals[:-1] + vals[1:]) / 2
+            even = np.where((bits[:-1] & 1) == 0, bits[:-1], bits[1:])
+            even = np.where((even == 0) & np.signbit(mid), np.uint16(0x8000), even)
+            if not np.array_equal(o.encode16_from_f64(mid, dtype), even):
+                return False
+            above = np.nextafter(mid, np.inf)
+            wa = np.where((bits[1:] == 0) & np.signbit(above), np.uint16(0x8000), bits[1:])
+            if not np.array_equal(o.encode16_from_f64(above, dtype), wa):
+                return False
+    except Exception:
+        return False
+    return True
+
+
+def _build(src_text: str, out_dir, name: str) -> str:
+    c = os.path.join(out_dir, name + ".c")
+    so = os.path.join(out_dir, name + ".so")
+    with open(c, "w") as f:
+        f.write(src_text)
+    subprocess.run(["gcc", "-O2", "-fno-fast-math", "-ffp-contract=off", "-std=c99", "-shared", "-fPIC",
+                    "-pthread", c, "-o", so, "-lm"], check=True)
+    return so
+
+
+def test_real_oracle_passes_core_pins(oracle_lib):
+    assert _core_pins(oracle_lib)
+
+
+@pytest.mark.parametrize("name", sorted(MUTATIONS))
+def test_planted_mistake_is_caught(oracle_lib, tmp_path, name):
+    old, new = MUTATIONS[name]
+    src = open(os.path.join(os.path.dirname(oracle_lib.__file__), "add_rmsnorm_oracle.c")).read()
+    assert src.count(old) >= 1, f"mutation anchor not found: {old}"
+    so = _build(src.replace(old, new), str(tmp_path), name)
+    saved = oracle_lib._lib
+    try:
+        oracle_lib._lib = oracle_lib._bind(so)
+        assert not _core_pins(oracle_lib), f"pins did not notice: {name}"
+    finally:
+        oracle_lib._lib = saved
