@@ -1,0 +1,307 @@
+/*
+ * rmsnorm_tuner.h - C ABI of the template-plus-search tuner for the fused
+ * residual-add + RMSNorm kernel on sm_100a (NVIDIA B200).
+ *
+ * The library holds three things, after the paper's Level 2 ("parameter search
+ * within the resource-feasible region", Algorithm 1) applied to one of its three
+ * evaluation kernels, `fused_add_rmsnorm` ("Kernels" paragraph, Experimental
+ * Setup):
+ *
+ *   1. the kernel as an explicitly parameterised template  (Templatize /
+ *      Instantiate(S~, theta), Section "Problem Formulation" and Algorithm 1);
+ *   2. the feasible-region deriver  (DeriveFeasibleSpace(S~, h, r(h)), Algorithm 1
+ *      and Section "Tuning parameter selection and search space derivation");
+ *   3. the guided search on measured device time with a correctness gate on every
+ *      candidate  (Search(S~, x, Theta_feasible), Algorithm 1; timing protocol of
+ *      "Performance Measurement": 20 warm-up runs then the mean of 100 runs;
+ *      correctness as in paragraph "Correctness": max_i d(S~(x_i), S(x_i)) <= eps).
+ *
+ * The operator, per token row t (rows are independent):
+ *     s_j  = fp32(x[t,j]) + fp32(r[t,j])               (one binary32 addition)
+ *     r_out[t,j] = round_to_nearest_even_dtype(s_j)
+ *     y[t,j] = round_dtype( s_j * rsqrt(mean_j(s_j^2) + eps) * w[j] )
+ * The normalisation uses the un-rounded fp32 sum s_j.
+ *
+ * Conventions
+ *   - Every function returns an rt_status (0 = RT_OK) unless stated; none throws,
+ *     aborts or exits.  rt_last_error() gives the text of the last failure on the
+ *     calling thread.
+ *   - "device" pointers are CUDA global-memory addresses on the current device;
+ *     "host" pointers are ordinary process memory.  The caller owns every buffer
+ *     it passes; the library never frees or keeps them.
+ *   - Tensors are row-major and contiguous: x, r, y, r_out are [n_tokens, hidden]
+ *     with row stride `hidden` elements; w is [hidden]; all of element type
+ *     `dtype`.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *   - Nothing here synchronises the device unless its comment says so.
+ */
+#ifndef RMSNORM_TUNER_H_
+#define RMSNORM_TUNER_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { RT_BF16 = 0, RT_FP16 = 1, RT_FP32 = 2 } rt_dtype;
+
+/* Where a row lives between the two passes over it. */
+typedef enum {
+    RT_STAGE_REG = 0,      /* ld.global vectors straight into registers, row kept as fp32 registers */
+    RT_STAGE_SMEM_LDG = 1, /* ld.global vectors, sum kept as fp32 in shared memory */
+    RT_STAGE_SMEM_TMA = 2  /* cp.async.bulk (TMA, one copy per row slice) into shared memory + mbarrier */
+} rt_stage;
+
+/* How the per-row sum of squares is combined. */
+typedef enum {
+    RT_REDUCE_SHFL = 0,   /* warp shuffle tree, then one shared-memory hop across warps */
+    RT_REDUCE_SMEM = 1,   /* shared-memory halving tree over all threads of the row */
+    RT_REDUCE_CLUSTER = 2 /* a row is split over a thread-block cluster; partials meet through
+                             distributed shared memory and barrier.cluster */
+} rt_reduce;
+
+/* theta: one point of the template's parameter space. */
+typedef struct {
+    int32_t threads_per_row; /* threads cooperating on one row (blockDim.x); power of two, 32..1024 */
+    int32_t rows_per_cta;    /* rows handled by one CTA (blockDim.y); 1..8 */
+    int32_t vec_bytes;       /* bytes per ld/st: 16 or 8 (4 and 2 exist as a narrow fall-back) */
+    int32_t unroll;          /* independent vector loads in flight per thread and tensor: 1, 2, 4 */
+    int32_t stage;           /* rt_stage */
+    int32_t reduce;          /* rt_reduce */
+    int32_t cluster_size;    /* CTAs per row when reduce == RT_REDUCE_CLUSTER (2, 4, 8), else 1 */
+} rt_params;
+
+typedef struct {
+    int64_t n_tokens;
+    int64_t hidden;
+    int32_t dtype;         /* rt_dtype */
+    int32_t min_ptr_align; /* largest power of two (bytes, <= 256) dividing all five base addresses */
+} rt_shape;
+
+/* r(h): the resource upper bounds the feasible region is derived from. */
+typedef struct {
+    int32_t sm_count;
+    int32_t warp_size;
+    int32_t max_threads_per_block;
+    int32_t max_threads_per_sm;
+    int32_t max_blocks_per_sm;
+    int32_t regs_per_block;
+    int32_t regs_per_sm;
+    int32_t max_regs_per_thread;
+    int32_t max_cluster_size;
+    int32_t have_device;            /* 1: per-kernel registers/spills and occupancy come from the CUDA
+                                       runtime; 0: from the closed-form model in the deriver */
+    int64_t smem_per_block_optin;   /* largest dynamic + static shared memory one CTA may ask for */
+    int64_t smem_per_sm;
+    int64_t smem_reserved_per_block;
+    int64_t l2_bytes;
+} rt_limits;
+
+/* Heuristic ("obvious inefficiency") pruning rules; hard rules are always applied. */
+enum {
+    RT_PRUNE_IDLE_THREADS = 1,  /* a thread of the row would never own a vector */
+    RT_PRUNE_DUPLICATES = 2,    /* unroll deeper than the per-thread vector count: same kernel again */
+    RT_PRUNE_CLUSTER_WAVES = 4, /* split rows over a cluster only while whole rows cannot fill the SMs */
+    RT_PRUNE_IDLE_ROWS = 8,     /* more rows per CTA than the batch has rows */
+    RT_PRUNE_DEFAULT = 15
+};
+
+typedef enum { RT_SEARCH_GUIDED = 0, RT_SEARCH_EXHAUSTIVE = 1 } rt_strategy;
+
+typedef struct {
+    int32_t max_evals;       /* budget in kernel evaluations (one evaluation = gate + warm-up + timed runs) */
+    int32_t warmup;          /* untimed launches per evaluation (paper: 20) */
+    int32_t iters;           /* timed launches per block (paper: 100); time = block time / iters */
+    int32_t repeats;         /* timed blocks per evaluation; the score is their median (>= 1) */
+    int32_t top_k;           /* finalists re-timed before the winner is declared (0 = none) */
+    int32_t strategy;        /* rt_strategy */
+    int32_t heuristics;      /* RT_PRUNE_* mask used for the candidate set */
+    int32_t use_graph;       /* 1: the timed block is one CUDA graph of `iters` launches */
+    const rt_params* seeds;  /* host; evaluated first when given (configs found on other shapes) */
+    int32_t n_seeds;
+    int32_t reserved;
+} rt_budget;
+
+typedef struct {
+    const void* x;     /* device, [ring_sets][n_tokens, hidden] */
+    const void* r;     /* device */
+    const void* w;     /* device, [hidden] */
+    void* y;           /* device; must not alias x here (launches repeat) */
+    void* r_out;       /* device; must not alias r here */
+    const void* y_ref; /* device, oracle y for rows [0, n_ref_tokens) of set 0 */
+    const void* r_ref; /* device, oracle r' for the same rows */
+    int64_t n_ref_tokens;     /* rows covered by the references, 1..n_tokens */
+    int64_t ring_stride_bytes;/* distance between consecutive sets of x, r, y, r_out (0 when ring_sets == 1) */
+    int32_t ring_sets;        /* >= 1; timed launches rotate over the sets (cold-L2 timing of small shapes) */
+    float eps;
+    void* stream;
+} rt_workspace;
+
+typedef enum { RT_PHASE_SEED = 0, RT_PHASE_GRID = 1, RT_PHASE_CLIMB = 2, RT_PHASE_TOPK = 3,
+               RT_PHASE_SWEEP = 4 } rt_phase;
+
+/* One line of the search log: every evaluated theta, its gate result and its time. */
+typedef struct {
+    rt_params params;
+    int32_t phase;      /* rt_phase */
+    int32_t eval_index; /* 0-based order of evaluation */
+    int32_t status;     /* RT_OK, RT_ERR_MISMATCH, RT_ERR_CUDA, ... for this candidate */
+    int32_t y_max_ulp;  /* 16-bit dtypes: worst distance of y from the reference in ulps */
+    int64_t y_bad;      /* elements of y beyond tolerance */
+    int64_t r_bad;      /* elements of r_out whose bits differ from the reference */
+    float y_max_rel;    /* fp32: worst relative error of y */
+    float us;           /* score: median over blocks of (block time / iters), microseconds */
+    float us_min_block; /* fastest block */
+    float us_mean;      /* mean over all blocks */
+    int32_t occupancy_blocks_per_sm;
+    int32_t regs_per_thread;
+} rt_eval_record;
+
+typedef struct {
+    rt_params best;
+    float best_us;
+    int32_t evals_used;
+    int32_t n_candidates; /* size of the feasible set searched */
+    int32_t n_log;        /* records written to the caller's log (<= log_cap) */
+    int32_t n_failed_gate;
+} rt_result;
+
+typedef enum {
+    RT_OK = 0,
+    RT_ERR_NULL = 1,           /* a required pointer is NULL */
+    RT_ERR_DTYPE = 2,
+    RT_ERR_SHAPE = 3,          /* n_tokens < 0, hidden <= 0, hidden too large */
+    RT_ERR_ALIGN = 4,          /* a pointer or the row length is not a multiple of vec_bytes (or of 16 for TMA) */
+    RT_ERR_INFEASIBLE = 5,     /* theta violates a hard limit; nothing was launched */
+    RT_ERR_CUDA = 6,           /* a CUDA runtime call failed; see rt_last_error() */
+    RT_ERR_MISMATCH = 7,       /* correctness gate failed (search: for every candidate) */
+    RT_ERR_BUDGET = 8,         /* the budget allows no evaluation */
+    RT_ERR_DEVICE_TIMEOUT = 9, /* a bounded device-side wait expired (read through rt_device_status) */
+    RT_ERR_CAPACITY = 10,      /* a caller-provided array or workspace is too small */
+    RT_ERR_NO_DEVICE = 11      /* no CUDA device is available */
+} rt_status;
+
+/* ---- 1. the template kernel ------------------------------------------------- */
+
+/*
+ * Instantiate(S~, theta) and launch it (Algorithm 1, Level 2; operator as defined at
+ * the top of this file).  Asynchronous on `stream`.
+ *   p        host; checked against the hard feasibility rules first - an infeasible
+ *            theta returns RT_ERR_INFEASIBLE / RT_ERR_ALIGN and launches nothing.
+ *   x, r, w  device, read only.   y, r_out  device, written.
+ *   Allowed aliasing: y == x and/or r_out == r (in-place use); any other overlap
+ *   is undefined.  n_tokens == 0 is a successful no-op.
+ *   Allocates nothing and never synchronises.
+ */
+int rmsnorm_template_launch(const rt_params* p, const void* x, const void* r, const void* w, void* y,
+                            void* r_out, int64_t n_tokens, int64_t hidden, float eps, int dtype,
+                            void* stream);
+
+/*
+ * The same operator on HOST buffers: copies x, r, w to the device, launches theta, copies y and
+ * r_out back, in row chunks so that the two copy directions and the kernel overlap.  `workspace`
+ * is device memory of at least rmsnorm_host_workspace_bytes(...) bytes, owned by the caller; host
+ * buffers should be page-locked for the copies to be asynchronous.  Synchronises `stream` before
+ * returning.  (End-to-end entry point; no counterpart in the paper, which times kernels only.)
+ */
+int rmsnorm_template_run_host(const rt_params* p, const void* x_host, const void* r_host,
+                              const void* w_host, void* y_host, void* r_out_host, int64_t n_tokens,
+                              int64_t hidden, float eps, int dtype, void* workspace,
+                              int64_t workspace_bytes, int64_t chunk_tokens, void* stream);
+int64_t rmsnorm_host_workspace_bytes(int64_t n_tokens, int64_t hidden, int dtype, int64_t chunk_tokens);
+
+/* ---- 2. the feasible region ----------------------------------------------------- */
+
+/* r(h) of the current CUDA device.  RT_ERR_NO_DEVICE when there is none. */
+int rt_query_limits(rt_limits* out);
+/* Documented sm_100a (B200) limits, for host-only use (have_device = 0). */
+void rt_limits_sm100_nominal(rt_limits* out);
+
+/*
+ * DeriveFeasibleSpace(S~, h, r(h)) (Algorithm 1; "Tuning parameter selection and search space
+ * derivation": ranges and discrete candidate sets from the hardware limits, pruning combinations
+ * that would not compile, not launch, or be obviously inefficient).
+ *   s      host.   out  host array of `cap` entries (may be NULL when cap == 0).
+ *   *n_out receives the size of the feasible set, which may exceed `cap`: call twice.
+ * Uses the current device's limits and, for every candidate, the compiled kernel's register count,
+ * spill size and occupancy.  tuner_derive_feasible_ex takes the limits and the heuristic mask
+ * explicitly (limits->have_device == 0 works without a GPU).
+ */
+int tuner_derive_feasible(const rt_shape* s, rt_params* out, int32_t cap, int32_t* n_out);
+int tuner_derive_feasible_ex(const rt_shape* s, const rt_limits* limits, int32_t heuristics,
+                             rt_params* out, int32_t cap, int32_t* n_out);
+/* Hard rules only, for one theta: RT_OK, RT_ERR_ALIGN or RT_ERR_INFEASIBLE (reason in rt_last_error). */
+int tuner_check_params(const rt_shape* s, const rt_limits* limits, const rt_params* p);
+/* The raw (unpruned) grid, for reporting how much the deriver removed. */
+int tuner_raw_grid(const rt_shape* s, rt_params* out, int32_t cap, int32_t* n_out);
+/*
+ * How the raw grid was pruned.  counts (host, n_counts >= 11): [0..7] points removed by a hard rule,
+ * by reason (0 unused, 1 arguments, 2 threads per CTA, 3 alignment, 4 registers, 5 shared memory,
+ * 6 cluster, 7 grid size); [8] removed by the heuristic rules; [9] feasible; [10] raw grid size.
+ */
+int tuner_derive_counts(const rt_shape* s, const rt_limits* limits, int32_t heuristics, int32_t* counts,
+                        int32_t n_counts);
+
+/* ---- 3. search -------------------------------------------------------------------- */
+
+/*
+ * Search(S~, x, Theta_feasible) for one input shape (Algorithm 1): seeds first, then a coarse
+ * grid over the feasible set, then steepest-descent hill-climbing over one-step neighbours on
+ * measured time, then a re-test of the top_k finalists ("Tuning agent": Top-K re-testing).
+ * Every candidate passes the correctness gate (r_out bit-exact, y within 2 ulp for 16-bit types or
+ * 1e-5 relative for fp32, against the uploaded references) before it is timed; candidates that
+ * fail the gate or the launch are logged and skipped.
+ *   log      host array of log_cap records (may be NULL).   Synchronises the stream repeatedly.
+ *   Allocates a few bytes of device memory on first use (freed by rt_shutdown).
+ * RT_ERR_MISMATCH when no candidate passed the gate; RT_ERR_BUDGET when max_evals < 1.
+ */
+int tuner_search(const rt_shape* s, const rt_budget* b, const rt_workspace* ws, rt_result* out,
+                 rt_eval_record* log, int32_t log_cap);
+
+/*
+ * The same search over a caller-supplied cost function instead of the device (host only; used to
+ * test the search logic and budget accounting).  `evaluate` returns the time of theta in
+ * microseconds, or a negative value / NaN for a candidate that fails its gate.
+ */
+typedef double (*rt_evaluate_fn)(const rt_params* p, void* user);
+int tuner_search_with(const rt_shape* s, const rt_limits* limits, const rt_budget* b,
+                      rt_evaluate_fn evaluate, void* user, rt_result* out, rt_eval_record* log,
+                      int32_t log_cap);
+
+/* Gate + timing of one theta with the protocol of `b` (warmup, iters, repeats, use_graph). */
+int tuner_evaluate(const rt_shape* s, const rt_params* p, const rt_budget* b, const rt_workspace* ws,
+                   rt_eval_record* out);
+
+typedef enum { RT_CMP_BITS = 0, RT_CMP_ULP16 = 1, RT_CMP_REL32 = 2 } rt_compare_mode;
+/*
+ * The distance d(.,.) of the correctness criterion, computed on the device.
+ *   got, ref  device, n elements of `dtype`.
+ *   RT_CMP_BITS : *n_bad = elements whose bit patterns differ; *max_err = 1 if any.
+ *   RT_CMP_ULP16: distance in units of the last place on the 16-bit type's value lattice
+ *                 (+0 == -0, NaN matches NaN); *n_bad = elements beyond `tol`.
+ *   RT_CMP_REL32: |got-ref| <= tol*|ref| + 1e-30 for fp32; *max_err = worst |got-ref|/|ref|.
+ *   max_err, n_bad: host.  Synchronises `stream`.
+ */
+int tuner_compare(const void* got, const void* ref, int64_t n, int dtype, int mode, double tol,
+                  double* max_err, int64_t* n_bad, void* stream);
+
+/* ---- housekeeping ------------------------------------------------------------------- */
+
+const char* rt_status_string(int status);
+const char* rt_last_error(void);
+/* Reads and clears the device status word (0, or RT_ERR_DEVICE_TIMEOUT).  Synchronises the device. */
+int rt_device_status(void);
+/* Number of compiled instances of the template, and the i-th one's coordinates (host query). */
+int32_t rt_num_kernel_instances(void);
+int rt_kernel_instance(int32_t i, int32_t* dtype, int32_t* vec_bytes, int32_t* stage, int32_t* reduce,
+                       int32_t* unroll, int32_t* reg_vectors);
+/* Kernel launches issued by this library in this process since load (all entry points). */
+int64_t rt_launch_count(void);
+/* Frees what the library allocated on the device.  Safe to call more than once. */
+void rt_shutdown(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RMSNORM_TUNER_H_ */

@@ -1,0 +1,339 @@
+"""ctypes binding of librmsnorm_tuner.so: the same names as the C ABI, argument marshalling only.
+
+Every step of the operator, of the feasible-region derivation and of the search runs inside the shared
+library.  torch is used here for device memory, streams and dtype bookkeeping; there is no CPU or
+PyTorch fall-back: if the library is missing, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, Structure, byref, c_char_p, c_double, c_float, c_int, c_int32, c_int64, c_void_p
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "librmsnorm_tuner.so")
+HEADER_PATH = os.path.join(os.path.dirname(_HERE), "include", "rmsnorm_tuner.h")
+
+RT_BF16, RT_FP16, RT_FP32 = 0, 1, 2
+RT_STAGE_REG, RT_STAGE_SMEM_LDG, RT_STAGE_SMEM_TMA = 0, 1, 2
+RT_REDUCE_SHFL, RT_REDUCE_SMEM, RT_REDUCE_CLUSTER = 0, 1, 2
+RT_PRUNE_IDLE_THREADS, RT_PRUNE_DUPLICATES, RT_PRUNE_CLUSTER_WAVES, RT_PRUNE_IDLE_ROWS = 1, 2, 4, 8
+RT_PRUNE_DEFAULT = 15
+RT_SEARCH_GUIDED, RT_SEARCH_EXHAUSTIVE = 0, 1
+RT_CMP_BITS, RT_CMP_ULP16, RT_CMP_REL32 = 0, 1, 2
+(RT_OK, RT_ERR_NULL, RT_ERR_DTYPE, RT_ERR_SHAPE, RT_ERR_ALIGN, RT_ERR_INFEASIBLE, RT_ERR_CUDA, RT_ERR_MISMATCH,
+ RT_ERR_BUDGET, RT_ERR_DEVICE_TIMEOUT, RT_ERR_CAPACITY, RT_ERR_NO_DEVICE) = range(12)
+PHASE_NAMES = {0: "seed", 1: "grid", 2: "climb", 3: "topk", 4: "sweep"}
+STAGE_NAMES = {0: "reg", 1: "smem_ldg", 2: "smem_tma"}
+REDUCE_NAMES = {0: "shfl", 1: "smem", 2: "cluster"}
+DTYPE_CODES = {"bf16": RT_BF16, "fp16": RT_FP16, "fp32": RT_FP32}
+
+
+class rt_params(Structure):
+    _fields_ = [("threads_per_row", c_int32), ("rows_per_cta", c_int32), ("vec_bytes", c_int32),
+                ("unroll", c_int32), ("stage", c_int32), ("reduce", c_int32), ("cluster_size", c_int32)]
+
+    def as_dict(self) -> dict:
+        return {k: int(getattr(self, k)) for k, _ in self._fields_}
+
+    def key(self) -> tuple:
+        return tuple(int(getattr(self, k)) for k, _ in self._fields_)
+
+    def __repr__(self):
+        return (f"theta(tpr={self.threads_per_row}, rpc={self.rows_per_cta}, vec={self.vec_bytes}, "
+                f"unroll={self.unroll}, stage={STAGE_NAMES.get(self.stage, self.stage)}, "
+                f"reduce={REDUCE_NAMES.get(self.reduce, self.reduce)}, cluster={self.cluster_size})")
+
+
+def make_params(threads_per_row=256, rows_per_cta=1, vec_bytes=16, unroll=1, stage=RT_STAGE_REG,
+                reduce=RT_REDUCE_SHFL, cluster_size=1) -> rt_params:
+    return rt_params(threads_per_row, rows_per_cta, vec_bytes, unroll, stage, reduce, cluster_size)
+
+
+class rt_shape(Structure):
+    _fields_ = [("n_tokens", c_int64), ("hidden", c_int64), ("dtype", c_int32), ("min_ptr_align", c_int32)]
+
+
+class rt_limits(Structure):
+    _fields_ = [("sm_count", c_int32), ("warp_size", c_int32), ("max_threads_per_block", c_int32),
+                ("max_threads_per_sm", c_int32), ("max_blocks_per_sm", c_int32), ("regs_per_block", c_int32),
+                ("regs_per_sm", c_int32), ("max_regs_per_thread", c_int32), ("max_cluster_size", c_int32),
+                ("have_device", c_int32), ("smem_per_block_optin", c_int64), ("smem_per_sm", c_int64),
+                ("smem_reserved_per_block", c_int64), ("l2_bytes", c_int64)]
+
+
+class rt_budget(Structure):
+    _fields_ = [("max_evals", c_int32), ("warmup", c_int32), ("iters", c_int32), ("repeats", c_int32),
+                ("top_k", c_int32), ("strategy", c_int32), ("heuristics", c_int32), ("use_graph", c_int32),
+                ("seeds", POINTER(rt_params)), ("n_seeds", c_int32), ("reserved", c_int32)]
+
+
+class rt_workspace(Structure):
+    _fields_ = [("x", c_void_p), ("r", c_void_p), ("w", c_void_p), ("y", c_void_p), ("r_out", c_void_p),
+                ("y_ref", c_void_p), ("r_ref", c_void_p), ("n_ref_tokens", c_int64),
+                ("ring_stride_bytes", c_int64), ("ring_sets", c_int32), ("eps", c_float), ("stream", c_void_p)]
+
+
+class rt_eval_record(Structure):
+    _fields_ = [("params", rt_params), ("phase", c_int32), ("eval_index", c_int32), ("status", c_int32),
+                ("y_max_ulp", c_int32), ("y_bad", c_int64), ("r_bad", c_int64), ("y_max_rel", c_float),
+                ("us", c_float), ("us_min_block", c_float), ("us_mean", c_float),
+                ("occupancy_blocks_per_sm", c_int32), ("regs_per_thread", c_int32)]
+
+    def as_dict(self) -> dict:
+        d = {k: getattr(self, k) for k, _ in self._fields_ if k != "params"}
+        d["params"] = self.params.as_dict()
+        d["phase"] = PHASE_NAMES.get(self.phase, self.phase)
+        return d
+
+
+class rt_result(Structure):
+    _fields_ = [("best", rt_params), ("best_us", c_float), ("evals_used", c_int32), ("n_candidates", c_int32),
+                ("n_log", c_int32), ("n_failed_gate", c_int32)]
+
+
+rt_evaluate_fn = ctypes.CFUNCTYPE(c_double, POINTER(rt_params), c_void_p)
+
+_SIGNATURES = {
+    "rmsnorm_template_launch": (c_int, [POINTER(rt_params), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                        c_int64, c_int64, c_float, c_int, c_void_p]),
+    "rmsnorm_template_run_host": (c_int, [POINTER(rt_params), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                          c_int64, c_int64, c_float, c_int, c_void_p, c_int64, c_int64, c_void_p]),
+    "rmsnorm_host_workspace_bytes": (c_int64, [c_int64, c_int64, c_int, c_int64]),
+    "rt_query_limits": (c_int, [POINTER(rt_limits)]),
+    "rt_limits_sm100_nominal": (None, [POINTER(rt_limits)]),
+    "tuner_derive_feasible": (c_int, [POINTER(rt_shape), POINTER(rt_params), c_int32, POINTER(c_int32)]),
+    "tuner_derive_feasible_ex": (c_int, [POINTER(rt_shape), POINTER(rt_limits), c_int32, POINTER(rt_params),
+                                         c_int32, POINTER(c_int32)]),
+    "tuner_check_params": (c_int, [POINTER(rt_shape), POINTER(rt_limits), POINTER(rt_params)]),
+    "tuner_raw_grid": (c_int, [POINTER(rt_shape), POINTER(rt_params), c_int32, POINTER(c_int32)]),
+    "tuner_derive_counts": (c_int, [POINTER(rt_shape), POINTER(rt_limits), c_int32, POINTER(c_int32), c_int32]),
+    "tuner_search": (c_int, [POINTER(rt_shape), POINTER(rt_budget), POINTER(rt_workspace), POINTER(rt_result),
+                             POINTER(rt_eval_record), c_int32]),
+    "tuner_search_with": (c_int, [POINTER(rt_shape), POINTER(rt_limits), POINTER(rt_budget), rt_evaluate_fn, c_void_p,
+                                  POINTER(rt_result), POINTER(rt_eval_record), c_int32]),
+    "tuner_evaluate": (c_int, [POINTER(rt_shape), POINTER(rt_params), POINTER(rt_budget), POINTER(rt_workspace),
+                               POINTER(rt_eval_record)]),
+    "tuner_compare": (c_int, [c_void_p, c_void_p, c_int64, c_int, c_int, c_double, POINTER(c_double),
+                              POINTER(c_int64), c_void_p]),
+    "rt_status_string": (c_char_p, [c_int]),
+    "rt_last_error": (c_char_p, []),
+    "rt_device_status": (c_int, []),
+    "rt_num_kernel_instances": (c_int32, []),
+    "rt_kernel_instance": (c_int, [c_int32] + [POINTER(c_int32)] * 6),
+    "rt_launch_count": (c_int64, []),
+    "rt_shutdown": (None, []),
+}
+EXPORTED = tuple(_SIGNATURES)
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2601_12698_b200.build` "
+                      "(there is no fall-back path)")
+lib = ctypes.CDLL(LIB_PATH)
+for _name, (_res, _args) in _SIGNATURES.items():
+    _fn = getattr(lib, _name)
+    _fn.restype = _res
+    _fn.argtypes = _args
+
+
+class TunerError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        text = lib.rt_status_string(status).decode()
+        detail = lib.rt_last_error().decode()
+        super().__init__(f"{where}: status {status} ({text}){': ' + detail if detail else ''}")
+
+
+def _check(status: int, where: str):
+    if status != RT_OK:
+        raise TunerError(status, where)
+
+
+def _dtype_code(t) -> int:
+    import torch
+    return {torch.bfloat16: RT_BF16, torch.float16: RT_FP16, torch.float32: RT_FP32}[t.dtype]
+
+
+def _stream_ptr(stream=None) -> int:
+    import torch
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return s.cuda_stream
+
+
+def _ptr_align(*tensors) -> int:
+    bits = 256
+    for t in tensors:
+        bits |= t.data_ptr()
+    return bits & -bits
+
+
+def shape_of(n_tokens: int, hidden: int, dtype, min_ptr_align: int = 256) -> rt_shape:
+    code = DTYPE_CODES[dtype] if isinstance(dtype, str) else int(dtype)
+    return rt_shape(n_tokens, hidden, code, min_ptr_align)
+
+
+def sm100_nominal_limits() -> rt_limits:
+    L = rt_limits()
+    lib.rt_limits_sm100_nominal(byref(L))
+    return L
+
+
+def rt_query_limits() -> rt_limits:
+    L = rt_limits()
+    _check(lib.rt_query_limits(byref(L)), "rt_query_limits")
+    return L
+
+
+# ---- 1. the template kernel -----------------------------------------------------------------------------
+
+def rmsnorm_template_launch(params: rt_params, x, r, w, y, r_out, eps: float, stream=None) -> None:
+    """Launch theta on device tensors (asynchronous on the stream).  y may be x, r_out may be r."""
+    if not (x.is_cuda and r.is_cuda and w.is_cuda and y.is_cuda and r_out.is_cuda):
+        raise ValueError("rmsnorm_template_launch takes CUDA tensors")
+    for t in (x, r, y, r_out):
+        if not t.is_contiguous() or t.shape != x.shape or t.dtype != x.dtype:
+            raise ValueError("x, r, y, r_out must be contiguous and alike")
+    n_tokens, hidden = x.shape
+    if w.shape != (hidden,) or w.dtype != x.dtype or not w.is_contiguous():
+        raise ValueError("w must be a contiguous [hidden] tensor of the same dtype")
+    _check(lib.rmsnorm_template_launch(byref(params), x.data_ptr(), r.data_ptr(), w.data_ptr(), y.data_ptr(),
+                                       r_out.data_ptr(), n_tokens, hidden, eps, _dtype_code(x), _stream_ptr(stream)),
+           "rmsnorm_template_launch")
+
+
+def rmsnorm_host_workspace_bytes(n_tokens: int, hidden: int, dtype, chunk_tokens: int = 0) -> int:
+    code = DTYPE_CODES[dtype] if isinstance(dtype, str) else int(dtype)
+    return int(lib.rmsnorm_host_workspace_bytes(n_tokens, hidden, code, chunk_tokens))
+
+
+def rmsnorm_template_run_host(params: rt_params, x, r, w, y, r_out, eps: float, workspace, chunk_tokens: int = 0,
+                              stream=None) -> None:
+    """The operator on host (ideally pinned) tensors through a device workspace; returns when y and r_out
+    are complete in host memory."""
+    for t in (x, r, w, y, r_out):
+        if t.is_cuda or not t.is_contiguous():
+            raise ValueError("rmsnorm_template_run_host takes contiguous host tensors")
+    n_tokens, hidden = x.shape
+    _check(lib.rmsnorm_template_run_host(byref(params), x.data_ptr(), r.data_ptr(), w.data_ptr(), y.data_ptr(),
+                                         r_out.data_ptr(), n_tokens, hidden, eps, _dtype_code(x),
+                                         workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                         chunk_tokens, _stream_ptr(stream)),
+           "rmsnorm_template_run_host")
+
+
+# ---- 2. the feasible region ---------------------------------------------------------------------------------
+
+def _collect(call, where: str) -> list[rt_params]:
+    n = c_int32(0)
+    _check(call(None, 0, byref(n)), where)
+    while True:
+        cap = max(1, n.value)
+        arr = (rt_params * cap)()
+        _check(call(arr, cap, byref(n)), where)
+        if n.value <= cap:
+            return [rt_params.from_buffer_copy(arr[i]) for i in range(n.value)]
+
+
+def tuner_derive_feasible(shape: rt_shape, limits: rt_limits | None = None,
+                          heuristics: int = RT_PRUNE_DEFAULT) -> list[rt_params]:
+    """Theta_feasible for a shape.  limits=None asks the current device."""
+    lim = byref(limits) if limits is not None else None
+    return _collect(lambda out, cap, n: lib.tuner_derive_feasible_ex(byref(shape), lim, heuristics, out, cap, n),
+                    "tuner_derive_feasible")
+
+
+def tuner_raw_grid(shape: rt_shape) -> list[rt_params]:
+    return _collect(lambda out, cap, n: lib.tuner_raw_grid(byref(shape), out, cap, n), "tuner_raw_grid")
+
+
+def tuner_derive_counts(shape: rt_shape, limits: rt_limits | None = None, heuristics: int = RT_PRUNE_DEFAULT) -> dict:
+    counts = (c_int32 * 11)()
+    lim = byref(limits) if limits is not None else None
+    _check(lib.tuner_derive_counts(byref(shape), lim, heuristics, counts, 11), "tuner_derive_counts")
+    names = ["unused", "arguments", "threads_per_cta", "alignment", "registers", "shared_memory", "cluster",
+             "grid", "heuristics", "feasible", "raw"]
+    return {k: int(v) for k, v in zip(names, counts) if k != "unused"}
+
+
+def tuner_check_params(shape: rt_shape, params: rt_params, limits: rt_limits | None = None) -> int:
+    lim = byref(limits) if limits is not None else None
+    return int(lib.tuner_check_params(byref(shape), lim, byref(params)))
+
+
+# ---- 3. search ------------------------------------------------------------------------------------------------
+
+def make_budget(max_evals=64, warmup=20, iters=100, repeats=3, top_k=5, strategy=RT_SEARCH_GUIDED,
+                heuristics=RT_PRUNE_DEFAULT, use_graph=False, seeds=None) -> rt_budget:
+    b = rt_budget(max_evals, warmup, iters, repeats, top_k, strategy, heuristics, int(use_graph), None, 0, 0)
+    if seeds:
+        arr = (rt_params * len(seeds))(*seeds)
+        b._seed_storage = arr  # keep alive
+        b.seeds = ctypes.cast(arr, POINTER(rt_params))
+        b.n_seeds = len(seeds)
+    return b
+
+
+def make_workspace(x, r, w, y, r_out, y_ref, r_ref, eps: float, n_ref_tokens: int | None = None, ring_sets: int = 1,
+                   ring_stride_bytes: int = 0, stream=None) -> rt_workspace:
+    """Device tensors for the tuner.  With ring_sets > 1, x, r, y, r_out are [ring_sets, T, H] and the
+    references cover set 0."""
+    T = x.shape[-2]
+    return rt_workspace(x.data_ptr(), r.data_ptr(), w.data_ptr(), y.data_ptr(), r_out.data_ptr(), y_ref.data_ptr(),
+                        r_ref.data_ptr(), n_ref_tokens if n_ref_tokens is not None else T, ring_stride_bytes,
+                        ring_sets, eps, _stream_ptr(stream))
+
+
+def tuner_search(shape: rt_shape, budget: rt_budget, ws: rt_workspace, log_cap: int = 4096):
+    """Returns (rt_result, [rt_eval_record...])."""
+    res = rt_result()
+    log = (rt_eval_record * log_cap)()
+    st = lib.tuner_search(byref(shape), byref(budget), byref(ws), byref(res), log, log_cap)
+    _check(st, "tuner_search")
+    return res, [rt_eval_record.from_buffer_copy(log[i]) for i in range(res.n_log)]
+
+
+def tuner_search_with(shape: rt_shape, limits: rt_limits, budget: rt_budget, evaluate, log_cap: int = 4096):
+    """The search over a Python cost function evaluate(theta) -> microseconds (negative: gate failed)."""
+    res = rt_result()
+    log = (rt_eval_record * log_cap)()
+    cb = rt_evaluate_fn(lambda p, _user: float(evaluate(p.contents)))
+    st = lib.tuner_search_with(byref(shape), byref(limits), byref(budget), cb, None, byref(res), log, log_cap)
+    _check(st, "tuner_search_with")
+    return res, [rt_eval_record.from_buffer_copy(log[i]) for i in range(res.n_log)]
+
+
+def tuner_evaluate(shape: rt_shape, params: rt_params, budget: rt_budget, ws: rt_workspace) -> rt_eval_record:
+    rec = rt_eval_record()
+    _check(lib.tuner_evaluate(byref(shape), byref(params), byref(budget), byref(ws), byref(rec)), "tuner_evaluate")
+    return rec
+
+
+def tuner_compare(got, ref, mode: int, tol: float = 0.0, stream=None):
+    """(max_err, n_bad) between two device tensors of one dtype."""
+    if got.shape != ref.shape or got.dtype != ref.dtype:
+        raise ValueError("got and ref must match")
+    worst, bad = c_double(0.0), c_int64(0)
+    _check(lib.tuner_compare(got.data_ptr(), ref.data_ptr(), got.numel(), _dtype_code(got), mode, tol, byref(worst),
+                             byref(bad), _stream_ptr(stream)), "tuner_compare")
+    return worst.value, bad.value
+
+
+def rt_device_status() -> int:
+    return int(lib.rt_device_status())
+
+
+def rt_launch_count() -> int:
+    return int(lib.rt_launch_count())
+
+
+def kernel_instances() -> list[dict]:
+    out = []
+    vals = [c_int32() for _ in range(6)]
+    for i in range(lib.rt_num_kernel_instances()):
+        _check(lib.rt_kernel_instance(i, *[byref(v) for v in vals]), "rt_kernel_instance")
+        out.append(dict(zip(("dtype", "vec_bytes", "stage", "reduce", "unroll", "reg_vectors"), (v.value for v in vals))))
+    return out
+
+
+def rt_shutdown() -> None:
+    lib.rt_shutdown()

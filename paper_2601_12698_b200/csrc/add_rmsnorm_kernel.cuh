@@ -1,0 +1,557 @@
+// Fused residual-add + RMSNorm as one explicitly parameterised kernel template (sm_100a).
+//
+// The template is the "parameterizable template" S~ of the paper's Algorithm 1 (Level 2) for the
+// kernel `fused_add_rmsnorm`; its axes are the execution-strategy dimensions named in "Tuning
+// parameter selection and search space derivation": thread-level granularity (threads per row,
+// rows per CTA: run-time block shape), vectorisation (VB bytes per ld/st), unrolling (U independent
+// loads in flight), and the organisation of shared memory and registers (STAGE, REDUCE).
+//
+// Compile-time axes: element type, VB, STAGE, REDUCE, U and - for the register stage - CAP, the
+// number of row vectors one thread keeps.  Run-time axes: blockDim.x = threads per row,
+// blockDim.y = rows per CTA, cluster size.
+//
+// Per row:  s = fp32(x) + fp32(r);  r_out = rn(s);  y = rn(s * rsqrt(mean(s^2) + eps) * w).
+// The sum of squares is combined in a fixed order (no atomics): results are deterministic.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <stdint.h>
+
+#include <type_traits>
+
+namespace rt {
+
+constexpr int kStageReg = 0;
+constexpr int kStageSmemLdg = 1;
+constexpr int kStageSmemTma = 2;
+constexpr int kReduceShfl = 0;
+constexpr int kReduceSmem = 1;
+constexpr int kReduceCluster = 2;
+
+constexpr int kMaxRowsPerCta = 8;
+constexpr int kMaxClusterSize = 8;
+constexpr int kDeviceTimeoutCode = 9;           // written to the status word when a bounded wait expires
+constexpr unsigned kMbarrierPollLimit = 1u << 24;        // polls of mbarrier.try_wait before giving up ...
+constexpr long long kMbarrierCycleLimit = 2000000000LL;  // ... or about one second of SM clock, whichever is first
+
+struct KernelArgs {
+    const void* x;
+    const void* r;
+    const void* w;
+    void* y;
+    void* r_out;
+    long long n_tokens;
+    int hidden;
+    int nvec;        // vectors of VB bytes in one row
+    int slice_nvec;  // vectors of one row owned by one CTA (== nvec unless the row is split over a cluster)
+    float eps;
+    int* status;     // device status word
+};
+
+// ---- vectors of VB bytes ------------------------------------------------------------------------
+
+template <int VB>
+struct Vec {
+    uint32_t w[(VB + 3) / 4];  // VB == 2 uses the low half of w[0]
+};
+
+// Streaming loads of x and r: read once, keep them out of L1.  Volatile, so that the order of
+// global loads and stores in the program is the order in the instruction stream: a batch of U loads
+// is issued together, and the next batch is not hoisted above this batch's stores.
+template <int VB>
+__device__ __forceinline__ Vec<VB> ld_stream(const void* p)
+{
+    Vec<VB> v;
+    if constexpr (VB == 16) {
+        asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(v.w[0]), "=r"(v.w[1]), "=r"(v.w[2]), "=r"(v.w[3]) : "l"(p));
+    } else if constexpr (VB == 8) {
+        asm volatile("ld.global.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(v.w[0]), "=r"(v.w[1]) : "l"(p));
+    } else if constexpr (VB == 4) {
+        asm volatile("ld.global.L1::no_allocate.u32 %0, [%1];" : "=r"(v.w[0]) : "l"(p));
+    } else {
+        unsigned short h;
+        asm volatile("ld.global.L1::no_allocate.u16 %0, [%1];" : "=h"(h) : "l"(p));
+        v.w[0] = h;
+    }
+    return v;
+}
+
+template <int VB>
+__device__ __forceinline__ void st_stream(void* p, const Vec<VB>& v)
+{
+    if constexpr (VB == 16) {
+        asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.w[0]), "r"(v.w[1]), "r"(v.w[2]),
+                     "r"(v.w[3]) : "memory");
+    } else if constexpr (VB == 8) {
+        asm volatile("st.global.v2.u32 [%0], {%1,%2};" ::"l"(p), "r"(v.w[0]), "r"(v.w[1]) : "memory");
+    } else if constexpr (VB == 4) {
+        asm volatile("st.global.u32 [%0], %1;" ::"l"(p), "r"(v.w[0]) : "memory");
+    } else {
+        asm volatile("st.global.u16 [%0], %1;" ::"l"(p), "h"((unsigned short)v.w[0]) : "memory");
+    }
+}
+
+// The weight vector is shared by every row: read-only path, cached.
+template <int VB>
+__device__ __forceinline__ Vec<VB> ld_weight(const void* p)
+{
+    Vec<VB> v;
+    if constexpr (VB == 16) {
+        const uint4 q = __ldg(reinterpret_cast<const uint4*>(p));
+        v.w[0] = q.x; v.w[1] = q.y; v.w[2] = q.z; v.w[3] = q.w;
+    } else if constexpr (VB == 8) {
+        const uint2 q = __ldg(reinterpret_cast<const uint2*>(p));
+        v.w[0] = q.x; v.w[1] = q.y;
+    } else if constexpr (VB == 4) {
+        v.w[0] = __ldg(reinterpret_cast<const unsigned int*>(p));
+    } else {
+        v.w[0] = __ldg(reinterpret_cast<const unsigned short*>(p));
+    }
+    return v;
+}
+
+template <int VB>
+__device__ __forceinline__ Vec<VB> ld_shared(const void* p)
+{
+    Vec<VB> v;
+    if constexpr (VB == 16) {
+        const uint4 q = *reinterpret_cast<const uint4*>(p);
+        v.w[0] = q.x; v.w[1] = q.y; v.w[2] = q.z; v.w[3] = q.w;
+    } else if constexpr (VB == 8) {
+        const uint2 q = *reinterpret_cast<const uint2*>(p);
+        v.w[0] = q.x; v.w[1] = q.y;
+    } else if constexpr (VB == 4) {
+        v.w[0] = *reinterpret_cast<const unsigned int*>(p);
+    } else {
+        v.w[0] = *reinterpret_cast<const unsigned short*>(p);
+    }
+    return v;
+}
+
+// ---- element codecs -----------------------------------------------------------------------------
+
+template <typename T, int VB>
+struct Codec {
+    static constexpr int EPV = VB / (int)sizeof(T);
+    static_assert(EPV >= 1, "vector narrower than one element");
+
+    static __device__ __forceinline__ void unpack(const Vec<VB>& v, float (&f)[EPV])
+    {
+        if constexpr (sizeof(T) == 4) {
+#pragma unroll
+            for (int i = 0; i < EPV; ++i) f[i] = __uint_as_float(v.w[i]);
+        } else if constexpr (EPV == 1) {
+            f[0] = to_float16(v.w[0] & 0xFFFFu);
+        } else {
+#pragma unroll
+            for (int i = 0; i < EPV / 2; ++i) {
+                f[2 * i] = to_float16(v.w[i] & 0xFFFFu);
+                f[2 * i + 1] = to_float16(v.w[i] >> 16);
+            }
+        }
+    }
+
+    static __device__ __forceinline__ Vec<VB> pack(const float (&f)[EPV])
+    {
+        Vec<VB> v;
+        if constexpr (sizeof(T) == 4) {
+#pragma unroll
+            for (int i = 0; i < EPV; ++i) v.w[i] = __float_as_uint(f[i]);
+        } else if constexpr (EPV == 1) {
+            v.w[0] = from_float16(f[0]);
+        } else {
+#pragma unroll
+            for (int i = 0; i < EPV / 2; ++i) v.w[i] = from_float16x2(f[2 * i], f[2 * i + 1]);
+        }
+        return v;
+    }
+
+    static __device__ __forceinline__ float to_float16(uint32_t bits)
+    {
+        if constexpr (sizeof(T) == 4) {
+            return 0.f;
+        } else if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+            return __uint_as_float(bits << 16);  // bf16 is the top half of a binary32
+        } else {
+            return __half2float(__ushort_as_half((unsigned short)bits));
+        }
+    }
+    static __device__ __forceinline__ uint32_t from_float16(float a)  // round to nearest even
+    {
+        if constexpr (sizeof(T) == 4) {
+            return 0u;
+        } else if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+            return __bfloat16_as_ushort(__float2bfloat16_rn(a));
+        } else {
+            return __half_as_ushort(__float2half_rn(a));
+        }
+    }
+    static __device__ __forceinline__ uint32_t from_float16x2(float lo, float hi)
+    {
+        if constexpr (sizeof(T) == 4) {
+            return 0u;
+        } else if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+            const __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
+            return *reinterpret_cast<const uint32_t*>(&p);
+        } else {
+            const __half2 p = __floats2half2_rn(lo, hi);
+            return *reinterpret_cast<const uint32_t*>(&p);
+        }
+    }
+};
+
+// ---- synchronisation helpers --------------------------------------------------------------------
+
+// Barrier over the threads of one row only (named barrier 1 + row); a warp-wide row needs no bar.
+__device__ __forceinline__ void row_sync(int row_in_cta, int threads_per_row)
+{
+    if (threads_per_row == 32) {
+        __syncwarp();
+    } else {
+        asm volatile("bar.sync %0, %1;" ::"r"(row_in_cta + 1), "r"(threads_per_row) : "memory");
+    }
+}
+
+__device__ __forceinline__ uint32_t cluster_cta_rank()
+{
+    uint32_t v;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(v));
+    return v;
+}
+__device__ __forceinline__ uint32_t cluster_num_ctas()
+{
+    uint32_t v;
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(v));
+    return v;
+}
+__device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_arrive_release() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait_acquire() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void st_cluster_f32(const float* local_slot, uint32_t peer_rank, float value)
+{
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(local_slot)), "r"(peer_rank));
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(value) : "memory");
+}
+
+__device__ __forceinline__ void mbarrier_init(uint64_t* bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbarrier_expect_tx(uint64_t* bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// One TMA bulk copy global -> this CTA's shared memory; completion is counted on `bar` in bytes.
+// Both addresses and the size are multiples of 16 bytes (checked on the host before launch).
+__device__ __forceinline__ void tma_bulk_load(void* smem_dst, const void* gmem_src, uint32_t bytes, uint64_t* bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(smem_dst)), "l"(gmem_src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+// Bounded wait for phase `parity` of `bar`.  Returns false when the poll limit is reached.
+__device__ __forceinline__ bool mbarrier_wait_bounded(uint64_t* bar, uint32_t parity)
+{
+    const uint32_t addr = smem_u32(bar);
+    const long long t0 = clock64();
+    for (unsigned it = 0; it < kMbarrierPollLimit; ++it) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done) : "r"(addr), "r"(parity) : "memory");
+        if (done) return true;
+        if ((it & 255u) == 255u && clock64() - t0 > kMbarrierCycleLimit) break;
+    }
+    return false;
+}
+
+// ---- the per-row reduction of the sum of squares ---------------------------------------------
+
+// Every thread of the row passes its partial; every thread of the row receives the row total.
+template <int REDUCE>
+__device__ __forceinline__ float row_reduce(float partial, int tx, int ty, int tpr, uint32_t crank, uint32_t csize)
+{
+    __shared__ float warp_part[kMaxRowsPerCta][32];
+    float total;
+    if constexpr (REDUCE == kReduceSmem) {
+        __shared__ float tree[1024];
+        float* mine = tree + ty * tpr;
+        mine[tx] = partial;
+        for (int stride = tpr >> 1; stride >= 1; stride >>= 1) {
+            row_sync(ty, tpr);
+            if (tx < stride) mine[tx] += mine[tx + stride];
+        }
+        row_sync(ty, tpr);
+        total = mine[0];
+    } else {
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) partial += __shfl_xor_sync(0xffffffffu, partial, off);
+        total = partial;
+        if (tpr > 32) {
+            const int lane = tx & 31, warp_in_row = tx >> 5, n_warps = tpr >> 5;
+            if (lane == 0) warp_part[ty][warp_in_row] = partial;
+            row_sync(ty, tpr);
+            float v = lane < n_warps ? warp_part[ty][lane] : 0.f;
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+            total = v;
+        }
+    }
+    if constexpr (REDUCE == kReduceCluster) {
+        // The row is split over the CTAs of a cluster: exchange CTA totals through distributed shared
+        // memory.  The first wait pairs with the arrive at kernel entry (all peers are running).
+        __shared__ float slot[kMaxRowsPerCta][kMaxClusterSize];
+        cluster_wait_acquire();
+        if (tx < (int)csize) st_cluster_f32(&slot[ty][crank], (uint32_t)tx, total);
+        cluster_arrive_release();
+        cluster_wait_acquire();
+        float v = 0.f;
+        for (uint32_t k = 0; k < csize; ++k) v += slot[ty][k];
+        total = v;
+    }
+    return total;
+}
+
+// ---- the kernel ---------------------------------------------------------------------------------
+
+// Shared-memory layout of the fp32 sums (STAGE == kStageSmemLdg): EPV floats of one vector are kept
+// as EPV/W chunks of W floats in separate planes, so that consecutive threads write consecutive
+// 16-byte (or 8/4-byte) chunks: no bank conflicts.
+template <int EPV>
+struct SumPlanes {
+    static constexpr int W = EPV >= 4 ? 4 : EPV;
+    static constexpr int PLANES = EPV / W;
+    static __device__ __forceinline__ void store(float* row_base, int slice_cap, int v, const float (&s)[EPV])
+    {
+#pragma unroll
+        for (int p = 0; p < PLANES; ++p) {
+            float* dst = row_base + ((size_t)p * slice_cap + v) * W;
+            if constexpr (W == 4) *reinterpret_cast<float4*>(dst) = make_float4(s[4 * p], s[4 * p + 1], s[4 * p + 2], s[4 * p + 3]);
+            else if constexpr (W == 2) *reinterpret_cast<float2*>(dst) = make_float2(s[0], s[1]);
+            else dst[0] = s[0];
+        }
+    }
+    static __device__ __forceinline__ void load(const float* row_base, int slice_cap, int v, float (&s)[EPV])
+    {
+#pragma unroll
+        for (int p = 0; p < PLANES; ++p) {
+            const float* src = row_base + ((size_t)p * slice_cap + v) * W;
+            if constexpr (W == 4) {
+                const float4 q = *reinterpret_cast<const float4*>(src);
+                s[4 * p] = q.x; s[4 * p + 1] = q.y; s[4 * p + 2] = q.z; s[4 * p + 3] = q.w;
+            } else if constexpr (W == 2) {
+                const float2 q = *reinterpret_cast<const float2*>(src);
+                s[0] = q.x; s[1] = q.y;
+            } else {
+                s[0] = src[0];
+            }
+        }
+    }
+};
+
+template <typename T, int VB, int STAGE, int REDUCE, int U, int CAP>
+__global__ void add_rmsnorm_kernel(const KernelArgs a)
+{
+    using C = Codec<T, VB>;
+    constexpr int EPV = C::EPV;
+    static_assert(STAGE != kStageReg || CAP % U == 0, "the unroll depth divides the per-thread vector count");
+    extern __shared__ __align__(128) unsigned char dyn_smem[];
+
+    const int tx = threadIdx.x, ty = threadIdx.y, tpr = blockDim.x;
+    uint32_t crank = 0, csize = 1;
+    long long row_block = blockIdx.x;
+    if constexpr (REDUCE == kReduceCluster) {
+        cluster_arrive_relaxed();  // matched by the first wait inside row_reduce
+        crank = cluster_cta_rank();
+        csize = cluster_num_ctas();
+        row_block = blockIdx.x / csize;
+    }
+    const long long row = row_block * blockDim.y + ty;
+    const int v_begin = (int)crank * a.slice_nvec;
+    int n = a.nvec - v_begin;              // vectors of this row owned by this CTA
+    if (n > a.slice_nvec) n = a.slice_nvec;
+    if (n < 0 || row >= a.n_tokens) n = 0;  // rows past the end and empty slices still reach every barrier
+
+    const size_t row_off = ((size_t)(row < a.n_tokens ? row : 0) * (size_t)a.nvec + (size_t)v_begin) * VB;
+    const unsigned char* xrow = reinterpret_cast<const unsigned char*>(a.x) + row_off;
+    const unsigned char* rrow = reinterpret_cast<const unsigned char*>(a.r) + row_off;
+    const unsigned char* wrow = reinterpret_cast<const unsigned char*>(a.w) + (size_t)v_begin * VB;
+    unsigned char* yrow = reinterpret_cast<unsigned char*>(a.y) + row_off;
+    unsigned char* orow = reinterpret_cast<unsigned char*>(a.r_out) + row_off;
+
+    float ss = 0.f;
+
+    if constexpr (STAGE == kStageReg) {
+        float s[CAP][EPV];
+#pragma unroll
+        for (int i0 = 0; i0 < CAP; i0 += U) {
+            Vec<VB> xv[U], rv[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int v = tx + (i0 + u) * tpr;
+                if (v < n) xv[u] = ld_stream<VB>(xrow + (size_t)v * VB);
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int v = tx + (i0 + u) * tpr;
+                if (v < n) rv[u] = ld_stream<VB>(rrow + (size_t)v * VB);
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int v = tx + (i0 + u) * tpr;
+                if (v < n) {
+                    float xf[EPV], rf[EPV];
+                    C::unpack(xv[u], xf);
+                    C::unpack(rv[u], rf);
+#pragma unroll
+                    for (int e = 0; e < EPV; ++e) {
+                        s[i0 + u][e] = xf[e] + rf[e];
+                        ss = fmaf(s[i0 + u][e], s[i0 + u][e], ss);
+                    }
+                    st_stream<VB>(orow + (size_t)v * VB, C::pack(s[i0 + u]));
+                }
+            }
+        }
+        const float total = row_reduce<REDUCE>(ss, tx, ty, tpr, crank, csize);
+        const float rho = __frsqrt_rn(total / (float)a.hidden + a.eps);
+#pragma unroll
+        for (int i = 0; i < CAP; ++i) {
+            const int v = tx + i * tpr;
+            if (v < n) {
+                float wf[EPV], yf[EPV];
+                C::unpack(ld_weight<VB>(wrow + (size_t)v * VB), wf);
+#pragma unroll
+                for (int e = 0; e < EPV; ++e) yf[e] = s[i][e] * rho * wf[e];
+                st_stream<VB>(yrow + (size_t)v * VB, C::pack(yf));
+            }
+        }
+    } else if constexpr (STAGE == kStageSmemLdg) {
+        using P = SumPlanes<EPV>;
+        float* srow = reinterpret_cast<float*>(dyn_smem) + (size_t)ty * a.slice_nvec * EPV;
+        for (int v0 = tx; v0 < n; v0 += U * tpr) {
+            Vec<VB> xv[U], rv[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int v = v0 + u * tpr;
+                if (v < n) xv[u] = ld_stream<VB>(xrow + (size_t)v * VB);
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int v = v0 + u * tpr;
+                if (v < n) rv[u] = ld_stream<VB>(rrow + (size_t)v * VB);
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int v = v0 + u * tpr;
+                if (v < n) {
+                    float xf[EPV], rf[EPV], s[EPV];
+                    C::unpack(xv[u], xf);
+                    C::unpack(rv[u], rf);
+#pragma unroll
+                    for (int e = 0; e < EPV; ++e) {
+                        s[e] = xf[e] + rf[e];
+                        ss = fmaf(s[e], s[e], ss);
+                    }
+                    st_stream<VB>(orow + (size_t)v * VB, C::pack(s));
+                    P::store(srow, a.slice_nvec, v, s);  // read back by this same thread only
+                }
+            }
+        }
+        const float total = row_reduce<REDUCE>(ss, tx, ty, tpr, crank, csize);
+        const float rho = __frsqrt_rn(total / (float)a.hidden + a.eps);
+        for (int v0 = tx; v0 < n; v0 += U * tpr) {
+            Vec<VB> wv[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int v = v0 + u * tpr;
+                if (v < n) wv[u] = ld_weight<VB>(wrow + (size_t)v * VB);
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int v = v0 + u * tpr;
+                if (v < n) {
+                    float s[EPV], wf[EPV], yf[EPV];
+                    P::load(srow, a.slice_nvec, v, s);
+                    C::unpack(wv[u], wf);
+#pragma unroll
+                    for (int e = 0; e < EPV; ++e) yf[e] = s[e] * rho * wf[e];
+                    st_stream<VB>(yrow + (size_t)v * VB, C::pack(yf));
+                }
+            }
+        }
+    } else {
+        // TMA: one thread per row posts two bulk copies (x slice, r slice) that complete on the row's
+        // mbarrier; the row's threads then work out of shared memory.
+        __shared__ __align__(8) uint64_t bars[kMaxRowsPerCta];
+        const size_t slice_bytes = (size_t)a.slice_nvec * VB;
+        unsigned char* xs = dyn_smem + (size_t)ty * 2 * slice_bytes;
+        unsigned char* rs = xs + slice_bytes;
+        if (tx == 0) {
+            mbarrier_init(&bars[ty], 1);
+            if (n > 0) {
+                const uint32_t bytes = (uint32_t)n * VB;
+                mbarrier_expect_tx(&bars[ty], 2 * bytes);
+                tma_bulk_load(xs, xrow, bytes, &bars[ty]);
+                tma_bulk_load(rs, rrow, bytes, &bars[ty]);
+            }
+        }
+        row_sync(ty, tpr);  // the barrier is initialised before anyone polls it
+        if (n > 0) {
+            bool landed = mbarrier_wait_bounded(&bars[ty], 0);
+            if (!landed) {
+                atomicExch(a.status, kDeviceTimeoutCode);
+                landed = mbarrier_wait_bounded(&bars[ty], 0);  // do not leave while the copies may still land
+            }
+        }
+        for (int v0 = tx; v0 < n; v0 += U * tpr) {
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int v = v0 + u * tpr;
+                if (v < n) {
+                    float xf[EPV], rf[EPV], s[EPV];
+                    C::unpack(ld_shared<VB>(xs + (size_t)v * VB), xf);
+                    C::unpack(ld_shared<VB>(rs + (size_t)v * VB), rf);
+#pragma unroll
+                    for (int e = 0; e < EPV; ++e) {
+                        s[e] = xf[e] + rf[e];
+                        ss = fmaf(s[e], s[e], ss);
+                    }
+                    st_stream<VB>(orow + (size_t)v * VB, C::pack(s));
+                }
+            }
+        }
+        const float total = row_reduce<REDUCE>(ss, tx, ty, tpr, crank, csize);
+        const float rho = __frsqrt_rn(total / (float)a.hidden + a.eps);
+        for (int v0 = tx; v0 < n; v0 += U * tpr) {
+            Vec<VB> wv[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int v = v0 + u * tpr;
+                if (v < n) wv[u] = ld_weight<VB>(wrow + (size_t)v * VB);
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int v = v0 + u * tpr;
+                if (v < n) {
+                    float xf[EPV], rf[EPV], wf[EPV], yf[EPV];
+                    C::unpack(ld_shared<VB>(xs + (size_t)v * VB), xf);
+                    C::unpack(ld_shared<VB>(rs + (size_t)v * VB), rf);
+                    C::unpack(wv[u], wf);
+#pragma unroll
+                    for (int e = 0; e < EPV; ++e) yf[e] = (xf[e] + rf[e]) * rho * wf[e];  // same binary32 sum as pass 1
+                    st_stream<VB>(yrow + (size_t)v * VB, C::pack(yf));
+                }
+            }
+        }
+    }
+}
+
+}  // namespace rt

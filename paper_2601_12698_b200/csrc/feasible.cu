@@ -1,0 +1,192 @@
+// DeriveFeasibleSpace(S~, h, r(h)): the raw parameter grid, the hard rules (make_plan) and the
+// switchable "obvious inefficiency" rules, after the paper's Section "Tuning parameter selection and
+// search space derivation".
+#include <string.h>
+
+#include "tuner_internal.h"
+
+namespace rt {
+
+namespace {
+
+const int kTprLevels[] = {32, 64, 128, 256, 512, 1024};
+const int kRpcLevels[] = {1, 2, 4, 8};
+const int kUnrollLevels[] = {1, 2, 4};
+struct Mode {
+    int reduce, cluster;
+};
+const Mode kReduceModes[] = {{RT_REDUCE_SHFL, 1}, {RT_REDUCE_SMEM, 1}, {RT_REDUCE_CLUSTER, 2},
+                             {RT_REDUCE_CLUSTER, 4}, {RT_REDUCE_CLUSTER, 8}};
+
+int next_pow2(int v)
+{
+    int p = 1;
+    while (p < v) p <<= 1;
+    return p;
+}
+
+// Vector widths offered for a shape: 16 and 8 bytes (the tuned axis); when the row length or a base
+// pointer allows neither, the widest narrower width that fits (a fall-back, not a tuned axis).
+std::vector<int> vec_levels(const rt_shape& s)
+{
+    const int eb = elem_bytes_of(s.dtype);
+    const int64_t row_bytes = s.hidden * eb;
+    auto fits = [&](int vb) { return vb >= eb && row_bytes % vb == 0 && s.min_ptr_align >= vb; };
+    if (fits(16) || fits(8)) return {16, 8};
+    if (fits(4)) return {4};
+    if (fits(2)) return {2};
+    return {16, 8};  // nothing fits: the hard rules reject every point and say why
+}
+
+}  // namespace
+
+uint64_t pack_params(const rt_params& p)
+{
+    return ((uint64_t)(uint16_t)p.threads_per_row) | ((uint64_t)(uint8_t)p.rows_per_cta << 16) |
+           ((uint64_t)(uint8_t)p.vec_bytes << 24) | ((uint64_t)(uint8_t)p.unroll << 32) |
+           ((uint64_t)(uint8_t)p.stage << 40) | ((uint64_t)(uint8_t)p.reduce << 44) |
+           ((uint64_t)(uint8_t)p.cluster_size << 48);
+}
+
+std::vector<rt_params> raw_grid(const rt_shape& s)
+{
+    std::vector<rt_params> out;
+    const std::vector<int> vecs = vec_levels(s);
+    for (int stage = 0; stage < 3; ++stage)
+        for (const Mode& m : kReduceModes)
+            for (int vb : vecs)
+                for (int tpr : kTprLevels)
+                    for (int rpc : kRpcLevels)
+                        for (int u : kUnrollLevels) {
+                            rt_params p;
+                            p.threads_per_row = tpr;
+                            p.rows_per_cta = rpc;
+                            p.vec_bytes = vb;
+                            p.unroll = u;
+                            p.stage = stage;
+                            p.reduce = m.reduce;
+                            p.cluster_size = m.cluster;
+                            out.push_back(p);
+                        }
+    return out;
+}
+
+// The heuristic rules.  Returns the RT_PRUNE_* bit of the first rule that removes theta, or 0.
+static int heuristic_reject(const rt_shape& s, const rt_limits& L, const rt_params& p, const Plan& plan, int mask)
+{
+    if ((mask & RT_PRUNE_IDLE_THREADS) && p.threads_per_row > plan.slice_nvec) return RT_PRUNE_IDLE_THREADS;
+    if (mask & RT_PRUNE_DUPLICATES) {
+        // A batch deeper than the vectors a thread owns only adds predicated-off slots.
+        if (p.unroll > next_pow2(plan.vec_per_thread)) return RT_PRUNE_DUPLICATES;
+    }
+    if ((mask & RT_PRUNE_CLUSTER_WAVES) && p.cluster_size > 1) {
+        // Splitting rows is for shapes with too few rows to occupy the SMs: allow a split into C only
+        // while the next smaller split still leaves SMs without a CTA.
+        const int64_t row_ctas = (s.n_tokens + p.rows_per_cta - 1) / p.rows_per_cta;
+        if (row_ctas * (p.cluster_size / 2) >= L.sm_count) return RT_PRUNE_CLUSTER_WAVES;
+    }
+    if ((mask & RT_PRUNE_IDLE_ROWS) && s.n_tokens > 0 && p.rows_per_cta > s.n_tokens) return RT_PRUNE_IDLE_ROWS;
+    return 0;
+}
+
+int derive_feasible(const rt_shape& s, const rt_limits& L, int heuristics, std::vector<rt_params>* out, int32_t* counts)
+{
+    int32_t local[kRejectReasons + 3];
+    memset(local, 0, sizeof(local));
+    if (s.dtype < 0 || s.dtype > 2) {
+        set_error("dtype %d is not one of bf16(0), fp16(1), fp32(2)", s.dtype);
+        return RT_ERR_DTYPE;
+    }
+    if (s.n_tokens < 0 || s.hidden <= 0 || s.hidden * elem_bytes_of(s.dtype) >= (int64_t)1 << 31) {
+        set_error("shape n_tokens=%lld hidden=%lld is out of range", (long long)s.n_tokens, (long long)s.hidden);
+        return RT_ERR_SHAPE;
+    }
+    const std::vector<rt_params> raw = raw_grid(s);
+    local[kRejectReasons + 2] = (int32_t)raw.size();
+    for (const rt_params& p : raw) {
+        Plan plan;
+        const int st = make_plan(&s, &p, &L, &plan);
+        if (st == RT_ERR_CUDA || st == RT_ERR_NO_DEVICE) return st;
+        if (st != RT_OK) {
+            local[plan.reject_reason < kRejectReasons ? plan.reject_reason : kRejectArgs]++;
+            continue;
+        }
+        if (plan_occupancy(plan, &L, nullptr) < 1) {
+            local[plan.dyn_smem > 0 ? kRejectSmem : kRejectRegisters]++;
+            continue;
+        }
+        if (heuristic_reject(s, L, p, plan, heuristics)) {
+            local[kRejectReasons]++;
+            continue;
+        }
+        local[kRejectReasons + 1]++;
+        if (out) out->push_back(p);
+    }
+    if (counts) memcpy(counts, local, sizeof(local));
+    return RT_OK;
+}
+
+}  // namespace rt
+
+extern "C" {
+
+int tuner_derive_feasible_ex(const rt_shape* s, const rt_limits* limits, int32_t heuristics, rt_params* out,
+                             int32_t cap, int32_t* n_out)
+{
+    if (!s || !n_out || (cap > 0 && !out)) {
+        rt::set_error("tuner_derive_feasible: NULL argument");
+        return RT_ERR_NULL;
+    }
+    rt_limits L;
+    if (!limits) {
+        int st = rt::current_limits(&L);
+        if (st != RT_OK) return st;
+        limits = &L;
+    }
+    std::vector<rt_params> v;
+    int st = rt::derive_feasible(*s, *limits, heuristics, &v, nullptr);
+    if (st != RT_OK) return st;
+    *n_out = (int32_t)v.size();
+    const int32_t n_copy = std::min<int32_t>(cap, (int32_t)v.size());
+    for (int32_t i = 0; i < n_copy; ++i) out[i] = v[i];
+    return RT_OK;
+}
+
+int tuner_derive_feasible(const rt_shape* s, rt_params* out, int32_t cap, int32_t* n_out)
+{
+    return tuner_derive_feasible_ex(s, nullptr, RT_PRUNE_DEFAULT, out, cap, n_out);
+}
+
+int tuner_derive_counts(const rt_shape* s, const rt_limits* limits, int32_t heuristics, int32_t* counts, int32_t n_counts)
+{
+    if (!s || !counts) {
+        rt::set_error("tuner_derive_counts: NULL argument");
+        return RT_ERR_NULL;
+    }
+    if (n_counts < rt::kRejectReasons + 3) {
+        rt::set_error("counts needs %d entries", rt::kRejectReasons + 3);
+        return RT_ERR_CAPACITY;
+    }
+    rt_limits L;
+    if (!limits) {
+        int st = rt::current_limits(&L);
+        if (st != RT_OK) return st;
+        limits = &L;
+    }
+    return rt::derive_feasible(*s, *limits, heuristics, nullptr, counts);
+}
+
+int tuner_raw_grid(const rt_shape* s, rt_params* out, int32_t cap, int32_t* n_out)
+{
+    if (!s || !n_out || (cap > 0 && !out)) {
+        rt::set_error("tuner_raw_grid: NULL argument");
+        return RT_ERR_NULL;
+    }
+    const std::vector<rt_params> v = rt::raw_grid(*s);
+    *n_out = (int32_t)v.size();
+    const int32_t n_copy = std::min<int32_t>(cap, (int32_t)v.size());
+    for (int32_t i = 0; i < n_copy; ++i) out[i] = v[i];
+    return RT_OK;
+}
+
+}  // extern "C"

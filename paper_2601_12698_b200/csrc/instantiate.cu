@@ -1,0 +1,67 @@
+// One instantiation unit of the kernel template.  Compiled once per line of instance_units.inc with
+//   -DRT_UNIT_NAME=<name> -DRT_UNIT_T=<element type> -DRT_UNIT_DTYPE=<0|1|2> -DRT_UNIT_VB=<bytes>
+//   -DRT_UNIT_GROUP=<0 register stage | 1 shared-memory stages | 2 narrow fall-back>
+//   -DRT_UNIT_REDUCE=<0|1|2>   (register-stage units only)
+//
+// Instance lists.  Register stage: CAP (row vectors kept per thread) in {1,2,4,8,16,32} while the row
+// stays within 128 fp32 registers per thread, unroll U in {1,2,4} with U <= CAP.  Shared-memory
+// stages: U in {1,2,4}, all three reductions.  Narrow fall-back (4- and 2-byte vectors, for rows whose
+// byte length is not a multiple of 8): register stage, shuffle reduction, U in {1,4}.
+#include "add_rmsnorm_kernel.cuh"
+#include "tuner_internal.h"
+
+namespace {
+
+using T = RT_UNIT_T;
+constexpr int kDtype = RT_UNIT_DTYPE;
+constexpr int kVB = RT_UNIT_VB;
+constexpr int kEPV = kVB / (int)sizeof(T);
+constexpr int kMaxRowRegisters = 128;
+
+template <int ST, int RD, int U, int CAP>
+rt::KernelEntry entry()
+{
+    if constexpr (ST == rt::kStageReg && CAP * kEPV > kMaxRowRegisters) {
+        return rt::KernelEntry{kDtype, kVB, ST, RD, U, CAP, nullptr};  // not instantiated
+    } else {
+        return rt::KernelEntry{kDtype, kVB, ST, RD, U, ST == rt::kStageReg ? CAP : 0,
+                               (const void*)&rt::add_rmsnorm_kernel<T, kVB, ST, RD, U, CAP>};
+    }
+}
+
+#define RT_REG_LIST(RD)                                                                                   \
+    entry<0, RD, 1, 1>(), entry<0, RD, 1, 2>(), entry<0, RD, 2, 2>(), entry<0, RD, 1, 4>(), entry<0, RD, 2, 4>(), \
+    entry<0, RD, 4, 4>(), entry<0, RD, 1, 8>(), entry<0, RD, 2, 8>(), entry<0, RD, 4, 8>(), entry<0, RD, 1, 16>(), \
+    entry<0, RD, 2, 16>(), entry<0, RD, 4, 16>(), entry<0, RD, 1, 32>(), entry<0, RD, 2, 32>(), entry<0, RD, 4, 32>()
+#define RT_SMEM_LIST(ST)                                                                                   \
+    entry<ST, 0, 1, 1>(), entry<ST, 0, 2, 1>(), entry<ST, 0, 4, 1>(), entry<ST, 1, 1, 1>(), entry<ST, 1, 2, 1>(), \
+    entry<ST, 1, 4, 1>(), entry<ST, 2, 1, 1>(), entry<ST, 2, 2, 1>(), entry<ST, 2, 4, 1>()
+
+std::vector<rt::KernelEntry> build_entries()
+{
+    std::vector<rt::KernelEntry> all = {
+#if RT_UNIT_GROUP == 0
+        RT_REG_LIST(RT_UNIT_REDUCE)
+#elif RT_UNIT_GROUP == 1
+        RT_SMEM_LIST(1), RT_SMEM_LIST(2)
+#else
+        entry<0, 0, 1, 1>(), entry<0, 0, 1, 2>(), entry<0, 0, 1, 4>(), entry<0, 0, 4, 4>(), entry<0, 0, 1, 8>(),
+        entry<0, 0, 4, 8>(), entry<0, 0, 1, 16>(), entry<0, 0, 4, 16>(), entry<0, 0, 1, 32>(), entry<0, 0, 4, 32>()
+#endif
+    };
+    std::vector<rt::KernelEntry> kept;
+    for (const rt::KernelEntry& e : all)
+        if (e.fn) kept.push_back(e);
+    return kept;
+}
+
+}  // namespace
+
+#define RT_CAT2(a, b) a##b
+#define RT_CAT(a, b) RT_CAT2(a, b)
+
+rt::KernelSlice RT_CAT(rt_kernel_slice_, RT_UNIT_NAME)()
+{
+    static const std::vector<rt::KernelEntry> entries = build_entries();
+    return rt::KernelSlice{entries.data(), (int)entries.size()};
+}

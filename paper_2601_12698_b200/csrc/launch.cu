@@ -1,0 +1,621 @@
+// Instance registry, resource limits r(h), the hard feasibility rules and the launch path.
+#include <cuda_runtime.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <atomic>
+#include <mutex>
+#include <unordered_map>
+
+#include "add_rmsnorm_kernel.cuh"
+#include "tuner_internal.h"
+
+// Each instantiation unit exports its slice of the instance table.
+#define RT_DECLARE_SLICE(name) rt::KernelSlice rt_kernel_slice_##name();
+#include "instance_units.inc"
+#undef RT_DECLARE_SLICE
+
+namespace rt {
+
+__device__ int g_status_word = 0;
+
+namespace {
+
+thread_local char tls_error[512] = "";
+std::atomic<int64_t> g_launches{0};
+std::mutex g_mutex;
+
+constexpr int kMaxDevices = 64;
+struct DeviceCache {
+    bool limits_ready = false;
+    rt_limits limits;
+    int* status_ptr = nullptr;
+    std::vector<KernelInfo> info;       // per instance
+    std::vector<char> info_ready;
+    std::vector<size_t> dyn_smem_set;   // largest dynamic shared memory opted in so far
+};
+DeviceCache g_dev[kMaxDevices];
+
+uint64_t key_of(int dtype, int vb, int stage, int reduce, int unroll, int cap)
+{
+    return ((uint64_t)dtype << 40) | ((uint64_t)vb << 32) | ((uint64_t)stage << 28) | ((uint64_t)reduce << 24) |
+           ((uint64_t)unroll << 16) | (uint64_t)cap;
+}
+
+struct Registry {
+    std::vector<KernelEntry> entries;
+    std::unordered_map<uint64_t, int> index;
+    Registry()
+    {
+#define RT_DECLARE_SLICE(name)                                             \
+    {                                                                      \
+        KernelSlice s = rt_kernel_slice_##name();                          \
+        for (int i = 0; i < s.n; ++i) entries.push_back(s.entries[i]);     \
+    }
+#include "instance_units.inc"
+#undef RT_DECLARE_SLICE
+        for (int i = 0; i < (int)entries.size(); ++i) {
+            const KernelEntry& e = entries[i];
+            index[key_of(e.dtype, e.vec_bytes, e.stage, e.reduce, e.unroll, e.cap)] = i;
+        }
+    }
+};
+Registry& reg()
+{
+    static Registry r;
+    return r;
+}
+
+int current_device_cache(DeviceCache** out)
+{
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        (void)cudaGetLastError();
+        set_error("no usable CUDA device (%s)", e == cudaSuccess ? "device index out of range" : cudaGetErrorString(e));
+        return RT_ERR_NO_DEVICE;
+    }
+    *out = &g_dev[dev];
+    return RT_OK;
+}
+
+int next_pow2(int v)
+{
+    int p = 1;
+    while (p < v) p <<= 1;
+    return p;
+}
+bool is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
+
+}  // namespace
+
+void set_error(const char* fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(tls_error, sizeof(tls_error), fmt, ap);
+    va_end(ap);
+}
+const char* last_error() { return tls_error; }
+void count_launch(int64_t n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+const std::vector<KernelEntry>& registry() { return reg().entries; }
+
+int find_kernel(int dtype, int vb, int stage, int reduce, int unroll, int cap)
+{
+    auto it = reg().index.find(key_of(dtype, vb, stage, reduce, unroll, cap));
+    return it == reg().index.end() ? -1 : it->second;
+}
+
+int current_limits(rt_limits* out)
+{
+    DeviceCache* dc;
+    int st = current_device_cache(&dc);
+    if (st != RT_OK) return st;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (!dc->limits_ready) {
+        int dev = 0;
+        RT_CUDA_OK(cudaGetDevice(&dev));
+        cudaDeviceProp prop;
+        RT_CUDA_OK(cudaGetDeviceProperties(&prop, dev));
+        rt_limits& l = dc->limits;
+        memset(&l, 0, sizeof(l));
+        l.sm_count = prop.multiProcessorCount;
+        l.warp_size = prop.warpSize;
+        l.max_threads_per_block = prop.maxThreadsPerBlock;
+        l.max_threads_per_sm = prop.maxThreadsPerMultiProcessor;
+        l.max_blocks_per_sm = prop.maxBlocksPerMultiProcessor;
+        l.regs_per_block = prop.regsPerBlock;
+        l.regs_per_sm = prop.regsPerMultiprocessor;
+        l.max_regs_per_thread = 255;
+        l.max_cluster_size = prop.major >= 9 ? 8 : 1;  // portable cluster size
+        l.have_device = 1;
+        l.smem_per_block_optin = (int64_t)prop.sharedMemPerBlockOptin;
+        l.smem_per_sm = (int64_t)prop.sharedMemPerMultiprocessor;
+        l.smem_reserved_per_block = (int64_t)prop.reservedSharedMemPerBlock;
+        l.l2_bytes = (int64_t)prop.l2CacheSize;
+        dc->limits_ready = true;
+    }
+    *out = dc->limits;
+    return RT_OK;
+}
+
+int kernel_info(int index, KernelInfo* out)
+{
+    DeviceCache* dc;
+    int st = current_device_cache(&dc);
+    if (st != RT_OK) return st;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    const size_t n = reg().entries.size();
+    if (dc->info.size() != n) {
+        dc->info.assign(n, KernelInfo{});
+        dc->info_ready.assign(n, 0);
+        dc->dyn_smem_set.assign(n, 48 * 1024);
+    }
+    if (!dc->info_ready[index]) {
+        cudaFuncAttributes fa;
+        RT_CUDA_OK(cudaFuncGetAttributes(&fa, reg().entries[index].fn));
+        KernelInfo& k = dc->info[index];
+        k.regs_per_thread = fa.numRegs;
+        k.local_bytes = (int)fa.localSizeBytes;
+        k.static_smem = (int)fa.sharedSizeBytes;
+        k.max_threads = fa.maxThreadsPerBlock;
+        dc->info_ready[index] = 1;
+    }
+    *out = dc->info[index];
+    return RT_OK;
+}
+
+// Kernels that need more than 48 KB of dynamic shared memory must opt in.  The opt-in is made once per
+// instance and device, to the largest size the device allows, so that occupancy queries and launches
+// see one fixed setting whatever order they come in.
+int ensure_dynamic_smem(int index, size_t bytes)
+{
+    if (bytes <= 48 * 1024) return RT_OK;
+    KernelInfo ki;
+    int st = kernel_info(index, &ki);  // also sizes the per-device tables
+    if (st != RT_OK) return st;
+    rt_limits L;
+    st = current_limits(&L);
+    if (st != RT_OK) return st;
+    DeviceCache* dc;
+    st = current_device_cache(&dc);
+    if (st != RT_OK) return st;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (dc->dyn_smem_set[index] < bytes) {
+        const size_t most = (size_t)L.smem_per_block_optin - (size_t)ki.static_smem;
+        if (bytes > most) {
+            set_error("%zu bytes of dynamic shared memory exceed the %zu this instance may opt in to", bytes, most);
+            return RT_ERR_INFEASIBLE;
+        }
+        RT_CUDA_OK(cudaFuncSetAttribute(reg().entries[index].fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)most));
+        dc->dyn_smem_set[index] = most;
+    }
+    return RT_OK;
+}
+
+int* device_status_word()
+{
+    DeviceCache* dc;
+    if (current_device_cache(&dc) != RT_OK) return nullptr;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (!dc->status_ptr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_status_word) != cudaSuccess) {
+            set_error("cudaGetSymbolAddress(status word) failed: %s", cudaGetErrorString(cudaGetLastError()));
+            return nullptr;
+        }
+        dc->status_ptr = (int*)p;
+    }
+    return dc->status_ptr;
+}
+
+int min_pointer_alignment(const void* a, const void* b, const void* c, const void* d, const void* e)
+{
+    const uintptr_t bits = (uintptr_t)a | (uintptr_t)b | (uintptr_t)c | (uintptr_t)d | (uintptr_t)e | 256u;
+    return (int)(bits & (~bits + 1));
+}
+
+// Registers per thread and static shared memory when no device can be asked: a plain model of what
+// the template needs (the row's fp32 sums, the loads in flight, addressing).
+static int model_regs(const KernelEntry& k, int elem_bytes)
+{
+    const int epv = k.vec_bytes / elem_bytes;
+    const int words = (k.vec_bytes + 3) / 4;
+    if (k.stage == kStageReg) return 28 + k.cap * epv + 2 * k.unroll * words;
+    return 36 + 2 * k.unroll * words + 2 * epv;
+}
+static int model_static_smem(const KernelEntry& k)
+{
+    int b = 1024;                                   // per-warp partials
+    if (k.reduce == kReduceSmem) b += 4096;         // halving tree
+    if (k.reduce == kReduceCluster) b += 256;       // cluster slots
+    if (k.stage == kStageSmemTma) b += 64;          // mbarriers
+    return b;
+}
+
+int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* plan)
+{
+    if (!s || !p || !L || !plan) {
+        set_error("make_plan: NULL argument");
+        return RT_ERR_NULL;
+    }
+    memset(plan, 0, sizeof(*plan));
+    if (s->dtype < 0 || s->dtype > 2) {
+        set_error("dtype %d is not one of bf16(0), fp16(1), fp32(2)", s->dtype);
+        plan->reject_reason = kRejectArgs;
+        return RT_ERR_DTYPE;
+    }
+    const int eb = elem_bytes_of(s->dtype);
+    if (s->n_tokens < 0 || s->hidden <= 0 || s->hidden * eb >= (int64_t)1 << 31) {
+        set_error("shape n_tokens=%lld hidden=%lld is out of range", (long long)s->n_tokens, (long long)s->hidden);
+        plan->reject_reason = kRejectArgs;
+        return RT_ERR_SHAPE;
+    }
+    const int tpr = p->threads_per_row, rpc = p->rows_per_cta, vb = p->vec_bytes;
+    if (!is_pow2(tpr) || tpr < L->warp_size || tpr > 1024) {
+        set_error("threads_per_row=%d must be a power of two between the warp size and 1024", tpr);
+        plan->reject_reason = kRejectThreads;
+        return RT_ERR_INFEASIBLE;
+    }
+    if (rpc < 1 || rpc > kMaxRowsPerCta) {
+        set_error("rows_per_cta=%d outside 1..%d", rpc, kMaxRowsPerCta);
+        plan->reject_reason = kRejectThreads;
+        return RT_ERR_INFEASIBLE;
+    }
+    if (tpr * rpc > L->max_threads_per_block) {
+        set_error("block of %d x %d threads exceeds the %d threads a CTA may have", tpr, rpc, L->max_threads_per_block);
+        plan->reject_reason = kRejectThreads;
+        return RT_ERR_INFEASIBLE;
+    }
+    if (!(vb == 16 || vb == 8 || vb == 4 || vb == 2) || vb < eb) {
+        set_error("vec_bytes=%d is not 16, 8, 4 or 2, or is narrower than one element", vb);
+        plan->reject_reason = kRejectArgs;
+        return RT_ERR_INFEASIBLE;
+    }
+    if (!(p->unroll == 1 || p->unroll == 2 || p->unroll == 4)) {
+        set_error("unroll=%d is not 1, 2 or 4", p->unroll);
+        plan->reject_reason = kRejectArgs;
+        return RT_ERR_INFEASIBLE;
+    }
+    if (p->stage < 0 || p->stage > 2 || p->reduce < 0 || p->reduce > 2) {
+        set_error("stage=%d or reduce=%d unknown", p->stage, p->reduce);
+        plan->reject_reason = kRejectArgs;
+        return RT_ERR_INFEASIBLE;
+    }
+    const int C = p->cluster_size;
+    if (p->reduce == RT_REDUCE_CLUSTER) {
+        if (!(C == 2 || C == 4 || C == 8) || C > L->max_cluster_size) {
+            set_error("cluster_size=%d is not 2, 4 or 8 within the device's limit of %d", C, L->max_cluster_size);
+            plan->reject_reason = kRejectCluster;
+        return RT_ERR_INFEASIBLE;
+        }
+    } else if (C != 1) {
+        set_error("cluster_size=%d without the cluster reduction", C);
+        plan->reject_reason = kRejectCluster;
+        return RT_ERR_INFEASIBLE;
+    }
+    const int64_t row_bytes = s->hidden * eb;
+    if (row_bytes % vb != 0) {
+        set_error("row of %lld bytes is not a multiple of vec_bytes=%d", (long long)row_bytes, vb);
+        plan->reject_reason = kRejectAlign;
+        return RT_ERR_ALIGN;
+    }
+    if (s->min_ptr_align < vb) {
+        set_error("a base pointer is only %d-byte aligned, vec_bytes=%d", s->min_ptr_align, vb);
+        plan->reject_reason = kRejectAlign;
+        return RT_ERR_ALIGN;
+    }
+    if (p->stage == RT_STAGE_SMEM_TMA && (row_bytes % 16 != 0 || s->min_ptr_align < 16)) {
+        set_error("TMA bulk copies need 16-byte aligned rows and pointers (row %lld bytes, pointers %d)",
+                  (long long)row_bytes, s->min_ptr_align);
+        plan->reject_reason = kRejectAlign;
+        return RT_ERR_ALIGN;
+    }
+
+    plan->elem_bytes = eb;
+    plan->nvec = (int)(row_bytes / vb);
+    int slice = (plan->nvec + C - 1) / C;
+    const int gran = vb < 16 ? 16 / vb : 1;  // slices start on 16-byte boundaries
+    slice = (slice + gran - 1) / gran * gran;
+    plan->slice_nvec = slice;
+    plan->vec_per_thread = (slice + tpr - 1) / tpr;
+    plan->cluster = C;
+    plan->block_x = tpr;
+    plan->block_y = rpc;
+    if ((int64_t)(C - 1) * slice >= plan->nvec && C > 1) {
+        set_error("a cluster of %d leaves a CTA without any part of the %d-vector row", C, plan->nvec);
+        plan->reject_reason = kRejectCluster;
+        return RT_ERR_INFEASIBLE;
+    }
+
+    int cap = 0, unroll = p->unroll;
+    if (p->stage == RT_STAGE_REG) {
+        cap = next_pow2(plan->vec_per_thread);
+        if (unroll > cap) unroll = cap;
+    }
+    plan->cap = cap;
+    plan->unroll_eff = unroll;
+    plan->kernel_index = find_kernel(s->dtype, vb, p->stage, p->reduce, unroll, cap);
+    if (plan->kernel_index < 0) {
+        if (p->stage == RT_STAGE_REG)
+            set_error("a row slice of %d vectors over %d threads needs %d vectors per thread: no register-stage "
+                      "instance that large (register budget)", slice, tpr, cap);
+        else
+            set_error("no compiled instance for dtype=%d vec=%d stage=%d reduce=%d unroll=%d", s->dtype, vb, p->stage,
+                      p->reduce, unroll);
+        plan->reject_reason = p->stage == RT_STAGE_REG ? kRejectRegisters : kRejectArgs;
+        return RT_ERR_INFEASIBLE;
+    }
+    const KernelEntry& k = registry()[plan->kernel_index];
+
+    if (p->stage == RT_STAGE_SMEM_LDG)
+        plan->dyn_smem = (size_t)rpc * slice * (vb / eb) * 4;
+    else if (p->stage == RT_STAGE_SMEM_TMA)
+        plan->dyn_smem = (size_t)rpc * 2 * slice * vb;
+
+    int regs, static_smem, local_bytes = 0, max_threads = L->max_threads_per_block;
+    if (L->have_device) {
+        KernelInfo ki;
+        int st = kernel_info(plan->kernel_index, &ki);
+        if (st != RT_OK) return st;
+        regs = ki.regs_per_thread;
+        static_smem = ki.static_smem;
+        local_bytes = ki.local_bytes;
+        max_threads = ki.max_threads;
+    } else {
+        regs = model_regs(k, eb);
+        static_smem = model_static_smem(k);
+    }
+    plan->static_smem_estimate = (size_t)static_smem;
+    if (regs > L->max_regs_per_thread || local_bytes > 0) {
+        set_error("instance needs %d registers per thread and spills %d bytes", regs, local_bytes);
+        plan->reject_reason = kRejectRegisters;
+        return RT_ERR_INFEASIBLE;
+    }
+    const int threads = tpr * rpc;
+    // registers are allocated per warp in units of 8 per thread
+    const int regs_alloc = (regs + 7) / 8 * 8;
+    if ((int64_t)regs_alloc * threads > L->regs_per_block || threads > max_threads) {
+        set_error("%d threads x %d registers exceed the %d registers of a CTA", threads, regs_alloc, L->regs_per_block);
+        plan->reject_reason = kRejectRegisters;
+        return RT_ERR_INFEASIBLE;
+    }
+    if ((int64_t)plan->dyn_smem + static_smem > L->smem_per_block_optin) {
+        set_error("%zu + %d bytes of shared memory exceed the %lld a CTA may opt in to", plan->dyn_smem, static_smem,
+                  (long long)L->smem_per_block_optin);
+        plan->reject_reason = kRejectSmem;
+        return RT_ERR_INFEASIBLE;
+    }
+    const int64_t row_blocks = (s->n_tokens + rpc - 1) / rpc;
+    if (row_blocks * C > 0x7fffffffLL) {
+        set_error("grid of %lld CTAs is too large", (long long)(row_blocks * C));
+        plan->reject_reason = kRejectGrid;
+        return RT_ERR_INFEASIBLE;
+    }
+    plan->grid_x = (unsigned)(row_blocks * C);
+    return RT_OK;
+}
+
+int plan_occupancy(const Plan& plan, const rt_limits* L, int* regs_per_thread)
+{
+    const KernelEntry& k = registry()[plan.kernel_index];
+    const int threads = plan.block_x * plan.block_y;
+    if (L->have_device) {
+        KernelInfo ki;
+        if (kernel_info(plan.kernel_index, &ki) != RT_OK) return 0;
+        if (regs_per_thread) *regs_per_thread = ki.regs_per_thread;
+        if (ensure_dynamic_smem(plan.kernel_index, plan.dyn_smem) != RT_OK) {
+            (void)cudaGetLastError();
+            return 0;
+        }
+        int blocks = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks, k.fn, threads, plan.dyn_smem) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return 0;
+        }
+        if (plan.cluster > 1 && blocks > 0) {
+            cudaLaunchConfig_t cfg;
+            memset(&cfg, 0, sizeof(cfg));
+            cfg.gridDim = dim3((unsigned)plan.cluster, 1, 1);
+            cfg.blockDim = dim3(plan.block_x, plan.block_y, 1);
+            cfg.dynamicSmemBytes = plan.dyn_smem;
+            cudaLaunchAttribute attr;
+            attr.id = cudaLaunchAttributeClusterDimension;
+            attr.val.clusterDim.x = plan.cluster;
+            attr.val.clusterDim.y = 1;
+            attr.val.clusterDim.z = 1;
+            cfg.attrs = &attr;
+            cfg.numAttrs = 1;
+            int clusters = 0;
+            if (cudaOccupancyMaxActiveClusters(&clusters, k.fn, &cfg) != cudaSuccess || clusters < 1) {
+                (void)cudaGetLastError();
+                return 0;
+            }
+        }
+        return blocks;
+    }
+    const int regs = model_regs(k, plan.elem_bytes);
+    if (regs_per_thread) *regs_per_thread = regs;
+    const int regs_alloc = (regs + 7) / 8 * 8;
+    int64_t blocks = L->max_blocks_per_sm;
+    blocks = std::min<int64_t>(blocks, L->max_threads_per_sm / threads);
+    blocks = std::min<int64_t>(blocks, L->regs_per_sm / ((int64_t)regs_alloc * threads));
+    const int64_t smem = (int64_t)plan.dyn_smem + (int64_t)plan.static_smem_estimate + L->smem_reserved_per_block;
+    blocks = std::min<int64_t>(blocks, L->smem_per_sm / smem);
+    return (int)blocks;
+}
+
+int launch_plan(const Plan& plan, const void* x, const void* r, const void* w, void* y, void* r_out,
+                int64_t n_tokens, int64_t hidden, float eps, cudaStream_t stream)
+{
+    if (n_tokens == 0) return RT_OK;
+    const KernelEntry& k = registry()[plan.kernel_index];
+    int st = ensure_dynamic_smem(plan.kernel_index, plan.dyn_smem);
+    if (st != RT_OK) return st;
+    KernelArgs a;
+    a.x = x; a.r = r; a.w = w; a.y = y; a.r_out = r_out;
+    a.n_tokens = n_tokens;
+    a.hidden = (int)hidden;
+    a.nvec = plan.nvec;
+    a.slice_nvec = plan.slice_nvec;
+    a.eps = eps;
+    a.status = device_status_word();
+    if (!a.status) return RT_ERR_CUDA;
+
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(plan.grid_x, 1, 1);
+    cfg.blockDim = dim3(plan.block_x, plan.block_y, 1);
+    cfg.dynamicSmemBytes = plan.dyn_smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    if (plan.cluster > 1) {
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = plan.cluster;
+        attr.val.clusterDim.y = 1;
+        attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+    }
+    void* params[] = {&a};
+    cudaError_t e = cudaLaunchKernelExC(&cfg, k.fn, params);
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        set_error("kernel launch failed: %s", cudaGetErrorString(e));
+        return RT_ERR_CUDA;
+    }
+    count_launch();
+    return RT_OK;
+}
+
+}  // namespace rt
+
+// ---- C ABI -------------------------------------------------------------------------------------
+
+extern "C" {
+
+int rmsnorm_template_launch(const rt_params* p, const void* x, const void* r, const void* w, void* y, void* r_out,
+                            int64_t n_tokens, int64_t hidden, float eps, int dtype, void* stream)
+{
+    if (!p) {
+        rt::set_error("params is NULL");
+        return RT_ERR_NULL;
+    }
+    if (n_tokens > 0 && (!x || !r || !w || !y || !r_out)) {
+        rt::set_error("a tensor pointer is NULL");
+        return RT_ERR_NULL;
+    }
+    rt_limits L;
+    int st = rt::current_limits(&L);
+    if (st != RT_OK) return st;
+    rt_shape s;
+    s.n_tokens = n_tokens;
+    s.hidden = hidden;
+    s.dtype = dtype;
+    s.min_ptr_align = n_tokens > 0 ? rt::min_pointer_alignment(x, r, w, y, r_out) : 256;
+    rt::Plan plan;
+    st = rt::make_plan(&s, p, &L, &plan);
+    if (st != RT_OK) return st;
+    return rt::launch_plan(plan, x, r, w, y, r_out, n_tokens, hidden, eps, (cudaStream_t)stream);
+}
+
+int rt_query_limits(rt_limits* out)
+{
+    if (!out) {
+        rt::set_error("limits is NULL");
+        return RT_ERR_NULL;
+    }
+    return rt::current_limits(out);
+}
+
+void rt_limits_sm100_nominal(rt_limits* out)
+{
+    if (!out) return;
+    memset(out, 0, sizeof(*out));
+    out->sm_count = 148;
+    out->warp_size = 32;
+    out->max_threads_per_block = 1024;
+    out->max_threads_per_sm = 2048;
+    out->max_blocks_per_sm = 32;
+    out->regs_per_block = 65536;
+    out->regs_per_sm = 65536;
+    out->max_regs_per_thread = 255;
+    out->max_cluster_size = 8;
+    out->have_device = 0;
+    out->smem_per_block_optin = 227 * 1024;
+    out->smem_per_sm = 228 * 1024;
+    out->smem_reserved_per_block = 1024;
+    out->l2_bytes = 126LL * 1024 * 1024;
+}
+
+int tuner_check_params(const rt_shape* s, const rt_limits* limits, const rt_params* p)
+{
+    rt_limits L;
+    if (!limits) {
+        int st = rt::current_limits(&L);
+        if (st != RT_OK) return st;
+        limits = &L;
+    }
+    rt::Plan plan;
+    return rt::make_plan(s, p, limits, &plan);
+}
+
+const char* rt_status_string(int status)
+{
+    switch (status) {
+        case RT_OK: return "ok";
+        case RT_ERR_NULL: return "a required pointer is NULL";
+        case RT_ERR_DTYPE: return "unknown dtype";
+        case RT_ERR_SHAPE: return "bad shape";
+        case RT_ERR_ALIGN: return "pointer or row length not aligned to the vector width";
+        case RT_ERR_INFEASIBLE: return "configuration outside the feasible region";
+        case RT_ERR_CUDA: return "CUDA runtime error";
+        case RT_ERR_MISMATCH: return "output differs from the reference beyond tolerance";
+        case RT_ERR_BUDGET: return "search budget allows no evaluation";
+        case RT_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+        case RT_ERR_CAPACITY: return "caller-provided buffer too small";
+        case RT_ERR_NO_DEVICE: return "no CUDA device";
+        default: return "unknown status";
+    }
+}
+
+const char* rt_last_error(void) { return rt::last_error(); }
+
+int rt_device_status(void)
+{
+    int* p = rt::device_status_word();
+    if (!p) return RT_ERR_CUDA;
+    int v = 0;
+    RT_CUDA_OK(cudaDeviceSynchronize());
+    RT_CUDA_OK(cudaMemcpy(&v, p, sizeof(int), cudaMemcpyDeviceToHost));
+    if (v != 0) {
+        RT_CUDA_OK(cudaMemset(p, 0, sizeof(int)));
+        rt::set_error("device status word = %d", v);
+    }
+    return v;
+}
+
+int32_t rt_num_kernel_instances(void) { return (int32_t)rt::registry().size(); }
+
+int rt_kernel_instance(int32_t i, int32_t* dtype, int32_t* vec_bytes, int32_t* stage, int32_t* reduce, int32_t* unroll,
+                       int32_t* reg_vectors)
+{
+    if (i < 0 || i >= (int32_t)rt::registry().size()) {
+        rt::set_error("instance index %d out of range", i);
+        return RT_ERR_CAPACITY;
+    }
+    const rt::KernelEntry& k = rt::registry()[i];
+    if (dtype) *dtype = k.dtype;
+    if (vec_bytes) *vec_bytes = k.vec_bytes;
+    if (stage) *stage = k.stage;
+    if (reduce) *reduce = k.reduce;
+    if (unroll) *unroll = k.unroll;
+    if (reg_vectors) *reg_vectors = k.cap;
+    return RT_OK;
+}
+
+int64_t rt_launch_count(void) { return rt::g_launches.load(); }
+
+}  // extern "C"

@@ -1,0 +1,722 @@
+// Search(S~, x, Theta_feasible): the correctness gate d(.,.) on the device, the timing protocol, and the
+// guided search (seeds -> coarse grid -> best-first hill-climb -> Top-K re-test), after Algorithm 1
+// (Level 2) and the "Tuning agent" / "Testing agent" roles of the paper.
+#include <math.h>
+#include <string.h>
+
+#include <mutex>
+#include <unordered_map>
+
+#include "tuner_internal.h"
+
+namespace rt {
+
+// ---- d(.,.): element-wise comparison on the device ---------------------------------------------------
+
+struct CompareAcc {
+    unsigned long long n_bad;
+    unsigned int max_bits;  // ULP16: max distance; REL32: float bits of the max relative error; BITS: 0/1
+    unsigned int pad;
+};
+
+__device__ __forceinline__ unsigned int ulp_distance16(unsigned int g, unsigned int q, unsigned int nan_above)
+{
+    const unsigned int gm = g & 0x7FFFu, qm = q & 0x7FFFu;
+    const bool gn = gm > nan_above, qn = qm > nan_above;
+    if (gn || qn) return (gn && qn) ? 0u : 65535u;
+    const int gi = (g & 0x8000u) ? -(int)gm : (int)gm;
+    const int qi = (q & 0x8000u) ? -(int)qm : (int)qm;
+    const int d = gi - qi;
+    return (unsigned int)(d < 0 ? -d : d);
+}
+
+template <int MODE>
+__device__ __forceinline__ void compare_word(unsigned int g, unsigned int q, int dtype, double tol,
+                                             unsigned long long& bad, unsigned int& worst)
+{
+    if constexpr (MODE == RT_CMP_BITS) {
+        if (dtype == RT_FP32) {
+            if (g != q) { ++bad; worst = 1u; }
+        } else {
+            if ((g & 0xFFFFu) != (q & 0xFFFFu)) { ++bad; worst = 1u; }
+            if ((g >> 16) != (q >> 16)) { ++bad; worst = 1u; }
+        }
+    } else if constexpr (MODE == RT_CMP_ULP16) {
+        const unsigned int nan_above = dtype == RT_BF16 ? 0x7F80u : 0x7C00u;
+        const unsigned int d0 = ulp_distance16(g & 0xFFFFu, q & 0xFFFFu, nan_above);
+        const unsigned int d1 = ulp_distance16(g >> 16, q >> 16, nan_above);
+        if ((double)d0 > tol) ++bad;
+        if ((double)d1 > tol) ++bad;
+        worst = max(worst, max(d0, d1));
+    } else {
+        const float gf = __uint_as_float(g), qf = __uint_as_float(q);
+        const bool gn = gf != gf, qn = qf != qf;
+        if (gn || qn) {
+            if (!(gn && qn)) { ++bad; worst = 0x7F800000u; }
+        } else if (gf != qf) {
+            const double err = fabs((double)gf - (double)qf);
+            const double mag = fabs((double)qf);
+            if (!(err <= tol * mag + 1e-30)) ++bad;
+            const float rel = (float)(err / fmax(mag, 1e-30));
+            worst = max(worst, __float_as_uint(rel));
+        }
+    }
+}
+
+// got/ref viewed as 32-bit words (n_words of them); a trailing 16-bit element, if any, is handled
+// by the last thread through the `tail` words (upper half zeroed on both sides).
+template <int MODE>
+__global__ void compare_kernel(const unsigned int* __restrict__ got, const unsigned int* __restrict__ ref,
+                               long long n_words, int has_tail, unsigned int tail_got, unsigned int tail_ref,
+                               int dtype, double tol, CompareAcc* acc)
+{
+    unsigned long long bad = 0;
+    unsigned int worst = 0;
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n_words; i += stride)
+        compare_word<MODE>(got[i], ref[i], dtype, tol, bad, worst);
+    if (has_tail && blockIdx.x == 0 && threadIdx.x == 0) {
+        unsigned long long b2 = 0;
+        compare_word<MODE>(tail_got, tail_ref, dtype, tol, b2, worst);
+        bad += b2 ? 1 : 0;  // the padded upper halves are equal and add nothing
+    }
+    for (int off = 16; off >= 1; off >>= 1) {
+        bad += __shfl_xor_sync(0xffffffffu, bad, off);
+        worst = max(worst, __shfl_xor_sync(0xffffffffu, worst, off));
+    }
+    if ((threadIdx.x & 31) == 0) {
+        if (bad) atomicAdd(&acc->n_bad, bad);
+        if (worst) atomicMax(&acc->max_bits, worst);
+    }
+}
+
+namespace {
+
+std::mutex g_scratch_mutex;
+struct Scratch {
+    CompareAcc* dev = nullptr;
+    CompareAcc* host = nullptr;  // page-locked
+};
+Scratch g_scratch[64];
+
+int get_scratch(Scratch** out)
+{
+    int dev = 0;
+    RT_CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) {
+        set_error("device index %d out of range", dev);
+        return RT_ERR_NO_DEVICE;
+    }
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    Scratch& s = g_scratch[dev];
+    if (!s.dev) {
+        RT_CUDA_OK(cudaMalloc((void**)&s.dev, 2 * sizeof(CompareAcc)));
+        RT_CUDA_OK(cudaMallocHost((void**)&s.host, 2 * sizeof(CompareAcc)));
+    }
+    *out = &s;
+    return RT_OK;
+}
+
+// Enqueue one comparison into accumulator slot `slot`; results are read after a stream sync.
+int enqueue_compare(const void* got, const void* ref, int64_t n, int dtype, int mode, double tol, CompareAcc* acc,
+                    cudaStream_t stream)
+{
+    const int eb = elem_bytes_of(dtype);
+    if (((uintptr_t)got | (uintptr_t)ref) & 3u) {
+        set_error("tuner_compare needs 4-byte aligned buffers");
+        return RT_ERR_ALIGN;
+    }
+    const long long n_words = (long long)(n * eb / 4);
+    const int has_tail = (n * eb) % 4 != 0;
+    unsigned int tail_got = 0, tail_ref = 0;
+    if (has_tail) {  // one trailing 16-bit element: fetch it to the host side of the launch
+        unsigned short tg = 0, tr = 0;
+        RT_CUDA_OK(cudaMemcpyAsync(&tg, (const char*)got + n_words * 4, 2, cudaMemcpyDeviceToHost, stream));
+        RT_CUDA_OK(cudaMemcpyAsync(&tr, (const char*)ref + n_words * 4, 2, cudaMemcpyDeviceToHost, stream));
+        RT_CUDA_OK(cudaStreamSynchronize(stream));
+        tail_got = tg;
+        tail_ref = tr;
+    }
+    const int threads = 256;
+    long long want = (n_words + threads * 8 - 1) / (threads * 8);
+    const int blocks = (int)std::max<long long>(1, std::min<long long>(want, 148 * 16));
+    const unsigned int* g = (const unsigned int*)got;
+    const unsigned int* q = (const unsigned int*)ref;
+    if (mode == RT_CMP_BITS)
+        compare_kernel<RT_CMP_BITS><<<blocks, threads, 0, stream>>>(g, q, n_words, has_tail, tail_got, tail_ref, dtype, tol, acc);
+    else if (mode == RT_CMP_ULP16)
+        compare_kernel<RT_CMP_ULP16><<<blocks, threads, 0, stream>>>(g, q, n_words, has_tail, tail_got, tail_ref, dtype, tol, acc);
+    else
+        compare_kernel<RT_CMP_REL32><<<blocks, threads, 0, stream>>>(g, q, n_words, has_tail, tail_got, tail_ref, dtype, tol, acc);
+    RT_CUDA_OK(cudaGetLastError());
+    count_launch();
+    return RT_OK;
+}
+
+int check_compare_args(const void* got, const void* ref, int64_t n, int dtype, int mode)
+{
+    if (!got || !ref) {
+        set_error("tuner_compare: NULL buffer");
+        return RT_ERR_NULL;
+    }
+    if (dtype < 0 || dtype > 2) {
+        set_error("dtype %d unknown", dtype);
+        return RT_ERR_DTYPE;
+    }
+    if (n < 0) {
+        set_error("n = %lld is negative", (long long)n);
+        return RT_ERR_SHAPE;
+    }
+    if (mode < RT_CMP_BITS || mode > RT_CMP_REL32 || (mode == RT_CMP_ULP16 && dtype == RT_FP32) ||
+        (mode == RT_CMP_REL32 && dtype != RT_FP32)) {
+        set_error("compare mode %d does not apply to dtype %d", mode, dtype);
+        return RT_ERR_DTYPE;
+    }
+    return RT_OK;
+}
+
+double acc_max_err(const CompareAcc& a, int mode)
+{
+    if (mode == RT_CMP_REL32) {
+        float f;
+        memcpy(&f, &a.max_bits, sizeof(f));
+        return (double)f;
+    }
+    return (double)a.max_bits;
+}
+
+}  // namespace
+
+// ---- evaluation of one theta: gate, then the timing protocol ----------------------------------------
+
+struct Evaluator {
+    virtual ~Evaluator() {}
+    // Fills rec->status, the gate statistics and the times.  Returns RT_OK unless the evaluation
+    // itself could not be carried out (a CUDA failure that is not specific to the candidate).
+    virtual int evaluate(const rt_params& p, rt_eval_record* rec) = 0;
+};
+
+static float median_of(std::vector<float> v)
+{
+    std::sort(v.begin(), v.end());
+    const size_t n = v.size();
+    return n % 2 ? v[n / 2] : 0.5f * (v[n / 2 - 1] + v[n / 2]);
+}
+
+struct DeviceEvaluator : Evaluator {
+    rt_shape shape;
+    rt_budget budget;
+    rt_workspace ws;
+    rt_limits limits;
+
+    int evaluate(const rt_params& p, rt_eval_record* rec) override
+    {
+        memset(rec, 0, sizeof(*rec));
+        rec->params = p;
+        cudaStream_t stream = (cudaStream_t)ws.stream;
+        const int eb = elem_bytes_of(shape.dtype);
+        Plan plan;
+        int st = make_plan(&shape, &p, &limits, &plan);
+        if (st != RT_OK) {
+            rec->status = st;
+            return RT_OK;
+        }
+        int regs = 0;
+        rec->occupancy_blocks_per_sm = plan_occupancy(plan, &limits, &regs);
+        rec->regs_per_thread = regs;
+
+        // Gate.  Outputs are poisoned first (all-ones is NaN in all three types), so that values left
+        // by an earlier candidate cannot pass for this one's.
+        const int64_t n_ref = ws.n_ref_tokens;
+        const size_t ref_bytes = (size_t)n_ref * shape.hidden * eb;
+        const size_t set_bytes = (size_t)shape.n_tokens * shape.hidden * eb;
+        Scratch* sc;
+        st = get_scratch(&sc);
+        if (st != RT_OK) return st;
+        RT_CUDA_OK(cudaMemsetAsync(ws.y, 0xFF, set_bytes, stream));
+        RT_CUDA_OK(cudaMemsetAsync(ws.r_out, 0xFF, set_bytes, stream));
+        RT_CUDA_OK(cudaMemsetAsync(sc->dev, 0, 2 * sizeof(CompareAcc), stream));
+        st = launch_plan(plan, ws.x, ws.r, ws.w, ws.y, ws.r_out, shape.n_tokens, shape.hidden, ws.eps, stream);
+        if (st != RT_OK) {
+            rec->status = st;
+            return RT_OK;
+        }
+        const int y_mode = shape.dtype == RT_FP32 ? RT_CMP_REL32 : RT_CMP_ULP16;
+        const double y_tol = shape.dtype == RT_FP32 ? 1e-5 : 2.0;
+        st = enqueue_compare(ws.r_out, ws.r_ref, n_ref * shape.hidden, shape.dtype, RT_CMP_BITS, 0.0, sc->dev, stream);
+        if (st != RT_OK) return st;
+        st = enqueue_compare(ws.y, ws.y_ref, n_ref * shape.hidden, shape.dtype, y_mode, y_tol, sc->dev + 1, stream);
+        if (st != RT_OK) return st;
+        (void)ref_bytes;
+        RT_CUDA_OK(cudaMemcpyAsync(sc->host, sc->dev, 2 * sizeof(CompareAcc), cudaMemcpyDeviceToHost, stream));
+        cudaError_t e = cudaStreamSynchronize(stream);
+        if (e != cudaSuccess) {
+            set_error("candidate faulted: %s", cudaGetErrorString(e));
+            return RT_ERR_CUDA;  // a sticky error: nothing further can run in this context
+        }
+        rec->r_bad = (int64_t)sc->host[0].n_bad;
+        rec->y_bad = (int64_t)sc->host[1].n_bad;
+        if (shape.dtype == RT_FP32)
+            rec->y_max_rel = (float)acc_max_err(sc->host[1], RT_CMP_REL32);
+        else
+            rec->y_max_ulp = (int32_t)sc->host[1].max_bits;
+        if (p.stage == RT_STAGE_SMEM_TMA) {
+            int flag = 0;
+            RT_CUDA_OK(cudaMemcpy(&flag, device_status_word(), sizeof(int), cudaMemcpyDeviceToHost));
+            if (flag) {
+                RT_CUDA_OK(cudaMemset(device_status_word(), 0, sizeof(int)));
+                rec->status = RT_ERR_DEVICE_TIMEOUT;
+                return RT_OK;
+            }
+        }
+        if (rec->r_bad || rec->y_bad) {
+            rec->status = RT_ERR_MISMATCH;
+            return RT_OK;
+        }
+
+        // Timing: `warmup` launches, then `repeats` blocks of `iters` launches between two events.
+        const int sets = ws.ring_sets > 0 ? ws.ring_sets : 1;
+        auto launch_set = [&](int k) {
+            const size_t off = (size_t)(k % sets) * (size_t)ws.ring_stride_bytes;
+            return launch_plan(plan, (const char*)ws.x + off, (const char*)ws.r + off, ws.w, (char*)ws.y + off,
+                               (char*)ws.r_out + off, shape.n_tokens, shape.hidden, ws.eps, stream);
+        };
+        for (int i = 0; i < budget.warmup; ++i) {
+            st = launch_set(i);
+            if (st != RT_OK) {
+                rec->status = st;
+                return RT_OK;
+            }
+        }
+        const int iters = budget.iters > 0 ? budget.iters : 1;
+        const int repeats = budget.repeats > 0 ? budget.repeats : 1;
+        cudaGraphExec_t graph_exec = nullptr;
+        if (budget.use_graph) {
+            if (!stream) {
+                set_error("use_graph needs a non-default stream");
+                return RT_ERR_CUDA;
+            }
+            cudaGraph_t graph = nullptr;
+            RT_CUDA_OK(cudaStreamBeginCapture(stream, cudaStreamCaptureModeThreadLocal));
+            int cap_st = RT_OK;
+            for (int i = 0; i < iters && cap_st == RT_OK; ++i) cap_st = launch_set(i);
+            cudaError_t ce = cudaStreamEndCapture(stream, &graph);
+            if (cap_st != RT_OK || ce != cudaSuccess) {
+                if (graph) cudaGraphDestroy(graph);
+                (void)cudaGetLastError();
+                rec->status = cap_st != RT_OK ? cap_st : RT_ERR_CUDA;
+                return RT_OK;
+            }
+            ce = cudaGraphInstantiate(&graph_exec, graph, 0);
+            cudaGraphDestroy(graph);
+            if (ce != cudaSuccess) {
+                set_error("cudaGraphInstantiate failed: %s", cudaGetErrorString(ce));
+                return RT_ERR_CUDA;
+            }
+            RT_CUDA_OK(cudaGraphLaunch(graph_exec, stream));  // one untimed replay
+        }
+        cudaEvent_t e0, e1;
+        RT_CUDA_OK(cudaEventCreate(&e0));
+        RT_CUDA_OK(cudaEventCreate(&e1));
+        std::vector<float> block_us;
+        int fail = RT_OK;
+        for (int rep = 0; rep < repeats && fail == RT_OK; ++rep) {
+            cudaEventRecord(e0, stream);
+            if (graph_exec) {
+                if (cudaGraphLaunch(graph_exec, stream) != cudaSuccess) fail = RT_ERR_CUDA;
+                count_launch(iters);
+            } else {
+                for (int i = 0; i < iters && fail == RT_OK; ++i) fail = launch_set(i);
+            }
+            cudaEventRecord(e1, stream);
+            if (cudaEventSynchronize(e1) != cudaSuccess) fail = RT_ERR_CUDA;
+            float ms = 0.f;
+            if (fail == RT_OK && cudaEventElapsedTime(&ms, e0, e1) == cudaSuccess) block_us.push_back(ms * 1000.f / iters);
+        }
+        cudaEventDestroy(e0);
+        cudaEventDestroy(e1);
+        if (graph_exec) cudaGraphExecDestroy(graph_exec);
+        if (fail != RT_OK || block_us.empty()) {
+            cudaError_t le = cudaGetLastError();
+            set_error("timing failed: %s", cudaGetErrorString(le));
+            return RT_ERR_CUDA;
+        }
+        float sum = 0.f, mn = block_us[0];
+        for (float v : block_us) {
+            sum += v;
+            mn = std::min(mn, v);
+        }
+        rec->us = median_of(block_us);
+        rec->us_min_block = mn;
+        rec->us_mean = sum / (float)block_us.size();
+        rec->status = RT_OK;
+        return RT_OK;
+    }
+};
+
+struct CallbackEvaluator : Evaluator {
+    rt_evaluate_fn fn;
+    void* user;
+    int evaluate(const rt_params& p, rt_eval_record* rec) override
+    {
+        memset(rec, 0, sizeof(*rec));
+        rec->params = p;
+        const double t = fn(&p, user);
+        if (!(t >= 0.0) || isinf(t)) {
+            rec->status = RT_ERR_MISMATCH;
+        } else {
+            rec->us = rec->us_min_block = rec->us_mean = (float)t;
+            rec->status = RT_OK;
+        }
+        return RT_OK;
+    }
+};
+
+// ---- the search --------------------------------------------------------------------------------------
+
+namespace {
+
+int level_of(const int* levels, int n, int v)
+{
+    for (int i = 0; i < n; ++i)
+        if (levels[i] == v) return i;
+    return -1;
+}
+const int kTpr[] = {32, 64, 128, 256, 512, 1024};
+const int kRpc[] = {1, 2, 4, 8};
+const int kUnr[] = {1, 2, 4};
+const int kVec[] = {2, 4, 8, 16};
+const int kClu[] = {1, 2, 4, 8};
+
+struct SearchState {
+    std::vector<rt_params> cand;
+    std::unordered_map<uint64_t, int> index;
+    std::vector<float> time_us;   // < 0: not evaluated; +inf: failed its gate
+    std::vector<char> expanded;
+    int used = 0, failed = 0;
+    int max_evals = 0;
+    rt_eval_record* log = nullptr;
+    int log_cap = 0, n_log = 0;
+    Evaluator* ev = nullptr;
+
+    int add(const rt_params& p)
+    {
+        auto it = index.find(pack_params(p));
+        if (it != index.end()) return it->second;
+        cand.push_back(p);
+        time_us.push_back(-1.f);
+        expanded.push_back(0);
+        index[pack_params(p)] = (int)cand.size() - 1;
+        return (int)cand.size() - 1;
+    }
+    bool budget_left(int reserve) const { return used < max_evals - reserve; }
+
+    // One evaluation (counts against the budget).  Returns a hard error or RT_OK.
+    int run(int idx, int phase, float* out_us)
+    {
+        rt_eval_record rec;
+        int st = ev->evaluate(cand[idx], &rec);
+        rec.phase = phase;
+        rec.eval_index = used;
+        ++used;
+        if (log && n_log < log_cap) log[n_log++] = rec;
+        if (st != RT_OK) return st;
+        if (rec.status != RT_OK) {
+            ++failed;
+            *out_us = INFINITY;
+        } else {
+            *out_us = rec.us;
+        }
+        return RT_OK;
+    }
+
+    // One-step neighbours: +-1 level on one ordered axis, or another stage, or another reduction.
+    std::vector<int> neighbours(int idx) const
+    {
+        std::vector<int> out;
+        const rt_params& p = cand[idx];
+        auto probe = [&](rt_params q) {
+            auto it = index.find(pack_params(q));
+            if (it != index.end() && it->second != idx) out.push_back(it->second);
+        };
+        auto step = [&](const int* levels, int n, int rt_params::*field) {
+            const int l = level_of(levels, n, p.*field);
+            for (int d = -1; d <= 1; d += 2) {
+                if (l + d < 0 || l + d >= n || l < 0) continue;
+                rt_params q = p;
+                q.*field = levels[l + d];
+                probe(q);
+            }
+        };
+        step(kTpr, 6, &rt_params::threads_per_row);
+        step(kRpc, 4, &rt_params::rows_per_cta);
+        step(kUnr, 3, &rt_params::unroll);
+        step(kVec, 4, &rt_params::vec_bytes);
+        for (int stage = 0; stage < 3; ++stage) {
+            rt_params q = p;
+            q.stage = stage;
+            probe(q);
+        }
+        for (int reduce = 0; reduce < 3; ++reduce)
+            for (int c : kClu) {
+                if ((reduce == RT_REDUCE_CLUSTER) != (c > 1)) continue;
+                rt_params q = p;
+                q.reduce = reduce;
+                q.cluster_size = c;
+                probe(q);
+            }
+        return out;
+    }
+};
+
+// The coarse grid: every other level of the ordered axes (threads per row 64/256/1024, rows per CTA
+// 1/4, unroll 1/4), the widest vector, every stage and reduction mode.
+bool on_coarse_grid(const rt_params& p, int widest_vec)
+{
+    const int lt = level_of(kTpr, 6, p.threads_per_row), lr = level_of(kRpc, 4, p.rows_per_cta),
+              lu = level_of(kUnr, 3, p.unroll);
+    return (lt % 2 == 1) && (lr % 2 == 0) && (lu % 2 == 0) && p.vec_bytes == widest_vec;
+}
+
+std::vector<int> thin(const std::vector<int>& v, int keep)
+{
+    if (keep <= 0) return {};
+    if ((int)v.size() <= keep) return v;
+    std::vector<int> out;
+    for (int i = 0; i < keep; ++i) out.push_back(v[(size_t)i * v.size() / keep]);
+    return out;
+}
+
+int run_search(const rt_shape& shape, const rt_limits& limits, const rt_budget& b, Evaluator& ev, rt_result* out,
+               rt_eval_record* log, int32_t log_cap)
+{
+    memset(out, 0, sizeof(*out));
+    if (b.max_evals < 1) {
+        set_error("max_evals = %d allows no evaluation", b.max_evals);
+        return RT_ERR_BUDGET;
+    }
+    std::vector<rt_params> feasible;
+    int st = derive_feasible(shape, limits, b.heuristics, &feasible, nullptr);
+    if (st != RT_OK) return st;
+    if (feasible.empty()) {
+        set_error("the feasible set is empty for this shape");
+        return RT_ERR_INFEASIBLE;
+    }
+    SearchState S;
+    S.ev = &ev;
+    S.max_evals = b.max_evals;
+    S.log = log;
+    S.log_cap = log ? log_cap : 0;
+    for (const rt_params& p : feasible) S.add(p);
+    out->n_candidates = (int32_t)feasible.size();
+
+    const int top_k = std::max(0, std::min<int>(b.top_k, b.max_evals / 4));  // re-tests are part of the budget
+    float t;
+
+    if (b.strategy == RT_SEARCH_EXHAUSTIVE) {
+        for (int i = 0; i < (int)S.cand.size() && S.budget_left(top_k); ++i) {
+            st = S.run(i, RT_PHASE_SWEEP, &t);
+            if (st != RT_OK) return st;
+            S.time_us[i] = t;
+        }
+    } else {
+        // 1. seeds: configurations found on other shapes, if they are feasible here
+        for (int k = 0; k < b.n_seeds && b.seeds && S.budget_left(top_k); ++k) {
+            Plan plan;
+            if (make_plan(&shape, &b.seeds[k], &limits, &plan) != RT_OK) continue;
+            const int idx = S.add(b.seeds[k]);
+            if (S.time_us[idx] >= 0.f) continue;
+            st = S.run(idx, RT_PHASE_SEED, &t);
+            if (st != RT_OK) return st;
+            S.time_us[idx] = t;
+        }
+        // 2. coarse grid, thinned to half of what is left of the budget
+        int widest = 0;
+        for (const rt_params& p : feasible) widest = std::max(widest, p.vec_bytes);
+        std::vector<int> coarse;
+        for (int i = 0; i < (int)feasible.size(); ++i)
+            if (on_coarse_grid(S.cand[i], widest)) coarse.push_back(i);
+        if (coarse.empty())
+            for (int i = 0; i < (int)feasible.size(); ++i) coarse.push_back(i);
+        const int grid_budget = std::max(1, (S.max_evals - top_k - S.used) / 2);
+        for (int idx : thin(coarse, grid_budget)) {
+            if (!S.budget_left(top_k)) break;
+            if (S.time_us[idx] >= 0.f) continue;
+            st = S.run(idx, RT_PHASE_GRID, &t);
+            if (st != RT_OK) return st;
+            S.time_us[idx] = t;
+        }
+        // 3. best-first hill-climb: expand the neighbours of the fastest point not yet expanded, among
+        //    the three fastest found so far; stop when those are all expanded or the budget is spent
+        while (S.budget_left(top_k)) {
+            std::vector<int> order;
+            for (int i = 0; i < (int)S.cand.size(); ++i)
+                if (S.time_us[i] >= 0.f && isfinite(S.time_us[i])) order.push_back(i);
+            std::sort(order.begin(), order.end(), [&](int a, int c) { return S.time_us[a] < S.time_us[c]; });
+            int pick = -1;
+            for (int k = 0; k < (int)order.size() && k < 3; ++k)
+                if (!S.expanded[order[k]]) {
+                    pick = order[k];
+                    break;
+                }
+            if (pick < 0) break;
+            S.expanded[pick] = 1;
+            for (int nb : S.neighbours(pick)) {
+                if (!S.budget_left(top_k)) break;
+                if (S.time_us[nb] >= 0.f) continue;
+                st = S.run(nb, RT_PHASE_CLIMB, &t);
+                if (st != RT_OK) return st;
+                S.time_us[nb] = t;
+            }
+        }
+    }
+
+    // 4. Top-K confirmation re-test: the finalists' scores become the mean of both measurements
+    std::vector<int> order;
+    for (int i = 0; i < (int)S.cand.size(); ++i)
+        if (S.time_us[i] >= 0.f && isfinite(S.time_us[i])) order.push_back(i);
+    std::sort(order.begin(), order.end(), [&](int a, int c) { return S.time_us[a] < S.time_us[c]; });
+    for (int k = 0; k < top_k && k < (int)order.size() && S.used < S.max_evals; ++k) {
+        st = S.run(order[k], RT_PHASE_TOPK, &t);
+        if (st != RT_OK) return st;
+        if (isfinite(t)) S.time_us[order[k]] = 0.5f * (S.time_us[order[k]] + t);
+    }
+    int best = -1;
+    for (int i : order)
+        if (best < 0 || S.time_us[i] < S.time_us[best]) best = i;
+
+    out->evals_used = S.used;
+    out->n_log = S.n_log;
+    out->n_failed_gate = S.failed;
+    if (best < 0) {
+        set_error("no candidate passed the correctness gate (%d evaluated)", S.used);
+        return RT_ERR_MISMATCH;
+    }
+    out->best = S.cand[best];
+    out->best_us = S.time_us[best];
+    return RT_OK;
+}
+
+int check_workspace(const rt_shape* s, const rt_workspace* ws)
+{
+    if (!s || !ws) {
+        set_error("shape or workspace is NULL");
+        return RT_ERR_NULL;
+    }
+    if (!ws->x || !ws->r || !ws->w || !ws->y || !ws->r_out || !ws->y_ref || !ws->r_ref) {
+        set_error("a workspace pointer is NULL");
+        return RT_ERR_NULL;
+    }
+    if (s->n_tokens < 1 || ws->n_ref_tokens < 1 || ws->n_ref_tokens > s->n_tokens) {
+        set_error("n_ref_tokens=%lld must lie in 1..n_tokens=%lld", (long long)ws->n_ref_tokens, (long long)s->n_tokens);
+        return RT_ERR_SHAPE;
+    }
+    if (ws->x == ws->y || ws->r == ws->r_out) {
+        set_error("the tuner's workspace must not alias inputs and outputs (launches repeat)");
+        return RT_ERR_SHAPE;
+    }
+    return RT_OK;
+}
+
+rt_budget normalised(const rt_budget* b)
+{
+    rt_budget n = *b;
+    if (n.warmup < 0) n.warmup = 0;
+    if (n.iters < 1) n.iters = 1;
+    if (n.repeats < 1) n.repeats = 1;
+    return n;
+}
+
+}  // namespace
+}  // namespace rt
+
+// ---- C ABI -------------------------------------------------------------------------------------------
+
+extern "C" {
+
+int tuner_compare(const void* got, const void* ref, int64_t n, int dtype, int mode, double tol, double* max_err,
+                  int64_t* n_bad, void* stream)
+{
+    int st = rt::check_compare_args(got, ref, n, dtype, mode);
+    if (st != RT_OK) return st;
+    if (!max_err || !n_bad) {
+        rt::set_error("tuner_compare: NULL result pointer");
+        return RT_ERR_NULL;
+    }
+    *max_err = 0.0;
+    *n_bad = 0;
+    if (n == 0) return RT_OK;
+    rt::Scratch* sc;
+    st = rt::get_scratch(&sc);
+    if (st != RT_OK) return st;
+    cudaStream_t s = (cudaStream_t)stream;
+    RT_CUDA_OK(cudaMemsetAsync(sc->dev, 0, sizeof(rt::CompareAcc), s));
+    st = rt::enqueue_compare(got, ref, n, dtype, mode, tol, sc->dev, s);
+    if (st != RT_OK) return st;
+    RT_CUDA_OK(cudaMemcpyAsync(sc->host, sc->dev, sizeof(rt::CompareAcc), cudaMemcpyDeviceToHost, s));
+    RT_CUDA_OK(cudaStreamSynchronize(s));
+    *max_err = rt::acc_max_err(sc->host[0], mode);
+    *n_bad = (int64_t)sc->host[0].n_bad;
+    return RT_OK;
+}
+
+int tuner_evaluate(const rt_shape* s, const rt_params* p, const rt_budget* b, const rt_workspace* ws, rt_eval_record* out)
+{
+    if (!p || !b || !out) {
+        rt::set_error("tuner_evaluate: NULL argument");
+        return RT_ERR_NULL;
+    }
+    int st = rt::check_workspace(s, ws);
+    if (st != RT_OK) return st;
+    rt::DeviceEvaluator ev;
+    ev.shape = *s;
+    ev.budget = rt::normalised(b);
+    ev.ws = *ws;
+    st = rt::current_limits(&ev.limits);
+    if (st != RT_OK) return st;
+    return ev.evaluate(*p, out);
+}
+
+int tuner_search(const rt_shape* s, const rt_budget* b, const rt_workspace* ws, rt_result* out, rt_eval_record* log,
+                 int32_t log_cap)
+{
+    if (!b || !out) {
+        rt::set_error("tuner_search: NULL argument");
+        return RT_ERR_NULL;
+    }
+    int st = rt::check_workspace(s, ws);
+    if (st != RT_OK) return st;
+    rt::DeviceEvaluator ev;
+    ev.shape = *s;
+    ev.budget = rt::normalised(b);
+    ev.ws = *ws;
+    st = rt::current_limits(&ev.limits);
+    if (st != RT_OK) return st;
+    return rt::run_search(*s, ev.limits, ev.budget, ev, out, log, log_cap);
+}
+
+int tuner_search_with(const rt_shape* s, const rt_limits* limits, const rt_budget* b, rt_evaluate_fn evaluate, void* user,
+                      rt_result* out, rt_eval_record* log, int32_t log_cap)
+{
+    if (!s || !limits || !b || !evaluate || !out) {
+        rt::set_error("tuner_search_with: NULL argument");
+        return RT_ERR_NULL;
+    }
+    rt::CallbackEvaluator ev;
+    ev.fn = evaluate;
+    ev.user = user;
+    return rt::run_search(*s, *limits, rt::normalised(b), ev, out, log, log_cap);
+}
+
+void rt_shutdown(void)
+{
+    std::lock_guard<std::mutex> lock(rt::g_scratch_mutex);
+    for (rt::Scratch& s : rt::g_scratch) {
+        if (s.dev) cudaFree(s.dev);
+        if (s.host) cudaFreeHost(s.host);
+        s.dev = nullptr;
+        s.host = nullptr;
+    }
+}
+
+}  // extern "C"
