@@ -286,6 +286,30 @@ typedef enum { RT_CMP_BITS = 0, RT_CMP_ULP16 = 1, RT_CMP_REL32 = 2 } rt_compare_
 int tuner_compare(const void* got, const void* ref, int64_t n, int dtype, int mode, double tol,
                   double* max_err, int64_t* n_bad, void* stream);
 
+/*
+ * tuner_compare without any allocation.  (No counterpart in the paper: it exists for callers that
+ * cannot allocate device memory.)
+ *
+ * Some callers must not reach cudaMalloc at all: a serving process that has handed the whole device
+ * to its own memory pool (a raw allocation there fails, or takes memory the pool counts on), and code
+ * on a latency path where the device-wide synchronisation that cudaMalloc and cudaFree imply is not
+ * acceptable.  tuner_compare allocates its accumulator (device and page-locked host memory) on first
+ * use; this entry point calls no cudaMalloc, cudaMallocHost, cudaFree or any other allocating routine,
+ * now or later.  Arguments, modes, results and errors are those of tuner_compare.
+ *
+ * Its accumulator lives in a fixed 256-byte array inside the library's device image: every GPU that
+ * loads the library holds those 256 bytes until the process exits.  The accumulator does not grow with
+ * n; n is limited to 2^40 elements (RT_ERR_CAPACITY beyond that, nothing is launched).
+ *
+ * The first call on each device looks up the array's device address (with that device current); make
+ * that first call before starting any stream capture.  All calls on a device share the one array: it is
+ * cleared at the start of every call, so calls in a row are independent, but two calls whose work
+ * overlaps on the GPU (different streams, different threads) race on it and return garbage - serialise
+ * them.  Synchronises `stream`.
+ */
+int tuner_compare_static(const void* got, const void* ref, int64_t n, int dtype, int mode, double tol,
+                         double* max_err, int64_t* n_bad, void* stream);
+
 /* ---- housekeeping ------------------------------------------------------------------- */
 
 const char* rt_status_string(int status);

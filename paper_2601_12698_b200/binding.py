@@ -116,6 +116,8 @@ _SIGNATURES = {
                                POINTER(rt_eval_record)]),
     "tuner_compare": (c_int, [c_void_p, c_void_p, c_int64, c_int, c_int, c_double, POINTER(c_double),
                               POINTER(c_int64), c_void_p]),
+    "tuner_compare_static": (c_int, [c_void_p, c_void_p, c_int64, c_int, c_int, c_double, POINTER(c_double),
+                                     POINTER(c_int64), c_void_p]),
     "rt_status_string": (c_char_p, [c_int]),
     "rt_last_error": (c_char_p, []),
     "rt_device_status": (c_int, []),
@@ -315,6 +317,17 @@ def tuner_compare(got, ref, mode: int, tol: float = 0.0, stream=None):
     worst, bad = c_double(0.0), c_int64(0)
     _check(lib.tuner_compare(got.data_ptr(), ref.data_ptr(), got.numel(), _dtype_code(got), mode, tol, byref(worst),
                              byref(bad), _stream_ptr(stream)), "tuner_compare")
+    return worst.value, bad.value
+
+
+def tuner_compare_static(got, ref, mode: int, tol: float = 0.0, stream=None):
+    """tuner_compare for callers that must not allocate: same result, accumulator in a fixed device array
+    (shared by all calls on the device, so calls must not overlap on the GPU)."""
+    if got.shape != ref.shape or got.dtype != ref.dtype:
+        raise ValueError("got and ref must match")
+    worst, bad = c_double(0.0), c_int64(0)
+    _check(lib.tuner_compare_static(got.data_ptr(), ref.data_ptr(), got.numel(), _dtype_code(got), mode, tol,
+                                    byref(worst), byref(bad), _stream_ptr(stream)), "tuner_compare_static")
     return worst.value, bad.value
 
 

@@ -90,9 +90,43 @@ __global__ void compare_kernel(const unsigned int* __restrict__ got, const unsig
     }
 }
 
+// Scratch of the allocation-free comparison entry point: one accumulator record, kept in a fixed
+// array that every device loading this library holds until the process exits.  In host code this name
+// is only a handle for cudaGetSymbolAddress, never an address a kernel may be given.
+constexpr int kStaticScratchBytes = 256;
+constexpr int64_t kStaticCompareMaxElems = (int64_t)1 << 40;
+static __device__ __align__(256) unsigned char g_static_compare_scratch[kStaticScratchBytes];
+static_assert(sizeof(CompareAcc) <= kStaticScratchBytes, "accumulator record larger than the static scratch");
+
 namespace {
 
 std::mutex g_scratch_mutex;
+CompareAcc* g_static_scratch_addr[64];  // device address of the static scratch, per device
+
+// Set-up of the static scratch for the current device: its device address, looked up once.
+int static_scratch(CompareAcc** out)
+{
+    int dev = 0;
+    RT_CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) {
+        set_error("device index %d out of range", dev);
+        return RT_ERR_NO_DEVICE;
+    }
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (!g_static_scratch_addr[dev]) {
+        void* p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&p, g_static_compare_scratch);
+        if (e != cudaSuccess || !p) {
+            (void)cudaGetLastError();
+            set_error("cudaGetSymbolAddress(static compare scratch) failed: %s", cudaGetErrorString(e));
+            return RT_ERR_CUDA;
+        }
+        g_static_scratch_addr[dev] = (CompareAcc*)p;
+    }
+    *out = g_static_scratch_addr[dev];
+    return RT_OK;
+}
+
 struct Scratch {
     CompareAcc* dev = nullptr;
     CompareAcc* host = nullptr;  // page-locked
@@ -657,6 +691,39 @@ int tuner_compare(const void* got, const void* ref, int64_t n, int dtype, int mo
     RT_CUDA_OK(cudaStreamSynchronize(s));
     *max_err = rt::acc_max_err(sc->host[0], mode);
     *n_bad = (int64_t)sc->host[0].n_bad;
+    return RT_OK;
+}
+
+int tuner_compare_static(const void* got, const void* ref, int64_t n, int dtype, int mode, double tol, double* max_err,
+                         int64_t* n_bad, void* stream)
+{
+    int st = rt::check_compare_args(got, ref, n, dtype, mode);
+    if (st != RT_OK) return st;
+    if (!max_err || !n_bad) {
+        rt::set_error("tuner_compare_static: NULL result pointer");
+        return RT_ERR_NULL;
+    }
+    if (n > rt::kStaticCompareMaxElems) {
+        rt::set_error("tuner_compare_static: n = %lld exceeds the limit of %lld elements", (long long)n,
+                      (long long)rt::kStaticCompareMaxElems);
+        return RT_ERR_CAPACITY;
+    }
+    *max_err = 0.0;
+    *n_bad = 0;
+    if (n == 0) return RT_OK;
+    rt::CompareAcc* acc = nullptr;
+    st = rt::static_scratch(&acc);
+    if (st != RT_OK) return st;
+    cudaStream_t s = (cudaStream_t)stream;
+    // The record still holds the previous call's result: clear it on the same stream first.
+    RT_CUDA_OK(cudaMemsetAsync(acc, 0, sizeof(rt::CompareAcc), s));
+    st = rt::enqueue_compare(got, ref, n, dtype, mode, tol, acc, s);
+    if (st != RT_OK) return st;
+    rt::CompareAcc result;
+    RT_CUDA_OK(cudaMemcpyAsync(&result, acc, sizeof(result), cudaMemcpyDeviceToHost, s));
+    RT_CUDA_OK(cudaStreamSynchronize(s));
+    *max_err = rt::acc_max_err(result, mode);
+    *n_bad = (int64_t)result.n_bad;
     return RT_OK;
 }
 
