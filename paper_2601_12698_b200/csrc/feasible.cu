@@ -74,7 +74,9 @@ std::vector<rt_params> raw_grid(const rt_shape& s)
 // The heuristic rules.  Returns the RT_PRUNE_* bit of the first rule that removes theta, or 0.
 static int heuristic_reject(const rt_shape& s, const rt_limits& L, const rt_params& p, const Plan& plan, int mask)
 {
-    if ((mask & RT_PRUNE_IDLE_THREADS) && p.threads_per_row > plan.slice_nvec) return RT_PRUNE_IDLE_THREADS;
+    // a row narrower than one warp keeps the smallest row width: something must remain feasible
+    if ((mask & RT_PRUNE_IDLE_THREADS) && p.threads_per_row > std::max(plan.slice_nvec, L.warp_size))
+        return RT_PRUNE_IDLE_THREADS;
     if (mask & RT_PRUNE_DUPLICATES) {
         // A batch deeper than the vectors a thread owns only adds predicated-off slots.
         if (p.unroll > next_pow2(plan.vec_per_thread)) return RT_PRUNE_DUPLICATES;

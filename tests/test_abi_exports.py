@@ -1,0 +1,66 @@
+"""The shared library loads without a GPU and exports every entry point the header declares."""
+import ctypes
+import os
+import re
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_functions():
+    text = open(os.path.join(ROOT, "include", "rmsnorm_tuner.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    names = re.findall(r"^\s*(?:const\s+)?(?:int|void|int32_t|int64_t|char\s*\*)\s*\*?\s*(\w+)\s*\(", text, flags=re.M)
+    return [n for n in names if not n.startswith("rt_evaluate_fn")]
+
+
+def test_library_exports_every_declared_symbol():
+    from paper_2601_12698_b200 import build
+    path = build.build()
+    lib = ctypes.CDLL(path)
+    declared = _declared_functions()
+    assert len(declared) >= 20 and "rmsnorm_template_launch" in declared and "tuner_search" in declared
+    assert "tuner_derive_feasible" in declared and "tuner_compare_static" in declared
+    missing = [n for n in declared if not hasattr(lib, n)]
+    assert not missing, missing
+
+
+def test_binding_covers_the_header():
+    from paper_2601_12698_b200 import binding
+    assert sorted(binding.EXPORTED) == sorted(_declared_functions())
+    assert binding.lib.rt_num_kernel_instances() == 410
+    assert binding.lib.rt_status_string(binding.RT_ERR_INFEASIBLE).decode().startswith("configuration outside")
+    inst = binding.kernel_instances()
+    assert {i["dtype"] for i in inst} == {0, 1, 2} and {i["stage"] for i in inst} == {0, 1, 2}
+    assert all(i["reg_vectors"] * (i["vec_bytes"] // (4 if i["dtype"] == 2 else 2)) <= 128 for i in inst)
+
+
+def test_struct_layouts_match_the_header_sizes():
+    """sizeof of each ctypes mirror equals what a C compiler gives for the header."""
+    import subprocess
+    import tempfile
+    from paper_2601_12698_b200 import binding as B
+    src = ('#include <stdio.h>\n#include "rmsnorm_tuner.h"\nint main(void){printf("%zu %zu %zu %zu %zu %zu %zu\\n",'
+           "sizeof(rt_params),sizeof(rt_shape),sizeof(rt_limits),sizeof(rt_budget),sizeof(rt_workspace),"
+           "sizeof(rt_eval_record),sizeof(rt_result));return 0;}\n")
+    with tempfile.TemporaryDirectory() as d:
+        c = os.path.join(d, "s.c")
+        open(c, "w").write(src)
+        exe = os.path.join(d, "s")
+        subprocess.run(["gcc", "-std=c99", "-I", os.path.join(ROOT, "include"), c, "-o", exe], check=True)
+        sizes = [int(v) for v in subprocess.run([exe], capture_output=True, text=True, check=True).stdout.split()]
+    mirrors = [B.rt_params, B.rt_shape, B.rt_limits, B.rt_budget, B.rt_workspace, B.rt_eval_record, B.rt_result]
+    assert sizes == [ctypes.sizeof(m) for m in mirrors]
+
+
+def test_no_device_is_reported_not_crashed():
+    import torch
+    if torch.cuda.is_available():
+        return
+    from paper_2601_12698_b200 import binding as B
+    L = B.rt_limits()
+    assert B.lib.rt_query_limits(ctypes.byref(L)) == B.RT_ERR_NO_DEVICE
+    n = ctypes.c_int32(0)
+    s = B.shape_of(4, 64, "bf16")
+    assert B.lib.tuner_derive_feasible(ctypes.byref(s), None, 0, ctypes.byref(n)) == B.RT_ERR_NO_DEVICE
+    th = B.make_params()
+    assert B.lib.rmsnorm_template_launch(ctypes.byref(th), 8, 8, 8, 8, 8, 4, 64, 1e-6, 0, None) == B.RT_ERR_NO_DEVICE

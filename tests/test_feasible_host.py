@@ -1,0 +1,92 @@
+"""The feasible-region deriver on the documented sm_100a limits (no GPU needed)."""
+import pytest
+
+from paper_2601_12698_b200 import binding as B
+
+
+@pytest.fixture(scope="module")
+def L():
+    return B.sm100_nominal_limits()
+
+
+def _keys(thetas):
+    return {t.key() for t in thetas}
+
+
+SHAPES = [(128, 4096, "bf16"), (1, 4096, "bf16"), (16384, 8192, "bf16"), (8192, 5120, "fp16"), (8192, 6152, "fp16"),
+          (8192, 6148, "fp16"), (32768, 12288, "fp32"), (64, 6146, "fp16"), (64, 6145, "fp16"), (3, 8, "fp32")]
+
+
+@pytest.mark.parametrize("T,H,dtype", SHAPES)
+def test_every_emitted_theta_passes_the_hard_rules_and_counts_add_up(L, T, H, dtype):
+    s = B.shape_of(T, H, dtype)
+    feasible = B.tuner_derive_feasible(s, L)
+    assert feasible, "empty feasible set"
+    assert len(_keys(feasible)) == len(feasible)  # no duplicates
+    for th in feasible:
+        assert B.tuner_check_params(s, th, L) == B.RT_OK
+        assert th.threads_per_row * th.rows_per_cta <= 1024
+        assert (H * (4 if dtype == "fp32" else 2)) % th.vec_bytes == 0
+        assert (th.reduce == B.RT_REDUCE_CLUSTER) == (th.cluster_size > 1)
+    c = B.tuner_derive_counts(s, L)
+    assert c["feasible"] == len(feasible)
+    assert sum(v for k, v in c.items() if k != "raw") == c["raw"] == len(B.tuner_raw_grid(s))
+
+
+def test_heuristics_only_remove_points(L):
+    s = B.shape_of(128, 4096, "bf16")
+    wide = _keys(B.tuner_derive_feasible(s, L, heuristics=0))
+    for mask in (B.RT_PRUNE_IDLE_THREADS, B.RT_PRUNE_DUPLICATES, B.RT_PRUNE_CLUSTER_WAVES, B.RT_PRUNE_IDLE_ROWS,
+                 B.RT_PRUNE_DEFAULT):
+        narrow = _keys(B.tuner_derive_feasible(s, L, heuristics=mask))
+        assert narrow <= wide
+    assert len(_keys(B.tuner_derive_feasible(s, L))) < len(wide)
+
+
+def test_rules_bite_where_they_should(L):
+    # 6148 fp16: row bytes = 8 mod 16 -> only 8-byte vectors, no TMA stage
+    f = B.tuner_derive_feasible(B.shape_of(8192, 6148, "fp16"), L)
+    assert {t.vec_bytes for t in f} == {8} and B.RT_STAGE_SMEM_TMA not in {t.stage for t in f}
+    # 6152 fp16: 769 16-byte vectors, both widths, all stages
+    f = B.tuner_derive_feasible(B.shape_of(8192, 6152, "fp16"), L)
+    assert {t.vec_bytes for t in f} == {8, 16} and {t.stage for t in f} == {0, 1, 2}
+    # rows that fit no 8-byte vector fall back to the widest narrow width
+    assert {t.vec_bytes for t in B.tuner_derive_feasible(B.shape_of(64, 6146, "fp16"), L)} == {4}
+    assert {t.vec_bytes for t in B.tuner_derive_feasible(B.shape_of(64, 6145, "fp16"), L)} == {2}
+    # pointers that are only 8-byte aligned remove the 16-byte vectors and TMA
+    f = B.tuner_derive_feasible(B.shape_of(128, 4096, "bf16", min_ptr_align=8), L)
+    assert {t.vec_bytes for t in f} == {8} and B.RT_STAGE_SMEM_TMA not in {t.stage for t in f}
+    # a single token: one row per CTA only; clusters are allowed (too few rows to fill the SMs)
+    f = B.tuner_derive_feasible(B.shape_of(1, 4096, "bf16"), L)
+    assert {t.rows_per_cta for t in f} == {1} and 8 in {t.cluster_size for t in f}
+    # the prefill shape fills the machine with whole rows: no cluster split survives
+    f = B.tuner_derive_feasible(B.shape_of(16384, 8192, "bf16"), L)
+    assert {t.cluster_size for t in f} == {1}
+    # register stage: a 32-thread row of 1024 vectors would need 32 vectors per thread (256 fp32): rejected
+    s = B.shape_of(16384, 8192, "bf16")
+    assert B.tuner_check_params(s, B.make_params(threads_per_row=32), L) == B.RT_ERR_INFEASIBLE
+    assert b"register" in B.lib.rt_last_error()
+    # shared-memory stage: 8 rows of fp32 12288 need 8 * 48 KB
+    s5 = B.shape_of(32768, 12288, "fp32")
+    assert B.tuner_check_params(s5, B.make_params(threads_per_row=128, rows_per_cta=8, stage=B.RT_STAGE_SMEM_LDG), L) == B.RT_ERR_INFEASIBLE
+    assert b"shared memory" in B.lib.rt_last_error()
+    assert B.tuner_check_params(s5, B.make_params(threads_per_row=128, rows_per_cta=2, stage=B.RT_STAGE_SMEM_TMA), L) == B.RT_OK
+    assert B.tuner_check_params(s5, B.make_params(threads_per_row=128, rows_per_cta=4, stage=B.RT_STAGE_SMEM_TMA), L) == B.RT_ERR_INFEASIBLE
+
+
+def test_argument_errors(L):
+    import ctypes
+    n = ctypes.c_int32(0)
+    assert B.lib.tuner_derive_feasible_ex(None, ctypes.byref(L), 15, None, 0, ctypes.byref(n)) == B.RT_ERR_NULL
+    bad = B.shape_of(4, 64, 7)
+    assert B.lib.tuner_derive_feasible_ex(ctypes.byref(bad), ctypes.byref(L), 15, None, 0, ctypes.byref(n)) == B.RT_ERR_DTYPE
+    bad = B.shape_of(-1, 64, "bf16")
+    assert B.lib.tuner_derive_feasible_ex(ctypes.byref(bad), ctypes.byref(L), 15, None, 0, ctypes.byref(n)) == B.RT_ERR_SHAPE
+    bad = B.shape_of(4, 0, "bf16")
+    assert B.lib.tuner_derive_feasible_ex(ctypes.byref(bad), ctypes.byref(L), 15, None, 0, ctypes.byref(n)) == B.RT_ERR_SHAPE
+    ok = B.shape_of(4, 4096, "bf16")
+    assert B.lib.tuner_derive_feasible_ex(ctypes.byref(ok), ctypes.byref(L), 15, None, 5, ctypes.byref(n)) == B.RT_ERR_NULL
+    # a small capacity still reports the full count
+    arr = (B.rt_params * 3)()
+    assert B.lib.tuner_derive_feasible_ex(ctypes.byref(ok), ctypes.byref(L), 15, arr, 3, ctypes.byref(n)) == B.RT_OK
+    assert n.value > 3

@@ -1,0 +1,143 @@
+"""The search on a synthetic cost function with a known optimum (host only): grid + hill-climb logic,
+budget accounting, seeds, gate failures, exhaustive mode."""
+import math
+
+import pytest
+
+from paper_2601_12698_b200 import binding as B
+
+
+@pytest.fixture(scope="module")
+def L():
+    return B.sm100_nominal_limits()
+
+
+SHAPE = (16384, 8192, "bf16")
+
+
+def _cost_factory(opt, noise=None, counter=None):
+    """Separable bowl over the ordered axes with a preferred stage/reduction: minimum 100 us at `opt`."""
+    def cost(p):
+        if counter is not None:
+            counter.append(p.key())
+        t = 100.0
+        t += 12.0 * abs(math.log2(p.threads_per_row) - math.log2(opt["tpr"]))
+        t += 7.0 * abs(math.log2(p.rows_per_cta) - math.log2(opt["rpc"]))
+        t += 5.0 * abs(math.log2(p.unroll) - math.log2(opt["unroll"]))
+        t += 9.0 * abs(math.log2(p.vec_bytes) - math.log2(opt["vec"]))
+        t += 0.0 if p.stage == opt["stage"] else 15.0
+        t += 0.0 if p.reduce == opt["reduce"] else 4.0
+        if noise is not None:
+            t *= 1.0 + noise(p)
+        return t
+    return cost
+
+
+OPTIMA = [dict(tpr=256, rpc=1, unroll=1, vec=16, stage=2, reduce=0),
+          dict(tpr=128, rpc=2, unroll=2, vec=16, stage=0, reduce=1),
+          dict(tpr=512, rpc=1, unroll=4, vec=8, stage=1, reduce=0),
+          dict(tpr=64, rpc=4, unroll=2, vec=16, stage=1, reduce=0)]
+
+
+@pytest.mark.parametrize("opt", OPTIMA)
+def test_guided_search_finds_the_known_optimum_within_budget(L, opt):
+    s = B.shape_of(*SHAPE)
+    feasible = B.tuner_derive_feasible(s, L)
+    target = [t for t in feasible if (t.threads_per_row, t.rows_per_cta, t.unroll, t.vec_bytes, t.stage, t.reduce) ==
+              (opt["tpr"], opt["rpc"], opt["unroll"], opt["vec"], opt["stage"], opt["reduce"])]
+    assert target, "the planted optimum must be feasible"
+    calls = []
+    budget = 80
+    res, log = B.tuner_search_with(s, L, B.make_budget(max_evals=budget, top_k=3), _cost_factory(opt, counter=calls))
+    assert res.best.key() == target[0].key(), (res.best, res.best_us)
+    assert abs(res.best_us - 100.0) < 1e-3
+    assert res.evals_used == len(calls) == len(log) <= budget
+    assert res.n_candidates == len(feasible) and budget < len(feasible) / 4
+    assert [r.eval_index for r in log] == list(range(len(log)))
+    phases = [r.phase for r in log]
+    assert phases == sorted(phases[:-3]) + [3, 3, 3]  # grid, then climb, then exactly top_k re-tests
+    # nothing but the re-tested finalists is evaluated twice
+    first = [r.params.key() for r in log if r.phase != 3]
+    assert len(set(first)) == len(first)
+
+
+def test_exhaustive_mode_visits_every_candidate_once(L):
+    s = B.shape_of(128, 4096, "bf16")
+    feasible = B.tuner_derive_feasible(s, L)
+    calls = []
+    res, log = B.tuner_search_with(s, L, B.make_budget(max_evals=len(feasible), top_k=0, strategy=B.RT_SEARCH_EXHAUSTIVE),
+                                   _cost_factory(dict(tpr=128, rpc=1, unroll=2, vec=16, stage=0, reduce=0), counter=calls))
+    assert res.evals_used == len(feasible) and sorted(calls) == sorted(t.key() for t in feasible)
+    assert all(r.phase == 4 for r in log) and abs(res.best_us - 100.0) < 1e-3
+    # a budget smaller than the set stops early and says so through evals_used
+    res2, _ = B.tuner_search_with(s, L, B.make_budget(max_evals=50, top_k=0, strategy=B.RT_SEARCH_EXHAUSTIVE),
+                                  _cost_factory(dict(tpr=128, rpc=1, unroll=2, vec=16, stage=0, reduce=0)))
+    assert res2.evals_used == 50
+
+
+def test_budget_is_never_exceeded_and_tiny_budgets_still_return(L):
+    s = B.shape_of(*SHAPE)
+    cost = _cost_factory(OPTIMA[0])
+    for budget in (1, 2, 3, 5, 8, 13, 40):
+        res, log = B.tuner_search_with(s, L, B.make_budget(max_evals=budget, top_k=5), cost)
+        assert 1 <= res.evals_used <= budget and len(log) == res.evals_used
+        assert res.best_us >= 100.0
+    with pytest.raises(B.TunerError) as e:
+        B.tuner_search_with(s, L, B.make_budget(max_evals=0), cost)
+    assert e.value.status == B.RT_ERR_BUDGET
+
+
+def test_seeds_are_evaluated_first_and_help(L):
+    s = B.shape_of(*SHAPE)
+    opt = OPTIMA[1]
+    seed = B.make_params(threads_per_row=opt["tpr"], rows_per_cta=opt["rpc"], vec_bytes=opt["vec"], unroll=opt["unroll"],
+                         stage=opt["stage"], reduce=opt["reduce"])
+    infeasible_seed = B.make_params(threads_per_row=1024, rows_per_cta=8)
+    res, log = B.tuner_search_with(s, L, B.make_budget(max_evals=12, top_k=2, seeds=[infeasible_seed, seed]),
+                                   _cost_factory(opt))
+    assert log[0].phase == 0 and log[0].params.key() == seed.key()  # the infeasible seed is skipped silently
+    assert sum(1 for r in log if r.phase == 0) == 1
+    assert res.best.key() == seed.key() and abs(res.best_us - 100.0) < 1e-3
+    # the same tiny budget without the seed does not reach the optimum
+    cold, _ = B.tuner_search_with(s, L, B.make_budget(max_evals=12, top_k=2), _cost_factory(opt))
+    assert cold.best_us > 100.0
+
+
+def test_candidates_that_fail_the_gate_are_skipped_and_counted(L):
+    s = B.shape_of(*SHAPE)
+    base = _cost_factory(OPTIMA[0])
+
+    def cost(p):  # every TMA candidate "fails parity", NaN for the shared-memory tree
+        if p.stage == B.RT_STAGE_SMEM_TMA:
+            return -1.0
+        if p.reduce == B.RT_REDUCE_SMEM:
+            return float("nan")
+        return base(p)
+    res, log = B.tuner_search_with(s, L, B.make_budget(max_evals=80, top_k=3), cost)
+    assert res.best.stage != B.RT_STAGE_SMEM_TMA and res.best.reduce != B.RT_REDUCE_SMEM
+    failed = [r for r in log if r.status != B.RT_OK]
+    assert res.n_failed_gate == len(failed) > 0 and all(r.status == B.RT_ERR_MISMATCH for r in failed)
+    assert abs(res.best_us - 115.0) < 1e-3  # the best point outside the failing stage
+    with pytest.raises(B.TunerError) as e:
+        B.tuner_search_with(s, L, B.make_budget(max_evals=20), lambda p: -1.0)
+    assert e.value.status == B.RT_ERR_MISMATCH
+
+
+def test_search_tolerates_timing_noise(L):
+    """3% multiplicative noise, deterministic per theta: the winner is within 3% of the optimum."""
+    s = B.shape_of(*SHAPE)
+
+    def noise(p):
+        h = hash(p.key()) & 0xFFFF
+        return 0.03 * (h / 65535.0 - 0.5)
+    res, _ = B.tuner_search_with(s, L, B.make_budget(max_evals=80, top_k=5), _cost_factory(OPTIMA[0], noise=noise))
+    clean = _cost_factory(OPTIMA[0])(res.best)
+    assert clean <= 103.0 + 7.0  # at most one small axis step away
+
+
+def test_empty_feasible_set_is_an_error_not_a_crash(L):
+    # fp32 rows of 3 elements: 12 bytes, only 4-byte vectors; with 2-byte pointer alignment nothing fits
+    s = B.shape_of(4, 3, "fp32", min_ptr_align=2)
+    with pytest.raises(B.TunerError) as e:
+        B.tuner_search_with(s, L, B.make_budget(max_evals=10), lambda p: 1.0)
+    assert e.value.status == B.RT_ERR_INFEASIBLE
