@@ -273,6 +273,13 @@ int tuner_search_with(const rt_shape* s, const rt_limits* limits, const rt_budge
 int tuner_evaluate(const rt_shape* s, const rt_params* p, const rt_budget* b, const rt_workspace* ws,
                    rt_eval_record* out);
 
+/*
+ * Time of an empty kernel under the same protocol (warmup, iters, repeats, use_graph of `b`), in
+ * microseconds per launch: the floor below which no candidate of a latency-bound shape can score.
+ * Synchronises `stream`.  (Measurement aid for "Performance Measurement"; the paper has no counterpart.)
+ */
+int tuner_launch_floor(const rt_budget* b, void* stream, float* us);
+
 typedef enum { RT_CMP_BITS = 0, RT_CMP_ULP16 = 1, RT_CMP_REL32 = 2 } rt_compare_mode;
 /*
  * The distance d(.,.) of the correctness criterion, computed on the device.

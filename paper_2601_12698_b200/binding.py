@@ -114,6 +114,7 @@ _SIGNATURES = {
                                   POINTER(rt_result), POINTER(rt_eval_record), c_int32]),
     "tuner_evaluate": (c_int, [POINTER(rt_shape), POINTER(rt_params), POINTER(rt_budget), POINTER(rt_workspace),
                                POINTER(rt_eval_record)]),
+    "tuner_launch_floor": (c_int, [POINTER(rt_budget), c_void_p, POINTER(c_float)]),
     "tuner_compare": (c_int, [c_void_p, c_void_p, c_int64, c_int, c_int, c_double, POINTER(c_double),
                               POINTER(c_int64), c_void_p]),
     "tuner_compare_static": (c_int, [c_void_p, c_void_p, c_int64, c_int, c_int, c_double, POINTER(c_double),
@@ -308,6 +309,13 @@ def tuner_evaluate(shape: rt_shape, params: rt_params, budget: rt_budget, ws: rt
     rec = rt_eval_record()
     _check(lib.tuner_evaluate(byref(shape), byref(params), byref(budget), byref(ws), byref(rec)), "tuner_evaluate")
     return rec
+
+
+def tuner_launch_floor(budget: rt_budget, stream=None) -> float:
+    """Microseconds per launch of an empty kernel under the budget's timing protocol."""
+    us = c_float(0.0)
+    _check(lib.tuner_launch_floor(byref(budget), _stream_ptr(stream), byref(us)), "tuner_launch_floor")
+    return us.value
 
 
 def tuner_compare(got, ref, mode: int, tol: float = 0.0, stream=None):

@@ -112,6 +112,27 @@ __device__ __forceinline__ Vec<VB> ld_weight(const void* p)
     return v;
 }
 
+// The same load pinned in program order (volatile): used to put the weight fetch ahead of the row
+// reduction, so that its latency overlaps the barrier instead of following it.
+template <int VB>
+__device__ __forceinline__ Vec<VB> ld_weight_early(const void* p)
+{
+    Vec<VB> v;
+    if constexpr (VB == 16) {
+        asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(v.w[0]), "=r"(v.w[1]), "=r"(v.w[2]), "=r"(v.w[3]) : "l"(p));
+    } else if constexpr (VB == 8) {
+        asm volatile("ld.global.nc.v2.u32 {%0,%1}, [%2];" : "=r"(v.w[0]), "=r"(v.w[1]) : "l"(p));
+    } else if constexpr (VB == 4) {
+        asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(v.w[0]) : "l"(p));
+    } else {
+        unsigned short h;
+        asm volatile("ld.global.nc.u16 %0, [%1];" : "=h"(h) : "l"(p));
+        v.w[0] = h;
+    }
+    return v;
+}
+
 template <int VB>
 __device__ __forceinline__ Vec<VB> ld_shared(const void* p)
 {
@@ -420,6 +441,18 @@ __global__ void add_rmsnorm_kernel(const KernelArgs a)
                 }
             }
         }
+        // A thread that owns at most two vectors (the latency-bound shapes) fetches its weights before the
+        // reduction: a few registers buy the overlap of that fetch with the barrier.  Threads that own
+        // more fetch them afterwards, where other CTAs' traffic hides the latency and registers are scarce.
+        constexpr bool kEarlyWeight = CAP <= 2;
+        Vec<VB> wv[kEarlyWeight ? CAP : 1];
+        if constexpr (kEarlyWeight) {
+#pragma unroll
+            for (int i = 0; i < CAP; ++i) {
+                const int v = tx + i * tpr;
+                if (v < n) wv[i] = ld_weight_early<VB>(wrow + (size_t)v * VB);
+            }
+        }
         const float total = row_reduce<REDUCE>(ss, tx, ty, tpr, crank, csize);
         const float rho = __frsqrt_rn(total / (float)a.hidden + a.eps);
 #pragma unroll
@@ -427,7 +460,8 @@ __global__ void add_rmsnorm_kernel(const KernelArgs a)
             const int v = tx + i * tpr;
             if (v < n) {
                 float wf[EPV], yf[EPV];
-                C::unpack(ld_weight<VB>(wrow + (size_t)v * VB), wf);
+                if constexpr (kEarlyWeight) C::unpack(wv[i], wf);
+                else C::unpack(ld_weight<VB>(wrow + (size_t)v * VB), wf);
 #pragma unroll
                 for (int e = 0; e < EPV; ++e) yf[e] = s[i][e] * rho * wf[e];
                 st_stream<VB>(yrow + (size_t)v * VB, C::pack(yf));

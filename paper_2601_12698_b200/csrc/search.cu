@@ -388,6 +388,61 @@ struct DeviceEvaluator : Evaluator {
     }
 };
 
+// The launch floor: an empty kernel timed with the same protocol, so that the share of launch overhead in
+// the time of a latency-bound shape is visible.
+__global__ void empty_kernel() {}
+
+static int time_launch_floor(const rt_budget& b, cudaStream_t stream, float* out_us)
+{
+    const int iters = b.iters > 0 ? b.iters : 1, repeats = b.repeats > 0 ? b.repeats : 1;
+    for (int i = 0; i < b.warmup; ++i) empty_kernel<<<1, 32, 0, stream>>>();
+    cudaGraphExec_t graph_exec = nullptr;
+    if (b.use_graph) {
+        if (!stream) {
+            set_error("use_graph needs a non-default stream");
+            return RT_ERR_CUDA;
+        }
+        cudaGraph_t graph = nullptr;
+        RT_CUDA_OK(cudaStreamBeginCapture(stream, cudaStreamCaptureModeThreadLocal));
+        for (int i = 0; i < iters; ++i) empty_kernel<<<1, 32, 0, stream>>>();
+        RT_CUDA_OK(cudaStreamEndCapture(stream, &graph));
+        cudaError_t ce = cudaGraphInstantiate(&graph_exec, graph, 0);
+        cudaGraphDestroy(graph);
+        if (ce != cudaSuccess) {
+            set_error("cudaGraphInstantiate failed: %s", cudaGetErrorString(ce));
+            return RT_ERR_CUDA;
+        }
+        RT_CUDA_OK(cudaGraphLaunch(graph_exec, stream));
+    }
+    cudaEvent_t e0, e1;
+    RT_CUDA_OK(cudaEventCreate(&e0));
+    RT_CUDA_OK(cudaEventCreate(&e1));
+    std::vector<float> block_us;
+    for (int rep = 0; rep < repeats; ++rep) {
+        cudaEventRecord(e0, stream);
+        if (graph_exec) {
+            cudaGraphLaunch(graph_exec, stream);
+        } else {
+            for (int i = 0; i < iters; ++i) empty_kernel<<<1, 32, 0, stream>>>();
+        }
+        cudaEventRecord(e1, stream);
+        float ms = 0.f;
+        if (cudaEventSynchronize(e1) == cudaSuccess && cudaEventElapsedTime(&ms, e0, e1) == cudaSuccess)
+            block_us.push_back(ms * 1000.f / iters);
+    }
+    count_launch((int64_t)repeats * iters + b.warmup);
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (graph_exec) cudaGraphExecDestroy(graph_exec);
+    RT_CUDA_OK(cudaGetLastError());
+    if (block_us.empty()) {
+        set_error("launch-floor timing failed");
+        return RT_ERR_CUDA;
+    }
+    *out_us = median_of(block_us);
+    return RT_OK;
+}
+
 struct CallbackEvaluator : Evaluator {
     rt_evaluate_fn fn;
     void* user;
@@ -773,6 +828,15 @@ int tuner_search_with(const rt_shape* s, const rt_limits* limits, const rt_budge
     ev.fn = evaluate;
     ev.user = user;
     return rt::run_search(*s, *limits, rt::normalised(b), ev, out, log, log_cap);
+}
+
+int tuner_launch_floor(const rt_budget* b, void* stream, float* us)
+{
+    if (!b || !us) {
+        rt::set_error("tuner_launch_floor: NULL argument");
+        return RT_ERR_NULL;
+    }
+    return rt::time_launch_floor(rt::normalised(b), (cudaStream_t)stream, us);
 }
 
 void rt_shutdown(void)
