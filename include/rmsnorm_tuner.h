@@ -280,6 +280,51 @@ int tuner_evaluate(const rt_shape* s, const rt_params* p, const rt_budget* b, co
  */
 int tuner_launch_floor(const rt_budget* b, void* stream, float* us);
 
+/* ---- 4. general configuration and specialised table -------------------------------------- */
+
+/* One row of D_spec: a shape and the best theta found for it. */
+typedef struct {
+    rt_shape shape;
+    rt_params best;
+    float best_us;
+    int32_t reserved;
+} rt_spec_entry;
+
+typedef enum { RT_FROM_TABLE_EXACT = 0, RT_FROM_TABLE_NEAREST = 1, RT_FROM_GENERAL = 2,
+               RT_FROM_FEASIBLE_SET = 3 } rt_theta_source;
+
+/*
+ * SelectGeneral (Algorithm 1; "Performance Measurement": the general configuration is the one with the
+ * best average performance across shapes).  Host only.
+ *   times_us  host, [n_candidates][n_shapes], the measured time of candidate c on shape x; a value <= 0,
+ *             NaN or inf marks "could not run / failed its gate on that shape".
+ * With T*(x) the best time on shape x over all candidates, the score of a candidate is the geometric mean
+ * over shapes of T*(x) / T(theta, x) (the paper's geometric-mean speedup with the per-shape optimum as the
+ * reference; 1.0 = best everywhere).  A candidate that cannot run on some shape scores 0 and is not
+ * eligible.  *best_index receives the eligible candidate with the highest score (first on ties);
+ * scores (may be NULL) receives every candidate's score.  RT_ERR_INFEASIBLE when none is eligible.
+ */
+int tuner_select_general(const float* times_us, int32_t n_candidates, int32_t n_shapes, int32_t* best_index,
+                         float* best_score, float* scores);
+
+/*
+ * BuildSpecialized's table put to use: theta for a query shape.  Host only (limits == NULL asks the
+ * current device).  Order of preference: the table entry of the same dtype nearest to the query (distance
+ * = 4 x octaves of hidden size + octaves of token count; distance 0 is an exact hit) whose theta passes the
+ * hard feasibility rules for the query; else `general` (may be NULL) if feasible; else the first point
+ * of the derived feasible set.  *source (may be NULL) receives an rt_theta_source.
+ */
+int tuner_table_lookup(const rt_spec_entry* table, int32_t n_entries, const rt_params* general,
+                       const rt_shape* query, const rt_limits* limits, rt_params* out, int32_t* source);
+
+/*
+ * rmsnorm_template_launch with theta taken from tuner_table_lookup for this call's shape and pointer
+ * alignment.  `used` (may be NULL) receives the theta launched.  Asynchronous, allocates nothing.
+ */
+int rmsnorm_launch_auto(const rt_spec_entry* table, int32_t n_entries, const rt_params* general,
+                        const void* x, const void* r, const void* w, void* y, void* r_out, int64_t n_tokens,
+                        int64_t hidden, float eps, int dtype, void* stream, rt_params* used);
+
 typedef enum { RT_CMP_BITS = 0, RT_CMP_ULP16 = 1, RT_CMP_REL32 = 2 } rt_compare_mode;
 /*
  * The distance d(.,.) of the correctness criterion, computed on the device.

@@ -92,6 +92,12 @@ class rt_result(Structure):
                 ("n_log", c_int32), ("n_failed_gate", c_int32)]
 
 
+class rt_spec_entry(Structure):
+    _fields_ = [("shape", rt_shape), ("best", rt_params), ("best_us", c_float), ("reserved", c_int32)]
+
+
+SOURCE_NAMES = {0: "table_exact", 1: "table_nearest", 2: "general", 3: "feasible_set"}
+
 rt_evaluate_fn = ctypes.CFUNCTYPE(c_double, POINTER(rt_params), c_void_p)
 
 _SIGNATURES = {
@@ -114,6 +120,12 @@ _SIGNATURES = {
                                   POINTER(rt_result), POINTER(rt_eval_record), c_int32]),
     "tuner_evaluate": (c_int, [POINTER(rt_shape), POINTER(rt_params), POINTER(rt_budget), POINTER(rt_workspace),
                                POINTER(rt_eval_record)]),
+    "tuner_select_general": (c_int, [POINTER(c_float), c_int32, c_int32, POINTER(c_int32), POINTER(c_float),
+                                     POINTER(c_float)]),
+    "tuner_table_lookup": (c_int, [POINTER(rt_spec_entry), c_int32, POINTER(rt_params), POINTER(rt_shape),
+                                   POINTER(rt_limits), POINTER(rt_params), POINTER(c_int32)]),
+    "rmsnorm_launch_auto": (c_int, [POINTER(rt_spec_entry), c_int32, POINTER(rt_params), c_void_p, c_void_p, c_void_p,
+                                    c_void_p, c_void_p, c_int64, c_int64, c_float, c_int, c_void_p, POINTER(rt_params)]),
     "tuner_launch_floor": (c_int, [POINTER(rt_budget), c_void_p, POINTER(c_float)]),
     "tuner_compare": (c_int, [c_void_p, c_void_p, c_int64, c_int, c_int, c_double, POINTER(c_double),
                               POINTER(c_int64), c_void_p]),
@@ -337,6 +349,74 @@ def tuner_compare_static(got, ref, mode: int, tol: float = 0.0, stream=None):
     _check(lib.tuner_compare_static(got.data_ptr(), ref.data_ptr(), got.numel(), _dtype_code(got), mode, tol,
                                     byref(worst), byref(bad), _stream_ptr(stream)), "tuner_compare_static")
     return worst.value, bad.value
+
+
+# ---- 4. general configuration and specialised table -------------------------------------------------------------
+
+def tuner_select_general(times_us) -> tuple[int, float, list[float]]:
+    """times_us[c][x] -> (index of theta_gen, its geometric-mean score, every candidate's score)."""
+    n_c, n_x = len(times_us), len(times_us[0])
+    flat = (c_float * (n_c * n_x))(*[float(v) for row in times_us for v in row])
+    best, score, scores = c_int32(-1), c_float(0.0), (c_float * n_c)()
+    _check(lib.tuner_select_general(flat, n_c, n_x, byref(best), byref(score), scores), "tuner_select_general")
+    return best.value, score.value, list(scores)
+
+
+class SpecTable:
+    """D_spec and theta_gen as the C arrays the library consumes, with JSON persistence (marshalling only)."""
+
+    def __init__(self, entries=(), general: rt_params | None = None, device_name: str = ""):
+        self.entries = list(entries)  # [(rt_shape, rt_params, best_us)]
+        self.general = general
+        self.device_name = device_name
+        self._pack()
+
+    def _pack(self):
+        self._arr = (rt_spec_entry * max(1, len(self.entries)))()
+        for i, (shape, theta, us) in enumerate(self.entries):
+            self._arr[i] = rt_spec_entry(shape, theta, us, 0)
+
+    def add(self, shape: rt_shape, theta: rt_params, best_us: float):
+        self.entries.append((shape, theta, best_us))
+        self._pack()
+
+    def lookup(self, shape: rt_shape, limits: rt_limits | None = None):
+        out, src = rt_params(), c_int32(-1)
+        _check(lib.tuner_table_lookup(self._arr, len(self.entries), byref(self.general) if self.general else None,
+                                      byref(shape), byref(limits) if limits is not None else None, byref(out),
+                                      byref(src)), "tuner_table_lookup")
+        return out, SOURCE_NAMES[src.value]
+
+    def launch(self, x, r, w, y, r_out, eps: float, stream=None) -> rt_params:
+        """rmsnorm_launch_auto on device tensors; returns the theta that was launched."""
+        n_tokens, hidden = x.shape
+        used = rt_params()
+        _check(lib.rmsnorm_launch_auto(self._arr, len(self.entries), byref(self.general) if self.general else None,
+                                       x.data_ptr(), r.data_ptr(), w.data_ptr(), y.data_ptr(), r_out.data_ptr(),
+                                       n_tokens, hidden, eps, _dtype_code(x), _stream_ptr(stream), byref(used)),
+               "rmsnorm_launch_auto")
+        return used
+
+    def to_json(self) -> dict:
+        names = {v: k for k, v in DTYPE_CODES.items()}
+        return {"device": self.device_name, "general": self.general.as_dict() if self.general else None,
+                "specialised": [{"dtype": names[s.dtype], "n_tokens": int(s.n_tokens), "hidden": int(s.hidden),
+                                 "theta": t.as_dict(), "us": round(float(us), 3)} for s, t, us in self.entries]}
+
+    @classmethod
+    def default(cls) -> "SpecTable":
+        """The table shipped with the package (tuned on a B200 with ``python -m paper_2601_12698_b200.tune``)."""
+        import json
+        with open(os.path.join(_HERE, "tables", "b200_default.json")) as f:
+            return cls.from_json(json.load(f))
+
+    @classmethod
+    def from_json(cls, d: dict) -> "SpecTable":
+        fields = [k for k, _ in rt_params._fields_]
+        mk = lambda t: rt_params(*[int(t[k]) for k in fields])
+        entries = [(shape_of(e["n_tokens"], e["hidden"], e["dtype"]), mk(e["theta"]), float(e["us"]))
+                   for e in d.get("specialised", [])]
+        return cls(entries, mk(d["general"]) if d.get("general") else None, d.get("device", ""))
 
 
 def rt_device_status() -> int:

@@ -23,7 +23,7 @@ LIB_PATH = os.path.join(HERE, "librmsnorm_tuner.so")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-std=c++17", "-O3", "-lineinfo",
               "-Xcompiler", "-fPIC", "-I", CSRC, "-I", INCLUDE]
-HOST_UNITS = ["launch.cu", "feasible.cu", "search.cu", "host_run.cu"]
+HOST_UNITS = ["launch.cu", "feasible.cu", "search.cu", "host_run.cu", "table.cu"]
 ELEMENT_TYPES = {"bf16": ("__nv_bfloat16", 0), "fp16": ("__half", 1), "fp32": ("float", 2)}
 GROUPS = {"reg": 0, "smem": 1, "narrow": 2}
 

@@ -1,0 +1,149 @@
+// SelectGeneral and BuildSpecialized of Algorithm 1: the general configuration theta_gen (one theta for all
+// shapes, chosen by geometric-mean speedup as in "Performance Measurement and Evaluation") and the
+// specialised table D_spec (shape -> its own best theta), with a launch entry point that consults them.
+#include <math.h>
+#include <string.h>
+
+#include "tuner_internal.h"
+
+namespace rt {
+
+// Distance between two shapes of one dtype: octaves of hidden size and of token count.  Hidden size
+// weighs more: it fixes vector counts, register and shared-memory footprints; the token count only
+// decides how full the machine is.
+static double shape_distance(const rt_shape& a, const rt_shape& b)
+{
+    const double dh = fabs(log2((double)a.hidden) - log2((double)b.hidden));
+    const double dt = fabs(log2((double)std::max<int64_t>(a.n_tokens, 1)) - log2((double)std::max<int64_t>(b.n_tokens, 1)));
+    return 4.0 * dh + dt;
+}
+
+int table_lookup(const rt_spec_entry* table, int32_t n, const rt_params* general, const rt_shape* query,
+                 const rt_limits* limits, rt_params* out, int32_t* source)
+{
+    int best = -1;
+    double best_d = 0.0;
+    for (int32_t i = 0; i < n; ++i) {
+        const rt_spec_entry& e = table[i];
+        if (e.shape.dtype != query->dtype) continue;
+        const double d = shape_distance(e.shape, *query);
+        if (best >= 0 && d >= best_d) continue;
+        Plan plan;
+        if (make_plan(query, &e.best, limits, &plan) != RT_OK) continue;  // not launchable on this shape
+        best = i;
+        best_d = d;
+    }
+    if (best >= 0) {
+        *out = table[best].best;
+        if (source) *source = best_d == 0.0 ? RT_FROM_TABLE_EXACT : RT_FROM_TABLE_NEAREST;
+        return RT_OK;
+    }
+    if (general) {
+        Plan plan;
+        if (make_plan(query, general, limits, &plan) == RT_OK) {
+            *out = *general;
+            if (source) *source = RT_FROM_GENERAL;
+            return RT_OK;
+        }
+    }
+    // Last resort: the first point of the feasible set (registers, shuffle, widest vector that fits).
+    std::vector<rt_params> feasible;
+    int st = derive_feasible(*query, *limits, RT_PRUNE_DEFAULT, &feasible, nullptr);
+    if (st != RT_OK) return st;
+    if (feasible.empty()) {
+        set_error("no feasible configuration for this shape");
+        return RT_ERR_INFEASIBLE;
+    }
+    *out = feasible[0];
+    if (source) *source = RT_FROM_FEASIBLE_SET;
+    return RT_OK;
+}
+
+}  // namespace rt
+
+extern "C" {
+
+int tuner_select_general(const float* times_us, int32_t n_candidates, int32_t n_shapes, int32_t* best_index,
+                         float* best_score, float* scores)
+{
+    if (!times_us || !best_index) {
+        rt::set_error("tuner_select_general: NULL argument");
+        return RT_ERR_NULL;
+    }
+    if (n_candidates < 1 || n_shapes < 1) {
+        rt::set_error("tuner_select_general: empty table");
+        return RT_ERR_SHAPE;
+    }
+    // T*(x): the best time on each shape over the candidates that ran there.
+    std::vector<double> best_time(n_shapes, INFINITY);
+    for (int32_t c = 0; c < n_candidates; ++c)
+        for (int32_t x = 0; x < n_shapes; ++x) {
+            const float t = times_us[(size_t)c * n_shapes + x];
+            if (t > 0.f && isfinite(t)) best_time[x] = std::min(best_time[x], (double)t);
+        }
+    int32_t best = -1;
+    double best_s = -1.0;
+    for (int32_t c = 0; c < n_candidates; ++c) {
+        // geometric mean over shapes of T*(x) / T(theta, x); a candidate that cannot run somewhere is out
+        double log_sum = 0.0;
+        bool everywhere = true;
+        for (int32_t x = 0; x < n_shapes && everywhere; ++x) {
+            const float t = times_us[(size_t)c * n_shapes + x];
+            if (!(t > 0.f) || !isfinite(t))
+                everywhere = false;
+            else
+                log_sum += log(best_time[x] / (double)t);
+        }
+        const double score = everywhere ? exp(log_sum / n_shapes) : 0.0;
+        if (scores) scores[c] = (float)score;
+        if (everywhere && score > best_s) {
+            best_s = score;
+            best = c;
+        }
+    }
+    if (best < 0) {
+        rt::set_error("no candidate ran on every shape");
+        return RT_ERR_INFEASIBLE;
+    }
+    *best_index = best;
+    if (best_score) *best_score = (float)best_s;
+    return RT_OK;
+}
+
+int tuner_table_lookup(const rt_spec_entry* table, int32_t n_entries, const rt_params* general, const rt_shape* query,
+                       const rt_limits* limits, rt_params* out, int32_t* source)
+{
+    if (!query || !out || (n_entries > 0 && !table)) {
+        rt::set_error("tuner_table_lookup: NULL argument");
+        return RT_ERR_NULL;
+    }
+    rt_limits L;
+    if (!limits) {
+        int st = rt::current_limits(&L);
+        if (st != RT_OK) return st;
+        limits = &L;
+    }
+    return rt::table_lookup(table, n_entries, general, query, limits, out, source);
+}
+
+int rmsnorm_launch_auto(const rt_spec_entry* table, int32_t n_entries, const rt_params* general, const void* x,
+                        const void* r, const void* w, void* y, void* r_out, int64_t n_tokens, int64_t hidden, float eps,
+                        int dtype, void* stream, rt_params* used)
+{
+    if (n_tokens > 0 && (!x || !r || !w || !y || !r_out)) {
+        rt::set_error("a tensor pointer is NULL");
+        return RT_ERR_NULL;
+    }
+    rt_shape s;
+    s.n_tokens = n_tokens;
+    s.hidden = hidden;
+    s.dtype = dtype;
+    s.min_ptr_align = n_tokens > 0 ? rt::min_pointer_alignment(x, r, w, y, r_out) : 256;
+    rt_params theta;
+    int st = tuner_table_lookup(table, n_entries, general, &s, nullptr, &theta, nullptr);
+    if (st != RT_OK) return st;
+    if (used) *used = theta;
+    return rmsnorm_template_launch(&theta, x, r, w, y, r_out, n_tokens, hidden, eps, dtype, stream);
+}
+
+}  // extern "C"
