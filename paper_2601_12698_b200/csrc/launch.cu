@@ -217,22 +217,41 @@ int min_pointer_alignment(const void* a, const void* b, const void* c, const voi
     return (int)(bits & (~bits + 1));
 }
 
-// Registers per thread and static shared memory when no device can be asked: a plain model of what
-// the template needs (the row's fp32 sums, the loads in flight, addressing).
+// Registers per thread, static shared memory and spill size of every instance as ptxas reported them for
+// this build (table generated by the build script).  Used when no device can be asked; with a device the
+// runtime's own figures are used instead.
+struct InstanceResources {
+    int dtype, vec_bytes, stage, reduce, unroll, cap, regs, static_smem, spill_bytes;
+};
+static const InstanceResources kInstanceResources[] = {
+#include "instance_resources.inc"
+};
+static const InstanceResources* build_resources(const KernelEntry& k)
+{
+    static std::unordered_map<uint64_t, const InstanceResources*> index = [] {
+        std::unordered_map<uint64_t, const InstanceResources*> m;
+        for (const InstanceResources& r : kInstanceResources)
+            m[key_of(r.dtype, r.vec_bytes, r.stage, r.reduce, r.unroll, r.cap)] = &r;
+        return m;
+    }();
+    auto it = index.find(key_of(k.dtype, k.vec_bytes, k.stage, k.reduce, k.unroll, k.cap));
+    return it == index.end() ? nullptr : it->second;
+}
 static int model_regs(const KernelEntry& k, int elem_bytes)
 {
-    const int epv = k.vec_bytes / elem_bytes;
-    const int words = (k.vec_bytes + 3) / 4;
-    if (k.stage == kStageReg) return 28 + k.cap * epv + 2 * k.unroll * words;
-    return 36 + 2 * k.unroll * words + 2 * epv;
+    (void)elem_bytes;
+    const InstanceResources* r = build_resources(k);
+    return r ? r->regs : 255;
 }
 static int model_static_smem(const KernelEntry& k)
 {
-    int b = 1024;                                   // per-warp partials
-    if (k.reduce == kReduceSmem) b += 4096;         // halving tree
-    if (k.reduce == kReduceCluster) b += 256;       // cluster slots
-    if (k.stage == kStageSmemTma) b += 64;          // mbarriers
-    return b;
+    const InstanceResources* r = build_resources(k);
+    return r ? r->static_smem : 8192;
+}
+static int model_spill(const KernelEntry& k)
+{
+    const InstanceResources* r = build_resources(k);
+    return r ? r->spill_bytes : 0;
 }
 
 int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* plan)
@@ -367,6 +386,7 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
     } else {
         regs = model_regs(k, eb);
         static_smem = model_static_smem(k);
+        local_bytes = model_spill(k);
     }
     plan->static_smem_estimate = (size_t)static_smem;
     if (regs > L->max_regs_per_thread || local_bytes > 0) {
