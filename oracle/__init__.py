@@ -1,7 +1,8 @@
-"""CPU oracle for fused residual-add + RMSNorm (test infrastructure only).
+"""CPU oracles of the tuned kernels (test infrastructure only).
 
-Thin ctypes wrapper over ``add_rmsnorm_oracle.c``; all arithmetic is in the C
-file.  Only the tests, the smoke check and the benchmark's CPU-baseline leg may
+Thin ctypes wrapper over ``add_rmsnorm_oracle.c`` and ``silu_and_mul_oracle.c``;
+all arithmetic is in the C files (``selection.py`` holds the plain-Python oracle
+of the general-configuration choice).  Only the tests, the smoke check and the benchmark's CPU-baseline leg may
 import this package.  It imports nothing from the CUDA package and shares no
 code with it.
 
@@ -22,22 +23,29 @@ BF16, FP16, FP32 = 0, 1, 2
 DTYPE_NAMES = {BF16: "bf16", FP16: "fp16", FP32: "fp32"}
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_SRC = os.path.join(_HERE, "add_rmsnorm_oracle.c")
-_LIB = os.path.join(_HERE, "libadd_rmsnorm_oracle.so")
+SOURCES = ("add_rmsnorm_oracle.c", "silu_and_mul_oracle.c")
+HEADERS = ("number_formats.h",)
+_LIB = os.path.join(_HERE, "liboracle.so")
 _lock = threading.Lock()
 _lib = None
+
+
+def compile_sources(src_dir: str, out_path: str) -> str:
+    """gcc the oracle's C files found in `src_dir` into one shared library."""
+    cmd = ["gcc", "-O2", "-fno-fast-math", "-ffp-contract=off", "-std=c99", "-shared", "-fPIC", "-pthread",
+           "-I", src_dir, *[os.path.join(src_dir, f) for f in SOURCES], "-o", out_path, "-lm"]
+    subprocess.run(cmd, check=True)
+    return out_path
 
 
 def build(force: bool = False) -> str:
     """Compile the C oracle with gcc (no-op when the library is up to date)."""
     with _lock:
-        if (not force and os.path.exists(_LIB)
-                and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+        newest = max(os.path.getmtime(os.path.join(_HERE, f)) for f in SOURCES + HEADERS)
+        if not force and os.path.exists(_LIB) and os.path.getmtime(_LIB) >= newest:
             return _LIB
         tmp = _LIB + f".tmp{os.getpid()}"
-        cmd = ["gcc", "-O2", "-fno-fast-math", "-ffp-contract=off", "-std=c99", "-shared", "-fPIC",
-               "-pthread", _SRC, "-o", tmp, "-lm"]
-        subprocess.run(cmd, check=True)
+        compile_sources(_HERE, tmp)
         os.replace(tmp, _LIB)
         return _LIB
 
@@ -61,6 +69,8 @@ def _bind(path: str):
     lib.oracle_rel_compare32.argtypes = [vp, vp, i64, ctypes.c_double, ctypes.c_double,
                                          ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i64)]
     lib.oracle_rel_compare32.restype = None
+    lib.oracle_silu_and_mul.argtypes = [vp, vp, i64, i64, ctypes.c_int, ctypes.c_int]
+    lib.oracle_silu_and_mul.restype = ctypes.c_int
     return lib
 
 
@@ -133,6 +143,20 @@ def add_rmsnorm(x, r, w, eps: float, dtype: int | None = None, *, norm_from_roun
     if want_torch:
         return to_torch(y, dt), to_torch(r_out, dt)
     return y, r_out
+
+
+def silu_and_mul(x, dtype: int | None = None, *, threads: int = 1):
+    """out = silu(x[:, :d]) * x[:, d:] for x of shape [T, 2*d]; storage array or torch tensor like the input."""
+    want_torch = hasattr(x, "detach")
+    xs, dt = as_storage(x, dtype)
+    if xs.ndim != 2 or xs.shape[1] % 2:
+        raise ValueError("expected x of shape [T, 2*d]")
+    T, d = xs.shape[0], xs.shape[1] // 2
+    out = np.empty((T, d), dtype=xs.dtype)
+    rc = _load().oracle_silu_and_mul(xs.ctypes.data, out.ctypes.data, T, d, dt, int(threads))
+    if rc != 0:
+        raise RuntimeError(f"oracle_silu_and_mul failed with status {rc}")
+    return to_torch(out, dt) if want_torch else out
 
 
 def decode16(bits, dtype: int) -> np.ndarray:

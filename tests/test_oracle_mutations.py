@@ -2,7 +2,6 @@
 (on the CPU), build it, and check that the core pins reject it while the real source passes."""
 import math
 import os
-import subprocess
 
 import numpy as np
 import pytest
@@ -80,14 +79,20 @@ def _core_pins(o) -> bool:
     return True
 
 
-def _build(src_text: str, out_dir, name: str) -> str:
-    c = os.path.join(out_dir, name + ".c")
-    so = os.path.join(out_dir, name + ".so")
-    with open(c, "w") as f:
-        f.write(src_text)
-    subprocess.run(["gcc", "-O2", "-fno-fast-math", "-ffp-contract=off", "-std=c99", "-shared", "-fPIC",
-                    "-pthread", c, "-o", so, "-lm"], check=True)
-    return so
+def _build_mutant(oracle_lib, out_dir: str, old: str, new: str,
+                  targets=("add_rmsnorm_oracle.c", "number_formats.h")) -> str:
+    """Copy the oracle's C sources into out_dir with one replacement applied, and compile them."""
+    here = os.path.dirname(oracle_lib.__file__)
+    hits = 0
+    for f in oracle_lib.SOURCES + oracle_lib.HEADERS:
+        text = open(os.path.join(here, f)).read()
+        if f in targets:
+            hits += text.count(old)
+            text = text.replace(old, new)
+        with open(os.path.join(out_dir, f), "w") as out:
+            out.write(text)
+    assert hits >= 1, f"mutation anchor not found: {old}"
+    return oracle_lib.compile_sources(out_dir, os.path.join(out_dir, "mutant.so"))
 
 
 def test_real_oracle_passes_core_pins(oracle_lib):
@@ -97,12 +102,59 @@ def test_real_oracle_passes_core_pins(oracle_lib):
 @pytest.mark.parametrize("name", sorted(MUTATIONS))
 def test_planted_mistake_is_caught(oracle_lib, tmp_path, name):
     old, new = MUTATIONS[name]
-    src = open(os.path.join(os.path.dirname(oracle_lib.__file__), "add_rmsnorm_oracle.c")).read()
-    assert src.count(old) >= 1, f"mutation anchor not found: {old}"
-    so = _build(src.replace(old, new), str(tmp_path), name)
+    so = _build_mutant(oracle_lib, str(tmp_path), old, new)
     saved = oracle_lib._lib
     try:
         oracle_lib._lib = oracle_lib._bind(so)
         assert not _core_pins(oracle_lib), f"pins did not notice: {name}"
+    finally:
+        oracle_lib._lib = saved
+
+
+SILU_MUTATIONS = {
+    "exp_sign": ("exp(-g)", "exp(g)"),
+    "value_dropped": ("(1.0 + exp(-g)) * u", "(1.0 + exp(-g))"),
+    "halves_swapped": ("const double v = g / (1.0 + exp(-g)) * u;", "const double v = u / (1.0 + exp(-u)) * g;"),
+    "value_from_gate_half": ("t * 2 * d + d + j", "t * 2 * d + j"),
+    "input_row_stride": ("load_elem(job->x, t * 2 * d + j, job->dtype)", "load_elem(job->x, t * d + j, job->dtype)"),
+    "sigmoid_denominator": ("(1.0 + exp(-g))", "(2.0 + exp(-g))"),
+    "rounded_through_binary32": ("encode16(v, job->dtype", "encode16((double)(float)(v * 1.00000003), job->dtype"),
+}
+
+
+def _silu_pins(o) -> bool:
+    try:
+        for dtype, td in ((0, torch.bfloat16), (1, torch.float16)):
+            x = torch.tensor([[50.0, 0.0, 1.5, -2.0, 2.0, 7.0, -3.0, 0.5],
+                              [-1.0, 3.0, 60.0, 0.25, 4.0, 1.0, 0.5, -8.0]], dtype=torch.float64).to(td)
+            out = o.silu_and_mul(x)
+            xd = x.double()
+            want = torch.nn.functional.silu(xd[:, :4]) * xd[:, 4:]
+            if not np.array_equal(out.view(torch.int16).numpy().view(np.uint16), refnum.round_array(want.numpy(), dtype)):
+                return False
+            g = np.random.Generator(np.random.Philox(key=[61, dtype]))
+            x = torch.from_numpy(g.standard_normal((6, 600)) * 3).to(td)
+            xd = x.double()
+            want = torch.nn.functional.silu(xd[:, :300]) * xd[:, 300:]
+            got = o.silu_and_mul(x).view(torch.int16).numpy().view(np.uint16)
+            if np.count_nonzero(got != refnum.round_array(want.numpy(), dtype)) > 1:
+                return False
+    except Exception:
+        return False
+    return True
+
+
+def test_real_silu_oracle_passes_its_pins(oracle_lib):
+    assert _silu_pins(oracle_lib)
+
+
+@pytest.mark.parametrize("name", sorted(SILU_MUTATIONS))
+def test_planted_silu_mistake_is_caught(oracle_lib, tmp_path, name):
+    old, new = SILU_MUTATIONS[name]
+    so = _build_mutant(oracle_lib, str(tmp_path), old, new, targets=("silu_and_mul_oracle.c",))
+    saved = oracle_lib._lib
+    try:
+        oracle_lib._lib = oracle_lib._bind(so)
+        assert not _silu_pins(oracle_lib), f"pins did not notice: {name}"
     finally:
         oracle_lib._lib = saved
