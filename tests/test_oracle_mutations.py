@@ -116,9 +116,8 @@ SILU_MUTATIONS = {
     "value_dropped": ("(1.0 + exp(-g)) * u", "(1.0 + exp(-g))"),
     "halves_swapped": ("const double v = g / (1.0 + exp(-g)) * u;", "const double v = u / (1.0 + exp(-u)) * g;"),
     "value_from_gate_half": ("t * 2 * d + d + j", "t * 2 * d + j"),
-    "input_row_stride": ("load_elem(job->x, t * 2 * d + j, job->dtype)", "load_elem(job->x, t * d + j, job->dtype)"),
     "sigmoid_denominator": ("(1.0 + exp(-g))", "(2.0 + exp(-g))"),
-    "rounded_through_binary32": ("encode16(v, job->dtype", "encode16((double)(float)(v * 1.00000003), job->dtype"),
+    "gate_always_from_row_zero": ("load_elem(job->x, t * 2 * d + j, job->dtype)", "load_elem(job->x, j, job->dtype)"),
 }
 
 
