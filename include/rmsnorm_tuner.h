@@ -46,6 +46,12 @@ extern "C" {
 
 typedef enum { RT_BF16 = 0, RT_FP16 = 1, RT_FP32 = 2 } rt_dtype;
 
+/* The kernels that have a template in this library (the paper tunes three serving kernels, "Kernels"). */
+typedef enum {
+    RT_OP_ADD_RMSNORM = 0,  /* fused residual-add + RMSNorm: the operator described above */
+    RT_OP_SILU_AND_MUL = 1  /* out[t,j] = silu(x[t,j]) * x[t,d+j] for x of shape [n_tokens, 2*d] */
+} rt_op;
+
 /* Where a row lives between the two passes over it. */
 typedef enum {
     RT_STAGE_REG = 0,      /* ld.global vectors straight into registers, row kept as fp32 registers */
@@ -74,9 +80,11 @@ typedef struct {
 
 typedef struct {
     int64_t n_tokens;
-    int64_t hidden;
+    int64_t hidden;        /* row width of the OUTPUT: hidden size, or d for silu_and_mul */
     int32_t dtype;         /* rt_dtype */
-    int32_t min_ptr_align; /* largest power of two (bytes, <= 256) dividing all five base addresses */
+    int32_t min_ptr_align; /* largest power of two (bytes, <= 256) dividing all base addresses */
+    int32_t op;            /* rt_op; 0 = add_rmsnorm */
+    int32_t reserved;
 } rt_shape;
 
 /* r(h): the resource upper bounds the feasible region is derived from. */
@@ -124,6 +132,8 @@ typedef struct {
     int32_t reserved;
 } rt_budget;
 
+/* For silu_and_mul: x is the [n_tokens, 2*d] input (ring stride 2 * ring_stride_bytes), y the output,
+ * y_ref its reference; r, w, r_out, r_ref are unused and may be NULL. */
 typedef struct {
     const void* x;     /* device, [ring_sets][n_tokens, hidden] */
     const void* r;     /* device */
@@ -211,6 +221,18 @@ int rmsnorm_template_run_host(const rt_params* p, const void* x_host, const void
                               int64_t hidden, float eps, int dtype, void* workspace,
                               int64_t workspace_bytes, int64_t chunk_tokens, void* stream);
 int64_t rmsnorm_host_workspace_bytes(int64_t n_tokens, int64_t hidden, int dtype, int64_t chunk_tokens);
+
+/*
+ * The gated activation silu_and_mul as an instance of its own template (second kernel of the paper's
+ * "Kernels" list; axes: threads per row, rows per CTA, vec_bytes, unroll, stage = registers or TMA bulk;
+ * it has no reduction: reduce must be RT_REDUCE_SHFL and cluster_size 1).
+ *   x    device, [n_tokens, 2*d]: gate in the first d columns of a row, value in the last d.
+ *   out  device, [n_tokens, d];  out = round_dtype(silu(gate) * value), silu(g) = g / (1 + exp(-g)),
+ *        computed in fp32 (ex2.approx and rcp.approx: 2 ulp of a 16-bit type, 1e-5 relative in fp32).
+ * Asynchronous on `stream`, allocates nothing; infeasible theta is refused without launching.
+ */
+int silu_and_mul_template_launch(const rt_params* p, const void* x, void* out, int64_t n_tokens, int64_t d,
+                                 int dtype, void* stream);
 
 /* ---- 2. the feasible region ----------------------------------------------------- */
 
@@ -373,6 +395,8 @@ int rt_device_status(void);
 int32_t rt_num_kernel_instances(void);
 int rt_kernel_instance(int32_t i, int32_t* dtype, int32_t* vec_bytes, int32_t* stage, int32_t* reduce,
                        int32_t* unroll, int32_t* reg_vectors);
+/* The rt_op the i-th instance belongs to (-1 when i is out of range). */
+int32_t rt_kernel_instance_op(int32_t i);
 /* Kernel launches issued by this library in this process since load (all entry points). */
 int64_t rt_launch_count(void);
 /* Frees what the library allocated on the device.  Safe to call more than once. */

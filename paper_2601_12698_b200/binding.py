@@ -15,6 +15,7 @@ LIB_PATH = os.path.join(_HERE, "librmsnorm_tuner.so")
 HEADER_PATH = os.path.join(os.path.dirname(_HERE), "include", "rmsnorm_tuner.h")
 
 RT_BF16, RT_FP16, RT_FP32 = 0, 1, 2
+RT_OP_ADD_RMSNORM, RT_OP_SILU_AND_MUL = 0, 1
 RT_STAGE_REG, RT_STAGE_SMEM_LDG, RT_STAGE_SMEM_TMA = 0, 1, 2
 RT_REDUCE_SHFL, RT_REDUCE_SMEM, RT_REDUCE_CLUSTER = 0, 1, 2
 RT_PRUNE_IDLE_THREADS, RT_PRUNE_DUPLICATES, RT_PRUNE_CLUSTER_WAVES, RT_PRUNE_IDLE_ROWS = 1, 2, 4, 8
@@ -51,7 +52,8 @@ def make_params(threads_per_row=256, rows_per_cta=1, vec_bytes=16, unroll=1, sta
 
 
 class rt_shape(Structure):
-    _fields_ = [("n_tokens", c_int64), ("hidden", c_int64), ("dtype", c_int32), ("min_ptr_align", c_int32)]
+    _fields_ = [("n_tokens", c_int64), ("hidden", c_int64), ("dtype", c_int32), ("min_ptr_align", c_int32),
+                ("op", c_int32), ("reserved", c_int32)]
 
 
 class rt_limits(Structure):
@@ -103,6 +105,7 @@ rt_evaluate_fn = ctypes.CFUNCTYPE(c_double, POINTER(rt_params), c_void_p)
 _SIGNATURES = {
     "rmsnorm_template_launch": (c_int, [POINTER(rt_params), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                         c_int64, c_int64, c_float, c_int, c_void_p]),
+    "silu_and_mul_template_launch": (c_int, [POINTER(rt_params), c_void_p, c_void_p, c_int64, c_int64, c_int, c_void_p]),
     "rmsnorm_template_run_host": (c_int, [POINTER(rt_params), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                           c_int64, c_int64, c_float, c_int, c_void_p, c_int64, c_int64, c_void_p]),
     "rmsnorm_host_workspace_bytes": (c_int64, [c_int64, c_int64, c_int, c_int64]),
@@ -136,6 +139,7 @@ _SIGNATURES = {
     "rt_device_status": (c_int, []),
     "rt_num_kernel_instances": (c_int32, []),
     "rt_kernel_instance": (c_int, [c_int32] + [POINTER(c_int32)] * 6),
+    "rt_kernel_instance_op": (c_int32, [c_int32]),
     "rt_launch_count": (c_int64, []),
     "rt_shutdown": (None, []),
 }
@@ -182,9 +186,10 @@ def _ptr_align(*tensors) -> int:
     return bits & -bits
 
 
-def shape_of(n_tokens: int, hidden: int, dtype, min_ptr_align: int = 256) -> rt_shape:
+def shape_of(n_tokens: int, hidden: int, dtype, min_ptr_align: int = 256, op: int = RT_OP_ADD_RMSNORM) -> rt_shape:
+    """hidden is the output row width (d for silu_and_mul)."""
     code = DTYPE_CODES[dtype] if isinstance(dtype, str) else int(dtype)
-    return rt_shape(n_tokens, hidden, code, min_ptr_align)
+    return rt_shape(n_tokens, hidden, code, min_ptr_align, op, 0)
 
 
 def sm100_nominal_limits() -> rt_limits:
@@ -214,6 +219,17 @@ def rmsnorm_template_launch(params: rt_params, x, r, w, y, r_out, eps: float, st
     _check(lib.rmsnorm_template_launch(byref(params), x.data_ptr(), r.data_ptr(), w.data_ptr(), y.data_ptr(),
                                        r_out.data_ptr(), n_tokens, hidden, eps, _dtype_code(x), _stream_ptr(stream)),
            "rmsnorm_template_launch")
+
+
+def silu_and_mul_template_launch(params: rt_params, x, out, stream=None) -> None:
+    """out[t, j] = silu(x[t, j]) * x[t, d + j] on device tensors x [T, 2d] and out [T, d] (asynchronous)."""
+    if not (x.is_cuda and out.is_cuda and x.is_contiguous() and out.is_contiguous()):
+        raise ValueError("silu_and_mul_template_launch takes contiguous CUDA tensors")
+    n_tokens, d = out.shape
+    if x.shape != (n_tokens, 2 * d) or x.dtype != out.dtype:
+        raise ValueError("x must be [n_tokens, 2*d] of the output's dtype")
+    _check(lib.silu_and_mul_template_launch(byref(params), x.data_ptr(), out.data_ptr(), n_tokens, d, _dtype_code(x),
+                                            _stream_ptr(stream)), "silu_and_mul_template_launch")
 
 
 def rmsnorm_host_workspace_bytes(n_tokens: int, hidden: int, dtype, chunk_tokens: int = 0) -> int:
@@ -291,10 +307,11 @@ def make_budget(max_evals=64, warmup=20, iters=100, repeats=3, top_k=5, strategy
 def make_workspace(x, r, w, y, r_out, y_ref, r_ref, eps: float, n_ref_tokens: int | None = None, ring_sets: int = 1,
                    ring_stride_bytes: int = 0, stream=None) -> rt_workspace:
     """Device tensors for the tuner.  With ring_sets > 1, x, r, y, r_out are [ring_sets, T, H] and the
-    references cover set 0."""
+    references cover set 0.  For silu_and_mul pass r = w = r_out = r_ref = None."""
     T = x.shape[-2]
-    return rt_workspace(x.data_ptr(), r.data_ptr(), w.data_ptr(), y.data_ptr(), r_out.data_ptr(), y_ref.data_ptr(),
-                        r_ref.data_ptr(), n_ref_tokens if n_ref_tokens is not None else T, ring_stride_bytes,
+    ptr = lambda t: t.data_ptr() if t is not None else None
+    return rt_workspace(ptr(x), ptr(r), ptr(w), ptr(y), ptr(r_out), ptr(y_ref), ptr(r_ref),
+                        n_ref_tokens if n_ref_tokens is not None else T, ring_stride_bytes,
                         ring_sets, eps, _stream_ptr(stream))
 
 
@@ -401,7 +418,8 @@ class SpecTable:
         names = {v: k for k, v in DTYPE_CODES.items()}
         return {"device": self.device_name, "general": self.general.as_dict() if self.general else None,
                 "specialised": [{"dtype": names[s.dtype], "n_tokens": int(s.n_tokens), "hidden": int(s.hidden),
-                                 "theta": t.as_dict(), "us": round(float(us), 3)} for s, t, us in self.entries]}
+                                 "op": int(s.op), "theta": t.as_dict(), "us": round(float(us), 3)}
+                                for s, t, us in self.entries]}
 
     @classmethod
     def default(cls) -> "SpecTable":
@@ -414,7 +432,7 @@ class SpecTable:
     def from_json(cls, d: dict) -> "SpecTable":
         fields = [k for k, _ in rt_params._fields_]
         mk = lambda t: rt_params(*[int(t[k]) for k in fields])
-        entries = [(shape_of(e["n_tokens"], e["hidden"], e["dtype"]), mk(e["theta"]), float(e["us"]))
+        entries = [(shape_of(e["n_tokens"], e["hidden"], e["dtype"], op=int(e.get("op", 0))), mk(e["theta"]), float(e["us"]))
                    for e in d.get("specialised", [])]
         return cls(entries, mk(d["general"]) if d.get("general") else None, d.get("device", ""))
 
@@ -433,6 +451,7 @@ def kernel_instances() -> list[dict]:
     for i in range(lib.rt_num_kernel_instances()):
         _check(lib.rt_kernel_instance(i, *[byref(v) for v in vals]), "rt_kernel_instance")
         out.append(dict(zip(("dtype", "vec_bytes", "stage", "reduce", "unroll", "reg_vectors"), (v.value for v in vals))))
+        out[-1]["op"] = int(lib.rt_kernel_instance_op(i))
     return out
 
 

@@ -52,9 +52,12 @@ std::vector<rt_params> raw_grid(const rt_shape& s)
 {
     std::vector<rt_params> out;
     const std::vector<int> vecs = vec_levels(s);
+    // silu_and_mul has no reduction and no ld.global -> shared stage: its grid is the remaining axes
+    const bool is_silu = s.op == RT_OP_SILU_AND_MUL;
     for (int stage = 0; stage < 3; ++stage)
         for (const Mode& m : kReduceModes)
-            for (int vb : vecs)
+            for (int vb : vecs) {
+                if (is_silu && (stage == RT_STAGE_SMEM_LDG || m.reduce != RT_REDUCE_SHFL)) continue;
                 for (int tpr : kTprLevels)
                     for (int rpc : kRpcLevels)
                         for (int u : kUnrollLevels) {
@@ -68,6 +71,7 @@ std::vector<rt_params> raw_grid(const rt_shape& s)
                             p.cluster_size = m.cluster;
                             out.push_back(p);
                         }
+            }
     return out;
 }
 

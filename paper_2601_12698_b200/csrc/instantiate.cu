@@ -1,13 +1,16 @@
 // One instantiation unit of the kernel template.  Compiled once per line of instance_units.inc with
 //   -DRT_UNIT_NAME=<name> -DRT_UNIT_T=<element type> -DRT_UNIT_DTYPE=<0|1|2> -DRT_UNIT_VB=<bytes>
-//   -DRT_UNIT_GROUP=<0 register stage | 1 shared-memory stages | 2 narrow fall-back>
+//   -DRT_UNIT_GROUP=<0 register stage | 1 shared-memory stages | 2 narrow fall-back | 3 silu_and_mul>
 //   -DRT_UNIT_REDUCE=<0|1|2>   (register-stage units only)
 //
 // Instance lists.  Register stage: CAP (row vectors kept per thread) in {1,2,4,8,16,32} while the row
 // stays within 128 fp32 registers per thread, unroll U in {1,2,4} with U <= CAP.  Shared-memory
 // stages: U in {1,2,4}, all three reductions.  Narrow fall-back (4- and 2-byte vectors, for rows whose
 // byte length is not a multiple of 8): register stage, shuffle reduction, U in {1,4}.
+// silu_and_mul (one unit per element type, every vector width): stages register and TMA bulk for 16- and
+// 8-byte vectors with U in {1,2,4}; register stage with U in {1,4} for the 4- and 2-byte fall-back.
 #include "add_rmsnorm_kernel.cuh"
+#include "silu_and_mul_kernel.cuh"
 #include "tuner_internal.h"
 
 namespace {
@@ -22,12 +25,26 @@ template <int ST, int RD, int U, int CAP>
 rt::KernelEntry entry()
 {
     if constexpr (ST == rt::kStageReg && CAP * kEPV > kMaxRowRegisters) {
-        return rt::KernelEntry{kDtype, kVB, ST, RD, U, CAP, nullptr};  // not instantiated
+        return rt::KernelEntry{RT_OP_ADD_RMSNORM, kDtype, kVB, ST, RD, U, CAP, nullptr};  // not instantiated
     } else {
-        return rt::KernelEntry{kDtype, kVB, ST, RD, U, ST == rt::kStageReg ? CAP : 0,
+        return rt::KernelEntry{RT_OP_ADD_RMSNORM, kDtype, kVB, ST, RD, U, ST == rt::kStageReg ? CAP : 0,
                                (const void*)&rt::add_rmsnorm_kernel<T, kVB, ST, RD, U, CAP>};
     }
 }
+
+template <int VB, int ST, int U>
+rt::KernelEntry silu_entry()
+{
+    if constexpr (VB < (int)sizeof(T)) {
+        return rt::KernelEntry{RT_OP_SILU_AND_MUL, kDtype, VB, ST, 0, U, 0, nullptr};  // narrower than an element
+    } else {
+        return rt::KernelEntry{RT_OP_SILU_AND_MUL, kDtype, VB, ST, 0, U, 0,
+                               (const void*)&rt::silu_and_mul_kernel<T, VB, ST, U>};
+    }
+}
+#define RT_SILU_WIDE(VB) \
+    silu_entry<VB, 0, 1>(), silu_entry<VB, 0, 2>(), silu_entry<VB, 0, 4>(), silu_entry<VB, 2, 1>(), \
+    silu_entry<VB, 2, 2>(), silu_entry<VB, 2, 4>()
 
 #define RT_REG_LIST(RD)                                                                                   \
     entry<0, RD, 1, 1>(), entry<0, RD, 1, 2>(), entry<0, RD, 2, 2>(), entry<0, RD, 1, 4>(), entry<0, RD, 2, 4>(), \
@@ -44,6 +61,9 @@ std::vector<rt::KernelEntry> build_entries()
         RT_REG_LIST(RT_UNIT_REDUCE)
 #elif RT_UNIT_GROUP == 1
         RT_SMEM_LIST(1), RT_SMEM_LIST(2)
+#elif RT_UNIT_GROUP == 3
+        RT_SILU_WIDE(16), RT_SILU_WIDE(8), silu_entry<4, 0, 1>(), silu_entry<4, 0, 4>(), silu_entry<2, 0, 1>(),
+        silu_entry<2, 0, 4>()
 #else
         entry<0, 0, 1, 1>(), entry<0, 0, 1, 2>(), entry<0, 0, 1, 4>(), entry<0, 0, 4, 4>(), entry<0, 0, 1, 8>(),
         entry<0, 0, 4, 8>(), entry<0, 0, 1, 16>(), entry<0, 0, 4, 16>(), entry<0, 0, 1, 32>(), entry<0, 0, 4, 32>()

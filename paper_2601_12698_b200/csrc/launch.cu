@@ -9,6 +9,7 @@
 #include <unordered_map>
 
 #include "add_rmsnorm_kernel.cuh"
+#include "silu_and_mul_kernel.cuh"
 #include "tuner_internal.h"
 
 // Each instantiation unit exports its slice of the instance table.
@@ -37,9 +38,9 @@ struct DeviceCache {
 };
 DeviceCache g_dev[kMaxDevices];
 
-uint64_t key_of(int dtype, int vb, int stage, int reduce, int unroll, int cap)
+uint64_t key_of(int op, int dtype, int vb, int stage, int reduce, int unroll, int cap)
 {
-    return ((uint64_t)dtype << 40) | ((uint64_t)vb << 32) | ((uint64_t)stage << 28) | ((uint64_t)reduce << 24) |
+    return ((uint64_t)op << 48) | ((uint64_t)dtype << 40) | ((uint64_t)vb << 32) | ((uint64_t)stage << 28) | ((uint64_t)reduce << 24) |
            ((uint64_t)unroll << 16) | (uint64_t)cap;
 }
 
@@ -57,7 +58,7 @@ struct Registry {
 #undef RT_DECLARE_SLICE
         for (int i = 0; i < (int)entries.size(); ++i) {
             const KernelEntry& e = entries[i];
-            index[key_of(e.dtype, e.vec_bytes, e.stage, e.reduce, e.unroll, e.cap)] = i;
+            index[key_of(e.op, e.dtype, e.vec_bytes, e.stage, e.reduce, e.unroll, e.cap)] = i;
         }
     }
 };
@@ -102,9 +103,9 @@ void count_launch(int64_t n) { g_launches.fetch_add(n, std::memory_order_relaxed
 
 const std::vector<KernelEntry>& registry() { return reg().entries; }
 
-int find_kernel(int dtype, int vb, int stage, int reduce, int unroll, int cap)
+int find_kernel(int op, int dtype, int vb, int stage, int reduce, int unroll, int cap)
 {
-    auto it = reg().index.find(key_of(dtype, vb, stage, reduce, unroll, cap));
+    auto it = reg().index.find(key_of(op, dtype, vb, stage, reduce, unroll, cap));
     return it == reg().index.end() ? -1 : it->second;
 }
 
@@ -221,7 +222,7 @@ int min_pointer_alignment(const void* a, const void* b, const void* c, const voi
 // this build (table generated by the build script).  Used when no device can be asked; with a device the
 // runtime's own figures are used instead.
 struct InstanceResources {
-    int dtype, vec_bytes, stage, reduce, unroll, cap, regs, static_smem, spill_bytes;
+    int op, dtype, vec_bytes, stage, reduce, unroll, cap, regs, static_smem, spill_bytes;
 };
 static const InstanceResources kInstanceResources[] = {
 #include "instance_resources.inc"
@@ -231,10 +232,10 @@ static const InstanceResources* build_resources(const KernelEntry& k)
     static std::unordered_map<uint64_t, const InstanceResources*> index = [] {
         std::unordered_map<uint64_t, const InstanceResources*> m;
         for (const InstanceResources& r : kInstanceResources)
-            m[key_of(r.dtype, r.vec_bytes, r.stage, r.reduce, r.unroll, r.cap)] = &r;
+            m[key_of(r.op, r.dtype, r.vec_bytes, r.stage, r.reduce, r.unroll, r.cap)] = &r;
         return m;
     }();
-    auto it = index.find(key_of(k.dtype, k.vec_bytes, k.stage, k.reduce, k.unroll, k.cap));
+    auto it = index.find(key_of(k.op, k.dtype, k.vec_bytes, k.stage, k.reduce, k.unroll, k.cap));
     return it == index.end() ? nullptr : it->second;
 }
 static int model_regs(const KernelEntry& k, int elem_bytes)
@@ -266,8 +267,15 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
         plan->reject_reason = kRejectArgs;
         return RT_ERR_DTYPE;
     }
+    if (s->op != RT_OP_ADD_RMSNORM && s->op != RT_OP_SILU_AND_MUL) {
+        set_error("op %d is not a kernel of this library", s->op);
+        plan->reject_reason = kRejectArgs;
+        return RT_ERR_SHAPE;
+    }
+    plan->op = s->op;
+    const bool is_silu = s->op == RT_OP_SILU_AND_MUL;
     const int eb = elem_bytes_of(s->dtype);
-    if (s->n_tokens < 0 || s->hidden <= 0 || s->hidden * eb >= (int64_t)1 << 31) {
+    if (s->n_tokens < 0 || s->hidden <= 0 || s->hidden * eb * (is_silu ? 2 : 1) >= (int64_t)1 << 31) {
         set_error("shape n_tokens=%lld hidden=%lld is out of range", (long long)s->n_tokens, (long long)s->hidden);
         plan->reject_reason = kRejectArgs;
         return RT_ERR_SHAPE;
@@ -303,6 +311,12 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
         plan->reject_reason = kRejectArgs;
         return RT_ERR_INFEASIBLE;
     }
+    if (is_silu && (p->reduce != RT_REDUCE_SHFL || p->cluster_size != 1 || p->stage == RT_STAGE_SMEM_LDG)) {
+        set_error("silu_and_mul has no reduction and no ld.global->shared stage (reduce=%d cluster=%d stage=%d)",
+                  p->reduce, p->cluster_size, p->stage);
+        plan->reject_reason = kRejectArgs;
+        return RT_ERR_INFEASIBLE;
+    }
     const int C = p->cluster_size;
     if (p->reduce == RT_REDUCE_CLUSTER) {
         if (!(C == 2 || C == 4 || C == 8) || C > L->max_cluster_size) {
@@ -326,6 +340,7 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
         plan->reject_reason = kRejectAlign;
         return RT_ERR_ALIGN;
     }
+    // silu_and_mul: an input row is 2 * row_bytes long, so 16-byte output rows give 16-byte input rows
     if (p->stage == RT_STAGE_SMEM_TMA && (row_bytes % 16 != 0 || s->min_ptr_align < 16)) {
         set_error("TMA bulk copies need 16-byte aligned rows and pointers (row %lld bytes, pointers %d)",
                   (long long)row_bytes, s->min_ptr_align);
@@ -350,21 +365,21 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
     }
 
     int cap = 0, unroll = p->unroll;
-    if (p->stage == RT_STAGE_REG) {
+    if (p->stage == RT_STAGE_REG && !is_silu) {
         cap = next_pow2(plan->vec_per_thread);
         if (unroll > cap) unroll = cap;
     }
     plan->cap = cap;
     plan->unroll_eff = unroll;
-    plan->kernel_index = find_kernel(s->dtype, vb, p->stage, p->reduce, unroll, cap);
+    plan->kernel_index = find_kernel(s->op, s->dtype, vb, p->stage, p->reduce, unroll, cap);
     if (plan->kernel_index < 0) {
-        if (p->stage == RT_STAGE_REG)
+        if (p->stage == RT_STAGE_REG && !is_silu)
             set_error("a row slice of %d vectors over %d threads needs %d vectors per thread: no register-stage "
                       "instance that large (register budget)", slice, tpr, cap);
         else
             set_error("no compiled instance for dtype=%d vec=%d stage=%d reduce=%d unroll=%d", s->dtype, vb, p->stage,
                       p->reduce, unroll);
-        plan->reject_reason = p->stage == RT_STAGE_REG ? kRejectRegisters : kRejectArgs;
+        plan->reject_reason = (p->stage == RT_STAGE_REG && !is_silu) ? kRejectRegisters : kRejectArgs;
         return RT_ERR_INFEASIBLE;
     }
     const KernelEntry& k = registry()[plan->kernel_index];
@@ -467,10 +482,48 @@ int plan_occupancy(const Plan& plan, const rt_limits* L, int* regs_per_thread)
     return (int)blocks;
 }
 
+int launch_silu_plan(const Plan& plan, const void* x, void* out, int64_t n_tokens, cudaStream_t stream)
+{
+    if (n_tokens == 0) return RT_OK;
+    if (plan.op != RT_OP_SILU_AND_MUL) {
+        set_error("plan belongs to another kernel");
+        return RT_ERR_INFEASIBLE;
+    }
+    const KernelEntry& k = registry()[plan.kernel_index];
+    int st = ensure_dynamic_smem(plan.kernel_index, plan.dyn_smem);
+    if (st != RT_OK) return st;
+    SiluArgs a;
+    a.x = x;
+    a.out = out;
+    a.n_tokens = n_tokens;
+    a.nvec = plan.nvec;
+    a.status = device_status_word();
+    if (!a.status) return RT_ERR_CUDA;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(plan.grid_x, 1, 1);
+    cfg.blockDim = dim3(plan.block_x, plan.block_y, 1);
+    cfg.dynamicSmemBytes = plan.dyn_smem;
+    cfg.stream = stream;
+    void* params[] = {&a};
+    cudaError_t e = cudaLaunchKernelExC(&cfg, k.fn, params);
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        set_error("kernel launch failed: %s", cudaGetErrorString(e));
+        return RT_ERR_CUDA;
+    }
+    count_launch();
+    return RT_OK;
+}
+
 int launch_plan(const Plan& plan, const void* x, const void* r, const void* w, void* y, void* r_out,
                 int64_t n_tokens, int64_t hidden, float eps, cudaStream_t stream)
 {
     if (n_tokens == 0) return RT_OK;
+    if (plan.op != RT_OP_ADD_RMSNORM) {
+        set_error("plan belongs to another kernel");
+        return RT_ERR_INFEASIBLE;
+    }
     const KernelEntry& k = registry()[plan.kernel_index];
     int st = ensure_dynamic_smem(plan.kernel_index, plan.dyn_smem);
     if (st != RT_OK) return st;
@@ -535,10 +588,39 @@ int rmsnorm_template_launch(const rt_params* p, const void* x, const void* r, co
     s.hidden = hidden;
     s.dtype = dtype;
     s.min_ptr_align = n_tokens > 0 ? rt::min_pointer_alignment(x, r, w, y, r_out) : 256;
+    s.op = RT_OP_ADD_RMSNORM;
+    s.reserved = 0;
     rt::Plan plan;
     st = rt::make_plan(&s, p, &L, &plan);
     if (st != RT_OK) return st;
     return rt::launch_plan(plan, x, r, w, y, r_out, n_tokens, hidden, eps, (cudaStream_t)stream);
+}
+
+int silu_and_mul_template_launch(const rt_params* p, const void* x, void* out, int64_t n_tokens, int64_t d, int dtype,
+                                 void* stream)
+{
+    if (!p) {
+        rt::set_error("params is NULL");
+        return RT_ERR_NULL;
+    }
+    if (n_tokens > 0 && (!x || !out)) {
+        rt::set_error("a tensor pointer is NULL");
+        return RT_ERR_NULL;
+    }
+    rt_limits L;
+    int st = rt::current_limits(&L);
+    if (st != RT_OK) return st;
+    rt_shape s;
+    s.n_tokens = n_tokens;
+    s.hidden = d;
+    s.dtype = dtype;
+    s.min_ptr_align = n_tokens > 0 ? rt::min_pointer_alignment(x, out, x, out, x) : 256;
+    s.op = RT_OP_SILU_AND_MUL;
+    s.reserved = 0;
+    rt::Plan plan;
+    st = rt::make_plan(&s, p, &L, &plan);
+    if (st != RT_OK) return st;
+    return rt::launch_silu_plan(plan, x, out, n_tokens, (cudaStream_t)stream);
 }
 
 int rt_query_limits(rt_limits* out)
@@ -634,6 +716,12 @@ int rt_kernel_instance(int32_t i, int32_t* dtype, int32_t* vec_bytes, int32_t* s
     if (unroll) *unroll = k.unroll;
     if (reg_vectors) *reg_vectors = k.cap;
     return RT_OK;
+}
+
+int32_t rt_kernel_instance_op(int32_t i)
+{
+    if (i < 0 || i >= (int32_t)rt::registry().size()) return -1;
+    return rt::registry()[i].op;
 }
 
 int64_t rt_launch_count(void) { return rt::g_launches.load(); }

@@ -267,18 +267,22 @@ struct DeviceEvaluator : Evaluator {
         Scratch* sc;
         st = get_scratch(&sc);
         if (st != RT_OK) return st;
+        const bool is_silu = shape.op == RT_OP_SILU_AND_MUL;
         RT_CUDA_OK(cudaMemsetAsync(ws.y, 0xFF, set_bytes, stream));
-        RT_CUDA_OK(cudaMemsetAsync(ws.r_out, 0xFF, set_bytes, stream));
+        if (!is_silu) RT_CUDA_OK(cudaMemsetAsync(ws.r_out, 0xFF, set_bytes, stream));
         RT_CUDA_OK(cudaMemsetAsync(sc->dev, 0, 2 * sizeof(CompareAcc), stream));
-        st = launch_plan(plan, ws.x, ws.r, ws.w, ws.y, ws.r_out, shape.n_tokens, shape.hidden, ws.eps, stream);
+        st = is_silu ? launch_silu_plan(plan, ws.x, ws.y, shape.n_tokens, stream)
+                     : launch_plan(plan, ws.x, ws.r, ws.w, ws.y, ws.r_out, shape.n_tokens, shape.hidden, ws.eps, stream);
         if (st != RT_OK) {
             rec->status = st;
             return RT_OK;
         }
         const int y_mode = shape.dtype == RT_FP32 ? RT_CMP_REL32 : RT_CMP_ULP16;
         const double y_tol = shape.dtype == RT_FP32 ? 1e-5 : 2.0;
-        st = enqueue_compare(ws.r_out, ws.r_ref, n_ref * shape.hidden, shape.dtype, RT_CMP_BITS, 0.0, sc->dev, stream);
-        if (st != RT_OK) return st;
+        if (!is_silu) {
+            st = enqueue_compare(ws.r_out, ws.r_ref, n_ref * shape.hidden, shape.dtype, RT_CMP_BITS, 0.0, sc->dev, stream);
+            if (st != RT_OK) return st;
+        }
         st = enqueue_compare(ws.y, ws.y_ref, n_ref * shape.hidden, shape.dtype, y_mode, y_tol, sc->dev + 1, stream);
         if (st != RT_OK) return st;
         (void)ref_bytes;
@@ -312,6 +316,8 @@ struct DeviceEvaluator : Evaluator {
         const int sets = ws.ring_sets > 0 ? ws.ring_sets : 1;
         auto launch_set = [&](int k) {
             const size_t off = (size_t)(k % sets) * (size_t)ws.ring_stride_bytes;
+            if (is_silu)  // the input rows are twice as long as the output rows
+                return launch_silu_plan(plan, (const char*)ws.x + 2 * off, (char*)ws.y + off, shape.n_tokens, stream);
             return launch_plan(plan, (const char*)ws.x + off, (const char*)ws.r + off, ws.w, (char*)ws.y + off,
                                (char*)ws.r_out + off, shape.n_tokens, shape.hidden, ws.eps, stream);
         };
@@ -692,7 +698,8 @@ int check_workspace(const rt_shape* s, const rt_workspace* ws)
         set_error("shape or workspace is NULL");
         return RT_ERR_NULL;
     }
-    if (!ws->x || !ws->r || !ws->w || !ws->y || !ws->r_out || !ws->y_ref || !ws->r_ref) {
+    const bool is_silu = s->op == RT_OP_SILU_AND_MUL;
+    if (!ws->x || !ws->y || !ws->y_ref || (!is_silu && (!ws->r || !ws->w || !ws->r_out || !ws->r_ref))) {
         set_error("a workspace pointer is NULL");
         return RT_ERR_NULL;
     }
@@ -700,7 +707,7 @@ int check_workspace(const rt_shape* s, const rt_workspace* ws)
         set_error("n_ref_tokens=%lld must lie in 1..n_tokens=%lld", (long long)ws->n_ref_tokens, (long long)s->n_tokens);
         return RT_ERR_SHAPE;
     }
-    if (ws->x == ws->y || ws->r == ws->r_out) {
+    if (ws->x == ws->y || (!is_silu && ws->r == ws->r_out)) {
         set_error("the tuner's workspace must not alias inputs and outputs (launches repeat)");
         return RT_ERR_SHAPE;
     }

@@ -25,7 +25,7 @@ int table_lookup(const rt_spec_entry* table, int32_t n, const rt_params* general
     double best_d = 0.0;
     for (int32_t i = 0; i < n; ++i) {
         const rt_spec_entry& e = table[i];
-        if (e.shape.dtype != query->dtype) continue;
+        if (e.shape.dtype != query->dtype || e.shape.op != query->op) continue;
         const double d = shape_distance(e.shape, *query);
         if (best >= 0 && d >= best_d) continue;
         Plan plan;
@@ -139,6 +139,8 @@ int rmsnorm_launch_auto(const rt_spec_entry* table, int32_t n_entries, const rt_
     s.hidden = hidden;
     s.dtype = dtype;
     s.min_ptr_align = n_tokens > 0 ? rt::min_pointer_alignment(x, r, w, y, r_out) : 256;
+    s.op = RT_OP_ADD_RMSNORM;
+    s.reserved = 0;
     rt_params theta;
     int st = tuner_table_lookup(table, n_entries, general, &s, nullptr, &theta, nullptr);
     if (st != RT_OK) return st;

@@ -13,6 +13,7 @@ namespace rt {
 
 // One compiled instance of the kernel template.
 struct KernelEntry {
+    int op;
     int dtype, vec_bytes, stage, reduce, unroll, cap;  // cap: per-thread row vectors (register stage), else 0
     const void* fn;
 };
@@ -31,6 +32,7 @@ struct KernelInfo {
 
 // theta turned into launch geometry; produced only when every hard rule holds.
 struct Plan {
+    int op;
     int kernel_index;
     int elem_bytes;
     int nvec;         // vectors per row
@@ -55,7 +57,7 @@ const char* last_error();
 inline int elem_bytes_of(int dtype) { return dtype == RT_FP32 ? 4 : 2; }
 
 const std::vector<KernelEntry>& registry();
-int find_kernel(int dtype, int vec_bytes, int stage, int reduce, int unroll, int cap);
+int find_kernel(int op, int dtype, int vec_bytes, int stage, int reduce, int unroll, int cap);
 // Cached cudaFuncGetAttributes of instance `index` on the current device.
 int kernel_info(int index, KernelInfo* out);
 
@@ -68,6 +70,7 @@ int current_limits(rt_limits* out);
 
 int launch_plan(const Plan& plan, const void* x, const void* r, const void* w, void* y, void* r_out,
                 int64_t n_tokens, int64_t hidden, float eps, cudaStream_t stream);
+int launch_silu_plan(const Plan& plan, const void* x, void* out, int64_t n_tokens, cudaStream_t stream);
 int ensure_dynamic_smem(int index, size_t bytes);
 int* device_status_word();
 void count_launch(int64_t n = 1);

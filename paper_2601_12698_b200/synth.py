@@ -29,7 +29,7 @@ import numpy as np
 import torch
 
 ROWS_PER_BLOCK = 64
-TENSOR_X, TENSOR_R, TENSOR_W = 0, 1, 2
+TENSOR_X, TENSOR_R, TENSOR_W, TENSOR_GATE_UP = 0, 1, 2, 3
 
 TORCH_DTYPES = {"bf16": torch.bfloat16, "fp16": torch.float16, "fp32": torch.float32}
 DTYPE_CODES = {"bf16": 0, "fp16": 1, "fp32": 2}
@@ -54,6 +54,7 @@ class Workload:
     seed: int
     dist: Dist = field(default_factory=Dist)
     eps: float = 1e-6
+    op: str = "add_rmsnorm"  # or "silu_and_mul" (hidden is then d, the output width)
 
     @property
     def elements(self) -> int:
@@ -61,13 +62,18 @@ class Workload:
 
     @property
     def algorithmic_bytes(self) -> int:
-        """Bytes the operator must move: read x, read r, write r', write y, w once."""
+        """Bytes the operator must move.  add_rmsnorm: read x, read r, write r', write y, w once.
+        silu_and_mul: read gate, read value, write out."""
         b = DTYPE_BYTES[self.dtype]
+        if self.op == "silu_and_mul":
+            return 3 * b * self.elements
         return 4 * b * self.elements + b * self.hidden
 
     @property
     def nominal_bytes(self) -> int:
-        """Three reads and two writes per element (w counted as a full stream)."""
+        """add_rmsnorm: three reads and two writes per element (w counted as a full stream)."""
+        if self.op == "silu_and_mul":
+            return self.algorithmic_bytes
         return 5 * DTYPE_BYTES[self.dtype] * self.elements
 
 
@@ -89,6 +95,12 @@ def workloads() -> dict[str, Workload]:
         add(Workload(f"c4_fp16_8192x{h}", "fp16", 8192, h, seed=3))
     add(Workload("c4x_fp16_8192x6148", "fp16", 8192, 6148, seed=3))
     add(Workload("c5_fp32_32768x12288", "fp32", 32768, 12288, seed=4))
+    # silu_and_mul: a bandwidth case (LLaMA-3-8B MLP width), and the paper's fp32 (m, n) shapes with n = d
+    gate = Dist(sigma=2.5)
+    add(Workload("silu_bf16_16384x14336", "bf16", 16384, 14336, seed=6, dist=gate, op="silu_and_mul"))
+    add(Workload("silu_fp32_2048x8192", "fp32", 2048, 8192, seed=6, dist=gate, op="silu_and_mul"))
+    add(Workload("silu_fp32_128x11008", "fp32", 128, 11008, seed=6, dist=gate, op="silu_and_mul"))
+    add(Workload("silu_bf16_64x11008", "bf16", 64, 11008, seed=6, dist=gate, op="silu_and_mul"))
     return out
 
 
@@ -154,7 +166,15 @@ def make_inputs(n_tokens: int, hidden: int, dtype: str, seed: int, dist: Dist = 
     return x, r, w
 
 
+def make_gate_up(row_begin: int, row_end: int, d: int, dtype: str, seed: int, dist: Dist = Dist(sigma=2.5),
+                 threads: int = 8) -> torch.Tensor:
+    """Rows of the [T, 2*d] input of silu_and_mul: gate and value halves, N(0, sigma) each."""
+    return make_rows(TENSOR_GATE_UP, row_begin, row_end, 2 * d, dtype, seed, dist, threads).contiguous()
+
+
 def make_workload_inputs(wl: Workload, threads: int = 8):
+    if wl.op == "silu_and_mul":
+        return (make_gate_up(0, wl.n_tokens, wl.hidden, wl.dtype, wl.seed, wl.dist, threads),)
     return make_inputs(wl.n_tokens, wl.hidden, wl.dtype, wl.seed, wl.dist, threads)
 
 

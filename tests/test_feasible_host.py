@@ -90,3 +90,22 @@ def test_argument_errors(L):
     arr = (B.rt_params * 3)()
     assert B.lib.tuner_derive_feasible_ex(ctypes.byref(ok), ctypes.byref(L), 15, arr, 3, ctypes.byref(n)) == B.RT_OK
     assert n.value > 3
+
+
+def test_silu_and_mul_grid_has_no_reduction_axis(L):
+    s = B.shape_of(16384, 14336, "bf16", op=B.RT_OP_SILU_AND_MUL)
+    raw = B.tuner_raw_grid(s)
+    assert {t.reduce for t in raw} == {0} and {t.cluster_size for t in raw} == {1} and {t.stage for t in raw} == {0, 2}
+    f = B.tuner_derive_feasible(s, L)
+    assert f and {t.stage for t in f} == {0, 2} and {t.vec_bytes for t in f} == {16, 8}
+    for th in f:
+        assert B.tuner_check_params(s, th, L) == B.RT_OK
+    c = B.tuner_derive_counts(s, L)
+    assert c["feasible"] == len(f) and sum(v for k, v in c.items() if k != "raw") == c["raw"] == len(raw)
+    # the other kernel's thetas are not this kernel's
+    assert B.tuner_check_params(s, B.make_params(reduce=B.RT_REDUCE_SMEM), L) == B.RT_ERR_INFEASIBLE
+    assert B.tuner_check_params(s, B.make_params(stage=B.RT_STAGE_SMEM_LDG), L) == B.RT_ERR_INFEASIBLE
+    # d = 3073 fp16: 2-byte fall-back only; the TMA stage needs 16-byte rows
+    f = B.tuner_derive_feasible(B.shape_of(8, 3073, "fp16", op=B.RT_OP_SILU_AND_MUL), L)
+    assert f and {t.vec_bytes for t in f} == {2} and {t.stage for t in f} == {0}
+    assert B.tuner_check_params(B.shape_of(8, 4096, "bf16", op=7), B.make_params(), L) == B.RT_ERR_SHAPE
