@@ -2,6 +2,8 @@
 // Rows are independent, so a tensor is cut into row chunks; three chunk slots rotate so that the
 // host-to-device copies of chunk i+1, the kernel of chunk i and the device-to-host copies of chunk
 // i-1 run at the same time on three streams.
+#include <string.h>
+
 #include <mutex>
 
 #include "tuner_internal.h"
@@ -115,6 +117,8 @@ int rmsnorm_template_run_host(const rt_params* p, const void* x_host, const void
 
     // Plans for a full chunk and for the ragged last chunk (device buffers are 256-byte aligned).
     rt_shape shape;
+    memset(&shape, 0, sizeof(shape));
+    shape.op = RT_OP_ADD_RMSNORM;
     shape.hidden = hidden;
     shape.dtype = dtype;
     shape.min_ptr_align = 256;
