@@ -1,6 +1,7 @@
 """CPU oracles of the tuned kernels (test infrastructure only).
 
-Thin ctypes wrapper over ``add_rmsnorm_oracle.c`` and ``silu_and_mul_oracle.c``;
+Thin ctypes wrapper over ``add_rmsnorm_oracle.c``, ``silu_and_mul_oracle.c`` and
+``merge_attn_states_oracle.c``;
 all arithmetic is in the C files (``selection.py`` holds the plain-Python oracle
 of the general-configuration choice).  Only the tests, the smoke check and the benchmark's CPU-baseline leg may
 import this package.  It imports nothing from the CUDA package and shares no
@@ -23,7 +24,7 @@ BF16, FP16, FP32 = 0, 1, 2
 DTYPE_NAMES = {BF16: "bf16", FP16: "fp16", FP32: "fp32"}
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-SOURCES = ("add_rmsnorm_oracle.c", "silu_and_mul_oracle.c")
+SOURCES = ("add_rmsnorm_oracle.c", "silu_and_mul_oracle.c", "merge_attn_states_oracle.c")
 HEADERS = ("number_formats.h",)
 _LIB = os.path.join(_HERE, "liboracle.so")
 _lock = threading.Lock()
@@ -71,6 +72,11 @@ def _bind(path: str):
     lib.oracle_rel_compare32.restype = None
     lib.oracle_silu_and_mul.argtypes = [vp, vp, i64, i64, ctypes.c_int, ctypes.c_int]
     lib.oracle_silu_and_mul.restype = ctypes.c_int
+    lib.oracle_merge_attn_states.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, ctypes.c_int]
+    lib.oracle_merge_attn_states.restype = ctypes.c_int
+    lib.oracle_mixed_compare.argtypes = [vp, vp, i64, ctypes.c_int, ctypes.c_double, ctypes.c_double,
+                                         ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i64)]
+    lib.oracle_mixed_compare.restype = None
     return lib
 
 
@@ -157,6 +163,42 @@ def silu_and_mul(x, dtype: int | None = None, *, threads: int = 1):
     if rc != 0:
         raise RuntimeError(f"oracle_silu_and_mul failed with status {rc}")
     return to_torch(out, dt) if want_torch else out
+
+
+def merge_attn_states(v_a, s_a, v_b, s_b, dtype: int | None = None):
+    """(v_out, s_out) for v_a, v_b of shape [n, h, d] and float32 log-sum-exps s_a, s_b of shape [n, h]."""
+    want_torch = hasattr(v_a, "detach")
+    va, dt = as_storage(v_a, dtype)
+    vb, dt_b = as_storage(v_b, dtype)
+    sa, _ = as_storage(s_a, FP32)
+    sb, _ = as_storage(s_b, FP32)
+    if dt != dt_b or va.ndim != 3 or vb.shape != va.shape or sa.shape != va.shape[:2] or sb.shape != sa.shape:
+        raise ValueError("expected v_a, v_b of shape [n, h, d] and s_a, s_b of shape [n, h]")
+    if sa.dtype != np.float32 or sb.dtype != np.float32:
+        raise TypeError("s_a and s_b must be float32")
+    n, h, d = va.shape
+    v_out = np.empty_like(va)
+    s_out = np.empty((n, h), dtype=np.float32)
+    rc = _load().oracle_merge_attn_states(va.ctypes.data, sa.ctypes.data, vb.ctypes.data, sb.ctypes.data,
+                                          v_out.ctypes.data, s_out.ctypes.data, n, h, d, dt)
+    if rc != 0:
+        raise RuntimeError(f"oracle_merge_attn_states failed with status {rc}")
+    if want_torch:
+        return to_torch(v_out, dt), to_torch(s_out, FP32)
+    return v_out, s_out
+
+
+def compare_mixed(got, ref, dtype: int | None = None, *, tol: float = 2.0, tol_abs: float = 1e-5):
+    """(largest absolute difference, count failing) where an element passes within `tol` (ulps for 16-bit
+    types, relative for fp32) OR within `tol_abs` absolutely."""
+    g, dt = as_storage(got, dtype)
+    q, dt2 = as_storage(ref, dtype)
+    if dt != dt2 or g.shape != q.shape:
+        raise ValueError("got and ref must match in dtype and shape")
+    worst, bad = ctypes.c_double(0.0), ctypes.c_int64(0)
+    _load().oracle_mixed_compare(g.ctypes.data, q.ctypes.data, g.size, dt, tol, tol_abs, ctypes.byref(worst),
+                                 ctypes.byref(bad))
+    return worst.value, bad.value
 
 
 def decode16(bits, dtype: int) -> np.ndarray:

@@ -39,7 +39,7 @@
  * Plain C99 + pthreads (threads only split independent rows).  The number-format code lives in
  * number_formats.h, shared by the oracle's C files only.  Build (oracle/__init__.py does this):
  *   gcc -O2 -fno-fast-math -ffp-contract=off -shared -fPIC -pthread \
- *       add_rmsnorm_oracle.c silu_and_mul_oracle.c -o liboracle.so -lm
+ *       add_rmsnorm_oracle.c silu_and_mul_oracle.c merge_attn_states_oracle.c -o liboracle.so -lm
  */
 #include <math.h>
 #include <pthread.h>

@@ -157,3 +157,58 @@ def test_planted_silu_mistake_is_caught(oracle_lib, tmp_path, name):
         assert not _silu_pins(oracle_lib), f"pins did not notice: {name}"
     finally:
         oracle_lib._lib = saved
+
+
+MERGE_MUTATIONS = {
+    "second_weight_is_first": ("(wa * a + wb * b) / D", "(wa * a + wa * b) / D"),
+    "not_normalised": ("(wa * a + wb * b) / D", "(wa * a + wb * b)"),
+    "log_dropped": ("(float)(m + log(D))", "(float)(m + D)"),
+    "shift_dropped": ("wb = exp(sb - m)", "wb = exp(sb)"),
+    "lse_indexed_by_token": ("const double sa = (double)s_a[row], sb = (double)s_b[row];",
+                             "const double sa = (double)s_a[t], sb = (double)s_b[row];"),
+    "parts_swapped_weights": ("const double wa = exp(sa - m), wb = exp(sb - m)", "const double wa = exp(sb - m), wb = exp(sa - m)"),
+    "empty_case_returns_garbage": ("s_out[row] = -INFINITY;", "s_out[row] = 0.0f;"),
+}
+
+
+def _merge_pins(o) -> bool:
+    try:
+        for dtype, td in ((0, torch.bfloat16), (2, torch.float32)):
+            g = torch.Generator().manual_seed(5)
+            n, h, d, k1, k2 = 4, 3, 8, 9, 5
+            q = torch.randn(n, h, d, generator=g, dtype=torch.float64)
+            K = torch.randn(h, k1 + k2, d, generator=g, dtype=torch.float64)
+            V = torch.randn(h, k1 + k2, d, generator=g, dtype=torch.float64)
+
+            def attend(lo, hi):
+                logits = torch.einsum("nhd,hkd->nhk", q, K[:, lo:hi]) / math.sqrt(d)
+                return torch.einsum("nhk,hkd->nhd", torch.softmax(logits, -1), V[:, lo:hi]), torch.logsumexp(logits, -1)
+            (o1, l1), (o2, l2), (oo, ll) = attend(0, k1), attend(k1, k1 + k2), attend(0, k1 + k2)
+            v, so = o.merge_attn_states(o1.to(td), l1.float(), o2.to(td), l2.float())
+            if not torch.allclose(v.double(), oo, rtol=0, atol=0.04 if dtype == 0 else 1e-5):
+                return False
+            if not torch.allclose(so.double(), ll, rtol=0, atol=2e-6):
+                return False
+            empty = torch.full((n, h), float("-inf"))
+            v, so = o.merge_attn_states(o1.to(td), empty, o2.to(td), empty)
+            if not (torch.equal(so, empty) and bool((v == 0).all())):
+                return False
+    except Exception:
+        return False
+    return True
+
+
+def test_real_merge_oracle_passes_its_pins(oracle_lib):
+    assert _merge_pins(oracle_lib)
+
+
+@pytest.mark.parametrize("name", sorted(MERGE_MUTATIONS))
+def test_planted_merge_mistake_is_caught(oracle_lib, tmp_path, name):
+    old, new = MERGE_MUTATIONS[name]
+    so = _build_mutant(oracle_lib, str(tmp_path), old, new, targets=("merge_attn_states_oracle.c",))
+    saved = oracle_lib._lib
+    try:
+        oracle_lib._lib = oracle_lib._bind(so)
+        assert not _merge_pins(oracle_lib), f"pins did not notice: {name}"
+    finally:
+        oracle_lib._lib = saved
