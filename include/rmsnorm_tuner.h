@@ -49,7 +49,8 @@ typedef enum { RT_BF16 = 0, RT_FP16 = 1, RT_FP32 = 2 } rt_dtype;
 /* The kernels that have a template in this library (the paper tunes three serving kernels, "Kernels"). */
 typedef enum {
     RT_OP_ADD_RMSNORM = 0,  /* fused residual-add + RMSNorm: the operator described above */
-    RT_OP_SILU_AND_MUL = 1  /* out[t,j] = silu(x[t,j]) * x[t,d+j] for x of shape [n_tokens, 2*d] */
+    RT_OP_SILU_AND_MUL = 1, /* out[t,j] = silu(x[t,j]) * x[t,d+j] for x of shape [n_tokens, 2*d] */
+    RT_OP_MERGE_ATTN_STATES = 2 /* two partial attention results merged by their log-sum-exps */
 } rt_op;
 
 /* Where a row lives between the two passes over it. */
@@ -80,11 +81,12 @@ typedef struct {
 
 typedef struct {
     int64_t n_tokens;
-    int64_t hidden;        /* row width of the OUTPUT: hidden size, or d for silu_and_mul */
+    int64_t hidden;        /* row width of the OUTPUT: hidden size; d for silu_and_mul; heads * d for
+                              merge_attn_states */
     int32_t dtype;         /* rt_dtype */
     int32_t min_ptr_align; /* largest power of two (bytes, <= 256) dividing all base addresses */
     int32_t op;            /* rt_op; 0 = add_rmsnorm */
-    int32_t reserved;
+    int32_t head_dim;      /* merge_attn_states: d (hidden = heads * d); 0 for the other kernels */
 } rt_shape;
 
 /* r(h): the resource upper bounds the feasible region is derived from. */
@@ -133,7 +135,9 @@ typedef struct {
 } rt_budget;
 
 /* For silu_and_mul: x is the [n_tokens, 2*d] input (ring stride 2 * ring_stride_bytes), y the output,
- * y_ref its reference; r, w, r_out, r_ref are unused and may be NULL. */
+ * y_ref its reference; r, w, r_out, r_ref are unused and may be NULL.
+ * For merge_attn_states: x = v_a, r = v_b, w = s_a, aux = s_b, y = v_out, r_out = s_out, y_ref and r_ref their
+ * references (the s tensors are binary32 [n_tokens, heads]; in a ring they advance by n_tokens*heads*4). */
 typedef struct {
     const void* x;     /* device, [ring_sets][n_tokens, hidden] */
     const void* r;     /* device */
@@ -147,6 +151,7 @@ typedef struct {
     int32_t ring_sets;        /* >= 1; timed launches rotate over the sets (cold-L2 timing of small shapes) */
     float eps;
     void* stream;
+    const void* aux;   /* device; merge_attn_states: s_b.  NULL otherwise */
 } rt_workspace;
 
 typedef enum { RT_PHASE_SEED = 0, RT_PHASE_GRID = 1, RT_PHASE_CLIMB = 2, RT_PHASE_TOPK = 3,
@@ -233,6 +238,21 @@ int64_t rmsnorm_host_workspace_bytes(int64_t n_tokens, int64_t hidden, int dtype
  */
 int silu_and_mul_template_launch(const rt_params* p, const void* x, void* out, int64_t n_tokens, int64_t d,
                                  int dtype, void* stream);
+
+/*
+ * merge_attn_states as an instance of its own template (third kernel of the paper's "Kernels" list, shapes
+ * (n, h, d); axes as for silu_and_mul: no reduction, stage = registers or TMA bulk).
+ *   v_a, v_b  device, [n_tokens, heads, head_dim] of `dtype`: normalised partial attention outputs.
+ *   s_a, s_b  device, [n_tokens, heads] binary32: natural log of each part's softmax denominator
+ *             (-inf = that part saw no keys).
+ *   v_out     device, [n_tokens, heads, head_dim];  s_out  device, [n_tokens, heads] binary32.
+ *   With m = max(s_a, s_b), w = exp(s - m), D = w_a + w_b:  v_out = round_dtype((w_a v_a + w_b v_b) / D),
+ *   s_out = m + ln D;  both parts empty: v_out = 0, s_out = -inf.  Computed in fp32.
+ * Asynchronous on `stream`, allocates nothing; infeasible theta is refused without launching.
+ */
+int merge_attn_states_template_launch(const rt_params* p, const void* v_a, const float* s_a, const void* v_b,
+                                      const float* s_b, void* v_out, float* s_out, int64_t n_tokens,
+                                      int64_t heads, int64_t head_dim, int dtype, void* stream);
 
 /* ---- 2. the feasible region ----------------------------------------------------- */
 
@@ -349,6 +369,14 @@ int rmsnorm_launch_auto(const rt_spec_entry* table, int32_t n_entries, const rt_
                         int64_t hidden, float eps, int dtype, void* stream, rt_params* used);
 
 typedef enum { RT_CMP_BITS = 0, RT_CMP_ULP16 = 1, RT_CMP_REL32 = 2 } rt_compare_mode;
+/*
+ * d(.,.) for outputs that may cancel (merge_attn_states): an element passes when it is within `tol` of the
+ * reference - units in the last place for the 16-bit types, relative for binary32 - OR within `tol_abs`
+ * absolutely.  *max_abs receives the largest absolute difference, *n_bad the failing elements.
+ * got, ref: device; max_abs, n_bad: host.  Synchronises `stream`.
+ */
+int tuner_compare_mixed(const void* got, const void* ref, int64_t n, int dtype, double tol, double tol_abs,
+                        double* max_abs, int64_t* n_bad, void* stream);
 /*
  * The distance d(.,.) of the correctness criterion, computed on the device.
  *   got, ref  device, n elements of `dtype`.

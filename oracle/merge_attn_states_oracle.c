@@ -93,7 +93,7 @@ void oracle_mixed_compare(const void* got, const void* ref, int64_t n, int dtype
         } else {
             diff = fabs(g - q);
             if (dtype == ORACLE_FP32) {
-                ok = diff <= tol_ulp_or_rel * fabs(q) + tol_abs;
+                ok = diff <= tol_ulp_or_rel * fabs(q) || diff <= tol_abs;
             } else {
                 const uint16_t gb = ((const uint16_t*)got)[i], qb = ((const uint16_t*)ref)[i];
                 int32_t gi = gb & 0x7FFF, qi = qb & 0x7FFF;

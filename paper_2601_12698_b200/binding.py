@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(_HERE, "librmsnorm_tuner.so")
 HEADER_PATH = os.path.join(os.path.dirname(_HERE), "include", "rmsnorm_tuner.h")
 
 RT_BF16, RT_FP16, RT_FP32 = 0, 1, 2
-RT_OP_ADD_RMSNORM, RT_OP_SILU_AND_MUL = 0, 1
+RT_OP_ADD_RMSNORM, RT_OP_SILU_AND_MUL, RT_OP_MERGE_ATTN_STATES = 0, 1, 2
 RT_STAGE_REG, RT_STAGE_SMEM_LDG, RT_STAGE_SMEM_TMA = 0, 1, 2
 RT_REDUCE_SHFL, RT_REDUCE_SMEM, RT_REDUCE_CLUSTER = 0, 1, 2
 RT_PRUNE_IDLE_THREADS, RT_PRUNE_DUPLICATES, RT_PRUNE_CLUSTER_WAVES, RT_PRUNE_IDLE_ROWS = 1, 2, 4, 8
@@ -53,7 +53,7 @@ def make_params(threads_per_row=256, rows_per_cta=1, vec_bytes=16, unroll=1, sta
 
 class rt_shape(Structure):
     _fields_ = [("n_tokens", c_int64), ("hidden", c_int64), ("dtype", c_int32), ("min_ptr_align", c_int32),
-                ("op", c_int32), ("reserved", c_int32)]
+                ("op", c_int32), ("head_dim", c_int32)]
 
 
 class rt_limits(Structure):
@@ -73,7 +73,8 @@ class rt_budget(Structure):
 class rt_workspace(Structure):
     _fields_ = [("x", c_void_p), ("r", c_void_p), ("w", c_void_p), ("y", c_void_p), ("r_out", c_void_p),
                 ("y_ref", c_void_p), ("r_ref", c_void_p), ("n_ref_tokens", c_int64),
-                ("ring_stride_bytes", c_int64), ("ring_sets", c_int32), ("eps", c_float), ("stream", c_void_p)]
+                ("ring_stride_bytes", c_int64), ("ring_sets", c_int32), ("eps", c_float), ("stream", c_void_p),
+                ("aux", c_void_p)]
 
 
 class rt_eval_record(Structure):
@@ -106,6 +107,8 @@ _SIGNATURES = {
     "rmsnorm_template_launch": (c_int, [POINTER(rt_params), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                         c_int64, c_int64, c_float, c_int, c_void_p]),
     "silu_and_mul_template_launch": (c_int, [POINTER(rt_params), c_void_p, c_void_p, c_int64, c_int64, c_int, c_void_p]),
+    "merge_attn_states_template_launch": (c_int, [POINTER(rt_params), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                                  c_void_p, c_int64, c_int64, c_int64, c_int, c_void_p]),
     "rmsnorm_template_run_host": (c_int, [POINTER(rt_params), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                           c_int64, c_int64, c_float, c_int, c_void_p, c_int64, c_int64, c_void_p]),
     "rmsnorm_host_workspace_bytes": (c_int64, [c_int64, c_int64, c_int, c_int64]),
@@ -132,6 +135,8 @@ _SIGNATURES = {
     "tuner_launch_floor": (c_int, [POINTER(rt_budget), c_void_p, POINTER(c_float)]),
     "tuner_compare": (c_int, [c_void_p, c_void_p, c_int64, c_int, c_int, c_double, POINTER(c_double),
                               POINTER(c_int64), c_void_p]),
+    "tuner_compare_mixed": (c_int, [c_void_p, c_void_p, c_int64, c_int, c_double, c_double, POINTER(c_double),
+                                    POINTER(c_int64), c_void_p]),
     "tuner_compare_static": (c_int, [c_void_p, c_void_p, c_int64, c_int, c_int, c_double, POINTER(c_double),
                                      POINTER(c_int64), c_void_p]),
     "rt_status_string": (c_char_p, [c_int]),
@@ -186,10 +191,11 @@ def _ptr_align(*tensors) -> int:
     return bits & -bits
 
 
-def shape_of(n_tokens: int, hidden: int, dtype, min_ptr_align: int = 256, op: int = RT_OP_ADD_RMSNORM) -> rt_shape:
-    """hidden is the output row width (d for silu_and_mul)."""
+def shape_of(n_tokens: int, hidden: int, dtype, min_ptr_align: int = 256, op: int = RT_OP_ADD_RMSNORM,
+             head_dim: int = 0) -> rt_shape:
+    """hidden is the output row width (d for silu_and_mul, heads * head_dim for merge_attn_states)."""
     code = DTYPE_CODES[dtype] if isinstance(dtype, str) else int(dtype)
-    return rt_shape(n_tokens, hidden, code, min_ptr_align, op, 0)
+    return rt_shape(n_tokens, hidden, code, min_ptr_align, op, head_dim)
 
 
 def sm100_nominal_limits() -> rt_limits:
@@ -230,6 +236,22 @@ def silu_and_mul_template_launch(params: rt_params, x, out, stream=None) -> None
         raise ValueError("x must be [n_tokens, 2*d] of the output's dtype")
     _check(lib.silu_and_mul_template_launch(byref(params), x.data_ptr(), out.data_ptr(), n_tokens, d, _dtype_code(x),
                                             _stream_ptr(stream)), "silu_and_mul_template_launch")
+
+
+def merge_attn_states_template_launch(params: rt_params, v_a, s_a, v_b, s_b, v_out, s_out, stream=None) -> None:
+    """Merge two partial attention results (device tensors; v: [n, h, d], s: float32 [n, h]); asynchronous."""
+    import torch
+    n, h, d = v_a.shape
+    for t in (v_a, v_b, v_out):
+        if not (t.is_cuda and t.is_contiguous() and t.shape == (n, h, d) and t.dtype == v_a.dtype):
+            raise ValueError("v_a, v_b, v_out must be contiguous CUDA tensors of one shape [n, h, d] and dtype")
+    for t in (s_a, s_b, s_out):
+        if not (t.is_cuda and t.is_contiguous() and t.shape == (n, h) and t.dtype == torch.float32):
+            raise ValueError("s_a, s_b, s_out must be contiguous float32 CUDA tensors of shape [n, h]")
+    _check(lib.merge_attn_states_template_launch(byref(params), v_a.data_ptr(), s_a.data_ptr(), v_b.data_ptr(),
+                                                 s_b.data_ptr(), v_out.data_ptr(), s_out.data_ptr(), n, h, d,
+                                                 _dtype_code(v_a), _stream_ptr(stream)),
+           "merge_attn_states_template_launch")
 
 
 def rmsnorm_host_workspace_bytes(n_tokens: int, hidden: int, dtype, chunk_tokens: int = 0) -> int:
@@ -305,14 +327,15 @@ def make_budget(max_evals=64, warmup=20, iters=100, repeats=3, top_k=5, strategy
 
 
 def make_workspace(x, r, w, y, r_out, y_ref, r_ref, eps: float, n_ref_tokens: int | None = None, ring_sets: int = 1,
-                   ring_stride_bytes: int = 0, stream=None) -> rt_workspace:
+                   ring_stride_bytes: int = 0, stream=None, aux=None) -> rt_workspace:
     """Device tensors for the tuner.  With ring_sets > 1, x, r, y, r_out are [ring_sets, T, H] and the
-    references cover set 0.  For silu_and_mul pass r = w = r_out = r_ref = None."""
+    references cover set 0.  For silu_and_mul pass r = w = r_out = r_ref = None; for merge_attn_states
+    x = v_a, r = v_b, w = s_a, aux = s_b, y = v_out, r_out = s_out."""
     T = x.shape[-2]
     ptr = lambda t: t.data_ptr() if t is not None else None
     return rt_workspace(ptr(x), ptr(r), ptr(w), ptr(y), ptr(r_out), ptr(y_ref), ptr(r_ref),
                         n_ref_tokens if n_ref_tokens is not None else T, ring_stride_bytes,
-                        ring_sets, eps, _stream_ptr(stream))
+                        ring_sets, eps, _stream_ptr(stream), ptr(aux))
 
 
 def tuner_search(shape: rt_shape, budget: rt_budget, ws: rt_workspace, log_cap: int = 4096):
@@ -354,6 +377,16 @@ def tuner_compare(got, ref, mode: int, tol: float = 0.0, stream=None):
     worst, bad = c_double(0.0), c_int64(0)
     _check(lib.tuner_compare(got.data_ptr(), ref.data_ptr(), got.numel(), _dtype_code(got), mode, tol, byref(worst),
                              byref(bad), _stream_ptr(stream)), "tuner_compare")
+    return worst.value, bad.value
+
+
+def tuner_compare_mixed(got, ref, tol: float, tol_abs: float, stream=None):
+    """(largest absolute difference, failing elements): pass within tol (ulps / relative) OR tol_abs absolutely."""
+    if got.shape != ref.shape or got.dtype != ref.dtype:
+        raise ValueError("got and ref must match")
+    worst, bad = c_double(0.0), c_int64(0)
+    _check(lib.tuner_compare_mixed(got.data_ptr(), ref.data_ptr(), got.numel(), _dtype_code(got), tol, tol_abs,
+                                   byref(worst), byref(bad), _stream_ptr(stream)), "tuner_compare_mixed")
     return worst.value, bad.value
 
 
@@ -418,7 +451,7 @@ class SpecTable:
         names = {v: k for k, v in DTYPE_CODES.items()}
         return {"device": self.device_name, "general": self.general.as_dict() if self.general else None,
                 "specialised": [{"dtype": names[s.dtype], "n_tokens": int(s.n_tokens), "hidden": int(s.hidden),
-                                 "op": int(s.op), "theta": t.as_dict(), "us": round(float(us), 3)}
+                                 "op": int(s.op), "head_dim": int(s.head_dim), "theta": t.as_dict(), "us": round(float(us), 3)}
                                 for s, t, us in self.entries]}
 
     @classmethod
@@ -432,7 +465,8 @@ class SpecTable:
     def from_json(cls, d: dict) -> "SpecTable":
         fields = [k for k, _ in rt_params._fields_]
         mk = lambda t: rt_params(*[int(t[k]) for k in fields])
-        entries = [(shape_of(e["n_tokens"], e["hidden"], e["dtype"], op=int(e.get("op", 0))), mk(e["theta"]), float(e["us"]))
+        entries = [(shape_of(e["n_tokens"], e["hidden"], e["dtype"], op=int(e.get("op", 0)),
+                             head_dim=int(e.get("head_dim", 0))), mk(e["theta"]), float(e["us"]))
                    for e in d.get("specialised", [])]
         return cls(entries, mk(d["general"]) if d.get("general") else None, d.get("device", ""))
 

@@ -31,7 +31,8 @@ std::vector<int> vec_levels(const rt_shape& s)
 {
     const int eb = elem_bytes_of(s.dtype);
     const int64_t row_bytes = s.hidden * eb;
-    auto fits = [&](int vb) { return vb >= eb && row_bytes % vb == 0 && s.min_ptr_align >= vb; };
+    const int64_t head_bytes = s.op == RT_OP_MERGE_ATTN_STATES && s.head_dim > 0 ? (int64_t)s.head_dim * eb : row_bytes;
+    auto fits = [&](int vb) { return vb >= eb && row_bytes % vb == 0 && head_bytes % vb == 0 && s.min_ptr_align >= vb; };
     if (fits(16) || fits(8)) return {16, 8};
     if (fits(4)) return {4};
     if (fits(2)) return {2};
@@ -52,8 +53,9 @@ std::vector<rt_params> raw_grid(const rt_shape& s)
 {
     std::vector<rt_params> out;
     const std::vector<int> vecs = vec_levels(s);
-    // silu_and_mul has no reduction and no ld.global -> shared stage: its grid is the remaining axes
-    const bool is_silu = s.op == RT_OP_SILU_AND_MUL;
+    // silu_and_mul and merge_attn_states have no reduction and no ld.global -> shared stage: their grid is
+    // the remaining axes
+    const bool is_silu = s.op == RT_OP_SILU_AND_MUL || s.op == RT_OP_MERGE_ATTN_STATES;  // no reduction axis
     for (int stage = 0; stage < 3; ++stage)
         for (const Mode& m : kReduceModes)
             for (int vb : vecs) {

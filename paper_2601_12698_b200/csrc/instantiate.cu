@@ -1,6 +1,6 @@
 // One instantiation unit of the kernel template.  Compiled once per line of instance_units.inc with
 //   -DRT_UNIT_NAME=<name> -DRT_UNIT_T=<element type> -DRT_UNIT_DTYPE=<0|1|2> -DRT_UNIT_VB=<bytes>
-//   -DRT_UNIT_GROUP=<0 register stage | 1 shared-memory stages | 2 narrow fall-back | 3 silu_and_mul>
+//   -DRT_UNIT_GROUP=<0 register stage | 1 shared-memory stages | 2 narrow fall-back | 3 silu_and_mul | 4 merge_attn_states>
 //   -DRT_UNIT_REDUCE=<0|1|2>   (register-stage units only)
 //
 // Instance lists.  Register stage: CAP (row vectors kept per thread) in {1,2,4,8,16,32} while the row
@@ -9,7 +9,9 @@
 // byte length is not a multiple of 8): register stage, shuffle reduction, U in {1,4}.
 // silu_and_mul (one unit per element type, every vector width): stages register and TMA bulk for 16- and
 // 8-byte vectors with U in {1,2,4}; register stage with U in {1,4} for the 4- and 2-byte fall-back.
+// merge_attn_states: the same instance list as silu_and_mul.
 #include "add_rmsnorm_kernel.cuh"
+#include "merge_attn_states_kernel.cuh"
 #include "silu_and_mul_kernel.cuh"
 #include "tuner_internal.h"
 
@@ -42,6 +44,19 @@ rt::KernelEntry silu_entry()
                                (const void*)&rt::silu_and_mul_kernel<T, VB, ST, U>};
     }
 }
+template <int VB, int ST, int U>
+rt::KernelEntry merge_entry()
+{
+    if constexpr (VB < (int)sizeof(T)) {
+        return rt::KernelEntry{RT_OP_MERGE_ATTN_STATES, kDtype, VB, ST, 0, U, 0, nullptr};
+    } else {
+        return rt::KernelEntry{RT_OP_MERGE_ATTN_STATES, kDtype, VB, ST, 0, U, 0,
+                               (const void*)&rt::merge_attn_states_kernel<T, VB, ST, U>};
+    }
+}
+#define RT_MERGE_WIDE(VB) \
+    merge_entry<VB, 0, 1>(), merge_entry<VB, 0, 2>(), merge_entry<VB, 0, 4>(), merge_entry<VB, 2, 1>(), \
+    merge_entry<VB, 2, 2>(), merge_entry<VB, 2, 4>()
 #define RT_SILU_WIDE(VB) \
     silu_entry<VB, 0, 1>(), silu_entry<VB, 0, 2>(), silu_entry<VB, 0, 4>(), silu_entry<VB, 2, 1>(), \
     silu_entry<VB, 2, 2>(), silu_entry<VB, 2, 4>()
@@ -64,6 +79,9 @@ std::vector<rt::KernelEntry> build_entries()
 #elif RT_UNIT_GROUP == 3
         RT_SILU_WIDE(16), RT_SILU_WIDE(8), silu_entry<4, 0, 1>(), silu_entry<4, 0, 4>(), silu_entry<2, 0, 1>(),
         silu_entry<2, 0, 4>()
+#elif RT_UNIT_GROUP == 4
+        RT_MERGE_WIDE(16), RT_MERGE_WIDE(8), merge_entry<4, 0, 1>(), merge_entry<4, 0, 4>(), merge_entry<2, 0, 1>(),
+        merge_entry<2, 0, 4>()
 #else
         entry<0, 0, 1, 1>(), entry<0, 0, 1, 2>(), entry<0, 0, 1, 4>(), entry<0, 0, 4, 4>(), entry<0, 0, 1, 8>(),
         entry<0, 0, 4, 8>(), entry<0, 0, 1, 16>(), entry<0, 0, 4, 16>(), entry<0, 0, 1, 32>(), entry<0, 0, 4, 32>()

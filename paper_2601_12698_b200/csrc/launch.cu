@@ -9,6 +9,7 @@
 #include <unordered_map>
 
 #include "add_rmsnorm_kernel.cuh"
+#include "merge_attn_states_kernel.cuh"
 #include "silu_and_mul_kernel.cuh"
 #include "tuner_internal.h"
 
@@ -267,13 +268,15 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
         plan->reject_reason = kRejectArgs;
         return RT_ERR_DTYPE;
     }
-    if (s->op != RT_OP_ADD_RMSNORM && s->op != RT_OP_SILU_AND_MUL) {
+    if (s->op != RT_OP_ADD_RMSNORM && s->op != RT_OP_SILU_AND_MUL && s->op != RT_OP_MERGE_ATTN_STATES) {
         set_error("op %d is not a kernel of this library", s->op);
         plan->reject_reason = kRejectArgs;
         return RT_ERR_SHAPE;
     }
     plan->op = s->op;
     const bool is_silu = s->op == RT_OP_SILU_AND_MUL;
+    const bool is_merge = s->op == RT_OP_MERGE_ATTN_STATES;
+    const bool no_reduction = is_silu || is_merge;  // element-wise kernels: no reduction axis, no CAP
     const int eb = elem_bytes_of(s->dtype);
     if (s->n_tokens < 0 || s->hidden <= 0 || s->hidden * eb * (is_silu ? 2 : 1) >= (int64_t)1 << 31) {
         set_error("shape n_tokens=%lld hidden=%lld is out of range", (long long)s->n_tokens, (long long)s->hidden);
@@ -311,8 +314,13 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
         plan->reject_reason = kRejectArgs;
         return RT_ERR_INFEASIBLE;
     }
-    if (is_silu && (p->reduce != RT_REDUCE_SHFL || p->cluster_size != 1 || p->stage == RT_STAGE_SMEM_LDG)) {
-        set_error("silu_and_mul has no reduction and no ld.global->shared stage (reduce=%d cluster=%d stage=%d)",
+    if (is_merge && (s->head_dim <= 0 || s->hidden % s->head_dim != 0)) {
+        set_error("head_dim=%d does not divide hidden=%lld", s->head_dim, (long long)s->hidden);
+        plan->reject_reason = kRejectArgs;
+        return RT_ERR_SHAPE;
+    }
+    if (no_reduction && (p->reduce != RT_REDUCE_SHFL || p->cluster_size != 1 || p->stage == RT_STAGE_SMEM_LDG)) {
+        set_error("this kernel has no reduction and no ld.global->shared stage (reduce=%d cluster=%d stage=%d)",
                   p->reduce, p->cluster_size, p->stage);
         plan->reject_reason = kRejectArgs;
         return RT_ERR_INFEASIBLE;
@@ -332,6 +340,11 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
     const int64_t row_bytes = s->hidden * eb;
     if (row_bytes % vb != 0) {
         set_error("row of %lld bytes is not a multiple of vec_bytes=%d", (long long)row_bytes, vb);
+        plan->reject_reason = kRejectAlign;
+        return RT_ERR_ALIGN;
+    }
+    if (is_merge && ((int64_t)s->head_dim * eb) % vb != 0) {
+        set_error("a head of %d bytes is not a multiple of vec_bytes=%d", s->head_dim * eb, vb);
         plan->reject_reason = kRejectAlign;
         return RT_ERR_ALIGN;
     }
@@ -356,6 +369,10 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
     plan->slice_nvec = slice;
     plan->vec_per_thread = (slice + tpr - 1) / tpr;
     plan->cluster = C;
+    if (is_merge) {
+        plan->vec_per_head = (int)((int64_t)s->head_dim * eb / vb);
+        plan->heads = (int)(s->hidden / s->head_dim);
+    }
     plan->block_x = tpr;
     plan->block_y = rpc;
     if ((int64_t)(C - 1) * slice >= plan->nvec && C > 1) {
@@ -365,7 +382,7 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
     }
 
     int cap = 0, unroll = p->unroll;
-    if (p->stage == RT_STAGE_REG && !is_silu) {
+    if (p->stage == RT_STAGE_REG && !no_reduction) {
         cap = next_pow2(plan->vec_per_thread);
         if (unroll > cap) unroll = cap;
     }
@@ -373,13 +390,13 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
     plan->unroll_eff = unroll;
     plan->kernel_index = find_kernel(s->op, s->dtype, vb, p->stage, p->reduce, unroll, cap);
     if (plan->kernel_index < 0) {
-        if (p->stage == RT_STAGE_REG && !is_silu)
+        if (p->stage == RT_STAGE_REG && !no_reduction)
             set_error("a row slice of %d vectors over %d threads needs %d vectors per thread: no register-stage "
                       "instance that large (register budget)", slice, tpr, cap);
         else
             set_error("no compiled instance for dtype=%d vec=%d stage=%d reduce=%d unroll=%d", s->dtype, vb, p->stage,
                       p->reduce, unroll);
-        plan->reject_reason = (p->stage == RT_STAGE_REG && !is_silu) ? kRejectRegisters : kRejectArgs;
+        plan->reject_reason = (p->stage == RT_STAGE_REG && !no_reduction) ? kRejectRegisters : kRejectArgs;
         return RT_ERR_INFEASIBLE;
     }
     const KernelEntry& k = registry()[plan->kernel_index];
@@ -480,6 +497,42 @@ int plan_occupancy(const Plan& plan, const rt_limits* L, int* regs_per_thread)
     const int64_t smem = (int64_t)plan.dyn_smem + (int64_t)plan.static_smem_estimate + L->smem_reserved_per_block;
     blocks = std::min<int64_t>(blocks, L->smem_per_sm / smem);
     return (int)blocks;
+}
+
+int launch_merge_plan(const Plan& plan, const void* v_a, const float* s_a, const void* v_b, const float* s_b, void* v_out,
+                      float* s_out, int64_t n_tokens, cudaStream_t stream)
+{
+    if (n_tokens == 0) return RT_OK;
+    if (plan.op != RT_OP_MERGE_ATTN_STATES) {
+        set_error("plan belongs to another kernel");
+        return RT_ERR_INFEASIBLE;
+    }
+    const KernelEntry& k = registry()[plan.kernel_index];
+    int st = ensure_dynamic_smem(plan.kernel_index, plan.dyn_smem);
+    if (st != RT_OK) return st;
+    MergeArgs a;
+    a.v_a = v_a; a.v_b = v_b; a.s_a = s_a; a.s_b = s_b; a.v_out = v_out; a.s_out = s_out;
+    a.n_tokens = n_tokens;
+    a.nvec = plan.nvec;
+    a.vec_per_head = plan.vec_per_head;
+    a.heads = plan.heads;
+    a.status = device_status_word();
+    if (!a.status) return RT_ERR_CUDA;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(plan.grid_x, 1, 1);
+    cfg.blockDim = dim3(plan.block_x, plan.block_y, 1);
+    cfg.dynamicSmemBytes = plan.dyn_smem;
+    cfg.stream = stream;
+    void* params[] = {&a};
+    cudaError_t e = cudaLaunchKernelExC(&cfg, k.fn, params);
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        set_error("kernel launch failed: %s", cudaGetErrorString(e));
+        return RT_ERR_CUDA;
+    }
+    count_launch();
+    return RT_OK;
 }
 
 int launch_silu_plan(const Plan& plan, const void* x, void* out, int64_t n_tokens, cudaStream_t stream)
@@ -589,7 +642,7 @@ int rmsnorm_template_launch(const rt_params* p, const void* x, const void* r, co
     s.dtype = dtype;
     s.min_ptr_align = n_tokens > 0 ? rt::min_pointer_alignment(x, r, w, y, r_out) : 256;
     s.op = RT_OP_ADD_RMSNORM;
-    s.reserved = 0;
+    s.head_dim = 0;
     rt::Plan plan;
     st = rt::make_plan(&s, p, &L, &plan);
     if (st != RT_OK) return st;
@@ -616,11 +669,47 @@ int silu_and_mul_template_launch(const rt_params* p, const void* x, void* out, i
     s.dtype = dtype;
     s.min_ptr_align = n_tokens > 0 ? rt::min_pointer_alignment(x, out, x, out, x) : 256;
     s.op = RT_OP_SILU_AND_MUL;
-    s.reserved = 0;
+    s.head_dim = 0;
     rt::Plan plan;
     st = rt::make_plan(&s, p, &L, &plan);
     if (st != RT_OK) return st;
     return rt::launch_silu_plan(plan, x, out, n_tokens, (cudaStream_t)stream);
+}
+
+int merge_attn_states_template_launch(const rt_params* p, const void* v_a, const float* s_a, const void* v_b,
+                                      const float* s_b, void* v_out, float* s_out, int64_t n_tokens, int64_t heads,
+                                      int64_t head_dim, int dtype, void* stream)
+{
+    if (!p) {
+        rt::set_error("params is NULL");
+        return RT_ERR_NULL;
+    }
+    if (n_tokens > 0 && (!v_a || !s_a || !v_b || !s_b || !v_out || !s_out)) {
+        rt::set_error("a tensor pointer is NULL");
+        return RT_ERR_NULL;
+    }
+    if (heads <= 0 || head_dim <= 0 || head_dim > 0x7fffffff) {
+        rt::set_error("heads=%lld head_dim=%lld out of range", (long long)heads, (long long)head_dim);
+        return RT_ERR_SHAPE;
+    }
+    if (n_tokens > 0 && (((uintptr_t)s_a | (uintptr_t)s_b | (uintptr_t)s_out) & 3u)) {
+        rt::set_error("the log-sum-exp tensors must be 4-byte aligned");
+        return RT_ERR_ALIGN;
+    }
+    rt_limits L;
+    int st = rt::current_limits(&L);
+    if (st != RT_OK) return st;
+    rt_shape s;
+    s.n_tokens = n_tokens;
+    s.hidden = heads * head_dim;
+    s.dtype = dtype;
+    s.min_ptr_align = n_tokens > 0 ? rt::min_pointer_alignment(v_a, v_b, v_out, v_a, v_b) : 256;
+    s.op = RT_OP_MERGE_ATTN_STATES;
+    s.head_dim = (int32_t)head_dim;
+    rt::Plan plan;
+    st = rt::make_plan(&s, p, &L, &plan);
+    if (st != RT_OK) return st;
+    return rt::launch_merge_plan(plan, v_a, s_a, v_b, s_b, v_out, s_out, n_tokens, (cudaStream_t)stream);
 }
 
 int rt_query_limits(rt_limits* out)

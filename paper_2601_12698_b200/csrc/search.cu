@@ -1,6 +1,7 @@
 // Search(S~, x, Theta_feasible): the correctness gate d(.,.) on the device, the timing protocol, and the
 // guided search (seeds -> coarse grid -> best-first hill-climb -> Top-K re-test), after Algorithm 1
 // (Level 2) and the "Tuning agent" / "Testing agent" roles of the paper.
+#include <cuda_fp16.h>
 #include <math.h>
 #include <string.h>
 
@@ -79,6 +80,54 @@ __global__ void compare_kernel(const unsigned int* __restrict__ got, const unsig
         unsigned long long b2 = 0;
         compare_word<MODE>(tail_got, tail_ref, dtype, tol, b2, worst);
         bad += b2 ? 1 : 0;  // the padded upper halves are equal and add nothing
+    }
+    for (int off = 16; off >= 1; off >>= 1) {
+        bad += __shfl_xor_sync(0xffffffffu, bad, off);
+        worst = max(worst, __shfl_xor_sync(0xffffffffu, worst, off));
+    }
+    if ((threadIdx.x & 31) == 0) {
+        if (bad) atomicAdd(&acc->n_bad, bad);
+        if (worst) atomicMax(&acc->max_bits, worst);
+    }
+}
+
+// Mixed tolerance (outputs that may cancel): pass within `tol` ulps (16-bit) / relative (binary32) OR within
+// `tol_abs` absolutely.  acc->max_bits receives the float bits of the largest absolute difference.
+__device__ __forceinline__ float decode_elem16(unsigned int bits, int dtype)
+{
+    return dtype == RT_BF16 ? __uint_as_float(bits << 16) : __half2float(__ushort_as_half((unsigned short)bits));
+}
+
+__device__ __forceinline__ void mixed_elem(float g, float q, unsigned int ulps, bool use_ulps, double tol, double tol_abs,
+                                           unsigned long long& bad, unsigned int& worst)
+{
+    const bool gn = g != g, qn = q != q;
+    if (gn || qn) {
+        if (!(gn && qn)) { ++bad; worst = 0x7F800000u; }
+        return;
+    }
+    if (g == q) return;
+    const double diff = fabs((double)g - (double)q);
+    const bool ok = diff <= tol_abs || (use_ulps ? (double)ulps <= tol : diff <= tol * fabs((double)q));
+    if (!ok) ++bad;
+    worst = max(worst, __float_as_uint((float)diff));
+}
+
+__global__ void compare_mixed_kernel(const void* __restrict__ got, const void* __restrict__ ref, long long n, int dtype,
+                                     double tol, double tol_abs, CompareAcc* acc)
+{
+    unsigned long long bad = 0;
+    unsigned int worst = 0;
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+        if (dtype == RT_FP32) {
+            mixed_elem(((const float*)got)[i], ((const float*)ref)[i], 0u, false, tol, tol_abs, bad, worst);
+        } else {
+            const unsigned int gb = ((const unsigned short*)got)[i], qb = ((const unsigned short*)ref)[i];
+            const unsigned int nan_above = dtype == RT_BF16 ? 0x7F80u : 0x7C00u;
+            mixed_elem(decode_elem16(gb, dtype), decode_elem16(qb, dtype), ulp_distance16(gb, qb, nan_above), true, tol,
+                       tol_abs, bad, worst);
+        }
     }
     for (int off = 16; off >= 1; off >>= 1) {
         bad += __shfl_xor_sync(0xffffffffu, bad, off);
@@ -187,6 +236,18 @@ int enqueue_compare(const void* got, const void* ref, int64_t n, int dtype, int 
     return RT_OK;
 }
 
+int enqueue_compare_mixed(const void* got, const void* ref, int64_t n, int dtype, double tol, double tol_abs,
+                          CompareAcc* acc, cudaStream_t stream)
+{
+    const int threads = 256;
+    const long long want = (n + threads * 8 - 1) / (threads * 8);
+    const int blocks = (int)std::max<long long>(1, std::min<long long>(want, 148 * 16));
+    compare_mixed_kernel<<<blocks, threads, 0, stream>>>(got, ref, n, dtype, tol, tol_abs, acc);
+    RT_CUDA_OK(cudaGetLastError());
+    count_launch();
+    return RT_OK;
+}
+
 int check_compare_args(const void* got, const void* ref, int64_t n, int dtype, int mode)
 {
     if (!got || !ref) {
@@ -268,23 +329,38 @@ struct DeviceEvaluator : Evaluator {
         st = get_scratch(&sc);
         if (st != RT_OK) return st;
         const bool is_silu = shape.op == RT_OP_SILU_AND_MUL;
+        const bool is_merge = shape.op == RT_OP_MERGE_ATTN_STATES;
+        const size_t lse_bytes = is_merge ? (size_t)shape.n_tokens * plan.heads * sizeof(float) : 0;  // one s tensor
         RT_CUDA_OK(cudaMemsetAsync(ws.y, 0xFF, set_bytes, stream));
-        if (!is_silu) RT_CUDA_OK(cudaMemsetAsync(ws.r_out, 0xFF, set_bytes, stream));
+        if (is_merge) RT_CUDA_OK(cudaMemsetAsync(ws.r_out, 0xFF, lse_bytes, stream));
+        else if (!is_silu) RT_CUDA_OK(cudaMemsetAsync(ws.r_out, 0xFF, set_bytes, stream));
         RT_CUDA_OK(cudaMemsetAsync(sc->dev, 0, 2 * sizeof(CompareAcc), stream));
-        st = is_silu ? launch_silu_plan(plan, ws.x, ws.y, shape.n_tokens, stream)
-                     : launch_plan(plan, ws.x, ws.r, ws.w, ws.y, ws.r_out, shape.n_tokens, shape.hidden, ws.eps, stream);
+        if (is_merge)
+            st = launch_merge_plan(plan, ws.x, (const float*)ws.w, ws.r, (const float*)ws.aux, ws.y, (float*)ws.r_out,
+                                   shape.n_tokens, stream);
+        else
+            st = is_silu ? launch_silu_plan(plan, ws.x, ws.y, shape.n_tokens, stream)
+                         : launch_plan(plan, ws.x, ws.r, ws.w, ws.y, ws.r_out, shape.n_tokens, shape.hidden, ws.eps, stream);
         if (st != RT_OK) {
             rec->status = st;
             return RT_OK;
         }
         const int y_mode = shape.dtype == RT_FP32 ? RT_CMP_REL32 : RT_CMP_ULP16;
         const double y_tol = shape.dtype == RT_FP32 ? 1e-5 : 2.0;
-        if (!is_silu) {
-            st = enqueue_compare(ws.r_out, ws.r_ref, n_ref * shape.hidden, shape.dtype, RT_CMP_BITS, 0.0, sc->dev, stream);
+        if (is_merge) {
+            // outputs that may cancel: 2 ulp / 1e-5 relative, or 1e-5 absolute; the merged log-sum-exp likewise
+            st = enqueue_compare_mixed(ws.r_out, ws.r_ref, n_ref * plan.heads, RT_FP32, 1e-5, 1e-5, sc->dev, stream);
+            if (st != RT_OK) return st;
+            st = enqueue_compare_mixed(ws.y, ws.y_ref, n_ref * shape.hidden, shape.dtype, y_tol, 1e-5, sc->dev + 1, stream);
+            if (st != RT_OK) return st;
+        } else {
+            if (!is_silu) {
+                st = enqueue_compare(ws.r_out, ws.r_ref, n_ref * shape.hidden, shape.dtype, RT_CMP_BITS, 0.0, sc->dev, stream);
+                if (st != RT_OK) return st;
+            }
+            st = enqueue_compare(ws.y, ws.y_ref, n_ref * shape.hidden, shape.dtype, y_mode, y_tol, sc->dev + 1, stream);
             if (st != RT_OK) return st;
         }
-        st = enqueue_compare(ws.y, ws.y_ref, n_ref * shape.hidden, shape.dtype, y_mode, y_tol, sc->dev + 1, stream);
-        if (st != RT_OK) return st;
         (void)ref_bytes;
         RT_CUDA_OK(cudaMemcpyAsync(sc->host, sc->dev, 2 * sizeof(CompareAcc), cudaMemcpyDeviceToHost, stream));
         cudaError_t e = cudaStreamSynchronize(stream);
@@ -294,8 +370,8 @@ struct DeviceEvaluator : Evaluator {
         }
         rec->r_bad = (int64_t)sc->host[0].n_bad;
         rec->y_bad = (int64_t)sc->host[1].n_bad;
-        if (shape.dtype == RT_FP32)
-            rec->y_max_rel = (float)acc_max_err(sc->host[1], RT_CMP_REL32);
+        if (shape.dtype == RT_FP32 || is_merge)
+            rec->y_max_rel = (float)acc_max_err(sc->host[1], RT_CMP_REL32);  // merge: largest absolute difference
         else
             rec->y_max_ulp = (int32_t)sc->host[1].max_bits;
         if (p.stage == RT_STAGE_SMEM_TMA) {
@@ -316,6 +392,12 @@ struct DeviceEvaluator : Evaluator {
         const int sets = ws.ring_sets > 0 ? ws.ring_sets : 1;
         auto launch_set = [&](int k) {
             const size_t off = (size_t)(k % sets) * (size_t)ws.ring_stride_bytes;
+            if (is_merge) {
+                const size_t so = (size_t)(k % sets) * lse_bytes;
+                return launch_merge_plan(plan, (const char*)ws.x + off, (const float*)((const char*)ws.w + so),
+                                         (const char*)ws.r + off, (const float*)((const char*)ws.aux + so),
+                                         (char*)ws.y + off, (float*)((char*)ws.r_out + so), shape.n_tokens, stream);
+            }
             if (is_silu)  // the input rows are twice as long as the output rows
                 return launch_silu_plan(plan, (const char*)ws.x + 2 * off, (char*)ws.y + off, shape.n_tokens, stream);
             return launch_plan(plan, (const char*)ws.x + off, (const char*)ws.r + off, ws.w, (char*)ws.y + off,
@@ -699,7 +781,8 @@ int check_workspace(const rt_shape* s, const rt_workspace* ws)
         return RT_ERR_NULL;
     }
     const bool is_silu = s->op == RT_OP_SILU_AND_MUL;
-    if (!ws->x || !ws->y || !ws->y_ref || (!is_silu && (!ws->r || !ws->w || !ws->r_out || !ws->r_ref))) {
+    if (!ws->x || !ws->y || !ws->y_ref || (!is_silu && (!ws->r || !ws->w || !ws->r_out || !ws->r_ref)) ||
+        (s->op == RT_OP_MERGE_ATTN_STATES && !ws->aux)) {
         set_error("a workspace pointer is NULL");
         return RT_ERR_NULL;
     }
@@ -752,6 +835,32 @@ int tuner_compare(const void* got, const void* ref, int64_t n, int dtype, int mo
     RT_CUDA_OK(cudaMemcpyAsync(sc->host, sc->dev, sizeof(rt::CompareAcc), cudaMemcpyDeviceToHost, s));
     RT_CUDA_OK(cudaStreamSynchronize(s));
     *max_err = rt::acc_max_err(sc->host[0], mode);
+    *n_bad = (int64_t)sc->host[0].n_bad;
+    return RT_OK;
+}
+
+int tuner_compare_mixed(const void* got, const void* ref, int64_t n, int dtype, double tol, double tol_abs,
+                        double* max_abs, int64_t* n_bad, void* stream)
+{
+    int st = rt::check_compare_args(got, ref, n, dtype, RT_CMP_BITS);
+    if (st != RT_OK) return st;
+    if (!max_abs || !n_bad) {
+        rt::set_error("tuner_compare_mixed: NULL result pointer");
+        return RT_ERR_NULL;
+    }
+    *max_abs = 0.0;
+    *n_bad = 0;
+    if (n == 0) return RT_OK;
+    rt::Scratch* sc;
+    st = rt::get_scratch(&sc);
+    if (st != RT_OK) return st;
+    cudaStream_t s = (cudaStream_t)stream;
+    RT_CUDA_OK(cudaMemsetAsync(sc->dev, 0, sizeof(rt::CompareAcc), s));
+    st = rt::enqueue_compare_mixed(got, ref, n, dtype, tol, tol_abs, sc->dev, s);
+    if (st != RT_OK) return st;
+    RT_CUDA_OK(cudaMemcpyAsync(sc->host, sc->dev, sizeof(rt::CompareAcc), cudaMemcpyDeviceToHost, s));
+    RT_CUDA_OK(cudaStreamSynchronize(s));
+    *max_abs = rt::acc_max_err(sc->host[0], RT_CMP_REL32);
     *n_bad = (int64_t)sc->host[0].n_bad;
     return RT_OK;
 }

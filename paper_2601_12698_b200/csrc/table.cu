@@ -140,7 +140,7 @@ int rmsnorm_launch_auto(const rt_spec_entry* table, int32_t n_entries, const rt_
     s.dtype = dtype;
     s.min_ptr_align = n_tokens > 0 ? rt::min_pointer_alignment(x, r, w, y, r_out) : 256;
     s.op = RT_OP_ADD_RMSNORM;
-    s.reserved = 0;
+    s.head_dim = 0;
     rt_params theta;
     int st = tuner_table_lookup(table, n_entries, general, &s, nullptr, &theta, nullptr);
     if (st != RT_OK) return st;

@@ -29,7 +29,7 @@ import numpy as np
 import torch
 
 ROWS_PER_BLOCK = 64
-TENSOR_X, TENSOR_R, TENSOR_W, TENSOR_GATE_UP = 0, 1, 2, 3
+TENSOR_X, TENSOR_R, TENSOR_W, TENSOR_GATE_UP, TENSOR_LSE_A, TENSOR_LSE_B = 0, 1, 2, 3, 4, 5
 
 TORCH_DTYPES = {"bf16": torch.bfloat16, "fp16": torch.float16, "fp32": torch.float32}
 DTYPE_CODES = {"bf16": 0, "fp16": 1, "fp32": 2}
@@ -54,7 +54,8 @@ class Workload:
     seed: int
     dist: Dist = field(default_factory=Dist)
     eps: float = 1e-6
-    op: str = "add_rmsnorm"  # or "silu_and_mul" (hidden is then d, the output width)
+    op: str = "add_rmsnorm"  # "silu_and_mul": hidden is d, the output width; "merge_attn_states": hidden = heads * head_dim
+    head_dim: int = 0
 
     @property
     def elements(self) -> int:
@@ -67,12 +68,14 @@ class Workload:
         b = DTYPE_BYTES[self.dtype]
         if self.op == "silu_and_mul":
             return 3 * b * self.elements
+        if self.op == "merge_attn_states":  # v_a, v_b in, v_out out; s_a, s_b in, s_out out (binary32 per head)
+            return 3 * b * self.elements + 3 * 4 * self.n_tokens * (self.hidden // self.head_dim)
         return 4 * b * self.elements + b * self.hidden
 
     @property
     def nominal_bytes(self) -> int:
         """add_rmsnorm: three reads and two writes per element (w counted as a full stream)."""
-        if self.op == "silu_and_mul":
+        if self.op != "add_rmsnorm":
             return self.algorithmic_bytes
         return 5 * DTYPE_BYTES[self.dtype] * self.elements
 
@@ -101,6 +104,10 @@ def workloads() -> dict[str, Workload]:
     add(Workload("silu_fp32_2048x8192", "fp32", 2048, 8192, seed=6, dist=gate, op="silu_and_mul"))
     add(Workload("silu_fp32_128x11008", "fp32", 128, 11008, seed=6, dist=gate, op="silu_and_mul"))
     add(Workload("silu_bf16_64x11008", "bf16", 64, 11008, seed=6, dist=gate, op="silu_and_mul"))
+    # merge_attn_states: the paper's (n, h, d) shapes in bf16, and a bandwidth case
+    for n, h, d in ((512, 32, 256), (512, 40, 128), (768, 32, 256), (768, 40, 128), (512, 64, 128)):
+        add(Workload(f"merge_bf16_{n}x{h}x{d}", "bf16", n, h * d, seed=7, op="merge_attn_states", head_dim=d))
+    add(Workload("merge_bf16_32768x32x128", "bf16", 32768, 32 * 128, seed=7, op="merge_attn_states", head_dim=128))
     return out
 
 
@@ -172,7 +179,26 @@ def make_gate_up(row_begin: int, row_end: int, d: int, dtype: str, seed: int, di
     return make_rows(TENSOR_GATE_UP, row_begin, row_end, 2 * d, dtype, seed, dist, threads).contiguous()
 
 
+def make_lse(tensor_id: int, row_begin: int, row_end: int, heads: int, seed: int, mean: float = 4.0,
+             sigma: float = 2.0) -> torch.Tensor:
+    """Rows of a float32 [T, heads] log-sum-exp tensor: N(mean, sigma), the spread two key blocks of unequal
+    length typically show."""
+    t = make_rows(tensor_id, row_begin, row_end, heads, "fp32", seed, Dist(sigma=sigma), threads=1).contiguous()
+    return (t + mean).contiguous()
+
+
+def make_merge_inputs(row_begin: int, row_end: int, heads: int, head_dim: int, dtype: str, seed: int, threads: int = 8):
+    """(v_a, s_a, v_b, s_b): partial outputs N(0, 1) of shape [T, heads, head_dim], float32 log-sum-exps [T, heads]."""
+    n = row_end - row_begin
+    v_a = make_rows(TENSOR_X, row_begin, row_end, heads * head_dim, dtype, seed, Dist(), threads).contiguous()
+    v_b = make_rows(TENSOR_R, row_begin, row_end, heads * head_dim, dtype, seed, Dist(), threads).contiguous()
+    return (v_a.view(n, heads, head_dim), make_lse(TENSOR_LSE_A, row_begin, row_end, heads, seed),
+            v_b.view(n, heads, head_dim), make_lse(TENSOR_LSE_B, row_begin, row_end, heads, seed))
+
+
 def make_workload_inputs(wl: Workload, threads: int = 8):
+    if wl.op == "merge_attn_states":
+        return make_merge_inputs(0, wl.n_tokens, wl.hidden // wl.head_dim, wl.head_dim, wl.dtype, wl.seed, threads)
     if wl.op == "silu_and_mul":
         return (make_gate_up(0, wl.n_tokens, wl.hidden, wl.dtype, wl.seed, wl.dist, threads),)
     return make_inputs(wl.n_tokens, wl.hidden, wl.dtype, wl.seed, wl.dist, threads)

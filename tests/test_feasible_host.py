@@ -109,3 +109,18 @@ def test_silu_and_mul_grid_has_no_reduction_axis(L):
     f = B.tuner_derive_feasible(B.shape_of(8, 3073, "fp16", op=B.RT_OP_SILU_AND_MUL), L)
     assert f and {t.vec_bytes for t in f} == {2} and {t.stage for t in f} == {0}
     assert B.tuner_check_params(B.shape_of(8, 4096, "bf16", op=7), B.make_params(), L) == B.RT_ERR_SHAPE
+
+
+def test_merge_attn_states_grid(L):
+    s = B.shape_of(512, 40 * 128, "bf16", op=B.RT_OP_MERGE_ATTN_STATES, head_dim=128)
+    f = B.tuner_derive_feasible(s, L)
+    assert f and {t.stage for t in f} == {0, 2} and {t.reduce for t in f} == {0} and {t.vec_bytes for t in f} == {16, 8}
+    assert all(B.tuner_check_params(s, t, L) == B.RT_OK for t in f)
+    # a vector may not straddle two heads: heads of 66 bf16 elements (132 bytes) allow 4-byte vectors only
+    f = B.tuner_derive_feasible(B.shape_of(4, 7 * 66, "bf16", op=B.RT_OP_MERGE_ATTN_STATES, head_dim=66), L)
+    assert f and {t.vec_bytes for t in f} == {4}
+    assert B.tuner_check_params(B.shape_of(4, 7 * 66, "bf16", op=B.RT_OP_MERGE_ATTN_STATES, head_dim=66),
+                                B.make_params(vec_bytes=8), L) == B.RT_ERR_ALIGN
+    # head_dim must divide hidden
+    assert B.tuner_check_params(B.shape_of(4, 1000, "bf16", op=B.RT_OP_MERGE_ATTN_STATES, head_dim=128), B.make_params(), L) == B.RT_ERR_SHAPE
+    assert B.tuner_check_params(B.shape_of(4, 1024, "bf16", op=B.RT_OP_MERGE_ATTN_STATES, head_dim=0), B.make_params(), L) == B.RT_ERR_SHAPE
