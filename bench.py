@@ -29,7 +29,12 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "fused_add_rmsnorm_hbm_gbs"
-METRICS = {"add_rmsnorm": METRIC, "silu_and_mul": "silu_and_mul_hbm_gbs"}
+METRICS = {"add_rmsnorm": METRIC, "silu_and_mul": "silu_and_mul_hbm_gbs", "merge_attn_states": "merge_attn_states_hbm_gbs"}
+BYTES_LABEL = {"add_rmsnorm": "algorithmic: 2 reads + 2 writes per element + w once",
+               "silu_and_mul": "algorithmic: 2 reads + 1 write per output element",
+               "merge_attn_states": "algorithmic: 2 reads + 1 write per element + 3 binary32 per (token, head)"}
+KERNEL_NAME = {"add_rmsnorm": "add_rmsnorm_kernel", "silu_and_mul": "silu_and_mul_kernel",
+               "merge_attn_states": "merge_attn_states_kernel"}
 UNIT = "GB/s"
 DEFAULT_WORKLOAD = "c3_prefill_bf16_16384x8192"
 FALLBACK_HBM_GBS = 6650.0  # used only when MEASURED_PEAKS.json is absent
@@ -136,7 +141,12 @@ def run_reference(args) -> None:
     cores = os.cpu_count() or 1
     is_silu = wl.op == "silu_and_mul"
 
+    is_merge = wl.op == "merge_attn_states"
+
     def sample(n_rows):
+        if is_merge:
+            va, sa, vb, sb = synth.make_merge_inputs(0, n_rows, wl.hidden // wl.head_dim, wl.head_dim, wl.dtype, wl.seed)
+            return lambda: oracle.merge_attn_states(va, sa, vb, sb)
         if is_silu:
             xs = synth.make_gate_up(0, n_rows, wl.hidden, wl.dtype, wl.seed, wl.dist)
             return lambda: oracle.silu_and_mul(xs, threads=cores)
@@ -160,7 +170,11 @@ def run_reference(args) -> None:
         run()
     elapsed = time.perf_counter() - t0
     b = synth.DTYPE_BYTES[wl.dtype]
-    step_bytes = 3 * b * rows * wl.hidden if is_silu else 4 * b * rows * wl.hidden + b * wl.hidden
+    if is_merge:
+        cores = 1  # this oracle is single-threaded
+        step_bytes = 3 * b * rows * wl.hidden + 12 * rows * (wl.hidden // wl.head_dim)
+    else:
+        step_bytes = 3 * b * rows * wl.hidden if is_silu else 4 * b * rows * wl.hidden + b * wl.hidden
     value = step_bytes * args.steps / elapsed / 1e9
     sample = f"first {rows} of {wl.n_tokens} rows of {wl.name} per step, {cores} threads"
     line = {
@@ -168,8 +182,7 @@ def run_reference(args) -> None:
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": elapsed * 1e3 / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
         "config": {"workload": wl.name, "n_tokens": wl.n_tokens, "hidden": wl.hidden, "sample_rows_per_step": rows,
-                   "bytes": ("algorithmic: 2 reads + 1 write per output element" if is_silu else
-                             "algorithmic: 2 reads + 2 writes per element + w once")},
+                   "bytes": BYTES_LABEL[wl.op]},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -196,10 +209,17 @@ def run_ours(args) -> None:
     T, H = wl.n_tokens, wl.hidden
 
     is_silu = wl.op == "silu_and_mul"
-    op_code = B.RT_OP_SILU_AND_MUL if is_silu else B.RT_OP_ADD_RMSNORM
+    is_merge = wl.op == "merge_attn_states"
+    op_code = {"add_rmsnorm": B.RT_OP_ADD_RMSNORM, "silu_and_mul": B.RT_OP_SILU_AND_MUL,
+               "merge_attn_states": B.RT_OP_MERGE_ATTN_STATES}[wl.op]
+    heads = H // wl.head_dim if is_merge else 0
+    sa = sb = None
 
     # Inputs: this rank's rows of the N-times larger job; w replicated.
-    if is_silu:
+    if is_merge:
+        va, sa, vb, sb = synth.make_merge_inputs(shard.row_begin, shard.row_end, heads, wl.head_dim, wl.dtype, wl.seed)
+        x, r, w = va.view(T, H), vb.view(T, H), None
+    elif is_silu:
         x = synth.make_gate_up(shard.row_begin, shard.row_end, H, wl.dtype, wl.seed, wl.dist)
         r = w = None
     else:
@@ -213,7 +233,11 @@ def run_ours(args) -> None:
     cores = os.cpu_count() or 1
     oracle.build()
     t0 = time.perf_counter()
-    if is_silu:
+    if is_merge:
+        cores = 1  # this oracle is single-threaded
+        v_ref, r_ref = oracle.merge_attn_states(va, sa, vb, sb)  # r_ref holds the merged log-sum-exps
+        y_ref = v_ref.view(T, H)
+    elif is_silu:
         y_ref, r_ref = oracle.silu_and_mul(x, threads=cores), None
     else:
         y_ref, r_ref = oracle.add_rmsnorm(x, r, w, wl.eps, threads=cores)
@@ -234,17 +258,23 @@ def run_ours(args) -> None:
     rd = ring(r) if r is not None else None
     wd = w.to(device) if w is not None else None
     yd = torch.empty((sets, T, H), dtype=xd.dtype, device=device)
-    od = torch.empty_like(yd) if not is_silu else None
+    od = torch.empty_like(yd) if not (is_silu or is_merge) else None
+    sad = sbd = None
+    if is_merge:
+        sad, sbd = ring(sa), ring(sb)
+        od = torch.empty_like(sad)  # s_out
     y_ref_d = y_ref.to(device)
     r_ref_d = r_ref.to(device) if r_ref is not None else None
     set_bytes = T * H * b  # one output-sized set; silu_and_mul's input sets are twice as long
     live = [t for t in (xd, rd, wd, yd, od) if t is not None]
     align = B._ptr_align(*live)
-    shape = B.shape_of(T, H, wl.dtype, align if set_bytes % 256 == 0 else min(align, set_bytes & -set_bytes), op=op_code)
+    shape = B.shape_of(T, H, wl.dtype, align if set_bytes % 256 == 0 else min(align, set_bytes & -set_bytes), op=op_code,
+                       head_dim=wl.head_dim)
     # warm: the paper's protocol (the same buffers every launch); cold: rotating over the ring
-    ws = B.make_workspace(xd, rd, wd, yd, od, y_ref_d, r_ref_d, wl.eps, stream=stream)
-    ws_cold = B.make_workspace(xd, rd, wd, yd, od, y_ref_d, r_ref_d, wl.eps, ring_sets=sets,
-                               ring_stride_bytes=set_bytes, stream=stream)
+    w_or_sa = sad if is_merge else wd
+    ws = B.make_workspace(xd, rd, w_or_sa, yd, od, y_ref_d, r_ref_d, wl.eps, n_ref_tokens=T, stream=stream, aux=sbd)
+    ws_cold = B.make_workspace(xd, rd, w_or_sa, yd, od, y_ref_d, r_ref_d, wl.eps, n_ref_tokens=T, ring_sets=sets,
+                               ring_stride_bytes=set_bytes, stream=stream, aux=sbd)
     use_graph = resident  # launch gaps would otherwise dominate kernels of a few microseconds
 
     # The tuner (not timed): exhaustive sweep as ground truth, then the guided search with a stated budget.
@@ -326,7 +356,18 @@ def run_ours(args) -> None:
     # Step k works on set k mod sets (one set when the workload exceeds L2 by itself).
     theta_ref = B.byref(theta)
     dtype_code, stream_ptr, eps = B.DTYPE_CODES[wl.dtype], stream.cuda_stream, wl.eps
-    if is_silu:
+    if is_merge:
+        launch = B.lib.merge_attn_states_template_launch
+        ptrs = [(xd[k].data_ptr(), sad[k].data_ptr(), rd[k].data_ptr(), sbd[k].data_ptr(), yd[k].data_ptr(),
+                 od[k].data_ptr()) for k in range(sets)]
+        head_dim = wl.head_dim
+
+        def step(k):
+            pa, psa, pb, psb, po, pso = ptrs[k % sets]
+            st = launch(theta_ref, pa, psa, pb, psb, po, pso, T, heads, head_dim, dtype_code, stream_ptr)
+            if st != 0:
+                raise B.TunerError(st, "merge_attn_states_template_launch")
+    elif is_silu:
         launch = B.lib.silu_and_mul_template_launch
         ptrs = [(xd[k].data_ptr(), yd[k].data_ptr()) for k in range(sets)]
 
@@ -366,8 +407,14 @@ def run_ours(args) -> None:
 
     # Parity of what was just timed, against the oracle (all rows; r' bit-exact, y within tolerance).
     last = (args.steps - 1) % sets  # the set the last timed step wrote
-    r_bad = 0 if is_silu else B.tuner_compare(od[last], r_ref_d, B.RT_CMP_BITS, stream=stream)[1]
-    if wl.dtype == "fp32":
+    if is_merge:
+        r_bad = B.tuner_compare_mixed(od[last], r_ref_d, 1e-5, 1e-5, stream=stream)[1]
+        y_worst, y_bad = B.tuner_compare_mixed(yd[last], y_ref_d, 1e-5 if wl.dtype == "fp32" else 2.0, 1e-5, stream=stream)
+    else:
+        r_bad = 0 if is_silu else B.tuner_compare(od[last], r_ref_d, B.RT_CMP_BITS, stream=stream)[1]
+    if is_merge:
+        pass
+    elif wl.dtype == "fp32":
         y_worst, y_bad = B.tuner_compare(yd[last], y_ref_d, B.RT_CMP_REL32, 1e-5, stream=stream)
     else:
         y_worst, y_bad = B.tuner_compare(yd[last], y_ref_d, B.RT_CMP_ULP16, 2.0, stream=stream)
@@ -379,7 +426,19 @@ def run_ours(args) -> None:
     # entry point (chunked, copies overlapped with the kernel); silu_and_mul has no such entry point, so its
     # end-to-end step is copy in, launch, copy out on the launch stream.
     e2e_steps = max(3, min(args.steps, args.e2e_steps))
-    if is_silu:
+    if is_merge:
+        xp, rp, sap, sbp = x.pin_memory(), r.pin_memory(), sa.pin_memory(), sb.pin_memory()
+        yp, sop = torch.empty((T, H), dtype=x.dtype).pin_memory(), torch.empty((T, heads)).pin_memory()
+        h2d_bytes, d2h_bytes = 2 * T * H * b + 8 * T * heads, T * H * b + 4 * T * heads
+
+        def e2e_step():
+            with torch.cuda.stream(stream):
+                xd[0].copy_(xp, non_blocking=True); rd[0].copy_(rp, non_blocking=True)
+                sad[0].copy_(sap, non_blocking=True); sbd[0].copy_(sbp, non_blocking=True)
+                step(0)
+                yp.copy_(yd[0], non_blocking=True); sop.copy_(od[0], non_blocking=True)
+            stream.synchronize()
+    elif is_silu:
         xp = x.pin_memory()
         yp = torch.empty((T, H), dtype=x.dtype).pin_memory()
         h2d_bytes, d2h_bytes = 2 * T * H * b, T * H * b
@@ -407,7 +466,13 @@ def run_ours(args) -> None:
     e2e_ms = dp.max_over_ranks((time.perf_counter() - t0) * 1e3, device)
     dp.barrier(device)
     e2e_value = dp.whole_job_rate(wl.algorithmic_bytes, e2e_steps, world, e2e_ms) / 1e9
-    if oracle.compare_y(yp[-64:], y_ref[-64:], tol_rel=1e-5)[1] or (not is_silu and oracle.bit_mismatches(op[:64], r_ref[:64])):
+    if is_merge:
+        e2e_bad = (oracle.compare_mixed(yp[-64:], y_ref[-64:], tol=1e-5 if wl.dtype == "fp32" else 2.0, tol_abs=1e-5)[1]
+                   or oracle.compare_mixed(sop[:64], r_ref[:64], tol=1e-5, tol_abs=1e-5)[1])
+    else:
+        e2e_bad = (oracle.compare_y(yp[-64:], y_ref[-64:], tol_rel=1e-5)[1]
+                   or (not is_silu and oracle.bit_mismatches(op[:64], r_ref[:64])))
+    if e2e_bad:
         raise RuntimeError("end-to-end path fails parity")
 
     if rank == 0:
@@ -425,13 +490,12 @@ def run_ours(args) -> None:
             "config": {"workload": wl.name, "n_tokens_per_gpu": T, "hidden": H, "eps": wl.eps,
                        "l2": ("inputs_exceed_l2" if not resident else
                               f"ring of {sets} input/output sets ({sets * wl.algorithmic_bytes >> 20} MiB) exceeds L2"),
-                       "bytes": ("algorithmic: 2 reads + 1 write per output element" if is_silu else
-                                 "algorithmic: 2 reads + 2 writes per element + w once"),
+                       "bytes": BYTES_LABEL[wl.op],
                        "parallelism": f"rows x{world}, no collective", "theta": theta_dict(theta)},
             "value_nominal_5_access_gbs": value * wl.nominal_bytes / wl.algorithmic_bytes,
             "frac_of_8TBs": value / world / NOMINAL_HBM_GBS,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": UNIT, "frac": achieved / peak,
-                         "traffic": traffic, "peak_kind": f"of {peak_kind}", "kernel": "silu_and_mul_kernel" if is_silu else "add_rmsnorm_kernel",
+                         "traffic": traffic, "peak_kind": f"of {peak_kind}", "kernel": KERNEL_NAME[wl.op],
                          "algorithmic_bytes_per_launch": wl.algorithmic_bytes},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d_bytes,
                     "d2h_bytes_per_step": d2h_bytes, "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},

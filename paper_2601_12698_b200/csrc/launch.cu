@@ -516,6 +516,9 @@ int launch_merge_plan(const Plan& plan, const void* v_a, const float* s_a, const
     a.nvec = plan.nvec;
     a.vec_per_head = plan.vec_per_head;
     a.heads = plan.heads;
+    a.head_shift = -1;
+    for (int sh = 0; sh < 31; ++sh)
+        if ((1 << sh) == plan.vec_per_head) a.head_shift = sh;
     a.status = device_status_word();
     if (!a.status) return RT_ERR_CUDA;
     cudaLaunchConfig_t cfg;

@@ -26,24 +26,28 @@ struct MergeArgs {
     int nvec;           // vectors of VB bytes in one token row (h * d elements)
     int vec_per_head;   // vectors in one head (d elements)
     int heads;
+    int head_shift;     // log2(vec_per_head) when it is a power of two, else -1
     int* status;        // device status word
 };
 
-// Normalised weights of the two parts and the merged log-sum-exp of one (token, head).
-__device__ __forceinline__ void merge_weights(float sa, float sb, float& wa, float& wb, float& s)
+// Normalised weights of the two parts of one (token, head), and D = w_a + w_b before normalisation.
+// e^x through ex2.approx, 1/D through rcp.approx: the weights carry a relative error of about 1e-6, far
+// inside the output tolerance; e^0 = 1, e^-inf = 0 and 1/1 = 1 come out exactly, so an empty part returns the
+// other part bit for bit.  Both parts empty (m = -inf): both weights are zero.
+__device__ __forceinline__ void merge_weights(float sa, float sb, float& wa, float& wb, float& m, float& d)
 {
-    const float m = fmaxf(sa, sb);
-    if (m == -INFINITY) {  // both parts empty
+    m = fmaxf(sa, sb);
+    if (m == -INFINITY) {
         wa = 0.f;
         wb = 0.f;
-        s = -INFINITY;
+        d = 0.f;
         return;
     }
-    const float ea = expf(sa - m), eb = expf(sb - m);
-    const float d = ea + eb;  // in [1, 2]
-    wa = ea / d;
-    wb = eb / d;
-    s = m + logf(d);
+    const float ea = exp2f((sa - m) * 1.4426950408889634f), eb = exp2f((sb - m) * 1.4426950408889634f);
+    d = ea + eb;  // in [1, 2]
+    const float inv = __fdividef(1.0f, d);
+    wa = ea * inv;
+    wb = eb * inv;
 }
 
 template <typename T, int VB, int STAGE, int U>
@@ -111,7 +115,7 @@ __global__ void merge_attn_states_kernel(const MergeArgs a)
         for (int u = 0; u < U; ++u) {
             const int v = v0 + u * tpr;
             if (v < n) {
-                const int head = v / a.vec_per_head;
+                const int head = a.head_shift >= 0 ? (v >> a.head_shift) : (v / a.vec_per_head);
                 fa[u] = __ldg(sa + head);
                 fb[u] = __ldg(sb + head);
             }
@@ -120,10 +124,11 @@ __global__ void merge_attn_states_kernel(const MergeArgs a)
         for (int u = 0; u < U; ++u) {
             const int v = v0 + u * tpr;
             if (v < n) {
-                float wa, wb, s;
-                merge_weights(fa[u], fb[u], wa, wb, s);
-                const int head = v / a.vec_per_head;
-                if (v - head * a.vec_per_head == 0) so[head] = s;  // the head's first vector writes s_out
+                float wa, wb, m, d;
+                merge_weights(fa[u], fb[u], wa, wb, m, d);
+                const int head = a.head_shift >= 0 ? (v >> a.head_shift) : (v / a.vec_per_head);
+                if (v - head * a.vec_per_head == 0)  // the head's first vector writes the merged log-sum-exp
+                    so[head] = d > 0.f ? m + logf(d) : -INFINITY;
                 float xf[EPV], yf[EPV], of[EPV];
                 C::unpack(av[u], xf);
                 C::unpack(bv[u], yf);
