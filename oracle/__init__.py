@@ -1,7 +1,7 @@
 """CPU oracles of the tuned kernels (test infrastructure only).
 
 Thin ctypes wrapper over ``add_rmsnorm_oracle.c``, ``silu_and_mul_oracle.c`` and
-``merge_attn_states_oracle.c``;
+``merge_attn_states_oracle.c`` / ``add_rmsnorm_fp8_oracle.c``;
 all arithmetic is in the C files (``selection.py`` holds the plain-Python oracle
 of the general-configuration choice).  Only the tests, the smoke check and the benchmark's CPU-baseline leg may
 import this package.  It imports nothing from the CUDA package and shares no
@@ -24,7 +24,8 @@ BF16, FP16, FP32 = 0, 1, 2
 DTYPE_NAMES = {BF16: "bf16", FP16: "fp16", FP32: "fp32"}
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-SOURCES = ("add_rmsnorm_oracle.c", "silu_and_mul_oracle.c", "merge_attn_states_oracle.c")
+SOURCES = ("add_rmsnorm_oracle.c", "silu_and_mul_oracle.c", "merge_attn_states_oracle.c",
+           "add_rmsnorm_fp8_oracle.c")
 HEADERS = ("number_formats.h",)
 _LIB = os.path.join(_HERE, "liboracle.so")
 _lock = threading.Lock()
@@ -77,6 +78,14 @@ def _bind(path: str):
     lib.oracle_mixed_compare.argtypes = [vp, vp, i64, ctypes.c_int, ctypes.c_double, ctypes.c_double,
                                          ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i64)]
     lib.oracle_mixed_compare.restype = None
+    lib.oracle_decode_e4m3.argtypes = [vp, vp, i64]
+    lib.oracle_decode_e4m3.restype = None
+    lib.oracle_encode_e4m3.argtypes = [vp, vp, i64]
+    lib.oracle_encode_e4m3.restype = None
+    lib.oracle_add_rmsnorm_fp8.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, ctypes.c_float, ctypes.c_int]
+    lib.oracle_add_rmsnorm_fp8.restype = ctypes.c_int
+    lib.oracle_e4m3_compare.argtypes = [vp, vp, i64, i32, ctypes.POINTER(i32), ctypes.POINTER(i64)]
+    lib.oracle_e4m3_compare.restype = None
     return lib
 
 
@@ -198,6 +207,55 @@ def compare_mixed(got, ref, dtype: int | None = None, *, tol: float = 2.0, tol_a
     worst, bad = ctypes.c_double(0.0), ctypes.c_int64(0)
     _load().oracle_mixed_compare(g.ctypes.data, q.ctypes.data, g.size, dt, tol, tol_abs, ctypes.byref(worst),
                                  ctypes.byref(bad))
+    return worst.value, bad.value
+
+
+def add_rmsnorm_fp8(x, r, w, eps: float, dtype: int | None = None):
+    """(q, scale, r_out): e4m3 codes as uint8 [T, H], float32 per-token scales [T], the rounded residual."""
+    want_torch = hasattr(x, "detach")
+    xs, dt = as_storage(x, dtype)
+    rs, dt_r = as_storage(r, dtype)
+    ws, dt_w = as_storage(w, dtype)
+    if not (dt == dt_r == dt_w):
+        raise TypeError("x, r and w must share one dtype")
+    if xs.ndim != 2 or rs.shape != xs.shape or ws.shape != (xs.shape[1],):
+        raise ValueError("expected x, r of shape [T, H] and w of shape [H]")
+    T, H = xs.shape
+    q = np.empty((T, H), dtype=np.uint8)
+    scale = np.empty((T,), dtype=np.float32)
+    r_out = np.empty_like(xs)
+    rc = _load().oracle_add_rmsnorm_fp8(xs.ctypes.data, rs.ctypes.data, ws.ctypes.data, q.ctypes.data,
+                                        scale.ctypes.data, r_out.ctypes.data, T, H, float(eps), dt)
+    if rc != 0:
+        raise RuntimeError(f"oracle_add_rmsnorm_fp8 failed with status {rc}")
+    if want_torch:
+        import torch
+        return torch.from_numpy(q), torch.from_numpy(scale), to_torch(r_out, dt)
+    return q, scale, r_out
+
+
+def decode_e4m3(bits) -> np.ndarray:
+    b = np.ascontiguousarray(bits, dtype=np.uint8)
+    out = np.empty(b.shape, dtype=np.float64)
+    _load().oracle_decode_e4m3(b.ctypes.data, out.ctypes.data, b.size)
+    return out
+
+
+def encode_e4m3(v) -> np.ndarray:
+    a = np.ascontiguousarray(v, dtype=np.float64)
+    out = np.empty(a.shape, dtype=np.uint8)
+    _load().oracle_encode_e4m3(a.ctypes.data, out.ctypes.data, a.size)
+    return out
+
+
+def compare_e4m3(got, ref, tol_steps: int = 1):
+    """(largest distance in e4m3 code steps, count beyond tol_steps) between two uint8 code arrays."""
+    g = np.ascontiguousarray(got.numpy() if hasattr(got, "numpy") else got, dtype=np.uint8)
+    q = np.ascontiguousarray(ref.numpy() if hasattr(ref, "numpy") else ref, dtype=np.uint8)
+    if g.shape != q.shape:
+        raise ValueError("got and ref must match in shape")
+    worst, bad = ctypes.c_int32(0), ctypes.c_int64(0)
+    _load().oracle_e4m3_compare(g.ctypes.data, q.ctypes.data, g.size, tol_steps, ctypes.byref(worst), ctypes.byref(bad))
     return worst.value, bad.value
 
 

@@ -212,3 +212,64 @@ def test_planted_merge_mistake_is_caught(oracle_lib, tmp_path, name):
         assert not _merge_pins(oracle_lib), f"pins did not notice: {name}"
     finally:
         oracle_lib._lib = saved
+
+
+FP8_MUTATIONS = {
+    "scale_from_448_wrong": ("(amax > 1e-12 ? amax : 1e-12) / 448.0", "(amax > 1e-12 ? amax : 1e-12) / 240.0"),
+    "amax_without_abs": ("if (fabs(y[j]) > amax) amax = fabs(y[j]);", "if (y[j] > amax) amax = y[j];"),
+    "weight_left_out_of_amax": ("y[j] = y[j] * (double)load32(w, j, dtype) / denom;\n            if (fabs(y[j]) > amax) amax = fabs(y[j]);",
+                                "if (fabs(y[j] / denom) > amax) amax = fabs(y[j] / denom);\n            y[j] = y[j] * (double)load32(w, j, dtype) / denom;"),
+    "ties_away": ("if (rem > 0.5 || (rem == 0.5 && (n & 1u))) n += 1;\n    uint32_t bits = E < emin", "if (rem >= 0.5) n += 1;\n    uint32_t bits = E < emin"),
+    "saturation_threshold": ("if (a >= 448.0) return (uint8_t)(sign | 0x7Eu);", "if (a >= 480.0) return (uint8_t)(sign | 0x7Eu);"),
+    "exponent_bias": ("((uint32_t)(E + 7) << 3)", "((uint32_t)(E + 8) << 3)"),
+    "scale_per_tensor": ("        double amax = 0.0;\n        for (int64_t j = 0; j < hidden; ++j) {\n            y[j] = y[j] *",
+                         "        static double amax = 0.0;\n        for (int64_t j = 0; j < hidden; ++j) {\n            y[j] = y[j] *"),
+}
+
+
+def _fp8_pins(o) -> bool:
+    try:
+        bits = torch.arange(256, dtype=torch.int16).to(torch.uint8)
+        vals = bits.view(torch.float8_e4m3fn).to(torch.float64).numpy()
+        fin = ~np.isnan(vals)
+        if not np.array_equal(o.encode_e4m3(vals[fin]), bits.numpy()[fin]):
+            return False
+        pos = np.sort(vals[fin & (bits.numpy() < 0x80)])
+        pb = o.encode_e4m3(pos)
+        mid = (pos[:-1] + pos[1:]) / 2
+        if not np.array_equal(o.encode_e4m3(mid), np.where((pb[:-1] & 1) == 0, pb[:-1], pb[1:])):
+            return False
+        if o.encode_e4m3(np.array([464.0, 470.0])).tolist() != [0x7E, 0x7E]:
+            return False
+        g = np.random.Generator(np.random.Philox(key=[81, 0]))
+        x = torch.from_numpy(g.standard_normal((6, 200)) * np.array([0.1, 1, 5, 1, 30, 1])[:, None]).to(torch.bfloat16)
+        r = torch.from_numpy(g.standard_normal((6, 200))).to(torch.bfloat16)
+        w = torch.from_numpy(-1.0 - 0.5 * np.abs(g.standard_normal(200))).to(torch.bfloat16)  # negative weights
+        q, scale, _ = o.add_rmsnorm_fp8(x, r, w, 1e-6)
+        s = (x.float() + r.float()).double()
+        y = s * torch.rsqrt(s.pow(2).mean(-1, keepdim=True) + float(np.float32(1e-6))) * w.double()
+        amax = y.abs().amax(-1)
+        if not torch.allclose(scale.double(), amax / 448.0, rtol=1.2e-7, atol=0):
+            return False
+        want = o.encode_e4m3((y / (amax / 448.0)[:, None]).numpy())
+        if np.count_nonzero(q.numpy() != want) > 1:
+            return False
+    except Exception:
+        return False
+    return True
+
+
+def test_real_fp8_oracle_passes_its_pins(oracle_lib):
+    assert _fp8_pins(oracle_lib)
+
+
+@pytest.mark.parametrize("name", sorted(FP8_MUTATIONS))
+def test_planted_fp8_mistake_is_caught(oracle_lib, tmp_path, name):
+    old, new = FP8_MUTATIONS[name]
+    so = _build_mutant(oracle_lib, str(tmp_path), old, new, targets=("add_rmsnorm_fp8_oracle.c",))
+    saved = oracle_lib._lib
+    try:
+        oracle_lib._lib = oracle_lib._bind(so)
+        assert not _fp8_pins(oracle_lib), f"pins did not notice: {name}"
+    finally:
+        oracle_lib._lib = saved
