@@ -50,7 +50,8 @@ typedef enum { RT_BF16 = 0, RT_FP16 = 1, RT_FP32 = 2 } rt_dtype;
 typedef enum {
     RT_OP_ADD_RMSNORM = 0,  /* fused residual-add + RMSNorm: the operator described above */
     RT_OP_SILU_AND_MUL = 1, /* out[t,j] = silu(x[t,j]) * x[t,d+j] for x of shape [n_tokens, 2*d] */
-    RT_OP_MERGE_ATTN_STATES = 2 /* two partial attention results merged by their log-sum-exps */
+    RT_OP_MERGE_ATTN_STATES = 2, /* two partial attention results merged by their log-sum-exps */
+    RT_OP_ADD_RMSNORM_FP8 = 3    /* add_rmsnorm whose y leaves as e4m3 bytes with one scale per token */
 } rt_op;
 
 /* Where a row lives between the two passes over it. */
@@ -137,7 +138,9 @@ typedef struct {
 /* For silu_and_mul: x is the [n_tokens, 2*d] input (ring stride 2 * ring_stride_bytes), y the output,
  * y_ref its reference; r, w, r_out, r_ref are unused and may be NULL.
  * For merge_attn_states: x = v_a, r = v_b, w = s_a, aux = s_b, y = v_out, r_out = s_out, y_ref and r_ref their
- * references (the s tensors are binary32 [n_tokens, heads]; in a ring they advance by n_tokens*heads*4). */
+ * references (the s tensors are binary32 [n_tokens, heads]; in a ring they advance by n_tokens*heads*4).
+ * For the fp8-output norm: y = q (bytes, ring stride ring_stride_bytes / 2), y_ref its reference codes,
+ * aux_out = scale ([n_tokens] binary32, ring stride n_tokens*4), aux_ref its reference. */
 typedef struct {
     const void* x;     /* device, [ring_sets][n_tokens, hidden] */
     const void* r;     /* device */
@@ -152,6 +155,8 @@ typedef struct {
     float eps;
     void* stream;
     const void* aux;   /* device; merge_attn_states: s_b.  NULL otherwise */
+    void* aux_out;     /* device; fp8-output norm: the per-token scales.  NULL otherwise */
+    const void* aux_ref; /* device; reference for aux_out */
 } rt_workspace;
 
 typedef enum { RT_PHASE_SEED = 0, RT_PHASE_GRID = 1, RT_PHASE_CLIMB = 2, RT_PHASE_TOPK = 3,
@@ -238,6 +243,21 @@ int64_t rmsnorm_host_workspace_bytes(int64_t n_tokens, int64_t hidden, int dtype
  */
 int silu_and_mul_template_launch(const rt_params* p, const void* x, void* out, int64_t n_tokens, int64_t d,
                                  int dtype, void* stream);
+
+/*
+ * add_rmsnorm with a quantised output for a following fp8 GEMM (a variant of the norm template: stage =
+ * registers or TMA bulk, 16-byte vectors, shuffle reduction; bf16 and fp16 inputs).  No counterpart kernel
+ * in the paper; it is one of the "organization of shared memory and registers" variants its template axes
+ * leave room for ("Tuning parameter selection and search space derivation").
+ *   x, r, w   device, as for rmsnorm_template_launch.     r_out  device, the rounded residual (bit-exact contract).
+ *   q         device, [n_tokens, hidden] bytes: e4m3 codes (4 exponent bits, bias 7, 3 significand bits, no
+ *             infinities, largest finite value 448) of y / scale, round to nearest even, saturating.
+ *   scale     device, [n_tokens] binary32: max(max_j |y_j|, 1e-12) / 448 with y the un-rounded norm output.
+ * Asynchronous on `stream`, allocates nothing; infeasible theta is refused without launching.
+ */
+int rmsnorm_fp8_template_launch(const rt_params* p, const void* x, const void* r, const void* w, void* q,
+                                float* scale, void* r_out, int64_t n_tokens, int64_t hidden, float eps, int dtype,
+                                void* stream);
 
 /*
  * merge_attn_states as an instance of its own template (third kernel of the paper's "Kernels" list, shapes
@@ -369,6 +389,12 @@ int rmsnorm_launch_auto(const rt_spec_entry* table, int32_t n_entries, const rt_
                         int64_t hidden, float eps, int dtype, void* stream, rt_params* used);
 
 typedef enum { RT_CMP_BITS = 0, RT_CMP_ULP16 = 1, RT_CMP_REL32 = 2 } rt_compare_mode;
+/*
+ * d(.,.) for e4m3 codes: distance in code steps on the format's value lattice (+0 == -0, NaN matches NaN).
+ * got, ref: device, n bytes.  *max_steps, *n_bad (elements beyond tol_steps): host.  Synchronises `stream`.
+ */
+int tuner_compare_e4m3(const void* got, const void* ref, int64_t n, int32_t tol_steps, int32_t* max_steps,
+                       int64_t* n_bad, void* stream);
 /*
  * d(.,.) for outputs that may cancel (merge_attn_states): an element passes when it is within `tol` of the
  * reference - units in the last place for the 16-bit types, relative for binary32 - OR within `tol_abs`

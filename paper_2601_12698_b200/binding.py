@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(_HERE, "librmsnorm_tuner.so")
 HEADER_PATH = os.path.join(os.path.dirname(_HERE), "include", "rmsnorm_tuner.h")
 
 RT_BF16, RT_FP16, RT_FP32 = 0, 1, 2
-RT_OP_ADD_RMSNORM, RT_OP_SILU_AND_MUL, RT_OP_MERGE_ATTN_STATES = 0, 1, 2
+RT_OP_ADD_RMSNORM, RT_OP_SILU_AND_MUL, RT_OP_MERGE_ATTN_STATES, RT_OP_ADD_RMSNORM_FP8 = 0, 1, 2, 3
 RT_STAGE_REG, RT_STAGE_SMEM_LDG, RT_STAGE_SMEM_TMA = 0, 1, 2
 RT_REDUCE_SHFL, RT_REDUCE_SMEM, RT_REDUCE_CLUSTER = 0, 1, 2
 RT_PRUNE_IDLE_THREADS, RT_PRUNE_DUPLICATES, RT_PRUNE_CLUSTER_WAVES, RT_PRUNE_IDLE_ROWS = 1, 2, 4, 8
@@ -74,7 +74,7 @@ class rt_workspace(Structure):
     _fields_ = [("x", c_void_p), ("r", c_void_p), ("w", c_void_p), ("y", c_void_p), ("r_out", c_void_p),
                 ("y_ref", c_void_p), ("r_ref", c_void_p), ("n_ref_tokens", c_int64),
                 ("ring_stride_bytes", c_int64), ("ring_sets", c_int32), ("eps", c_float), ("stream", c_void_p),
-                ("aux", c_void_p)]
+                ("aux", c_void_p), ("aux_out", c_void_p), ("aux_ref", c_void_p)]
 
 
 class rt_eval_record(Structure):
@@ -107,6 +107,8 @@ _SIGNATURES = {
     "rmsnorm_template_launch": (c_int, [POINTER(rt_params), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                         c_int64, c_int64, c_float, c_int, c_void_p]),
     "silu_and_mul_template_launch": (c_int, [POINTER(rt_params), c_void_p, c_void_p, c_int64, c_int64, c_int, c_void_p]),
+    "rmsnorm_fp8_template_launch": (c_int, [POINTER(rt_params), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                            c_int64, c_int64, c_float, c_int, c_void_p]),
     "merge_attn_states_template_launch": (c_int, [POINTER(rt_params), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                                   c_void_p, c_int64, c_int64, c_int64, c_int, c_void_p]),
     "rmsnorm_template_run_host": (c_int, [POINTER(rt_params), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
@@ -135,6 +137,7 @@ _SIGNATURES = {
     "tuner_launch_floor": (c_int, [POINTER(rt_budget), c_void_p, POINTER(c_float)]),
     "tuner_compare": (c_int, [c_void_p, c_void_p, c_int64, c_int, c_int, c_double, POINTER(c_double),
                               POINTER(c_int64), c_void_p]),
+    "tuner_compare_e4m3": (c_int, [c_void_p, c_void_p, c_int64, c_int32, POINTER(c_int32), POINTER(c_int64), c_void_p]),
     "tuner_compare_mixed": (c_int, [c_void_p, c_void_p, c_int64, c_int, c_double, c_double, POINTER(c_double),
                                     POINTER(c_int64), c_void_p]),
     "tuner_compare_static": (c_int, [c_void_p, c_void_p, c_int64, c_int, c_int, c_double, POINTER(c_double),
@@ -238,6 +241,20 @@ def silu_and_mul_template_launch(params: rt_params, x, out, stream=None) -> None
                                             _stream_ptr(stream)), "silu_and_mul_template_launch")
 
 
+def rmsnorm_fp8_template_launch(params: rt_params, x, r, w, q, scale, r_out, eps: float, stream=None) -> None:
+    """add_rmsnorm with e4m3 output: q uint8 [T, H], scale float32 [T], r_out like x (device tensors; asynchronous)."""
+    import torch
+    n_tokens, hidden = x.shape
+    ok = (all(t.is_cuda and t.is_contiguous() for t in (x, r, w, q, scale, r_out)) and r.shape == x.shape
+          and r_out.shape == x.shape and q.shape == x.shape and q.dtype == torch.uint8 and scale.shape == (n_tokens,)
+          and scale.dtype == torch.float32 and w.shape == (hidden,) and r.dtype == x.dtype == w.dtype == r_out.dtype)
+    if not ok:
+        raise ValueError("rmsnorm_fp8_template_launch: tensors of the wrong device, layout, shape or dtype")
+    _check(lib.rmsnorm_fp8_template_launch(byref(params), x.data_ptr(), r.data_ptr(), w.data_ptr(), q.data_ptr(),
+                                           scale.data_ptr(), r_out.data_ptr(), n_tokens, hidden, eps, _dtype_code(x),
+                                           _stream_ptr(stream)), "rmsnorm_fp8_template_launch")
+
+
 def merge_attn_states_template_launch(params: rt_params, v_a, s_a, v_b, s_b, v_out, s_out, stream=None) -> None:
     """Merge two partial attention results (device tensors; v: [n, h, d], s: float32 [n, h]); asynchronous."""
     import torch
@@ -327,15 +344,16 @@ def make_budget(max_evals=64, warmup=20, iters=100, repeats=3, top_k=5, strategy
 
 
 def make_workspace(x, r, w, y, r_out, y_ref, r_ref, eps: float, n_ref_tokens: int | None = None, ring_sets: int = 1,
-                   ring_stride_bytes: int = 0, stream=None, aux=None) -> rt_workspace:
+                   ring_stride_bytes: int = 0, stream=None, aux=None, aux_out=None, aux_ref=None) -> rt_workspace:
     """Device tensors for the tuner.  With ring_sets > 1, x, r, y, r_out are [ring_sets, T, H] and the
     references cover set 0.  For silu_and_mul pass r = w = r_out = r_ref = None; for merge_attn_states
-    x = v_a, r = v_b, w = s_a, aux = s_b, y = v_out, r_out = s_out."""
+    x = v_a, r = v_b, w = s_a, aux = s_b, y = v_out, r_out = s_out; for the fp8-output norm y = q (uint8),
+    aux_out = scale, aux_ref its reference."""
     T = x.shape[-2]
     ptr = lambda t: t.data_ptr() if t is not None else None
     return rt_workspace(ptr(x), ptr(r), ptr(w), ptr(y), ptr(r_out), ptr(y_ref), ptr(r_ref),
                         n_ref_tokens if n_ref_tokens is not None else T, ring_stride_bytes,
-                        ring_sets, eps, _stream_ptr(stream), ptr(aux))
+                        ring_sets, eps, _stream_ptr(stream), ptr(aux), ptr(aux_out), ptr(aux_ref))
 
 
 def tuner_search(shape: rt_shape, budget: rt_budget, ws: rt_workspace, log_cap: int = 4096):
@@ -377,6 +395,16 @@ def tuner_compare(got, ref, mode: int, tol: float = 0.0, stream=None):
     worst, bad = c_double(0.0), c_int64(0)
     _check(lib.tuner_compare(got.data_ptr(), ref.data_ptr(), got.numel(), _dtype_code(got), mode, tol, byref(worst),
                              byref(bad), _stream_ptr(stream)), "tuner_compare")
+    return worst.value, bad.value
+
+
+def tuner_compare_e4m3(got, ref, tol_steps: int = 1, stream=None):
+    """(largest distance in e4m3 code steps, elements beyond tol_steps) between two uint8 device tensors."""
+    if got.shape != ref.shape:
+        raise ValueError("got and ref must match")
+    worst, bad = c_int32(0), c_int64(0)
+    _check(lib.tuner_compare_e4m3(got.data_ptr(), ref.data_ptr(), got.numel(), tol_steps, byref(worst), byref(bad),
+                                  _stream_ptr(stream)), "tuner_compare_e4m3")
     return worst.value, bad.value
 
 

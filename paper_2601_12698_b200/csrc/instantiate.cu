@@ -1,6 +1,6 @@
 // One instantiation unit of the kernel template.  Compiled once per line of instance_units.inc with
 //   -DRT_UNIT_NAME=<name> -DRT_UNIT_T=<element type> -DRT_UNIT_DTYPE=<0|1|2> -DRT_UNIT_VB=<bytes>
-//   -DRT_UNIT_GROUP=<0 register stage | 1 shared-memory stages | 2 narrow fall-back | 3 silu_and_mul | 4 merge_attn_states>
+//   -DRT_UNIT_GROUP=<0 register stage | 1 shared-memory stages | 2 narrow fall-back | 3 silu_and_mul | 4 merge_attn_states | 5 fp8-output norm>
 //   -DRT_UNIT_REDUCE=<0|1|2>   (register-stage units only)
 //
 // Instance lists.  Register stage: CAP (row vectors kept per thread) in {1,2,4,8,16,32} while the row
@@ -10,6 +10,9 @@
 // silu_and_mul (one unit per element type, every vector width): stages register and TMA bulk for 16- and
 // 8-byte vectors with U in {1,2,4}; register stage with U in {1,4} for the 4- and 2-byte fall-back.
 // merge_attn_states: the same instance list as silu_and_mul.
+// fp8-output norm (16-bit element types, 16-byte vectors, shuffle reduction): register stage with CAP in
+// {1,2,4,8,16} and U <= CAP, TMA stage with U in {1,2,4}.
+#include "add_rmsnorm_fp8_kernel.cuh"
 #include "add_rmsnorm_kernel.cuh"
 #include "merge_attn_states_kernel.cuh"
 #include "silu_and_mul_kernel.cuh"
@@ -44,6 +47,17 @@ rt::KernelEntry silu_entry()
                                (const void*)&rt::silu_and_mul_kernel<T, VB, ST, U>};
     }
 }
+template <int ST, int U, int CAP>
+rt::KernelEntry fp8_entry()
+{
+    if constexpr (sizeof(T) != 2) {
+        return rt::KernelEntry{RT_OP_ADD_RMSNORM_FP8, kDtype, 16, ST, 0, U, CAP, nullptr};
+    } else {
+        return rt::KernelEntry{RT_OP_ADD_RMSNORM_FP8, kDtype, 16, ST, 0, U, ST == rt::kStageReg ? CAP : 0,
+                               (const void*)&rt::add_rmsnorm_fp8_kernel<T, ST, U, CAP>};
+    }
+}
+
 template <int VB, int ST, int U>
 rt::KernelEntry merge_entry()
 {
@@ -79,6 +93,10 @@ std::vector<rt::KernelEntry> build_entries()
 #elif RT_UNIT_GROUP == 3
         RT_SILU_WIDE(16), RT_SILU_WIDE(8), silu_entry<4, 0, 1>(), silu_entry<4, 0, 4>(), silu_entry<2, 0, 1>(),
         silu_entry<2, 0, 4>()
+#elif RT_UNIT_GROUP == 5
+        fp8_entry<0, 1, 1>(), fp8_entry<0, 1, 2>(), fp8_entry<0, 2, 2>(), fp8_entry<0, 1, 4>(), fp8_entry<0, 2, 4>(),
+        fp8_entry<0, 4, 4>(), fp8_entry<0, 1, 8>(), fp8_entry<0, 2, 8>(), fp8_entry<0, 4, 8>(), fp8_entry<0, 1, 16>(),
+        fp8_entry<0, 2, 16>(), fp8_entry<0, 4, 16>(), fp8_entry<2, 1, 1>(), fp8_entry<2, 2, 1>(), fp8_entry<2, 4, 1>()
 #elif RT_UNIT_GROUP == 4
         RT_MERGE_WIDE(16), RT_MERGE_WIDE(8), merge_entry<4, 0, 1>(), merge_entry<4, 0, 4>(), merge_entry<2, 0, 1>(),
         merge_entry<2, 0, 4>()

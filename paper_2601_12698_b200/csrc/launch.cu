@@ -8,6 +8,7 @@
 #include <mutex>
 #include <unordered_map>
 
+#include "add_rmsnorm_fp8_kernel.cuh"
 #include "add_rmsnorm_kernel.cuh"
 #include "merge_attn_states_kernel.cuh"
 #include "silu_and_mul_kernel.cuh"
@@ -268,7 +269,7 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
         plan->reject_reason = kRejectArgs;
         return RT_ERR_DTYPE;
     }
-    if (s->op != RT_OP_ADD_RMSNORM && s->op != RT_OP_SILU_AND_MUL && s->op != RT_OP_MERGE_ATTN_STATES) {
+    if (s->op < RT_OP_ADD_RMSNORM || s->op > RT_OP_ADD_RMSNORM_FP8) {
         set_error("op %d is not a kernel of this library", s->op);
         plan->reject_reason = kRejectArgs;
         return RT_ERR_SHAPE;
@@ -277,6 +278,7 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
     const bool is_silu = s->op == RT_OP_SILU_AND_MUL;
     const bool is_merge = s->op == RT_OP_MERGE_ATTN_STATES;
     const bool no_reduction = is_silu || is_merge;  // element-wise kernels: no reduction axis, no CAP
+    const bool is_fp8 = s->op == RT_OP_ADD_RMSNORM_FP8;
     const int eb = elem_bytes_of(s->dtype);
     if (s->n_tokens < 0 || s->hidden <= 0 || s->hidden * eb * (is_silu ? 2 : 1) >= (int64_t)1 << 31) {
         set_error("shape n_tokens=%lld hidden=%lld is out of range", (long long)s->n_tokens, (long long)s->hidden);
@@ -318,6 +320,14 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
         set_error("head_dim=%d does not divide hidden=%lld", s->head_dim, (long long)s->hidden);
         plan->reject_reason = kRejectArgs;
         return RT_ERR_SHAPE;
+    }
+    if (is_fp8 && (s->dtype == RT_FP32 || p->vec_bytes != 16 || p->reduce != RT_REDUCE_SHFL || p->cluster_size != 1 ||
+                   p->stage == RT_STAGE_SMEM_LDG)) {
+        set_error("the fp8-output norm takes bf16/fp16, 16-byte vectors, the shuffle reduction and the register or TMA "
+                  "stage (dtype=%d vec=%d reduce=%d cluster=%d stage=%d)", s->dtype, p->vec_bytes, p->reduce,
+                  p->cluster_size, p->stage);
+        plan->reject_reason = kRejectArgs;
+        return s->dtype == RT_FP32 ? RT_ERR_DTYPE : RT_ERR_INFEASIBLE;
     }
     if (no_reduction && (p->reduce != RT_REDUCE_SHFL || p->cluster_size != 1 || p->stage == RT_STAGE_SMEM_LDG)) {
         set_error("this kernel has no reduction and no ld.global->shared stage (reduce=%d cluster=%d stage=%d)",
@@ -499,6 +509,42 @@ int plan_occupancy(const Plan& plan, const rt_limits* L, int* regs_per_thread)
     return (int)blocks;
 }
 
+int launch_fp8_plan(const Plan& plan, const void* x, const void* r, const void* w, void* q, float* scale, void* r_out,
+                    int64_t n_tokens, int64_t hidden, float eps, cudaStream_t stream)
+{
+    if (n_tokens == 0) return RT_OK;
+    if (plan.op != RT_OP_ADD_RMSNORM_FP8) {
+        set_error("plan belongs to another kernel");
+        return RT_ERR_INFEASIBLE;
+    }
+    const KernelEntry& k = registry()[plan.kernel_index];
+    int st = ensure_dynamic_smem(plan.kernel_index, plan.dyn_smem);
+    if (st != RT_OK) return st;
+    Fp8Args a;
+    a.x = x; a.r = r; a.w = w; a.q = q; a.scale = scale; a.r_out = r_out;
+    a.n_tokens = n_tokens;
+    a.hidden = (int)hidden;
+    a.nvec = plan.nvec;
+    a.eps = eps;
+    a.status = device_status_word();
+    if (!a.status) return RT_ERR_CUDA;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(plan.grid_x, 1, 1);
+    cfg.blockDim = dim3(plan.block_x, plan.block_y, 1);
+    cfg.dynamicSmemBytes = plan.dyn_smem;
+    cfg.stream = stream;
+    void* params[] = {&a};
+    cudaError_t e = cudaLaunchKernelExC(&cfg, k.fn, params);
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        set_error("kernel launch failed: %s", cudaGetErrorString(e));
+        return RT_ERR_CUDA;
+    }
+    count_launch();
+    return RT_OK;
+}
+
 int launch_merge_plan(const Plan& plan, const void* v_a, const float* s_a, const void* v_b, const float* s_b, void* v_out,
                       float* s_out, int64_t n_tokens, cudaStream_t stream)
 {
@@ -677,6 +723,37 @@ int silu_and_mul_template_launch(const rt_params* p, const void* x, void* out, i
     st = rt::make_plan(&s, p, &L, &plan);
     if (st != RT_OK) return st;
     return rt::launch_silu_plan(plan, x, out, n_tokens, (cudaStream_t)stream);
+}
+
+int rmsnorm_fp8_template_launch(const rt_params* p, const void* x, const void* r, const void* w, void* q, float* scale,
+                                void* r_out, int64_t n_tokens, int64_t hidden, float eps, int dtype, void* stream)
+{
+    if (!p) {
+        rt::set_error("params is NULL");
+        return RT_ERR_NULL;
+    }
+    if (n_tokens > 0 && (!x || !r || !w || !q || !scale || !r_out)) {
+        rt::set_error("a tensor pointer is NULL");
+        return RT_ERR_NULL;
+    }
+    if (n_tokens > 0 && (((uintptr_t)scale & 3u) || ((uintptr_t)q & 7u))) {
+        rt::set_error("scale must be 4-byte and q 8-byte aligned");
+        return RT_ERR_ALIGN;
+    }
+    rt_limits L;
+    int st = rt::current_limits(&L);
+    if (st != RT_OK) return st;
+    rt_shape s;
+    s.n_tokens = n_tokens;
+    s.hidden = hidden;
+    s.dtype = dtype;
+    s.min_ptr_align = n_tokens > 0 ? rt::min_pointer_alignment(x, r, w, r_out, x) : 256;
+    s.op = RT_OP_ADD_RMSNORM_FP8;
+    s.head_dim = 0;
+    rt::Plan plan;
+    st = rt::make_plan(&s, p, &L, &plan);
+    if (st != RT_OK) return st;
+    return rt::launch_fp8_plan(plan, x, r, w, q, scale, r_out, n_tokens, hidden, eps, (cudaStream_t)stream);
 }
 
 int merge_attn_states_template_launch(const rt_params* p, const void* v_a, const float* s_a, const void* v_b,

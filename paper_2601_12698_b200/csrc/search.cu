@@ -14,6 +14,7 @@ namespace rt {
 
 // ---- d(.,.): element-wise comparison on the device ---------------------------------------------------
 
+constexpr int kAccSlots = 4;  // accumulator records one evaluation may fill before it reads them back
 struct CompareAcc {
     unsigned long long n_bad;
     unsigned int max_bits;  // ULP16: max distance; REL32: float bits of the max relative error; BITS: 0/1
@@ -80,6 +81,37 @@ __global__ void compare_kernel(const unsigned int* __restrict__ got, const unsig
         unsigned long long b2 = 0;
         compare_word<MODE>(tail_got, tail_ref, dtype, tol, b2, worst);
         bad += b2 ? 1 : 0;  // the padded upper halves are equal and add nothing
+    }
+    for (int off = 16; off >= 1; off >>= 1) {
+        bad += __shfl_xor_sync(0xffffffffu, bad, off);
+        worst = max(worst, __shfl_xor_sync(0xffffffffu, worst, off));
+    }
+    if ((threadIdx.x & 31) == 0) {
+        if (bad) atomicAdd(&acc->n_bad, bad);
+        if (worst) atomicMax(&acc->max_bits, worst);
+    }
+}
+
+// e4m3 codes: distance in code steps on the value lattice (+0 == -0, NaN matches NaN).
+__global__ void compare_e4m3_kernel(const unsigned char* __restrict__ got, const unsigned char* __restrict__ ref,
+                                    long long n, int tol_steps, CompareAcc* acc)
+{
+    unsigned long long bad = 0;
+    unsigned int worst = 0;
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+        const unsigned int g = got[i], q = ref[i];
+        const bool gn = (g & 0x7Fu) == 0x7Fu, qn = (q & 0x7Fu) == 0x7Fu;
+        unsigned int d;
+        if (gn || qn) {
+            d = (gn && qn) ? 0u : 255u;
+        } else {
+            const int gi = (g & 0x80u) ? -(int)(g & 0x7Fu) : (int)(g & 0x7Fu);
+            const int qi = (q & 0x80u) ? -(int)(q & 0x7Fu) : (int)(q & 0x7Fu);
+            d = (unsigned int)(gi > qi ? gi - qi : qi - gi);
+        }
+        if ((int)d > tol_steps) ++bad;
+        worst = max(worst, d);
     }
     for (int off = 16; off >= 1; off >>= 1) {
         bad += __shfl_xor_sync(0xffffffffu, bad, off);
@@ -193,8 +225,8 @@ int get_scratch(Scratch** out)
     std::lock_guard<std::mutex> lock(g_scratch_mutex);
     Scratch& s = g_scratch[dev];
     if (!s.dev) {
-        RT_CUDA_OK(cudaMalloc((void**)&s.dev, 2 * sizeof(CompareAcc)));
-        RT_CUDA_OK(cudaMallocHost((void**)&s.host, 2 * sizeof(CompareAcc)));
+        RT_CUDA_OK(cudaMalloc((void**)&s.dev, kAccSlots * sizeof(CompareAcc)));
+        RT_CUDA_OK(cudaMallocHost((void**)&s.host, kAccSlots * sizeof(CompareAcc)));
     }
     *out = &s;
     return RT_OK;
@@ -231,6 +263,17 @@ int enqueue_compare(const void* got, const void* ref, int64_t n, int dtype, int 
         compare_kernel<RT_CMP_ULP16><<<blocks, threads, 0, stream>>>(g, q, n_words, has_tail, tail_got, tail_ref, dtype, tol, acc);
     else
         compare_kernel<RT_CMP_REL32><<<blocks, threads, 0, stream>>>(g, q, n_words, has_tail, tail_got, tail_ref, dtype, tol, acc);
+    RT_CUDA_OK(cudaGetLastError());
+    count_launch();
+    return RT_OK;
+}
+
+int enqueue_compare_e4m3(const void* got, const void* ref, int64_t n, int tol_steps, CompareAcc* acc, cudaStream_t stream)
+{
+    const int threads = 256;
+    const long long want = (n + threads * 16 - 1) / (threads * 16);
+    const int blocks = (int)std::max<long long>(1, std::min<long long>(want, 148 * 16));
+    compare_e4m3_kernel<<<blocks, threads, 0, stream>>>((const unsigned char*)got, (const unsigned char*)ref, n, tol_steps, acc);
     RT_CUDA_OK(cudaGetLastError());
     count_launch();
     return RT_OK;
@@ -330,12 +373,17 @@ struct DeviceEvaluator : Evaluator {
         if (st != RT_OK) return st;
         const bool is_silu = shape.op == RT_OP_SILU_AND_MUL;
         const bool is_merge = shape.op == RT_OP_MERGE_ATTN_STATES;
+        const bool is_fp8 = shape.op == RT_OP_ADD_RMSNORM_FP8;
         const size_t lse_bytes = is_merge ? (size_t)shape.n_tokens * plan.heads * sizeof(float) : 0;  // one s tensor
-        RT_CUDA_OK(cudaMemsetAsync(ws.y, 0xFF, set_bytes, stream));
+        RT_CUDA_OK(cudaMemsetAsync(ws.y, 0xFF, is_fp8 ? set_bytes / eb : set_bytes, stream));
+        if (is_fp8) RT_CUDA_OK(cudaMemsetAsync(ws.aux_out, 0xFF, (size_t)shape.n_tokens * sizeof(float), stream));
         if (is_merge) RT_CUDA_OK(cudaMemsetAsync(ws.r_out, 0xFF, lse_bytes, stream));
         else if (!is_silu) RT_CUDA_OK(cudaMemsetAsync(ws.r_out, 0xFF, set_bytes, stream));
-        RT_CUDA_OK(cudaMemsetAsync(sc->dev, 0, 2 * sizeof(CompareAcc), stream));
-        if (is_merge)
+        RT_CUDA_OK(cudaMemsetAsync(sc->dev, 0, kAccSlots * sizeof(CompareAcc), stream));
+        if (is_fp8)
+            st = launch_fp8_plan(plan, ws.x, ws.r, ws.w, ws.y, (float*)ws.aux_out, ws.r_out, shape.n_tokens, shape.hidden,
+                                 ws.eps, stream);
+        else if (is_merge)
             st = launch_merge_plan(plan, ws.x, (const float*)ws.w, ws.r, (const float*)ws.aux, ws.y, (float*)ws.r_out,
                                    shape.n_tokens, stream);
         else
@@ -347,7 +395,15 @@ struct DeviceEvaluator : Evaluator {
         }
         const int y_mode = shape.dtype == RT_FP32 ? RT_CMP_REL32 : RT_CMP_ULP16;
         const double y_tol = shape.dtype == RT_FP32 ? 1e-5 : 2.0;
-        if (is_merge) {
+        if (is_fp8) {
+            // residual bit-exact; codes within one e4m3 step; per-token scales within 1e-5 relative
+            st = enqueue_compare(ws.r_out, ws.r_ref, n_ref * shape.hidden, shape.dtype, RT_CMP_BITS, 0.0, sc->dev, stream);
+            if (st != RT_OK) return st;
+            st = enqueue_compare_e4m3(ws.y, ws.y_ref, n_ref * shape.hidden, 1, sc->dev + 1, stream);
+            if (st != RT_OK) return st;
+            st = enqueue_compare(ws.aux_out, ws.aux_ref, n_ref, RT_FP32, RT_CMP_REL32, 1e-5, sc->dev + 2, stream);
+            if (st != RT_OK) return st;
+        } else if (is_merge) {
             // outputs that may cancel: 2 ulp / 1e-5 relative, or 1e-5 absolute; the merged log-sum-exp likewise
             st = enqueue_compare_mixed(ws.r_out, ws.r_ref, n_ref * plan.heads, RT_FP32, 1e-5, 1e-5, sc->dev, stream);
             if (st != RT_OK) return st;
@@ -362,15 +418,17 @@ struct DeviceEvaluator : Evaluator {
             if (st != RT_OK) return st;
         }
         (void)ref_bytes;
-        RT_CUDA_OK(cudaMemcpyAsync(sc->host, sc->dev, 2 * sizeof(CompareAcc), cudaMemcpyDeviceToHost, stream));
+        RT_CUDA_OK(cudaMemcpyAsync(sc->host, sc->dev, kAccSlots * sizeof(CompareAcc), cudaMemcpyDeviceToHost, stream));
         cudaError_t e = cudaStreamSynchronize(stream);
         if (e != cudaSuccess) {
             set_error("candidate faulted: %s", cudaGetErrorString(e));
             return RT_ERR_CUDA;  // a sticky error: nothing further can run in this context
         }
         rec->r_bad = (int64_t)sc->host[0].n_bad;
-        rec->y_bad = (int64_t)sc->host[1].n_bad;
-        if (shape.dtype == RT_FP32 || is_merge)
+        rec->y_bad = (int64_t)sc->host[1].n_bad + (is_fp8 ? (int64_t)sc->host[2].n_bad : 0);
+        if (is_fp8)
+            rec->y_max_ulp = (int32_t)sc->host[1].max_bits;  // e4m3 code steps
+        else if (shape.dtype == RT_FP32 || is_merge)
             rec->y_max_rel = (float)acc_max_err(sc->host[1], RT_CMP_REL32);  // merge: largest absolute difference
         else
             rec->y_max_ulp = (int32_t)sc->host[1].max_bits;
@@ -392,6 +450,10 @@ struct DeviceEvaluator : Evaluator {
         const int sets = ws.ring_sets > 0 ? ws.ring_sets : 1;
         auto launch_set = [&](int k) {
             const size_t off = (size_t)(k % sets) * (size_t)ws.ring_stride_bytes;
+            if (is_fp8)
+                return launch_fp8_plan(plan, (const char*)ws.x + off, (const char*)ws.r + off, ws.w, (char*)ws.y + off / eb,
+                                       (float*)((char*)ws.aux_out + (size_t)(k % sets) * shape.n_tokens * sizeof(float)),
+                                       (char*)ws.r_out + off, shape.n_tokens, shape.hidden, ws.eps, stream);
             if (is_merge) {
                 const size_t so = (size_t)(k % sets) * lse_bytes;
                 return launch_merge_plan(plan, (const char*)ws.x + off, (const float*)((const char*)ws.w + so),
@@ -782,7 +844,7 @@ int check_workspace(const rt_shape* s, const rt_workspace* ws)
     }
     const bool is_silu = s->op == RT_OP_SILU_AND_MUL;
     if (!ws->x || !ws->y || !ws->y_ref || (!is_silu && (!ws->r || !ws->w || !ws->r_out || !ws->r_ref)) ||
-        (s->op == RT_OP_MERGE_ATTN_STATES && !ws->aux)) {
+        (s->op == RT_OP_MERGE_ATTN_STATES && !ws->aux) || (s->op == RT_OP_ADD_RMSNORM_FP8 && (!ws->aux_out || !ws->aux_ref))) {
         set_error("a workspace pointer is NULL");
         return RT_ERR_NULL;
     }
@@ -835,6 +897,34 @@ int tuner_compare(const void* got, const void* ref, int64_t n, int dtype, int mo
     RT_CUDA_OK(cudaMemcpyAsync(sc->host, sc->dev, sizeof(rt::CompareAcc), cudaMemcpyDeviceToHost, s));
     RT_CUDA_OK(cudaStreamSynchronize(s));
     *max_err = rt::acc_max_err(sc->host[0], mode);
+    *n_bad = (int64_t)sc->host[0].n_bad;
+    return RT_OK;
+}
+
+int tuner_compare_e4m3(const void* got, const void* ref, int64_t n, int32_t tol_steps, int32_t* max_steps, int64_t* n_bad,
+                       void* stream)
+{
+    if (!got || !ref || !max_steps || !n_bad) {
+        rt::set_error("tuner_compare_e4m3: NULL argument");
+        return RT_ERR_NULL;
+    }
+    if (n < 0) {
+        rt::set_error("n = %lld is negative", (long long)n);
+        return RT_ERR_SHAPE;
+    }
+    *max_steps = 0;
+    *n_bad = 0;
+    if (n == 0) return RT_OK;
+    rt::Scratch* sc;
+    int st = rt::get_scratch(&sc);
+    if (st != RT_OK) return st;
+    cudaStream_t s = (cudaStream_t)stream;
+    RT_CUDA_OK(cudaMemsetAsync(sc->dev, 0, sizeof(rt::CompareAcc), s));
+    st = rt::enqueue_compare_e4m3(got, ref, n, tol_steps, sc->dev, s);
+    if (st != RT_OK) return st;
+    RT_CUDA_OK(cudaMemcpyAsync(sc->host, sc->dev, sizeof(rt::CompareAcc), cudaMemcpyDeviceToHost, s));
+    RT_CUDA_OK(cudaStreamSynchronize(s));
+    *max_steps = (int32_t)sc->host[0].max_bits;
     *n_bad = (int64_t)sc->host[0].n_bad;
     return RT_OK;
 }

@@ -72,6 +72,8 @@ int current_limits(rt_limits* out);
 
 int launch_plan(const Plan& plan, const void* x, const void* r, const void* w, void* y, void* r_out,
                 int64_t n_tokens, int64_t hidden, float eps, cudaStream_t stream);
+int launch_fp8_plan(const Plan& plan, const void* x, const void* r, const void* w, void* q, float* scale, void* r_out,
+                    int64_t n_tokens, int64_t hidden, float eps, cudaStream_t stream);
 int launch_merge_plan(const Plan& plan, const void* v_a, const float* s_a, const void* v_b, const float* s_b, void* v_out,
                       float* s_out, int64_t n_tokens, cudaStream_t stream);
 int launch_silu_plan(const Plan& plan, const void* x, void* out, int64_t n_tokens, cudaStream_t stream);

@@ -68,6 +68,8 @@ class Workload:
         b = DTYPE_BYTES[self.dtype]
         if self.op == "silu_and_mul":
             return 3 * b * self.elements
+        if self.op == "add_rmsnorm_fp8":  # read x, r; write r' and one byte of q per element; w once; a scale per token
+            return (3 * b + 1) * self.elements + b * self.hidden + 4 * self.n_tokens
         if self.op == "merge_attn_states":  # v_a, v_b in, v_out out; s_a, s_b in, s_out out (binary32 per head)
             return 3 * b * self.elements + 3 * 4 * self.n_tokens * (self.hidden // self.head_dim)
         return 4 * b * self.elements + b * self.hidden
@@ -104,6 +106,8 @@ def workloads() -> dict[str, Workload]:
     add(Workload("silu_fp32_2048x8192", "fp32", 2048, 8192, seed=6, dist=gate, op="silu_and_mul"))
     add(Workload("silu_fp32_128x11008", "fp32", 128, 11008, seed=6, dist=gate, op="silu_and_mul"))
     add(Workload("silu_bf16_64x11008", "bf16", 64, 11008, seed=6, dist=gate, op="silu_and_mul"))
+    # the fp8-output variant of the norm on the prefill shape
+    add(Workload("c3q_prefill_bf16_16384x8192_fp8out", "bf16", 16384, 8192, seed=2, dist=_PREFILL_DIST, op="add_rmsnorm_fp8"))
     # merge_attn_states: the paper's (n, h, d) shapes in bf16, and a bandwidth case
     for n, h, d in ((512, 32, 256), (512, 40, 128), (768, 32, 256), (768, 40, 128), (512, 64, 128)):
         add(Workload(f"merge_bf16_{n}x{h}x{d}", "bf16", n, h * d, seed=7, op="merge_attn_states", head_dim=d))

@@ -124,3 +124,14 @@ def test_merge_attn_states_grid(L):
     # head_dim must divide hidden
     assert B.tuner_check_params(B.shape_of(4, 1000, "bf16", op=B.RT_OP_MERGE_ATTN_STATES, head_dim=128), B.make_params(), L) == B.RT_ERR_SHAPE
     assert B.tuner_check_params(B.shape_of(4, 1024, "bf16", op=B.RT_OP_MERGE_ATTN_STATES, head_dim=0), B.make_params(), L) == B.RT_ERR_SHAPE
+
+
+def test_fp8_output_norm_grid(L):
+    s = B.shape_of(16384, 8192, "bf16", op=B.RT_OP_ADD_RMSNORM_FP8)
+    f = B.tuner_derive_feasible(s, L)
+    assert f and {t.vec_bytes for t in f} == {16} and {t.stage for t in f} == {0, 2} and {t.reduce for t in f} == {0}
+    assert all(B.tuner_check_params(s, t, L) == B.RT_OK for t in f)
+    assert B.tuner_check_params(B.shape_of(64, 4096, "fp32", op=B.RT_OP_ADD_RMSNORM_FP8), B.make_params(), L) == B.RT_ERR_DTYPE
+    assert B.tuner_check_params(s, B.make_params(vec_bytes=8), L) == B.RT_ERR_INFEASIBLE
+    # rows that are not 16-byte multiples have no instance of this variant
+    assert B.tuner_derive_feasible(B.shape_of(64, 6148, "fp16", op=B.RT_OP_ADD_RMSNORM_FP8), L) == []
