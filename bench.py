@@ -29,12 +29,14 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "fused_add_rmsnorm_hbm_gbs"
-METRICS = {"add_rmsnorm": METRIC, "silu_and_mul": "silu_and_mul_hbm_gbs", "merge_attn_states": "merge_attn_states_hbm_gbs"}
+METRICS = {"add_rmsnorm": METRIC, "silu_and_mul": "silu_and_mul_hbm_gbs", "merge_attn_states": "merge_attn_states_hbm_gbs",
+           "add_rmsnorm_fp8": "fused_add_rmsnorm_fp8out_hbm_gbs"}
 BYTES_LABEL = {"add_rmsnorm": "algorithmic: 2 reads + 2 writes per element + w once",
                "silu_and_mul": "algorithmic: 2 reads + 1 write per output element",
-               "merge_attn_states": "algorithmic: 2 reads + 1 write per element + 3 binary32 per (token, head)"}
+               "merge_attn_states": "algorithmic: 2 reads + 1 write per element + 3 binary32 per (token, head)",
+               "add_rmsnorm_fp8": "algorithmic: 2 reads + 1 write per element + 1 byte of q per element + w once + a scale per token"}
 KERNEL_NAME = {"add_rmsnorm": "add_rmsnorm_kernel", "silu_and_mul": "silu_and_mul_kernel",
-               "merge_attn_states": "merge_attn_states_kernel"}
+               "merge_attn_states": "merge_attn_states_kernel", "add_rmsnorm_fp8": "add_rmsnorm_fp8_kernel"}
 UNIT = "GB/s"
 DEFAULT_WORKLOAD = "c3_prefill_bf16_16384x8192"
 FALLBACK_HBM_GBS = 6650.0  # used only when MEASURED_PEAKS.json is absent
@@ -147,6 +149,11 @@ def run_reference(args) -> None:
         if is_merge:
             va, sa, vb, sb = synth.make_merge_inputs(0, n_rows, wl.hidden // wl.head_dim, wl.head_dim, wl.dtype, wl.seed)
             return lambda: oracle.merge_attn_states(va, sa, vb, sb)
+        if wl.op == "add_rmsnorm_fp8":
+            w = synth.make_weight(wl.hidden, wl.dtype, wl.seed, wl.dist)
+            xs = synth.make_rows(synth.TENSOR_X, 0, n_rows, wl.hidden, wl.dtype, wl.seed, wl.dist).contiguous()
+            rs = synth.make_rows(synth.TENSOR_R, 0, n_rows, wl.hidden, wl.dtype, wl.seed, wl.dist).contiguous()
+            return lambda: oracle.add_rmsnorm_fp8(xs, rs, w, wl.eps)
         if is_silu:
             xs = synth.make_gate_up(0, n_rows, wl.hidden, wl.dtype, wl.seed, wl.dist)
             return lambda: oracle.silu_and_mul(xs, threads=cores)
@@ -170,7 +177,10 @@ def run_reference(args) -> None:
         run()
     elapsed = time.perf_counter() - t0
     b = synth.DTYPE_BYTES[wl.dtype]
-    if is_merge:
+    if wl.op == "add_rmsnorm_fp8":
+        cores = 1  # this oracle is single-threaded
+        step_bytes = (3 * b + 1) * rows * wl.hidden + b * wl.hidden + 4 * rows
+    elif is_merge:
         cores = 1  # this oracle is single-threaded
         step_bytes = 3 * b * rows * wl.hidden + 12 * rows * (wl.hidden // wl.head_dim)
     else:
@@ -210,8 +220,10 @@ def run_ours(args) -> None:
 
     is_silu = wl.op == "silu_and_mul"
     is_merge = wl.op == "merge_attn_states"
+    is_fp8 = wl.op == "add_rmsnorm_fp8"
     op_code = {"add_rmsnorm": B.RT_OP_ADD_RMSNORM, "silu_and_mul": B.RT_OP_SILU_AND_MUL,
-               "merge_attn_states": B.RT_OP_MERGE_ATTN_STATES}[wl.op]
+               "merge_attn_states": B.RT_OP_MERGE_ATTN_STATES, "add_rmsnorm_fp8": B.RT_OP_ADD_RMSNORM_FP8}[wl.op]
+    scale_ref = None
     heads = H // wl.head_dim if is_merge else 0
     sa = sb = None
 
@@ -233,7 +245,10 @@ def run_ours(args) -> None:
     cores = os.cpu_count() or 1
     oracle.build()
     t0 = time.perf_counter()
-    if is_merge:
+    if is_fp8:
+        cores = 1  # this oracle is single-threaded
+        y_ref, scale_ref, r_ref = oracle.add_rmsnorm_fp8(x, r, w, wl.eps)  # y_ref holds the e4m3 codes
+    elif is_merge:
         cores = 1  # this oracle is single-threaded
         v_ref, r_ref = oracle.merge_attn_states(va, sa, vb, sb)  # r_ref holds the merged log-sum-exps
         y_ref = v_ref.view(T, H)
@@ -257,8 +272,10 @@ def run_ours(args) -> None:
     xd = ring(x)
     rd = ring(r) if r is not None else None
     wd = w.to(device) if w is not None else None
-    yd = torch.empty((sets, T, H), dtype=xd.dtype, device=device)
-    od = torch.empty_like(yd) if not (is_silu or is_merge) else None
+    yd = torch.empty((sets, T, H), dtype=torch.uint8 if is_fp8 else xd.dtype, device=device)
+    scaled = torch.empty((sets, T), dtype=torch.float32, device=device) if is_fp8 else None
+    scale_ref_d = scale_ref.to(device) if is_fp8 else None
+    od = torch.empty_like(xd) if not (is_silu or is_merge) else None
     sad = sbd = None
     if is_merge:
         sad, sbd = ring(sa), ring(sb)
@@ -266,15 +283,16 @@ def run_ours(args) -> None:
     y_ref_d = y_ref.to(device)
     r_ref_d = r_ref.to(device) if r_ref is not None else None
     set_bytes = T * H * b  # one output-sized set; silu_and_mul's input sets are twice as long
-    live = [t for t in (xd, rd, wd, yd, od) if t is not None]
+    live = [t for t in (xd, rd, wd, od if is_fp8 else yd, od) if t is not None]
     align = B._ptr_align(*live)
     shape = B.shape_of(T, H, wl.dtype, align if set_bytes % 256 == 0 else min(align, set_bytes & -set_bytes), op=op_code,
                        head_dim=wl.head_dim)
     # warm: the paper's protocol (the same buffers every launch); cold: rotating over the ring
     w_or_sa = sad if is_merge else wd
-    ws = B.make_workspace(xd, rd, w_or_sa, yd, od, y_ref_d, r_ref_d, wl.eps, n_ref_tokens=T, stream=stream, aux=sbd)
+    ws = B.make_workspace(xd, rd, w_or_sa, yd, od, y_ref_d, r_ref_d, wl.eps, n_ref_tokens=T, stream=stream, aux=sbd,
+                          aux_out=scaled, aux_ref=scale_ref_d)
     ws_cold = B.make_workspace(xd, rd, w_or_sa, yd, od, y_ref_d, r_ref_d, wl.eps, n_ref_tokens=T, ring_sets=sets,
-                               ring_stride_bytes=set_bytes, stream=stream, aux=sbd)
+                               ring_stride_bytes=set_bytes, stream=stream, aux=sbd, aux_out=scaled, aux_ref=scale_ref_d)
     use_graph = resident  # launch gaps would otherwise dominate kernels of a few microseconds
 
     # The tuner (not timed): exhaustive sweep as ground truth, then the guided search with a stated budget.
@@ -356,7 +374,18 @@ def run_ours(args) -> None:
     # Step k works on set k mod sets (one set when the workload exceeds L2 by itself).
     theta_ref = B.byref(theta)
     dtype_code, stream_ptr, eps = B.DTYPE_CODES[wl.dtype], stream.cuda_stream, wl.eps
-    if is_merge:
+    if is_fp8:
+        launch = B.lib.rmsnorm_fp8_template_launch
+        ptrs = [(xd[k].data_ptr(), rd[k].data_ptr(), yd[k].data_ptr(), scaled[k].data_ptr(), od[k].data_ptr())
+                for k in range(sets)]
+        w_ptr = wd.data_ptr()
+
+        def step(k):
+            px, pr, pq, ps, po = ptrs[k % sets]
+            st = launch(theta_ref, px, pr, w_ptr, pq, ps, po, T, H, eps, dtype_code, stream_ptr)
+            if st != 0:
+                raise B.TunerError(st, "rmsnorm_fp8_template_launch")
+    elif is_merge:
         launch = B.lib.merge_attn_states_template_launch
         ptrs = [(xd[k].data_ptr(), sad[k].data_ptr(), rd[k].data_ptr(), sbd[k].data_ptr(), yd[k].data_ptr(),
                  od[k].data_ptr()) for k in range(sets)]
@@ -407,12 +436,16 @@ def run_ours(args) -> None:
 
     # Parity of what was just timed, against the oracle (all rows; r' bit-exact, y within tolerance).
     last = (args.steps - 1) % sets  # the set the last timed step wrote
-    if is_merge:
+    if is_fp8:
+        r_bad = B.tuner_compare(od[last], r_ref_d, B.RT_CMP_BITS, stream=stream)[1]
+        y_worst, y_bad = B.tuner_compare_e4m3(yd[last], y_ref_d, 1, stream=stream)
+        y_bad += B.tuner_compare(scaled[last], scale_ref_d, B.RT_CMP_REL32, 1e-5, stream=stream)[1]
+    elif is_merge:
         r_bad = B.tuner_compare_mixed(od[last], r_ref_d, 1e-5, 1e-5, stream=stream)[1]
         y_worst, y_bad = B.tuner_compare_mixed(yd[last], y_ref_d, 1e-5 if wl.dtype == "fp32" else 2.0, 1e-5, stream=stream)
     else:
         r_bad = 0 if is_silu else B.tuner_compare(od[last], r_ref_d, B.RT_CMP_BITS, stream=stream)[1]
-    if is_merge:
+    if is_merge or is_fp8:
         pass
     elif wl.dtype == "fp32":
         y_worst, y_bad = B.tuner_compare(yd[last], y_ref_d, B.RT_CMP_REL32, 1e-5, stream=stream)
@@ -426,7 +459,18 @@ def run_ours(args) -> None:
     # entry point (chunked, copies overlapped with the kernel); silu_and_mul has no such entry point, so its
     # end-to-end step is copy in, launch, copy out on the launch stream.
     e2e_steps = max(3, min(args.steps, args.e2e_steps))
-    if is_merge:
+    if is_fp8:
+        xp, rp, wp = x.pin_memory(), r.pin_memory(), w.pin_memory()
+        yp, op, sp = torch.empty((T, H), dtype=torch.uint8).pin_memory(), torch.empty_like(xp).pin_memory(), torch.empty(T).pin_memory()
+        h2d_bytes, d2h_bytes = 2 * T * H * b + H * b, T * H * b + T * H + 4 * T
+
+        def e2e_step():
+            with torch.cuda.stream(stream):
+                xd[0].copy_(xp, non_blocking=True); rd[0].copy_(rp, non_blocking=True); wd.copy_(wp, non_blocking=True)
+                step(0)
+                yp.copy_(yd[0], non_blocking=True); op.copy_(od[0], non_blocking=True); sp.copy_(scaled[0], non_blocking=True)
+            stream.synchronize()
+    elif is_merge:
         xp, rp, sap, sbp = x.pin_memory(), r.pin_memory(), sa.pin_memory(), sb.pin_memory()
         yp, sop = torch.empty((T, H), dtype=x.dtype).pin_memory(), torch.empty((T, heads)).pin_memory()
         h2d_bytes, d2h_bytes = 2 * T * H * b + 8 * T * heads, T * H * b + 4 * T * heads
@@ -466,7 +510,10 @@ def run_ours(args) -> None:
     e2e_ms = dp.max_over_ranks((time.perf_counter() - t0) * 1e3, device)
     dp.barrier(device)
     e2e_value = dp.whole_job_rate(wl.algorithmic_bytes, e2e_steps, world, e2e_ms) / 1e9
-    if is_merge:
+    if is_fp8:
+        e2e_bad = (oracle.compare_e4m3(yp[-64:], y_ref[-64:], tol_steps=1)[1] or oracle.bit_mismatches(op[:64], r_ref[:64])
+                   or oracle.compare_y(sp, scale_ref, tol_rel=1e-5)[1])
+    elif is_merge:
         e2e_bad = (oracle.compare_mixed(yp[-64:], y_ref[-64:], tol=1e-5 if wl.dtype == "fp32" else 2.0, tol_abs=1e-5)[1]
                    or oracle.compare_mixed(sop[:64], r_ref[:64], tol=1e-5, tol_abs=1e-5)[1])
     else:
