@@ -717,12 +717,37 @@ bool on_coarse_grid(const rt_params& p, int widest_vec)
     return (lt % 2 == 1) && (lr % 2 == 0) && (lu % 2 == 0) && p.vec_bytes == widest_vec;
 }
 
-std::vector<int> thin(const std::vector<int>& v, int keep)
+// When the budget cannot cover the whole coarse grid, the part that is evaluated must still touch every
+// stage x reduction mode: the grid points are ordered mode by mode in rounds - first every mode's point
+// nearest the middle of the ordered axes (256 threads per row, one row per CTA, unroll 1), then every mode's
+// second nearest, and so on - and the first `keep` of that order are taken.
+std::vector<int> stratified(const std::vector<int>& coarse, const std::vector<rt_params>& cand, int keep)
 {
     if (keep <= 0) return {};
-    if ((int)v.size() <= keep) return v;
+    if ((int)coarse.size() <= keep) return coarse;
+    auto mode_of = [](const rt_params& p) { return (p.reduce * 16 + p.cluster_size) * 4 + p.stage; };
+    auto off_centre = [](const rt_params& p) {
+        return 2 * abs(level_of(kTpr, 6, p.threads_per_row) - 3) + level_of(kRpc, 4, p.rows_per_cta) +
+               level_of(kUnr, 3, p.unroll);
+    };
+    std::vector<int> order = coarse;
+    std::stable_sort(order.begin(), order.end(), [&](int x, int y) {
+        const int mx = mode_of(cand[x]), my = mode_of(cand[y]);
+        if (mx != my) return mx < my;
+        return off_centre(cand[x]) < off_centre(cand[y]);
+    });
+    // rank of each point inside its mode, then round-robin over the modes
+    std::vector<std::pair<int, int>> keyed;  // (rank in mode, position in `order`)
+    int rank = 0;
+    for (size_t i = 0; i < order.size(); ++i) {
+        rank = (i > 0 && mode_of(cand[order[i]]) == mode_of(cand[order[i - 1]])) ? rank + 1 : 0;
+        keyed.push_back({rank, (int)i});
+    }
+    std::stable_sort(keyed.begin(), keyed.end(), [](const std::pair<int, int>& x, const std::pair<int, int>& y) {
+        return x.first < y.first;
+    });
     std::vector<int> out;
-    for (int i = 0; i < keep; ++i) out.push_back(v[(size_t)i * v.size() / keep]);
+    for (int i = 0; i < keep; ++i) out.push_back(order[keyed[i].second]);
     return out;
 }
 
@@ -769,7 +794,7 @@ int run_search(const rt_shape& shape, const rt_limits& limits, const rt_budget& 
             if (st != RT_OK) return st;
             S.time_us[idx] = t;
         }
-        // 2. coarse grid, thinned to half of what is left of the budget
+        // 2. coarse grid, cut to half of what is left of the budget (mode by mode, nearest the middle first)
         int widest = 0;
         for (const rt_params& p : feasible) widest = std::max(widest, p.vec_bytes);
         std::vector<int> coarse;
@@ -778,7 +803,7 @@ int run_search(const rt_shape& shape, const rt_limits& limits, const rt_budget& 
         if (coarse.empty())
             for (int i = 0; i < (int)feasible.size(); ++i) coarse.push_back(i);
         const int grid_budget = std::max(1, (S.max_evals - top_k - S.used) / 2);
-        for (int idx : thin(coarse, grid_budget)) {
+        for (int idx : stratified(coarse, S.cand, grid_budget)) {
             if (!S.budget_left(top_k)) break;
             if (S.time_us[idx] >= 0.f) continue;
             st = S.run(idx, RT_PHASE_GRID, &t);

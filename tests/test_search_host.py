@@ -141,3 +141,17 @@ def test_empty_feasible_set_is_an_error_not_a_crash(L):
     with pytest.raises(B.TunerError) as e:
         B.tuner_search_with(s, L, B.make_budget(max_evals=10), lambda p: 1.0)
     assert e.value.status == B.RT_ERR_INFEASIBLE
+
+
+def test_a_small_budget_still_touches_every_stage_and_reduction_mode(L):
+    """The coarse grid is cut mode by mode: with room for 12 grid points every (stage, reduction) pair of the prefill
+    shape (3 x 2) is visited before any pair is visited a third time."""
+    s = B.shape_of(*SHAPE)
+    res, log = B.tuner_search_with(s, L, B.make_budget(max_evals=30, top_k=5), _cost_factory(OPTIMA[0]))
+    grid = [r for r in log if r.phase == 1]
+    assert len(grid) == 12
+    modes = [(r.params.stage, r.params.reduce) for r in grid]
+    assert set(modes[:6]) == {(st, rd) for st in (0, 1, 2) for rd in (0, 1)}
+    assert all(modes.count(m) == 2 for m in set(modes))
+    # the first point of every mode is the one nearest the middle of the ordered axes
+    assert all(r.params.threads_per_row == 256 and r.params.rows_per_cta == 1 and r.params.unroll == 1 for r in grid[:6])
