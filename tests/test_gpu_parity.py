@@ -238,3 +238,33 @@ def test_host_buffer_entry_point(B, oracle_lib):
     with pytest.raises(B.TunerError) as e:
         B.rmsnorm_template_run_host(B.make_params(), xp, rp, wp, y, ro, EPS, small)
     assert e.value.status == B.RT_ERR_CAPACITY
+
+
+def test_more_than_2_to_31_elements(B, oracle_lib):
+    """A batch whose element count and byte offsets exceed 32 bits: rows are a 4096-row seeded block repeated on the
+    device, and sampled rows from the whole range (the far end above all) are checked against the oracle."""
+    synth = _synth()
+    H, block, reps = 8192, 4096, 66                      # 270 336 rows, 2.21e9 elements, 4.4 GB per tensor
+    T = block * reps
+    x, r, w = synth.make_inputs(block, H, "bf16", seed=77)
+    y_ref, r_ref = oracle_lib.add_rmsnorm(x, r, w, EPS, threads=8)
+    xd = x.cuda().repeat(reps, 1); rd = r.cuda().repeat(reps, 1); wd = w.cuda()
+    assert xd.numel() > 2**31 and xd.shape == (T, H)
+    y, ro = torch.empty_like(xd), torch.empty_like(xd)
+    rows = sorted({0, 1, block - 1, block, 131072, 131073, 262143, 262144, T - 2, T - 1} |
+                  {int(v) for v in torch.randint(0, T, (48,), generator=torch.Generator().manual_seed(1))})
+    idx = torch.tensor(rows)
+    shape = B.shape_of(T, H, "bf16")
+    feasible = B.tuner_derive_feasible(shape)
+    picks = [next(t for t in feasible if t.stage == s) for s in (0, 1, 2)] + [B.make_params(threads_per_row=256, rows_per_cta=4)]
+    for th in picks:
+        y.fill_(float("nan")); ro.fill_(float("nan"))
+        B.rmsnorm_template_launch(th, xd, rd, wd, y, ro, EPS)
+        assert oracle_lib.bit_mismatches(ro[idx].cpu(), r_ref[idx % block]) == 0, repr(th)
+        assert oracle_lib.compare_y(y[idx].cpu(), y_ref[idx % block])[1] == 0, repr(th)
+        assert not bool(torch.isnan(y[-4096:]).any()) and not bool(torch.isnan(ro[-4096:]).any())
+    # the device comparator over the whole far half (offsets past 2^32 bytes)
+    half = (reps // 2) * block
+    want = y_ref.cuda().repeat(reps - reps // 2, 1)
+    assert B.tuner_compare(y[half:], want, B.RT_CMP_ULP16, 2.0)[1] == 0
+    assert B.rt_device_status() == 0
