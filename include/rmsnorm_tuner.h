@@ -383,6 +383,8 @@ int tuner_table_lookup(const rt_spec_entry* table, int32_t n_entries, const rt_p
 /*
  * rmsnorm_template_launch with theta taken from tuner_table_lookup for this call's shape and pointer
  * alignment.  `used` (may be NULL) receives the theta launched.  Asynchronous, allocates nothing.
+ * Each thread remembers its last lookup (table address, entry count, shape), so a loop over one shape pays for
+ * the lookup once: do not edit a table in place while it is in use - build a new array instead.
  */
 int rmsnorm_launch_auto(const rt_spec_entry* table, int32_t n_entries, const rt_params* general,
                         const void* x, const void* r, const void* w, void* y, void* r_out, int64_t n_tokens,
@@ -410,7 +412,8 @@ int tuner_compare_mixed(const void* got, const void* ref, int64_t n, int dtype, 
  *   RT_CMP_ULP16: distance in units of the last place on the 16-bit type's value lattice
  *                 (+0 == -0, NaN matches NaN); *n_bad = elements beyond `tol`.
  *   RT_CMP_REL32: |got-ref| <= tol*|ref| + 1e-30 for fp32; *max_err = worst |got-ref|/|ref|.
- *   max_err, n_bad: host.  Synchronises `stream`.
+ *   max_err, n_bad: host.  Synchronises `stream`.  The comparison entry points (this one, _mixed, _e4m3) and
+ *   the tuner's evaluations share one accumulator block per device and are serialised by a lock.
  */
 int tuner_compare(const void* got, const void* ref, int64_t n, int dtype, int mode, double tol,
                   double* max_err, int64_t* n_bad, void* stream);

@@ -61,6 +61,24 @@ int get_pipe(HostPipe** out)
 }
 
 }  // namespace
+
+void host_pipe_shutdown()
+{
+    std::lock_guard<std::mutex> lock(g_pipe_mutex);
+    for (HostPipe& p : g_pipe) {
+        if (!p.ready) continue;
+        cudaStreamDestroy(p.h2d);
+        cudaStreamDestroy(p.d2h);
+        for (int i = 0; i < kSlots; ++i) {
+            cudaEventDestroy(p.loaded[i]);
+            cudaEventDestroy(p.computed[i]);
+            cudaEventDestroy(p.drained[i]);
+        }
+        cudaEventDestroy(p.start);
+        p.ready = false;
+    }
+}
+
 }  // namespace rt
 
 extern "C" {

@@ -181,6 +181,15 @@ static_assert(sizeof(CompareAcc) <= kStaticScratchBytes, "accumulator record lar
 
 namespace {
 
+// Upper bound of the comparison kernels' grids: 16 CTAs of 256 threads per SM of the current device.
+int compare_grid_cap()
+{
+    rt_limits L;
+    return current_limits(&L) == RT_OK ? 16 * std::max(1, L.sm_count) : 16 * 132;
+}
+
+// The comparison entry points and the evaluator share one accumulator block per device: calls are serialised.
+std::mutex g_compare_mutex;
 std::mutex g_scratch_mutex;
 CompareAcc* g_static_scratch_addr[64];  // device address of the static scratch, per device
 
@@ -254,7 +263,7 @@ int enqueue_compare(const void* got, const void* ref, int64_t n, int dtype, int 
     }
     const int threads = 256;
     long long want = (n_words + threads * 8 - 1) / (threads * 8);
-    const int blocks = (int)std::max<long long>(1, std::min<long long>(want, 148 * 16));
+    const int blocks = (int)std::max<long long>(1, std::min<long long>(want, (long long)compare_grid_cap()));
     const unsigned int* g = (const unsigned int*)got;
     const unsigned int* q = (const unsigned int*)ref;
     if (mode == RT_CMP_BITS)
@@ -272,7 +281,7 @@ int enqueue_compare_e4m3(const void* got, const void* ref, int64_t n, int tol_st
 {
     const int threads = 256;
     const long long want = (n + threads * 16 - 1) / (threads * 16);
-    const int blocks = (int)std::max<long long>(1, std::min<long long>(want, 148 * 16));
+    const int blocks = (int)std::max<long long>(1, std::min<long long>(want, (long long)compare_grid_cap()));
     compare_e4m3_kernel<<<blocks, threads, 0, stream>>>((const unsigned char*)got, (const unsigned char*)ref, n, tol_steps, acc);
     RT_CUDA_OK(cudaGetLastError());
     count_launch();
@@ -284,7 +293,7 @@ int enqueue_compare_mixed(const void* got, const void* ref, int64_t n, int dtype
 {
     const int threads = 256;
     const long long want = (n + threads * 8 - 1) / (threads * 8);
-    const int blocks = (int)std::max<long long>(1, std::min<long long>(want, 148 * 16));
+    const int blocks = (int)std::max<long long>(1, std::min<long long>(want, (long long)compare_grid_cap()));
     compare_mixed_kernel<<<blocks, threads, 0, stream>>>(got, ref, n, dtype, tol, tol_abs, acc);
     RT_CUDA_OK(cudaGetLastError());
     count_launch();
@@ -349,6 +358,7 @@ struct DeviceEvaluator : Evaluator {
 
     int evaluate(const rt_params& p, rt_eval_record* rec) override
     {
+        std::lock_guard<std::mutex> serial(g_compare_mutex);
         memset(rec, 0, sizeof(*rec));
         rec->params = p;
         cudaStream_t stream = (cudaStream_t)ws.stream;
@@ -903,6 +913,7 @@ extern "C" {
 int tuner_compare(const void* got, const void* ref, int64_t n, int dtype, int mode, double tol, double* max_err,
                   int64_t* n_bad, void* stream)
 {
+    std::lock_guard<std::mutex> serial(rt::g_compare_mutex);
     int st = rt::check_compare_args(got, ref, n, dtype, mode);
     if (st != RT_OK) return st;
     if (!max_err || !n_bad) {
@@ -929,6 +940,7 @@ int tuner_compare(const void* got, const void* ref, int64_t n, int dtype, int mo
 int tuner_compare_e4m3(const void* got, const void* ref, int64_t n, int32_t tol_steps, int32_t* max_steps, int64_t* n_bad,
                        void* stream)
 {
+    std::lock_guard<std::mutex> serial(rt::g_compare_mutex);
     if (!got || !ref || !max_steps || !n_bad) {
         rt::set_error("tuner_compare_e4m3: NULL argument");
         return RT_ERR_NULL;
@@ -957,6 +969,7 @@ int tuner_compare_e4m3(const void* got, const void* ref, int64_t n, int32_t tol_
 int tuner_compare_mixed(const void* got, const void* ref, int64_t n, int dtype, double tol, double tol_abs,
                         double* max_abs, int64_t* n_bad, void* stream)
 {
+    std::lock_guard<std::mutex> serial(rt::g_compare_mutex);
     int st = rt::check_compare_args(got, ref, n, dtype, RT_CMP_BITS);
     if (st != RT_OK) return st;
     if (!max_abs || !n_bad) {
@@ -1072,6 +1085,8 @@ int tuner_launch_floor(const rt_budget* b, void* stream, float* us)
 
 void rt_shutdown(void)
 {
+    rt::host_pipe_shutdown();
+    std::lock_guard<std::mutex> serial(rt::g_compare_mutex);
     std::lock_guard<std::mutex> lock(rt::g_scratch_mutex);
     for (rt::Scratch& s : rt::g_scratch) {
         if (s.dev) cudaFree(s.dev);

@@ -79,6 +79,7 @@ int launch_merge_plan(const Plan& plan, const void* v_a, const float* s_a, const
 int launch_silu_plan(const Plan& plan, const void* x, void* out, int64_t n_tokens, cudaStream_t stream);
 int ensure_dynamic_smem(int index, size_t bytes);
 int* device_status_word();
+void host_pipe_shutdown();  // streams and events of the host-buffer pipeline
 void count_launch(int64_t n = 1);
 
 // Raw grid and feasible set (feasible.cu).  counts, when given, has kRejectReasons + 3 entries:
