@@ -178,6 +178,8 @@ def _check(status: int, where: str):
 
 def _dtype_code(t) -> int:
     import torch
+    if isinstance(t, int):
+        return t
     return {torch.bfloat16: RT_BF16, torch.float16: RT_FP16, torch.float32: RT_FP32}[t.dtype]
 
 
@@ -441,13 +443,21 @@ def tuner_select_general(times_us) -> tuple[int, float, list[float]]:
 
 
 class SpecTable:
-    """D_spec and theta_gen as the C arrays the library consumes, with JSON persistence (marshalling only)."""
+    """D_spec and theta_gen as the C arrays the library consumes, with JSON persistence (marshalling only).
 
-    def __init__(self, entries=(), general: rt_params | None = None, device_name: str = ""):
+    Entries of every kernel (rt_shape.op) live in one table; there is one general configuration per kernel."""
+
+    def __init__(self, entries=(), general: rt_params | None = None, device_name: str = "", generals: dict | None = None):
         self.entries = list(entries)  # [(rt_shape, rt_params, best_us)]
-        self.general = general
+        self.generals = dict(generals or {})  # rt_op -> rt_params
+        if general is not None:
+            self.generals[RT_OP_ADD_RMSNORM] = general
         self.device_name = device_name
         self._pack()
+
+    @property
+    def general(self) -> rt_params | None:
+        return self.generals.get(RT_OP_ADD_RMSNORM)
 
     def _pack(self):
         self._arr = (rt_spec_entry * max(1, len(self.entries)))()
@@ -460,7 +470,8 @@ class SpecTable:
 
     def lookup(self, shape: rt_shape, limits: rt_limits | None = None):
         out, src = rt_params(), c_int32(-1)
-        _check(lib.tuner_table_lookup(self._arr, len(self.entries), byref(self.general) if self.general else None,
+        general = self.generals.get(int(shape.op))
+        _check(lib.tuner_table_lookup(self._arr, len(self.entries), byref(general) if general else None,
                                       byref(shape), byref(limits) if limits is not None else None, byref(out),
                                       byref(src)), "tuner_table_lookup")
         return out, SOURCE_NAMES[src.value]
@@ -469,15 +480,37 @@ class SpecTable:
         """rmsnorm_launch_auto on device tensors; returns the theta that was launched."""
         n_tokens, hidden = x.shape
         used = rt_params()
-        _check(lib.rmsnorm_launch_auto(self._arr, len(self.entries), byref(self.general) if self.general else None,
+        general = self.general
+        _check(lib.rmsnorm_launch_auto(self._arr, len(self.entries), byref(general) if general else None,
                                        x.data_ptr(), r.data_ptr(), w.data_ptr(), y.data_ptr(), r_out.data_ptr(),
                                        n_tokens, hidden, eps, _dtype_code(x), _stream_ptr(stream), byref(used)),
                "rmsnorm_launch_auto")
         return used
 
+    def launch_silu_and_mul(self, x, out, stream=None) -> rt_params:
+        """Table lookup (in the library) for this shape, then silu_and_mul_template_launch."""
+        n_tokens, d = out.shape
+        theta, _ = self.lookup(shape_of(n_tokens, d, _dtype_code(out), _ptr_align(x, out), op=RT_OP_SILU_AND_MUL))
+        silu_and_mul_template_launch(theta, x, out, stream)
+        return theta
+
+    def launch_merge_attn_states(self, v_a, s_a, v_b, s_b, v_out, s_out, stream=None) -> rt_params:
+        n, h, d = v_a.shape
+        theta, _ = self.lookup(shape_of(n, h * d, _dtype_code(v_a), _ptr_align(v_a, v_b, v_out),
+                                        op=RT_OP_MERGE_ATTN_STATES, head_dim=d))
+        merge_attn_states_template_launch(theta, v_a, s_a, v_b, s_b, v_out, s_out, stream)
+        return theta
+
+    def launch_rmsnorm_fp8(self, x, r, w, q, scale, r_out, eps: float, stream=None) -> rt_params:
+        n_tokens, hidden = x.shape
+        theta, _ = self.lookup(shape_of(n_tokens, hidden, _dtype_code(x), _ptr_align(x, r, w, r_out), op=RT_OP_ADD_RMSNORM_FP8))
+        rmsnorm_fp8_template_launch(theta, x, r, w, q, scale, r_out, eps, stream)
+        return theta
+
     def to_json(self) -> dict:
         names = {v: k for k, v in DTYPE_CODES.items()}
         return {"device": self.device_name, "general": self.general.as_dict() if self.general else None,
+                "generals": {str(op): th.as_dict() for op, th in sorted(self.generals.items())},
                 "specialised": [{"dtype": names[s.dtype], "n_tokens": int(s.n_tokens), "hidden": int(s.hidden),
                                  "op": int(s.op), "head_dim": int(s.head_dim), "theta": t.as_dict(), "us": round(float(us), 3)}
                                 for s, t, us in self.entries]}
@@ -496,7 +529,8 @@ class SpecTable:
         entries = [(shape_of(e["n_tokens"], e["hidden"], e["dtype"], op=int(e.get("op", 0)),
                              head_dim=int(e.get("head_dim", 0))), mk(e["theta"]), float(e["us"]))
                    for e in d.get("specialised", [])]
-        return cls(entries, mk(d["general"]) if d.get("general") else None, d.get("device", ""))
+        generals = {int(op): mk(th) for op, th in (d.get("generals") or {}).items()}
+        return cls(entries, mk(d["general"]) if d.get("general") else None, d.get("device", ""), generals)
 
 
 def rt_device_status() -> int:

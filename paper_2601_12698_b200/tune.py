@@ -2,9 +2,10 @@
 
     python -m paper_2601_12698_b200.tune --shapes bf16:128x4096,bf16:16384x8192,fp32:2048x8192 \
         --budget 64 --out rmsnorm_table.json
+    python -m paper_2601_12698_b200.tune --shapes silu/bf16:4096x14336,merge/bf16:512x32x128,fp8/bf16:4096x8192
 
-For every shape: seeded synthetic inputs, a guided search (Algorithm 1: DeriveFeasibleSpace, Search), then
-SelectGeneral over the shapes' finalists timed on every shape and BuildSpecialized as a JSON table that
+For every (kernel, shape): seeded synthetic inputs, a guided search (Algorithm 1: DeriveFeasibleSpace, Search),
+then, per kernel, SelectGeneral over the shapes' finalists timed on every shape, and BuildSpecialized as a JSON table that
 ``binding.SpecTable`` loads for ``rmsnorm_launch_auto``.
 
 The correctness gate needs reference outputs.  As in the paper's protocol (every candidate is compared with
@@ -24,12 +25,19 @@ from . import binding as B
 from . import synth
 
 
+OPS = {"norm": B.RT_OP_ADD_RMSNORM, "silu": B.RT_OP_SILU_AND_MUL, "merge": B.RT_OP_MERGE_ATTN_STATES,
+       "fp8": B.RT_OP_ADD_RMSNORM_FP8}
+
+
 def parse_shapes(text: str):
+    """[kernel/]dtype:dims, comma separated.  kernel: norm (default, TOKENSxHIDDEN), silu (TOKENSxD),
+    merge (TOKENSxHEADSxHEAD_DIM), fp8 (the norm with e4m3 output, TOKENSxHIDDEN)."""
     out = []
     for item in text.split(","):
-        dtype, dims = item.strip().split(":")
-        t, h = dims.lower().split("x")
-        out.append((dtype, int(t), int(h)))
+        item = item.strip()
+        kernel, rest = item.split("/") if "/" in item else ("norm", item)
+        dtype, dims = rest.split(":")
+        out.append((kernel, dtype, tuple(int(v) for v in dims.lower().split("x"))))
     return out
 
 
@@ -43,29 +51,67 @@ def reference_theta(shape: B.rt_shape) -> B.rt_params:
 
 
 class ShapeProblem:
-    """Device buffers of one shape: inputs, outputs, reference outputs from S_ref."""
+    """Device buffers of one (kernel, shape): inputs, outputs, reference outputs from S_ref."""
 
-    def __init__(self, dtype: str, n_tokens: int, hidden: int, seed: int, eps: float, stream):
-        self.dtype, self.n_tokens, self.hidden, self.eps = dtype, n_tokens, hidden, eps
-        x, r, w = synth.make_inputs(n_tokens, hidden, dtype, seed)
-        self.x, self.r, self.w = x.cuda(), r.cuda(), w.cuda()
-        self.y, self.r_out = torch.empty_like(self.x), torch.empty_like(self.x)
-        self.y_ref, self.r_ref = torch.empty_like(self.x), torch.empty_like(self.x)
-        self.shape = B.shape_of(n_tokens, hidden, dtype, B._ptr_align(self.x, self.r, self.w, self.y, self.r_out))
-        self.ref_theta = reference_theta(self.shape)
-        B.rmsnorm_template_launch(self.ref_theta, self.x, self.r, self.w, self.y_ref, self.r_ref, eps, stream=stream)
+    def __init__(self, kernel: str, dtype: str, dims: tuple, seed: int, eps: float, stream):
+        self.kernel, self.dtype, self.dims, self.eps = kernel, dtype, dims, eps
+        op = OPS[kernel]
+        n_tokens = dims[0]
+        if kernel == "silu":
+            d = dims[1]
+            x = synth.make_gate_up(0, n_tokens, d, dtype, seed).cuda()
+            y, y_ref = (torch.empty(n_tokens, d, dtype=x.dtype, device="cuda") for _ in range(2))
+            self.shape = B.shape_of(n_tokens, d, dtype, B._ptr_align(x, y), op=op)
+            self.ref_theta = reference_theta(self.shape)
+            B.silu_and_mul_template_launch(self.ref_theta, x, y_ref, stream=stream)
+            self.ws = B.make_workspace(x, None, None, y, None, y_ref, None, eps, stream=stream)
+            moved = 3 * x.element_size() * n_tokens * d
+            self.keep = (x, y, y_ref)
+        elif kernel == "merge":
+            h, d = dims[1], dims[2]
+            va, sa, vb, sb = (t.cuda() for t in synth.make_merge_inputs(0, n_tokens, h, d, dtype, seed))
+            vo, vo_ref, so, so_ref = torch.empty_like(va), torch.empty_like(va), torch.empty_like(sa), torch.empty_like(sa)
+            self.shape = B.shape_of(n_tokens, h * d, dtype, B._ptr_align(va, vb, vo), op=op, head_dim=d)
+            self.ref_theta = reference_theta(self.shape)
+            B.merge_attn_states_template_launch(self.ref_theta, va, sa, vb, sb, vo_ref, so_ref, stream=stream)
+            self.ws = B.make_workspace(va, vb, sa, vo, so, vo_ref, so_ref, eps, stream=stream, aux=sb)
+            moved = 3 * va.element_size() * va.numel()
+            self.keep = (va, sa, vb, sb, vo, vo_ref, so, so_ref)
+        else:
+            hidden = dims[1]
+            x, r, w = (t.cuda() for t in synth.make_inputs(n_tokens, hidden, dtype, seed))
+            r_out, r_ref = torch.empty_like(x), torch.empty_like(x)
+            if kernel == "fp8":
+                y, y_ref = (torch.empty(n_tokens, hidden, dtype=torch.uint8, device="cuda") for _ in range(2))
+                sc, sc_ref = (torch.empty(n_tokens, dtype=torch.float32, device="cuda") for _ in range(2))
+                self.shape = B.shape_of(n_tokens, hidden, dtype, B._ptr_align(x, r, w, r_out), op=op)
+                self.ref_theta = reference_theta(self.shape)
+                B.rmsnorm_fp8_template_launch(self.ref_theta, x, r, w, y_ref, sc_ref, r_ref, eps, stream=stream)
+                self.ws = B.make_workspace(x, r, w, y, r_out, y_ref, r_ref, eps, stream=stream, aux_out=sc, aux_ref=sc_ref)
+                self.keep = (x, r, w, y, y_ref, r_out, r_ref, sc, sc_ref)
+            else:
+                y, y_ref = torch.empty_like(x), torch.empty_like(x)
+                self.shape = B.shape_of(n_tokens, hidden, dtype, B._ptr_align(x, r, w, y, r_out), op=op)
+                self.ref_theta = reference_theta(self.shape)
+                B.rmsnorm_template_launch(self.ref_theta, x, r, w, y_ref, r_ref, eps, stream=stream)
+                self.ws = B.make_workspace(x, r, w, y, r_out, y_ref, r_ref, eps, stream=stream)
+                self.keep = (x, r, w, y, y_ref, r_out, r_ref)
+            moved = 4 * x.element_size() * x.numel()
         stream.synchronize()
-        self.ws = B.make_workspace(self.x, self.r, self.w, self.y, self.r_out, self.y_ref, self.r_ref, eps, stream=stream)
-        limits = B.rt_query_limits()
-        self.use_graph = 4 * x.numel() * x.element_size() <= 2 * limits.l2_bytes
+        self.use_graph = moved <= 2 * B.rt_query_limits().l2_bytes
+
+    @property
+    def label(self) -> str:
+        return f"{self.kernel}/{self.dtype}:" + "x".join(str(v) for v in self.dims)
 
 
 def tune(shapes, budget: int = 64, top_k: int = 5, finalists: int = 3, seed: int = 0, eps: float = 1e-6, verbose=False):
-    """Returns (SpecTable, report dict)."""
+    """shapes: [(kernel, dtype, dims)] or, for the norm, [(dtype, n_tokens, hidden)].  Returns (SpecTable, report)."""
+    shapes = [s if isinstance(s[2], tuple) else ("norm", s[0], (s[1], s[2])) for s in shapes]
     stream = torch.cuda.Stream()
-    problems, per_shape, candidates = [], [], {}
-    for dtype, t, h in shapes:
-        p = ShapeProblem(dtype, t, h, seed, eps, stream)
+    per_shape, candidates = [], {}  # candidates: kernel -> {theta key: theta}
+    for kernel, dtype, dims in shapes:
+        p = ShapeProblem(kernel, dtype, dims, seed, eps, stream)
         res, log = B.tuner_search(p.shape, B.make_budget(max_evals=budget, top_k=top_k, use_graph=p.use_graph), p.ws)
         ranked = sorted((rec for rec in log if rec.status == B.RT_OK), key=lambda rec: rec.us)
         seen = []
@@ -75,49 +121,53 @@ def tune(shapes, budget: int = 64, top_k: int = 5, finalists: int = 3, seed: int
             if len(seen) == finalists:
                 break
         for key in [res.best.key()] + seen:
-            candidates.setdefault(key, B.rt_params(*key))
-        per_shape.append((p.shape, res.best, res.best_us, res.evals_used))
-        problems.append((dtype, t, h))
+            candidates.setdefault(kernel, {}).setdefault(key, B.rt_params(*key))
+        per_shape.append((p.shape, res.best, res.best_us, res.evals_used, p.label))
         if verbose:
-            print(f"{dtype}:{t}x{h}: {res.best} {res.best_us:.2f} us ({res.evals_used} evaluations)", file=sys.stderr)
+            print(f"{p.label}: {res.best} {res.best_us:.2f} us ({res.evals_used} evaluations)", file=sys.stderr)
         del p
         torch.cuda.empty_cache()
 
-    # SelectGeneral: every finalist timed on every shape (paper protocol), then the geometric-mean choice
-    cand = list(candidates.values())
-    times = [[-1.0] * len(problems) for _ in cand]
-    for xi, (dtype, t, h) in enumerate(problems):
-        p = ShapeProblem(dtype, t, h, seed, eps, stream)
-        proto = B.make_budget(warmup=20, iters=100, repeats=3, use_graph=p.use_graph)
-        for ci, th in enumerate(cand):
-            if B.tuner_check_params(p.shape, th) != B.RT_OK:
-                continue
-            rec = B.tuner_evaluate(p.shape, th, proto, p.ws)
-            if rec.status == B.RT_OK:
-                times[ci][xi] = rec.us
-        del p
-        torch.cuda.empty_cache()
-    general, report = None, {"shapes": [f"{d}:{t}x{h}" for d, t, h in problems]}
-    try:
-        gi, score, scores = B.tuner_select_general(times)
-        general = cand[gi]
-        report.update({"general": general.as_dict(), "general_geomean_vs_specialised": round(score, 4),
-                       "general_us": [round(v, 3) for v in times[gi]]})
-    except B.TunerError as err:
-        report["general"] = None
-        report["general_error"] = str(err)
-    best_per_shape = [min((times[c][x] for c in range(len(cand)) if times[c][x] > 0), default=-1.0)
-                      for x in range(len(problems))]
-    report["specialised_us"] = [round(v, 3) for v in best_per_shape]
-    report["specialised"] = [th.as_dict() for _, th, _, _ in per_shape]
-    report["evaluations"] = [n for _, _, _, n in per_shape]
-    table = B.SpecTable([(s, th, us) for s, th, us, _ in per_shape], general, torch.cuda.get_device_name())
+    # SelectGeneral, kernel by kernel: every finalist timed on every shape of its kernel (paper protocol), then
+    # the geometric-mean choice
+    generals, report = {}, {"shapes": [label for *_, label in per_shape], "kernels": {}}
+    for kernel, cand_map in candidates.items():
+        cand = list(cand_map.values())
+        mine = [(k, d, dims) for k, d, dims in shapes if k == kernel]
+        times = [[-1.0] * len(mine) for _ in cand]
+        for xi, (k, dtype, dims) in enumerate(mine):
+            p = ShapeProblem(k, dtype, dims, seed, eps, stream)
+            proto = B.make_budget(warmup=20, iters=100, repeats=3, use_graph=p.use_graph)
+            for ci, th in enumerate(cand):
+                if B.tuner_check_params(p.shape, th) != B.RT_OK:
+                    continue
+                rec = B.tuner_evaluate(p.shape, th, proto, p.ws)
+                if rec.status == B.RT_OK:
+                    times[ci][xi] = rec.us
+            del p
+            torch.cuda.empty_cache()
+        entry = {"specialised_us": [round(min((times[c][x] for c in range(len(cand)) if times[c][x] > 0), default=-1.0), 3)
+                                    for x in range(len(mine))]}
+        try:
+            gi, score, _ = B.tuner_select_general(times)
+            generals[OPS[kernel]] = cand[gi]
+            entry.update({"general": cand[gi].as_dict(), "general_geomean_vs_specialised": round(score, 4),
+                          "general_us": [round(v, 3) for v in times[gi]]})
+        except B.TunerError as err:
+            entry.update({"general": None, "general_error": str(err)})
+        report["kernels"][kernel] = entry
+    norm = report["kernels"].get("norm", {})
+    report.update({k: norm.get(k) for k in ("general", "general_geomean_vs_specialised", "general_us", "specialised_us")})
+    report["specialised"] = [th.as_dict() for _, th, _, _, _ in per_shape]
+    report["evaluations"] = [n for _, _, _, n, _ in per_shape]
+    table = B.SpecTable([(s, th, us) for s, th, us, _, _ in per_shape], None, torch.cuda.get_device_name(), generals)
     return table, report
 
 
 def main() -> None:
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
-    ap.add_argument("--shapes", required=True, help="comma-separated dtype:TOKENSxHIDDEN, e.g. bf16:128x4096")
+    ap.add_argument("--shapes", required=True, help="comma-separated [kernel/]dtype:dims, e.g. bf16:128x4096,"
+                    "silu/bf16:4096x14336,merge/bf16:512x32x128,fp8/bf16:4096x8192")
     ap.add_argument("--budget", type=int, default=64, help="kernel evaluations per shape")
     ap.add_argument("--out", default="", help="write the table as JSON here")
     ap.add_argument("--seed", type=int, default=0)

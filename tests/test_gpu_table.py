@@ -60,3 +60,32 @@ def test_launch_auto_matches_the_oracle(B, oracle_lib, tuned, dtype, T, H, want_
     elif want_source is not None:
         assert source == want_source
     assert B.rt_device_status() == 0
+
+
+def test_tuning_and_auto_launch_for_the_other_kernels(B, oracle_lib):
+    from paper_2601_12698_b200 import synth, tune
+    table, report = tune.tune([("silu", "bf16", (64, 2048)), ("silu", "bf16", (512, 5504)), ("merge", "bf16", (128, 8, 128)),
+                               ("fp8", "bf16", (256, 4096))], budget=16, top_k=2)
+    assert set(table.generals) == {B.RT_OP_SILU_AND_MUL, B.RT_OP_MERGE_ATTN_STATES, B.RT_OP_ADD_RMSNORM_FP8}
+    assert 0.5 < report["kernels"]["silu"]["general_geomean_vs_specialised"] <= 1.0 + 1e-6
+    again = B.SpecTable.from_json(table.to_json())
+    assert {op: th.key() for op, th in again.generals.items()} == {op: th.key() for op, th in table.generals.items()}
+    # silu_and_mul on a shape that is not in the table
+    x = synth.make_gate_up(0, 100, 2048, "bf16", seed=3)
+    out = torch.empty(100, 2048, dtype=torch.bfloat16, device="cuda")
+    used = again.launch_silu_and_mul(x.cuda(), out)
+    assert oracle_lib.compare_y(out.cpu(), oracle_lib.silu_and_mul(x))[1] == 0 and used.reduce == 0
+    # merge_attn_states, exact shape
+    va, sa, vb, sb = synth.make_merge_inputs(0, 128, 8, 128, "bf16", seed=3)
+    vo, so = torch.empty_like(va, device="cuda"), torch.empty_like(sa, device="cuda")
+    again.launch_merge_attn_states(va.cuda(), sa.cuda(), vb.cuda(), sb.cuda(), vo, so)
+    v_ref, s_ref = oracle_lib.merge_attn_states(va, sa, vb, sb)
+    assert oracle_lib.compare_mixed(vo.cpu(), v_ref)[1] == 0 and oracle_lib.compare_mixed(so.cpu(), s_ref, tol=1e-5)[1] == 0
+    # the fp8-output norm on another token count
+    xx, rr, ww = synth.make_inputs(77, 4096, "bf16", seed=3)
+    q = torch.empty(77, 4096, dtype=torch.uint8, device="cuda"); sc = torch.empty(77, device="cuda")
+    ro = torch.empty(77, 4096, dtype=torch.bfloat16, device="cuda")
+    again.launch_rmsnorm_fp8(xx.cuda(), rr.cuda(), ww.cuda(), q, sc, ro, EPS)
+    q_ref, sc_ref, r_ref = oracle_lib.add_rmsnorm_fp8(xx, rr, ww, EPS)
+    assert oracle_lib.compare_e4m3(q.cpu(), q_ref)[1] == 0 and oracle_lib.compare_y(sc.cpu(), sc_ref)[1] == 0
+    assert oracle_lib.bit_mismatches(ro.cpu(), r_ref) == 0
