@@ -15,7 +15,9 @@ static double shape_distance(const rt_shape& a, const rt_shape& b)
 {
     const double dh = fabs(log2((double)a.hidden) - log2((double)b.hidden));
     const double dt = fabs(log2((double)std::max<int64_t>(a.n_tokens, 1)) - log2((double)std::max<int64_t>(b.n_tokens, 1)));
-    return 4.0 * dh + dt;
+    double dd = 0.0;  // merge_attn_states: the same hidden size may be cut into heads differently
+    if (a.head_dim > 0 && b.head_dim > 0) dd = fabs(log2((double)a.head_dim) - log2((double)b.head_dim));
+    return 4.0 * dh + dt + 2.0 * dd;
 }
 
 int table_lookup(const rt_spec_entry* table, int32_t n, const rt_params* general, const rt_shape* query,
