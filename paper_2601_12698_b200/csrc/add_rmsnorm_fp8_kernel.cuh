@@ -95,7 +95,7 @@ __global__ void add_rmsnorm_fp8_kernel(const Fp8Args a)
         Vec<8> out;
         out.w[0] = pack_e4m3x2(t[0], t[1]) | (pack_e4m3x2(t[2], t[3]) << 16);
         out.w[1] = pack_e4m3x2(t[4], t[5]) | (pack_e4m3x2(t[6], t[7]) << 16);
-        st_stream<8>(qrow + (size_t)v * 8, out);
+        st_stream<8, STAGE == kStageReg>(qrow + (size_t)v * 8, out);
     };
     auto finish_row = [&](float& rho, float& inv_scale) {
         row_reduce_sum_max(ss, amax, tx, ty, tpr);
@@ -135,7 +135,7 @@ __global__ void add_rmsnorm_fp8_kernel(const Fp8Args a)
                         ss = fmaf(s[i0 + u][e], s[i0 + u][e], ss);
                         amax = fmaxf(amax, fabsf(s[i0 + u][e] * wf[e]));
                     }
-                    st_stream<VB>(orow + (size_t)v * VB, C::pack(s[i0 + u]));
+                    st_stream<VB, STAGE == kStageReg>(orow + (size_t)v * VB, C::pack(s[i0 + u]));
                 }
             }
         }
@@ -186,7 +186,7 @@ __global__ void add_rmsnorm_fp8_kernel(const Fp8Args a)
                         ss = fmaf(s[e], s[e], ss);
                         amax = fmaxf(amax, fabsf(s[e] * wf[e]));
                     }
-                    st_stream<VB>(orow + (size_t)v * VB, C::pack(s));
+                    st_stream<VB, STAGE == kStageReg>(orow + (size_t)v * VB, C::pack(s));
                 }
             }
         }

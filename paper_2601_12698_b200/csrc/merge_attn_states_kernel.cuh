@@ -134,7 +134,7 @@ __global__ void merge_attn_states_kernel(const MergeArgs a)
                 C::unpack(bv[u], yf);
 #pragma unroll
                 for (int e = 0; e < EPV; ++e) of[e] = fmaf(wa, xf[e], wb * yf[e]);
-                st_stream<VB>(po + (size_t)v * VB, C::pack(of));
+                st_stream<VB, STAGE == kStageReg>(po + (size_t)v * VB, C::pack(of));
             }
         }
     }

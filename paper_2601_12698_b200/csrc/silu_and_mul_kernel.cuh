@@ -92,7 +92,7 @@ __global__ void silu_and_mul_kernel(const SiluArgs a)
                 C::unpack(uv[u], uf);
 #pragma unroll
                 for (int e = 0; e < EPV; ++e) of[e] = silu_mul(gf[e], uf[e]);
-                st_stream<VB>(out + (size_t)v * VB, C::pack(of));
+                st_stream<VB, STAGE == kStageReg>(out + (size_t)v * VB, C::pack(of));
             }
         }
     }
