@@ -25,7 +25,7 @@ DTYPE_NAMES = {BF16: "bf16", FP16: "fp16", FP32: "fp32"}
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 SOURCES = ("add_rmsnorm_oracle.c", "silu_and_mul_oracle.c", "merge_attn_states_oracle.c",
-           "add_rmsnorm_fp8_oracle.c")
+           "add_rmsnorm_fp8_oracle.c", "allreduce_add_rmsnorm_oracle.c")
 HEADERS = ("number_formats.h",)
 _LIB = os.path.join(_HERE, "liboracle.so")
 _lock = threading.Lock()
@@ -84,6 +84,9 @@ def _bind(path: str):
     lib.oracle_encode_e4m3.restype = None
     lib.oracle_add_rmsnorm_fp8.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, ctypes.c_float, ctypes.c_int]
     lib.oracle_add_rmsnorm_fp8.restype = ctypes.c_int
+    lib.oracle_allreduce_add_rmsnorm.argtypes = [vp, ctypes.c_int, vp, vp, vp, vp, i64, i64, ctypes.c_float,
+                                                 ctypes.c_int, ctypes.c_int]
+    lib.oracle_allreduce_add_rmsnorm.restype = ctypes.c_int
     lib.oracle_e4m3_compare.argtypes = [vp, vp, i64, i32, ctypes.POINTER(i32), ctypes.POINTER(i64)]
     lib.oracle_e4m3_compare.restype = None
     return lib
@@ -232,6 +235,29 @@ def add_rmsnorm_fp8(x, r, w, eps: float, dtype: int | None = None):
         import torch
         return torch.from_numpy(q), torch.from_numpy(scale), to_torch(r_out, dt)
     return q, scale, r_out
+
+
+def allreduce_add_rmsnorm(x_parts, r, w, eps: float, dtype: int | None = None, *, threads: int = 1):
+    """y, r_out for x given as parts: x_parts [N, T, H] summed in binary32 in rank order, then the residual, then
+    the norm.  Storage arrays for numpy input, torch tensors for torch input."""
+    want_torch = hasattr(x_parts, "detach")
+    xs, dt = as_storage(x_parts, dtype)
+    rs, dt_r = as_storage(r, dtype)
+    ws, dt_w = as_storage(w, dtype)
+    if not (dt == dt_r == dt_w):
+        raise TypeError("x_parts, r and w must share one dtype")
+    if xs.ndim != 3 or xs.shape[0] < 1 or rs.shape != xs.shape[1:] or ws.shape != (xs.shape[2],):
+        raise ValueError("expected x_parts of shape [N, T, H], r of shape [T, H] and w of shape [H]")
+    N, T, H = xs.shape
+    y = np.empty_like(rs)
+    r_out = np.empty_like(rs)
+    rc = _load().oracle_allreduce_add_rmsnorm(xs.ctypes.data, N, rs.ctypes.data, ws.ctypes.data, y.ctypes.data,
+                                              r_out.ctypes.data, T, H, float(eps), dt, int(threads))
+    if rc != 0:
+        raise RuntimeError(f"oracle_allreduce_add_rmsnorm failed with status {rc}")
+    if want_torch:
+        return to_torch(y, dt), to_torch(r_out, dt)
+    return y, r_out
 
 
 def decode_e4m3(bits) -> np.ndarray:
