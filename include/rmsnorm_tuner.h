@@ -46,12 +46,17 @@ extern "C" {
 
 typedef enum { RT_BF16 = 0, RT_FP16 = 1, RT_FP32 = 2 } rt_dtype;
 
+/* Most partial inputs and most destinations one launch of the all-reduce-fused norm takes. */
+#define RT_MAX_PARTS 8
+
 /* The kernels that have a template in this library (the paper tunes three serving kernels, "Kernels"). */
 typedef enum {
     RT_OP_ADD_RMSNORM = 0,  /* fused residual-add + RMSNorm: the operator described above */
     RT_OP_SILU_AND_MUL = 1, /* out[t,j] = silu(x[t,j]) * x[t,d+j] for x of shape [n_tokens, 2*d] */
     RT_OP_MERGE_ATTN_STATES = 2, /* two partial attention results merged by their log-sum-exps */
-    RT_OP_ADD_RMSNORM_FP8 = 3    /* add_rmsnorm whose y leaves as e4m3 bytes with one scale per token */
+    RT_OP_ADD_RMSNORM_FP8 = 3,   /* add_rmsnorm whose y leaves as e4m3 bytes with one scale per token */
+    RT_OP_ADD_RMSNORM_ALLREDUCE = 4 /* add_rmsnorm whose x arrives as n_parts partial results (one per rank of a
+                                       tensor-parallel group) that are summed while they are loaded */
 } rt_op;
 
 /* Where a row lives between the two passes over it. */
@@ -88,6 +93,8 @@ typedef struct {
     int32_t min_ptr_align; /* largest power of two (bytes, <= 256) dividing all base addresses */
     int32_t op;            /* rt_op; 0 = add_rmsnorm */
     int32_t head_dim;      /* merge_attn_states: d (hidden = heads * d); 0 for the other kernels */
+    int32_t n_parts;       /* all-reduce-fused norm: partial inputs summed per element (2, 4 or 8); 0 otherwise */
+    int32_t reserved;      /* 0 */
 } rt_shape;
 
 /* r(h): the resource upper bounds the feasible region is derived from. */
@@ -140,7 +147,10 @@ typedef struct {
  * For merge_attn_states: x = v_a, r = v_b, w = s_a, aux = s_b, y = v_out, r_out = s_out, y_ref and r_ref their
  * references (the s tensors are binary32 [n_tokens, heads]; in a ring they advance by n_tokens*heads*4).
  * For the fp8-output norm: y = q (bytes, ring stride ring_stride_bytes / 2), y_ref its reference codes,
- * aux_out = scale ([n_tokens] binary32, ring stride n_tokens*4), aux_ref its reference. */
+ * aux_out = scale ([n_tokens] binary32, ring stride n_tokens*4), aux_ref its reference.
+ * For the all-reduce-fused norm: x holds the n_parts partial inputs one after the other, part k at byte offset
+ * k * n_tokens * hidden * sizeof(element) (ring stride n_parts * ring_stride_bytes); everything else as for
+ * add_rmsnorm.  The tuner times the form with one destination. */
 typedef struct {
     const void* x;     /* device, [ring_sets][n_tokens, hidden] */
     const void* r;     /* device */
@@ -258,6 +268,37 @@ int silu_and_mul_template_launch(const rt_params* p, const void* x, void* out, i
 int rmsnorm_fp8_template_launch(const rt_params* p, const void* x, const void* r, const void* w, void* q,
                                 float* scale, void* r_out, int64_t n_tokens, int64_t hidden, float eps, int dtype,
                                 void* stream);
+
+/*
+ * The tensor-parallel form of add_rmsnorm: the all-reduce that precedes the operator in tensor-parallel
+ * serving is folded into the kernel (a variant of the norm template: register stage, 16-byte vectors, shuffle
+ * reduction; axes threads per row, rows per CTA, unroll).  No counterpart in the paper, whose experiments run
+ * on one GPU; the operator is its `fused_add_rmsnorm` ("Kernels") with x = sum over ranks of x^(k).
+ *
+ * One launch computes rows [row_begin, row_begin + row_count) of the tensors:
+ *     a = fp32(x^(0));  a = a + fp32(x^(k)) for k = 1 .. n_parts-1, in this order, each a binary32 addition;
+ *     s = a + fp32(r);  r_out = round_dtype(s);  y = round_dtype(s * rsqrt(mean(s^2) + eps) * w)
+ * and writes those rows of y and r_out into EVERY destination given.  With rank k of an n-rank group calling it
+ * on its own block of rows, with all ranks' partials as x_parts and all ranks' output tensors as destinations,
+ * every rank ends with the complete y and r_out (reduce-scatter + operator + all-gather in one kernel, the
+ * transfers being the kernel's own loads and stores over peer-mapped memory).  With one destination and all
+ * rows it is the one-shot form (every rank reduces everything for itself).
+ *   x_parts   HOST array of n_parts (2, 4 or 8) DEVICE pointers, part k = rank k's partial x, each a full
+ *             [n_rows_total, hidden] tensor addressable from the current device (its own memory or a
+ *             peer-mapped allocation); read only.
+ *   r, w      device (current GPU), r a full [n_rows_total, hidden] tensor, w [hidden].
+ *   y_outs, r_outs  HOST arrays of n_outs (1..8) DEVICE pointers to full [n_rows_total, hidden] tensors; only the
+ *             launch's rows are written.  A destination may be the tensor r itself (in-place residual), never
+ *             a part of x.
+ *   All tensor pointers must be 16-byte aligned and the row length a multiple of 16 bytes (RT_ERR_ALIGN).
+ * The kernel contains no wait: the caller orders the launch after every rank's partial is complete and lets
+ * no rank read the outputs before every rank's launch has finished (a barrier of the group on both sides).
+ * Asynchronous on `stream`, allocates nothing; infeasible theta is refused without launching.
+ */
+int rmsnorm_allreduce_template_launch(const rt_params* p, const void* const* x_parts, int32_t n_parts, const void* r,
+                                      const void* w, void* const* y_outs, void* const* r_outs, int32_t n_outs,
+                                      int64_t row_begin, int64_t row_count, int64_t hidden, float eps, int dtype,
+                                      void* stream);
 
 /*
  * merge_attn_states as an instance of its own template (third kernel of the paper's "Kernels" list, shapes
@@ -455,6 +496,8 @@ int rt_kernel_instance(int32_t i, int32_t* dtype, int32_t* vec_bytes, int32_t* s
                        int32_t* unroll, int32_t* reg_vectors);
 /* The rt_op the i-th instance belongs to (-1 when i is out of range). */
 int32_t rt_kernel_instance_op(int32_t i);
+/* Partial inputs the i-th instance sums per element (all-reduce-fused norm; 0 for the others, -1 out of range). */
+int32_t rt_kernel_instance_parts(int32_t i);
 /* Kernel launches issued by this library in this process since load (all entry points). */
 int64_t rt_launch_count(void);
 /* Frees what the library allocated on the device.  Safe to call more than once. */

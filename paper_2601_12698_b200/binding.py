@@ -16,6 +16,8 @@ HEADER_PATH = os.path.join(os.path.dirname(_HERE), "include", "rmsnorm_tuner.h")
 
 RT_BF16, RT_FP16, RT_FP32 = 0, 1, 2
 RT_OP_ADD_RMSNORM, RT_OP_SILU_AND_MUL, RT_OP_MERGE_ATTN_STATES, RT_OP_ADD_RMSNORM_FP8 = 0, 1, 2, 3
+RT_OP_ADD_RMSNORM_ALLREDUCE = 4
+RT_MAX_PARTS = 8
 RT_STAGE_REG, RT_STAGE_SMEM_LDG, RT_STAGE_SMEM_TMA = 0, 1, 2
 RT_REDUCE_SHFL, RT_REDUCE_SMEM, RT_REDUCE_CLUSTER = 0, 1, 2
 RT_PRUNE_IDLE_THREADS, RT_PRUNE_DUPLICATES, RT_PRUNE_CLUSTER_WAVES, RT_PRUNE_IDLE_ROWS = 1, 2, 4, 8
@@ -53,7 +55,7 @@ def make_params(threads_per_row=256, rows_per_cta=1, vec_bytes=16, unroll=1, sta
 
 class rt_shape(Structure):
     _fields_ = [("n_tokens", c_int64), ("hidden", c_int64), ("dtype", c_int32), ("min_ptr_align", c_int32),
-                ("op", c_int32), ("head_dim", c_int32)]
+                ("op", c_int32), ("head_dim", c_int32), ("n_parts", c_int32), ("reserved", c_int32)]
 
 
 class rt_limits(Structure):
@@ -109,6 +111,10 @@ _SIGNATURES = {
     "silu_and_mul_template_launch": (c_int, [POINTER(rt_params), c_void_p, c_void_p, c_int64, c_int64, c_int, c_void_p]),
     "rmsnorm_fp8_template_launch": (c_int, [POINTER(rt_params), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                             c_int64, c_int64, c_float, c_int, c_void_p]),
+    "rmsnorm_allreduce_template_launch": (c_int, [POINTER(rt_params), POINTER(c_void_p), c_int32, c_void_p, c_void_p,
+                                                  POINTER(c_void_p), POINTER(c_void_p), c_int32, c_int64, c_int64,
+                                                  c_int64, c_float, c_int, c_void_p]),
+    "rt_kernel_instance_parts": (c_int32, [c_int32]),
     "merge_attn_states_template_launch": (c_int, [POINTER(rt_params), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                                   c_void_p, c_int64, c_int64, c_int64, c_int, c_void_p]),
     "rmsnorm_template_run_host": (c_int, [POINTER(rt_params), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
@@ -197,10 +203,11 @@ def _ptr_align(*tensors) -> int:
 
 
 def shape_of(n_tokens: int, hidden: int, dtype, min_ptr_align: int = 256, op: int = RT_OP_ADD_RMSNORM,
-             head_dim: int = 0) -> rt_shape:
-    """hidden is the output row width (d for silu_and_mul, heads * head_dim for merge_attn_states)."""
+             head_dim: int = 0, n_parts: int = 0) -> rt_shape:
+    """hidden is the output row width (d for silu_and_mul, heads * head_dim for merge_attn_states); n_parts is the
+    number of partial inputs of the all-reduce-fused norm."""
     code = DTYPE_CODES[dtype] if isinstance(dtype, str) else int(dtype)
-    return rt_shape(n_tokens, hidden, code, min_ptr_align, op, head_dim)
+    return rt_shape(n_tokens, hidden, code, min_ptr_align, op, head_dim, n_parts, 0)
 
 
 def sm100_nominal_limits() -> rt_limits:
@@ -255,6 +262,27 @@ def rmsnorm_fp8_template_launch(params: rt_params, x, r, w, q, scale, r_out, eps
     _check(lib.rmsnorm_fp8_template_launch(byref(params), x.data_ptr(), r.data_ptr(), w.data_ptr(), q.data_ptr(),
                                            scale.data_ptr(), r_out.data_ptr(), n_tokens, hidden, eps, _dtype_code(x),
                                            _stream_ptr(stream)), "rmsnorm_fp8_template_launch")
+
+
+def rmsnorm_allreduce_template_launch(params: rt_params, x_parts, r, w, y_outs, r_outs, row_begin: int, row_count: int,
+                                      eps: float, stream=None) -> None:
+    """The tensor-parallel form of add_rmsnorm on rows [row_begin, row_begin + row_count): x_parts is a list of 2, 4
+    or 8 device tensors [T, H] (one partial x per rank, each addressable from the current device), y_outs / r_outs
+    lists of 1..8 destination tensors [T, H] that all receive those rows.  Asynchronous."""
+    n_rows, hidden = r.shape
+    tensors = list(x_parts) + [r] + list(y_outs) + list(r_outs)
+    ok = (all(t.is_cuda and t.is_contiguous() and t.shape == (n_rows, hidden) and t.dtype == r.dtype for t in tensors)
+          and w.is_cuda and w.is_contiguous() and w.shape == (hidden,) and w.dtype == r.dtype
+          and len(y_outs) == len(r_outs) and 0 <= row_begin and row_begin + row_count <= n_rows)
+    if not ok:
+        raise ValueError("rmsnorm_allreduce_template_launch: tensors of the wrong device, layout, shape or dtype, "
+                         "or rows out of range")
+    xp = (c_void_p * len(x_parts))(*[t.data_ptr() for t in x_parts])
+    yo = (c_void_p * len(y_outs))(*[t.data_ptr() for t in y_outs])
+    ro = (c_void_p * len(r_outs))(*[t.data_ptr() for t in r_outs])
+    _check(lib.rmsnorm_allreduce_template_launch(byref(params), xp, len(x_parts), r.data_ptr(), w.data_ptr(), yo, ro,
+                                                 len(y_outs), row_begin, row_count, hidden, eps, _dtype_code(r),
+                                                 _stream_ptr(stream)), "rmsnorm_allreduce_template_launch")
 
 
 def merge_attn_states_template_launch(params: rt_params, v_a, s_a, v_b, s_b, v_out, s_out, stream=None) -> None:
@@ -512,7 +540,7 @@ class SpecTable:
         return {"device": self.device_name, "general": self.general.as_dict() if self.general else None,
                 "generals": {str(op): th.as_dict() for op, th in sorted(self.generals.items())},
                 "specialised": [{"dtype": names[s.dtype], "n_tokens": int(s.n_tokens), "hidden": int(s.hidden),
-                                 "op": int(s.op), "head_dim": int(s.head_dim), "theta": t.as_dict(), "us": round(float(us), 3)}
+                                 "op": int(s.op), "head_dim": int(s.head_dim), "n_parts": int(s.n_parts), "theta": t.as_dict(), "us": round(float(us), 3)}
                                 for s, t, us in self.entries]}
 
     @classmethod
@@ -527,7 +555,7 @@ class SpecTable:
         fields = [k for k, _ in rt_params._fields_]
         mk = lambda t: rt_params(*[int(t[k]) for k in fields])
         entries = [(shape_of(e["n_tokens"], e["hidden"], e["dtype"], op=int(e.get("op", 0)),
-                             head_dim=int(e.get("head_dim", 0))), mk(e["theta"]), float(e["us"]))
+                             head_dim=int(e.get("head_dim", 0)), n_parts=int(e.get("n_parts", 0))), mk(e["theta"]), float(e["us"]))
                    for e in d.get("specialised", [])]
         generals = {int(op): mk(th) for op, th in (d.get("generals") or {}).items()}
         return cls(entries, mk(d["general"]) if d.get("general") else None, d.get("device", ""), generals)
@@ -548,6 +576,7 @@ def kernel_instances() -> list[dict]:
         _check(lib.rt_kernel_instance(i, *[byref(v) for v in vals]), "rt_kernel_instance")
         out.append(dict(zip(("dtype", "vec_bytes", "stage", "reduce", "unroll", "reg_vectors"), (v.value for v in vals))))
         out[-1]["op"] = int(lib.rt_kernel_instance_op(i))
+        out[-1]["parts"] = int(lib.rt_kernel_instance_parts(i))
     return out
 
 

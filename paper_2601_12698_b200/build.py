@@ -30,7 +30,7 @@ NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-std=c++17", "-O3",
               "-Xcompiler", "-fPIC", "-I", CSRC, "-I", INCLUDE]
 HOST_UNITS = ["launch.cu", "feasible.cu", "search.cu", "host_run.cu", "table.cu"]
 ELEMENT_TYPES = {"bf16": ("__nv_bfloat16", 0), "fp16": ("__half", 1), "fp32": ("float", 2)}
-GROUPS = {"reg": 0, "smem": 1, "narrow": 2, "silu": 3, "merge": 4, "fp8out": 5}
+GROUPS = {"reg": 0, "smem": 1, "narrow": 2, "silu": 3, "merge": 4, "fp8out": 5, "allreduce": 6}
 
 
 def instance_units() -> list[str]:
@@ -39,7 +39,7 @@ def instance_units() -> list[str]:
 
 
 def unit_flags(name: str) -> list[str]:
-    m = re.fullmatch(r"(bf16|fp16|fp32)_v(\d+)_(reg|smem|narrow|silu|merge|fp8out)(?:_r(\d))?", name)
+    m = re.fullmatch(r"(bf16|fp16|fp32)_v(\d+)_(reg|smem|narrow|silu|merge|fp8out|allreduce)(?:_r(\d))?", name)
     if not m:
         raise ValueError(f"cannot parse instantiation unit name {name!r}")
     ctype, code = ELEMENT_TYPES[m.group(1)]
@@ -67,33 +67,41 @@ _FP8_ENTRY = re.compile(r"Compiling entry function '_ZN2rt22add_rmsnorm_fp8_kern
                         r"EEvNS_7Fp8ArgsE'.*?(\d+) bytes spill stores.*?Used (\d+) registers(?:.*?(\d+) bytes smem)?", re.S)
 
 
+_ALLREDUCE_ENTRY = re.compile(r"Compiling entry function '_ZN2rt28add_rmsnorm_allreduce_kernelI(\w+?)Li(\d+)ELi(\d+)ELi(\d+)E"
+                              r"EEvNS_13AllreduceArgsE'.*?(\d+) bytes spill stores.*?Used (\d+) registers(?:.*?(\d+) bytes smem)?", re.S)
+
+
 def parse_ptxas(log: str) -> list[tuple]:
-    """(op, dtype, vec, stage, reduce, unroll, cap, registers, static smem, spill bytes) per entry function."""
+    """(op, dtype, vec, stage, reduce, unroll, cap, registers, static smem, spill bytes, parts) per entry function."""
     rows = []
     for m in _ENTRY.finditer(log):
         t, vb, st, rd, u, cap, spill, regs, smem = m.groups()
         rows.append((0, _MANGLED_DTYPE[t], int(vb), int(st), int(rd), int(u), int(cap) if int(st) == 0 else 0,
-                     int(regs), int(smem), int(spill)))
+                     int(regs), int(smem), int(spill), 0))
     for block in log.split("ptxas info    : Compiling entry function")[1:]:
         for op, pattern in ((1, _SILU_ENTRY), (2, _MERGE_ENTRY)):
             m = pattern.search("Compiling entry function" + block)
             if m:
                 t, vb, st, u, spill, regs, smem = m.groups()
-                rows.append((op, _MANGLED_DTYPE[t], int(vb), int(st), 0, int(u), 0, int(regs), int(smem or 0), int(spill)))
+                rows.append((op, _MANGLED_DTYPE[t], int(vb), int(st), 0, int(u), 0, int(regs), int(smem or 0), int(spill), 0))
     for block in log.split("ptxas info    : Compiling entry function")[1:]:
         m = _FP8_ENTRY.search("Compiling entry function" + block)
         if m:
             t, st, u, cap, spill, regs, smem = m.groups()
             rows.append((3, _MANGLED_DTYPE[t], 16, int(st), 0, int(u), int(cap) if int(st) == 0 else 0, int(regs),
-                         int(smem or 0), int(spill)))
+                         int(smem or 0), int(spill), 0))
+        m = _ALLREDUCE_ENTRY.search("Compiling entry function" + block)
+        if m:
+            t, parts, u, cap, spill, regs, smem = m.groups()
+            rows.append((4, _MANGLED_DTYPE[t], 16, 0, 0, int(u), int(cap), int(regs), int(smem or 0), int(spill), int(parts)))
     return rows
 
 
 def write_resource_table(rows: list[tuple]) -> str:
     path = os.path.join(OBJ_DIR, "instance_resources.inc")
     lines = ["// Generated by build.py from the ptxas reports of the instantiation units: per instance\n"
-             "// {op, dtype, vec_bytes, stage, reduce, unroll, cap, registers per thread, static smem, spill bytes}.\n"]
-    lines += ["{%d, %d, %d, %d, %d, %d, %d, %d, %d, %d},\n" % r for r in sorted(set(rows))]
+             "// {op, dtype, vec_bytes, stage, reduce, unroll, cap, registers per thread, static smem, spill bytes, parts}.\n"]
+    lines += ["{%d, %d, %d, %d, %d, %d, %d, %d, %d, %d, %d},\n" % r for r in sorted(set(rows))]
     text = "".join(lines)
     if not os.path.exists(path) or open(path).read() != text:
         with open(path, "w") as f:

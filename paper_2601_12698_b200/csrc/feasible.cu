@@ -63,6 +63,9 @@ std::vector<rt_params> raw_grid(const rt_shape& s)
                 // the fp8-output norm: 16-byte vectors, shuffle reduction, register or TMA stage
                 if (s.op == RT_OP_ADD_RMSNORM_FP8 && (stage == RT_STAGE_SMEM_LDG || m.reduce != RT_REDUCE_SHFL || vb != 16))
                     continue;
+                // the all-reduce-fused norm: 16-byte vectors, shuffle reduction, register stage
+                if (s.op == RT_OP_ADD_RMSNORM_ALLREDUCE && (stage != RT_STAGE_REG || m.reduce != RT_REDUCE_SHFL || vb != 16))
+                    continue;
                 for (int tpr : kTprLevels)
                     for (int rpc : kRpcLevels)
                         for (int u : kUnrollLevels) {

@@ -1,6 +1,6 @@
 // One instantiation unit of the kernel template.  Compiled once per line of instance_units.inc with
 //   -DRT_UNIT_NAME=<name> -DRT_UNIT_T=<element type> -DRT_UNIT_DTYPE=<0|1|2> -DRT_UNIT_VB=<bytes>
-//   -DRT_UNIT_GROUP=<0 register stage | 1 shared-memory stages | 2 narrow fall-back | 3 silu_and_mul | 4 merge_attn_states | 5 fp8-output norm>
+//   -DRT_UNIT_GROUP=<0 register stage | 1 shared-memory stages | 2 narrow fall-back | 3 silu_and_mul | 4 merge_attn_states | 5 fp8-output norm | 6 all-reduce-fused norm>
 //   -DRT_UNIT_REDUCE=<0|1|2>   (register-stage units only)
 //
 // Instance lists.  Register stage: CAP (row vectors kept per thread) in {1,2,4,8,16,32} while the row
@@ -12,6 +12,10 @@
 // merge_attn_states: the same instance list as silu_and_mul.
 // fp8-output norm (16-bit element types, 16-byte vectors, shuffle reduction): register stage with CAP in
 // {1,2,4,8,16} and U <= CAP, TMA stage with U in {1,2,4}.
+// all-reduce-fused norm (16-byte vectors, register stage, shuffle reduction): 2, 4 and 8 parts, CAP in
+// {1,2,4,8,16} while the row stays within 128 fp32 registers per thread, U <= CAP with U * parts <= 16 loads of x
+// in flight per thread.
+#include "add_rmsnorm_allreduce_kernel.cuh"
 #include "add_rmsnorm_fp8_kernel.cuh"
 #include "add_rmsnorm_kernel.cuh"
 #include "merge_attn_states_kernel.cuh"
@@ -58,6 +62,21 @@ rt::KernelEntry fp8_entry()
     }
 }
 
+template <int NP, int U, int CAP>
+rt::KernelEntry allreduce_entry()
+{
+    if constexpr (CAP * (16 / (int)sizeof(T)) > kMaxRowRegisters || U * NP > 16) {
+        return rt::KernelEntry{RT_OP_ADD_RMSNORM_ALLREDUCE, kDtype, 16, 0, 0, U, CAP, nullptr, NP};
+    } else {
+        return rt::KernelEntry{RT_OP_ADD_RMSNORM_ALLREDUCE, kDtype, 16, 0, 0, U, CAP,
+                               (const void*)&rt::add_rmsnorm_allreduce_kernel<T, NP, U, CAP>, NP};
+    }
+}
+#define RT_ALLREDUCE_LIST(NP)                                                                                     \
+    allreduce_entry<NP, 1, 1>(), allreduce_entry<NP, 1, 2>(), allreduce_entry<NP, 2, 2>(), allreduce_entry<NP, 1, 4>(), \
+    allreduce_entry<NP, 2, 4>(), allreduce_entry<NP, 4, 4>(), allreduce_entry<NP, 1, 8>(), allreduce_entry<NP, 2, 8>(), \
+    allreduce_entry<NP, 4, 8>(), allreduce_entry<NP, 1, 16>(), allreduce_entry<NP, 2, 16>(), allreduce_entry<NP, 4, 16>()
+
 template <int VB, int ST, int U>
 rt::KernelEntry merge_entry()
 {
@@ -97,6 +116,8 @@ std::vector<rt::KernelEntry> build_entries()
         fp8_entry<0, 1, 1>(), fp8_entry<0, 1, 2>(), fp8_entry<0, 2, 2>(), fp8_entry<0, 1, 4>(), fp8_entry<0, 2, 4>(),
         fp8_entry<0, 4, 4>(), fp8_entry<0, 1, 8>(), fp8_entry<0, 2, 8>(), fp8_entry<0, 4, 8>(), fp8_entry<0, 1, 16>(),
         fp8_entry<0, 2, 16>(), fp8_entry<0, 4, 16>(), fp8_entry<2, 1, 1>(), fp8_entry<2, 2, 1>(), fp8_entry<2, 4, 1>()
+#elif RT_UNIT_GROUP == 6
+        RT_ALLREDUCE_LIST(2), RT_ALLREDUCE_LIST(4), RT_ALLREDUCE_LIST(8)
 #elif RT_UNIT_GROUP == 4
         RT_MERGE_WIDE(16), RT_MERGE_WIDE(8), merge_entry<4, 0, 1>(), merge_entry<4, 0, 4>(), merge_entry<2, 0, 1>(),
         merge_entry<2, 0, 4>()

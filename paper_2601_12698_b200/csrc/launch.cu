@@ -8,6 +8,7 @@
 #include <mutex>
 #include <unordered_map>
 
+#include "add_rmsnorm_allreduce_kernel.cuh"
 #include "add_rmsnorm_fp8_kernel.cuh"
 #include "add_rmsnorm_kernel.cuh"
 #include "merge_attn_states_kernel.cuh"
@@ -20,6 +21,8 @@
 #undef RT_DECLARE_SLICE
 
 namespace rt {
+
+static_assert(kMaxParts == RT_MAX_PARTS, "the kernel's argument arrays hold RT_MAX_PARTS pointers");
 
 __device__ int g_status_word = 0;
 
@@ -40,9 +43,9 @@ struct DeviceCache {
 };
 DeviceCache g_dev[kMaxDevices];
 
-uint64_t key_of(int op, int dtype, int vb, int stage, int reduce, int unroll, int cap)
+uint64_t key_of(int op, int dtype, int vb, int stage, int reduce, int unroll, int cap, int parts = 0)
 {
-    return ((uint64_t)op << 48) | ((uint64_t)dtype << 40) | ((uint64_t)vb << 32) | ((uint64_t)stage << 28) | ((uint64_t)reduce << 24) |
+    return ((uint64_t)parts << 56) | ((uint64_t)op << 48) | ((uint64_t)dtype << 40) | ((uint64_t)vb << 32) | ((uint64_t)stage << 28) | ((uint64_t)reduce << 24) |
            ((uint64_t)unroll << 16) | (uint64_t)cap;
 }
 
@@ -60,7 +63,7 @@ struct Registry {
 #undef RT_DECLARE_SLICE
         for (int i = 0; i < (int)entries.size(); ++i) {
             const KernelEntry& e = entries[i];
-            index[key_of(e.op, e.dtype, e.vec_bytes, e.stage, e.reduce, e.unroll, e.cap)] = i;
+            index[key_of(e.op, e.dtype, e.vec_bytes, e.stage, e.reduce, e.unroll, e.cap, e.parts)] = i;
         }
     }
 };
@@ -105,9 +108,9 @@ void count_launch(int64_t n) { g_launches.fetch_add(n, std::memory_order_relaxed
 
 const std::vector<KernelEntry>& registry() { return reg().entries; }
 
-int find_kernel(int op, int dtype, int vb, int stage, int reduce, int unroll, int cap)
+int find_kernel(int op, int dtype, int vb, int stage, int reduce, int unroll, int cap, int parts)
 {
-    auto it = reg().index.find(key_of(op, dtype, vb, stage, reduce, unroll, cap));
+    auto it = reg().index.find(key_of(op, dtype, vb, stage, reduce, unroll, cap, parts));
     return it == reg().index.end() ? -1 : it->second;
 }
 
@@ -224,7 +227,7 @@ int min_pointer_alignment(const void* a, const void* b, const void* c, const voi
 // this build (table generated by the build script).  Used when no device can be asked; with a device the
 // runtime's own figures are used instead.
 struct InstanceResources {
-    int op, dtype, vec_bytes, stage, reduce, unroll, cap, regs, static_smem, spill_bytes;
+    int op, dtype, vec_bytes, stage, reduce, unroll, cap, regs, static_smem, spill_bytes, parts;
 };
 static const InstanceResources kInstanceResources[] = {
 #include "instance_resources.inc"
@@ -234,10 +237,10 @@ static const InstanceResources* build_resources(const KernelEntry& k)
     static std::unordered_map<uint64_t, const InstanceResources*> index = [] {
         std::unordered_map<uint64_t, const InstanceResources*> m;
         for (const InstanceResources& r : kInstanceResources)
-            m[key_of(r.op, r.dtype, r.vec_bytes, r.stage, r.reduce, r.unroll, r.cap)] = &r;
+            m[key_of(r.op, r.dtype, r.vec_bytes, r.stage, r.reduce, r.unroll, r.cap, r.parts)] = &r;
         return m;
     }();
-    auto it = index.find(key_of(k.op, k.dtype, k.vec_bytes, k.stage, k.reduce, k.unroll, k.cap));
+    auto it = index.find(key_of(k.op, k.dtype, k.vec_bytes, k.stage, k.reduce, k.unroll, k.cap, k.parts));
     return it == index.end() ? nullptr : it->second;
 }
 static int model_regs(const KernelEntry& k, int elem_bytes)
@@ -269,7 +272,7 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
         plan->reject_reason = kRejectArgs;
         return RT_ERR_DTYPE;
     }
-    if (s->op < RT_OP_ADD_RMSNORM || s->op > RT_OP_ADD_RMSNORM_FP8) {
+    if (s->op < RT_OP_ADD_RMSNORM || s->op > RT_OP_ADD_RMSNORM_ALLREDUCE) {
         set_error("op %d is not a kernel of this library", s->op);
         plan->reject_reason = kRejectArgs;
         return RT_ERR_SHAPE;
@@ -279,6 +282,7 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
     const bool is_merge = s->op == RT_OP_MERGE_ATTN_STATES;
     const bool no_reduction = is_silu || is_merge;  // element-wise kernels: no reduction axis, no CAP
     const bool is_fp8 = s->op == RT_OP_ADD_RMSNORM_FP8;
+    const bool is_allreduce = s->op == RT_OP_ADD_RMSNORM_ALLREDUCE;
     const int eb = elem_bytes_of(s->dtype);
     if (s->n_tokens < 0 || s->hidden <= 0 || s->hidden * eb * (is_silu ? 2 : 1) >= (int64_t)1 << 31) {
         set_error("shape n_tokens=%lld hidden=%lld is out of range", (long long)s->n_tokens, (long long)s->hidden);
@@ -328,6 +332,17 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
                   p->cluster_size, p->stage);
         plan->reject_reason = kRejectArgs;
         return s->dtype == RT_FP32 ? RT_ERR_DTYPE : RT_ERR_INFEASIBLE;
+    }
+    if (is_allreduce && !(s->n_parts == 2 || s->n_parts == 4 || s->n_parts == 8)) {
+        set_error("n_parts=%d is not 2, 4 or 8", s->n_parts);
+        plan->reject_reason = kRejectArgs;
+        return RT_ERR_SHAPE;
+    }
+    if (is_allreduce && (p->vec_bytes != 16 || p->reduce != RT_REDUCE_SHFL || p->cluster_size != 1 || p->stage != RT_STAGE_REG)) {
+        set_error("the all-reduce-fused norm takes 16-byte vectors, the shuffle reduction and the register stage "
+                  "(vec=%d reduce=%d cluster=%d stage=%d)", p->vec_bytes, p->reduce, p->cluster_size, p->stage);
+        plan->reject_reason = kRejectArgs;
+        return RT_ERR_INFEASIBLE;
     }
     if (no_reduction && (p->reduce != RT_REDUCE_SHFL || p->cluster_size != 1 || p->stage == RT_STAGE_SMEM_LDG)) {
         set_error("this kernel has no reduction and no ld.global->shared stage (reduce=%d cluster=%d stage=%d)",
@@ -398,7 +413,7 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
     }
     plan->cap = cap;
     plan->unroll_eff = unroll;
-    plan->kernel_index = find_kernel(s->op, s->dtype, vb, p->stage, p->reduce, unroll, cap);
+    plan->kernel_index = find_kernel(s->op, s->dtype, vb, p->stage, p->reduce, unroll, cap, is_allreduce ? s->n_parts : 0);
     if (plan->kernel_index < 0) {
         if (p->stage == RT_STAGE_REG && !no_reduction)
             set_error("a row slice of %d vectors over %d threads needs %d vectors per thread: no register-stage "
@@ -533,6 +548,50 @@ int launch_fp8_plan(const Plan& plan, const void* x, const void* r, const void* 
     cfg.gridDim = dim3(plan.grid_x, 1, 1);
     cfg.blockDim = dim3(plan.block_x, plan.block_y, 1);
     cfg.dynamicSmemBytes = plan.dyn_smem;
+    cfg.stream = stream;
+    void* params[] = {&a};
+    cudaError_t e = cudaLaunchKernelExC(&cfg, k.fn, params);
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        set_error("kernel launch failed: %s", cudaGetErrorString(e));
+        return RT_ERR_CUDA;
+    }
+    count_launch();
+    return RT_OK;
+}
+
+int launch_allreduce_plan(const Plan& plan, const void* const* x_parts, int n_parts, const void* r, const void* w,
+                          void* const* y_outs, void* const* r_outs, int n_outs, int64_t row_begin, int64_t row_count,
+                          int64_t hidden, float eps, cudaStream_t stream)
+{
+    if (row_count == 0) return RT_OK;
+    const KernelEntry& k = registry()[plan.kernel_index];
+    if (plan.op != RT_OP_ADD_RMSNORM_ALLREDUCE || k.parts != n_parts) {
+        set_error("plan belongs to another kernel");
+        return RT_ERR_INFEASIBLE;
+    }
+    if (n_outs < 1 || n_outs > kMaxParts) {
+        set_error("n_outs=%d outside 1..%d", n_outs, kMaxParts);
+        return RT_ERR_SHAPE;
+    }
+    AllreduceArgs a;
+    memset(&a, 0, sizeof(a));
+    for (int i = 0; i < n_parts; ++i) a.x_parts[i] = x_parts[i];
+    for (int i = 0; i < n_outs; ++i) {
+        a.y_outs[i] = y_outs[i];
+        a.r_outs[i] = r_outs[i];
+    }
+    a.r = r; a.w = w;
+    a.n_outs = n_outs;
+    a.row_begin = row_begin;
+    a.row_end = row_begin + row_count;
+    a.hidden = (int)hidden;
+    a.nvec = plan.nvec;
+    a.eps = eps;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(plan.grid_x, 1, 1);
+    cfg.blockDim = dim3(plan.block_x, plan.block_y, 1);
     cfg.stream = stream;
     void* params[] = {&a};
     cudaError_t e = cudaLaunchKernelExC(&cfg, k.fn, params);
@@ -685,7 +744,7 @@ int rmsnorm_template_launch(const rt_params* p, const void* x, const void* r, co
     rt_limits L;
     int st = rt::current_limits(&L);
     if (st != RT_OK) return st;
-    rt_shape s;
+    rt_shape s = {};
     s.n_tokens = n_tokens;
     s.hidden = hidden;
     s.dtype = dtype;
@@ -712,7 +771,7 @@ int silu_and_mul_template_launch(const rt_params* p, const void* x, void* out, i
     rt_limits L;
     int st = rt::current_limits(&L);
     if (st != RT_OK) return st;
-    rt_shape s;
+    rt_shape s = {};
     s.n_tokens = n_tokens;
     s.hidden = d;
     s.dtype = dtype;
@@ -743,7 +802,7 @@ int rmsnorm_fp8_template_launch(const rt_params* p, const void* x, const void* r
     rt_limits L;
     int st = rt::current_limits(&L);
     if (st != RT_OK) return st;
-    rt_shape s;
+    rt_shape s = {};
     s.n_tokens = n_tokens;
     s.hidden = hidden;
     s.dtype = dtype;
@@ -754,6 +813,70 @@ int rmsnorm_fp8_template_launch(const rt_params* p, const void* x, const void* r
     st = rt::make_plan(&s, p, &L, &plan);
     if (st != RT_OK) return st;
     return rt::launch_fp8_plan(plan, x, r, w, q, scale, r_out, n_tokens, hidden, eps, (cudaStream_t)stream);
+}
+
+int rmsnorm_allreduce_template_launch(const rt_params* p, const void* const* x_parts, int32_t n_parts, const void* r,
+                                      const void* w, void* const* y_outs, void* const* r_outs, int32_t n_outs,
+                                      int64_t row_begin, int64_t row_count, int64_t hidden, float eps, int dtype,
+                                      void* stream)
+{
+    if (!p) {
+        rt::set_error("params is NULL");
+        return RT_ERR_NULL;
+    }
+    if (!(n_parts == 2 || n_parts == 4 || n_parts == 8)) {
+        rt::set_error("n_parts=%d is not 2, 4 or 8", n_parts);
+        return RT_ERR_SHAPE;
+    }
+    if (n_outs < 1 || n_outs > rt::kMaxParts) {
+        rt::set_error("n_outs=%d outside 1..%d", n_outs, rt::kMaxParts);
+        return RT_ERR_SHAPE;
+    }
+    if (row_begin < 0 || row_count < 0) {
+        rt::set_error("row_begin=%lld row_count=%lld out of range", (long long)row_begin, (long long)row_count);
+        return RT_ERR_SHAPE;
+    }
+    if (row_count > 0 && (!x_parts || !y_outs || !r_outs || !r || !w)) {
+        rt::set_error("a tensor pointer is NULL");
+        return RT_ERR_NULL;
+    }
+    uintptr_t bits = (uintptr_t)r | (uintptr_t)w | 256u;
+    if (row_count > 0) {
+        for (int i = 0; i < n_parts; ++i) {
+            if (!x_parts[i]) {
+                rt::set_error("x_parts[%d] is NULL", i);
+                return RT_ERR_NULL;
+            }
+            bits |= (uintptr_t)x_parts[i];
+        }
+        for (int i = 0; i < n_outs; ++i) {
+            if (!y_outs[i] || !r_outs[i]) {
+                rt::set_error("destination %d is NULL", i);
+                return RT_ERR_NULL;
+            }
+            bits |= (uintptr_t)y_outs[i] | (uintptr_t)r_outs[i];
+            for (int k = 0; k < n_parts; ++k)
+                if (y_outs[i] == x_parts[k] || r_outs[i] == x_parts[k]) {
+                    rt::set_error("destination %d is part %d of x", i, k);
+                    return RT_ERR_SHAPE;
+                }
+        }
+    }
+    rt_limits L;
+    int st = rt::current_limits(&L);
+    if (st != RT_OK) return st;
+    rt_shape s = {};
+    s.n_tokens = row_count;
+    s.hidden = hidden;
+    s.dtype = dtype;
+    s.min_ptr_align = (int32_t)(bits & (~bits + 1));
+    s.op = RT_OP_ADD_RMSNORM_ALLREDUCE;
+    s.n_parts = n_parts;
+    rt::Plan plan;
+    st = rt::make_plan(&s, p, &L, &plan);
+    if (st != RT_OK) return st;
+    return rt::launch_allreduce_plan(plan, x_parts, n_parts, r, w, y_outs, r_outs, n_outs, row_begin, row_count, hidden, eps,
+                                     (cudaStream_t)stream);
 }
 
 int merge_attn_states_template_launch(const rt_params* p, const void* v_a, const float* s_a, const void* v_b,
@@ -779,7 +902,7 @@ int merge_attn_states_template_launch(const rt_params* p, const void* v_a, const
     rt_limits L;
     int st = rt::current_limits(&L);
     if (st != RT_OK) return st;
-    rt_shape s;
+    rt_shape s = {};
     s.n_tokens = n_tokens;
     s.hidden = heads * head_dim;
     s.dtype = dtype;
@@ -891,6 +1014,12 @@ int32_t rt_kernel_instance_op(int32_t i)
 {
     if (i < 0 || i >= (int32_t)rt::registry().size()) return -1;
     return rt::registry()[i].op;
+}
+
+int32_t rt_kernel_instance_parts(int32_t i)
+{
+    if (i < 0 || i >= (int32_t)rt::registry().size()) return -1;
+    return rt::registry()[i].parts;
 }
 
 int64_t rt_launch_count(void) { return rt::g_launches.load(); }

@@ -384,13 +384,26 @@ struct DeviceEvaluator : Evaluator {
         const bool is_silu = shape.op == RT_OP_SILU_AND_MUL;
         const bool is_merge = shape.op == RT_OP_MERGE_ATTN_STATES;
         const bool is_fp8 = shape.op == RT_OP_ADD_RMSNORM_FP8;
+        const bool is_allreduce = shape.op == RT_OP_ADD_RMSNORM_ALLREDUCE;
+        // the all-reduce-fused norm: the parts of x lie one after the other in ws.x; one destination
+        auto launch_allreduce = [&](size_t off) {
+            const void* parts[RT_MAX_PARTS];
+            for (int k = 0; k < shape.n_parts; ++k)
+                parts[k] = (const char*)ws.x + (size_t)shape.n_parts * off + (size_t)k * set_bytes;
+            void* y_out = (char*)ws.y + off;
+            void* r_out = (char*)ws.r_out + off;
+            return launch_allreduce_plan(plan, parts, shape.n_parts, (const char*)ws.r + off, ws.w, &y_out, &r_out, 1, 0,
+                                         shape.n_tokens, shape.hidden, ws.eps, stream);
+        };
         const size_t lse_bytes = is_merge ? (size_t)shape.n_tokens * plan.heads * sizeof(float) : 0;  // one s tensor
         RT_CUDA_OK(cudaMemsetAsync(ws.y, 0xFF, is_fp8 ? set_bytes / eb : set_bytes, stream));
         if (is_fp8) RT_CUDA_OK(cudaMemsetAsync(ws.aux_out, 0xFF, (size_t)shape.n_tokens * sizeof(float), stream));
         if (is_merge) RT_CUDA_OK(cudaMemsetAsync(ws.r_out, 0xFF, lse_bytes, stream));
         else if (!is_silu) RT_CUDA_OK(cudaMemsetAsync(ws.r_out, 0xFF, set_bytes, stream));
         RT_CUDA_OK(cudaMemsetAsync(sc->dev, 0, kAccSlots * sizeof(CompareAcc), stream));
-        if (is_fp8)
+        if (is_allreduce)
+            st = launch_allreduce(0);
+        else if (is_fp8)
             st = launch_fp8_plan(plan, ws.x, ws.r, ws.w, ws.y, (float*)ws.aux_out, ws.r_out, shape.n_tokens, shape.hidden,
                                  ws.eps, stream);
         else if (is_merge)
@@ -460,6 +473,7 @@ struct DeviceEvaluator : Evaluator {
         const int sets = ws.ring_sets > 0 ? ws.ring_sets : 1;
         auto launch_set = [&](int k) {
             const size_t off = (size_t)(k % sets) * (size_t)ws.ring_stride_bytes;
+            if (is_allreduce) return launch_allreduce(off);
             if (is_fp8)
                 return launch_fp8_plan(plan, (const char*)ws.x + off, (const char*)ws.r + off, ws.w, (char*)ws.y + off / eb,
                                        (float*)((char*)ws.aux_out + (size_t)(k % sets) * shape.n_tokens * sizeof(float)),

@@ -17,6 +17,8 @@ static double shape_distance(const rt_shape& a, const rt_shape& b)
     const double dt = fabs(log2((double)std::max<int64_t>(a.n_tokens, 1)) - log2((double)std::max<int64_t>(b.n_tokens, 1)));
     double dd = 0.0;  // merge_attn_states: the same hidden size may be cut into heads differently
     if (a.head_dim > 0 && b.head_dim > 0) dd = fabs(log2((double)a.head_dim) - log2((double)b.head_dim));
+    // all-reduce-fused norm: the part count multiplies the loads in flight per thread
+    if (a.n_parts > 0 && b.n_parts > 0) dd += fabs(log2((double)a.n_parts) - log2((double)b.n_parts));
     return 4.0 * dh + dt + 2.0 * dd;
 }
 
@@ -136,7 +138,7 @@ int rmsnorm_launch_auto(const rt_spec_entry* table, int32_t n_entries, const rt_
         rt::set_error("a tensor pointer is NULL");
         return RT_ERR_NULL;
     }
-    rt_shape s;
+    rt_shape s = {};
     s.n_tokens = n_tokens;
     s.hidden = hidden;
     s.dtype = dtype;

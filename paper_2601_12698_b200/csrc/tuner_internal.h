@@ -16,6 +16,7 @@ struct KernelEntry {
     int op;
     int dtype, vec_bytes, stage, reduce, unroll, cap;  // cap: per-thread row vectors (register stage), else 0
     const void* fn;
+    int parts = 0;  // all-reduce-fused norm: partial inputs summed per element
 };
 struct KernelSlice {
     const KernelEntry* entries;
@@ -59,7 +60,7 @@ const char* last_error();
 inline int elem_bytes_of(int dtype) { return dtype == RT_FP32 ? 4 : 2; }
 
 const std::vector<KernelEntry>& registry();
-int find_kernel(int op, int dtype, int vec_bytes, int stage, int reduce, int unroll, int cap);
+int find_kernel(int op, int dtype, int vec_bytes, int stage, int reduce, int unroll, int cap, int parts = 0);
 // Cached cudaFuncGetAttributes of instance `index` on the current device.
 int kernel_info(int index, KernelInfo* out);
 
@@ -74,6 +75,9 @@ int launch_plan(const Plan& plan, const void* x, const void* r, const void* w, v
                 int64_t n_tokens, int64_t hidden, float eps, cudaStream_t stream);
 int launch_fp8_plan(const Plan& plan, const void* x, const void* r, const void* w, void* q, float* scale, void* r_out,
                     int64_t n_tokens, int64_t hidden, float eps, cudaStream_t stream);
+int launch_allreduce_plan(const Plan& plan, const void* const* x_parts, int n_parts, const void* r, const void* w,
+                          void* const* y_outs, void* const* r_outs, int n_outs, int64_t row_begin, int64_t row_count,
+                          int64_t hidden, float eps, cudaStream_t stream);
 int launch_merge_plan(const Plan& plan, const void* v_a, const float* s_a, const void* v_b, const float* s_b, void* v_out,
                       float* s_out, int64_t n_tokens, cudaStream_t stream);
 int launch_silu_plan(const Plan& plan, const void* x, void* out, int64_t n_tokens, cudaStream_t stream);

@@ -30,6 +30,7 @@ import torch
 
 ROWS_PER_BLOCK = 64
 TENSOR_X, TENSOR_R, TENSOR_W, TENSOR_GATE_UP, TENSOR_LSE_A, TENSOR_LSE_B = 0, 1, 2, 3, 4, 5
+TENSOR_PART0 = 16  # partial inputs of the tensor-parallel norm: tensor ids 16, 17, ...
 
 TORCH_DTYPES = {"bf16": torch.bfloat16, "fp16": torch.float16, "fp32": torch.float32}
 DTYPE_CODES = {"bf16": 0, "fp16": 1, "fp32": 2}
@@ -56,6 +57,7 @@ class Workload:
     eps: float = 1e-6
     op: str = "add_rmsnorm"  # "silu_and_mul": hidden is d, the output width; "merge_attn_states": hidden = heads * head_dim
     head_dim: int = 0
+    n_parts: int = 0  # "add_rmsnorm_allreduce": partial inputs per element (the tensor-parallel group size)
 
     @property
     def elements(self) -> int:
@@ -72,6 +74,8 @@ class Workload:
             return (3 * b + 1) * self.elements + b * self.hidden + 4 * self.n_tokens
         if self.op == "merge_attn_states":  # v_a, v_b in, v_out out; s_a, s_b in, s_out out (binary32 per head)
             return 3 * b * self.elements + 3 * 4 * self.n_tokens * (self.hidden // self.head_dim)
+        if self.op == "add_rmsnorm_allreduce":  # n_parts partial x, r; write r' and y once; w once
+            return (self.n_parts + 3) * b * self.elements + b * self.hidden
         return 4 * b * self.elements + b * self.hidden
 
     @property
@@ -108,6 +112,11 @@ def workloads() -> dict[str, Workload]:
     add(Workload("silu_bf16_64x11008", "bf16", 64, 11008, seed=6, dist=gate, op="silu_and_mul"))
     # the fp8-output variant of the norm on the prefill shape
     add(Workload("c3q_prefill_bf16_16384x8192_fp8out", "bf16", 16384, 8192, seed=2, dist=_PREFILL_DIST, op="add_rmsnorm_fp8"))
+    # the tensor-parallel form of the norm on the prefill shape cut to a quarter of its rows, and a decode shape
+    for n in (2, 4, 8):
+        add(Workload(f"c3ar{n}_prefill_bf16_4096x8192", "bf16", 4096, 8192, seed=2, dist=_PREFILL_DIST,
+                     op="add_rmsnorm_allreduce", n_parts=n))
+    add(Workload("c2ar8_decode_bf16_64x8192", "bf16", 64, 8192, seed=1, op="add_rmsnorm_allreduce", n_parts=8))
     # merge_attn_states: the paper's (n, h, d) shapes in bf16, and a bandwidth case
     for n, h, d in ((512, 32, 256), (512, 40, 128), (768, 32, 256), (768, 40, 128), (512, 64, 128)):
         add(Workload(f"merge_bf16_{n}x{h}x{d}", "bf16", n, h * d, seed=7, op="merge_attn_states", head_dim=d))
@@ -177,6 +186,16 @@ def make_inputs(n_tokens: int, hidden: int, dtype: str, seed: int, dist: Dist = 
     return x, r, w
 
 
+def make_parts(row_begin: int, row_end: int, hidden: int, dtype: str, seed: int, n_parts: int, dist: Dist = Dist(),
+               threads: int = 8) -> torch.Tensor:
+    """Rows of the n_parts partial inputs of the tensor-parallel norm as one [n_parts, rows, hidden] tensor: part k
+    is N(0, sigma / sqrt(n_parts)) with the same outlier mix, so that the sum over parts has the spread of x."""
+    scaled = Dist(sigma=dist.sigma / float(np.sqrt(n_parts)), outlier_p=dist.outlier_p,
+                  outlier_sigma=dist.outlier_sigma / float(np.sqrt(n_parts)), w_mean=dist.w_mean, w_sigma=dist.w_sigma)
+    parts = [make_rows(TENSOR_PART0 + k, row_begin, row_end, hidden, dtype, seed, scaled, threads) for k in range(n_parts)]
+    return torch.stack(parts).contiguous()
+
+
 def make_gate_up(row_begin: int, row_end: int, d: int, dtype: str, seed: int, dist: Dist = Dist(sigma=2.5),
                  threads: int = 8) -> torch.Tensor:
     """Rows of the [T, 2*d] input of silu_and_mul: gate and value halves, N(0, sigma) each."""
@@ -205,6 +224,9 @@ def make_workload_inputs(wl: Workload, threads: int = 8):
         return make_merge_inputs(0, wl.n_tokens, wl.hidden // wl.head_dim, wl.head_dim, wl.dtype, wl.seed, threads)
     if wl.op == "silu_and_mul":
         return (make_gate_up(0, wl.n_tokens, wl.hidden, wl.dtype, wl.seed, wl.dist, threads),)
+    if wl.op == "add_rmsnorm_allreduce":
+        _, r, w = make_inputs(wl.n_tokens, wl.hidden, wl.dtype, wl.seed, wl.dist, threads)
+        return make_parts(0, wl.n_tokens, wl.hidden, wl.dtype, wl.seed, wl.n_parts, wl.dist, threads), r, w
     return make_inputs(wl.n_tokens, wl.hidden, wl.dtype, wl.seed, wl.dist, threads)
 
 

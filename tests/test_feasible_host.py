@@ -135,3 +135,28 @@ def test_fp8_output_norm_grid(L):
     assert B.tuner_check_params(s, B.make_params(vec_bytes=8), L) == B.RT_ERR_INFEASIBLE
     # rows that are not 16-byte multiples have no instance of this variant
     assert B.tuner_derive_feasible(B.shape_of(64, 6148, "fp16", op=B.RT_OP_ADD_RMSNORM_FP8), L) == []
+
+
+def test_allreduce_fused_norm_grid(L):
+    s = B.shape_of(4096, 8192, "bf16", op=B.RT_OP_ADD_RMSNORM_ALLREDUCE, n_parts=4)
+    f = B.tuner_derive_feasible(s, L)
+    assert f and {t.vec_bytes for t in f} == {16} and {t.stage for t in f} == {0} and {t.reduce for t in f} == {0}
+    assert all(B.tuner_check_params(s, t, L) == B.RT_OK for t in f)
+    c = B.tuner_derive_counts(s, L)
+    assert c["feasible"] == len(f) and sum(v for k, v in c.items() if k != "raw") == c["raw"] == len(B.tuner_raw_grid(s))
+    # eight parts leave no instance with four vectors per part in flight
+    s8 = B.shape_of(4096, 8192, "bf16", op=B.RT_OP_ADD_RMSNORM_ALLREDUCE, n_parts=8)
+    f8 = B.tuner_derive_feasible(s8, L)
+    assert f8 and 4 not in {t.unroll for t in f8} and len(f8) < len(f)
+    # the part count is 2, 4 or 8
+    for bad in (0, 1, 3, 16):
+        assert B.tuner_check_params(B.shape_of(64, 4096, "bf16", op=B.RT_OP_ADD_RMSNORM_ALLREDUCE, n_parts=bad),
+                                    B.make_params(), L) == B.RT_ERR_SHAPE
+    # the other stages, reductions and vector widths are not this variant's
+    assert B.tuner_check_params(s, B.make_params(stage=B.RT_STAGE_SMEM_TMA), L) == B.RT_ERR_INFEASIBLE
+    assert B.tuner_check_params(s, B.make_params(reduce=B.RT_REDUCE_SMEM), L) == B.RT_ERR_INFEASIBLE
+    assert B.tuner_check_params(s, B.make_params(vec_bytes=8), L) == B.RT_ERR_INFEASIBLE
+    # rows that are not 16-byte multiples have no instance
+    assert B.tuner_derive_feasible(B.shape_of(64, 6148, "fp16", op=B.RT_OP_ADD_RMSNORM_ALLREDUCE, n_parts=2), L) == []
+    # fp32 rows work too
+    assert B.tuner_derive_feasible(B.shape_of(64, 4096, "fp32", op=B.RT_OP_ADD_RMSNORM_ALLREDUCE, n_parts=2), L)
