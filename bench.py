@@ -30,13 +30,17 @@ if ROOT not in sys.path:
 
 METRIC = "fused_add_rmsnorm_hbm_gbs"
 METRICS = {"add_rmsnorm": METRIC, "silu_and_mul": "silu_and_mul_hbm_gbs", "merge_attn_states": "merge_attn_states_hbm_gbs",
-           "add_rmsnorm_fp8": "fused_add_rmsnorm_fp8out_hbm_gbs"}
+           "add_rmsnorm_fp8": "fused_add_rmsnorm_fp8out_hbm_gbs",
+           "add_rmsnorm_allreduce": "fused_allreduce_add_rmsnorm_hbm_gbs"}
 BYTES_LABEL = {"add_rmsnorm": "algorithmic: 2 reads + 2 writes per element + w once",
                "silu_and_mul": "algorithmic: 2 reads + 1 write per output element",
                "merge_attn_states": "algorithmic: 2 reads + 1 write per element + 3 binary32 per (token, head)",
-               "add_rmsnorm_fp8": "algorithmic: 2 reads + 1 write per element + 1 byte of q per element + w once + a scale per token"}
+               "add_rmsnorm_fp8": "algorithmic: 2 reads + 1 write per element + 1 byte of q per element + w once + a scale per token",
+               "add_rmsnorm_allreduce": "algorithmic: n_parts + 1 reads + 2 writes per element + w once (all parts and the one "
+                                        "destination in this GPU's memory)"}
 KERNEL_NAME = {"add_rmsnorm": "add_rmsnorm_kernel", "silu_and_mul": "silu_and_mul_kernel",
-               "merge_attn_states": "merge_attn_states_kernel", "add_rmsnorm_fp8": "add_rmsnorm_fp8_kernel"}
+               "merge_attn_states": "merge_attn_states_kernel", "add_rmsnorm_fp8": "add_rmsnorm_fp8_kernel",
+               "add_rmsnorm_allreduce": "add_rmsnorm_allreduce_kernel"}
 UNIT = "GB/s"
 DEFAULT_WORKLOAD = "c3_prefill_bf16_16384x8192"
 FALLBACK_HBM_GBS = 6650.0  # used only when MEASURED_PEAKS.json is absent
@@ -159,6 +163,11 @@ def run_reference(args) -> None:
         if is_silu:
             xs = synth.make_gate_up(0, n_rows, wl.hidden, wl.dtype, wl.seed, wl.dist)
             return lambda: oracle.silu_and_mul(xs, threads=cores)
+        if wl.op == "add_rmsnorm_allreduce":
+            w = synth.make_weight(wl.hidden, wl.dtype, wl.seed, wl.dist)
+            ps = synth.make_parts(0, n_rows, wl.hidden, wl.dtype, wl.seed, wl.n_parts, wl.dist)
+            rs = synth.make_rows(synth.TENSOR_R, 0, n_rows, wl.hidden, wl.dtype, wl.seed, wl.dist).contiguous()
+            return lambda: oracle.allreduce_add_rmsnorm(ps, rs, w, wl.eps, threads=cores)
         w = synth.make_weight(wl.hidden, wl.dtype, wl.seed, wl.dist)
         xs = synth.make_rows(synth.TENSOR_X, 0, n_rows, wl.hidden, wl.dtype, wl.seed, wl.dist).contiguous()
         rs = synth.make_rows(synth.TENSOR_R, 0, n_rows, wl.hidden, wl.dtype, wl.seed, wl.dist).contiguous()
@@ -185,6 +194,8 @@ def run_reference(args) -> None:
     elif is_merge:
         cores = 1  # this oracle is single-threaded
         step_bytes = 3 * b * rows * wl.hidden + 12 * rows * (wl.hidden // wl.head_dim)
+    elif wl.op == "add_rmsnorm_allreduce":
+        step_bytes = (wl.n_parts + 3) * b * rows * wl.hidden + b * wl.hidden
     else:
         step_bytes = 3 * b * rows * wl.hidden if is_silu else 4 * b * rows * wl.hidden + b * wl.hidden
     value = step_bytes * args.steps / elapsed / 1e9
@@ -223,8 +234,10 @@ def run_ours(args) -> None:
     is_silu = wl.op == "silu_and_mul"
     is_merge = wl.op == "merge_attn_states"
     is_fp8 = wl.op == "add_rmsnorm_fp8"
+    is_allreduce = wl.op == "add_rmsnorm_allreduce"  # all parts and the one destination on this GPU (one-shot form)
     op_code = {"add_rmsnorm": B.RT_OP_ADD_RMSNORM, "silu_and_mul": B.RT_OP_SILU_AND_MUL,
-               "merge_attn_states": B.RT_OP_MERGE_ATTN_STATES, "add_rmsnorm_fp8": B.RT_OP_ADD_RMSNORM_FP8}[wl.op]
+               "merge_attn_states": B.RT_OP_MERGE_ATTN_STATES, "add_rmsnorm_fp8": B.RT_OP_ADD_RMSNORM_FP8,
+               "add_rmsnorm_allreduce": B.RT_OP_ADD_RMSNORM_ALLREDUCE}[wl.op]
     scale_ref = None
     heads = H // wl.head_dim if is_merge else 0
     sa = sb = None
@@ -236,6 +249,10 @@ def run_ours(args) -> None:
     elif is_silu:
         x = synth.make_gate_up(shard.row_begin, shard.row_end, H, wl.dtype, wl.seed, wl.dist)
         r = w = None
+    elif is_allreduce:
+        x = synth.make_parts(shard.row_begin, shard.row_end, H, wl.dtype, wl.seed, wl.n_parts, wl.dist)  # [N, T, H]
+        r = synth.make_rows(synth.TENSOR_R, shard.row_begin, shard.row_end, H, wl.dtype, wl.seed, wl.dist).contiguous()
+        w = synth.make_weight(H, wl.dtype, wl.seed, wl.dist)
     else:
         x = synth.make_rows(synth.TENSOR_X, shard.row_begin, shard.row_end, H, wl.dtype, wl.seed, wl.dist).contiguous()
         r = synth.make_rows(synth.TENSOR_R, shard.row_begin, shard.row_end, H, wl.dtype, wl.seed, wl.dist).contiguous()
@@ -256,6 +273,8 @@ def run_ours(args) -> None:
         y_ref = v_ref.view(T, H)
     elif is_silu:
         y_ref, r_ref = oracle.silu_and_mul(x, threads=cores), None
+    elif is_allreduce:
+        y_ref, r_ref = oracle.allreduce_add_rmsnorm(x, r, w, wl.eps, threads=cores)
     else:
         y_ref, r_ref = oracle.add_rmsnorm(x, r, w, wl.eps, threads=cores)
     oracle_s = time.perf_counter() - t0
@@ -270,14 +289,14 @@ def run_ours(args) -> None:
     # every timed launch reads from DRAM; the large workloads exceed L2 on their own.
     resident = wl.algorithmic_bytes <= 2 * limits.l2_bytes
     sets = 1 if not resident else int(min(4096, -(-3 * limits.l2_bytes // wl.algorithmic_bytes)))
-    ring = lambda t: t.to(device).unsqueeze(0).repeat(sets, 1, 1).contiguous()
+    ring = lambda t: t.to(device).unsqueeze(0).repeat(sets, *([1] * t.dim())).contiguous()
     xd = ring(x)
     rd = ring(r) if r is not None else None
     wd = w.to(device) if w is not None else None
     yd = torch.empty((sets, T, H), dtype=torch.uint8 if is_fp8 else xd.dtype, device=device)
     scaled = torch.empty((sets, T), dtype=torch.float32, device=device) if is_fp8 else None
     scale_ref_d = scale_ref.to(device) if is_fp8 else None
-    od = torch.empty_like(xd) if not (is_silu or is_merge) else None
+    od = torch.empty((sets, T, H), dtype=xd.dtype, device=device) if not (is_silu or is_merge) else None
     sad = sbd = None
     if is_merge:
         sad, sbd = ring(sa), ring(sb)
@@ -288,7 +307,7 @@ def run_ours(args) -> None:
     live = [t for t in (xd, rd, wd, od if is_fp8 else yd, od) if t is not None]
     align = B._ptr_align(*live)
     shape = B.shape_of(T, H, wl.dtype, align if set_bytes % 256 == 0 else min(align, set_bytes & -set_bytes), op=op_code,
-                       head_dim=wl.head_dim)
+                       head_dim=wl.head_dim, n_parts=wl.n_parts)
     # warm: the paper's protocol (the same buffers every launch); cold: rotating over the ring
     w_or_sa = sad if is_merge else wd
     ws = B.make_workspace(xd, rd, w_or_sa, yd, od, y_ref_d, r_ref_d, wl.eps, n_ref_tokens=T, stream=stream, aux=sbd,
@@ -398,6 +417,18 @@ def run_ours(args) -> None:
             st = launch(theta_ref, pa, psa, pb, psb, po, pso, T, heads, head_dim, dtype_code, stream_ptr)
             if st != 0:
                 raise B.TunerError(st, "merge_attn_states_template_launch")
+    elif is_allreduce:
+        launch = B.lib.rmsnorm_allreduce_template_launch
+        vp, n_parts = B.c_void_p, wl.n_parts
+        ptrs = [((vp * n_parts)(*[xd[k, j].data_ptr() for j in range(n_parts)]), rd[k].data_ptr(),
+                 (vp * 1)(yd[k].data_ptr()), (vp * 1)(od[k].data_ptr())) for k in range(sets)]
+        w_ptr = wd.data_ptr()
+
+        def step(k):
+            px, pr, py, po = ptrs[k % sets]
+            st = launch(theta_ref, px, n_parts, pr, w_ptr, py, po, 1, 0, T, H, eps, dtype_code, stream_ptr)
+            if st != 0:
+                raise B.TunerError(st, "rmsnorm_allreduce_template_launch")
     elif is_silu:
         launch = B.lib.silu_and_mul_template_launch
         ptrs = [(xd[k].data_ptr(), yd[k].data_ptr()) for k in range(sets)]
@@ -483,6 +514,17 @@ def run_ours(args) -> None:
                 sad[0].copy_(sap, non_blocking=True); sbd[0].copy_(sbp, non_blocking=True)
                 step(0)
                 yp.copy_(yd[0], non_blocking=True); sop.copy_(od[0], non_blocking=True)
+            stream.synchronize()
+    elif is_allreduce:
+        xp, rp, wp = x.pin_memory(), r.pin_memory(), w.pin_memory()
+        yp, op = torch.empty_like(rp).pin_memory(), torch.empty_like(rp).pin_memory()
+        h2d_bytes, d2h_bytes = (wl.n_parts + 1) * T * H * b + H * b, 2 * T * H * b
+
+        def e2e_step():
+            with torch.cuda.stream(stream):
+                xd[0].copy_(xp, non_blocking=True); rd[0].copy_(rp, non_blocking=True); wd.copy_(wp, non_blocking=True)
+                step(0)
+                yp.copy_(yd[0], non_blocking=True); op.copy_(od[0], non_blocking=True)
             stream.synchronize()
     elif is_silu:
         xp = x.pin_memory()

@@ -535,6 +535,16 @@ class SpecTable:
         rmsnorm_fp8_template_launch(theta, x, r, w, q, scale, r_out, eps, stream)
         return theta
 
+    def launch_rmsnorm_allreduce(self, x_parts, r, w, y_outs, r_outs, row_begin: int, row_count: int, eps: float,
+                                 stream=None) -> rt_params:
+        """The tensor-parallel form of the norm with the table's theta for (row_count, hidden, parts)."""
+        n_rows, hidden = r.shape
+        shape = shape_of(max(1, row_count), hidden, _dtype_code(r), _ptr_align(*x_parts, r, w, *y_outs, *r_outs),
+                         op=RT_OP_ADD_RMSNORM_ALLREDUCE, n_parts=len(x_parts))
+        theta, _ = self.lookup(shape)
+        rmsnorm_allreduce_template_launch(theta, x_parts, r, w, y_outs, r_outs, row_begin, row_count, eps, stream)
+        return theta
+
     def to_json(self) -> dict:
         names = {v: k for k, v in DTYPE_CODES.items()}
         return {"device": self.device_name, "general": self.general.as_dict() if self.general else None,

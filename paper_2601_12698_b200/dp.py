@@ -103,3 +103,88 @@ def whole_job_rate(units_per_rank_per_step: float, steps: int, world: int, max_m
 def shutdown() -> None:
     if dist.is_initialized():
         dist.destroy_process_group()
+
+
+# ---- the tensor-parallel form of the norm: all-reduce folded into the kernel ---------------------------------
+
+@dataclass
+class FusedAllreduceNorm:
+    """One rank's view of a tensor-parallel group for the all-reduce-fused norm.
+
+    ``x_parts[k]`` is rank k's partial x, ``y_outs[k]`` / ``r_outs[k]`` rank k's output tensors, all [n_rows, hidden]
+    and all addressable from this rank's GPU (index ``rank`` is this rank's own memory, the others are peer
+    mappings).  A call runs this rank's block of rows: it reads every rank's partial for those rows, and writes
+    the rows of y and r_out into every rank's outputs, so that after all ranks' calls each rank holds all rows.
+
+    The kernel never waits for another rank.  The group meets in stream order instead: a one-element all-reduce
+    on the launch stream before the kernel (every rank's partial is complete once it returns) and one after it
+    (every rank's rows have been written once it returns).  ``launch`` is
+    ``binding.rmsnorm_allreduce_template_launch``; it is a parameter so that the host logic can run without a GPU.
+    """
+    rank: int
+    world: int
+    n_rows: int
+    x_parts: list
+    y_outs: list
+    r_outs: list
+    launch: object
+    sync: object = None  # callable run before and after the launch; default: a one-element all-reduce
+
+    def __post_init__(self):
+        if self.world not in (2, 4, 8):
+            raise ValueError("the all-reduce-fused norm takes groups of 2, 4 or 8 ranks")
+        if not (len(self.x_parts) == len(self.y_outs) == len(self.r_outs) == self.world):
+            raise ValueError("one partial input and one pair of outputs per rank, in rank order")
+        if not (0 <= self.rank < self.world):
+            raise ValueError("rank outside the group")
+
+    @property
+    def shard(self) -> Shard:
+        return strong_shard(self.n_rows, self.rank, self.world)
+
+    def _meet(self, device) -> None:
+        if self.sync is not None:
+            self.sync()
+        elif dist.is_initialized():
+            flag = torch.zeros(1, dtype=torch.int32, device=device)
+            dist.all_reduce(flag)  # stream-ordered on NCCL: returns on the stream once every rank has reached it
+
+    def __call__(self, theta, r, w, eps: float, stream=None) -> Shard:
+        """r: this rank's residual [n_rows, hidden] (the same values on every rank); w: [hidden]."""
+        sh = self.shard
+        self._meet(r.device)
+        self.launch(theta, self.x_parts, r, w, self.y_outs, self.r_outs, sh.row_begin, sh.rows, eps, stream)
+        self._meet(r.device)
+        return sh
+
+
+def gather_in_rank_order(obj) -> list:
+    """Every rank's ``obj`` as a list indexed by rank (the list [obj] without a process group)."""
+    if not dist.is_initialized():
+        return [obj]
+    out = [None] * dist.get_world_size()
+    dist.all_gather_object(out, obj)
+    return out
+
+
+def symmetric_group_buffers(n_rows: int, hidden: int, dtype: torch.dtype, device: torch.device, names=("x", "y", "r_out")):
+    """Allocate one [n_rows, hidden] tensor per name in symmetric memory and return, per name, the list of all
+    ranks' tensors in rank order as seen from this GPU (own memory at this rank's index, peer mappings elsewhere).
+    Needs an initialised NCCL process group whose ranks share one node."""
+    import torch.distributed._symmetric_memory as symm_mem
+    world, group = dist.get_world_size(), dist.group.WORLD
+    out = {}
+    for name in names:
+        local = symm_mem.empty((n_rows, hidden), dtype=dtype, device=device)
+        handle = symm_mem.rendezvous(local, group)
+        out[name] = [local if k == dist.get_rank() else handle.get_buffer(k, (n_rows, hidden), dtype) for k in range(world)]
+    return out
+
+
+def fused_allreduce_norm(n_rows: int, hidden: int, dtype: torch.dtype, device: torch.device) -> FusedAllreduceNorm:
+    """The group's buffers in symmetric memory, wired to the CUDA entry point.  Each rank writes its partial x into
+    ``x_parts[rank]`` and reads the results from ``y_outs[rank]`` / ``r_outs[rank]``."""
+    from . import binding
+    bufs = symmetric_group_buffers(n_rows, hidden, dtype, device)
+    return FusedAllreduceNorm(dist.get_rank(), dist.get_world_size(), n_rows, bufs["x"], bufs["y"], bufs["r_out"],
+                              binding.rmsnorm_allreduce_template_launch)

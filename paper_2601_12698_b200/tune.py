@@ -3,6 +3,7 @@
     python -m paper_2601_12698_b200.tune --shapes bf16:128x4096,bf16:16384x8192,fp32:2048x8192 \
         --budget 64 --out rmsnorm_table.json
     python -m paper_2601_12698_b200.tune --shapes silu/bf16:4096x14336,merge/bf16:512x32x128,fp8/bf16:4096x8192
+    python -m paper_2601_12698_b200.tune --shapes allreduce/bf16:4096x8192x4
 
 For every (kernel, shape): seeded synthetic inputs, a guided search (Algorithm 1: DeriveFeasibleSpace, Search),
 then, per kernel, SelectGeneral over the shapes' finalists timed on every shape, and BuildSpecialized as a JSON table that
@@ -26,12 +27,13 @@ from . import synth
 
 
 OPS = {"norm": B.RT_OP_ADD_RMSNORM, "silu": B.RT_OP_SILU_AND_MUL, "merge": B.RT_OP_MERGE_ATTN_STATES,
-       "fp8": B.RT_OP_ADD_RMSNORM_FP8}
+       "fp8": B.RT_OP_ADD_RMSNORM_FP8, "allreduce": B.RT_OP_ADD_RMSNORM_ALLREDUCE}
 
 
 def parse_shapes(text: str):
     """[kernel/]dtype:dims, comma separated.  kernel: norm (default, TOKENSxHIDDEN), silu (TOKENSxD),
-    merge (TOKENSxHEADSxHEAD_DIM), fp8 (the norm with e4m3 output, TOKENSxHIDDEN)."""
+    merge (TOKENSxHEADSxHEAD_DIM), fp8 (the norm with e4m3 output, TOKENSxHIDDEN), allreduce (the norm with its x
+    given as PARTS partial inputs, TOKENSxHIDDENxPARTS)."""
     out = []
     for item in text.split(","):
         item = item.strip()
@@ -77,6 +79,18 @@ class ShapeProblem:
             self.ws = B.make_workspace(va, vb, sa, vo, so, vo_ref, so_ref, eps, stream=stream, aux=sb)
             moved = 3 * va.element_size() * va.numel()
             self.keep = (va, sa, vb, sb, vo, vo_ref, so, so_ref)
+        elif kernel == "allreduce":
+            hidden, n_parts = dims[1], dims[2]
+            _, r, w = (t.cuda() for t in synth.make_inputs(n_tokens, hidden, dtype, seed))
+            parts = synth.make_parts(0, n_tokens, hidden, dtype, seed, n_parts).cuda()  # [parts, tokens, hidden]
+            y, y_ref, r_out, r_ref = (torch.empty_like(r) for _ in range(4))
+            self.shape = B.shape_of(n_tokens, hidden, dtype, B._ptr_align(parts, r, w, y, r_out), op=op, n_parts=n_parts)
+            self.ref_theta = reference_theta(self.shape)
+            B.rmsnorm_allreduce_template_launch(self.ref_theta, [parts[k] for k in range(n_parts)], r, w, [y_ref], [r_ref],
+                                                0, n_tokens, eps, stream=stream)
+            self.ws = B.make_workspace(parts, r, w, y, r_out, y_ref, r_ref, eps, stream=stream)
+            moved = (n_parts + 3) * r.element_size() * r.numel()
+            self.keep = (parts, r, w, y, y_ref, r_out, r_ref)
         else:
             hidden = dims[1]
             x, r, w = (t.cuda() for t in synth.make_inputs(n_tokens, hidden, dtype, seed))

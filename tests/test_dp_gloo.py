@@ -77,3 +77,84 @@ def test_shard_arithmetic():
     # single process: the helpers are the identity
     cpu = torch.device("cpu")
     assert dp.max_over_ranks(3.5, cpu) == 3.5 and dp.broadcast_ints([1, 2], cpu) == [1, 2]
+
+
+# ---- the tensor-parallel form of the norm: host logic of the group on CPU --------------------------------------
+
+def _tp_worker(rank: int, world: int, port: int, shared: dict, out_dir: str):
+    sys.path.insert(0, ROOT)
+    os.environ.update(RANK=str(rank), WORLD_SIZE=str(world), LOCAL_RANK=str(rank), MASTER_ADDR="127.0.0.1",
+                      MASTER_PORT=str(port))
+    import torch.distributed as dist
+    from paper_2601_12698_b200 import dp
+    import oracle
+    device = torch.device("cpu")
+    assert dp.init(backend="gloo", device=device) is True
+    n_rows, hidden = shared["r"].shape
+    calls = []
+
+    # Stand-in for the CUDA entry point with the same signature: the oracle on the requested rows, written to every
+    # destination.  Shared-memory tensors stand in for peer-mapped GPU memory.
+    def launch(theta, x_parts, r, w, y_outs, r_outs, row_begin, row_count, eps, stream):
+        calls.append((tuple(theta), row_begin, row_count, len(x_parts), len(y_outs)))
+        rows = slice(row_begin, row_begin + row_count)
+        stacked = torch.stack([p[rows] for p in x_parts]).contiguous()
+        y, ro = oracle.allreduce_add_rmsnorm(stacked, r[rows].contiguous(), w, eps)
+        for k in range(len(y_outs)):
+            y_outs[k][rows] = y
+            r_outs[k][rows] = ro
+
+    # every rank fills its own partial, then the group runs the fused operator
+    g = torch.Generator().manual_seed(100 + rank)
+    shared["x"][rank].copy_(torch.randn(n_rows, hidden, generator=g).to(torch.bfloat16))
+    ranks_seen = dp.gather_in_rank_order(("rank", rank))
+    assert ranks_seen == [("rank", k) for k in range(world)]
+    op = dp.FusedAllreduceNorm(rank, world, n_rows, list(shared["x"]), list(shared["y"]), list(shared["r_out"]), launch,
+                               sync=dist.barrier)
+    sh = op((256, 1, 16, 1, 0, 0, 1), shared["r"], shared["w"], 1e-6)
+    assert (sh.row_begin, sh.row_end) == ((0, 19), (19, 37))[rank]          # 37 rows over two ranks: 19 + 18
+    assert calls == [((256, 1, 16, 1, 0, 0, 1), sh.row_begin, sh.rows, world, world)]
+    # after the second meeting this rank's outputs hold every row
+    torch.save({"y": shared["y"][rank].clone(), "ro": shared["r_out"][rank].clone()}, os.path.join(out_dir, f"tp{rank}.pt"))
+    dp.barrier(device)
+    dp.shutdown()
+
+
+def test_two_gloo_ranks_tensor_parallel_norm(tmp_path):
+    sys.path.insert(0, ROOT)
+    import oracle
+    world, n_rows, hidden = 2, 37, 64
+    g = torch.Generator().manual_seed(9)
+    shared = {
+        "x": [torch.zeros(n_rows, hidden, dtype=torch.bfloat16).share_memory_() for _ in range(world)],
+        "y": [torch.zeros(n_rows, hidden, dtype=torch.bfloat16).share_memory_() for _ in range(world)],
+        "r_out": [torch.zeros(n_rows, hidden, dtype=torch.bfloat16).share_memory_() for _ in range(world)],
+        "r": torch.randn(n_rows, hidden, generator=g).to(torch.bfloat16).share_memory_(),
+        "w": (1 + 0.1 * torch.randn(hidden, generator=g)).to(torch.bfloat16).share_memory_(),
+    }
+    mp.spawn(_tp_worker, args=(world, _free_port(), shared, str(tmp_path)), nprocs=world, join=True)
+    got = [torch.load(os.path.join(tmp_path, f"tp{k}.pt")) for k in range(world)]
+    y_ref, r_ref = oracle.allreduce_add_rmsnorm(torch.stack(shared["x"]).contiguous(), shared["r"], shared["w"], 1e-6)
+    for k in range(world):
+        assert torch.equal(got[k]["y"].view(torch.int16), y_ref.view(torch.int16))
+        assert torch.equal(got[k]["ro"].view(torch.int16), r_ref.view(torch.int16))
+
+
+def test_fused_allreduce_norm_argument_checks():
+    sys.path.insert(0, ROOT)
+    from paper_2601_12698_b200 import dp
+    t = [torch.zeros(4, 8)] * 2
+    with pytest.raises(ValueError):
+        dp.FusedAllreduceNorm(0, 3, 4, t + t[:1], t + t[:1], t + t[:1], None)     # a group of three
+    with pytest.raises(ValueError):
+        dp.FusedAllreduceNorm(0, 2, 4, t, t[:1], t, None)                           # a destination missing
+    with pytest.raises(ValueError):
+        dp.FusedAllreduceNorm(2, 2, 4, t, t, t, None)                               # rank outside the group
+    assert dp.gather_in_rank_order("alone") == ["alone"]
+    # the blocks of rows tile the job for every group size
+    for world in (2, 4, 8):
+        for n_rows in (1, 7, 64, 1001):
+            blocks = [dp.FusedAllreduceNorm(k, world, n_rows, [None] * world, [None] * world, [None] * world, None).shard
+                      for k in range(world)]
+            assert blocks[0].row_begin == 0 and blocks[-1].row_end == n_rows
+            assert all(a.row_end == b.row_begin for a, b in zip(blocks, blocks[1:]))
