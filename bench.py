@@ -426,7 +426,7 @@ def run_ours(args) -> None:
 
         def step(k):
             px, pr, py, po = ptrs[k % sets]
-            st = launch(theta_ref, px, n_parts, pr, w_ptr, py, po, 1, 0, T, H, eps, dtype_code, stream_ptr)
+            st = launch(theta_ref, px, n_parts, pr, w_ptr, py, 1, po, 1, 0, T, H, eps, dtype_code, stream_ptr)
             if st != 0:
                 raise B.TunerError(st, "rmsnorm_allreduce_template_launch")
     elif is_silu:

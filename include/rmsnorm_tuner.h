@@ -278,27 +278,29 @@ int rmsnorm_fp8_template_launch(const rt_params* p, const void* x, const void* r
  * One launch computes rows [row_begin, row_begin + row_count) of the tensors:
  *     a = fp32(x^(0));  a = a + fp32(x^(k)) for k = 1 .. n_parts-1, in this order, each a binary32 addition;
  *     s = a + fp32(r);  r_out = round_dtype(s);  y = round_dtype(s * rsqrt(mean(s^2) + eps) * w)
- * and writes those rows of y and r_out into EVERY destination given.  With rank k of an n-rank group calling it
- * on its own block of rows, with all ranks' partials as x_parts and all ranks' output tensors as destinations,
- * every rank ends with the complete y and r_out (reduce-scatter + operator + all-gather in one kernel, the
- * transfers being the kernel's own loads and stores over peer-mapped memory).  With one destination and all
- * rows it is the one-shot form (every rank reduces everything for itself).
+ * and writes those rows of y into EVERY y destination and those rows of r_out into EVERY r_out destination.
+ * With rank k of an n-rank group calling it on its own block of rows, with all ranks' partials as x_parts and
+ * all ranks' y tensors as y destinations, every rank ends with the complete y (reduce-scatter + operator +
+ * all-gather in one kernel, the transfers being the kernel's own loads and stores over peer-mapped memory).  The
+ * residual usually has one destination, the rank's own tensor: the rank's next norm needs the residual of its
+ * own rows only, so each link direction carries 2 (n-1)/n tensor sizes, as much as an all-reduce of x alone.
+ * With one y destination and all rows it is the one-shot form (every rank reduces everything for itself).
  *   x_parts   HOST array of n_parts (2, 4 or 8) DEVICE pointers, part k = rank k's partial x, each a full
  *             [n_rows_total, hidden] tensor addressable from the current device (its own memory or a
  *             peer-mapped allocation); read only.
  *   r, w      device (current GPU), r a full [n_rows_total, hidden] tensor, w [hidden].
- *   y_outs, r_outs  HOST arrays of n_outs (1..8) DEVICE pointers to full [n_rows_total, hidden] tensors; only the
- *             launch's rows are written.  A destination may be the tensor r itself (in-place residual), never
- *             a part of x.
+ *   y_outs    HOST array of n_y_outs (1..RT_MAX_PARTS) DEVICE pointers to full [n_rows_total, hidden] tensors;
+ *   r_outs    HOST array of n_r_outs (1..RT_MAX_PARTS) such pointers.  Only the launch's rows are written.  An
+ *             r_out destination may be the tensor r itself (in-place residual); no destination may be a part of x.
  *   All tensor pointers must be 16-byte aligned and the row length a multiple of 16 bytes (RT_ERR_ALIGN).
  * The kernel contains no wait: the caller orders the launch after every rank's partial is complete and lets
  * no rank read the outputs before every rank's launch has finished (a barrier of the group on both sides).
  * Asynchronous on `stream`, allocates nothing; infeasible theta is refused without launching.
  */
 int rmsnorm_allreduce_template_launch(const rt_params* p, const void* const* x_parts, int32_t n_parts, const void* r,
-                                      const void* w, void* const* y_outs, void* const* r_outs, int32_t n_outs,
-                                      int64_t row_begin, int64_t row_count, int64_t hidden, float eps, int dtype,
-                                      void* stream);
+                                      const void* w, void* const* y_outs, int32_t n_y_outs, void* const* r_outs,
+                                      int32_t n_r_outs, int64_t row_begin, int64_t row_count, int64_t hidden,
+                                      float eps, int dtype, void* stream);
 
 /*
  * merge_attn_states as an instance of its own template (third kernel of the paper's "Kernels" list, shapes

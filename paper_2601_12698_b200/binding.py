@@ -112,8 +112,8 @@ _SIGNATURES = {
     "rmsnorm_fp8_template_launch": (c_int, [POINTER(rt_params), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                             c_int64, c_int64, c_float, c_int, c_void_p]),
     "rmsnorm_allreduce_template_launch": (c_int, [POINTER(rt_params), POINTER(c_void_p), c_int32, c_void_p, c_void_p,
-                                                  POINTER(c_void_p), POINTER(c_void_p), c_int32, c_int64, c_int64,
-                                                  c_int64, c_float, c_int, c_void_p]),
+                                                  POINTER(c_void_p), c_int32, POINTER(c_void_p), c_int32, c_int64,
+                                                  c_int64, c_int64, c_float, c_int, c_void_p]),
     "rt_kernel_instance_parts": (c_int32, [c_int32]),
     "merge_attn_states_template_launch": (c_int, [POINTER(rt_params), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                                   c_void_p, c_int64, c_int64, c_int64, c_int, c_void_p]),
@@ -267,22 +267,23 @@ def rmsnorm_fp8_template_launch(params: rt_params, x, r, w, q, scale, r_out, eps
 def rmsnorm_allreduce_template_launch(params: rt_params, x_parts, r, w, y_outs, r_outs, row_begin: int, row_count: int,
                                       eps: float, stream=None) -> None:
     """The tensor-parallel form of add_rmsnorm on rows [row_begin, row_begin + row_count): x_parts is a list of 2, 4
-    or 8 device tensors [T, H] (one partial x per rank, each addressable from the current device), y_outs / r_outs
-    lists of 1..8 destination tensors [T, H] that all receive those rows.  Asynchronous."""
+    or 8 device tensors [T, H] (one partial x per rank, each addressable from the current device); y_outs and r_outs
+    are lists of 1..8 destination tensors [T, H]: every y destination receives those rows of y, every r_out
+    destination those rows of the new residual.  Asynchronous."""
     n_rows, hidden = r.shape
     tensors = list(x_parts) + [r] + list(y_outs) + list(r_outs)
     ok = (all(t.is_cuda and t.is_contiguous() and t.shape == (n_rows, hidden) and t.dtype == r.dtype for t in tensors)
           and w.is_cuda and w.is_contiguous() and w.shape == (hidden,) and w.dtype == r.dtype
-          and len(y_outs) == len(r_outs) and 0 <= row_begin and row_begin + row_count <= n_rows)
+          and 0 <= row_begin and row_begin + row_count <= n_rows)
     if not ok:
         raise ValueError("rmsnorm_allreduce_template_launch: tensors of the wrong device, layout, shape or dtype, "
                          "or rows out of range")
     xp = (c_void_p * len(x_parts))(*[t.data_ptr() for t in x_parts])
     yo = (c_void_p * len(y_outs))(*[t.data_ptr() for t in y_outs])
     ro = (c_void_p * len(r_outs))(*[t.data_ptr() for t in r_outs])
-    _check(lib.rmsnorm_allreduce_template_launch(byref(params), xp, len(x_parts), r.data_ptr(), w.data_ptr(), yo, ro,
-                                                 len(y_outs), row_begin, row_count, hidden, eps, _dtype_code(r),
-                                                 _stream_ptr(stream)), "rmsnorm_allreduce_template_launch")
+    _check(lib.rmsnorm_allreduce_template_launch(byref(params), xp, len(x_parts), r.data_ptr(), w.data_ptr(), yo,
+                                                 len(y_outs), ro, len(r_outs), row_begin, row_count, hidden, eps,
+                                                 _dtype_code(r), _stream_ptr(stream)), "rmsnorm_allreduce_template_launch")
 
 
 def merge_attn_states_template_launch(params: rt_params, v_a, s_a, v_b, s_b, v_out, s_out, stream=None) -> None:

@@ -2,10 +2,11 @@
 // x of the operator is the sum over the ranks of a group of each rank's partial result.  One launch handles a
 // block of rows: it reads the rows of every rank's partial (plain loads; a peer's memory over NVLink is read the
 // same way as this GPU's own), sums them in rank order in binary32, adds the residual, normalises, and writes
-// y and r_out for those rows into every destination it is given (this GPU's and, for the gather half of the
-// all-reduce, each peer's).  With each rank launching it on its own block of rows, every rank ends with the full
-// y and r_out: reduce-scatter, the operator and all-gather in one kernel, with no wait inside the kernel - the
-// ranks meet on the host (or in stream order) before and after the launch.
+// y for those rows into every y destination it is given (this GPU's and, for the gather half of the all-reduce,
+// each peer's) and r_out into every r_out destination (usually this GPU's only: the next norm of the same rank
+// needs the residual of its own rows only).  With each rank launching it on its own block of rows, every rank
+// ends with the full y: reduce-scatter, the operator and all-gather in one kernel, with no wait inside the
+// kernel - the ranks meet on the host (or in stream order) before and after the launch.
 //
 // Per row:  a = fp32(x^(0));  a += fp32(x^(k)) for k = 1..NP-1 in this order;  s = a + fp32(r);
 //           r_out = rn(s);  y = rn(s * rsqrt(mean(s^2) + eps) * w).
@@ -23,9 +24,9 @@ struct AllreduceArgs {
     const void* x_parts[kMaxParts];  // part k: [*, hidden] rows, indexed by absolute row
     const void* r;
     const void* w;
-    void* y_outs[kMaxParts];         // destinations 0..n_outs-1 receive the rows of this launch
-    void* r_outs[kMaxParts];
-    int n_outs;
+    void* y_outs[kMaxParts];         // destinations 0..n_y_outs-1 receive the rows of y of this launch
+    void* r_outs[kMaxParts];         // destinations 0..n_r_outs-1 the rows of r_out
+    int n_y_outs, n_r_outs;
     long long row_begin, row_end;    // absolute rows handled by this launch
     int hidden;
     int nvec;                        // 16-byte vectors in one row
@@ -49,10 +50,10 @@ __global__ void add_rmsnorm_allreduce_kernel(const AllreduceArgs a)
     const unsigned char* wrow = reinterpret_cast<const unsigned char*>(a.w);
 
     // the same vector to every destination; the destination count is uniform over the grid
-    auto store_all = [&](void* const (&dst)[kMaxParts], size_t off, const Vec<VB>& v) {
+    auto store_all = [&](void* const (&dst)[kMaxParts], int n_dst, size_t off, const Vec<VB>& v) {
 #pragma unroll
         for (int d = 0; d < kMaxParts; ++d)
-            if (d < a.n_outs) st_stream<VB, true>(reinterpret_cast<unsigned char*>(dst[d]) + off, v);
+            if (d < n_dst) st_stream<VB, true>(reinterpret_cast<unsigned char*>(dst[d]) + off, v);
     };
 
     float ss = 0.f;
@@ -92,7 +93,7 @@ __global__ void add_rmsnorm_allreduce_kernel(const AllreduceArgs a)
                     s[i0 + u][e] = __fadd_rn(acc[e], pf[e]);
                     ss = fmaf(s[i0 + u][e], s[i0 + u][e], ss);
                 }
-                store_all(a.r_outs, row_off + (size_t)v * VB, C::pack(s[i0 + u]));
+                store_all(a.r_outs, a.n_r_outs, row_off + (size_t)v * VB, C::pack(s[i0 + u]));
             }
         }
     }
@@ -106,7 +107,7 @@ __global__ void add_rmsnorm_allreduce_kernel(const AllreduceArgs a)
             C::unpack(ld_weight<VB>(wrow + (size_t)v * VB), wf);
 #pragma unroll
             for (int e = 0; e < EPV; ++e) yf[e] = s[i][e] * rho * wf[e];
-            store_all(a.y_outs, row_off + (size_t)v * VB, C::pack(yf));
+            store_all(a.y_outs, a.n_y_outs, row_off + (size_t)v * VB, C::pack(yf));
         }
     }
 }

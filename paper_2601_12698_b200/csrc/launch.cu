@@ -561,8 +561,8 @@ int launch_fp8_plan(const Plan& plan, const void* x, const void* r, const void* 
 }
 
 int launch_allreduce_plan(const Plan& plan, const void* const* x_parts, int n_parts, const void* r, const void* w,
-                          void* const* y_outs, void* const* r_outs, int n_outs, int64_t row_begin, int64_t row_count,
-                          int64_t hidden, float eps, cudaStream_t stream)
+                          void* const* y_outs, int n_y_outs, void* const* r_outs, int n_r_outs, int64_t row_begin,
+                          int64_t row_count, int64_t hidden, float eps, cudaStream_t stream)
 {
     if (row_count == 0) return RT_OK;
     const KernelEntry& k = registry()[plan.kernel_index];
@@ -570,19 +570,18 @@ int launch_allreduce_plan(const Plan& plan, const void* const* x_parts, int n_pa
         set_error("plan belongs to another kernel");
         return RT_ERR_INFEASIBLE;
     }
-    if (n_outs < 1 || n_outs > kMaxParts) {
-        set_error("n_outs=%d outside 1..%d", n_outs, kMaxParts);
+    if (n_y_outs < 1 || n_y_outs > kMaxParts || n_r_outs < 1 || n_r_outs > kMaxParts) {
+        set_error("n_y_outs=%d or n_r_outs=%d outside 1..%d", n_y_outs, n_r_outs, kMaxParts);
         return RT_ERR_SHAPE;
     }
     AllreduceArgs a;
     memset(&a, 0, sizeof(a));
     for (int i = 0; i < n_parts; ++i) a.x_parts[i] = x_parts[i];
-    for (int i = 0; i < n_outs; ++i) {
-        a.y_outs[i] = y_outs[i];
-        a.r_outs[i] = r_outs[i];
-    }
+    for (int i = 0; i < n_y_outs; ++i) a.y_outs[i] = y_outs[i];
+    for (int i = 0; i < n_r_outs; ++i) a.r_outs[i] = r_outs[i];
     a.r = r; a.w = w;
-    a.n_outs = n_outs;
+    a.n_y_outs = n_y_outs;
+    a.n_r_outs = n_r_outs;
     a.row_begin = row_begin;
     a.row_end = row_begin + row_count;
     a.hidden = (int)hidden;
@@ -816,9 +815,9 @@ int rmsnorm_fp8_template_launch(const rt_params* p, const void* x, const void* r
 }
 
 int rmsnorm_allreduce_template_launch(const rt_params* p, const void* const* x_parts, int32_t n_parts, const void* r,
-                                      const void* w, void* const* y_outs, void* const* r_outs, int32_t n_outs,
-                                      int64_t row_begin, int64_t row_count, int64_t hidden, float eps, int dtype,
-                                      void* stream)
+                                      const void* w, void* const* y_outs, int32_t n_y_outs, void* const* r_outs,
+                                      int32_t n_r_outs, int64_t row_begin, int64_t row_count, int64_t hidden, float eps,
+                                      int dtype, void* stream)
 {
     if (!p) {
         rt::set_error("params is NULL");
@@ -828,8 +827,8 @@ int rmsnorm_allreduce_template_launch(const rt_params* p, const void* const* x_p
         rt::set_error("n_parts=%d is not 2, 4 or 8", n_parts);
         return RT_ERR_SHAPE;
     }
-    if (n_outs < 1 || n_outs > rt::kMaxParts) {
-        rt::set_error("n_outs=%d outside 1..%d", n_outs, rt::kMaxParts);
+    if (n_y_outs < 1 || n_y_outs > rt::kMaxParts || n_r_outs < 1 || n_r_outs > rt::kMaxParts) {
+        rt::set_error("n_y_outs=%d or n_r_outs=%d outside 1..%d", n_y_outs, n_r_outs, rt::kMaxParts);
         return RT_ERR_SHAPE;
     }
     if (row_begin < 0 || row_count < 0) {
@@ -849,17 +848,21 @@ int rmsnorm_allreduce_template_launch(const rt_params* p, const void* const* x_p
             }
             bits |= (uintptr_t)x_parts[i];
         }
-        for (int i = 0; i < n_outs; ++i) {
-            if (!y_outs[i] || !r_outs[i]) {
-                rt::set_error("destination %d is NULL", i);
-                return RT_ERR_NULL;
-            }
-            bits |= (uintptr_t)y_outs[i] | (uintptr_t)r_outs[i];
-            for (int k = 0; k < n_parts; ++k)
-                if (y_outs[i] == x_parts[k] || r_outs[i] == x_parts[k]) {
-                    rt::set_error("destination %d is part %d of x", i, k);
-                    return RT_ERR_SHAPE;
+        for (int pass = 0; pass < 2; ++pass) {
+            void* const* outs = pass == 0 ? y_outs : r_outs;
+            const int n_dst = pass == 0 ? n_y_outs : n_r_outs;
+            for (int i = 0; i < n_dst; ++i) {
+                if (!outs[i]) {
+                    rt::set_error("%s destination %d is NULL", pass == 0 ? "y" : "r_out", i);
+                    return RT_ERR_NULL;
                 }
+                bits |= (uintptr_t)outs[i];
+                for (int k = 0; k < n_parts; ++k)
+                    if (outs[i] == x_parts[k]) {
+                        rt::set_error("%s destination %d is part %d of x", pass == 0 ? "y" : "r_out", i, k);
+                        return RT_ERR_SHAPE;
+                    }
+            }
         }
     }
     rt_limits L;
@@ -875,8 +878,8 @@ int rmsnorm_allreduce_template_launch(const rt_params* p, const void* const* x_p
     rt::Plan plan;
     st = rt::make_plan(&s, p, &L, &plan);
     if (st != RT_OK) return st;
-    return rt::launch_allreduce_plan(plan, x_parts, n_parts, r, w, y_outs, r_outs, n_outs, row_begin, row_count, hidden, eps,
-                                     (cudaStream_t)stream);
+    return rt::launch_allreduce_plan(plan, x_parts, n_parts, r, w, y_outs, n_y_outs, r_outs, n_r_outs, row_begin, row_count,
+                                     hidden, eps, (cudaStream_t)stream);
 }
 
 int merge_attn_states_template_launch(const rt_params* p, const void* v_a, const float* s_a, const void* v_b,

@@ -392,7 +392,7 @@ struct DeviceEvaluator : Evaluator {
                 parts[k] = (const char*)ws.x + (size_t)shape.n_parts * off + (size_t)k * set_bytes;
             void* y_out = (char*)ws.y + off;
             void* r_out = (char*)ws.r_out + off;
-            return launch_allreduce_plan(plan, parts, shape.n_parts, (const char*)ws.r + off, ws.w, &y_out, &r_out, 1, 0,
+            return launch_allreduce_plan(plan, parts, shape.n_parts, (const char*)ws.r + off, ws.w, &y_out, 1, &r_out, 1, 0,
                                          shape.n_tokens, shape.hidden, ws.eps, stream);
         };
         const size_t lse_bytes = is_merge ? (size_t)shape.n_tokens * plan.heads * sizeof(float) : 0;  // one s tensor

@@ -76,8 +76,8 @@ int launch_plan(const Plan& plan, const void* x, const void* r, const void* w, v
 int launch_fp8_plan(const Plan& plan, const void* x, const void* r, const void* w, void* q, float* scale, void* r_out,
                     int64_t n_tokens, int64_t hidden, float eps, cudaStream_t stream);
 int launch_allreduce_plan(const Plan& plan, const void* const* x_parts, int n_parts, const void* r, const void* w,
-                          void* const* y_outs, void* const* r_outs, int n_outs, int64_t row_begin, int64_t row_count,
-                          int64_t hidden, float eps, cudaStream_t stream);
+                          void* const* y_outs, int n_y_outs, void* const* r_outs, int n_r_outs, int64_t row_begin,
+                          int64_t row_count, int64_t hidden, float eps, cudaStream_t stream);
 int launch_merge_plan(const Plan& plan, const void* v_a, const float* s_a, const void* v_b, const float* s_b, void* v_out,
                       float* s_out, int64_t n_tokens, cudaStream_t stream);
 int launch_silu_plan(const Plan& plan, const void* x, void* out, int64_t n_tokens, cudaStream_t stream);

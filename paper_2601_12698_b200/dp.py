@@ -114,7 +114,9 @@ class FusedAllreduceNorm:
     ``x_parts[k]`` is rank k's partial x, ``y_outs[k]`` / ``r_outs[k]`` rank k's output tensors, all [n_rows, hidden]
     and all addressable from this rank's GPU (index ``rank`` is this rank's own memory, the others are peer
     mappings).  A call runs this rank's block of rows: it reads every rank's partial for those rows, and writes
-    the rows of y and r_out into every rank's outputs, so that after all ranks' calls each rank holds all rows.
+    the rows of y into every rank's y, so that after all ranks' calls each rank holds all rows of y.  The new
+    residual of those rows goes to this rank's own r_out only - the rank's next norm reads the residual of its
+    own block and nothing else - unless ``gather_residual`` asks for every rank to receive it too.
 
     The kernel never waits for another rank.  The group meets in stream order instead: a one-element all-reduce
     on the launch stream before the kernel (every rank's partial is complete once it returns) and one after it
@@ -129,6 +131,7 @@ class FusedAllreduceNorm:
     r_outs: list
     launch: object
     sync: object = None  # callable run before and after the launch; default: a one-element all-reduce
+    gather_residual: bool = False
 
     def __post_init__(self):
         if self.world not in (2, 4, 8):
@@ -153,7 +156,8 @@ class FusedAllreduceNorm:
         """r: this rank's residual [n_rows, hidden] (the same values on every rank); w: [hidden]."""
         sh = self.shard
         self._meet(r.device)
-        self.launch(theta, self.x_parts, r, w, self.y_outs, self.r_outs, sh.row_begin, sh.rows, eps, stream)
+        r_outs = self.r_outs if self.gather_residual else [self.r_outs[self.rank]]
+        self.launch(theta, self.x_parts, r, w, self.y_outs, r_outs, sh.row_begin, sh.rows, eps, stream)
         self._meet(r.device)
         return sh
 

@@ -96,13 +96,14 @@ def _tp_worker(rank: int, world: int, port: int, shared: dict, out_dir: str):
     # Stand-in for the CUDA entry point with the same signature: the oracle on the requested rows, written to every
     # destination.  Shared-memory tensors stand in for peer-mapped GPU memory.
     def launch(theta, x_parts, r, w, y_outs, r_outs, row_begin, row_count, eps, stream):
-        calls.append((tuple(theta), row_begin, row_count, len(x_parts), len(y_outs)))
+        calls.append((tuple(theta), row_begin, row_count, len(x_parts), len(y_outs), len(r_outs)))
         rows = slice(row_begin, row_begin + row_count)
         stacked = torch.stack([p[rows] for p in x_parts]).contiguous()
         y, ro = oracle.allreduce_add_rmsnorm(stacked, r[rows].contiguous(), w, eps)
-        for k in range(len(y_outs)):
-            y_outs[k][rows] = y
-            r_outs[k][rows] = ro
+        for dst in y_outs:
+            dst[rows] = y
+        for dst in r_outs:
+            dst[rows] = ro
 
     # every rank fills its own partial, then the group runs the fused operator
     g = torch.Generator().manual_seed(100 + rank)
@@ -113,9 +114,16 @@ def _tp_worker(rank: int, world: int, port: int, shared: dict, out_dir: str):
                                sync=dist.barrier)
     sh = op((256, 1, 16, 1, 0, 0, 1), shared["r"], shared["w"], 1e-6)
     assert (sh.row_begin, sh.row_end) == ((0, 19), (19, 37))[rank]          # 37 rows over two ranks: 19 + 18
-    assert calls == [((256, 1, 16, 1, 0, 0, 1), sh.row_begin, sh.rows, world, world)]
-    # after the second meeting this rank's outputs hold every row
-    torch.save({"y": shared["y"][rank].clone(), "ro": shared["r_out"][rank].clone()}, os.path.join(out_dir, f"tp{rank}.pt"))
+    assert calls == [((256, 1, 16, 1, 0, 0, 1), sh.row_begin, sh.rows, world, world, 1)]
+    # after the second meeting this rank's y holds every row, its r_out the rows of its own block
+    torch.save({"y": shared["y"][rank].clone(), "ro": shared["r_out"][rank].clone(), "rows": (sh.row_begin, sh.row_end)},
+               os.path.join(out_dir, f"tp{rank}.pt"))
+    # the same again with the residual sent to every rank
+    dp.barrier(device)
+    op.gather_residual = True
+    op((256, 1, 16, 1, 0, 0, 1), shared["r"], shared["w"], 1e-6)
+    assert calls[-1][-1] == world
+    torch.save({"ro_all": shared["r_out"][rank].clone()}, os.path.join(out_dir, f"tpg{rank}.pt"))
     dp.barrier(device)
     dp.shutdown()
 
@@ -137,7 +145,12 @@ def test_two_gloo_ranks_tensor_parallel_norm(tmp_path):
     y_ref, r_ref = oracle.allreduce_add_rmsnorm(torch.stack(shared["x"]).contiguous(), shared["r"], shared["w"], 1e-6)
     for k in range(world):
         assert torch.equal(got[k]["y"].view(torch.int16), y_ref.view(torch.int16))
-        assert torch.equal(got[k]["ro"].view(torch.int16), r_ref.view(torch.int16))
+        lo, hi = got[k]["rows"]
+        assert torch.equal(got[k]["ro"][lo:hi].view(torch.int16), r_ref[lo:hi].view(torch.int16))
+        outside = torch.cat([got[k]["ro"][:lo], got[k]["ro"][hi:]])
+        assert bool((outside == 0).all())                                   # another rank's rows were not sent here
+        gathered = torch.load(os.path.join(tmp_path, f"tpg{k}.pt"))["ro_all"]
+        assert torch.equal(gathered.view(torch.int16), r_ref.view(torch.int16))
 
 
 def test_fused_allreduce_norm_argument_checks():

@@ -122,39 +122,68 @@ def test_refusals(B):
     x = [torch.zeros(T, H, dtype=torch.bfloat16, device="cuda") for _ in range(4)]
     r = torch.zeros(T, H, dtype=torch.bfloat16, device="cuda"); w = torch.ones(H, dtype=torch.bfloat16, device="cuda")
     y = torch.full_like(r, 9.0); ro = torch.full_like(r, 9.0)
-    call = B.lib.rmsnorm_allreduce_template_launch
     vp = B.c_void_p
 
     def arr(ts):
         return (vp * len(ts))(*[t.data_ptr() if t is not None else None for t in ts])
 
+    def call(th, xs=x, n_parts=None, r_=r, w_=w, ys=(y,), ros=(ro,), n_y=None, n_r=None, row_begin=0, rows=T, hidden=H,
+             dtype=B.RT_BF16):
+        return B.lib.rmsnorm_allreduce_template_launch(
+            B.byref(th), arr(list(xs)) if xs is not None else None, len(xs) if n_parts is None else n_parts,
+            r_.data_ptr() if r_ is not None else None, w_.data_ptr(), arr(list(ys)), len(ys) if n_y is None else n_y,
+            arr(list(ros)), len(ros) if n_r is None else n_r, row_begin, rows, hidden, EPS, dtype, None)
+
     th = B.make_params()
     before = B.rt_launch_count()
-    ok_tail = (0, T, H, EPS, B.RT_BF16, None)
     for bad in (B.make_params(vec_bytes=8), B.make_params(reduce=B.RT_REDUCE_SMEM), B.make_params(stage=B.RT_STAGE_SMEM_TMA),
                 B.make_params(stage=B.RT_STAGE_SMEM_LDG), B.make_params(reduce=B.RT_REDUCE_CLUSTER, cluster_size=2),
                 B.make_params(unroll=3), B.make_params(threads_per_row=48)):
-        assert call(B.byref(bad), arr(x), 4, r.data_ptr(), w.data_ptr(), arr([y]), arr([ro]), 1, *ok_tail) == B.RT_ERR_INFEASIBLE, repr(bad)
-    assert call(B.byref(th), arr(x[:3]), 3, r.data_ptr(), w.data_ptr(), arr([y]), arr([ro]), 1, *ok_tail) == B.RT_ERR_SHAPE
-    assert call(B.byref(th), arr(x), 4, r.data_ptr(), w.data_ptr(), arr([y]), arr([ro]), 0, *ok_tail) == B.RT_ERR_SHAPE
-    assert call(B.byref(th), arr(x), 4, r.data_ptr(), w.data_ptr(), arr([y] * 9), arr([ro] * 9), 9, *ok_tail) == B.RT_ERR_SHAPE
-    assert call(B.byref(th), arr(x), 4, r.data_ptr(), w.data_ptr(), arr([y]), arr([ro]), 1, -1, T, H, EPS, B.RT_BF16, None) == B.RT_ERR_SHAPE
-    assert call(B.byref(th), arr(x), 4, r.data_ptr(), w.data_ptr(), arr([x[1]]), arr([ro]), 1, *ok_tail) == B.RT_ERR_SHAPE  # writes a part
-    assert call(B.byref(th), arr(x[:3] + [None]), 4, r.data_ptr(), w.data_ptr(), arr([y]), arr([ro]), 1, *ok_tail) == B.RT_ERR_NULL
-    assert call(B.byref(th), arr(x), 4, None, w.data_ptr(), arr([y]), arr([ro]), 1, *ok_tail) == B.RT_ERR_NULL
-    assert call(B.byref(th), None, 4, r.data_ptr(), w.data_ptr(), arr([y]), arr([ro]), 1, *ok_tail) == B.RT_ERR_NULL
-    assert call(B.byref(th), arr(x), 4, r.data_ptr(), w.data_ptr(), arr([y]), arr([ro]), 1, 0, T, 4100, EPS, B.RT_BF16, None) == B.RT_ERR_ALIGN
+        assert call(bad) == B.RT_ERR_INFEASIBLE, repr(bad)
+    assert call(th, xs=x[:3]) == B.RT_ERR_SHAPE                        # three parts
+    assert call(th, n_y=0) == B.RT_ERR_SHAPE and call(th, n_r=0) == B.RT_ERR_SHAPE
+    assert call(th, ys=[y] * 9) == B.RT_ERR_SHAPE and call(th, ros=[ro] * 9) == B.RT_ERR_SHAPE
+    assert call(th, row_begin=-1) == B.RT_ERR_SHAPE and call(th, rows=-2) == B.RT_ERR_SHAPE
+    assert call(th, ys=[x[1]]) == B.RT_ERR_SHAPE and call(th, ros=[ro, x[3]]) == B.RT_ERR_SHAPE   # would overwrite a part
+    assert call(th, xs=x[:3] + [None]) == B.RT_ERR_NULL
+    assert call(th, r_=None) == B.RT_ERR_NULL
+    assert call(th, xs=None, n_parts=4) == B.RT_ERR_NULL
+    assert call(th, ys=[y, None]) == B.RT_ERR_NULL
+    assert call(th, hidden=4100) == B.RT_ERR_ALIGN
     off = torch.zeros(T * H + 8, dtype=torch.bfloat16, device="cuda")[4:4 + T * H].view(T, H)   # 8-byte aligned only
-    assert call(B.byref(th), arr([off] + x[1:]), 4, r.data_ptr(), w.data_ptr(), arr([y]), arr([ro]), 1, *ok_tail) == B.RT_ERR_ALIGN
-    assert call(B.byref(th), arr(x), 4, r.data_ptr(), w.data_ptr(), arr([y]), arr([ro]), 1, 0, T, H, EPS, 7, None) == B.RT_ERR_DTYPE
+    assert call(th, xs=[off] + x[1:]) == B.RT_ERR_ALIGN
+    assert call(th, dtype=7) == B.RT_ERR_DTYPE
     # a 32-thread row of 1024 vectors would keep 32 vectors per thread: no such instance
-    wide = B.make_params(threads_per_row=32)
     x8 = [torch.zeros(2, 8192, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
     r8 = torch.zeros(2, 8192, dtype=torch.bfloat16, device="cuda"); w8 = torch.ones(8192, dtype=torch.bfloat16, device="cuda")
-    assert call(B.byref(wide), arr(x8), 2, r8.data_ptr(), w8.data_ptr(), arr([r8.clone()]), arr([r8.clone()]), 1, 0, 2, 8192, EPS,
-                B.RT_BF16, None) == B.RT_ERR_INFEASIBLE
+    assert call(B.make_params(threads_per_row=32), xs=x8, r_=r8, w_=w8, ys=[r8.clone()], ros=[r8.clone()], rows=2,
+                hidden=8192) == B.RT_ERR_INFEASIBLE
     torch.cuda.synchronize()
     assert B.rt_launch_count() == before and bool((y == 9.0).all()) and bool((ro == 9.0).all())
+
+
+def test_residual_stays_with_the_owner_of_the_rows(B, oracle_lib):
+    """The usual group form: y goes to every rank, the new residual only to the rank that owns the rows."""
+    from paper_2601_12698_b200 import dp
+    T, H, n_parts = 45, 2048, 4
+    parts, r, w = _inputs(T, H, "bf16", n_parts, seed=633)
+    y_ref, r_ref = oracle_lib.allreduce_add_rmsnorm(parts, r, w, EPS)
+    pd, wd = parts.cuda(), w.cuda()
+    x_parts = [pd[k] for k in range(n_parts)]
+    residual = [r.cuda() for _ in range(n_parts)]                      # every rank's copy of the residual stream
+    y_outs = [torch.full((T, H), float("nan"), dtype=torch.bfloat16, device="cuda") for _ in range(n_parts)]
+    th = B.make_params(threads_per_row=256)
+    for rank in range(n_parts):
+        sh = dp.strong_shard(T, rank, n_parts)
+        B.rmsnorm_allreduce_template_launch(th, x_parts, residual[rank], wd, y_outs, [residual[rank]], sh.row_begin, sh.rows, EPS)
+    for rank in range(n_parts):
+        sh = dp.strong_shard(T, rank, n_parts)
+        worst, bad = oracle_lib.compare_y(y_outs[rank].cpu(), y_ref)
+        assert bad == 0, (rank, worst)
+        own = slice(sh.row_begin, sh.row_end)
+        assert oracle_lib.bit_mismatches(residual[rank][own].cpu().contiguous(), r_ref[own].contiguous()) == 0
+        others = torch.ones(T, dtype=torch.bool); others[own] = False
+        assert torch.equal(residual[rank].cpu()[others].view(torch.int16), r[others].view(torch.int16))  # untouched
 
 
 @pytest.mark.parametrize("name", ["c2ar8_decode_bf16_64x8192", "c3ar4_prefill_bf16_4096x8192"])
