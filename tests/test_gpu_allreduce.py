@@ -209,3 +209,19 @@ def test_search_on_the_stacked_workspace_and_sampled_parity(B, oracle_lib, name)
     B.rmsnorm_allreduce_template_launch(res.best, [pd[k] for k in range(wl.n_parts)], rd, wd, [y], [ro], 0, wl.n_tokens, wl.eps)
     _assert_matches(oracle_lib, y[rows], ro[rows], y_rows, r_rows, repr(res.best))
     assert not bool(torch.isnan(y.float()).any()) and not bool(torch.isnan(ro.float()).any())
+
+
+def test_shipped_table_drives_the_launch(B, oracle_lib):
+    table = B.SpecTable.default()
+    assert B.RT_OP_ADD_RMSNORM_ALLREDUCE in table.generals
+    for n_parts, T, H in ((8, 64, 8192), (4, 300, 8192), (2, 9, 1024)):
+        parts, r, w = _inputs(T, H, "bf16", n_parts, seed=650 + n_parts)
+        y_ref, r_ref = oracle_lib.allreduce_add_rmsnorm(parts, r, w, EPS)
+        pd, rd, wd = parts.cuda(), r.cuda(), w.cuda()
+        y, ro = torch.full_like(rd, float("nan")), torch.full_like(rd, float("nan"))
+        theta = table.launch_rmsnorm_allreduce([pd[k] for k in range(n_parts)], rd, wd, [y], [ro], 0, T, EPS)
+        shape = B.shape_of(T, H, "bf16", op=B.RT_OP_ADD_RMSNORM_ALLREDUCE, n_parts=n_parts)
+        assert B.tuner_check_params(shape, theta) == B.RT_OK
+        if (n_parts, T, H) == (8, 64, 8192):
+            assert table.lookup(shape)[1] == "table_exact"
+        _assert_matches(oracle_lib, y, ro, y_ref, r_ref, (n_parts, T, H, repr(theta)))
