@@ -500,6 +500,19 @@ int rt_kernel_instance(int32_t i, int32_t* dtype, int32_t* vec_bytes, int32_t* s
 int32_t rt_kernel_instance_op(int32_t i);
 /* Partial inputs the i-th instance sums per element (all-reduce-fused norm; 0 for the others, -1 out of range). */
 int32_t rt_kernel_instance_parts(int32_t i);
+/*
+ * Process-wide launch options.  RT_OPTION_PROGRAMMATIC_LAUNCH (0 or 1, default 1): launch every kernel of the
+ * library with the programmatic-stream-serialization attribute, so that a launch's CTAs may be scheduled, and
+ * run their prologue, while the previous kernel of the stream is still finishing; each kernel waits
+ * (griddepcontrol.wait) for that kernel to complete, and for its writes to be visible, before it touches memory,
+ * so results do not depend on the option.  Measured on B200: 10-13% on the latency-bound shapes inside a CUDA
+ * graph, 40% on them in a plain stream of launches, 1-3.5% on the bandwidth-bound shapes.  Set it to 0 to launch
+ * with full stream serialization.
+ * rt_set_option returns RT_ERR_SHAPE for an unknown option or value; rt_get_option returns -1 for an unknown option.
+ */
+enum { RT_OPTION_PROGRAMMATIC_LAUNCH = 0 };
+int rt_set_option(int32_t option, int32_t value);
+int32_t rt_get_option(int32_t option);
 /* Kernel launches issued by this library in this process since load (all entry points). */
 int64_t rt_launch_count(void);
 /* Frees what the library allocated on the device.  Safe to call more than once. */

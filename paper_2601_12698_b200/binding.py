@@ -18,6 +18,7 @@ RT_BF16, RT_FP16, RT_FP32 = 0, 1, 2
 RT_OP_ADD_RMSNORM, RT_OP_SILU_AND_MUL, RT_OP_MERGE_ATTN_STATES, RT_OP_ADD_RMSNORM_FP8 = 0, 1, 2, 3
 RT_OP_ADD_RMSNORM_ALLREDUCE = 4
 RT_MAX_PARTS = 8
+RT_OPTION_PROGRAMMATIC_LAUNCH = 0
 RT_STAGE_REG, RT_STAGE_SMEM_LDG, RT_STAGE_SMEM_TMA = 0, 1, 2
 RT_REDUCE_SHFL, RT_REDUCE_SMEM, RT_REDUCE_CLUSTER = 0, 1, 2
 RT_PRUNE_IDLE_THREADS, RT_PRUNE_DUPLICATES, RT_PRUNE_CLUSTER_WAVES, RT_PRUNE_IDLE_ROWS = 1, 2, 4, 8
@@ -115,6 +116,8 @@ _SIGNATURES = {
                                                   POINTER(c_void_p), c_int32, POINTER(c_void_p), c_int32, c_int64,
                                                   c_int64, c_int64, c_float, c_int, c_void_p]),
     "rt_kernel_instance_parts": (c_int32, [c_int32]),
+    "rt_set_option": (c_int, [c_int32, c_int32]),
+    "rt_get_option": (c_int32, [c_int32]),
     "merge_attn_states_template_launch": (c_int, [POINTER(rt_params), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                                   c_void_p, c_int64, c_int64, c_int64, c_int, c_void_p]),
     "rmsnorm_template_run_host": (c_int, [POINTER(rt_params), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,

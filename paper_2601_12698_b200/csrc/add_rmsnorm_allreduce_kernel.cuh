@@ -48,6 +48,7 @@ __global__ void add_rmsnorm_allreduce_kernel(const AllreduceArgs a)
     const size_t row_off = (size_t)(row < a.row_end ? row : a.row_begin) * (size_t)a.nvec * VB;
     const unsigned char* rrow = reinterpret_cast<const unsigned char*>(a.r) + row_off;
     const unsigned char* wrow = reinterpret_cast<const unsigned char*>(a.w);
+    wait_for_previous_kernel();
 
     // the same vector to every destination; the destination count is uniform over the grid
     auto store_all = [&](void* const (&dst)[kMaxParts], int n_dst, size_t off, const Vec<VB>& v) {

@@ -84,6 +84,7 @@ __global__ void add_rmsnorm_fp8_kernel(const Fp8Args a)
     const unsigned char* wrow = reinterpret_cast<const unsigned char*>(a.w);
     unsigned char* orow = reinterpret_cast<unsigned char*>(a.r_out) + row_off;
     unsigned char* qrow = reinterpret_cast<unsigned char*>(a.q) + row_off / 2;  // one byte per element
+    wait_for_previous_kernel();
 
     float ss = 0.f, amax = 0.f;
 

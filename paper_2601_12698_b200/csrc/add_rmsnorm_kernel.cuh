@@ -302,6 +302,17 @@ __device__ __forceinline__ bool mbarrier_wait_bounded(uint64_t* bar, uint32_t pa
     return false;
 }
 
+// Programmatic dependent launch.  When the kernel is launched with the programmatic-stream-serialization
+// attribute, its CTAs may be scheduled while the previous kernel of the stream is still draining; everything above
+// this call (index arithmetic) overlaps that kernel's tail, and the call returns once that kernel has completed
+// and its writes are visible, so nothing below it can see unfinished data.  Without the attribute it is a no-op.
+// The kernels never signal their own dependents early (no griddepcontrol.launch_dependents): measured on B200,
+// dependents that start while this kernel still streams only take SM slots from it.
+__device__ __forceinline__ void wait_for_previous_kernel()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // ---- the per-row reduction of the sum of squares ---------------------------------------------
 
 // Every thread of the row passes its partial; every thread of the row receives the row total.
@@ -416,6 +427,7 @@ __global__ void add_rmsnorm_kernel(const KernelArgs a)
     unsigned char* yrow = reinterpret_cast<unsigned char*>(a.y) + row_off;
     unsigned char* orow = reinterpret_cast<unsigned char*>(a.r_out) + row_off;
 
+    wait_for_previous_kernel();
     float ss = 0.f;
 
     if constexpr (STAGE == kStageReg) {

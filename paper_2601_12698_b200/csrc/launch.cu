@@ -30,6 +30,7 @@ namespace {
 
 thread_local char tls_error[512] = "";
 std::atomic<int64_t> g_launches{0};
+std::atomic<int> g_programmatic_launch{1};
 std::mutex g_mutex;
 
 constexpr int kMaxDevices = 64;
@@ -524,6 +525,29 @@ int plan_occupancy(const Plan& plan, const rt_limits* L, int* regs_per_thread)
     return (int)blocks;
 }
 
+// Launch attributes common to every kernel of the library: the cluster shape, and - unless switched off through
+// rt_set_option - programmatic stream serialization (the kernels wait for their predecessor themselves).
+struct LaunchAttrs {
+    cudaLaunchAttribute a[2];
+};
+static void set_launch_attrs(cudaLaunchConfig_t* cfg, LaunchAttrs* la, int cluster)
+{
+    cfg->numAttrs = 0;
+    if (cluster > 1) {
+        cudaLaunchAttribute& attr = la->a[cfg->numAttrs++];
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = cluster;
+        attr.val.clusterDim.y = 1;
+        attr.val.clusterDim.z = 1;
+    }
+    if (g_programmatic_launch.load(std::memory_order_relaxed)) {
+        cudaLaunchAttribute& attr = la->a[cfg->numAttrs++];
+        attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr.val.programmaticStreamSerializationAllowed = 1;
+    }
+    cfg->attrs = cfg->numAttrs ? la->a : nullptr;
+}
+
 int launch_fp8_plan(const Plan& plan, const void* x, const void* r, const void* w, void* q, float* scale, void* r_out,
                     int64_t n_tokens, int64_t hidden, float eps, cudaStream_t stream)
 {
@@ -549,6 +573,8 @@ int launch_fp8_plan(const Plan& plan, const void* x, const void* r, const void* 
     cfg.blockDim = dim3(plan.block_x, plan.block_y, 1);
     cfg.dynamicSmemBytes = plan.dyn_smem;
     cfg.stream = stream;
+    LaunchAttrs la;
+    set_launch_attrs(&cfg, &la, 1);
     void* params[] = {&a};
     cudaError_t e = cudaLaunchKernelExC(&cfg, k.fn, params);
     if (e != cudaSuccess) {
@@ -592,6 +618,8 @@ int launch_allreduce_plan(const Plan& plan, const void* const* x_parts, int n_pa
     cfg.gridDim = dim3(plan.grid_x, 1, 1);
     cfg.blockDim = dim3(plan.block_x, plan.block_y, 1);
     cfg.stream = stream;
+    LaunchAttrs la;
+    set_launch_attrs(&cfg, &la, 1);
     void* params[] = {&a};
     cudaError_t e = cudaLaunchKernelExC(&cfg, k.fn, params);
     if (e != cudaSuccess) {
@@ -631,6 +659,8 @@ int launch_merge_plan(const Plan& plan, const void* v_a, const float* s_a, const
     cfg.blockDim = dim3(plan.block_x, plan.block_y, 1);
     cfg.dynamicSmemBytes = plan.dyn_smem;
     cfg.stream = stream;
+    LaunchAttrs la;
+    set_launch_attrs(&cfg, &la, 1);
     void* params[] = {&a};
     cudaError_t e = cudaLaunchKernelExC(&cfg, k.fn, params);
     if (e != cudaSuccess) {
@@ -665,6 +695,8 @@ int launch_silu_plan(const Plan& plan, const void* x, void* out, int64_t n_token
     cfg.blockDim = dim3(plan.block_x, plan.block_y, 1);
     cfg.dynamicSmemBytes = plan.dyn_smem;
     cfg.stream = stream;
+    LaunchAttrs la;
+    set_launch_attrs(&cfg, &la, 1);
     void* params[] = {&a};
     cudaError_t e = cudaLaunchKernelExC(&cfg, k.fn, params);
     if (e != cudaSuccess) {
@@ -703,15 +735,8 @@ int launch_plan(const Plan& plan, const void* x, const void* r, const void* w, v
     cfg.blockDim = dim3(plan.block_x, plan.block_y, 1);
     cfg.dynamicSmemBytes = plan.dyn_smem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr;
-    if (plan.cluster > 1) {
-        attr.id = cudaLaunchAttributeClusterDimension;
-        attr.val.clusterDim.x = plan.cluster;
-        attr.val.clusterDim.y = 1;
-        attr.val.clusterDim.z = 1;
-        cfg.attrs = &attr;
-        cfg.numAttrs = 1;
-    }
+    LaunchAttrs la;
+    set_launch_attrs(&cfg, &la, plan.cluster);
     void* params[] = {&a};
     cudaError_t e = cudaLaunchKernelExC(&cfg, k.fn, params);
     if (e != cudaSuccess) {
@@ -1017,6 +1042,21 @@ int32_t rt_kernel_instance_op(int32_t i)
 {
     if (i < 0 || i >= (int32_t)rt::registry().size()) return -1;
     return rt::registry()[i].op;
+}
+
+int rt_set_option(int32_t option, int32_t value)
+{
+    if (option != RT_OPTION_PROGRAMMATIC_LAUNCH || (value != 0 && value != 1)) {
+        rt::set_error("unknown option %d or value %d", option, value);
+        return RT_ERR_SHAPE;
+    }
+    rt::g_programmatic_launch.store(value);
+    return RT_OK;
+}
+
+int32_t rt_get_option(int32_t option)
+{
+    return option == RT_OPTION_PROGRAMMATIC_LAUNCH ? rt::g_programmatic_launch.load() : -1;
 }
 
 int32_t rt_kernel_instance_parts(int32_t i)

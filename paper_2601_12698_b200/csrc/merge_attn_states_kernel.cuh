@@ -67,6 +67,7 @@ __global__ void merge_attn_states_kernel(const MergeArgs a)
     const float* sa = a.s_a + safe_row * a.heads;
     const float* sb = a.s_b + safe_row * a.heads;
     float* so = a.s_out + safe_row * a.heads;
+    wait_for_previous_kernel();
 
     if constexpr (STAGE == kStageSmemTma) {
         __shared__ __align__(8) uint64_t bars[kMaxRowsPerCta];

@@ -42,6 +42,7 @@ __global__ void silu_and_mul_kernel(const SiluArgs a)
     const unsigned char* gate = reinterpret_cast<const unsigned char*>(a.x) + safe_row * 2 * half_bytes;
     const unsigned char* value = gate + half_bytes;
     unsigned char* out = reinterpret_cast<unsigned char*>(a.out) + safe_row * half_bytes;
+    wait_for_previous_kernel();
 
     if constexpr (STAGE == kStageSmemTma) {
         __shared__ __align__(8) uint64_t bars[kMaxRowsPerCta];

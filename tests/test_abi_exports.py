@@ -69,3 +69,15 @@ def test_no_device_is_reported_not_crashed():
     assert B.lib.tuner_derive_feasible(ctypes.byref(s), None, 0, ctypes.byref(n)) == B.RT_ERR_NO_DEVICE
     th = B.make_params()
     assert B.lib.rmsnorm_template_launch(ctypes.byref(th), 8, 8, 8, 8, 8, 4, 64, 1e-6, 0, None) == B.RT_ERR_NO_DEVICE
+
+
+def test_launch_option_is_validated_and_remembered():
+    from paper_2601_12698_b200 import binding as B
+    opt = B.RT_OPTION_PROGRAMMATIC_LAUNCH
+    assert B.lib.rt_get_option(opt) == 1                       # the default
+    try:
+        assert B.lib.rt_set_option(opt, 0) == B.RT_OK and B.lib.rt_get_option(opt) == 0
+        assert B.lib.rt_set_option(opt, 2) == B.RT_ERR_SHAPE and B.lib.rt_get_option(opt) == 0
+        assert B.lib.rt_set_option(7, 1) == B.RT_ERR_SHAPE and B.lib.rt_get_option(7) == -1
+    finally:
+        assert B.lib.rt_set_option(opt, 1) == B.RT_OK

@@ -268,3 +268,42 @@ def test_more_than_2_to_31_elements(B, oracle_lib):
     want = y_ref.cuda().repeat(reps - reps // 2, 1)
     assert B.tuner_compare(y[half:], want, B.RT_CMP_ULP16, 2.0)[1] == 0
     assert B.rt_device_status() == 0
+
+
+def test_programmatic_launch_option_does_not_change_results(B):
+    """Back-to-back in-place launches (each consumes what the previous one wrote) with and without the
+    programmatic-stream-serialization attribute: the bits must agree, in a plain stream and inside a CUDA graph."""
+    from paper_2601_12698_b200 import synth
+    x, r, w = synth.make_inputs(64, 4096, "bf16", seed=77)
+    w = (w * 0 + 1).to(w.dtype)
+    thetas = [B.make_params(threads_per_row=512), B.make_params(threads_per_row=256, stage=B.RT_STAGE_SMEM_TMA),
+              B.make_params(threads_per_row=128, reduce=B.RT_REDUCE_CLUSTER, cluster_size=4)]
+    opt = B.RT_OPTION_PROGRAMMATIC_LAUNCH
+    results = {}
+    try:
+        for value in (0, 1):
+            assert B.lib.rt_set_option(opt, value) == B.RT_OK
+            for mode in ("stream", "graph"):
+                xd, rd, wd = x.cuda(), r.cuda(), w.cuda()
+                stream = torch.cuda.Stream()
+                stream.wait_stream(torch.cuda.current_stream())
+
+                def chain():
+                    for i in range(12):  # y over x, r' over r: every launch depends on the one before
+                        B.rmsnorm_template_launch(thetas[i % len(thetas)], xd, rd, wd, xd, rd, 1e-6, stream=stream)
+                if mode == "graph":
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g, stream=stream):
+                        chain()
+                    g.replay()
+                    torch.cuda.synchronize()
+                else:
+                    chain()
+                    stream.synchronize()
+                results[(value, mode)] = (xd.cpu().view(torch.int16).clone(), rd.cpu().view(torch.int16).clone())
+    finally:
+        assert B.lib.rt_set_option(opt, 1) == B.RT_OK
+    base = results[(0, "stream")]
+    for key, got in results.items():
+        assert torch.equal(got[0], base[0]) and torch.equal(got[1], base[1]), key
+    assert B.rt_device_status() == 0
