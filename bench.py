@@ -49,12 +49,12 @@ NOMINAL_HBM_GBS = 8000.0
 # DRAM traffic of one launch of the top kernel from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum), valid only for the kernel source and theta it was taken on.
 NCU_TRAFFIC = {
-    "kernel_sha256_16": "1bb03ec60e25a158",
+    "kernel_sha256_16": "a5caaa4fd7831901",
     "workload": "c3_prefill_bf16_16384x8192",
     # (threads_per_row, rows_per_cta, vec_bytes, unroll, stage, reduce, cluster_size) -> DRAM bytes per launch
     "bytes_per_launch": {
-        (256, 1, 16, 1, 2, 0, 1): 1021075968,  # 537.02 MB read + 484.06 MB written
-        (256, 1, 16, 4, 0, 0, 1): 1022077184,  # 536.90 MB read + 485.18 MB written
+        (256, 1, 16, 1, 2, 0, 1): 1021228032,  # 536.93 MB read + 484.30 MB written
+        (256, 1, 16, 4, 0, 0, 1): 1020643840,  # 536.92 MB read + 483.72 MB written
     },
 }
 
