@@ -55,6 +55,13 @@ NCU_TRAFFIC = {
     "bytes_per_launch": {
         (256, 1, 16, 1, 2, 0, 1): 1021228032,  # 536.93 MB read + 484.30 MB written
         (256, 1, 16, 4, 0, 0, 1): 1020643840,  # 536.92 MB read + 483.72 MB written
+        # the other configurations the search has returned on this shape (dram__bytes metrics only, first of two launches)
+        (256, 1, 16, 2, 0, 0, 1): 1020540928,
+        (256, 1, 16, 2, 2, 0, 1): 1020514048,
+        (256, 1, 16, 4, 2, 0, 1): 1022055424,
+        (512, 1, 16, 1, 2, 0, 1): 1021512704,
+        (512, 1, 16, 2, 0, 0, 1): 1019790592,
+        (512, 1, 16, 4, 0, 0, 1): 1019570944,
     },
 }
 
