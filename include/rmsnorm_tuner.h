@@ -353,8 +353,9 @@ int tuner_derive_counts(const rt_shape* s, const rt_limits* limits, int32_t heur
 
 /*
  * Search(S~, x, Theta_feasible) for one input shape (Algorithm 1): seeds first, then a coarse
- * grid over the feasible set, then steepest-descent hill-climbing over one-step neighbours on
- * measured time, then a re-test of the top_k finalists ("Tuning agent": Top-K re-testing).
+ * grid over the feasible set, then best-first hill-climbing over one-step neighbours on
+ * measured time (around the three fastest points, then, while budget remains, around up to the
+ * twelve fastest), then a re-test of the top_k finalists ("Tuning agent": Top-K re-testing).
  * Every candidate passes the correctness gate (r_out bit-exact, y within 2 ulp for 16-bit types or
  * 1e-5 relative for fp32, against the uploaded references) before it is timed; candidates that
  * fail the gate or the launch are logged and skipped.

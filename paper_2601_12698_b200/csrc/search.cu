@@ -835,19 +835,27 @@ int run_search(const rt_shape& shape, const rt_limits& limits, const rt_budget& 
             S.time_us[idx] = t;
         }
         // 3. best-first hill-climb: expand the neighbours of the fastest point not yet expanded, among
-        //    the three fastest found so far; stop when those are all expanded or the budget is spent
+        //    the three fastest found so far.  When those are all expanded and budget is left, the frontier
+        //    widens by three at a time (up to the twelve fastest): an optimum two steps away from every
+        //    leader - a narrower vector that only pays with a deeper unroll, say - is reached through a
+        //    runner-up.  Stops when the widest frontier is expanded or the budget is spent.
+        int frontier = 3;
         while (S.budget_left(top_k)) {
             std::vector<int> order;
             for (int i = 0; i < (int)S.cand.size(); ++i)
                 if (S.time_us[i] >= 0.f && isfinite(S.time_us[i])) order.push_back(i);
             std::sort(order.begin(), order.end(), [&](int a, int c) { return S.time_us[a] < S.time_us[c]; });
             int pick = -1;
-            for (int k = 0; k < (int)order.size() && k < 3; ++k)
+            for (int k = 0; k < (int)order.size() && k < frontier; ++k)
                 if (!S.expanded[order[k]]) {
                     pick = order[k];
                     break;
                 }
-            if (pick < 0) break;
+            if (pick < 0) {
+                if (frontier >= 12 || frontier >= (int)order.size()) break;
+                frontier += 3;
+                continue;
+            }
             S.expanded[pick] = 1;
             for (int nb : S.neighbours(pick)) {
                 if (!S.budget_left(top_k)) break;

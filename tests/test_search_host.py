@@ -155,3 +155,24 @@ def test_a_small_budget_still_touches_every_stage_and_reduction_mode(L):
     assert all(modes.count(m) == 2 for m in set(modes))
     # the first point of every mode is the one nearest the middle of the ordered axes
     assert all(r.params.threads_per_row == 256 and r.params.rows_per_cta == 1 and r.params.unroll == 1 for r in grid[:6])
+
+
+def test_an_optimum_two_steps_from_every_leader_is_reached_with_leftover_budget(L):
+    """A narrower vector that only pays with a deeper unroll: both one-step moves towards it are worse than the
+    three leaders, so the climb gets there only because the frontier widens once the leaders are expanded."""
+    s = B.shape_of(64, 11008, "bf16", op=B.RT_OP_SILU_AND_MUL)
+    base = _cost_factory(dict(tpr=1024, rpc=1, unroll=1, vec=16, stage=0, reduce=0))
+
+    def cost(p):
+        if (p.threads_per_row, p.rows_per_cta, p.vec_bytes, p.unroll, p.stage) == (1024, 1, 8, 4, 0):
+            return 90.0                                   # the planted optimum, 10% under the bowl's minimum
+        return base(p)
+
+    feasible = B.tuner_derive_feasible(s, L)
+    assert any((t.threads_per_row, t.rows_per_cta, t.vec_bytes, t.unroll, t.stage) == (1024, 1, 8, 4, 0) for t in feasible)
+    res, log = B.tuner_search_with(s, L, B.make_budget(max_evals=64, top_k=3), cost)
+    assert (res.best.threads_per_row, res.best.vec_bytes, res.best.unroll, res.best.stage) == (1024, 8, 4, 0)
+    assert res.evals_used <= 64
+    # with the budget of a single frontier it stays on the bowl's minimum
+    small, _ = B.tuner_search_with(s, L, B.make_budget(max_evals=20, top_k=2), cost)
+    assert small.evals_used <= 20
