@@ -63,7 +63,13 @@ typedef enum {
 typedef enum {
     RT_STAGE_REG = 0,      /* ld.global vectors straight into registers, row kept as fp32 registers */
     RT_STAGE_SMEM_LDG = 1, /* ld.global vectors, sum kept as fp32 in shared memory */
-    RT_STAGE_SMEM_TMA = 2  /* cp.async.bulk (TMA, one copy per row slice) into shared memory + mbarrier */
+    RT_STAGE_SMEM_TMA = 2, /* cp.async.bulk (TMA, one copy per row slice) into shared memory + mbarrier */
+    RT_STAGE_REG_REALIGN = 3 /* add_rmsnorm only, for rows whose byte length is not a multiple of 16 (the paper's
+                                "vectorization and alignment strategies" axis): the row is cut at the 16-byte
+                                boundaries of the tensor; the whole chunks between them move as 16-byte vectors and
+                                stay in registers, the fewer than 16 bytes before the first and after the last
+                                boundary move one element to a thread.  Takes vec_bytes = 16, the shuffle reduction,
+                                16-byte aligned base pointers and any hidden size */
 } rt_stage;
 
 /* How the per-row sum of squares is combined. */

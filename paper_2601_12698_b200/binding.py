@@ -19,7 +19,7 @@ RT_OP_ADD_RMSNORM, RT_OP_SILU_AND_MUL, RT_OP_MERGE_ATTN_STATES, RT_OP_ADD_RMSNOR
 RT_OP_ADD_RMSNORM_ALLREDUCE = 4
 RT_MAX_PARTS = 8
 RT_OPTION_PROGRAMMATIC_LAUNCH = 0
-RT_STAGE_REG, RT_STAGE_SMEM_LDG, RT_STAGE_SMEM_TMA = 0, 1, 2
+RT_STAGE_REG, RT_STAGE_SMEM_LDG, RT_STAGE_SMEM_TMA, RT_STAGE_REG_REALIGN = 0, 1, 2, 3
 RT_REDUCE_SHFL, RT_REDUCE_SMEM, RT_REDUCE_CLUSTER = 0, 1, 2
 RT_PRUNE_IDLE_THREADS, RT_PRUNE_DUPLICATES, RT_PRUNE_CLUSTER_WAVES, RT_PRUNE_IDLE_ROWS = 1, 2, 4, 8
 RT_PRUNE_DEFAULT = 15
@@ -28,7 +28,7 @@ RT_CMP_BITS, RT_CMP_ULP16, RT_CMP_REL32 = 0, 1, 2
 (RT_OK, RT_ERR_NULL, RT_ERR_DTYPE, RT_ERR_SHAPE, RT_ERR_ALIGN, RT_ERR_INFEASIBLE, RT_ERR_CUDA, RT_ERR_MISMATCH,
  RT_ERR_BUDGET, RT_ERR_DEVICE_TIMEOUT, RT_ERR_CAPACITY, RT_ERR_NO_DEVICE) = range(12)
 PHASE_NAMES = {0: "seed", 1: "grid", 2: "climb", 3: "topk", 4: "sweep"}
-STAGE_NAMES = {0: "reg", 1: "smem_ldg", 2: "smem_tma"}
+STAGE_NAMES = {0: "reg", 1: "smem_ldg", 2: "smem_tma", 3: "reg_realign"}
 REDUCE_NAMES = {0: "shfl", 1: "smem", 2: "cluster"}
 DTYPE_CODES = {"bf16": RT_BF16, "fp16": RT_FP16, "fp32": RT_FP32}
 

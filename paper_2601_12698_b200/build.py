@@ -30,7 +30,7 @@ NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-std=c++17", "-O3",
               "-Xcompiler", "-fPIC", "-I", CSRC, "-I", INCLUDE]
 HOST_UNITS = ["launch.cu", "feasible.cu", "search.cu", "host_run.cu", "table.cu"]
 ELEMENT_TYPES = {"bf16": ("__nv_bfloat16", 0), "fp16": ("__half", 1), "fp32": ("float", 2)}
-GROUPS = {"reg": 0, "smem": 1, "narrow": 2, "silu": 3, "merge": 4, "fp8out": 5, "allreduce": 6}
+GROUPS = {"reg": 0, "smem": 1, "narrow": 2, "silu": 3, "merge": 4, "fp8out": 5, "allreduce": 6, "realign": 7}
 
 
 def instance_units() -> list[str]:
@@ -39,7 +39,7 @@ def instance_units() -> list[str]:
 
 
 def unit_flags(name: str) -> list[str]:
-    m = re.fullmatch(r"(bf16|fp16|fp32)_v(\d+)_(reg|smem|narrow|silu|merge|fp8out|allreduce)(?:_r(\d))?", name)
+    m = re.fullmatch(r"(bf16|fp16|fp32)_v(\d+)_(reg|smem|narrow|silu|merge|fp8out|allreduce|realign)(?:_r(\d))?", name)
     if not m:
         raise ValueError(f"cannot parse instantiation unit name {name!r}")
     ctype, code = ELEMENT_TYPES[m.group(1)]
@@ -76,7 +76,7 @@ def parse_ptxas(log: str) -> list[tuple]:
     rows = []
     for m in _ENTRY.finditer(log):
         t, vb, st, rd, u, cap, spill, regs, smem = m.groups()
-        rows.append((0, _MANGLED_DTYPE[t], int(vb), int(st), int(rd), int(u), int(cap) if int(st) == 0 else 0,
+        rows.append((0, _MANGLED_DTYPE[t], int(vb), int(st), int(rd), int(u), int(cap) if int(st) in (0, 3) else 0,
                      int(regs), int(smem), int(spill), 0))
     for block in log.split("ptxas info    : Compiling entry function")[1:]:
         for op, pattern in ((1, _SILU_ENTRY), (2, _MERGE_ENTRY)):

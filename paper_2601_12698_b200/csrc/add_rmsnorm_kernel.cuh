@@ -6,7 +6,7 @@
 // rows per CTA: run-time block shape), vectorisation (VB bytes per ld/st), unrolling (U independent
 // loads in flight), and the organisation of shared memory and registers (STAGE, REDUCE).
 //
-// Compile-time axes: element type, VB, STAGE, REDUCE, U and - for the register stage - CAP, the
+// Compile-time axes: element type, VB, STAGE, REDUCE, U and - for the two register stages - CAP, the
 // number of row vectors one thread keeps.  Run-time axes: blockDim.x = threads per row,
 // blockDim.y = rows per CTA, cluster size.
 //
@@ -16,6 +16,7 @@
 
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
+#include <stddef.h>
 #include <stdint.h>
 
 #include <type_traits>
@@ -25,6 +26,7 @@ namespace rt {
 constexpr int kStageReg = 0;
 constexpr int kStageSmemLdg = 1;
 constexpr int kStageSmemTma = 2;
+constexpr int kStageRegRealign = 3;
 constexpr int kReduceShfl = 0;
 constexpr int kReduceSmem = 1;
 constexpr int kReduceCluster = 2;
@@ -231,6 +233,59 @@ struct Codec {
     }
 };
 
+// ---- ragged rows (STAGE == kStageRegRealign) -----------------------------------------------------
+//
+// A row whose byte length is not a multiple of 16 starts at a different offset inside a 16-byte chunk from one
+// row to the next, so no vector wider than the row length's alignment divides it.  This stage cuts the row at
+// the 16-byte boundaries of the tensor instead: a head of fewer than EPV elements up to the first boundary,
+// the whole aligned chunks (moved as 16-byte vectors, kept in registers like the register stage), and a tail of
+// fewer than EPV elements.  Head and tail elements go one to a thread, so no byte outside the row is touched.
+// Only the weights are then out of step: the weights of a whole chunk start `phase` bytes past a 16-byte
+// boundary of w, the same phase for every chunk of the row.
+
+// Sixteen bytes of w from address p (a multiple of the element size, `phase` = p modulo 16 > 0): the two aligned
+// vectors around p, shifted together.  The caller guarantees that both lie inside w.
+__device__ __forceinline__ Vec<16> ld_weight_shifted(const unsigned char* p, int phase)
+{
+    const Vec<16> lo = ld_weight<16>(p - phase), hi = ld_weight<16>(p - phase + 16);
+    const uint32_t sh = (uint32_t)(phase & 3) * 8u;  // 0 or 16 bits inside a word
+    Vec<16> v;
+    switch (phase >> 2) {
+        case 0:
+            v.w[0] = __funnelshift_r(lo.w[0], lo.w[1], sh); v.w[1] = __funnelshift_r(lo.w[1], lo.w[2], sh);
+            v.w[2] = __funnelshift_r(lo.w[2], lo.w[3], sh); v.w[3] = __funnelshift_r(lo.w[3], hi.w[0], sh);
+            break;
+        case 1:
+            v.w[0] = __funnelshift_r(lo.w[1], lo.w[2], sh); v.w[1] = __funnelshift_r(lo.w[2], lo.w[3], sh);
+            v.w[2] = __funnelshift_r(lo.w[3], hi.w[0], sh); v.w[3] = __funnelshift_r(hi.w[0], hi.w[1], sh);
+            break;
+        case 2:
+            v.w[0] = __funnelshift_r(lo.w[2], lo.w[3], sh); v.w[1] = __funnelshift_r(lo.w[3], hi.w[0], sh);
+            v.w[2] = __funnelshift_r(hi.w[0], hi.w[1], sh); v.w[3] = __funnelshift_r(hi.w[1], hi.w[2], sh);
+            break;
+        default:
+            v.w[0] = __funnelshift_r(lo.w[3], hi.w[0], sh); v.w[1] = __funnelshift_r(hi.w[0], hi.w[1], sh);
+            v.w[2] = __funnelshift_r(hi.w[1], hi.w[2], sh); v.w[3] = __funnelshift_r(hi.w[2], hi.w[3], sh);
+            break;
+    }
+    return v;
+}
+
+// The same sixteen bytes element by element: for the one chunk whose second aligned vector would reach past w.
+template <typename T>
+__device__ __forceinline__ Vec<16> ld_weight_elements(const unsigned char* p)
+{
+    Vec<16> v;
+    if constexpr (sizeof(T) == 4) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) v.w[k] = ld_weight<4>(p + 4 * k).w[0];
+    } else {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) v.w[k] = ld_weight<2>(p + 4 * k).w[0] | (ld_weight<2>(p + 4 * k + 2).w[0] << 16);
+    }
+    return v;
+}
+
 // ---- synchronisation helpers --------------------------------------------------------------------
 
 // Barrier over the threads of one row only (named barrier 1 + row); a warp-wide row needs no bar.
@@ -402,7 +457,7 @@ __global__ void add_rmsnorm_kernel(const KernelArgs a)
 {
     using C = Codec<T, VB>;
     constexpr int EPV = C::EPV;
-    static_assert(STAGE != kStageReg || CAP % U == 0, "the unroll depth divides the per-thread vector count");
+    static_assert((STAGE != kStageReg && STAGE != kStageRegRealign) || CAP % U == 0, "the unroll depth divides the per-thread vector count");
     extern __shared__ __align__(128) unsigned char dyn_smem[];
 
     const int tx = threadIdx.x, ty = threadIdx.y, tpr = blockDim.x;
@@ -486,6 +541,89 @@ __global__ void add_rmsnorm_kernel(const KernelArgs a)
                 for (int e = 0; e < EPV; ++e) yf[e] = s[i][e] * rho * wf[e];
                 st_stream<VB, true>(yrow + (size_t)v * VB, C::pack(yf));
             }
+        }
+    } else if constexpr (STAGE == kStageRegRealign) {
+        static_assert(VB == 16 && REDUCE != kReduceCluster, "ragged rows: 16-byte chunks, one CTA per row");
+        constexpr int EB = (int)sizeof(T);
+        using C1 = Codec<T, EB>;  // one element
+        const bool live = row < a.n_tokens;
+        const size_t row_byte = (size_t)(live ? row : 0) * (size_t)a.hidden * EB;
+        int head = (int)((16u - (unsigned)(row_byte & 15u)) & 15u) / EB;  // elements before the first 16-byte boundary
+        if (head > a.hidden) head = a.hidden;
+        const int n_whole = live ? (a.hidden - head) / EPV : 0;            // aligned chunks wholly inside the row
+        const int tail = a.hidden - head - n_whole * EPV;                  // elements after the last of them
+        const int n_edge = live ? head + tail : 0;                         // < 2 * EPV <= 32: one thread each
+        const int edge_col = tx < head ? tx : head + n_whole * EPV + (tx - head);
+        const int phase = (head * EB) & 15;                                // address of a chunk's weights, modulo 16
+        const size_t chunk_off = row_byte + (size_t)head * EB;
+        const unsigned char* xc = reinterpret_cast<const unsigned char*>(a.x) + chunk_off;
+        const unsigned char* rc = reinterpret_cast<const unsigned char*>(a.r) + chunk_off;
+        const unsigned char* wc = reinterpret_cast<const unsigned char*>(a.w) + (size_t)head * EB;
+        unsigned char* yc = reinterpret_cast<unsigned char*>(a.y) + chunk_off;
+        unsigned char* oc = reinterpret_cast<unsigned char*>(a.r_out) + chunk_off;
+        const size_t edge_off = row_byte + (size_t)edge_col * EB;
+        // the chunk whose second aligned weight vector would end past w is read element by element
+        const int v_unsafe = (phase != 0 && tail * EB < 16 - phase) ? n_whole - 1 : -1;
+        float s[CAP][EPV];
+        float s_edge = 0.f;
+#pragma unroll
+        for (int i0 = 0; i0 < CAP; i0 += U) {
+            Vec<VB> xv[U], rv[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int v = tx + (i0 + u) * tpr;
+                if (v < n_whole) xv[u] = ld_stream<VB>(xc + (size_t)v * VB);
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int v = tx + (i0 + u) * tpr;
+                if (v < n_whole) rv[u] = ld_stream<VB>(rc + (size_t)v * VB);
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int v = tx + (i0 + u) * tpr;
+                if (v < n_whole) {
+                    float xf[EPV], rf[EPV];
+                    C::unpack(xv[u], xf);
+                    C::unpack(rv[u], rf);
+#pragma unroll
+                    for (int e = 0; e < EPV; ++e) {
+                        s[i0 + u][e] = xf[e] + rf[e];
+                        ss = fmaf(s[i0 + u][e], s[i0 + u][e], ss);
+                    }
+                    st_stream<VB, true>(oc + (size_t)v * VB, C::pack(s[i0 + u]));
+                }
+            }
+        }
+        if (tx < n_edge) {
+            float xf[1], rf[1], sf[1];
+            C1::unpack(ld_stream<EB>(reinterpret_cast<const unsigned char*>(a.x) + edge_off), xf);
+            C1::unpack(ld_stream<EB>(reinterpret_cast<const unsigned char*>(a.r) + edge_off), rf);
+            sf[0] = s_edge = xf[0] + rf[0];
+            ss = fmaf(s_edge, s_edge, ss);
+            st_stream<EB>(reinterpret_cast<unsigned char*>(a.r_out) + edge_off, C1::pack(sf));
+        }
+        const float total = row_reduce<REDUCE>(ss, tx, ty, tpr, crank, csize);
+        const float rho = __frsqrt_rn(total / (float)a.hidden + a.eps);
+#pragma unroll
+        for (int k = 0; k < CAP; ++k) {
+            const int v = tx + k * tpr;
+            if (v < n_whole) {
+                float wf[EPV], yf[EPV];
+                const unsigned char* wp = wc + (size_t)v * VB;
+                if (phase == 0) C::unpack(ld_weight<VB>(wp), wf);
+                else if (v != v_unsafe) C::unpack(ld_weight_shifted(wp, phase), wf);
+                else C::unpack(ld_weight_elements<T>(wp), wf);
+#pragma unroll
+                for (int e = 0; e < EPV; ++e) yf[e] = s[k][e] * rho * wf[e];
+                st_stream<VB, true>(yc + (size_t)v * VB, C::pack(yf));
+            }
+        }
+        if (tx < n_edge) {
+            float wf[1], yf[1];
+            C1::unpack(ld_weight<EB>(reinterpret_cast<const unsigned char*>(a.w) + (size_t)edge_col * EB), wf);
+            yf[0] = s_edge * rho * wf[0];
+            st_stream<EB>(reinterpret_cast<unsigned char*>(a.y) + edge_off, C1::pack(yf));
         }
     } else if constexpr (STAGE == kStageSmemLdg) {
         using P = SumPlanes<EPV>;

@@ -80,6 +80,22 @@ std::vector<rt_params> raw_grid(const rt_shape& s)
                             out.push_back(p);
                         }
             }
+    // Rows whose byte length is not a multiple of 16 also get the ragged-row register stage, which keeps 16-byte
+    // accesses on such rows; on aligned rows it would only repeat the register stage with extra bookkeeping.
+    if (s.op == RT_OP_ADD_RMSNORM && (s.hidden * elem_bytes_of(s.dtype)) % 16 != 0)
+        for (int tpr : kTprLevels)
+            for (int rpc : kRpcLevels)
+                for (int u : kUnrollLevels) {
+                    rt_params p;
+                    p.threads_per_row = tpr;
+                    p.rows_per_cta = rpc;
+                    p.vec_bytes = 16;
+                    p.unroll = u;
+                    p.stage = RT_STAGE_REG_REALIGN;
+                    p.reduce = RT_REDUCE_SHFL;
+                    p.cluster_size = 1;
+                    out.push_back(p);
+                }
     return out;
 }
 

@@ -1,12 +1,13 @@
 // One instantiation unit of the kernel template.  Compiled once per line of instance_units.inc with
 //   -DRT_UNIT_NAME=<name> -DRT_UNIT_T=<element type> -DRT_UNIT_DTYPE=<0|1|2> -DRT_UNIT_VB=<bytes>
-//   -DRT_UNIT_GROUP=<0 register stage | 1 shared-memory stages | 2 narrow fall-back | 3 silu_and_mul | 4 merge_attn_states | 5 fp8-output norm | 6 all-reduce-fused norm>
+//   -DRT_UNIT_GROUP=<0 register stage | 1 shared-memory stages | 2 narrow fall-back | 3 silu_and_mul | 4 merge_attn_states | 5 fp8-output norm | 6 all-reduce-fused norm | 7 ragged-row register stage>
 //   -DRT_UNIT_REDUCE=<0|1|2>   (register-stage units only)
 //
 // Instance lists.  Register stage: CAP (row vectors kept per thread) in {1,2,4,8,16,32} while the row
 // stays within 128 fp32 registers per thread, unroll U in {1,2,4} with U <= CAP.  Shared-memory
 // stages: U in {1,2,4}, all three reductions.  Narrow fall-back (4- and 2-byte vectors, for rows whose
 // byte length is not a multiple of 8): register stage, shuffle reduction, U in {1,4}.
+// Ragged-row register stage (16-byte chunks, shuffle reduction): the register stage's (CAP, U) list.
 // silu_and_mul (one unit per element type, every vector width): stages register and TMA bulk for 16- and
 // 8-byte vectors with U in {1,2,4}; register stage with U in {1,4} for the 4- and 2-byte fall-back.
 // merge_attn_states: the same instance list as silu_and_mul.
@@ -33,10 +34,11 @@ constexpr int kMaxRowRegisters = 128;
 template <int ST, int RD, int U, int CAP>
 rt::KernelEntry entry()
 {
-    if constexpr (ST == rt::kStageReg && CAP * kEPV > kMaxRowRegisters) {
+    constexpr bool kInRegisters = ST == rt::kStageReg || ST == rt::kStageRegRealign;
+    if constexpr (kInRegisters && CAP * kEPV > kMaxRowRegisters) {
         return rt::KernelEntry{RT_OP_ADD_RMSNORM, kDtype, kVB, ST, RD, U, CAP, nullptr};  // not instantiated
     } else {
-        return rt::KernelEntry{RT_OP_ADD_RMSNORM, kDtype, kVB, ST, RD, U, ST == rt::kStageReg ? CAP : 0,
+        return rt::KernelEntry{RT_OP_ADD_RMSNORM, kDtype, kVB, ST, RD, U, kInRegisters ? CAP : 0,
                                (const void*)&rt::add_rmsnorm_kernel<T, kVB, ST, RD, U, CAP>};
     }
 }
@@ -98,6 +100,10 @@ rt::KernelEntry merge_entry()
     entry<0, RD, 1, 1>(), entry<0, RD, 1, 2>(), entry<0, RD, 2, 2>(), entry<0, RD, 1, 4>(), entry<0, RD, 2, 4>(), \
     entry<0, RD, 4, 4>(), entry<0, RD, 1, 8>(), entry<0, RD, 2, 8>(), entry<0, RD, 4, 8>(), entry<0, RD, 1, 16>(), \
     entry<0, RD, 2, 16>(), entry<0, RD, 4, 16>(), entry<0, RD, 1, 32>(), entry<0, RD, 2, 32>(), entry<0, RD, 4, 32>()
+#define RT_REALIGN_LIST                                                                                   \
+    entry<3, 0, 1, 1>(), entry<3, 0, 1, 2>(), entry<3, 0, 2, 2>(), entry<3, 0, 1, 4>(), entry<3, 0, 2, 4>(), \
+    entry<3, 0, 4, 4>(), entry<3, 0, 1, 8>(), entry<3, 0, 2, 8>(), entry<3, 0, 4, 8>(), entry<3, 0, 1, 16>(), \
+    entry<3, 0, 2, 16>(), entry<3, 0, 4, 16>(), entry<3, 0, 1, 32>(), entry<3, 0, 2, 32>(), entry<3, 0, 4, 32>()
 #define RT_SMEM_LIST(ST)                                                                                   \
     entry<ST, 0, 1, 1>(), entry<ST, 0, 2, 1>(), entry<ST, 0, 4, 1>(), entry<ST, 1, 1, 1>(), entry<ST, 1, 2, 1>(), \
     entry<ST, 1, 4, 1>(), entry<ST, 2, 1, 1>(), entry<ST, 2, 2, 1>(), entry<ST, 2, 4, 1>()
@@ -118,6 +124,8 @@ std::vector<rt::KernelEntry> build_entries()
         fp8_entry<0, 2, 16>(), fp8_entry<0, 4, 16>(), fp8_entry<2, 1, 1>(), fp8_entry<2, 2, 1>(), fp8_entry<2, 4, 1>()
 #elif RT_UNIT_GROUP == 6
         RT_ALLREDUCE_LIST(2), RT_ALLREDUCE_LIST(4), RT_ALLREDUCE_LIST(8)
+#elif RT_UNIT_GROUP == 7
+        RT_REALIGN_LIST
 #elif RT_UNIT_GROUP == 4
         RT_MERGE_WIDE(16), RT_MERGE_WIDE(8), merge_entry<4, 0, 1>(), merge_entry<4, 0, 4>(), merge_entry<2, 0, 1>(),
         merge_entry<2, 0, 4>()

@@ -316,8 +316,15 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
         plan->reject_reason = kRejectArgs;
         return RT_ERR_INFEASIBLE;
     }
-    if (p->stage < 0 || p->stage > 2 || p->reduce < 0 || p->reduce > 2) {
+    if (p->stage < 0 || p->stage > RT_STAGE_REG_REALIGN || p->reduce < 0 || p->reduce > 2) {
         set_error("stage=%d or reduce=%d unknown", p->stage, p->reduce);
+        plan->reject_reason = kRejectArgs;
+        return RT_ERR_INFEASIBLE;
+    }
+    const bool realign = p->stage == RT_STAGE_REG_REALIGN;
+    if (realign && (s->op != RT_OP_ADD_RMSNORM || p->vec_bytes != 16 || p->reduce != RT_REDUCE_SHFL || p->cluster_size != 1)) {
+        set_error("the ragged-row stage belongs to add_rmsnorm and takes 16-byte chunks and the shuffle reduction "
+                  "(op=%d vec=%d reduce=%d cluster=%d)", s->op, p->vec_bytes, p->reduce, p->cluster_size);
         plan->reject_reason = kRejectArgs;
         return RT_ERR_INFEASIBLE;
     }
@@ -364,7 +371,7 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
         return RT_ERR_INFEASIBLE;
     }
     const int64_t row_bytes = s->hidden * eb;
-    if (row_bytes % vb != 0) {
+    if (row_bytes % vb != 0 && !realign) {  // the ragged-row stage covers a row of any length with aligned chunks
         set_error("row of %lld bytes is not a multiple of vec_bytes=%d", (long long)row_bytes, vb);
         plan->reject_reason = kRejectAlign;
         return RT_ERR_ALIGN;
@@ -388,7 +395,8 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
     }
 
     plan->elem_bytes = eb;
-    plan->nvec = (int)(row_bytes / vb);
+    // ragged rows: the most whole 16-byte chunks a row can hold (its head and tail elements go one to a thread)
+    plan->nvec = realign ? (int)std::max<int64_t>(1, row_bytes / 16) : (int)(row_bytes / vb);
     int slice = (plan->nvec + C - 1) / C;
     const int gran = vb < 16 ? 16 / vb : 1;  // slices start on 16-byte boundaries
     slice = (slice + gran - 1) / gran * gran;
@@ -408,7 +416,8 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
     }
 
     int cap = 0, unroll = p->unroll;
-    if (p->stage == RT_STAGE_REG && !no_reduction) {
+    const bool row_in_registers = (p->stage == RT_STAGE_REG || realign) && !no_reduction;
+    if (row_in_registers) {
         cap = next_pow2(plan->vec_per_thread);
         if (unroll > cap) unroll = cap;
     }
@@ -416,13 +425,13 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
     plan->unroll_eff = unroll;
     plan->kernel_index = find_kernel(s->op, s->dtype, vb, p->stage, p->reduce, unroll, cap, is_allreduce ? s->n_parts : 0);
     if (plan->kernel_index < 0) {
-        if (p->stage == RT_STAGE_REG && !no_reduction)
+        if (row_in_registers)
             set_error("a row slice of %d vectors over %d threads needs %d vectors per thread: no register-stage "
                       "instance that large (register budget)", slice, tpr, cap);
         else
             set_error("no compiled instance for dtype=%d vec=%d stage=%d reduce=%d unroll=%d", s->dtype, vb, p->stage,
                       p->reduce, unroll);
-        plan->reject_reason = (p->stage == RT_STAGE_REG && !no_reduction) ? kRejectRegisters : kRejectArgs;
+        plan->reject_reason = row_in_registers ? kRejectRegisters : kRejectArgs;
         return RT_ERR_INFEASIBLE;
     }
     const KernelEntry& k = registry()[plan->kernel_index];

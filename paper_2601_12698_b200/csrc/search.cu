@@ -715,9 +715,18 @@ struct SearchState {
         step(kRpc, 4, &rt_params::rows_per_cta);
         step(kUnr, 3, &rt_params::unroll);
         step(kVec, 4, &rt_params::vec_bytes);
-        for (int stage = 0; stage < 3; ++stage) {
+        // another stage at the same vector width; where that stage has no such point (the ragged-row stage is
+        // all 16-byte chunks while the other stages of a misaligned shape are narrower), at its widest width
+        for (int stage = 0; stage <= RT_STAGE_REG_REALIGN; ++stage) {
             rt_params q = p;
             q.stage = stage;
+            if (index.find(pack_params(q)) == index.end()) {
+                if (stage == RT_STAGE_REG_REALIGN) q.reduce = RT_REDUCE_SHFL, q.cluster_size = 1;
+                for (int k = 3; k >= 0; --k) {
+                    q.vec_bytes = kVec[k];
+                    if (index.find(pack_params(q)) != index.end()) break;
+                }
+            }
             probe(q);
         }
         for (int reduce = 0; reduce < 3; ++reduce)
@@ -733,7 +742,7 @@ struct SearchState {
 };
 
 // The coarse grid: every other level of the ordered axes (threads per row 64/256/1024, rows per CTA
-// 1/4, unroll 1/4), the widest vector, every stage and reduction mode.
+// 1/4, unroll 1/4), the widest vector of the point's stage, every stage and reduction mode.
 bool on_coarse_grid(const rt_params& p, int widest_vec)
 {
     const int lt = level_of(kTpr, 6, p.threads_per_row), lr = level_of(kRpc, 4, p.rows_per_cta),
@@ -819,11 +828,11 @@ int run_search(const rt_shape& shape, const rt_limits& limits, const rt_budget& 
             S.time_us[idx] = t;
         }
         // 2. coarse grid, cut to half of what is left of the budget (mode by mode, nearest the middle first)
-        int widest = 0;
-        for (const rt_params& p : feasible) widest = std::max(widest, p.vec_bytes);
+        int widest[RT_STAGE_REG_REALIGN + 1] = {0, 0, 0, 0};  // per stage: the ragged-row stage is wider than the others
+        for (const rt_params& p : feasible) widest[p.stage] = std::max(widest[p.stage], p.vec_bytes);
         std::vector<int> coarse;
         for (int i = 0; i < (int)feasible.size(); ++i)
-            if (on_coarse_grid(S.cand[i], widest)) coarse.push_back(i);
+            if (on_coarse_grid(S.cand[i], widest[S.cand[i].stage])) coarse.push_back(i);
         if (coarse.empty())
             for (int i = 0; i < (int)feasible.size(); ++i) coarse.push_back(i);
         const int grid_budget = std::max(1, (S.max_evals - top_k - S.used) / 2);

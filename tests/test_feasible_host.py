@@ -26,7 +26,10 @@ def test_every_emitted_theta_passes_the_hard_rules_and_counts_add_up(L, T, H, dt
     for th in feasible:
         assert B.tuner_check_params(s, th, L) == B.RT_OK
         assert th.threads_per_row * th.rows_per_cta <= 1024
-        assert (H * (4 if dtype == "fp32" else 2)) % th.vec_bytes == 0
+        if th.stage == B.RT_STAGE_REG_REALIGN:  # aligned 16-byte chunks over rows of any length
+            assert th.vec_bytes == 16 and th.reduce == B.RT_REDUCE_SHFL and (H * (4 if dtype == "fp32" else 2)) % 16 != 0
+        else:
+            assert (H * (4 if dtype == "fp32" else 2)) % th.vec_bytes == 0
         assert (th.reduce == B.RT_REDUCE_CLUSTER) == (th.cluster_size > 1)
     c = B.tuner_derive_counts(s, L)
     assert c["feasible"] == len(feasible)
@@ -44,18 +47,41 @@ def test_heuristics_only_remove_points(L):
 
 
 def test_rules_bite_where_they_should(L):
-    # 6148 fp16: row bytes = 8 mod 16 -> only 8-byte vectors, no TMA stage
+    ragged = B.RT_STAGE_REG_REALIGN
+
+    def row_vectors(f):  # the stages whose vectors must divide the row
+        return [t for t in f if t.stage != ragged]
+
+    # 6148 fp16: row bytes = 8 mod 16 -> only 8-byte row vectors, no TMA stage; the ragged-row stage keeps 16-byte chunks
     f = B.tuner_derive_feasible(B.shape_of(8192, 6148, "fp16"), L)
-    assert {t.vec_bytes for t in f} == {8} and B.RT_STAGE_SMEM_TMA not in {t.stage for t in f}
-    # 6152 fp16: 769 16-byte vectors, both widths, all stages
+    assert {t.vec_bytes for t in row_vectors(f)} == {8} and {t.stage for t in f} == {0, 1, ragged}
+    assert {t.vec_bytes for t in f if t.stage == ragged} == {16}
+    # 6152 fp16: 769 16-byte vectors, both widths, the three aligned stages and no ragged-row stage
     f = B.tuner_derive_feasible(B.shape_of(8192, 6152, "fp16"), L)
     assert {t.vec_bytes for t in f} == {8, 16} and {t.stage for t in f} == {0, 1, 2}
-    # rows that fit no 8-byte vector fall back to the widest narrow width
-    assert {t.vec_bytes for t in B.tuner_derive_feasible(B.shape_of(64, 6146, "fp16"), L)} == {4}
-    assert {t.vec_bytes for t in B.tuner_derive_feasible(B.shape_of(64, 6145, "fp16"), L)} == {2}
-    # pointers that are only 8-byte aligned remove the 16-byte vectors and TMA
+    # rows that fit no 8-byte vector fall back to the widest narrow width, or take the ragged-row stage
+    for hidden, narrow in ((6146, 4), (6145, 2)):
+        f = B.tuner_derive_feasible(B.shape_of(64, hidden, "fp16"), L)
+        assert {t.vec_bytes for t in row_vectors(f)} == {narrow} and {t.stage for t in row_vectors(f)} == {0}
+        assert any(t.stage == ragged for t in f)
+    # pointers that are only 8-byte aligned remove the 16-byte vectors, TMA and the ragged-row stage
     f = B.tuner_derive_feasible(B.shape_of(128, 4096, "bf16", min_ptr_align=8), L)
-    assert {t.vec_bytes for t in f} == {8} and B.RT_STAGE_SMEM_TMA not in {t.stage for t in f}
+    assert {t.vec_bytes for t in f} == {8} and not {B.RT_STAGE_SMEM_TMA, ragged} & {t.stage for t in f}
+    f = B.tuner_derive_feasible(B.shape_of(128, 4100, "bf16", min_ptr_align=8), L)
+    assert f and {t.vec_bytes for t in f} == {8} and ragged not in {t.stage for t in f}
+    # the ragged-row stage: add_rmsnorm only, 16-byte chunks, shuffle reduction, one CTA per row; it also runs on
+    # aligned rows (where the deriver does not offer it)
+    s_odd = B.shape_of(64, 6145, "fp16")
+    assert B.tuner_check_params(s_odd, B.make_params(stage=ragged), L) == B.RT_OK
+    assert B.tuner_check_params(s_odd, B.make_params(stage=ragged, vec_bytes=8), L) == B.RT_ERR_INFEASIBLE
+    assert B.tuner_check_params(s_odd, B.make_params(stage=ragged, reduce=B.RT_REDUCE_SMEM), L) == B.RT_ERR_INFEASIBLE
+    assert B.tuner_check_params(s_odd, B.make_params(stage=ragged, reduce=B.RT_REDUCE_CLUSTER, cluster_size=2), L) == B.RT_ERR_INFEASIBLE
+    assert B.tuner_check_params(s_odd, B.make_params(stage=4), L) == B.RT_ERR_INFEASIBLE
+    assert B.tuner_check_params(B.shape_of(64, 6145, "fp16", min_ptr_align=8), B.make_params(stage=ragged), L) == B.RT_ERR_ALIGN
+    assert B.tuner_check_params(B.shape_of(128, 4096, "bf16"), B.make_params(stage=ragged), L) == B.RT_OK
+    assert B.tuner_check_params(B.shape_of(64, 6145, "fp16", op=B.RT_OP_SILU_AND_MUL), B.make_params(stage=ragged), L) == B.RT_ERR_INFEASIBLE
+    # a 32-thread row of fp32 12289 would keep 96 chunks per thread: no instance that large
+    assert B.tuner_check_params(B.shape_of(64, 12289, "fp32"), B.make_params(threads_per_row=32, stage=ragged), L) == B.RT_ERR_INFEASIBLE
     # a single token: one row per CTA only; clusters are allowed (too few rows to fill the SMs)
     f = B.tuner_derive_feasible(B.shape_of(1, 4096, "bf16"), L)
     assert {t.rows_per_cta for t in f} == {1} and 8 in {t.cluster_size for t in f}

@@ -80,6 +80,49 @@ def test_every_feasible_theta_matches_oracle(B, oracle_lib, dtype, T, H):
     assert not failures, f"{len(failures)} of {n_run} configurations differ: {failures[:5]}"
 
 
+RAGGED_SHAPES = [(1, 1), (9, 1), (5, 3), (9, 7), (4, 9), (7, 33), (5, 1001), (3, 4097), (5, 6145), (4, 6146), (3, 6148),
+                 (2, 12289), (5, 4096)]
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp16", "fp32"])
+@pytest.mark.parametrize("T,H", RAGGED_SHAPES)
+def test_ragged_row_stage_matches_oracle(B, oracle_lib, dtype, T, H):
+    """Rows of any byte length through the aligned-chunk stage: every block shape and unroll depth that passes the
+    hard rules, written between canaries (the end chunks of a row are shared with its neighbours, or reach past
+    the tensor), then in place."""
+    synth = _synth()
+    x, r, w = synth.make_inputs(T, H, dtype, seed=300 + H % 89)
+    y_ref, r_ref = oracle_lib.add_rmsnorm(x, r, w, EPS)
+    xd, rd, wd = x.cuda(), r.cuda(), w.cuda()
+    y_ref_d, r_ref_d = y_ref.cuda(), r_ref.cuda()
+    y, _, y_ok = _padded((T, H), TD[dtype])
+    ro, _, ro_ok = _padded((T, H), TD[dtype])
+    shape = B.shape_of(T, H, dtype, B._ptr_align(xd, rd, wd, y, ro))
+    thetas = [B.make_params(threads_per_row=tpr, rows_per_cta=rpc, unroll=u, stage=B.RT_STAGE_REG_REALIGN)
+              for tpr in (32, 64, 128, 256, 512, 1024) for rpc in (1, 2, 4, 8) for u in (1, 2, 4)]
+    thetas = [th for th in thetas if B.tuner_check_params(shape, th) == B.RT_OK]
+    assert thetas
+    if (H * (4 if dtype == "fp32" else 2)) % 16 != 0:  # the deriver offers the stage exactly on such rows
+        offered = {t.key() for t in B.tuner_derive_feasible(shape, heuristics=0) if t.stage == B.RT_STAGE_REG_REALIGN}
+        assert offered == {t.key() for t in thetas}
+    failures = []
+    for th in thetas:
+        y.fill_(float("nan")); ro.fill_(float("nan"))
+        B.rmsnorm_template_launch(th, xd, rd, wd, y, ro, EPS)
+        r_bad, y_bad, worst = _gate(B, oracle_lib, y, ro, y_ref_d, r_ref_d, dtype)
+        if r_bad or y_bad:
+            failures.append((repr(th), r_bad, y_bad, worst))
+    assert B.rt_device_status() == 0
+    assert y_ok() and ro_ok(), "a kernel wrote outside its output"
+    assert not failures, f"{len(failures)} of {len(thetas)} configurations differ: {failures[:5]}"
+    # in place: y over x and r_out over r, neighbours' rows untouched where a chunk is shared
+    for th in thetas[::5]:
+        x2, r2 = x.cuda(), r.cuda()
+        B.rmsnorm_template_launch(th, x2, r2, wd, x2, r2, EPS)
+        r_bad, y_bad, _ = _gate(B, oracle_lib, x2, r2, y_ref_d, r_ref_d, dtype)
+        assert (r_bad, y_bad) == (0, 0), repr(th)
+
+
 @pytest.mark.parametrize("dtype", ["bf16", "fp16", "fp32"])
 def test_device_comparator_agrees_with_oracle_comparator(B, oracle_lib, dtype):
     """The gate's own metric is checked against the oracle's comparison routine on perturbed data."""
@@ -191,7 +234,7 @@ def test_narrow_fallback_for_rows_that_fit_no_wide_vector(B, oracle_lib):
         y_ref, r_ref = oracle_lib.add_rmsnorm(x, r, w, EPS)
         xd, rd, wd = x.cuda(), r.cuda(), w.cuda()
         shape = B.shape_of(9, H, "fp16")
-        thetas = B.tuner_derive_feasible(shape)
+        thetas = [t for t in B.tuner_derive_feasible(shape) if t.stage != B.RT_STAGE_REG_REALIGN]  # the row-vector stages
         assert thetas and all(t.vec_bytes == want_vec for t in thetas)
         for th in thetas:
             y, ro = torch.empty_like(xd), torch.empty_like(xd)
