@@ -103,6 +103,9 @@ def workloads() -> dict[str, Workload]:
     for h in (5120, 7168, 6152):
         add(Workload(f"c4_fp16_8192x{h}", "fp16", 8192, h, seed=3))
     add(Workload("c4x_fp16_8192x6148", "fp16", 8192, 6148, seed=3))
+    # rows that are only 4- and 2-byte multiples: no 8-byte vector divides them (narrow fall-back or the ragged-row stage)
+    add(Workload("c4x_fp16_8192x6146", "fp16", 8192, 6146, seed=3))
+    add(Workload("c4x_fp16_8192x6145", "fp16", 8192, 6145, seed=3))
     add(Workload("c5_fp32_32768x12288", "fp32", 32768, 12288, seed=4))
     # silu_and_mul: a bandwidth case (LLaMA-3-8B MLP width), and the paper's fp32 (m, n) shapes with n = d
     gate = Dist(sigma=2.5)
