@@ -49,19 +49,22 @@ NOMINAL_HBM_GBS = 8000.0
 # DRAM traffic of one launch of the top kernel from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum), valid only for the kernel source and theta it was taken on.
 NCU_TRAFFIC = {
-    "kernel_sha256_16": "a5caaa4fd7831901",
-    "workload": "c3_prefill_bf16_16384x8192",
-    # (threads_per_row, rows_per_cta, vec_bytes, unroll, stage, reduce, cluster_size) -> DRAM bytes per launch
+    "kernel_sha256_16": "a1a203764915b554",
+    # workload -> (threads_per_row, rows_per_cta, vec_bytes, unroll, stage, reduce, cluster_size) -> DRAM bytes per launch
     "bytes_per_launch": {
-        (256, 1, 16, 1, 2, 0, 1): 1021228032,  # 536.93 MB read + 484.30 MB written
-        (256, 1, 16, 4, 0, 0, 1): 1020643840,  # 536.92 MB read + 483.72 MB written
-        # the other configurations the search has returned on this shape (dram__bytes metrics only, first of two launches)
-        (256, 1, 16, 2, 0, 0, 1): 1020540928,
-        (256, 1, 16, 2, 2, 0, 1): 1020514048,
-        (256, 1, 16, 4, 2, 0, 1): 1022055424,
-        (512, 1, 16, 1, 2, 0, 1): 1021512704,
-        (512, 1, 16, 2, 0, 0, 1): 1019790592,
-        (512, 1, 16, 4, 0, 0, 1): 1019570944,
+        "c3_prefill_bf16_16384x8192": {
+            (256, 1, 16, 1, 2, 0, 1): 1020595456,  # 536.90 MB read + 483.69 MB written
+            (256, 1, 16, 4, 0, 0, 1): 1019879168,  # 536.90 MB read + 482.98 MB written
+            # the other configurations the search has returned on this shape (dram__bytes metrics only, first of two launches)
+            (256, 1, 16, 2, 0, 0, 1): 1020492288,
+            (256, 1, 16, 2, 2, 0, 1): 1020761088,
+            (256, 1, 16, 4, 2, 0, 1): 1020097024,
+            (512, 1, 16, 1, 2, 0, 1): 1020931328,
+            (512, 1, 16, 2, 0, 0, 1): 1019459072,
+            (512, 1, 16, 4, 0, 0, 1): 1019613952,
+        },
+        # the ragged-row stage; 201.41 MB read + 150.33 MB written (a quarter of the output is still dirty in L2 at the end)
+        "c4x_fp16_8192x6145": {(256, 1, 16, 4, 3, 0, 1): 351735040},
     },
 }
 
@@ -578,8 +581,8 @@ def run_ours(args) -> None:
         per_launch_ms = ms_local / args.steps
         achieved = wl.algorithmic_bytes / (per_launch_ms * 1e-3) / 1e9
         traffic = None
-        if NCU_TRAFFIC["kernel_sha256_16"] == kernel_source_hash() and NCU_TRAFFIC["workload"] == wl.name:
-            traffic = NCU_TRAFFIC["bytes_per_launch"].get(tuple(theta_dict(theta).values()))
+        if NCU_TRAFFIC["kernel_sha256_16"] == kernel_source_hash():
+            traffic = NCU_TRAFFIC["bytes_per_launch"].get(wl.name, {}).get(tuple(theta_dict(theta).values()))
         line = {
             "metric": METRICS[wl.op], "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",

@@ -30,6 +30,9 @@ int table_lookup(const rt_spec_entry* table, int32_t n, const rt_params* general
     for (int32_t i = 0; i < n; ++i) {
         const rt_spec_entry& e = table[i];
         if (e.shape.dtype != query->dtype || e.shape.op != query->op) continue;
+        // the ragged-row stage runs on any row length, but on 16-byte rows it is the register stage plus
+        // bookkeeping: an entry tuned on a misaligned shape is not a neighbour of an aligned one
+        if (e.best.stage == RT_STAGE_REG_REALIGN && (query->hidden * elem_bytes_of(query->dtype)) % 16 == 0) continue;
         const double d = shape_distance(e.shape, *query);
         if (best >= 0 && d >= best_d) continue;
         Plan plan;
@@ -50,7 +53,7 @@ int table_lookup(const rt_spec_entry* table, int32_t n, const rt_params* general
             return RT_OK;
         }
     }
-    // Last resort: the first point of the feasible set (registers, shuffle, widest vector that fits).
+    // Last resort: a point of the feasible set (registers, shuffle, widest vector that fits).
     std::vector<rt_params> feasible;
     int st = derive_feasible(*query, *limits, RT_PRUNE_DEFAULT, &feasible, nullptr);
     if (st != RT_OK) return st;
@@ -59,6 +62,20 @@ int table_lookup(const rt_spec_entry* table, int32_t n, const rt_params* general
         return RT_ERR_INFEASIBLE;
     }
     *out = feasible[0];
+    // rows that are not 16-byte multiples: the ragged-row stage near 256 threads per row, one row per CTA, deepest
+    // unroll is what the searches return on such shapes, and is far ahead of the narrow row vectors
+    int best_rank = -1;
+    for (const rt_params& p : feasible) {
+        if (p.stage != RT_STAGE_REG_REALIGN) continue;
+        int away = 0;
+        for (int t = p.threads_per_row; t < 256; t <<= 1) ++away;
+        for (int t = p.threads_per_row; t > 256; t >>= 1) ++away;
+        const int rank = 100 - 10 * away - 4 * (p.rows_per_cta - 1) + p.unroll;
+        if (rank > best_rank) {
+            best_rank = rank;
+            *out = p;
+        }
+    }
     if (source) *source = RT_FROM_FEASIBLE_SET;
     return RT_OK;
 }

@@ -84,9 +84,23 @@ def test_table_lookup_prefers_exact_then_nearest_then_general():
                       B.make_params(vec_bytes=8, threads_per_row=512))
     theta, src = t16.lookup(B.shape_of(8192, 6148, "fp16"), L)
     assert (theta.vec_bytes, src) == (8, "general")
-    # nothing usable at all: the first point of the feasible set
+    # nothing usable at all: a point of the feasible set - on rows that are not 16-byte multiples the ragged-row stage
     theta, src = B.SpecTable([], None).lookup(B.shape_of(64, 6146, "fp16"), L)
-    assert src == "feasible_set" and theta.vec_bytes == 4
+    assert src == "feasible_set" and (theta.stage, theta.vec_bytes, theta.threads_per_row, theta.rows_per_cta) == \
+        (B.RT_STAGE_REG_REALIGN, 16, 256, 1)
+    theta, src = B.SpecTable([], None).lookup(B.shape_of(64, 6146, "fp16", min_ptr_align=4), L)  # pointers rule it out
+    assert src == "feasible_set" and (theta.stage, theta.vec_bytes) == (B.RT_STAGE_REG, 4)
+    theta, src = B.SpecTable([], None).lookup(B.shape_of(64, 4096, "fp16"), L)
+    assert src == "feasible_set" and theta.stage == B.RT_STAGE_REG and theta.vec_bytes == 16
+    # an entry tuned on ragged rows serves other ragged rows of its dtype, never rows that are 16-byte multiples
+    ragged = B.make_params(unroll=4, stage=B.RT_STAGE_REG_REALIGN)
+    tr = B.SpecTable([(B.shape_of(8192, 6145, "fp16"), ragged, 65.0), (B.shape_of(8192, 5120, "fp16"), th_fp32, 51.0)], general)
+    theta, src = tr.lookup(B.shape_of(4096, 6146, "fp16"), L)
+    assert (theta.key(), src) == (ragged.key(), "table_nearest")
+    theta, src = tr.lookup(B.shape_of(8192, 5121, "fp16"), L)  # the aligned neighbour's theta cannot run here
+    assert (theta.key(), src) == (ragged.key(), "table_nearest")
+    theta, src = tr.lookup(B.shape_of(8192, 6144, "fp16"), L)  # 6145 is nearer, but its theta is for ragged rows
+    assert (theta.key(), src) == (th_fp32.key(), "table_nearest")
     # JSON round trip
     again = B.SpecTable.from_json(table.to_json())
     assert [(s.n_tokens, s.hidden, s.dtype, t.key()) for s, t, _ in again.entries] == \
@@ -104,4 +118,6 @@ def test_shipped_table_loads_and_every_entry_is_feasible_for_its_shape():
         assert got.key() == theta.key() and source == "table_exact"
     # every kernel has a general configuration, and it runs on every shape of its kernel in the table
     assert set(table.generals) == {0, 1, 2, 3, 4}
-    assert all(B.tuner_check_params(s, table.generals[int(s.op)], L) == B.RT_OK for s, _, _ in table.entries)
+    # (rows that are not 16-byte multiples are served by their own entries: the general 16-byte vectors do not divide them)
+    assert all(B.tuner_check_params(s, table.generals[int(s.op)], L) == B.RT_OK for s, _, _ in table.entries
+               if (s.hidden * (4 if s.dtype == B.RT_FP32 else 2)) % 16 == 0)
