@@ -243,13 +243,35 @@ struct Codec {
 // Only the weights are then out of step: the weights of a whole chunk start `phase` bytes past a 16-byte
 // boundary of w, the same phase for every chunk of the row.
 
-// Sixteen bytes of w from address p (a multiple of the element size, `phase` = p modulo 16 > 0): the two aligned
-// vectors around p, shifted together.  The caller guarantees that both lie inside w.
-__device__ __forceinline__ Vec<16> ld_weight_shifted(const unsigned char* p, int phase)
+template <int VB, bool EARLY>
+__device__ __forceinline__ Vec<VB> ld_weight_at(const void* p)
 {
-    const Vec<16> lo = ld_weight<16>(p - phase), hi = ld_weight<16>(p - phase + 16);
-    const uint32_t sh = (uint32_t)(phase & 3) * 8u;  // 0 or 16 bits inside a word
+    if constexpr (EARLY) return ld_weight_early<VB>(p);
+    else return ld_weight<VB>(p);
+}
+
+// Sixteen bytes of w from address p (a multiple of the element size; `phase` = p modulo 16, the same for every
+// chunk of a row).  phase = 0: one aligned vector.  Otherwise the two aligned vectors around p, shifted together
+// (`whole_pair`: both lie inside w), or - for the one chunk per row whose second vector would reach past the end of
+// w - element by element.  EARLY pins the loads in program order, for a fetch ahead of the row reduction.
+template <typename T, bool EARLY>
+__device__ __forceinline__ Vec<16> ld_weight_ragged(const unsigned char* p, int phase, bool whole_pair)
+{
+    if (phase == 0) return ld_weight_at<16, EARLY>(p);
     Vec<16> v;
+    if (!whole_pair) {
+        if constexpr (sizeof(T) == 4) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) v.w[k] = ld_weight_at<4, EARLY>(p + 4 * k).w[0];
+        } else {
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                v.w[k] = ld_weight_at<2, EARLY>(p + 4 * k).w[0] | (ld_weight_at<2, EARLY>(p + 4 * k + 2).w[0] << 16);
+        }
+        return v;
+    }
+    const Vec<16> lo = ld_weight_at<16, EARLY>(p - phase), hi = ld_weight_at<16, EARLY>(p - phase + 16);
+    const uint32_t sh = (uint32_t)(phase & 3) * 8u;  // 0 or 16 bits inside a word
     switch (phase >> 2) {
         case 0:
             v.w[0] = __funnelshift_r(lo.w[0], lo.w[1], sh); v.w[1] = __funnelshift_r(lo.w[1], lo.w[2], sh);
@@ -267,21 +289,6 @@ __device__ __forceinline__ Vec<16> ld_weight_shifted(const unsigned char* p, int
             v.w[0] = __funnelshift_r(lo.w[3], hi.w[0], sh); v.w[1] = __funnelshift_r(hi.w[0], hi.w[1], sh);
             v.w[2] = __funnelshift_r(hi.w[1], hi.w[2], sh); v.w[3] = __funnelshift_r(hi.w[2], hi.w[3], sh);
             break;
-    }
-    return v;
-}
-
-// The same sixteen bytes element by element: for the one chunk whose second aligned vector would reach past w.
-template <typename T>
-__device__ __forceinline__ Vec<16> ld_weight_elements(const unsigned char* p)
-{
-    Vec<16> v;
-    if constexpr (sizeof(T) == 4) {
-#pragma unroll
-        for (int k = 0; k < 4; ++k) v.w[k] = ld_weight<4>(p + 4 * k).w[0];
-    } else {
-#pragma unroll
-        for (int k = 0; k < 4; ++k) v.w[k] = ld_weight<2>(p + 4 * k).w[0] | (ld_weight<2>(p + 4 * k + 2).w[0] << 16);
     }
     return v;
 }
@@ -603,6 +610,19 @@ __global__ void add_rmsnorm_kernel(const KernelArgs a)
             ss = fmaf(s_edge, s_edge, ss);
             st_stream<EB>(reinterpret_cast<unsigned char*>(a.r_out) + edge_off, C1::pack(sf));
         }
+        // As in the register stage, a thread that owns at most two chunks fetches its weights ahead of the
+        // reduction; the one weight of a head or tail element always is.
+        constexpr bool kEarlyWeight = CAP <= 2;
+        Vec<VB> wv[kEarlyWeight ? CAP : 1];
+        Vec<EB> w_edge;
+        if constexpr (kEarlyWeight) {
+#pragma unroll
+            for (int k = 0; k < CAP; ++k) {
+                const int v = tx + k * tpr;
+                if (v < n_whole) wv[k] = ld_weight_ragged<T, true>(wc + (size_t)v * VB, phase, v != v_unsafe);
+            }
+        }
+        if (tx < n_edge) w_edge = ld_weight_early<EB>(reinterpret_cast<const unsigned char*>(a.w) + (size_t)edge_col * EB);
         const float total = row_reduce<REDUCE>(ss, tx, ty, tpr, crank, csize);
         const float rho = __frsqrt_rn(total / (float)a.hidden + a.eps);
 #pragma unroll
@@ -610,10 +630,8 @@ __global__ void add_rmsnorm_kernel(const KernelArgs a)
             const int v = tx + k * tpr;
             if (v < n_whole) {
                 float wf[EPV], yf[EPV];
-                const unsigned char* wp = wc + (size_t)v * VB;
-                if (phase == 0) C::unpack(ld_weight<VB>(wp), wf);
-                else if (v != v_unsafe) C::unpack(ld_weight_shifted(wp, phase), wf);
-                else C::unpack(ld_weight_elements<T>(wp), wf);
+                if constexpr (kEarlyWeight) C::unpack(wv[k], wf);
+                else C::unpack(ld_weight_ragged<T, false>(wc + (size_t)v * VB, phase, v != v_unsafe), wf);
 #pragma unroll
                 for (int e = 0; e < EPV; ++e) yf[e] = s[k][e] * rho * wf[e];
                 st_stream<VB, true>(yc + (size_t)v * VB, C::pack(yf));
@@ -621,7 +639,7 @@ __global__ void add_rmsnorm_kernel(const KernelArgs a)
         }
         if (tx < n_edge) {
             float wf[1], yf[1];
-            C1::unpack(ld_weight<EB>(reinterpret_cast<const unsigned char*>(a.w) + (size_t)edge_col * EB), wf);
+            C1::unpack(w_edge, wf);
             yf[0] = s_edge * rho * wf[0];
             st_stream<EB>(reinterpret_cast<unsigned char*>(a.y) + edge_off, C1::pack(yf));
         }
