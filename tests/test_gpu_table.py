@@ -89,3 +89,26 @@ def test_tuning_and_auto_launch_for_the_other_kernels(B, oracle_lib):
     q_ref, sc_ref, r_ref = oracle_lib.add_rmsnorm_fp8(xx, rr, ww, EPS)
     assert oracle_lib.compare_e4m3(q.cpu(), q_ref)[1] == 0 and oracle_lib.compare_y(sc.cpu(), sc_ref)[1] == 0
     assert oracle_lib.bit_mismatches(ro.cpu(), r_ref) == 0
+
+
+@pytest.mark.parametrize("dtype,T,H,want_stage", [
+    ("fp16", 100, 6145, 3), ("fp16", 8192, 6146, 3), ("bf16", 7, 4099, 3), ("fp32", 50, 4097, 3), ("bf16", 33, 1001, 3),
+    ("fp16", 100, 6144, None), ("bf16", 16, 4096, None)])
+def test_shipped_table_serves_ragged_rows_with_the_ragged_row_stage(B, oracle_lib, dtype, T, H, want_stage):
+    """The table shipped with the package: rows that are not 16-byte multiples get an entry tuned on such rows (the
+    ragged-row stage), rows that are never do; either way the launch matches the oracle."""
+    from paper_2601_12698_b200 import synth
+    table = B.SpecTable.default()
+    x, r, w = synth.make_inputs(T, H, dtype, seed=47)
+    y_ref, r_ref = oracle_lib.add_rmsnorm(x, r, w, EPS)
+    xd, rd, wd = x.cuda(), r.cuda(), w.cuda()
+    y, ro = torch.empty_like(xd), torch.empty_like(xd)
+    used = table.launch(xd, rd, wd, y, ro, EPS)
+    torch.cuda.synchronize()
+    assert oracle_lib.bit_mismatches(ro.cpu(), r_ref) == 0, repr(used)
+    assert oracle_lib.compare_y(y.cpu(), y_ref)[1] == 0, repr(used)
+    if want_stage is None:
+        assert used.stage != B.RT_STAGE_REG_REALIGN
+    else:
+        assert used.stage == want_stage and used.vec_bytes == 16
+    assert B.rt_device_status() == 0
