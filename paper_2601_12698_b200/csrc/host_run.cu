@@ -28,9 +28,11 @@ int64_t pick_chunk(int64_t n_tokens, int64_t hidden, int dtype, int64_t chunk_to
 {
     if (n_tokens <= 0) return 1;
     if (chunk_tokens <= 0) {
-        // about 32 MB per tensor per chunk: large enough for full copy bandwidth, small enough to overlap
+        // about 16 MB per tensor per chunk: measured on B200 over PCIe Gen5 x16 (bf16 16384 x 8192, both
+        // directions busy), 8-16 MB chunks give the shortest step; 32 MB loses 5% to the pipeline's fill and
+        // drain, 2 MB and below lose more to per-copy overhead
         const int64_t row_bytes = hidden * elem_bytes_of(dtype);
-        chunk_tokens = std::max<int64_t>(1, (32LL << 20) / std::max<int64_t>(1, row_bytes));
+        chunk_tokens = std::max<int64_t>(1, (16LL << 20) / std::max<int64_t>(1, row_bytes));
     }
     return std::min(chunk_tokens, n_tokens);
 }
