@@ -84,7 +84,8 @@ typedef enum {
 typedef struct {
     int32_t threads_per_row; /* threads cooperating on one row (blockDim.x); power of two, 32..1024 */
     int32_t rows_per_cta;    /* rows handled by one CTA (blockDim.y); 1..8 */
-    int32_t vec_bytes;       /* bytes per ld/st: 16 or 8 (4 and 2 exist as a narrow fall-back) */
+    int32_t vec_bytes;       /* bytes per ld/st: 16 or 8 (4 and 2 exist as a narrow fall-back); 16 with
+                                RT_STAGE_REG_REALIGN, whatever the row length */
     int32_t unroll;          /* independent vector loads in flight per thread and tensor: 1, 2, 4 */
     int32_t stage;           /* rt_stage */
     int32_t reduce;          /* rt_reduce */
@@ -209,7 +210,8 @@ typedef enum {
     RT_ERR_NULL = 1,           /* a required pointer is NULL */
     RT_ERR_DTYPE = 2,
     RT_ERR_SHAPE = 3,          /* n_tokens < 0, hidden <= 0, hidden too large */
-    RT_ERR_ALIGN = 4,          /* a pointer or the row length is not a multiple of vec_bytes (or of 16 for TMA) */
+    RT_ERR_ALIGN = 4,          /* a pointer or the row length is not a multiple of vec_bytes (or of 16 for TMA);
+                                  RT_STAGE_REG_REALIGN constrains the pointers only */
     RT_ERR_INFEASIBLE = 5,     /* theta violates a hard limit; nothing was launched */
     RT_ERR_CUDA = 6,           /* a CUDA runtime call failed; see rt_last_error() */
     RT_ERR_MISMATCH = 7,       /* correctness gate failed (search: for every candidate) */
@@ -246,6 +248,7 @@ int rmsnorm_template_run_host(const rt_params* p, const void* x_host, const void
                               const void* w_host, void* y_host, void* r_out_host, int64_t n_tokens,
                               int64_t hidden, float eps, int dtype, void* workspace,
                               int64_t workspace_bytes, int64_t chunk_tokens, void* stream);
+/* chunk_tokens <= 0 picks rows worth about 16 MB per tensor, the fastest chunk measured over PCIe Gen5 x16. */
 int64_t rmsnorm_host_workspace_bytes(int64_t n_tokens, int64_t hidden, int dtype, int64_t chunk_tokens);
 
 /*
