@@ -3,7 +3,8 @@
 // The template is the "parameterizable template" S~ of the paper's Algorithm 1 (Level 2) for the
 // kernel `fused_add_rmsnorm`; its axes are the execution-strategy dimensions named in "Tuning
 // parameter selection and search space derivation": thread-level granularity (threads per row,
-// rows per CTA: run-time block shape), vectorisation (VB bytes per ld/st), unrolling (U independent
+// rows per CTA: run-time block shape), vectorisation (VB bytes per ld/st: 32 - the 256-bit global accesses
+// of sm_100 -, 16 or 8), unrolling (U independent
 // loads in flight), and the organisation of shared memory and registers (STAGE, REDUCE).
 //
 // Compile-time axes: element type, VB, STAGE, REDUCE, U and - for the two register stages - CAP, the
@@ -65,7 +66,11 @@ template <int VB>
 __device__ __forceinline__ Vec<VB> ld_stream(const void* p)
 {
     Vec<VB> v;
-    if constexpr (VB == 16) {
+    if constexpr (VB == 32) {
+        asm volatile("ld.global.L1::no_allocate.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                     : "=r"(v.w[0]), "=r"(v.w[1]), "=r"(v.w[2]), "=r"(v.w[3]), "=r"(v.w[4]), "=r"(v.w[5]), "=r"(v.w[6]),
+                       "=r"(v.w[7]) : "l"(p));
+    } else if constexpr (VB == 16) {
         asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                      : "=r"(v.w[0]), "=r"(v.w[1]), "=r"(v.w[2]), "=r"(v.w[3]) : "l"(p));
     } else if constexpr (VB == 8) {
@@ -86,7 +91,13 @@ __device__ __forceinline__ Vec<VB> ld_stream(const void* p)
 template <int VB, bool EVICT_FIRST = false>
 __device__ __forceinline__ void st_stream(void* p, const Vec<VB>& v)
 {
-    if constexpr (VB == 16 && EVICT_FIRST) {
+    if constexpr (VB == 32 && EVICT_FIRST) {
+        asm volatile("st.global.cs.v8.u32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(v.w[0]), "r"(v.w[1]), "r"(v.w[2]),
+                     "r"(v.w[3]), "r"(v.w[4]), "r"(v.w[5]), "r"(v.w[6]), "r"(v.w[7]) : "memory");
+    } else if constexpr (VB == 32) {
+        asm volatile("st.global.v8.u32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(v.w[0]), "r"(v.w[1]), "r"(v.w[2]),
+                     "r"(v.w[3]), "r"(v.w[4]), "r"(v.w[5]), "r"(v.w[6]), "r"(v.w[7]) : "memory");
+    } else if constexpr (VB == 16 && EVICT_FIRST) {
         asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.w[0]), "r"(v.w[1]), "r"(v.w[2]),
                      "r"(v.w[3]) : "memory");
     } else if constexpr (VB == 8 && EVICT_FIRST) {
@@ -108,7 +119,11 @@ template <int VB>
 __device__ __forceinline__ Vec<VB> ld_weight(const void* p)
 {
     Vec<VB> v;
-    if constexpr (VB == 16) {
+    if constexpr (VB == 32) {
+        const uint4 q = __ldg(reinterpret_cast<const uint4*>(p)), h = __ldg(reinterpret_cast<const uint4*>(p) + 1);
+        v.w[0] = q.x; v.w[1] = q.y; v.w[2] = q.z; v.w[3] = q.w;
+        v.w[4] = h.x; v.w[5] = h.y; v.w[6] = h.z; v.w[7] = h.w;
+    } else if constexpr (VB == 16) {
         const uint4 q = __ldg(reinterpret_cast<const uint4*>(p));
         v.w[0] = q.x; v.w[1] = q.y; v.w[2] = q.z; v.w[3] = q.w;
     } else if constexpr (VB == 8) {
@@ -128,7 +143,12 @@ template <int VB>
 __device__ __forceinline__ Vec<VB> ld_weight_early(const void* p)
 {
     Vec<VB> v;
-    if constexpr (VB == 16) {
+    if constexpr (VB == 32) {
+        asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(v.w[0]), "=r"(v.w[1]), "=r"(v.w[2]), "=r"(v.w[3]) : "l"(p));
+        asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(v.w[4]), "=r"(v.w[5]), "=r"(v.w[6]), "=r"(v.w[7]) : "l"(reinterpret_cast<const unsigned char*>(p) + 16));
+    } else if constexpr (VB == 16) {
         asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];"
                      : "=r"(v.w[0]), "=r"(v.w[1]), "=r"(v.w[2]), "=r"(v.w[3]) : "l"(p));
     } else if constexpr (VB == 8) {
@@ -147,7 +167,11 @@ template <int VB>
 __device__ __forceinline__ Vec<VB> ld_shared(const void* p)
 {
     Vec<VB> v;
-    if constexpr (VB == 16) {
+    if constexpr (VB == 32) {
+        const uint4 q = *reinterpret_cast<const uint4*>(p), h = *(reinterpret_cast<const uint4*>(p) + 1);
+        v.w[0] = q.x; v.w[1] = q.y; v.w[2] = q.z; v.w[3] = q.w;
+        v.w[4] = h.x; v.w[5] = h.y; v.w[6] = h.z; v.w[7] = h.w;
+    } else if constexpr (VB == 16) {
         const uint4 q = *reinterpret_cast<const uint4*>(p);
         v.w[0] = q.x; v.w[1] = q.y; v.w[2] = q.z; v.w[3] = q.w;
     } else if constexpr (VB == 8) {

@@ -648,7 +648,7 @@ int level_of(const int* levels, int n, int v)
 const int kTpr[] = {32, 64, 128, 256, 512, 1024};
 const int kRpc[] = {1, 2, 4, 8};
 const int kUnr[] = {1, 2, 4};
-const int kVec[] = {2, 4, 8, 16};
+const int kVec[] = {2, 4, 8, 16, 32};
 const int kClu[] = {1, 2, 4, 8};
 
 struct SearchState {
@@ -714,7 +714,7 @@ struct SearchState {
         step(kTpr, 6, &rt_params::threads_per_row);
         step(kRpc, 4, &rt_params::rows_per_cta);
         step(kUnr, 3, &rt_params::unroll);
-        step(kVec, 4, &rt_params::vec_bytes);
+        step(kVec, 5, &rt_params::vec_bytes);
         // another stage at the same vector width; where that stage has no such point (the ragged-row stage is
         // all 16-byte chunks while the other stages of a misaligned shape are narrower), at its widest width
         for (int stage = 0; stage <= RT_STAGE_REG_REALIGN; ++stage) {
@@ -722,7 +722,7 @@ struct SearchState {
             q.stage = stage;
             if (index.find(pack_params(q)) == index.end()) {
                 if (stage == RT_STAGE_REG_REALIGN) q.reduce = RT_REDUCE_SHFL, q.cluster_size = 1;
-                for (int k = 3; k >= 0; --k) {
+                for (int k = 4; k >= 0; --k) {
                     q.vec_bytes = kVec[k];
                     if (index.find(pack_params(q)) != index.end()) break;
                 }

@@ -27,7 +27,7 @@ def test_library_exports_every_declared_symbol():
 def test_binding_covers_the_header():
     from paper_2601_12698_b200 import binding
     assert sorted(binding.EXPORTED) == sorted(_declared_functions())
-    assert binding.lib.rt_num_kernel_instances() == 670  # 449 norm (39 of them the ragged-row stage) + 46 silu_and_mul + 46 merge_attn_states + 30 fp8-output + 99 all-reduce-fused
+    assert binding.lib.rt_num_kernel_instances() == 814  # 593 norm (39 of them the ragged-row stage, 144 with 32-byte vectors) + 46 silu_and_mul + 46 merge_attn_states + 30 fp8-output + 99 all-reduce-fused
     assert binding.lib.rt_status_string(binding.RT_ERR_INFEASIBLE).decode().startswith("configuration outside")
     inst = binding.kernel_instances()
     assert {i["dtype"] for i in inst} == {0, 1, 2} and {i["stage"] for i in inst} == {0, 1, 2, 3}

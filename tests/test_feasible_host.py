@@ -56,7 +56,12 @@ def test_rules_bite_where_they_should(L):
     f = B.tuner_derive_feasible(B.shape_of(8192, 6148, "fp16"), L)
     assert {t.vec_bytes for t in row_vectors(f)} == {8} and {t.stage for t in f} == {0, 1, ragged}
     assert {t.vec_bytes for t in f if t.stage == ragged} == {16}
-    # 6152 fp16: 769 16-byte vectors, both widths, the three aligned stages and no ragged-row stage
+    # rows of 8192 bf16 elements: all three widths of the vector axis; other kernels' grids stop at 16 bytes
+    f = B.tuner_derive_feasible(B.shape_of(16384, 8192, "bf16"), L)
+    assert {t.vec_bytes for t in f} == {8, 16, 32} and {t.stage for t in f if t.vec_bytes == 32} == {0, 1, 2}
+    assert B.tuner_check_params(B.shape_of(16384, 8192, "bf16", min_ptr_align=16), B.make_params(vec_bytes=32), L) == B.RT_ERR_ALIGN
+    assert B.tuner_check_params(B.shape_of(64, 8192, "bf16", op=B.RT_OP_SILU_AND_MUL), B.make_params(vec_bytes=32), L) == B.RT_ERR_INFEASIBLE
+    # 6152 fp16: 769 16-byte vectors (no 32-byte ones), both widths, the three aligned stages and no ragged-row stage
     f = B.tuner_derive_feasible(B.shape_of(8192, 6152, "fp16"), L)
     assert {t.vec_bytes for t in f} == {8, 16} and {t.stage for t in f} == {0, 1, 2}
     # rows that fit no 8-byte vector fall back to the widest narrow width, or take the ragged-row stage

@@ -38,7 +38,7 @@ def test_tuning_builds_a_table_and_a_general_configuration(B, tuned, tmp_path):
 
 @pytest.mark.parametrize("dtype,T,H,want_source", [
     ("bf16", 64, 4096, "table_exact"), ("bf16", 2048, 8192, "table_exact"), ("bf16", 77, 4096, "table_nearest"),
-    ("bf16", 4096, 7168, "table_nearest"), ("fp16", 300, 6152, "table_nearest"), ("fp16", 300, 6148, None),
+    ("bf16", 4096, 7168, "table_nearest"), ("fp16", 300, 6152, "nearest_or_general"), ("fp16", 300, 6148, None),
     ("fp32", 33, 12288, "general_or_feasible"), ("fp16", 9, 6146, "feasible_set"), ("bf16", 1, 8, None)])
 def test_launch_auto_matches_the_oracle(B, oracle_lib, tuned, dtype, T, H, want_source):
     from paper_2601_12698_b200 import synth
@@ -55,7 +55,9 @@ def test_launch_auto_matches_the_oracle(B, oracle_lib, tuned, dtype, T, H, want_
     assert B.tuner_check_params(shape, used) == B.RT_OK
     theta, source = table.lookup(shape)
     assert theta.key() == used.key()
-    if want_source == "general_or_feasible":
+    if want_source == "nearest_or_general":  # rows of 6152 fp16 take no 32-byte vectors: an entry that uses them is skipped
+        assert source in ("table_nearest", "general")
+    elif want_source == "general_or_feasible":
         assert source in ("general", "feasible_set")
     elif want_source is not None:
         assert source == want_source

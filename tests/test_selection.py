@@ -91,7 +91,7 @@ def test_table_lookup_prefers_exact_then_nearest_then_general():
     theta, src = B.SpecTable([], None).lookup(B.shape_of(64, 6146, "fp16", min_ptr_align=4), L)  # pointers rule it out
     assert src == "feasible_set" and (theta.stage, theta.vec_bytes) == (B.RT_STAGE_REG, 4)
     theta, src = B.SpecTable([], None).lookup(B.shape_of(64, 4096, "fp16"), L)
-    assert src == "feasible_set" and theta.stage == B.RT_STAGE_REG and theta.vec_bytes == 16
+    assert src == "feasible_set" and theta.stage == B.RT_STAGE_REG and theta.vec_bytes == 32  # the widest that fits
     # an entry tuned on ragged rows serves other ragged rows of its dtype, never rows that are 16-byte multiples
     ragged = B.make_params(unroll=4, stage=B.RT_STAGE_REG_REALIGN)
     tr = B.SpecTable([(B.shape_of(8192, 6145, "fp16"), ragged, 65.0), (B.shape_of(8192, 5120, "fp16"), th_fp32, 51.0)], general)
