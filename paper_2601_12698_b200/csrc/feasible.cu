@@ -25,7 +25,7 @@ int next_pow2(int v)
     return p;
 }
 
-// Vector widths offered for a shape: 32 (add_rmsnorm), 16 and 8 bytes (the tuned axis); when the row length or a base
+// Vector widths offered for a shape: 32, 16 and 8 bytes (the tuned axis); when the row length or a base
 // pointer allows neither, the widest narrower width that fits (a fall-back, not a tuned axis).
 std::vector<int> vec_levels(const rt_shape& s)
 {
@@ -34,9 +34,10 @@ std::vector<int> vec_levels(const rt_shape& s)
     const int64_t head_bytes = s.op == RT_OP_MERGE_ATTN_STATES && s.head_dim > 0 ? (int64_t)s.head_dim * eb : row_bytes;
     auto fits = [&](int vb) { return vb >= eb && row_bytes % vb == 0 && head_bytes % vb == 0 && s.min_ptr_align >= vb; };
     if (fits(32) || fits(16) || fits(8)) {
-        // the 256-bit accesses of sm_100 are a level of the norm template's vector axis only
-        if (s.op == RT_OP_ADD_RMSNORM) return {32, 16, 8};
-        return {16, 8};
+        // the 256-bit accesses of sm_100: a level of the vector axis of the three tuned kernels; the two
+        // variants of the norm are instantiated with 16-byte vectors only
+        if (s.op == RT_OP_ADD_RMSNORM_FP8 || s.op == RT_OP_ADD_RMSNORM_ALLREDUCE) return {16, 8};
+        return {32, 16, 8};
     }
     if (fits(4)) return {4};
     if (fits(2)) return {2};

@@ -8,7 +8,7 @@
 // stages: U in {1,2,4}, all three reductions.  Narrow fall-back (4- and 2-byte vectors, for rows whose
 // byte length is not a multiple of 8): register stage, shuffle reduction, U in {1,4}.
 // Ragged-row register stage (16-byte chunks, shuffle reduction): the register stage's (CAP, U) list.
-// silu_and_mul (one unit per element type, every vector width): stages register and TMA bulk for 16- and
+// silu_and_mul (one unit per element type, every vector width): stages register and TMA bulk for 32-, 16- and
 // 8-byte vectors with U in {1,2,4}; register stage with U in {1,4} for the 4- and 2-byte fall-back.
 // merge_attn_states: the same instance list as silu_and_mul.
 // fp8-output norm (16-bit element types, 16-byte vectors, shuffle reduction): register stage with CAP in
@@ -116,7 +116,7 @@ std::vector<rt::KernelEntry> build_entries()
 #elif RT_UNIT_GROUP == 1
         RT_SMEM_LIST(1), RT_SMEM_LIST(2)
 #elif RT_UNIT_GROUP == 3
-        RT_SILU_WIDE(16), RT_SILU_WIDE(8), silu_entry<4, 0, 1>(), silu_entry<4, 0, 4>(), silu_entry<2, 0, 1>(),
+        RT_SILU_WIDE(32), RT_SILU_WIDE(16), RT_SILU_WIDE(8), silu_entry<4, 0, 1>(), silu_entry<4, 0, 4>(), silu_entry<2, 0, 1>(),
         silu_entry<2, 0, 4>()
 #elif RT_UNIT_GROUP == 5
         fp8_entry<0, 1, 1>(), fp8_entry<0, 1, 2>(), fp8_entry<0, 2, 2>(), fp8_entry<0, 1, 4>(), fp8_entry<0, 2, 4>(),
@@ -127,7 +127,7 @@ std::vector<rt::KernelEntry> build_entries()
 #elif RT_UNIT_GROUP == 7
         RT_REALIGN_LIST
 #elif RT_UNIT_GROUP == 4
-        RT_MERGE_WIDE(16), RT_MERGE_WIDE(8), merge_entry<4, 0, 1>(), merge_entry<4, 0, 4>(), merge_entry<2, 0, 1>(),
+        RT_MERGE_WIDE(32), RT_MERGE_WIDE(16), RT_MERGE_WIDE(8), merge_entry<4, 0, 1>(), merge_entry<4, 0, 4>(), merge_entry<2, 0, 1>(),
         merge_entry<2, 0, 4>()
 #else
         entry<0, 0, 1, 1>(), entry<0, 0, 1, 2>(), entry<0, 0, 1, 4>(), entry<0, 0, 4, 4>(), entry<0, 0, 1, 8>(),

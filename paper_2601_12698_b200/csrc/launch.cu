@@ -306,8 +306,9 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
         plan->reject_reason = kRejectThreads;
         return RT_ERR_INFEASIBLE;
     }
-    if (!(vb == 32 || vb == 16 || vb == 8 || vb == 4 || vb == 2) || vb < eb || (vb == 32 && s->op != RT_OP_ADD_RMSNORM)) {
-        set_error("vec_bytes=%d is not 32 (add_rmsnorm only), 16, 8, 4 or 2, or is narrower than one element", vb);
+    if (!(vb == 32 || vb == 16 || vb == 8 || vb == 4 || vb == 2) || vb < eb || (vb == 32 && (is_fp8 || is_allreduce))) {
+        set_error("vec_bytes=%d is not 32 (not for the fp8-output and all-reduce-fused norms), 16, 8, 4 or 2, or is narrower "
+                  "than one element", vb);
         plan->reject_reason = kRejectArgs;
         return RT_ERR_INFEASIBLE;
     }

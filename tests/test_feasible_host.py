@@ -56,11 +56,14 @@ def test_rules_bite_where_they_should(L):
     f = B.tuner_derive_feasible(B.shape_of(8192, 6148, "fp16"), L)
     assert {t.vec_bytes for t in row_vectors(f)} == {8} and {t.stage for t in f} == {0, 1, ragged}
     assert {t.vec_bytes for t in f if t.stage == ragged} == {16}
-    # rows of 8192 bf16 elements: all three widths of the vector axis; other kernels' grids stop at 16 bytes
+    # rows of 8192 bf16 elements: all three widths of the vector axis; the two variants of the norm stop at 16 bytes
     f = B.tuner_derive_feasible(B.shape_of(16384, 8192, "bf16"), L)
     assert {t.vec_bytes for t in f} == {8, 16, 32} and {t.stage for t in f if t.vec_bytes == 32} == {0, 1, 2}
     assert B.tuner_check_params(B.shape_of(16384, 8192, "bf16", min_ptr_align=16), B.make_params(vec_bytes=32), L) == B.RT_ERR_ALIGN
-    assert B.tuner_check_params(B.shape_of(64, 8192, "bf16", op=B.RT_OP_SILU_AND_MUL), B.make_params(vec_bytes=32), L) == B.RT_ERR_INFEASIBLE
+    assert B.tuner_check_params(B.shape_of(64, 8192, "bf16", op=B.RT_OP_SILU_AND_MUL), B.make_params(vec_bytes=32), L) == B.RT_OK
+    assert B.tuner_check_params(B.shape_of(64, 8192, "bf16", op=B.RT_OP_ADD_RMSNORM_FP8), B.make_params(vec_bytes=32), L) == B.RT_ERR_INFEASIBLE
+    assert B.tuner_check_params(B.shape_of(64, 8192, "bf16", op=B.RT_OP_ADD_RMSNORM_ALLREDUCE, n_parts=2),
+                                B.make_params(vec_bytes=32), L) == B.RT_ERR_INFEASIBLE
     # 6152 fp16: 769 16-byte vectors (no 32-byte ones), both widths, the three aligned stages and no ragged-row stage
     f = B.tuner_derive_feasible(B.shape_of(8192, 6152, "fp16"), L)
     assert {t.vec_bytes for t in f} == {8, 16} and {t.stage for t in f} == {0, 1, 2}
@@ -128,7 +131,7 @@ def test_silu_and_mul_grid_has_no_reduction_axis(L):
     raw = B.tuner_raw_grid(s)
     assert {t.reduce for t in raw} == {0} and {t.cluster_size for t in raw} == {1} and {t.stage for t in raw} == {0, 2}
     f = B.tuner_derive_feasible(s, L)
-    assert f and {t.stage for t in f} == {0, 2} and {t.vec_bytes for t in f} == {16, 8}
+    assert f and {t.stage for t in f} == {0, 2} and {t.vec_bytes for t in f} == {32, 16, 8}
     for th in f:
         assert B.tuner_check_params(s, th, L) == B.RT_OK
     c = B.tuner_derive_counts(s, L)
@@ -145,8 +148,11 @@ def test_silu_and_mul_grid_has_no_reduction_axis(L):
 def test_merge_attn_states_grid(L):
     s = B.shape_of(512, 40 * 128, "bf16", op=B.RT_OP_MERGE_ATTN_STATES, head_dim=128)
     f = B.tuner_derive_feasible(s, L)
-    assert f and {t.stage for t in f} == {0, 2} and {t.reduce for t in f} == {0} and {t.vec_bytes for t in f} == {16, 8}
+    assert f and {t.stage for t in f} == {0, 2} and {t.reduce for t in f} == {0} and {t.vec_bytes for t in f} == {32, 16, 8}
     assert all(B.tuner_check_params(s, t, L) == B.RT_OK for t in f)
+    # heads of 72 bf16 elements (144 bytes): 16-byte vectors fit a head, 32-byte ones would straddle two
+    f72 = B.tuner_derive_feasible(B.shape_of(64, 8 * 72, "bf16", op=B.RT_OP_MERGE_ATTN_STATES, head_dim=72), L)
+    assert f72 and {t.vec_bytes for t in f72} == {16, 8}
     # a vector may not straddle two heads: heads of 66 bf16 elements (132 bytes) allow 4-byte vectors only
     f = B.tuner_derive_feasible(B.shape_of(4, 7 * 66, "bf16", op=B.RT_OP_MERGE_ATTN_STATES, head_dim=66), L)
     assert f and {t.vec_bytes for t in f} == {4}
