@@ -742,12 +742,15 @@ struct SearchState {
 };
 
 // The coarse grid: every other level of the ordered axes (threads per row 64/256/1024, rows per CTA
-// 1/4, unroll 1/4), the widest vector of the point's stage, every stage and reduction mode.
-bool on_coarse_grid(const rt_params& p, int widest_vec)
+// 1/4, unroll 1 and the deepest feasible), the widest vector of the point's stage, every stage and reduction mode.
+bool on_coarse_grid(const rt_params& p, int widest_vec, bool deepest_unroll)
 {
     const int lt = level_of(kTpr, 6, p.threads_per_row), lr = level_of(kRpc, 4, p.rows_per_cta),
               lu = level_of(kUnr, 3, p.unroll);
-    return (lt % 2 == 1) && (lr % 2 == 0) && (lu % 2 == 0) && p.vec_bytes == widest_vec;
+    // the two ends of the unroll axis: 1, and the deepest unroll that is feasible beside these other parameters
+    // (4 where a thread owns that many vectors; with wide vectors and many threads per row it is 2, and the
+    // step from 1 to 2 can be the steepest of the whole space)
+    return (lt % 2 == 1) && (lr % 2 == 0) && (lu == 0 || deepest_unroll) && p.vec_bytes == widest_vec;
 }
 
 // When the budget cannot cover the whole coarse grid, the part that is evaluated must still touch every
@@ -831,8 +834,15 @@ int run_search(const rt_shape& shape, const rt_limits& limits, const rt_budget& 
         int widest[RT_STAGE_REG_REALIGN + 1] = {0, 0, 0, 0};  // per stage: the ragged-row stage is wider than the others
         for (const rt_params& p : feasible) widest[p.stage] = std::max(widest[p.stage], p.vec_bytes);
         std::vector<int> coarse;
-        for (int i = 0; i < (int)feasible.size(); ++i)
-            if (on_coarse_grid(S.cand[i], widest[S.cand[i].stage])) coarse.push_back(i);
+        for (int i = 0; i < (int)feasible.size(); ++i) {
+            bool deepest = true;  // no feasible point with these parameters and a deeper unroll
+            for (int u = S.cand[i].unroll * 2; u <= 4 && deepest; u *= 2) {
+                rt_params q = S.cand[i];
+                q.unroll = u;
+                if (S.index.find(pack_params(q)) != S.index.end()) deepest = false;
+            }
+            if (on_coarse_grid(S.cand[i], widest[S.cand[i].stage], deepest)) coarse.push_back(i);
+        }
         if (coarse.empty())
             for (int i = 0; i < (int)feasible.size(); ++i) coarse.push_back(i);
         const int grid_budget = std::max(1, (S.max_evals - top_k - S.used) / 2);
