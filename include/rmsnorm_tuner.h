@@ -84,7 +84,8 @@ typedef enum {
 typedef struct {
     int32_t threads_per_row; /* threads cooperating on one row (blockDim.x); power of two, 32..1024 */
     int32_t rows_per_cta;    /* rows handled by one CTA (blockDim.y); 1..8 */
-    int32_t vec_bytes;       /* bytes per ld/st: 32 (add_rmsnorm only: the 256-bit global accesses of sm_100), 16
+    int32_t vec_bytes;       /* bytes per ld/st: 32 (the 256-bit global accesses of sm_100; not for the fp8-output and
+                                all-reduce-fused norms), 16
                                 or 8 (4 and 2 exist as a narrow fall-back); 16 with
                                 RT_STAGE_REG_REALIGN, whatever the row length */
     int32_t unroll;          /* independent vector loads in flight per thread and tensor: 1, 2, 4 */
