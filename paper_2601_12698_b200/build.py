@@ -63,7 +63,7 @@ _MERGE_ENTRY = re.compile(r"Compiling entry function '_ZN2rt24merge_attn_states_
                           r"EEvNS_9MergeArgsE'.*?(\d+) bytes spill stores.*?Used (\d+) registers(?:.*?(\d+) bytes smem)?", re.S)
 
 
-_FP8_ENTRY = re.compile(r"Compiling entry function '_ZN2rt22add_rmsnorm_fp8_kernelI(\w+?)Li(\d+)ELi(\d+)ELi(\d+)E"
+_FP8_ENTRY = re.compile(r"Compiling entry function '_ZN2rt22add_rmsnorm_fp8_kernelI(\w+?)Li(\d+)ELi(\d+)ELi(\d+)ELi(\d+)E"
                         r"EEvNS_7Fp8ArgsE'.*?(\d+) bytes spill stores.*?Used (\d+) registers(?:.*?(\d+) bytes smem)?", re.S)
 
 
@@ -87,8 +87,8 @@ def parse_ptxas(log: str) -> list[tuple]:
     for block in log.split("ptxas info    : Compiling entry function")[1:]:
         m = _FP8_ENTRY.search("Compiling entry function" + block)
         if m:
-            t, st, u, cap, spill, regs, smem = m.groups()
-            rows.append((3, _MANGLED_DTYPE[t], 16, int(st), 0, int(u), int(cap) if int(st) == 0 else 0, int(regs),
+            t, vb, st, u, cap, spill, regs, smem = m.groups()
+            rows.append((3, _MANGLED_DTYPE[t], int(vb), int(st), 0, int(u), int(cap) if int(st) == 0 else 0, int(regs),
                          int(smem or 0), int(spill), 0))
         m = _ALLREDUCE_ENTRY.search("Compiling entry function" + block)
         if m:

@@ -1,6 +1,6 @@
 // Fused residual-add + RMSNorm with a per-token fp8 (e4m3) quantised output: the norm template's variant
 // for a following fp8 GEMM.  Same row mapping and stages as add_rmsnorm_kernel (registers or TMA bulk),
-// 16-byte vectors of a 16-bit element type, shuffle reduction.
+// 16- or 32-byte vectors of a 16-bit element type, shuffle reduction.
 //
 // Per row:  s = fp32(x) + fp32(r);  r_out = rn(s);  y = s * rsqrt(mean(s^2) + eps) * w   (not rounded);
 //           scale = max(max_j |y_j|, 1e-12) / 448;   q_j = rn_e4m3_satfinite(y_j / scale).
@@ -21,7 +21,7 @@ struct Fp8Args {
     void* r_out;
     long long n_tokens;
     int hidden;
-    int nvec;       // 16-byte vectors in one row
+    int nvec;       // vectors (16 or 32 bytes) in one row
     float eps;
     int* status;
 };
@@ -64,12 +64,12 @@ __device__ __forceinline__ void row_reduce_sum_max(float& sum, float& mx, int tx
     }
 }
 
-template <typename T, int STAGE, int U, int CAP>
+template <typename T, int VB, int STAGE, int U, int CAP>
 __global__ void add_rmsnorm_fp8_kernel(const Fp8Args a)
 {
-    constexpr int VB = 16;
+    static_assert(VB == 16 || VB == 32, "16- or 32-byte vectors of x and r; q leaves as 8 or 16 bytes");
     using C = Codec<T, VB>;
-    constexpr int EPV = C::EPV;  // 8
+    constexpr int EPV = C::EPV;  // 8 or 16
     static_assert(sizeof(T) == 2, "the fp8-output variant takes 16-bit inputs");
     static_assert(STAGE != kStageReg || CAP % U == 0, "the unroll depth divides the per-thread vector count");
     extern __shared__ __align__(128) unsigned char dyn_smem[];
@@ -88,15 +88,16 @@ __global__ void add_rmsnorm_fp8_kernel(const Fp8Args a)
 
     float ss = 0.f, amax = 0.f;
 
-    // y_j * inv_scale -> 8 bytes
+    // y_j * inv_scale -> one byte per element: 8 or 16 bytes per vector
     auto quantise_store = [&](int v, const float (&s)[EPV], const float (&wf)[EPV], float rho, float inv_scale) {
         float t[EPV];
 #pragma unroll
         for (int e = 0; e < EPV; ++e) t[e] = s[e] * rho * wf[e] * inv_scale;
-        Vec<8> out;
-        out.w[0] = pack_e4m3x2(t[0], t[1]) | (pack_e4m3x2(t[2], t[3]) << 16);
-        out.w[1] = pack_e4m3x2(t[4], t[5]) | (pack_e4m3x2(t[6], t[7]) << 16);
-        st_stream<8, STAGE == kStageReg>(qrow + (size_t)v * 8, out);
+        Vec<EPV> out;
+#pragma unroll
+        for (int k = 0; k < EPV / 4; ++k)
+            out.w[k] = pack_e4m3x2(t[4 * k], t[4 * k + 1]) | (pack_e4m3x2(t[4 * k + 2], t[4 * k + 3]) << 16);
+        st_stream<EPV, STAGE == kStageReg>(qrow + (size_t)v * EPV, out);
     };
     auto finish_row = [&](float& rho, float& inv_scale) {
         row_reduce_sum_max(ss, amax, tx, ty, tpr);

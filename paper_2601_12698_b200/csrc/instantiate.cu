@@ -11,8 +11,8 @@
 // silu_and_mul (one unit per element type, every vector width): stages register and TMA bulk for 32-, 16- and
 // 8-byte vectors with U in {1,2,4}; register stage with U in {1,4} for the 4- and 2-byte fall-back.
 // merge_attn_states: the same instance list as silu_and_mul.
-// fp8-output norm (16-bit element types, 16-byte vectors, shuffle reduction): register stage with CAP in
-// {1,2,4,8,16} and U <= CAP, TMA stage with U in {1,2,4}.
+// fp8-output norm (16-bit element types, 32- and 16-byte vectors, shuffle reduction): register stage with CAP in
+// {1,2,4,8,16} (while the row stays within 128 fp32 registers per thread) and U <= CAP, TMA stage with U in {1,2,4}.
 // all-reduce-fused norm (16-byte vectors, register stage, shuffle reduction): 2, 4 and 8 parts, CAP in
 // {1,2,4,8,16} while the row stays within 128 fp32 registers per thread, U <= CAP with U * parts <= 16 loads of x
 // in flight per thread.
@@ -53,16 +53,21 @@ rt::KernelEntry silu_entry()
                                (const void*)&rt::silu_and_mul_kernel<T, VB, ST, U>};
     }
 }
-template <int ST, int U, int CAP>
+template <int VB, int ST, int U, int CAP>
 rt::KernelEntry fp8_entry()
 {
-    if constexpr (sizeof(T) != 2) {
-        return rt::KernelEntry{RT_OP_ADD_RMSNORM_FP8, kDtype, 16, ST, 0, U, CAP, nullptr};
+    if constexpr (sizeof(T) != 2 || (ST == rt::kStageReg && CAP * (VB / 2) > kMaxRowRegisters)) {
+        return rt::KernelEntry{RT_OP_ADD_RMSNORM_FP8, kDtype, VB, ST, 0, U, CAP, nullptr};
     } else {
-        return rt::KernelEntry{RT_OP_ADD_RMSNORM_FP8, kDtype, 16, ST, 0, U, ST == rt::kStageReg ? CAP : 0,
-                               (const void*)&rt::add_rmsnorm_fp8_kernel<T, ST, U, CAP>};
+        return rt::KernelEntry{RT_OP_ADD_RMSNORM_FP8, kDtype, VB, ST, 0, U, ST == rt::kStageReg ? CAP : 0,
+                               (const void*)&rt::add_rmsnorm_fp8_kernel<T, VB, ST, U, CAP>};
     }
 }
+#define RT_FP8_LIST(VB)                                                                                             \
+    fp8_entry<VB, 0, 1, 1>(), fp8_entry<VB, 0, 1, 2>(), fp8_entry<VB, 0, 2, 2>(), fp8_entry<VB, 0, 1, 4>(),          \
+    fp8_entry<VB, 0, 2, 4>(), fp8_entry<VB, 0, 4, 4>(), fp8_entry<VB, 0, 1, 8>(), fp8_entry<VB, 0, 2, 8>(),          \
+    fp8_entry<VB, 0, 4, 8>(), fp8_entry<VB, 0, 1, 16>(), fp8_entry<VB, 0, 2, 16>(), fp8_entry<VB, 0, 4, 16>(),       \
+    fp8_entry<VB, 2, 1, 1>(), fp8_entry<VB, 2, 2, 1>(), fp8_entry<VB, 2, 4, 1>()
 
 template <int NP, int U, int CAP>
 rt::KernelEntry allreduce_entry()
@@ -119,9 +124,7 @@ std::vector<rt::KernelEntry> build_entries()
         RT_SILU_WIDE(32), RT_SILU_WIDE(16), RT_SILU_WIDE(8), silu_entry<4, 0, 1>(), silu_entry<4, 0, 4>(), silu_entry<2, 0, 1>(),
         silu_entry<2, 0, 4>()
 #elif RT_UNIT_GROUP == 5
-        fp8_entry<0, 1, 1>(), fp8_entry<0, 1, 2>(), fp8_entry<0, 2, 2>(), fp8_entry<0, 1, 4>(), fp8_entry<0, 2, 4>(),
-        fp8_entry<0, 4, 4>(), fp8_entry<0, 1, 8>(), fp8_entry<0, 2, 8>(), fp8_entry<0, 4, 8>(), fp8_entry<0, 1, 16>(),
-        fp8_entry<0, 2, 16>(), fp8_entry<0, 4, 16>(), fp8_entry<2, 1, 1>(), fp8_entry<2, 2, 1>(), fp8_entry<2, 4, 1>()
+        RT_FP8_LIST(32), RT_FP8_LIST(16)
 #elif RT_UNIT_GROUP == 6
         RT_ALLREDUCE_LIST(2), RT_ALLREDUCE_LIST(4), RT_ALLREDUCE_LIST(8)
 #elif RT_UNIT_GROUP == 7

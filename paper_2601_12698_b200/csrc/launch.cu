@@ -306,9 +306,9 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
         plan->reject_reason = kRejectThreads;
         return RT_ERR_INFEASIBLE;
     }
-    if (!(vb == 32 || vb == 16 || vb == 8 || vb == 4 || vb == 2) || vb < eb || (vb == 32 && (is_fp8 || is_allreduce))) {
-        set_error("vec_bytes=%d is not 32 (not for the fp8-output and all-reduce-fused norms), 16, 8, 4 or 2, or is narrower "
-                  "than one element", vb);
+    if (!(vb == 32 || vb == 16 || vb == 8 || vb == 4 || vb == 2) || vb < eb || (vb == 32 && is_allreduce)) {
+        set_error("vec_bytes=%d is not 32 (not for the all-reduce-fused norm), 16, 8, 4 or 2, or is narrower than one "
+                  "element", vb);
         plan->reject_reason = kRejectArgs;
         return RT_ERR_INFEASIBLE;
     }
@@ -334,9 +334,9 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
         plan->reject_reason = kRejectArgs;
         return RT_ERR_SHAPE;
     }
-    if (is_fp8 && (s->dtype == RT_FP32 || p->vec_bytes != 16 || p->reduce != RT_REDUCE_SHFL || p->cluster_size != 1 ||
+    if (is_fp8 && (s->dtype == RT_FP32 || p->vec_bytes < 16 || p->reduce != RT_REDUCE_SHFL || p->cluster_size != 1 ||
                    p->stage == RT_STAGE_SMEM_LDG)) {
-        set_error("the fp8-output norm takes bf16/fp16, 16-byte vectors, the shuffle reduction and the register or TMA "
+        set_error("the fp8-output norm takes bf16/fp16, 32- or 16-byte vectors, the shuffle reduction and the register or TMA "
                   "stage (dtype=%d vec=%d reduce=%d cluster=%d stage=%d)", s->dtype, p->vec_bytes, p->reduce,
                   p->cluster_size, p->stage);
         plan->reject_reason = kRejectArgs;
@@ -829,8 +829,10 @@ int rmsnorm_fp8_template_launch(const rt_params* p, const void* x, const void* r
         rt::set_error("a tensor pointer is NULL");
         return RT_ERR_NULL;
     }
-    if (n_tokens > 0 && (((uintptr_t)scale & 3u) || ((uintptr_t)q & 7u))) {
-        rt::set_error("scale must be 4-byte and q 8-byte aligned");
+    // q leaves as one vector of vec_bytes / 2 bytes per vector of x
+    const uintptr_t q_mask = p->vec_bytes == 32 ? 15u : 7u;
+    if (n_tokens > 0 && (((uintptr_t)scale & 3u) || ((uintptr_t)q & q_mask))) {
+        rt::set_error("scale must be 4-byte and q %d-byte aligned", (int)q_mask + 1);
         return RT_ERR_ALIGN;
     }
     rt_limits L;

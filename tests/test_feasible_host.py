@@ -56,12 +56,12 @@ def test_rules_bite_where_they_should(L):
     f = B.tuner_derive_feasible(B.shape_of(8192, 6148, "fp16"), L)
     assert {t.vec_bytes for t in row_vectors(f)} == {8} and {t.stage for t in f} == {0, 1, ragged}
     assert {t.vec_bytes for t in f if t.stage == ragged} == {16}
-    # rows of 8192 bf16 elements: all three widths of the vector axis; the two variants of the norm stop at 16 bytes
+    # rows of 8192 bf16 elements: all three widths of the vector axis; the all-reduce-fused norm stops at 16 bytes
     f = B.tuner_derive_feasible(B.shape_of(16384, 8192, "bf16"), L)
     assert {t.vec_bytes for t in f} == {8, 16, 32} and {t.stage for t in f if t.vec_bytes == 32} == {0, 1, 2}
     assert B.tuner_check_params(B.shape_of(16384, 8192, "bf16", min_ptr_align=16), B.make_params(vec_bytes=32), L) == B.RT_ERR_ALIGN
     assert B.tuner_check_params(B.shape_of(64, 8192, "bf16", op=B.RT_OP_SILU_AND_MUL), B.make_params(vec_bytes=32), L) == B.RT_OK
-    assert B.tuner_check_params(B.shape_of(64, 8192, "bf16", op=B.RT_OP_ADD_RMSNORM_FP8), B.make_params(vec_bytes=32), L) == B.RT_ERR_INFEASIBLE
+    assert B.tuner_check_params(B.shape_of(64, 8192, "bf16", op=B.RT_OP_ADD_RMSNORM_FP8), B.make_params(vec_bytes=32), L) == B.RT_OK
     assert B.tuner_check_params(B.shape_of(64, 8192, "bf16", op=B.RT_OP_ADD_RMSNORM_ALLREDUCE, n_parts=2),
                                 B.make_params(vec_bytes=32), L) == B.RT_ERR_INFEASIBLE
     # 6152 fp16: 769 16-byte vectors (no 32-byte ones), both widths, the three aligned stages and no ragged-row stage
@@ -166,8 +166,11 @@ def test_merge_attn_states_grid(L):
 def test_fp8_output_norm_grid(L):
     s = B.shape_of(16384, 8192, "bf16", op=B.RT_OP_ADD_RMSNORM_FP8)
     f = B.tuner_derive_feasible(s, L)
-    assert f and {t.vec_bytes for t in f} == {16} and {t.stage for t in f} == {0, 2} and {t.reduce for t in f} == {0}
+    assert f and {t.vec_bytes for t in f} == {16, 32} and {t.stage for t in f} == {0, 2} and {t.reduce for t in f} == {0}
     assert all(B.tuner_check_params(s, t, L) == B.RT_OK for t in f)
+    # rows of 4104 bf16 elements: 16-byte vectors only
+    f16 = B.tuner_derive_feasible(B.shape_of(64, 4104, "bf16", op=B.RT_OP_ADD_RMSNORM_FP8), L)
+    assert f16 and {t.vec_bytes for t in f16} == {16}
     assert B.tuner_check_params(B.shape_of(64, 4096, "fp32", op=B.RT_OP_ADD_RMSNORM_FP8), B.make_params(), L) == B.RT_ERR_DTYPE
     assert B.tuner_check_params(s, B.make_params(vec_bytes=8), L) == B.RT_ERR_INFEASIBLE
     # rows that are not 16-byte multiples have no instance of this variant

@@ -41,7 +41,8 @@ def test_every_feasible_theta_matches_oracle(B, oracle_lib, dtype, T, H):
     ro = torch.empty_like(xd)
     shape = B.shape_of(T, H, dtype, B._ptr_align(xd, rd, wd, ro), op=B.RT_OP_ADD_RMSNORM_FP8)
     thetas = B.tuner_derive_feasible(shape, heuristics=0)
-    assert thetas and {t.vec_bytes for t in thetas} == {16} and {t.reduce for t in thetas} == {0}
+    assert thetas and 16 in {t.vec_bytes for t in thetas} and {t.vec_bytes for t in thetas} <= {16, 32}
+    assert {t.reduce for t in thetas} == {0} and ((H * 2) % 32 != 0 or 32 in {t.vec_bytes for t in thetas})
     q_ref_d, scale_ref_d, r_ref_d = q_ref.cuda(), scale_ref.cuda(), r_ref.cuda()
     bad = []
     for th in thetas:
