@@ -84,8 +84,8 @@ typedef enum {
 typedef struct {
     int32_t threads_per_row; /* threads cooperating on one row (blockDim.x); power of two, 32..1024 */
     int32_t rows_per_cta;    /* rows handled by one CTA (blockDim.y); 1..8 */
-    int32_t vec_bytes;       /* bytes per ld/st: 32 (the 256-bit global accesses of sm_100; not for the fp8-output and
-                                all-reduce-fused norms), 16
+    int32_t vec_bytes;       /* bytes per ld/st: 32 (the 256-bit global accesses of sm_100; not for the all-reduce-fused
+                                norm), 16
                                 or 8 (4 and 2 exist as a narrow fall-back); 16 with
                                 RT_STAGE_REG_REALIGN, whatever the row length */
     int32_t unroll;          /* independent vector loads in flight per thread and tensor: 1, 2, 4 */
@@ -267,12 +267,13 @@ int silu_and_mul_template_launch(const rt_params* p, const void* x, void* out, i
 
 /*
  * add_rmsnorm with a quantised output for a following fp8 GEMM (a variant of the norm template: stage =
- * registers or TMA bulk, 16-byte vectors, shuffle reduction; bf16 and fp16 inputs).  No counterpart kernel
+ * registers or TMA bulk, 32- or 16-byte vectors, shuffle reduction; bf16 and fp16 inputs).  No counterpart kernel
  * in the paper; it is one of the "organization of shared memory and registers" variants its template axes
  * leave room for ("Tuning parameter selection and search space derivation").
  *   x, r, w   device, as for rmsnorm_template_launch.     r_out  device, the rounded residual (bit-exact contract).
  *   q         device, [n_tokens, hidden] bytes: e4m3 codes (4 exponent bits, bias 7, 3 significand bits, no
- *             infinities, largest finite value 448) of y / scale, round to nearest even, saturating.
+ *             infinities, largest finite value 448) of y / scale, round to nearest even, saturating.  Aligned to
+ *             vec_bytes / 2 bytes (8 or 16; RT_ERR_ALIGN otherwise).
  *   scale     device, [n_tokens] binary32: max(max_j |y_j|, 1e-12) / 448 with y the un-rounded norm output.
  * Asynchronous on `stream`, allocates nothing; infeasible theta is refused without launching.
  */
