@@ -67,7 +67,7 @@ _FP8_ENTRY = re.compile(r"Compiling entry function '_ZN2rt22add_rmsnorm_fp8_kern
                         r"EEvNS_7Fp8ArgsE'.*?(\d+) bytes spill stores.*?Used (\d+) registers(?:.*?(\d+) bytes smem)?", re.S)
 
 
-_ALLREDUCE_ENTRY = re.compile(r"Compiling entry function '_ZN2rt28add_rmsnorm_allreduce_kernelI(\w+?)Li(\d+)ELi(\d+)ELi(\d+)E"
+_ALLREDUCE_ENTRY = re.compile(r"Compiling entry function '_ZN2rt28add_rmsnorm_allreduce_kernelI(\w+?)Li(\d+)ELi(\d+)ELi(\d+)ELi(\d+)E"
                               r"EEvNS_13AllreduceArgsE'.*?(\d+) bytes spill stores.*?Used (\d+) registers(?:.*?(\d+) bytes smem)?", re.S)
 
 
@@ -92,8 +92,8 @@ def parse_ptxas(log: str) -> list[tuple]:
                          int(smem or 0), int(spill), 0))
         m = _ALLREDUCE_ENTRY.search("Compiling entry function" + block)
         if m:
-            t, parts, u, cap, spill, regs, smem = m.groups()
-            rows.append((4, _MANGLED_DTYPE[t], 16, 0, 0, int(u), int(cap), int(regs), int(smem or 0), int(spill), int(parts)))
+            t, vb, parts, u, cap, spill, regs, smem = m.groups()
+            rows.append((4, _MANGLED_DTYPE[t], int(vb), 0, 0, int(u), int(cap), int(regs), int(smem or 0), int(spill), int(parts)))
     return rows
 
 

@@ -29,14 +29,14 @@ struct AllreduceArgs {
     int n_y_outs, n_r_outs;
     long long row_begin, row_end;    // absolute rows handled by this launch
     int hidden;
-    int nvec;                        // 16-byte vectors in one row
+    int nvec;                        // vectors (16 or 32 bytes) in one row
     float eps;
 };
 
-template <typename T, int NP, int U, int CAP>
+template <typename T, int VB, int NP, int U, int CAP>
 __global__ void add_rmsnorm_allreduce_kernel(const AllreduceArgs a)
 {
-    constexpr int VB = 16;
+    static_assert(VB == 16 || VB == 32, "16- or 32-byte vectors");
     using C = Codec<T, VB>;
     constexpr int EPV = C::EPV;
     static_assert(NP >= 2 && NP <= kMaxParts, "2..8 parts");

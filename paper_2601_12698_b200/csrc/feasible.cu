@@ -34,10 +34,7 @@ std::vector<int> vec_levels(const rt_shape& s)
     const int64_t head_bytes = s.op == RT_OP_MERGE_ATTN_STATES && s.head_dim > 0 ? (int64_t)s.head_dim * eb : row_bytes;
     auto fits = [&](int vb) { return vb >= eb && row_bytes % vb == 0 && head_bytes % vb == 0 && s.min_ptr_align >= vb; };
     if (fits(32) || fits(16) || fits(8)) {
-        // the 256-bit accesses of sm_100: a level of the vector axis of every kernel but the all-reduce-fused
-        // norm, which is instantiated with 16-byte vectors only
-        if (s.op == RT_OP_ADD_RMSNORM_ALLREDUCE) return {16, 8};
-        return {32, 16, 8};
+        return {32, 16, 8};  // 32: the 256-bit global accesses of sm_100
     }
     if (fits(4)) return {4};
     if (fits(2)) return {2};
@@ -68,8 +65,8 @@ std::vector<rt_params> raw_grid(const rt_shape& s)
                 // the fp8-output norm: 32- or 16-byte vectors, shuffle reduction, register or TMA stage
                 if (s.op == RT_OP_ADD_RMSNORM_FP8 && (stage == RT_STAGE_SMEM_LDG || m.reduce != RT_REDUCE_SHFL || vb < 16))
                     continue;
-                // the all-reduce-fused norm: 16-byte vectors, shuffle reduction, register stage
-                if (s.op == RT_OP_ADD_RMSNORM_ALLREDUCE && (stage != RT_STAGE_REG || m.reduce != RT_REDUCE_SHFL || vb != 16))
+                // the all-reduce-fused norm: 32- or 16-byte vectors, shuffle reduction, register stage
+                if (s.op == RT_OP_ADD_RMSNORM_ALLREDUCE && (stage != RT_STAGE_REG || m.reduce != RT_REDUCE_SHFL || vb < 16))
                     continue;
                 for (int tpr : kTprLevels)
                     for (int rpc : kRpcLevels)

@@ -13,9 +13,9 @@
 // merge_attn_states: the same instance list as silu_and_mul.
 // fp8-output norm (16-bit element types, 32- and 16-byte vectors, shuffle reduction): register stage with CAP in
 // {1,2,4,8,16} (while the row stays within 128 fp32 registers per thread) and U <= CAP, TMA stage with U in {1,2,4}.
-// all-reduce-fused norm (16-byte vectors, register stage, shuffle reduction): 2, 4 and 8 parts, CAP in
-// {1,2,4,8,16} while the row stays within 128 fp32 registers per thread, U <= CAP with U * parts <= 16 loads of x
-// in flight per thread.
+// all-reduce-fused norm (32- and 16-byte vectors, register stage, shuffle reduction): 2, 4 and 8 parts, CAP in
+// {1,2,4,8,16} while the row stays within 128 fp32 registers per thread, U <= CAP with at most 256 bytes of x in flight
+// per thread (U * parts <= 16 with 16-byte vectors, <= 8 with 32-byte ones).
 #include "add_rmsnorm_allreduce_kernel.cuh"
 #include "add_rmsnorm_fp8_kernel.cuh"
 #include "add_rmsnorm_kernel.cuh"
@@ -69,20 +69,22 @@ rt::KernelEntry fp8_entry()
     fp8_entry<VB, 0, 4, 8>(), fp8_entry<VB, 0, 1, 16>(), fp8_entry<VB, 0, 2, 16>(), fp8_entry<VB, 0, 4, 16>(),       \
     fp8_entry<VB, 2, 1, 1>(), fp8_entry<VB, 2, 2, 1>(), fp8_entry<VB, 2, 4, 1>()
 
-template <int NP, int U, int CAP>
+template <int VB, int NP, int U, int CAP>
 rt::KernelEntry allreduce_entry()
 {
-    if constexpr (CAP * (16 / (int)sizeof(T)) > kMaxRowRegisters || U * NP > 16) {
-        return rt::KernelEntry{RT_OP_ADD_RMSNORM_ALLREDUCE, kDtype, 16, 0, 0, U, CAP, nullptr, NP};
+    // the row within 128 fp32 registers per thread, and at most 256 bytes of x in flight per thread
+    if constexpr (CAP * (VB / (int)sizeof(T)) > kMaxRowRegisters || U * NP * VB > 256) {
+        return rt::KernelEntry{RT_OP_ADD_RMSNORM_ALLREDUCE, kDtype, VB, 0, 0, U, CAP, nullptr, NP};
     } else {
-        return rt::KernelEntry{RT_OP_ADD_RMSNORM_ALLREDUCE, kDtype, 16, 0, 0, U, CAP,
-                               (const void*)&rt::add_rmsnorm_allreduce_kernel<T, NP, U, CAP>, NP};
+        return rt::KernelEntry{RT_OP_ADD_RMSNORM_ALLREDUCE, kDtype, VB, 0, 0, U, CAP,
+                               (const void*)&rt::add_rmsnorm_allreduce_kernel<T, VB, NP, U, CAP>, NP};
     }
 }
-#define RT_ALLREDUCE_LIST(NP)                                                                                     \
-    allreduce_entry<NP, 1, 1>(), allreduce_entry<NP, 1, 2>(), allreduce_entry<NP, 2, 2>(), allreduce_entry<NP, 1, 4>(), \
-    allreduce_entry<NP, 2, 4>(), allreduce_entry<NP, 4, 4>(), allreduce_entry<NP, 1, 8>(), allreduce_entry<NP, 2, 8>(), \
-    allreduce_entry<NP, 4, 8>(), allreduce_entry<NP, 1, 16>(), allreduce_entry<NP, 2, 16>(), allreduce_entry<NP, 4, 16>()
+#define RT_ALLREDUCE_LIST(VB, NP)                                                                                      \
+    allreduce_entry<VB, NP, 1, 1>(), allreduce_entry<VB, NP, 1, 2>(), allreduce_entry<VB, NP, 2, 2>(),                  \
+    allreduce_entry<VB, NP, 1, 4>(), allreduce_entry<VB, NP, 2, 4>(), allreduce_entry<VB, NP, 4, 4>(),                  \
+    allreduce_entry<VB, NP, 1, 8>(), allreduce_entry<VB, NP, 2, 8>(), allreduce_entry<VB, NP, 4, 8>(),                  \
+    allreduce_entry<VB, NP, 1, 16>(), allreduce_entry<VB, NP, 2, 16>(), allreduce_entry<VB, NP, 4, 16>()
 
 template <int VB, int ST, int U>
 rt::KernelEntry merge_entry()
@@ -126,7 +128,8 @@ std::vector<rt::KernelEntry> build_entries()
 #elif RT_UNIT_GROUP == 5
         RT_FP8_LIST(32), RT_FP8_LIST(16)
 #elif RT_UNIT_GROUP == 6
-        RT_ALLREDUCE_LIST(2), RT_ALLREDUCE_LIST(4), RT_ALLREDUCE_LIST(8)
+        RT_ALLREDUCE_LIST(32, 2), RT_ALLREDUCE_LIST(32, 4), RT_ALLREDUCE_LIST(32, 8), RT_ALLREDUCE_LIST(16, 2),
+        RT_ALLREDUCE_LIST(16, 4), RT_ALLREDUCE_LIST(16, 8)
 #elif RT_UNIT_GROUP == 7
         RT_REALIGN_LIST
 #elif RT_UNIT_GROUP == 4

@@ -306,9 +306,8 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
         plan->reject_reason = kRejectThreads;
         return RT_ERR_INFEASIBLE;
     }
-    if (!(vb == 32 || vb == 16 || vb == 8 || vb == 4 || vb == 2) || vb < eb || (vb == 32 && is_allreduce)) {
-        set_error("vec_bytes=%d is not 32 (not for the all-reduce-fused norm), 16, 8, 4 or 2, or is narrower than one "
-                  "element", vb);
+    if (!(vb == 32 || vb == 16 || vb == 8 || vb == 4 || vb == 2) || vb < eb) {
+        set_error("vec_bytes=%d is not 32, 16, 8, 4 or 2, or is narrower than one element", vb);
         plan->reject_reason = kRejectArgs;
         return RT_ERR_INFEASIBLE;
     }
@@ -347,8 +346,8 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
         plan->reject_reason = kRejectArgs;
         return RT_ERR_SHAPE;
     }
-    if (is_allreduce && (p->vec_bytes != 16 || p->reduce != RT_REDUCE_SHFL || p->cluster_size != 1 || p->stage != RT_STAGE_REG)) {
-        set_error("the all-reduce-fused norm takes 16-byte vectors, the shuffle reduction and the register stage "
+    if (is_allreduce && (p->vec_bytes < 16 || p->reduce != RT_REDUCE_SHFL || p->cluster_size != 1 || p->stage != RT_STAGE_REG)) {
+        set_error("the all-reduce-fused norm takes 32- or 16-byte vectors, the shuffle reduction and the register stage "
                   "(vec=%d reduce=%d cluster=%d stage=%d)", p->vec_bytes, p->reduce, p->cluster_size, p->stage);
         plan->reject_reason = kRejectArgs;
         return RT_ERR_INFEASIBLE;

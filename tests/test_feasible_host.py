@@ -56,14 +56,14 @@ def test_rules_bite_where_they_should(L):
     f = B.tuner_derive_feasible(B.shape_of(8192, 6148, "fp16"), L)
     assert {t.vec_bytes for t in row_vectors(f)} == {8} and {t.stage for t in f} == {0, 1, ragged}
     assert {t.vec_bytes for t in f if t.stage == ragged} == {16}
-    # rows of 8192 bf16 elements: all three widths of the vector axis; the all-reduce-fused norm stops at 16 bytes
+    # rows of 8192 bf16 elements: all three widths of the vector axis, for every kernel
     f = B.tuner_derive_feasible(B.shape_of(16384, 8192, "bf16"), L)
     assert {t.vec_bytes for t in f} == {8, 16, 32} and {t.stage for t in f if t.vec_bytes == 32} == {0, 1, 2}
     assert B.tuner_check_params(B.shape_of(16384, 8192, "bf16", min_ptr_align=16), B.make_params(vec_bytes=32), L) == B.RT_ERR_ALIGN
     assert B.tuner_check_params(B.shape_of(64, 8192, "bf16", op=B.RT_OP_SILU_AND_MUL), B.make_params(vec_bytes=32), L) == B.RT_OK
     assert B.tuner_check_params(B.shape_of(64, 8192, "bf16", op=B.RT_OP_ADD_RMSNORM_FP8), B.make_params(vec_bytes=32), L) == B.RT_OK
     assert B.tuner_check_params(B.shape_of(64, 8192, "bf16", op=B.RT_OP_ADD_RMSNORM_ALLREDUCE, n_parts=2),
-                                B.make_params(vec_bytes=32), L) == B.RT_ERR_INFEASIBLE
+                                B.make_params(vec_bytes=32), L) == B.RT_OK
     # 6152 fp16: 769 16-byte vectors (no 32-byte ones), both widths, the three aligned stages and no ragged-row stage
     f = B.tuner_derive_feasible(B.shape_of(8192, 6152, "fp16"), L)
     assert {t.vec_bytes for t in f} == {8, 16} and {t.stage for t in f} == {0, 1, 2}
@@ -180,8 +180,10 @@ def test_fp8_output_norm_grid(L):
 def test_allreduce_fused_norm_grid(L):
     s = B.shape_of(4096, 8192, "bf16", op=B.RT_OP_ADD_RMSNORM_ALLREDUCE, n_parts=4)
     f = B.tuner_derive_feasible(s, L)
-    assert f and {t.vec_bytes for t in f} == {16} and {t.stage for t in f} == {0} and {t.reduce for t in f} == {0}
+    assert f and {t.vec_bytes for t in f} == {16, 32} and {t.stage for t in f} == {0} and {t.reduce for t in f} == {0}
     assert all(B.tuner_check_params(s, t, L) == B.RT_OK for t in f)
+    # at most 256 bytes of x in flight per thread: four parts of 32-byte vectors allow unroll 1 and 2 only
+    assert {t.unroll for t in f if t.vec_bytes == 32} == {1, 2} and {t.unroll for t in f if t.vec_bytes == 16} == {1, 2, 4}
     c = B.tuner_derive_counts(s, L)
     assert c["feasible"] == len(f) and sum(v for k, v in c.items() if k != "raw") == c["raw"] == len(B.tuner_raw_grid(s))
     # eight parts leave no instance with four vectors per part in flight

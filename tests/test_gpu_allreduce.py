@@ -48,7 +48,8 @@ def test_group_emulated_on_one_gpu_every_theta(B, oracle_lib, dtype, n_parts, T,
     y_ref_d, r_ref_d = y_ref.cuda(), r_ref.cuda()
     shape = B.shape_of(max(1, (T + n_parts - 1) // n_parts), H, dtype, op=B.RT_OP_ADD_RMSNORM_ALLREDUCE, n_parts=n_parts)
     thetas = B.tuner_derive_feasible(shape, heuristics=0)
-    assert thetas and {t.stage for t in thetas} == {0} and {t.vec_bytes for t in thetas} == {16}
+    assert thetas and {t.stage for t in thetas} == {0} and 16 in {t.vec_bytes for t in thetas} and \
+        {t.vec_bytes for t in thetas} <= {16, 32}
     # guard bands around every destination
     n = T * H
     y_full = torch.zeros(n_parts, n + 256, dtype=pd.dtype, device="cuda")
