@@ -84,8 +84,7 @@ typedef enum {
 typedef struct {
     int32_t threads_per_row; /* threads cooperating on one row (blockDim.x); power of two, 32..1024 */
     int32_t rows_per_cta;    /* rows handled by one CTA (blockDim.y); 1..8 */
-    int32_t vec_bytes;       /* bytes per ld/st: 32 (the 256-bit global accesses of sm_100; not for the all-reduce-fused
-                                norm), 16
+    int32_t vec_bytes;       /* bytes per ld/st: 32 (the 256-bit global accesses of sm_100), 16
                                 or 8 (4 and 2 exist as a narrow fall-back); 16 with
                                 RT_STAGE_REG_REALIGN, whatever the row length */
     int32_t unroll;          /* independent vector loads in flight per thread and tensor: 1, 2, 4 */
@@ -283,7 +282,7 @@ int rmsnorm_fp8_template_launch(const rt_params* p, const void* x, const void* r
 
 /*
  * The tensor-parallel form of add_rmsnorm: the all-reduce that precedes the operator in tensor-parallel
- * serving is folded into the kernel (a variant of the norm template: register stage, 16-byte vectors, shuffle
+ * serving is folded into the kernel (a variant of the norm template: register stage, 32- or 16-byte vectors, shuffle
  * reduction; axes threads per row, rows per CTA, unroll).  No counterpart in the paper, whose experiments run
  * on one GPU; the operator is its `fused_add_rmsnorm` ("Kernels") with x = sum over ranks of x^(k).
  *
