@@ -8,8 +8,11 @@ seeded synthetic input.  The workload is the prefill configuration (bf16, 16384 
 bandwidth metric is quoted on.  Before the timed region the tuner runs once (not timed): the guided search,
 and the exhaustive sweep it is compared with.  Rank 0 prints one JSON line.
 
-N > 1 (torchrun): every rank owns its own block of rows of an N-times larger job (weak scaling); there is
-no data-path collective, only a barrier and the max over ranks of the measured time.
+N > 1: one process per GPU.  Under a launcher (RANK / WORLD_SIZE in the environment, e.g. torchrun) this process
+is one rank; started plainly with --gpus N > 1 it starts the N ranks itself.  Every rank owns its own block of rows
+of an N-times larger job (weak scaling); there is no data-path collective, only a barrier and the max over ranks of
+the measured time.  The c3ar* workloads (the tensor-parallel form of the norm) are the exception: with N equal to
+their group size they run the all-reduce-fused kernel over the ranks' peer-mapped buffers.
 
 --impl reference times the CPU oracle (the deliberately plain checker) on the host cores, on a bounded
 sample of the same workload.
@@ -20,8 +23,10 @@ import argparse
 import hashlib
 import json
 import os
+import socket
+import subprocess
 import sys
-import threading
+import tempfile
 import time
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
@@ -46,28 +51,26 @@ DEFAULT_WORKLOAD = "c3_prefill_bf16_16384x8192"
 FALLBACK_HBM_GBS = 6650.0  # used only when MEASURED_PEAKS.json is absent
 NOMINAL_HBM_GBS = 8000.0
 
-# DRAM traffic of one launch of the top kernel from an ncu capture (dram__bytes_read.sum +
-# dram__bytes_write.sum), valid only for the kernel source and theta it was taken on.
+# DRAM traffic of one launch of the top kernel from ncu captures (dram__bytes_read.sum + dram__bytes_write.sum),
+# keyed by workload and theta (tpr, rpc, vec, unroll, stage, reduce, cluster).  Each entry names the hash of the kernel
+# header it was captured on: the bench prints the figure as `traffic` only while that hash is the current one, and
+# prints the capture with both hashes beside it either way (`traffic_capture`).
 NCU_TRAFFIC = {
-    "kernel_sha256_16": "ca1f28704284bed6",
-    # workload -> (threads_per_row, rows_per_cta, vec_bytes, unroll, stage, reduce, cluster_size) -> DRAM bytes per launch
-    "bytes_per_launch": {
-        "c3_prefill_bf16_16384x8192": {
-            (256, 1, 32, 2, 0, 0, 1): 1020995584,  # 536.94 MB read + 484.06 MB written (--set full capture)
-            (256, 1, 16, 1, 2, 0, 1): 1020571136,  # 536.91 MB read + 483.67 MB written (--set full capture)
-            # the other configurations the search has returned on this shape (dram__bytes metrics only, first of two launches)
-            (256, 2, 32, 2, 0, 0, 1): 1020452352,
-            (256, 1, 32, 2, 0, 1, 1): 1019887104,
-            (512, 1, 32, 1, 0, 0, 1): 1026409216,
-            (256, 1, 32, 1, 2, 0, 1): 1022494720,
-            (256, 2, 32, 2, 2, 0, 1): 1022360832,
-            (256, 1, 16, 4, 0, 0, 1): 1019570944,
-            (512, 1, 16, 2, 0, 0, 1): 1019498752,
-            (256, 1, 16, 2, 2, 0, 1): 1019478272,
-        },
-        # the ragged-row stage; 201.42 MB read + 153.50 MB written (a quarter of the output is still dirty in L2 at the end)
-        "c4x_fp16_8192x6145": {(256, 1, 16, 4, 3, 0, 1): 354928640},
+    "c3_prefill_bf16_16384x8192": {
+        (256, 1, 32, 2, 0, 0, 1): (1020995584, "ca1f28704284bed6"),  # 536.94 MB read + 484.06 MB written (--set full)
+        (256, 1, 16, 1, 2, 0, 1): (1020571136, "ca1f28704284bed6"),  # 536.91 MB read + 483.67 MB written (--set full)
+        # the other configurations the search has returned on this shape (dram__bytes metrics only, first of two launches)
+        (256, 2, 32, 2, 0, 0, 1): (1020452352, "ca1f28704284bed6"),
+        (256, 1, 32, 2, 0, 1, 1): (1019887104, "ca1f28704284bed6"),
+        (512, 1, 32, 1, 0, 0, 1): (1026409216, "ca1f28704284bed6"),
+        (256, 1, 32, 1, 2, 0, 1): (1022494720, "ca1f28704284bed6"),
+        (256, 2, 32, 2, 2, 0, 1): (1022360832, "ca1f28704284bed6"),
+        (256, 1, 16, 4, 0, 0, 1): (1019570944, "ca1f28704284bed6"),
+        (512, 1, 16, 2, 0, 0, 1): (1019498752, "ca1f28704284bed6"),
+        (256, 1, 16, 2, 2, 0, 1): (1019478272, "ca1f28704284bed6"),
     },
+    # the ragged-row stage; 201.42 MB read + 153.50 MB written (a quarter of the output is still dirty in L2 at the end)
+    "c4x_fp16_8192x6145": {(256, 1, 16, 4, 3, 0, 1): (354928640, "ca1f28704284bed6")},
 }
 
 
@@ -76,65 +79,126 @@ def kernel_source_hash() -> str:
     return hashlib.sha256(open(path, "rb").read()).hexdigest()[:16]
 
 
+def ncu_traffic(workload: str, theta_key: tuple):
+    """(traffic or None, description of the capture or None) for the roofline object."""
+    hit = NCU_TRAFFIC.get(workload, {}).get(tuple(theta_key))
+    if hit is None:
+        return None, None
+    nbytes, captured_on = hit
+    current = kernel_source_hash()
+    info = {"bytes_per_launch": nbytes, "kernel_sha256_16_at_capture": captured_on, "kernel_sha256_16_now": current,
+            "current": captured_on == current}
+    return (nbytes if captured_on == current else None), info
+
+
+_SAMPLER_SOURCE = r"""
+import sys, time
+import pynvml as nv
+nv.nvmlInit()
+uuid, index, period = sys.argv[1], int(sys.argv[2]), float(sys.argv[3])
+try:
+    h = nv.nvmlDeviceGetHandleByUUID(uuid.encode()) if uuid else nv.nvmlDeviceGetHandleByIndex(index)
+except Exception:
+    h = nv.nvmlDeviceGetHandleByIndex(index)
+sys.stdout.write("max %d\n" % nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM))
+sys.stdout.flush()
+while True:
+    t = time.monotonic()
+    mhz = nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)
+    try:
+        bits = nv.nvmlDeviceGetCurrentClocksEventReasons(h)
+    except Exception:
+        bits = nv.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+    sys.stdout.write("%.6f %d %d\n" % (t, mhz, bits))
+    sys.stdout.flush()
+    time.sleep(period)
+"""
+
+
 class ClockSampler:
-    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
+    """SM clock and clock-event reasons of one GPU, read through NVML (reading only) by a child process while the
+    measurements run.  A child process, not a thread: the timed loop holds the interpreter, and a sampling thread
+    would get a turn every few milliseconds at best.  Samples carry CLOCK_MONOTONIC times, so any interval of this
+    process's own clock can be looked up afterwards."""
 
     REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
                0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting"}
 
-    def __init__(self, torch_device, period_s: float = 0.002):
-        self.period = period_s
-        self.samples: list[int] = []
-        self.reason_bits = 0
+    def __init__(self, torch_device, period_s: float = 0.0005):
+        self.proc = None
         self.max_mhz = None
-        self.handle = None
-        self._stop = threading.Event()
-        self._thread = None
+        self.samples: list[tuple[float, int, int]] = []
+        self._parsed = 0
         try:
-            import pynvml
             import torch
-            self.nv = pynvml
-            pynvml.nvmlInit()
             props = torch.cuda.get_device_properties(torch_device)
-            try:
-                self.handle = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + str(props.uuid)).encode())
-            except Exception:
-                self.handle = pynvml.nvmlDeviceGetHandleByIndex(torch_device.index or 0)
-            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM))
+            uuid = "GPU-" + str(props.uuid) if getattr(props, "uuid", None) is not None else ""
+            self.out = tempfile.NamedTemporaryFile("w+", prefix="clocks_", suffix=".txt", delete=True)
+            self.proc = subprocess.Popen([sys.executable, "-c", _SAMPLER_SOURCE, uuid, str(torch_device.index or 0),
+                                          str(period_s)], stdout=self.out, stderr=subprocess.DEVNULL)
         except Exception:
-            self.handle = None
+            self.proc = None
 
-    def _loop(self):
-        nv = self.nv
-        while not self._stop.is_set():
+    def wait_ready(self, timeout_s: float = 20.0) -> None:
+        """Returns once the child has delivered its first sample (or has died, or the time is up)."""
+        t0 = time.monotonic()
+        while self.proc is not None and self.proc.poll() is None and time.monotonic() - t0 < timeout_s:
+            if len(self._read()) > 0:
+                return
+            time.sleep(0.01)
+
+    def _read(self):
+        if self.proc is None:
+            return self.samples
+        with open(self.out.name) as f:
+            f.seek(self._parsed)
+            text = f.read()
+        done = text.rfind("\n") + 1  # whole lines only: a line cut off in mid-write comes again complete
+        for line in text[:done].splitlines():
+            parts = line.split()
+            if len(parts) == 2 and parts[0] == "max":
+                self.max_mhz = int(parts[1])
+            elif len(parts) == 3:
+                self.samples.append((float(parts[0]), int(parts[1]), int(parts[2])))
+        self._parsed += done
+        return self.samples
+
+    def stop(self) -> None:
+        if self.proc is not None:
+            self._read()
+            self.proc.terminate()  # this very child, by its handle
             try:
-                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.handle, nv.NVML_CLOCK_SM)))
-                try:
-                    bits = nv.nvmlDeviceGetCurrentClocksEventReasons(self.handle)
-                except Exception:
-                    bits = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle)
-                self.reason_bits |= int(bits)
+                self.proc.wait(timeout=5)
             except Exception:
-                pass
-            time.sleep(self.period)
+                self.proc.kill()
+            self._read()
+            self.proc = None
 
-    def __enter__(self):
-        if self.handle is not None:
-            self._thread = threading.Thread(target=self._loop, daemon=True)
-            self._thread.start()
-        return self
-
-    def __exit__(self, *exc):
-        self._stop.set()
-        if self._thread is not None:
-            self._thread.join()
-
-    def summary(self) -> dict:
-        if not self.samples:
+    def window(self, t_begin: float, t_end: float, widen_to: int = 3) -> dict:
+        """Median SM clock and the union of the reasons over [t_begin, t_end] (time.monotonic() values).  A window
+        with fewer than `widen_to` samples is widened to its nearest samples on either side, and says so."""
+        samples = self._read()
+        inside = [s for s in samples if t_begin <= s[0] <= t_end]
+        widened = False
+        if len(inside) < widen_to and samples:
+            mid = 0.5 * (t_begin + t_end)
+            inside = sorted(samples, key=lambda s: abs(s[0] - mid))[:widen_to]
+            widened = True
+        if not inside:
             return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
-        s = sorted(self.samples)
-        return {"sm_mhz": s[len(s) // 2], "sm_max_mhz": self.max_mhz, "samples": len(s),
-                "reasons": sorted(name for bit, name in self.REASONS.items() if self.reason_bits & bit)}
+        mhz = sorted(s[1] for s in inside)
+        bits = 0
+        for s in inside:
+            bits |= s[2]
+        out = {"sm_mhz": mhz[len(mhz) // 2], "sm_min_mhz": mhz[0], "sm_max_mhz": self.max_mhz, "samples": len(inside),
+               "reasons": sorted(name for bit, name in self.REASONS.items() if bits & bit)}
+        if widened:
+            out["window"] = "widened to the nearest samples around the timed region"
+        return out
+
+    def median_mhz(self, t_begin: float, t_end: float):
+        w = self.window(t_begin, t_end, widen_to=1)
+        return w["sm_mhz"]
 
 
 def measured_hbm_peak() -> tuple[float, str]:
@@ -216,13 +280,44 @@ def run_reference(args) -> None:
         "impl": "reference", "metric": METRICS[wl.op], "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": elapsed * 1e3 / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
-        "config": {"workload": wl.name, "n_tokens": wl.n_tokens, "hidden": wl.hidden, "sample_rows_per_step": rows,
-                   "bytes": BYTES_LABEL[wl.op]},
+        "config": {"workload": wl.name, "n_tokens_per_gpu": wl.n_tokens, "hidden": wl.hidden, "eps": wl.eps,
+                   "sample_rows_per_step": rows, "bytes": BYTES_LABEL[wl.op]},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line), flush=True)
+
+
+def fastest_of(log, k: int) -> list:
+    """The k fastest distinct thetas of a search log that passed their gate (a theta's last record counts)."""
+    last = {}
+    for rec in log:
+        last[rec.params.key()] = rec
+    good = sorted((rec for rec in last.values() if rec.status == 0), key=lambda rec: rec.us)
+    return [rec.params for rec in good[:k]]
+
+
+def resume_seeds(path: str, workload: str, k: int = 8) -> list:
+    """Resume: the fastest thetas of an earlier search log (the JSONL file --log writes) become the seeds of this
+    search, so it starts where that one stopped.  Records of other workloads in the file are seeds as well, after
+    this workload's own (configurations found on other shapes; the tuner skips those that are infeasible here)."""
+    from paper_2601_12698_b200 import binding as B
+    own, other = {}, {}
+    with open(path) as f:
+        for line in f:
+            line = line.strip()
+            if not line:
+                continue
+            rec = json.loads(line)
+            if rec.get("status") != 0 or not rec.get("us"):
+                continue
+            th = rec["params"]
+            key = tuple(int(th[name]) for name, _ in B.rt_params._fields_)
+            table = own if rec.get("workload") == workload else other
+            table[key] = min(float(rec["us"]), table.get(key, float("inf")))
+    ranked = sorted(own, key=own.get)[:k] + sorted(other, key=other.get)[:k]
+    return [B.rt_params(*key) for key in ranked]
 
 
 # ---- our arm ----------------------------------------------------------------------------------------------------
@@ -239,6 +334,8 @@ def run_ours(args) -> None:
     torch.cuda.set_device(device)
     dp.init(device=device)
     wl = synth.workloads()[args.workload]
+    if wl.op == "add_rmsnorm_allreduce" and world > 1:
+        return run_tensor_parallel(args, wl, rank, world, device)
     shard = dp.weak_shard(wl.n_tokens, rank, world)
     b = synth.DTYPE_BYTES[wl.dtype]
     T, H = wl.n_tokens, wl.hidden
@@ -294,8 +391,19 @@ def run_ours(args) -> None:
     if world == 1:
         cpu_baseline = {"value": wl.algorithmic_bytes / oracle_s / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
                         "sample": f"one pass over all {T} rows of {wl.name}, {cores} threads, {oracle_s:.2f} s"}
+        if wl.op == "add_rmsnorm":
+            # the same oracle on one thread, on the first rows of the workload (about two seconds of work)
+            rows1 = int(max(1, min(T, T * 2.0 / max(oracle_s * cores, 1e-6))))
+            t0 = time.perf_counter()
+            oracle.add_rmsnorm(x[:rows1], r[:rows1], w, wl.eps, threads=1)
+            one_s = time.perf_counter() - t0
+            cpu_baseline["single_thread"] = {
+                "value": (4 * b * rows1 * H + b * H) / one_s / 1e9, "unit": UNIT, "cores": 1,
+                "sample": f"first {rows1} of {T} rows, 1 thread, {one_s:.2f} s"}
 
     stream = torch.cuda.Stream(device=device)
+    clock_sampler = ClockSampler(device)  # a child process that only reads NVML; stopped before the line is printed
+    clock_sampler.wait_ready()
     limits = B.rt_query_limits()
     # A workload that fits in L2 is timed over a ring of identical input/output sets larger than L2, so that
     # every timed launch reads from DRAM; the large workloads exceed L2 on their own.
@@ -338,36 +446,76 @@ def run_ours(args) -> None:
         tuner = {"skipped": "theta given on the command line"}
     elif rank == 0:
         counts = B.tuner_derive_counts(shape)
+        # Both searches time every candidate with the paper's protocol (20 warm-up launches, blocks of 100).
         t0 = time.perf_counter()
-        sweep, sweep_log = B.tuner_search(shape, B.make_budget(max_evals=counts["feasible"] + args.top_k, warmup=10,
-                                                               iters=50, repeats=2, top_k=args.top_k,
-                                                               strategy=B.RT_SEARCH_EXHAUSTIVE, use_graph=use_graph), ws)
+        sweep, sweep_log = B.tuner_search(shape, B.make_budget(max_evals=counts["feasible"], warmup=20, iters=100, repeats=2,
+                                                               top_k=0, strategy=B.RT_SEARCH_EXHAUSTIVE,
+                                                               use_graph=use_graph), ws)
         sweep_s = time.perf_counter() - t0
+        seeds = resume_seeds(args.resume, wl.name) if args.resume else None
         t0 = time.perf_counter()
         guided, guided_log = B.tuner_search(shape, B.make_budget(max_evals=args.search_budget, warmup=20, iters=100,
-                                                                 repeats=3, top_k=args.top_k, use_graph=use_graph), ws)
+                                                                 repeats=3, top_k=args.top_k, use_graph=use_graph,
+                                                                 seeds=seeds), ws)
         guided_s = time.perf_counter() - t0
-        # head-to-head re-timing of the two winners with the paper's protocol (20 warm-up, 100 timed)
-        proto = B.make_budget(warmup=20, iters=100, repeats=5, use_graph=use_graph)
-        t_guided = B.tuner_evaluate(shape, guided.best, proto, ws)
-        t_sweep = B.tuner_evaluate(shape, sweep.best, proto, ws)
-        t_cold = B.tuner_evaluate(shape, guided.best, proto, ws_cold)
-        floor_us = B.tuner_launch_floor(proto, stream=stream)
+        # Search-best against exhaustive-best, measured side by side: the sweep's fastest --retest-top points, the
+        # guided winner and its runner-up are re-timed together, block by block in rotation (20 warm-up + 100 timed
+        # launches per block), so that every candidate meets the same clocks.  exhaustive_best is the fastest of
+        # that set (the guided winner belongs to the feasible set the sweep covers, so it is a member by right).
+        finalists = []
+        for th in (fastest_of(sweep_log, args.retest_top) + [guided.best] + fastest_of(guided_log, 2)):
+            if th.key() not in [f.key() for f in finalists]:
+                finalists.append(th)
+        proto = B.make_budget(warmup=20, iters=100, repeats=1, use_graph=use_graph)
+        recs, blocks = B.tuner_retest_interleaved(shape, finalists, proto, ws, args.retest_rounds)
+        i_guided = [f.key() for f in finalists].index(guided.best.key())
+        ok = [i for i, rec in enumerate(recs) if rec.status == 0]
+        if i_guided not in ok:
+            raise RuntimeError(f"the guided winner failed its re-test: status {recs[i_guided].status}")
+        i_best = min(ok, key=lambda i: recs[i].us)
+        per = {i: [blk for blk in blocks if blk.theta_index == i] for i in ok}
+        mhz = {i: [clock_sampler.median_mhz(blk.t_begin_s, blk.t_end_s) for blk in per[i]] for i in ok}
+
+        def normalised(i):  # median over blocks of (time x SM clock): cycles per launch, in us x MHz
+            vals = sorted(blk.us * m for blk, m in zip(per[i], mhz[i]) if m)
+            return vals[len(vals) // 2] if vals else None
+        round_ratio = sorted(per[i_guided][k].us / min(per[i][k].us for i in ok) for k in range(args.retest_rounds))
+        norm_guided, norm_best = normalised(i_guided), min((normalised(i) for i in ok if normalised(i)), default=None)
+        t_guided, t_sweep = recs[i_guided], recs[i_best]
+        t_cold = B.tuner_evaluate(shape, guided.best, B.make_budget(warmup=20, iters=100, repeats=5, use_graph=use_graph), ws_cold)
+        floor_us = B.tuner_launch_floor(B.make_budget(warmup=20, iters=100, repeats=5, use_graph=use_graph), stream=stream)
         theta = guided.best
         tuner = {
             "feasible": counts["feasible"], "raw_grid": counts["raw"], "pruned": {k: v for k, v in counts.items()
                                                                                  if k not in ("feasible", "raw") and v},
             "search_budget_evals": args.search_budget, "search_evals_used": guided.evals_used,
             "search_best": theta_dict(guided.best), "search_best_us": round(t_guided.us, 3),
-            "exhaustive_best": theta_dict(sweep.best), "exhaustive_best_us": round(t_sweep.us, 3),
+            "exhaustive_best": theta_dict(finalists[i_best]), "exhaustive_best_us": round(t_sweep.us, 3),
             "exhaustive_evals": sweep.evals_used, "failed_gate": guided.n_failed_gate + sweep.n_failed_gate,
             "search_vs_exhaustive": round(t_guided.us / t_sweep.us, 4),
+            "search_vs_exhaustive_clock_normalised": (round(norm_guided / norm_best, 4) if norm_guided and norm_best else None),
+            "retest": {
+                "rule": ("sweep top-%d + guided winner + guided runner-up re-timed together, %d rounds in rotation, "
+                         "20 warm-up + 100 timed launches per block; score = median block; exhaustive_best = fastest "
+                         "of the set" % (args.retest_top, args.retest_rounds)),
+                "per_round_ratio_min_median_max": [round(round_ratio[0], 4), round(round_ratio[len(round_ratio) // 2], 4),
+                                                   round(round_ratio[-1], 4)],
+                "candidates": [{"theta": list(finalists[i].key()), "us": round(recs[i].us, 3),
+                                "us_min": round(recs[i].us_min_block, 3),
+                                "spread": round((max(blk.us for blk in per[i]) - recs[i].us_min_block) / recs[i].us, 4),
+                                "sm_mhz": sorted(m for m in mhz[i] if m)[len([m for m in mhz[i] if m]) // 2] if any(mhz[i]) else None,
+                                "us_x_mhz": round(normalised(i), 1) if normalised(i) else None,
+                                "from": ("guided" if i == i_guided else "sweep" if i < args.retest_top else "guided runner-up")}
+                               for i in ok],
+            },
             "timing": ("CUDA graph of 100 launches, same buffers (L2-warm)" if use_graph else
                        "100 back-to-back launches, same buffers (exceed L2)"),
             "search_best_cold_us": round(t_cold.us, 3), "ring_sets": sets, "empty_kernel_us": round(floor_us, 3),
             "search_seconds": round(guided_s, 2), "exhaustive_seconds": round(sweep_s, 2),
             "occupancy_blocks_per_sm": t_guided.occupancy_blocks_per_sm, "regs_per_thread": t_guided.regs_per_thread,
         }
+        if seeds:
+            tuner["resumed_seeds"] = len(seeds)
         if args.seed_thetas:
             # Cross-shape transfer: the same small budget, cold and seeded with configurations found on other
             # shapes; "evaluations to within 3%" counts evaluations until one scores within 3% of the
@@ -461,20 +609,24 @@ def run_ours(args) -> None:
             if st != 0:
                 raise B.TunerError(st, "rmsnorm_template_launch")
 
+    t_warm = time.monotonic()
     for k in range(args.warmup):
         step(k)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     dp.barrier(device)
     launches_before = B.rt_launch_count()
-    with ClockSampler(device) as clocks:
-        with torch.cuda.stream(stream):
-            e0.record(stream)
-            for k in range(args.steps):
-                step(k)
-            e1.record(stream)
-        e1.synchronize()
-        dp.barrier(device)
+    t_begin = time.monotonic()
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        for k in range(args.steps):
+            step(k)
+        e1.record(stream)
+    e1.synchronize()
+    t_end = time.monotonic()
+    dp.barrier(device)
     gpu_launches = B.rt_launch_count() - launches_before
+    clocks = clock_sampler.window(t_begin, t_end)
+    clocks["warmup_and_timed"] = clock_sampler.window(t_warm, t_end)
     ms_local = e0.elapsed_time(e1)
     ms = dp.max_over_ranks(ms_local, device)
     value = dp.whole_job_rate(wl.algorithmic_bytes, args.steps, world, ms) / 1e9
@@ -582,9 +734,7 @@ def run_ours(args) -> None:
         peak, peak_kind = measured_hbm_peak()
         per_launch_ms = ms_local / args.steps
         achieved = wl.algorithmic_bytes / (per_launch_ms * 1e-3) / 1e9
-        traffic = None
-        if NCU_TRAFFIC["kernel_sha256_16"] == kernel_source_hash():
-            traffic = NCU_TRAFFIC["bytes_per_launch"].get(wl.name, {}).get(tuple(theta_dict(theta).values()))
+        traffic, traffic_capture = ncu_traffic(wl.name, theta.key())
         line = {
             "metric": METRICS[wl.op], "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
@@ -597,20 +747,171 @@ def run_ours(args) -> None:
             "value_nominal_5_access_gbs": value * wl.nominal_bytes / wl.algorithmic_bytes,
             "frac_of_8TBs": value / world / NOMINAL_HBM_GBS,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": UNIT, "frac": achieved / peak,
-                         "traffic": traffic, "peak_kind": f"of {peak_kind}", "kernel": KERNEL_NAME[wl.op],
+                         "traffic": traffic, "traffic_capture": traffic_capture, "peak_kind": f"of {peak_kind}",
+                         "kernel": KERNEL_NAME[wl.op],
                          "algorithmic_bytes_per_launch": wl.algorithmic_bytes},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d_bytes,
                     "d2h_bytes_per_step": d2h_bytes, "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
             "gpu_launches": int(gpu_launches),
-            "clocks": clocks.summary(),
+            "clocks": clocks,
             "parity": {"r_out_bit_mismatches": int(r_bad), "y_beyond_tolerance": int(y_bad), "y_worst": y_worst,
                        "rows_checked": T},
             "tuner": tuner,
         }
         if cpu_baseline is not None:
             line["cpu_baseline"] = cpu_baseline
+        clock_sampler.stop()
         print(json.dumps(line), flush=True)
+    clock_sampler.stop()
     dp.shutdown()
+
+
+NVLINK_PEER_GBS = 770.0  # measured peer copy per direction on this kind of machine (nominal 900)
+
+
+def run_tensor_parallel(args, wl, rank: int, world: int, device) -> None:
+    """The c3ar* workloads on a real group: world == the workload's group size, one rank per GPU, every rank's partial
+    x, y and r_out in symmetric memory.  A step is dp.FusedAllreduceNorm: the group meets, each rank's launch reads
+    its block of rows of every rank's partial through plain peer loads and stores its rows of y into every rank's
+    tensor, the group meets again.  No TMA and no multicast of any kind is involved."""
+    import torch
+    from paper_2601_12698_b200 import binding as B
+    from paper_2601_12698_b200 import dp, synth
+    import oracle
+    if world != wl.n_parts:
+        raise SystemExit(f"{wl.name} is a group of {wl.n_parts}: start it with --gpus {wl.n_parts} (got {world} ranks)")
+    T, H, b = wl.n_tokens, wl.hidden, synth.DTYPE_BYTES[wl.dtype]
+    tdtype = synth.TORCH_DTYPES[wl.dtype]
+    stream = torch.cuda.Stream(device=device)
+    group = dp.fused_allreduce_norm(T, H, tdtype, device)
+    shard = group.shard
+    parts = synth.make_parts(0, T, H, wl.dtype, wl.seed, world, wl.dist)       # every rank draws all parts: the oracle needs them
+    r = synth.make_rows(synth.TENSOR_R, 0, T, H, wl.dtype, wl.seed, wl.dist).contiguous()
+    w = synth.make_weight(H, wl.dtype, wl.seed, wl.dist)
+    y_ref, r_ref = oracle.allreduce_add_rmsnorm(parts, r, w, wl.eps, threads=os.cpu_count() or 1)
+    mine_host = parts[rank].contiguous().pin_memory()
+    group.x_parts[rank].copy_(mine_host)
+    rd, wd = r.to(device), w.to(device)
+    # theta: the shipped table's entry for (rows of one block, hidden, parts); rank 0 decides for the group
+    shape = B.shape_of(max(1, shard.rows), H, wl.dtype, op=B.RT_OP_ADD_RMSNORM_ALLREDUCE, n_parts=world)
+    key = list(B.SpecTable.default().lookup(shape)[0].key()) if rank == 0 else [0] * 7
+    theta = B.rt_params(*dp.broadcast_ints(key, device))
+    clock_sampler = ClockSampler(device)
+    clock_sampler.wait_ready()
+
+    def step():
+        group(theta, rd, wd, wl.eps, stream=stream)
+    for _ in range(args.warmup):
+        step()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    dp.barrier(device)
+    launches_before = B.rt_launch_count()
+    t_begin = time.monotonic()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    e1.synchronize()
+    t_end = time.monotonic()
+    dp.barrier(device)
+    gpu_launches = B.rt_launch_count() - launches_before
+    ms = dp.max_over_ranks(e0.elapsed_time(e1), device)
+    # parity: this rank's copy of every row of y, and the residual of its own block
+    y_worst, y_bad = B.tuner_compare(group.y_outs[rank], y_ref.to(device), B.RT_CMP_REL32 if wl.dtype == "fp32" else B.RT_CMP_ULP16,
+                                     1e-5 if wl.dtype == "fp32" else 2.0, stream=stream)
+    rows = slice(shard.row_begin, shard.row_end)
+    r_bad = B.tuner_compare(group.r_outs[rank][rows], r_ref[rows].to(device), B.RT_CMP_BITS, stream=stream)[1] if shard.rows else 0
+    bad = dp.sum_over_ranks(float(y_bad + r_bad), device)
+    if bad or B.rt_device_status() != 0:
+        raise RuntimeError(f"rank {rank}: the group's outputs differ from the oracle (y_bad={y_bad}, r_bad={r_bad})")
+    # end to end: this rank's partial comes from pinned host memory and its y goes back, inside the timed region
+    y_host = torch.empty((T, H), dtype=tdtype).pin_memory()
+    e2e_steps = max(3, min(args.steps, args.e2e_steps))
+
+    def e2e_step():
+        with torch.cuda.stream(stream):
+            group.x_parts[rank].copy_(mine_host, non_blocking=True)
+        step()
+        with torch.cuda.stream(stream):
+            y_host.copy_(group.y_outs[rank], non_blocking=True)
+        stream.synchronize()
+    e2e_step()
+    dp.barrier(device)
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e2e_ms = dp.max_over_ranks((time.perf_counter() - t0) * 1e3, device)
+    dp.barrier(device)
+    if oracle.compare_y(y_host[-64:], y_ref[-64:], tol_rel=1e-5)[1]:
+        raise RuntimeError("end-to-end path fails parity")
+    if rank == 0:
+        step_s = ms * 1e-3 / args.steps
+        link_bytes = 2.0 * (world - 1) / world * T * H * b   # per GPU and direction: peers' parts in, y out
+        hbm_bytes = (3 + 2.0 / world) * T * H * b + H * b     # per GPU: parts and y of all rows, r and r' of its block
+        hbm_peak, peak_kind = measured_hbm_peak()
+        bound_s = max(link_bytes / (NVLINK_PEER_GBS * 1e9), hbm_bytes / (hbm_peak * 1e9))
+        line = {
+            "metric": METRICS[wl.op], "value": wl.algorithmic_bytes / step_s / 1e9, "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+            "scaling": "strong", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
+            "config": {"workload": wl.name, "n_tokens": T, "hidden": H, "eps": wl.eps, "l2": "inputs_exceed_l2",
+                       "bytes": "per element: one partial per rank and r read, y and r' written once (what the group must move)",
+                       "parallelism": f"tensor-parallel group of {world}: all-reduce fused into the norm over peer-mapped memory",
+                       "theta": theta_dict(theta)},
+            "roofline": {"bound": "nvlink" if link_bytes / NVLINK_PEER_GBS > hbm_bytes / hbm_peak else "hbm",
+                         "achieved": link_bytes / step_s / 1e9, "peak": NVLINK_PEER_GBS, "unit": UNIT,
+                         "frac": bound_s / step_s, "traffic": None, "peak_kind": f"slower of link bytes / {NVLINK_PEER_GBS:.0f} GB/s "
+                         f"per direction and HBM bytes / copy peak (of {peak_kind}); includes the two group meetings per step",
+                         "kernel": KERNEL_NAME[wl.op], "link_bytes_per_direction_per_gpu": link_bytes,
+                         "hbm_bytes_per_gpu": hbm_bytes},
+            "e2e": {"value": wl.algorithmic_bytes * e2e_steps / (e2e_ms * 1e-3) / 1e9, "unit": UNIT,
+                    "h2d_bytes_per_step": T * H * b, "d2h_bytes_per_step": T * H * b, "steps": e2e_steps,
+                    "ms_per_step": e2e_ms / e2e_steps},
+            "gpu_launches": int(gpu_launches), "clocks": clock_sampler.window(t_begin, t_end),
+            "parity": {"r_out_bit_mismatches": 0, "y_beyond_tolerance": 0, "y_worst": y_worst, "rows_checked": T,
+                       "ranks_checked": world},
+            "tuner": {"theta_from": "shipped table (nearest entry for this block of rows)"},
+        }
+        clock_sampler.stop()
+        print(json.dumps(line), flush=True)
+    clock_sampler.stop()
+    dp.shutdown()
+
+
+def spawn_ranks(n: int, argv: list, script: str | None = None, extra_env: dict | None = None, timeout_s: float | None = None) -> int:
+    """Start `n` ranks of `script` (this file by default), one process per GPU: RANK = LOCAL_RANK = 0..n-1, WORLD_SIZE = n,
+    rendezvous on 127.0.0.1 at a port that is free now.  The ranks inherit stdout and stderr (rank 0 prints the JSON
+    line; NCCL's own messages stay at their default).  Returns the largest exit code; when one rank fails the others
+    are ended, each by its own handle."""
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    procs = []
+    for rank in range(n):
+        env = dict(os.environ, RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(n), LOCAL_WORLD_SIZE=str(n),
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        env.update(extra_env or {})
+        procs.append(subprocess.Popen([sys.executable, script or os.path.abspath(__file__), *argv], env=env))
+    worst, t0 = 0, time.monotonic()
+    pending = list(procs)
+    while pending:
+        for pr in list(pending):
+            rc = pr.poll()
+            if rc is None:
+                continue
+            pending.remove(pr)
+            worst = max(worst, abs(rc))
+        if pending and (worst != 0 or (timeout_s is not None and time.monotonic() - t0 > timeout_s)):
+            for pr in pending:
+                pr.terminate()
+            for pr in pending:
+                try:
+                    pr.wait(timeout=10)
+                except subprocess.TimeoutExpired:
+                    pr.kill()
+            return worst or 124
+        time.sleep(0.05)
+    return worst
 
 
 def main() -> None:
@@ -628,9 +929,15 @@ def main() -> None:
                     "cold-versus-seeded transfer experiment")
     ap.add_argument("--transfer-budget", type=int, default=24)
     ap.add_argument("--log", default="", help="write every evaluated theta of both searches to this JSONL file")
+    ap.add_argument("--resume", default="", help="a JSONL file written by --log: its fastest thetas seed the guided search")
+    ap.add_argument("--retest-top", type=int, default=8, help="points of the sweep re-timed beside the guided winner")
+    ap.add_argument("--retest-rounds", type=int, default=7, help="rounds of the side-by-side re-test")
     args = ap.parse_args()
     if args.steps < 1 or args.warmup < 0:
         raise SystemExit("--steps must be >= 1 and --warmup >= 0")
+    if args.gpus > 1 and "RANK" not in os.environ:
+        # started plainly: be the launcher - one process per GPU, this same command line in each
+        raise SystemExit(spawn_ranks(args.gpus, sys.argv[1:]))
     if args.impl == "reference":
         run_reference(args)
     else:

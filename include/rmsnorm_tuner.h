@@ -64,12 +64,19 @@ typedef enum {
     RT_STAGE_REG = 0,      /* ld.global vectors straight into registers, row kept as fp32 registers */
     RT_STAGE_SMEM_LDG = 1, /* ld.global vectors, sum kept as fp32 in shared memory */
     RT_STAGE_SMEM_TMA = 2, /* cp.async.bulk (TMA, one copy per row slice) into shared memory + mbarrier */
-    RT_STAGE_REG_REALIGN = 3 /* add_rmsnorm only, for rows whose byte length is not a multiple of 16 (the paper's
+    RT_STAGE_REG_REALIGN = 3, /* add_rmsnorm only, for rows whose byte length is not a multiple of 16 (the paper's
                                 "vectorization and alignment strategies" axis): the row is cut at the 16-byte
                                 boundaries of the tensor; the whole chunks between them move as 16-byte vectors and
                                 stay in registers, the fewer than 16 bytes before the first and after the last
                                 boundary move one element to a thread.  Takes vec_bytes = 16, the shuffle reduction,
                                 16-byte aligned base pointers and any hidden size */
+    RT_STAGE_TMA_PIPELINE = 4 /* add_rmsnorm only ("loop scheduling" in the paper's list of tuning dimensions): a
+                                 persistent grid - as many CTAs as stay resident on the device, each walking over row
+                                 blocks b, b + grid, ... - with a ring of `unroll` shared-memory stages per row slot
+                                 (1, 2 or 4), so that the TMA bulk copies of the CTA's next `unroll` - 1 row blocks
+                                 are in flight while the current one is reduced and stored.  Same alignment rules as
+                                 RT_STAGE_SMEM_TMA; shuffle or shared-memory reduction, no cluster.  Left out of the
+                                 derived feasible set unless RT_PRUNE_PIPELINE_STAGE is cleared from the mask */
 } rt_stage;
 
 /* How the per-row sum of squares is combined. */
@@ -131,7 +138,9 @@ enum {
     RT_PRUNE_DUPLICATES = 2,    /* unroll deeper than the per-thread vector count: same kernel again */
     RT_PRUNE_CLUSTER_WAVES = 4, /* split rows over a cluster only while whole rows cannot fill the SMs */
     RT_PRUNE_IDLE_ROWS = 8,     /* more rows per CTA than the batch has rows */
-    RT_PRUNE_DEFAULT = 15
+    RT_PRUNE_PIPELINE_STAGE = 16, /* RT_STAGE_TMA_PIPELINE: measured on B200 it wins on no shape tried, so the
+                                     default search does not pay for its points; clear the bit to include them */
+    RT_PRUNE_DEFAULT = 31
 };
 
 typedef enum { RT_SEARCH_GUIDED = 0, RT_SEARCH_EXHAUSTIVE = 1 } rt_strategy;
@@ -366,7 +375,10 @@ int tuner_derive_counts(const rt_shape* s, const rt_limits* limits, int32_t heur
  * Search(S~, x, Theta_feasible) for one input shape (Algorithm 1): seeds first, then a coarse
  * grid over the feasible set, then best-first hill-climbing over one-step neighbours on
  * measured time (around the three fastest points, then, while budget remains, around up to the
- * twelve fastest), then a re-test of the top_k finalists ("Tuning agent": Top-K re-testing).
+ * twelve fastest), then a re-test of the top_k finalists ("Tuning agent": Top-K re-testing): they are
+ * re-timed side by side as tuner_retest_interleaved does, each counts as one evaluation, the winner is the
+ * fastest finalist that passes again, and a finalist that fails its re-test is replaced by the next runner-up
+ * while budget remains.
  * Every candidate passes the correctness gate (r_out bit-exact, y within 2 ulp for 16-bit types or
  * 1e-5 relative for fp32, against the uploaded references) before it is timed; candidates that
  * fail the gate or the launch are logged and skipped.
@@ -390,6 +402,35 @@ int tuner_search_with(const rt_shape* s, const rt_limits* limits, const rt_budge
 /* Gate + timing of one theta with the protocol of `b` (warmup, iters, repeats, use_graph). */
 int tuner_evaluate(const rt_shape* s, const rt_params* p, const rt_budget* b, const rt_workspace* ws,
                    rt_eval_record* out);
+
+/* One timed block of tuner_retest_interleaved. */
+typedef struct {
+    int32_t theta_index; /* index into the caller's theta array */
+    int32_t round;       /* 0-based round the block belongs to */
+    float us;            /* block time / iters, microseconds */
+    int32_t reserved;    /* 0 */
+    double t_begin_s;    /* host CLOCK_MONOTONIC seconds just before the block's first timed launch ... */
+    double t_end_s;      /* ... and just after its last one completed: for matching clock samples to blocks */
+} rt_block_record;
+
+/*
+ * Top-K re-test as a measurement of its own ("Tuning agent": Top-K re-testing before the convergence decision;
+ * protocol of "Performance Measurement" per block): several thetas re-timed side by side.  Every theta passes the
+ * gate once; then `rounds` rounds follow, and in each round every theta runs one block - b->warmup untimed launches,
+ * then b->iters launches between two events (one CUDA graph when b->use_graph) - before any theta runs its next
+ * block; the order rotates by one from round to round.  A clock or power change during the measurement therefore
+ * meets every theta alike, which back-to-back evaluations of one theta after the other do not give.
+ *   thetas  host, n_thetas entries.      out  host, n_thetas records: status and gate statistics of theta i,
+ *           us = median over its blocks, us_min_block, us_mean.  A theta that is refused or fails the gate has
+ *           its status set and takes no further part.
+ *   blocks  host, rounds * n_thetas records, or NULL: every block in the order it ran (fewer when thetas drop out;
+ *           *n_blocks, may be NULL, receives the count).
+ * tuner_search runs its own Top-K confirmation through the same routine (rounds = b->repeats).  Synchronises the
+ * stream repeatedly.
+ */
+int tuner_retest_interleaved(const rt_shape* s, const rt_params* thetas, int32_t n_thetas, const rt_budget* b,
+                             const rt_workspace* ws, int32_t rounds, rt_eval_record* out, rt_block_record* blocks,
+                             int32_t* n_blocks);
 
 /*
  * Time of an empty kernel under the same protocol (warmup, iters, repeats, use_graph of `b`), in
@@ -521,8 +562,17 @@ int32_t rt_kernel_instance_parts(int32_t i);
  * graph, 40% on them in a plain stream of launches, 1-3.5% on the bandwidth-bound shapes.  Set it to 0 to launch
  * with full stream serialization.
  * rt_set_option returns RT_ERR_SHAPE for an unknown option or value; rt_get_option returns -1 for an unknown option.
+ *
+ * RT_OPTION_TMA_WAIT_POLL_LIMIT (1 .. 2^24, default 2^24): how many times a thread of add_rmsnorm's TMA stages polls
+ * its row's mbarrier before it gives up, writes RT_ERR_DEVICE_TIMEOUT into the device status word, waits once more
+ * with the same limit and then carries on to every barrier of the CTA (the launch completes; its outputs are not
+ * valid).  The default is about a second of polling; a copy that has not landed by then never will.
+ * RT_OPTION_DEBUG_DROP_TMA_COPIES (0 or 1, default 0): diagnostic switch for exercising that path without a
+ * fault - the TMA stages of add_rmsnorm initialise their mbarriers but post no copy, so every wait runs out at the
+ * poll limit and the launch reports RT_ERR_DEVICE_TIMEOUT.  Nothing out of bounds is read or written.  Lower the
+ * poll limit to a few thousand first, or every row waits the full default.
  */
-enum { RT_OPTION_PROGRAMMATIC_LAUNCH = 0 };
+enum { RT_OPTION_PROGRAMMATIC_LAUNCH = 0, RT_OPTION_TMA_WAIT_POLL_LIMIT = 1, RT_OPTION_DEBUG_DROP_TMA_COPIES = 2 };
 int rt_set_option(int32_t option, int32_t value);
 int32_t rt_get_option(int32_t option);
 /* Kernel launches issued by this library in this process since load (all entry points). */

@@ -221,10 +221,19 @@ static int is_nan16(uint16_t b, fmt16 f)
     return ((b >> f.mbits) & emax_field) == emax_field && (b & ((1 << f.mbits) - 1));
 }
 
+static int is_inf16(uint16_t b, fmt16 f)
+{
+    const int emax_field = (1 << f.ebits) - 1;
+    return ((b >> f.mbits) & emax_field) == emax_field && !(b & ((1 << f.mbits) - 1));
+}
+
 /*
  * Distance in units of the last place between two arrays of 16-bit values.
  * Writes the maximum distance and how many elements exceed `tol_ulp`.
  * NaN matches NaN (distance 0); NaN against a number counts as 65535.
+ * The lattice is that of the finite values: an infinity matches only the same
+ * infinity (distance 0) and is 65535 away from everything else, so an output
+ * that overflowed is never "one step" from the largest finite value.
  */
 void oracle_ulp_compare16(const uint16_t* got, const uint16_t* ref, int64_t n, int dtype,
                           int32_t tol_ulp, int32_t* max_ulp, int64_t* n_bad)
@@ -237,6 +246,8 @@ void oracle_ulp_compare16(const uint16_t* got, const uint16_t* ref, int64_t n, i
         const int gn = is_nan16(got[i], f), rn = is_nan16(ref[i], f);
         if (gn || rn)
             d = (gn && rn) ? 0 : 65535;
+        else if (is_inf16(got[i], f) || is_inf16(ref[i], f))
+            d = got[i] == ref[i] ? 0 : 65535;
         else {
             d = lattice16(got[i]) - lattice16(ref[i]);
             if (d < 0) d = -d;
@@ -264,6 +275,8 @@ void oracle_rel_compare32(const float* got, const float* ref, int64_t n, double 
             e = (isnan(g) && isnan(q)) ? 0.0 : INFINITY;
         else if (g == q)
             e = 0.0;
+        else if (isinf(g) || isinf(q))
+            e = INFINITY; /* an infinity matches only itself */
         else {
             double den = fabs(q);
             if (den < abs_floor) den = abs_floor;

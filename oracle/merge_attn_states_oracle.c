@@ -93,14 +93,15 @@ void oracle_mixed_compare(const void* got, const void* ref, int64_t n, int dtype
         } else {
             diff = fabs(g - q);
             if (dtype == ORACLE_FP32) {
-                ok = diff <= tol_ulp_or_rel * fabs(q) || diff <= tol_abs;
+                ok = !isinf(g) && !isinf(q) && (diff <= tol_ulp_or_rel * fabs(q) || diff <= tol_abs);
             } else {
                 const uint16_t gb = ((const uint16_t*)got)[i], qb = ((const uint16_t*)ref)[i];
                 int32_t gi = gb & 0x7FFF, qi = qb & 0x7FFF;
                 if (gb & 0x8000u) gi = -gi;
                 if (qb & 0x8000u) qi = -qi;
                 const double ulps = fabs((double)gi - (double)qi);
-                ok = ulps <= tol_ulp_or_rel || diff <= tol_abs;
+                /* g != q here: an infinity on either side is no neighbour of any finite value */
+                ok = !isinf(g) && !isinf(q) && (ulps <= tol_ulp_or_rel || diff <= tol_abs);
             }
         }
         if (!ok) ++bad;

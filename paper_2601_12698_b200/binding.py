@@ -18,17 +18,18 @@ RT_BF16, RT_FP16, RT_FP32 = 0, 1, 2
 RT_OP_ADD_RMSNORM, RT_OP_SILU_AND_MUL, RT_OP_MERGE_ATTN_STATES, RT_OP_ADD_RMSNORM_FP8 = 0, 1, 2, 3
 RT_OP_ADD_RMSNORM_ALLREDUCE = 4
 RT_MAX_PARTS = 8
-RT_OPTION_PROGRAMMATIC_LAUNCH = 0
-RT_STAGE_REG, RT_STAGE_SMEM_LDG, RT_STAGE_SMEM_TMA, RT_STAGE_REG_REALIGN = 0, 1, 2, 3
+RT_OPTION_PROGRAMMATIC_LAUNCH, RT_OPTION_TMA_WAIT_POLL_LIMIT, RT_OPTION_DEBUG_DROP_TMA_COPIES = 0, 1, 2
+RT_STAGE_REG, RT_STAGE_SMEM_LDG, RT_STAGE_SMEM_TMA, RT_STAGE_REG_REALIGN, RT_STAGE_TMA_PIPELINE = 0, 1, 2, 3, 4
 RT_REDUCE_SHFL, RT_REDUCE_SMEM, RT_REDUCE_CLUSTER = 0, 1, 2
 RT_PRUNE_IDLE_THREADS, RT_PRUNE_DUPLICATES, RT_PRUNE_CLUSTER_WAVES, RT_PRUNE_IDLE_ROWS = 1, 2, 4, 8
-RT_PRUNE_DEFAULT = 15
+RT_PRUNE_PIPELINE_STAGE = 16
+RT_PRUNE_DEFAULT = 31
 RT_SEARCH_GUIDED, RT_SEARCH_EXHAUSTIVE = 0, 1
 RT_CMP_BITS, RT_CMP_ULP16, RT_CMP_REL32 = 0, 1, 2
 (RT_OK, RT_ERR_NULL, RT_ERR_DTYPE, RT_ERR_SHAPE, RT_ERR_ALIGN, RT_ERR_INFEASIBLE, RT_ERR_CUDA, RT_ERR_MISMATCH,
  RT_ERR_BUDGET, RT_ERR_DEVICE_TIMEOUT, RT_ERR_CAPACITY, RT_ERR_NO_DEVICE) = range(12)
 PHASE_NAMES = {0: "seed", 1: "grid", 2: "climb", 3: "topk", 4: "sweep"}
-STAGE_NAMES = {0: "reg", 1: "smem_ldg", 2: "smem_tma", 3: "reg_realign"}
+STAGE_NAMES = {0: "reg", 1: "smem_ldg", 2: "smem_tma", 3: "reg_realign", 4: "tma_pipeline"}
 REDUCE_NAMES = {0: "shfl", 1: "smem", 2: "cluster"}
 DTYPE_CODES = {"bf16": RT_BF16, "fp16": RT_FP16, "fp32": RT_FP32}
 
@@ -93,6 +94,11 @@ class rt_eval_record(Structure):
         return d
 
 
+class rt_block_record(Structure):
+    _fields_ = [("theta_index", c_int32), ("round", c_int32), ("us", c_float), ("reserved", c_int32),
+                ("t_begin_s", c_double), ("t_end_s", c_double)]
+
+
 class rt_result(Structure):
     _fields_ = [("best", rt_params), ("best_us", c_float), ("evals_used", c_int32), ("n_candidates", c_int32),
                 ("n_log", c_int32), ("n_failed_gate", c_int32)]
@@ -137,6 +143,9 @@ _SIGNATURES = {
                                   POINTER(rt_result), POINTER(rt_eval_record), c_int32]),
     "tuner_evaluate": (c_int, [POINTER(rt_shape), POINTER(rt_params), POINTER(rt_budget), POINTER(rt_workspace),
                                POINTER(rt_eval_record)]),
+    "tuner_retest_interleaved": (c_int, [POINTER(rt_shape), POINTER(rt_params), c_int32, POINTER(rt_budget),
+                                         POINTER(rt_workspace), c_int32, POINTER(rt_eval_record),
+                                         POINTER(rt_block_record), POINTER(c_int32)]),
     "tuner_select_general": (c_int, [POINTER(c_float), c_int32, c_int32, POINTER(c_int32), POINTER(c_float),
                                      POINTER(c_float)]),
     "tuner_table_lookup": (c_int, [POINTER(rt_spec_entry), c_int32, POINTER(rt_params), POINTER(rt_shape),
@@ -413,6 +422,20 @@ def tuner_evaluate(shape: rt_shape, params: rt_params, budget: rt_budget, ws: rt
     rec = rt_eval_record()
     _check(lib.tuner_evaluate(byref(shape), byref(params), byref(budget), byref(ws), byref(rec)), "tuner_evaluate")
     return rec
+
+
+def tuner_retest_interleaved(shape: rt_shape, thetas, budget: rt_budget, ws: rt_workspace, rounds: int):
+    """Several thetas re-timed side by side, round-robin block by block.  Returns ([rt_eval_record per theta],
+    [rt_block_record per block, in the order the blocks ran])."""
+    n = len(thetas)
+    arr = (rt_params * n)(*thetas)
+    recs = (rt_eval_record * n)()
+    blocks = (rt_block_record * (n * rounds))()
+    ran = c_int32(0)
+    _check(lib.tuner_retest_interleaved(byref(shape), arr, n, byref(budget), byref(ws), rounds, recs, blocks, byref(ran)),
+           "tuner_retest_interleaved")
+    return ([rt_eval_record.from_buffer_copy(recs[i]) for i in range(n)],
+            [rt_block_record.from_buffer_copy(blocks[i]) for i in range(ran.value)])
 
 
 def tuner_launch_floor(budget: rt_budget, stream=None) -> float:

@@ -50,6 +50,8 @@ struct KernelArgs {
     int slice_nvec;  // vectors of one row owned by one CTA (== nvec unless the row is split over a cluster)
     float eps;
     int* status;     // device status word
+    unsigned wait_polls;  // polls a bounded mbarrier wait may take (kMbarrierPollLimit unless the caller lowered it)
+    int drop_copies;      // diagnostic: 1 = the TMA stages post no copy, so their waits run out and report it
 };
 
 // ---- vectors of VB bytes ------------------------------------------------------------------------
@@ -371,11 +373,11 @@ __device__ __forceinline__ void tma_bulk_load(void* smem_dst, const void* gmem_s
                  ::"r"(smem_u32(smem_dst)), "l"(gmem_src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 // Bounded wait for phase `parity` of `bar`.  Returns false when the poll limit is reached.
-__device__ __forceinline__ bool mbarrier_wait_bounded(uint64_t* bar, uint32_t parity)
+__device__ __forceinline__ bool mbarrier_wait_bounded(uint64_t* bar, uint32_t parity, unsigned poll_limit = kMbarrierPollLimit)
 {
     const uint32_t addr = smem_u32(bar);
     const long long t0 = clock64();
-    for (unsigned it = 0; it < kMbarrierPollLimit; ++it) {
+    for (unsigned it = 0; it < poll_limit; ++it) {
         uint32_t done;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
@@ -518,6 +520,17 @@ __global__ void add_rmsnorm_kernel(const KernelArgs a)
 
     if constexpr (STAGE == kStageReg) {
         float s[CAP][EPV];
+        // A thread that owns at most two vectors (the latency-bound shapes) fetches its weights ahead of the
+        // reduction: a few registers buy the overlap of that fetch with the barrier.  With a single vector it
+        // fetches them first of all, so that the fetch also overlaps the loads of x and r (with two vectors that
+        // order costs four registers and, at 256 threads, a resident CTA on the bandwidth-bound shapes).  Threads that
+        // own more fetch them after the reduction, where other CTAs' traffic hides the latency and registers are scarce.
+        constexpr bool kEarlyWeight = CAP <= 2;
+        constexpr bool kWeightFirst = CAP == 1;
+        Vec<VB> wv[kEarlyWeight ? CAP : 1];
+        if constexpr (kWeightFirst) {
+            if (tx < n) wv[0] = ld_weight_early<VB>(wrow + (size_t)tx * VB);
+        }
 #pragma unroll
         for (int i0 = 0; i0 < CAP; i0 += U) {
             Vec<VB> xv[U], rv[U];
@@ -538,21 +551,18 @@ __global__ void add_rmsnorm_kernel(const KernelArgs a)
                     float xf[EPV], rf[EPV];
                     C::unpack(xv[u], xf);
                     C::unpack(rv[u], rf);
+                    float sv = 0.f;  // this vector's sum of squares: the thread's running sum takes one addition per vector
 #pragma unroll
                     for (int e = 0; e < EPV; ++e) {
                         s[i0 + u][e] = xf[e] + rf[e];
-                        ss = fmaf(s[i0 + u][e], s[i0 + u][e], ss);
+                        sv = fmaf(s[i0 + u][e], s[i0 + u][e], sv);
                     }
+                    ss += sv;
                     st_stream<VB, true>(orow + (size_t)v * VB, C::pack(s[i0 + u]));
                 }
             }
         }
-        // A thread that owns at most two vectors (the latency-bound shapes) fetches its weights before the
-        // reduction: a few registers buy the overlap of that fetch with the barrier.  Threads that own
-        // more fetch them afterwards, where other CTAs' traffic hides the latency and registers are scarce.
-        constexpr bool kEarlyWeight = CAP <= 2;
-        Vec<VB> wv[kEarlyWeight ? CAP : 1];
-        if constexpr (kEarlyWeight) {
+        if constexpr (kEarlyWeight && !kWeightFirst) {
 #pragma unroll
             for (int i = 0; i < CAP; ++i) {
                 const int v = tx + i * tpr;
@@ -617,11 +627,13 @@ __global__ void add_rmsnorm_kernel(const KernelArgs a)
                     float xf[EPV], rf[EPV];
                     C::unpack(xv[u], xf);
                     C::unpack(rv[u], rf);
+                    float sv = 0.f;  // this vector's sum of squares: the thread's running sum takes one addition per vector
 #pragma unroll
                     for (int e = 0; e < EPV; ++e) {
                         s[i0 + u][e] = xf[e] + rf[e];
-                        ss = fmaf(s[i0 + u][e], s[i0 + u][e], ss);
+                        sv = fmaf(s[i0 + u][e], s[i0 + u][e], sv);
                     }
+                    ss += sv;
                     st_stream<VB, true>(oc + (size_t)v * VB, C::pack(s[i0 + u]));
                 }
             }
@@ -689,11 +701,13 @@ __global__ void add_rmsnorm_kernel(const KernelArgs a)
                     float xf[EPV], rf[EPV], s[EPV];
                     C::unpack(xv[u], xf);
                     C::unpack(rv[u], rf);
+                    float sv = 0.f;
 #pragma unroll
                     for (int e = 0; e < EPV; ++e) {
                         s[e] = xf[e] + rf[e];
-                        ss = fmaf(s[e], s[e], ss);
+                        sv = fmaf(s[e], s[e], sv);
                     }
+                    ss += sv;
                     st_stream<VB, true>(orow + (size_t)v * VB, C::pack(s));
                     P::store(srow, a.slice_nvec, v, s);  // read back by this same thread only
                 }
@@ -730,7 +744,7 @@ __global__ void add_rmsnorm_kernel(const KernelArgs a)
         unsigned char* rs = xs + slice_bytes;
         if (tx == 0) {
             mbarrier_init(&bars[ty], 1);
-            if (n > 0) {
+            if (n > 0 && !a.drop_copies) {
                 const uint32_t bytes = (uint32_t)n * VB;
                 mbarrier_expect_tx(&bars[ty], 2 * bytes);
                 tma_bulk_load(xs, xrow, bytes, &bars[ty]);
@@ -739,10 +753,10 @@ __global__ void add_rmsnorm_kernel(const KernelArgs a)
         }
         row_sync(ty, tpr);  // the barrier is initialised before anyone polls it
         if (n > 0) {
-            bool landed = mbarrier_wait_bounded(&bars[ty], 0);
+            bool landed = mbarrier_wait_bounded(&bars[ty], 0, a.wait_polls);
             if (!landed) {
                 atomicExch(a.status, kDeviceTimeoutCode);
-                landed = mbarrier_wait_bounded(&bars[ty], 0);  // do not leave while the copies may still land
+                landed = mbarrier_wait_bounded(&bars[ty], 0, a.wait_polls);  // do not leave while the copies may still land
             }
         }
         for (int v0 = tx; v0 < n; v0 += U * tpr) {
@@ -753,11 +767,13 @@ __global__ void add_rmsnorm_kernel(const KernelArgs a)
                     float xf[EPV], rf[EPV], s[EPV];
                     C::unpack(ld_shared<VB>(xs + (size_t)v * VB), xf);
                     C::unpack(ld_shared<VB>(rs + (size_t)v * VB), rf);
+                    float sv = 0.f;
 #pragma unroll
                     for (int e = 0; e < EPV; ++e) {
                         s[e] = xf[e] + rf[e];
-                        ss = fmaf(s[e], s[e], ss);
+                        sv = fmaf(s[e], s[e], sv);
                     }
+                    ss += sv;
                     st_stream<VB>(orow + (size_t)v * VB, C::pack(s));
                 }
             }

@@ -31,6 +31,8 @@ namespace {
 thread_local char tls_error[512] = "";
 std::atomic<int64_t> g_launches{0};
 std::atomic<int> g_programmatic_launch{1};
+std::atomic<int> g_wait_polls{(int)kMbarrierPollLimit};
+std::atomic<int> g_drop_tma_copies{0};
 std::mutex g_mutex;
 
 constexpr int kMaxDevices = 64;
@@ -737,6 +739,8 @@ int launch_plan(const Plan& plan, const void* x, const void* r, const void* w, v
     a.eps = eps;
     a.status = device_status_word();
     if (!a.status) return RT_ERR_CUDA;
+    a.wait_polls = (unsigned)g_wait_polls.load(std::memory_order_relaxed);
+    a.drop_copies = g_drop_tma_copies.load(std::memory_order_relaxed);
 
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
@@ -1057,17 +1061,27 @@ int32_t rt_kernel_instance_op(int32_t i)
 
 int rt_set_option(int32_t option, int32_t value)
 {
-    if (option != RT_OPTION_PROGRAMMATIC_LAUNCH || (value != 0 && value != 1)) {
+    if (option == RT_OPTION_PROGRAMMATIC_LAUNCH && (value == 0 || value == 1)) {
+        rt::g_programmatic_launch.store(value);
+    } else if (option == RT_OPTION_TMA_WAIT_POLL_LIMIT && value >= 1 && value <= (int32_t)rt::kMbarrierPollLimit) {
+        rt::g_wait_polls.store(value);
+    } else if (option == RT_OPTION_DEBUG_DROP_TMA_COPIES && (value == 0 || value == 1)) {
+        rt::g_drop_tma_copies.store(value);
+    } else {
         rt::set_error("unknown option %d or value %d", option, value);
         return RT_ERR_SHAPE;
     }
-    rt::g_programmatic_launch.store(value);
     return RT_OK;
 }
 
 int32_t rt_get_option(int32_t option)
 {
-    return option == RT_OPTION_PROGRAMMATIC_LAUNCH ? rt::g_programmatic_launch.load() : -1;
+    switch (option) {
+        case RT_OPTION_PROGRAMMATIC_LAUNCH: return rt::g_programmatic_launch.load();
+        case RT_OPTION_TMA_WAIT_POLL_LIMIT: return rt::g_wait_polls.load();
+        case RT_OPTION_DEBUG_DROP_TMA_COPIES: return rt::g_drop_tma_copies.load();
+        default: return -1;
+    }
 }
 
 int32_t rt_kernel_instance_parts(int32_t i)

@@ -4,6 +4,7 @@
 #include <cuda_fp16.h>
 #include <math.h>
 #include <string.h>
+#include <time.h>
 
 #include <mutex>
 #include <unordered_map>
@@ -26,6 +27,8 @@ __device__ __forceinline__ unsigned int ulp_distance16(unsigned int g, unsigned 
     const unsigned int gm = g & 0x7FFFu, qm = q & 0x7FFFu;
     const bool gn = gm > nan_above, qn = qm > nan_above;
     if (gn || qn) return (gn && qn) ? 0u : 65535u;
+    // nan_above is the pattern of infinity: an overflowed value is not "one step" from the largest finite one
+    if (gm == nan_above || qm == nan_above) return g == q ? 0u : 65535u;
     const int gi = (g & 0x8000u) ? -(int)gm : (int)gm;
     const int qi = (q & 0x8000u) ? -(int)qm : (int)qm;
     const int d = gi - qi;
@@ -55,6 +58,9 @@ __device__ __forceinline__ void compare_word(unsigned int g, unsigned int q, int
         const bool gn = gf != gf, qn = qf != qf;
         if (gn || qn) {
             if (!(gn && qn)) { ++bad; worst = 0x7F800000u; }
+        } else if (gf != qf && (isinf(gf) || isinf(qf))) {
+            ++bad;  // an infinity matches only itself
+            worst = 0x7F800000u;
         } else if (gf != qf) {
             const double err = fabs((double)gf - (double)qf);
             const double mag = fabs((double)qf);
@@ -139,6 +145,11 @@ __device__ __forceinline__ void mixed_elem(float g, float q, unsigned int ulps, 
         return;
     }
     if (g == q) return;
+    if (isinf(g) || isinf(q)) {  // an infinity matches only itself
+        ++bad;
+        worst = 0x7F800000u;
+        return;
+    }
     const double diff = fabs((double)g - (double)q);
     const bool ok = diff <= tol_abs || (use_ulps ? (double)ulps <= tol : diff <= tol * fabs((double)q));
     if (!ok) ++bad;
@@ -341,6 +352,18 @@ struct Evaluator {
     // Fills rec->status, the gate statistics and the times.  Returns RT_OK unless the evaluation
     // itself could not be carried out (a CUDA failure that is not specific to the candidate).
     virtual int evaluate(const rt_params& p, rt_eval_record* rec) = 0;
+    // Top-K re-test of `n` finalists: one record per finalist.  The default measures them one after the other.
+    virtual int retest(const rt_params* ps, int n, rt_eval_record* recs)
+    {
+        for (int i = 0; i < n; ++i) {
+            const int st = evaluate(ps[i], &recs[i]);
+            if (st != RT_OK) return st;
+        }
+        return RT_OK;
+    }
+    // true: a finalist's score becomes its re-test time (all finalists were re-timed side by side, under one clock
+    // regime); false: the mean of its two measurements.
+    virtual bool retest_replaces() const { return false; }
 };
 
 static float median_of(std::vector<float> v)
@@ -350,68 +373,113 @@ static float median_of(std::vector<float> v)
     return n % 2 ? v[n / 2] : 0.5f * (v[n / 2 - 1] + v[n / 2]);
 }
 
+static double monotonic_seconds()
+{
+    timespec ts;
+    clock_gettime(CLOCK_MONOTONIC, &ts);
+    return (double)ts.tv_sec + 1e-9 * (double)ts.tv_nsec;
+}
+
 struct DeviceEvaluator : Evaluator {
     rt_shape shape;
     rt_budget budget;
     rt_workspace ws;
     rt_limits limits;
 
-    int evaluate(const rt_params& p, rt_eval_record* rec) override
+    cudaStream_t stream() const { return (cudaStream_t)ws.stream; }
+    int elem_bytes() const { return elem_bytes_of(shape.dtype); }
+    size_t set_bytes() const { return (size_t)shape.n_tokens * shape.hidden * elem_bytes(); }
+    size_t lse_bytes(const Plan& plan) const  // merge_attn_states: one log-sum-exp tensor
     {
-        std::lock_guard<std::mutex> serial(g_compare_mutex);
+        return shape.op == RT_OP_MERGE_ATTN_STATES ? (size_t)shape.n_tokens * plan.heads * sizeof(float) : 0;
+    }
+
+    // One launch of the plan on ring set k (set 0 when the workspace has one set).
+    int launch_set(const Plan& plan, int k) const
+    {
+        const int sets = ws.ring_sets > 0 ? ws.ring_sets : 1;
+        const int eb = elem_bytes();
+        const size_t set = (size_t)(k % sets);
+        const size_t off = set * (size_t)ws.ring_stride_bytes;
+        switch (shape.op) {
+            case RT_OP_ADD_RMSNORM_ALLREDUCE: {
+                // the parts of x lie one after the other in ws.x; one destination
+                const void* parts[RT_MAX_PARTS];
+                for (int j = 0; j < shape.n_parts; ++j)
+                    parts[j] = (const char*)ws.x + (size_t)shape.n_parts * off + (size_t)j * set_bytes();
+                void* y_out = (char*)ws.y + off;
+                void* r_out = (char*)ws.r_out + off;
+                return launch_allreduce_plan(plan, parts, shape.n_parts, (const char*)ws.r + off, ws.w, &y_out, 1, &r_out, 1,
+                                             0, shape.n_tokens, shape.hidden, ws.eps, stream());
+            }
+            case RT_OP_ADD_RMSNORM_FP8:
+                return launch_fp8_plan(plan, (const char*)ws.x + off, (const char*)ws.r + off, ws.w, (char*)ws.y + off / eb,
+                                       (float*)((char*)ws.aux_out + set * shape.n_tokens * sizeof(float)),
+                                       (char*)ws.r_out + off, shape.n_tokens, shape.hidden, ws.eps, stream());
+            case RT_OP_MERGE_ATTN_STATES: {
+                const size_t so = set * lse_bytes(plan);
+                return launch_merge_plan(plan, (const char*)ws.x + off, (const float*)((const char*)ws.w + so),
+                                         (const char*)ws.r + off, (const float*)((const char*)ws.aux + so),
+                                         (char*)ws.y + off, (float*)((char*)ws.r_out + so), shape.n_tokens, stream());
+            }
+            case RT_OP_SILU_AND_MUL:  // the input rows are twice as long as the output rows
+                return launch_silu_plan(plan, (const char*)ws.x + 2 * off, (char*)ws.y + off, shape.n_tokens, stream());
+            default:
+                return launch_plan(plan, (const char*)ws.x + off, (const char*)ws.r + off, ws.w, (char*)ws.y + off,
+                                   (char*)ws.r_out + off, shape.n_tokens, shape.hidden, ws.eps, stream());
+        }
+    }
+
+    // Reads and clears the device status word.  A bounded wait that expired marks the candidate, not the search.
+    int status_word_clear(rt_eval_record* rec) const
+    {
+        int* word = device_status_word();
+        if (!word) return RT_ERR_CUDA;
+        int flag = 0;
+        RT_CUDA_OK(cudaMemcpy(&flag, word, sizeof(int), cudaMemcpyDeviceToHost));
+        if (flag) {
+            RT_CUDA_OK(cudaMemset(word, 0, sizeof(int)));
+            rec->status = RT_ERR_DEVICE_TIMEOUT;
+        }
+        return RT_OK;
+    }
+
+    // theta -> plan; rec->status carries a refusal.  Returns false when the candidate was refused.
+    bool plan_for(const rt_params& p, Plan* plan, rt_eval_record* rec) const
+    {
         memset(rec, 0, sizeof(*rec));
         rec->params = p;
-        cudaStream_t stream = (cudaStream_t)ws.stream;
-        const int eb = elem_bytes_of(shape.dtype);
-        Plan plan;
-        int st = make_plan(&shape, &p, &limits, &plan);
+        const int st = make_plan(&shape, &p, &limits, plan);
         if (st != RT_OK) {
             rec->status = st;
-            return RT_OK;
+            return false;
         }
         int regs = 0;
-        rec->occupancy_blocks_per_sm = plan_occupancy(plan, &limits, &regs);
+        rec->occupancy_blocks_per_sm = plan_occupancy(*plan, &limits, &regs);
         rec->regs_per_thread = regs;
+        return true;
+    }
 
-        // Gate.  Outputs are poisoned first (all-ones is NaN in all three types), so that values left
-        // by an earlier candidate cannot pass for this one's.
+    // The correctness gate: one launch on set 0 compared with the uploaded references.  rec->status = RT_OK,
+    // RT_ERR_MISMATCH, RT_ERR_DEVICE_TIMEOUT or the launch's refusal.  Outputs are poisoned first (all-ones is NaN
+    // in all three types), so that values left by an earlier candidate cannot pass for this one's.
+    int gate(const rt_params& p, const Plan& plan, rt_eval_record* rec) const
+    {
+        const int eb = elem_bytes();
         const int64_t n_ref = ws.n_ref_tokens;
-        const size_t ref_bytes = (size_t)n_ref * shape.hidden * eb;
-        const size_t set_bytes = (size_t)shape.n_tokens * shape.hidden * eb;
         Scratch* sc;
-        st = get_scratch(&sc);
+        int st = get_scratch(&sc);
         if (st != RT_OK) return st;
         const bool is_silu = shape.op == RT_OP_SILU_AND_MUL;
         const bool is_merge = shape.op == RT_OP_MERGE_ATTN_STATES;
         const bool is_fp8 = shape.op == RT_OP_ADD_RMSNORM_FP8;
-        const bool is_allreduce = shape.op == RT_OP_ADD_RMSNORM_ALLREDUCE;
-        // the all-reduce-fused norm: the parts of x lie one after the other in ws.x; one destination
-        auto launch_allreduce = [&](size_t off) {
-            const void* parts[RT_MAX_PARTS];
-            for (int k = 0; k < shape.n_parts; ++k)
-                parts[k] = (const char*)ws.x + (size_t)shape.n_parts * off + (size_t)k * set_bytes;
-            void* y_out = (char*)ws.y + off;
-            void* r_out = (char*)ws.r_out + off;
-            return launch_allreduce_plan(plan, parts, shape.n_parts, (const char*)ws.r + off, ws.w, &y_out, 1, &r_out, 1, 0,
-                                         shape.n_tokens, shape.hidden, ws.eps, stream);
-        };
-        const size_t lse_bytes = is_merge ? (size_t)shape.n_tokens * plan.heads * sizeof(float) : 0;  // one s tensor
-        RT_CUDA_OK(cudaMemsetAsync(ws.y, 0xFF, is_fp8 ? set_bytes / eb : set_bytes, stream));
-        if (is_fp8) RT_CUDA_OK(cudaMemsetAsync(ws.aux_out, 0xFF, (size_t)shape.n_tokens * sizeof(float), stream));
-        if (is_merge) RT_CUDA_OK(cudaMemsetAsync(ws.r_out, 0xFF, lse_bytes, stream));
-        else if (!is_silu) RT_CUDA_OK(cudaMemsetAsync(ws.r_out, 0xFF, set_bytes, stream));
-        RT_CUDA_OK(cudaMemsetAsync(sc->dev, 0, kAccSlots * sizeof(CompareAcc), stream));
-        if (is_allreduce)
-            st = launch_allreduce(0);
-        else if (is_fp8)
-            st = launch_fp8_plan(plan, ws.x, ws.r, ws.w, ws.y, (float*)ws.aux_out, ws.r_out, shape.n_tokens, shape.hidden,
-                                 ws.eps, stream);
-        else if (is_merge)
-            st = launch_merge_plan(plan, ws.x, (const float*)ws.w, ws.r, (const float*)ws.aux, ws.y, (float*)ws.r_out,
-                                   shape.n_tokens, stream);
-        else
-            st = is_silu ? launch_silu_plan(plan, ws.x, ws.y, shape.n_tokens, stream)
-                         : launch_plan(plan, ws.x, ws.r, ws.w, ws.y, ws.r_out, shape.n_tokens, shape.hidden, ws.eps, stream);
+        cudaStream_t s = stream();
+        RT_CUDA_OK(cudaMemsetAsync(ws.y, 0xFF, is_fp8 ? set_bytes() / eb : set_bytes(), s));
+        if (is_fp8) RT_CUDA_OK(cudaMemsetAsync(ws.aux_out, 0xFF, (size_t)shape.n_tokens * sizeof(float), s));
+        if (is_merge) RT_CUDA_OK(cudaMemsetAsync(ws.r_out, 0xFF, lse_bytes(plan), s));
+        else if (!is_silu) RT_CUDA_OK(cudaMemsetAsync(ws.r_out, 0xFF, set_bytes(), s));
+        RT_CUDA_OK(cudaMemsetAsync(sc->dev, 0, kAccSlots * sizeof(CompareAcc), s));
+        st = launch_set(plan, 0);
         if (st != RT_OK) {
             rec->status = st;
             return RT_OK;
@@ -420,29 +488,28 @@ struct DeviceEvaluator : Evaluator {
         const double y_tol = shape.dtype == RT_FP32 ? 1e-5 : 2.0;
         if (is_fp8) {
             // residual bit-exact; codes within one e4m3 step; per-token scales within 1e-5 relative
-            st = enqueue_compare(ws.r_out, ws.r_ref, n_ref * shape.hidden, shape.dtype, RT_CMP_BITS, 0.0, sc->dev, stream);
+            st = enqueue_compare(ws.r_out, ws.r_ref, n_ref * shape.hidden, shape.dtype, RT_CMP_BITS, 0.0, sc->dev, s);
             if (st != RT_OK) return st;
-            st = enqueue_compare_e4m3(ws.y, ws.y_ref, n_ref * shape.hidden, 1, sc->dev + 1, stream);
+            st = enqueue_compare_e4m3(ws.y, ws.y_ref, n_ref * shape.hidden, 1, sc->dev + 1, s);
             if (st != RT_OK) return st;
-            st = enqueue_compare(ws.aux_out, ws.aux_ref, n_ref, RT_FP32, RT_CMP_REL32, 1e-5, sc->dev + 2, stream);
+            st = enqueue_compare(ws.aux_out, ws.aux_ref, n_ref, RT_FP32, RT_CMP_REL32, 1e-5, sc->dev + 2, s);
             if (st != RT_OK) return st;
         } else if (is_merge) {
             // outputs that may cancel: 2 ulp / 1e-5 relative, or 1e-5 absolute; the merged log-sum-exp likewise
-            st = enqueue_compare_mixed(ws.r_out, ws.r_ref, n_ref * plan.heads, RT_FP32, 1e-5, 1e-5, sc->dev, stream);
+            st = enqueue_compare_mixed(ws.r_out, ws.r_ref, n_ref * plan.heads, RT_FP32, 1e-5, 1e-5, sc->dev, s);
             if (st != RT_OK) return st;
-            st = enqueue_compare_mixed(ws.y, ws.y_ref, n_ref * shape.hidden, shape.dtype, y_tol, 1e-5, sc->dev + 1, stream);
+            st = enqueue_compare_mixed(ws.y, ws.y_ref, n_ref * shape.hidden, shape.dtype, y_tol, 1e-5, sc->dev + 1, s);
             if (st != RT_OK) return st;
         } else {
             if (!is_silu) {
-                st = enqueue_compare(ws.r_out, ws.r_ref, n_ref * shape.hidden, shape.dtype, RT_CMP_BITS, 0.0, sc->dev, stream);
+                st = enqueue_compare(ws.r_out, ws.r_ref, n_ref * shape.hidden, shape.dtype, RT_CMP_BITS, 0.0, sc->dev, s);
                 if (st != RT_OK) return st;
             }
-            st = enqueue_compare(ws.y, ws.y_ref, n_ref * shape.hidden, shape.dtype, y_mode, y_tol, sc->dev + 1, stream);
+            st = enqueue_compare(ws.y, ws.y_ref, n_ref * shape.hidden, shape.dtype, y_mode, y_tol, sc->dev + 1, s);
             if (st != RT_OK) return st;
         }
-        (void)ref_bytes;
-        RT_CUDA_OK(cudaMemcpyAsync(sc->host, sc->dev, kAccSlots * sizeof(CompareAcc), cudaMemcpyDeviceToHost, stream));
-        cudaError_t e = cudaStreamSynchronize(stream);
+        RT_CUDA_OK(cudaMemcpyAsync(sc->host, sc->dev, kAccSlots * sizeof(CompareAcc), cudaMemcpyDeviceToHost, s));
+        cudaError_t e = cudaStreamSynchronize(s);
         if (e != cudaSuccess) {
             set_error("candidate faulted: %s", cudaGetErrorString(e));
             return RT_ERR_CUDA;  // a sticky error: nothing further can run in this context
@@ -455,42 +522,93 @@ struct DeviceEvaluator : Evaluator {
             rec->y_max_rel = (float)acc_max_err(sc->host[1], RT_CMP_REL32);  // merge: largest absolute difference
         else
             rec->y_max_ulp = (int32_t)sc->host[1].max_bits;
-        if (p.stage == RT_STAGE_SMEM_TMA) {
-            int flag = 0;
-            RT_CUDA_OK(cudaMemcpy(&flag, device_status_word(), sizeof(int), cudaMemcpyDeviceToHost));
-            if (flag) {
-                RT_CUDA_OK(cudaMemset(device_status_word(), 0, sizeof(int)));
-                rec->status = RT_ERR_DEVICE_TIMEOUT;
-                return RT_OK;
-            }
+        if (p.stage == RT_STAGE_SMEM_TMA || p.stage == RT_STAGE_TMA_PIPELINE) {
+            st = status_word_clear(rec);
+            if (st != RT_OK) return st;
+            if (rec->status != RT_OK) return RT_OK;
         }
-        if (rec->r_bad || rec->y_bad) {
-            rec->status = RT_ERR_MISMATCH;
+        if (rec->r_bad || rec->y_bad) rec->status = RT_ERR_MISMATCH;
+        return RT_OK;
+    }
+
+    // The timed block as one CUDA graph of `iters` launches, replayed once untimed.  A candidate that cannot be
+    // captured gets rec->status; *exec stays NULL.
+    int capture_block(const Plan& plan, int iters, cudaGraphExec_t* exec, rt_eval_record* rec) const
+    {
+        *exec = nullptr;
+        if (!stream()) {
+            set_error("use_graph needs a non-default stream");
+            return RT_ERR_CUDA;
+        }
+        cudaGraph_t graph = nullptr;
+        RT_CUDA_OK(cudaStreamBeginCapture(stream(), cudaStreamCaptureModeThreadLocal));
+        int cap_st = RT_OK;
+        for (int i = 0; i < iters && cap_st == RT_OK; ++i) cap_st = launch_set(plan, i);
+        cudaError_t ce = cudaStreamEndCapture(stream(), &graph);
+        if (cap_st != RT_OK || ce != cudaSuccess) {
+            if (graph) cudaGraphDestroy(graph);
+            (void)cudaGetLastError();
+            rec->status = cap_st != RT_OK ? cap_st : RT_ERR_CUDA;
             return RT_OK;
         }
+        ce = cudaGraphInstantiate(exec, graph, 0);
+        cudaGraphDestroy(graph);
+        if (ce != cudaSuccess) {
+            *exec = nullptr;
+            set_error("cudaGraphInstantiate failed: %s", cudaGetErrorString(ce));
+            return RT_ERR_CUDA;
+        }
+        RT_CUDA_OK(cudaGraphLaunch(*exec, stream()));  // one untimed replay
+        return RT_OK;
+    }
+
+    // `iters` launches between two events; *us = block time / iters.
+    int timed_block(const Plan& plan, cudaGraphExec_t exec, int iters, cudaEvent_t e0, cudaEvent_t e1, float* us) const
+    {
+        int fail = RT_OK;
+        cudaEventRecord(e0, stream());
+        if (exec) {
+            if (cudaGraphLaunch(exec, stream()) != cudaSuccess) fail = RT_ERR_CUDA;
+            count_launch(iters);
+        } else {
+            for (int i = 0; i < iters && fail == RT_OK; ++i) fail = launch_set(plan, i);
+        }
+        cudaEventRecord(e1, stream());
+        if (cudaEventSynchronize(e1) != cudaSuccess) fail = RT_ERR_CUDA;
+        float ms = 0.f;
+        if (fail == RT_OK && cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess) fail = RT_ERR_CUDA;
+        if (fail != RT_OK) {
+            cudaError_t le = cudaGetLastError();
+            set_error("timing failed: %s", cudaGetErrorString(le));
+            return RT_ERR_CUDA;
+        }
+        *us = ms * 1000.f / (float)iters;
+        return RT_OK;
+    }
+
+    static void fill_times(const std::vector<float>& block_us, rt_eval_record* rec)
+    {
+        float sum = 0.f, mn = block_us[0];
+        for (float v : block_us) {
+            sum += v;
+            mn = std::min(mn, v);
+        }
+        rec->us = median_of(block_us);
+        rec->us_min_block = mn;
+        rec->us_mean = sum / (float)block_us.size();
+    }
+
+    int evaluate(const rt_params& p, rt_eval_record* rec) override
+    {
+        std::lock_guard<std::mutex> serial(g_compare_mutex);
+        Plan plan;
+        if (!plan_for(p, &plan, rec)) return RT_OK;
+        int st = gate(p, plan, rec);
+        if (st != RT_OK || rec->status != RT_OK) return st;
 
         // Timing: `warmup` launches, then `repeats` blocks of `iters` launches between two events.
-        const int sets = ws.ring_sets > 0 ? ws.ring_sets : 1;
-        auto launch_set = [&](int k) {
-            const size_t off = (size_t)(k % sets) * (size_t)ws.ring_stride_bytes;
-            if (is_allreduce) return launch_allreduce(off);
-            if (is_fp8)
-                return launch_fp8_plan(plan, (const char*)ws.x + off, (const char*)ws.r + off, ws.w, (char*)ws.y + off / eb,
-                                       (float*)((char*)ws.aux_out + (size_t)(k % sets) * shape.n_tokens * sizeof(float)),
-                                       (char*)ws.r_out + off, shape.n_tokens, shape.hidden, ws.eps, stream);
-            if (is_merge) {
-                const size_t so = (size_t)(k % sets) * lse_bytes;
-                return launch_merge_plan(plan, (const char*)ws.x + off, (const float*)((const char*)ws.w + so),
-                                         (const char*)ws.r + off, (const float*)((const char*)ws.aux + so),
-                                         (char*)ws.y + off, (float*)((char*)ws.r_out + so), shape.n_tokens, stream);
-            }
-            if (is_silu)  // the input rows are twice as long as the output rows
-                return launch_silu_plan(plan, (const char*)ws.x + 2 * off, (char*)ws.y + off, shape.n_tokens, stream);
-            return launch_plan(plan, (const char*)ws.x + off, (const char*)ws.r + off, ws.w, (char*)ws.y + off,
-                               (char*)ws.r_out + off, shape.n_tokens, shape.hidden, ws.eps, stream);
-        };
         for (int i = 0; i < budget.warmup; ++i) {
-            st = launch_set(i);
+            st = launch_set(plan, i);
             if (st != RT_OK) {
                 rec->status = st;
                 return RT_OK;
@@ -500,66 +618,115 @@ struct DeviceEvaluator : Evaluator {
         const int repeats = budget.repeats > 0 ? budget.repeats : 1;
         cudaGraphExec_t graph_exec = nullptr;
         if (budget.use_graph) {
-            if (!stream) {
-                set_error("use_graph needs a non-default stream");
-                return RT_ERR_CUDA;
-            }
-            cudaGraph_t graph = nullptr;
-            RT_CUDA_OK(cudaStreamBeginCapture(stream, cudaStreamCaptureModeThreadLocal));
-            int cap_st = RT_OK;
-            for (int i = 0; i < iters && cap_st == RT_OK; ++i) cap_st = launch_set(i);
-            cudaError_t ce = cudaStreamEndCapture(stream, &graph);
-            if (cap_st != RT_OK || ce != cudaSuccess) {
-                if (graph) cudaGraphDestroy(graph);
-                (void)cudaGetLastError();
-                rec->status = cap_st != RT_OK ? cap_st : RT_ERR_CUDA;
-                return RT_OK;
-            }
-            ce = cudaGraphInstantiate(&graph_exec, graph, 0);
-            cudaGraphDestroy(graph);
-            if (ce != cudaSuccess) {
-                set_error("cudaGraphInstantiate failed: %s", cudaGetErrorString(ce));
-                return RT_ERR_CUDA;
-            }
-            RT_CUDA_OK(cudaGraphLaunch(graph_exec, stream));  // one untimed replay
+            st = capture_block(plan, iters, &graph_exec, rec);
+            if (st != RT_OK || rec->status != RT_OK) return st;
         }
         cudaEvent_t e0, e1;
         RT_CUDA_OK(cudaEventCreate(&e0));
         RT_CUDA_OK(cudaEventCreate(&e1));
         std::vector<float> block_us;
-        int fail = RT_OK;
-        for (int rep = 0; rep < repeats && fail == RT_OK; ++rep) {
-            cudaEventRecord(e0, stream);
-            if (graph_exec) {
-                if (cudaGraphLaunch(graph_exec, stream) != cudaSuccess) fail = RT_ERR_CUDA;
-                count_launch(iters);
-            } else {
-                for (int i = 0; i < iters && fail == RT_OK; ++i) fail = launch_set(i);
-            }
-            cudaEventRecord(e1, stream);
-            if (cudaEventSynchronize(e1) != cudaSuccess) fail = RT_ERR_CUDA;
-            float ms = 0.f;
-            if (fail == RT_OK && cudaEventElapsedTime(&ms, e0, e1) == cudaSuccess) block_us.push_back(ms * 1000.f / iters);
+        st = RT_OK;
+        for (int rep = 0; rep < repeats && st == RT_OK; ++rep) {
+            float us = 0.f;
+            st = timed_block(plan, graph_exec, iters, e0, e1, &us);
+            if (st == RT_OK) block_us.push_back(us);
         }
         cudaEventDestroy(e0);
         cudaEventDestroy(e1);
         if (graph_exec) cudaGraphExecDestroy(graph_exec);
-        if (fail != RT_OK || block_us.empty()) {
-            cudaError_t le = cudaGetLastError();
-            set_error("timing failed: %s", cudaGetErrorString(le));
-            return RT_ERR_CUDA;
-        }
-        float sum = 0.f, mn = block_us[0];
-        for (float v : block_us) {
-            sum += v;
-            mn = std::min(mn, v);
-        }
-        rec->us = median_of(block_us);
-        rec->us_min_block = mn;
-        rec->us_mean = sum / (float)block_us.size();
-        rec->status = RT_OK;
+        if (st != RT_OK) return st;
+        fill_times(block_us, rec);
+        // a bounded wait may also expire in a timed launch: such a time is not a time of the operator
+        if (p.stage == RT_STAGE_SMEM_TMA || p.stage == RT_STAGE_TMA_PIPELINE) return status_word_clear(rec);
         return RT_OK;
     }
+
+    // Re-timing of several thetas side by side: every theta passes the gate once, then `rounds` rounds; in a round
+    // every theta runs one block (warm-up launches, then `iters` timed launches) before any theta runs its next
+    // block, and the order rotates by one from round to round.  Clock and power changes during the measurement
+    // therefore meet every theta alike.  recs[i]: status, gate statistics, median / fastest / mean block of theta i;
+    // blocks (may be NULL): one record per (round, theta) block in the order they ran.
+    int interleaved(const rt_params* ps, int n, int rounds, rt_eval_record* recs, rt_block_record* blocks,
+                    int* n_blocks_out = nullptr)
+    {
+        std::lock_guard<std::mutex> serial(g_compare_mutex);
+        const int iters = budget.iters > 0 ? budget.iters : 1;
+        std::vector<Plan> plans((size_t)n);
+        std::vector<cudaGraphExec_t> execs((size_t)n, nullptr);
+        std::vector<std::vector<float>> times((size_t)n);
+        int st = RT_OK;
+        for (int i = 0; i < n && st == RT_OK; ++i) {
+            if (!plan_for(ps[i], &plans[i], &recs[i])) continue;
+            st = gate(ps[i], plans[i], &recs[i]);
+            if (st == RT_OK && recs[i].status == RT_OK && budget.use_graph)
+                st = capture_block(plans[i], iters, &execs[i], &recs[i]);
+        }
+        cudaEvent_t e0 = nullptr, e1 = nullptr;
+        if (st == RT_OK && (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess)) {
+            set_error("cudaEventCreate failed");
+            st = RT_ERR_CUDA;
+        }
+        int n_blocks = 0;
+        for (int round = 0; round < rounds && st == RT_OK; ++round)
+            for (int j = 0; j < n && st == RT_OK; ++j) {
+                const int i = (j + round) % n;
+                if (recs[i].status != RT_OK) continue;
+                for (int k = 0; k < budget.warmup && st == RT_OK; ++k) st = launch_set(plans[i], k);
+                if (st != RT_OK) break;
+                if (cudaStreamSynchronize(stream()) != cudaSuccess) {
+                    set_error("warm-up faulted");
+                    st = RT_ERR_CUDA;
+                    break;
+                }
+                float us = 0.f;
+                const double t0 = monotonic_seconds();
+                st = timed_block(plans[i], execs[i], iters, e0, e1, &us);
+                const double t1 = monotonic_seconds();
+                if (st != RT_OK) break;
+                times[i].push_back(us);
+                if (blocks) {
+                    rt_block_record& b = blocks[n_blocks];
+                    b.theta_index = i;
+                    b.round = round;
+                    b.us = us;
+                    b.reserved = 0;
+                    b.t_begin_s = t0;
+                    b.t_end_s = t1;
+                }
+                ++n_blocks;
+            }
+        if (n_blocks_out) *n_blocks_out = n_blocks;
+        if (e0) cudaEventDestroy(e0);
+        if (e1) cudaEventDestroy(e1);
+        for (cudaGraphExec_t g : execs)
+            if (g) cudaGraphExecDestroy(g);
+        if (st != RT_OK) return st;
+        for (int i = 0; i < n; ++i) {
+            if (recs[i].status != RT_OK) continue;
+            if (times[i].empty()) {
+                recs[i].status = RT_ERR_BUDGET;  // rounds < 1: gated, not timed
+                continue;
+            }
+            fill_times(times[i], &recs[i]);
+            if (ps[i].stage == RT_STAGE_SMEM_TMA || ps[i].stage == RT_STAGE_TMA_PIPELINE) {
+                // the word is shared: an expired wait is charged to every TMA candidate of this re-test
+                rt_eval_record probe = recs[i];
+                st = status_word_clear(&probe);
+                if (st != RT_OK) return st;
+                if (probe.status != RT_OK)
+                    for (int k = 0; k < n; ++k)
+                        if (recs[k].status == RT_OK && (ps[k].stage == RT_STAGE_SMEM_TMA || ps[k].stage == RT_STAGE_TMA_PIPELINE))
+                            recs[k].status = RT_ERR_DEVICE_TIMEOUT;
+            }
+        }
+        return RT_OK;
+    }
+
+    int retest(const rt_params* ps, int n, rt_eval_record* recs) override
+    {
+        return interleaved(ps, n, budget.repeats > 0 ? budget.repeats : 1, recs, nullptr);
+    }
+    bool retest_replaces() const override { return true; }
 };
 
 // The launch floor: an empty kernel timed with the same protocol, so that the share of launch overhead in
@@ -886,19 +1053,49 @@ int run_search(const rt_shape& shape, const rt_limits& limits, const rt_budget& 
         }
     }
 
-    // 4. Top-K confirmation re-test: the finalists' scores become the mean of both measurements
+    // 4. Top-K confirmation re-test ("Tuning agent": the finalists are measured again before the winner is
+    //    declared).  The K fastest are re-timed together (on the device: interleaved block by block, so that they
+    //    share one clock regime) and the winner is the fastest of those that pass again; a finalist that fails
+    //    its re-test - a gate that passes once and fails once is what the re-test is there to catch - drops out,
+    //    and while budget remains the next runner-up is re-tested in its place.
     std::vector<int> order;
     for (int i = 0; i < (int)S.cand.size(); ++i)
         if (S.time_us[i] >= 0.f && isfinite(S.time_us[i])) order.push_back(i);
     std::sort(order.begin(), order.end(), [&](int a, int c) { return S.time_us[a] < S.time_us[c]; });
-    for (int k = 0; k < top_k && k < (int)order.size() && S.used < S.max_evals; ++k) {
-        st = S.run(order[k], RT_PHASE_TOPK, &t);
+    std::vector<int> confirmed;
+    size_t next = 0;
+    int want = top_k;
+    for (int pass = 0; pass < 2 && want > 0; ++pass) {
+        std::vector<int> batch;
+        while (next < order.size() && (int)batch.size() < want && S.used + (int)batch.size() < S.max_evals)
+            batch.push_back(order[next++]);
+        if (batch.empty()) break;
+        std::vector<rt_params> ps;
+        for (int idx : batch) ps.push_back(S.cand[idx]);
+        std::vector<rt_eval_record> recs(batch.size());
+        st = ev.retest(ps.data(), (int)ps.size(), recs.data());
+        int dropped = 0;
+        for (size_t k = 0; k < batch.size(); ++k) {
+            rt_eval_record& rec = recs[k];
+            rec.phase = RT_PHASE_TOPK;
+            rec.eval_index = S.used++;
+            if (S.log && S.n_log < S.log_cap) S.log[S.n_log++] = rec;
+            if (st != RT_OK) continue;
+            if (rec.status != RT_OK) {
+                ++S.failed;
+                ++dropped;
+                S.time_us[batch[k]] = INFINITY;
+            } else {
+                S.time_us[batch[k]] = ev.retest_replaces() ? rec.us : 0.5f * (S.time_us[batch[k]] + rec.us);
+                confirmed.push_back(batch[k]);
+            }
+        }
         if (st != RT_OK) return st;
-        if (isfinite(t)) S.time_us[order[k]] = 0.5f * (S.time_us[order[k]] + t);
+        want = dropped;
     }
     int best = -1;
-    for (int i : order)
-        if (best < 0 || S.time_us[i] < S.time_us[best]) best = i;
+    for (int i : confirmed.empty() ? order : confirmed)
+        if (isfinite(S.time_us[i]) && (best < 0 || S.time_us[i] < S.time_us[best])) best = i;
 
     out->evals_used = S.used;
     out->n_log = S.n_log;
@@ -932,7 +1129,43 @@ int check_workspace(const rt_shape* s, const rt_workspace* ws)
         set_error("the tuner's workspace must not alias inputs and outputs (launches repeat)");
         return RT_ERR_SHAPE;
     }
+    if (ws->ring_sets > 1 && ws->ring_stride_bytes <= 0) {
+        set_error("ring_sets=%d needs a positive ring_stride_bytes", ws->ring_sets);
+        return RT_ERR_SHAPE;
+    }
+    // the comparison kernels read 32-bit words
+    if (((uintptr_t)ws->y | (uintptr_t)ws->y_ref | (uintptr_t)ws->r_out | (uintptr_t)ws->r_ref | (uintptr_t)ws->aux_out |
+         (uintptr_t)ws->aux_ref) & 3u) {
+        set_error("outputs and references must be 4-byte aligned");
+        return RT_ERR_ALIGN;
+    }
     return RT_OK;
+}
+
+// The alignment every address the evaluator will hand to a kernel is known to have: the caller's claim
+// (rt_shape.min_ptr_align) cut down to what the workspace pointers, the ring stride and the offsets derived from
+// them (the parts of the all-reduce-fused norm, the byte-wide codes of the fp8-output norm) really share.  The
+// feasible set and every plan are derived from this value, so a sliced tensor or an odd ring stride narrows the
+// vectors or refuses the TMA stages instead of launching a misaligned access.
+int32_t effective_alignment(const rt_shape& s, const rt_workspace& ws)
+{
+    const int eb = elem_bytes_of(s.dtype);
+    uintptr_t bits = (uintptr_t)ws.x | (uintptr_t)ws.y | 256u;
+    const bool vectors_in_r = s.op != RT_OP_SILU_AND_MUL;
+    if (vectors_in_r) bits |= (uintptr_t)ws.r;
+    if (s.op == RT_OP_ADD_RMSNORM_FP8) {
+        // q leaves as vectors half as wide as those of x: its alignment counts double
+        bits = ((uintptr_t)ws.x | (uintptr_t)ws.r | (uintptr_t)ws.w | (uintptr_t)ws.r_out | ((uintptr_t)ws.y << 1) | 256u);
+    } else if (s.op != RT_OP_MERGE_ATTN_STATES && s.op != RT_OP_SILU_AND_MUL) {
+        bits |= (uintptr_t)ws.w | (uintptr_t)ws.r_out;  // merge_attn_states: w and r_out are binary32 scalars per head
+    }
+    if (ws.ring_sets > 1) {
+        bits |= (uintptr_t)ws.ring_stride_bytes;
+        if (s.op == RT_OP_ADD_RMSNORM_FP8) bits |= (uintptr_t)(ws.ring_stride_bytes / eb) << 1;
+    }
+    if (s.op == RT_OP_ADD_RMSNORM_ALLREDUCE) bits |= (uintptr_t)((uint64_t)s.n_tokens * (uint64_t)s.hidden * eb);
+    const int32_t have = (int32_t)(bits & (~bits + 1));
+    return std::min<int32_t>(s.min_ptr_align > 0 ? s.min_ptr_align : 1, have);
 }
 
 rt_budget normalised(const rt_budget* b)
@@ -1077,11 +1310,40 @@ int tuner_evaluate(const rt_shape* s, const rt_params* p, const rt_budget* b, co
     if (st != RT_OK) return st;
     rt::DeviceEvaluator ev;
     ev.shape = *s;
+    ev.shape.min_ptr_align = rt::effective_alignment(*s, *ws);
     ev.budget = rt::normalised(b);
     ev.ws = *ws;
     st = rt::current_limits(&ev.limits);
     if (st != RT_OK) return st;
     return ev.evaluate(*p, out);
+}
+
+int tuner_retest_interleaved(const rt_shape* s, const rt_params* thetas, int32_t n_thetas, const rt_budget* b,
+                             const rt_workspace* ws, int32_t rounds, rt_eval_record* out, rt_block_record* blocks,
+                             int32_t* n_blocks)
+{
+    if (!thetas || !b || !out) {
+        rt::set_error("tuner_retest_interleaved: NULL argument");
+        return RT_ERR_NULL;
+    }
+    if (n_thetas < 1 || rounds < 1) {
+        rt::set_error("tuner_retest_interleaved: n_thetas=%d and rounds=%d must be positive", n_thetas, rounds);
+        return RT_ERR_BUDGET;
+    }
+    int st = rt::check_workspace(s, ws);
+    if (st != RT_OK) return st;
+    rt::DeviceEvaluator ev;
+    ev.shape = *s;
+    ev.shape.min_ptr_align = rt::effective_alignment(*s, *ws);
+    ev.budget = rt::normalised(b);
+    ev.ws = *ws;
+    st = rt::current_limits(&ev.limits);
+    if (st != RT_OK) return st;
+    if (blocks) memset(blocks, 0, sizeof(rt_block_record) * (size_t)rounds * (size_t)n_thetas);
+    int ran = 0;
+    st = ev.interleaved(thetas, n_thetas, rounds, out, blocks, &ran);
+    if (n_blocks) *n_blocks = ran;
+    return st;
 }
 
 int tuner_search(const rt_shape* s, const rt_budget* b, const rt_workspace* ws, rt_result* out, rt_eval_record* log,
@@ -1095,11 +1357,12 @@ int tuner_search(const rt_shape* s, const rt_budget* b, const rt_workspace* ws, 
     if (st != RT_OK) return st;
     rt::DeviceEvaluator ev;
     ev.shape = *s;
+    ev.shape.min_ptr_align = rt::effective_alignment(*s, *ws);
     ev.budget = rt::normalised(b);
     ev.ws = *ws;
     st = rt::current_limits(&ev.limits);
     if (st != RT_OK) return st;
-    return rt::run_search(*s, ev.limits, ev.budget, ev, out, log, log_cap);
+    return rt::run_search(ev.shape, ev.limits, ev.budget, ev, out, log, log_cap);
 }
 
 int tuner_search_with(const rt_shape* s, const rt_limits* limits, const rt_budget* b, rt_evaluate_fn evaluate, void* user,

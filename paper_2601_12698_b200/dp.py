@@ -119,8 +119,9 @@ class FusedAllreduceNorm:
     own block and nothing else - unless ``gather_residual`` asks for every rank to receive it too.
 
     The kernel never waits for another rank.  The group meets in stream order instead: a one-element all-reduce
-    on the launch stream before the kernel (every rank's partial is complete once it returns) and one after it
-    (every rank's rows have been written once it returns).  ``launch`` is
+    on the launch stream before the kernel (every rank's partial is complete once it has run) and one after it
+    (every rank's rows have been written once it has run).  Whatever produced this rank's partial must be ordered
+    before the call on that same stream.  ``launch`` is
     ``binding.rmsnorm_allreduce_template_launch``; it is a parameter so that the host logic can run without a GPU.
     """
     rank: int
@@ -130,8 +131,9 @@ class FusedAllreduceNorm:
     y_outs: list
     r_outs: list
     launch: object
-    sync: object = None  # callable run before and after the launch; default: a one-element all-reduce
+    sync: object = None  # callable(stream) run before and after the launch; default: a one-element all-reduce on it
     gather_residual: bool = False
+    _flag: object = None  # the meeting's one-element tensor, allocated once (no allocation per step)
 
     def __post_init__(self):
         if self.world not in (2, 4, 8):
@@ -145,20 +147,32 @@ class FusedAllreduceNorm:
     def shard(self) -> Shard:
         return strong_shard(self.n_rows, self.rank, self.world)
 
-    def _meet(self, device) -> None:
+    def _meet(self, device, stream) -> None:
+        """One meeting of the group, ordered on `stream` (None = the current stream): both the collective and the
+        kernel between the two meetings must sit on one stream, or the kernel is ordered against neither."""
         if self.sync is not None:
-            self.sync()
-        elif dist.is_initialized():
-            flag = torch.zeros(1, dtype=torch.int32, device=device)
-            dist.all_reduce(flag)  # stream-ordered on NCCL: returns on the stream once every rank has reached it
+            self.sync(stream)
+            return
+        if not dist.is_initialized():
+            return
+        if device.type == "cuda" and stream is not None:
+            with torch.cuda.stream(stream):  # the collective is ordered against the stream that is current at the call
+                if self._flag is None:
+                    self._flag = torch.zeros(1, dtype=torch.int32, device=device)
+                dist.all_reduce(self._flag)
+        else:
+            if self._flag is None:
+                self._flag = torch.zeros(1, dtype=torch.int32, device=device)
+            dist.all_reduce(self._flag)  # stream-ordered on NCCL: complete on the stream once every rank has reached it
 
     def __call__(self, theta, r, w, eps: float, stream=None) -> Shard:
-        """r: this rank's residual [n_rows, hidden] (the same values on every rank); w: [hidden]."""
+        """r: this rank's residual [n_rows, hidden] (the same values on every rank); w: [hidden].  The two meetings
+        and the launch between them are issued on `stream` (None: torch's current stream for all three)."""
         sh = self.shard
-        self._meet(r.device)
+        self._meet(r.device, stream)
         r_outs = self.r_outs if self.gather_residual else [self.r_outs[self.rank]]
         self.launch(theta, self.x_parts, r, w, self.y_outs, r_outs, sh.row_begin, sh.rows, eps, stream)
-        self._meet(r.device)
+        self._meet(r.device, stream)
         return sh
 
 

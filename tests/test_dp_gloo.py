@@ -95,7 +95,15 @@ def _tp_worker(rank: int, world: int, port: int, shared: dict, out_dir: str):
 
     # Stand-in for the CUDA entry point with the same signature: the oracle on the requested rows, written to every
     # destination.  Shared-memory tensors stand in for peer-mapped GPU memory.
+    met_on = []  # the stream each meeting of the group was issued on
+
+    def sync(stream):
+        met_on.append(stream)
+        dist.barrier()
+
     def launch(theta, x_parts, r, w, y_outs, r_outs, row_begin, row_count, eps, stream):
+        # the launch sits between two meetings and on the very stream the first one was issued on
+        assert len(met_on) % 2 == 1 and stream is met_on[-1]
         calls.append((tuple(theta), row_begin, row_count, len(x_parts), len(y_outs), len(r_outs)))
         rows = slice(row_begin, row_begin + row_count)
         stacked = torch.stack([p[rows] for p in x_parts]).contiguous()
@@ -111,8 +119,10 @@ def _tp_worker(rank: int, world: int, port: int, shared: dict, out_dir: str):
     ranks_seen = dp.gather_in_rank_order(("rank", rank))
     assert ranks_seen == [("rank", k) for k in range(world)]
     op = dp.FusedAllreduceNorm(rank, world, n_rows, list(shared["x"]), list(shared["y"]), list(shared["r_out"]), launch,
-                               sync=dist.barrier)
-    sh = op((256, 1, 16, 1, 0, 0, 1), shared["r"], shared["w"], 1e-6)
+                               sync=sync)
+    side_stream = object()  # stands for a CUDA stream that is not the current one
+    sh = op((256, 1, 16, 1, 0, 0, 1), shared["r"], shared["w"], 1e-6, stream=side_stream)
+    assert met_on == [side_stream, side_stream]                             # both meetings on the launch stream
     assert (sh.row_begin, sh.row_end) == ((0, 19), (19, 37))[rank]          # 37 rows over two ranks: 19 + 18
     assert calls == [((256, 1, 16, 1, 0, 0, 1), sh.row_begin, sh.rows, world, world, 1)]
     # after the second meeting this rank's y holds every row, its r_out the rows of its own block
@@ -122,8 +132,14 @@ def _tp_worker(rank: int, world: int, port: int, shared: dict, out_dir: str):
     dp.barrier(device)
     op.gather_residual = True
     op((256, 1, 16, 1, 0, 0, 1), shared["r"], shared["w"], 1e-6)
-    assert calls[-1][-1] == world
+    assert calls[-1][-1] == world and met_on[2:] == [None, None]
     torch.save({"ro_all": shared["r_out"][rank].clone()}, os.path.join(out_dir, f"tpg{rank}.pt"))
+    # the default meeting (a one-element all-reduce of the process group) in place of the test's barrier
+    dp.barrier(device)
+    met_on.append(None)  # keep the launch's "between two meetings" check in step
+    op.sync = None
+    op((256, 1, 16, 1, 0, 0, 1), shared["r"], shared["w"], 1e-6)
+    assert int(op._flag.item()) == 0 and len(calls) == 3
     dp.barrier(device)
     dp.shutdown()
 

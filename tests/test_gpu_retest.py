@@ -1,0 +1,153 @@
+"""The side-by-side re-test (Top-K re-testing as a measurement of its own) and the alignment the tuner derives from
+its workspace, on the device."""
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2601_12698_b200 import binding
+    torch.cuda.set_device(0)
+    return binding
+
+
+def _workspace(B, oracle_lib, wl, **kw):
+    from paper_2601_12698_b200 import synth
+    x, r, w = synth.make_workload_inputs(wl)
+    y_ref, r_ref = oracle_lib.add_rmsnorm(x, r, w, wl.eps)
+    t = dict(x=x.cuda(), r=r.cuda(), w=w.cuda(), y_ref=y_ref.cuda(), r_ref=r_ref.cuda())
+    t["y"], t["r_out"] = torch.empty_like(t["x"]), torch.empty_like(t["x"])
+    t["stream"] = torch.cuda.Stream()
+    ws = B.make_workspace(t["x"], t["r"], t["w"], t["y"], t["r_out"], t["y_ref"], t["r_ref"], wl.eps, stream=t["stream"], **kw)
+    return t, ws
+
+
+@pytest.mark.parametrize("graph", [False, True])
+def test_blocks_rotate_over_the_candidates(B, oracle_lib, graph):
+    from paper_2601_12698_b200 import synth
+    wl = synth.Workload("t", "bf16", 256, 4096, seed=3)
+    t, ws = _workspace(B, oracle_lib, wl)
+    shape = B.shape_of(wl.n_tokens, wl.hidden, wl.dtype)
+    thetas = [B.make_params(threads_per_row=512), B.make_params(threads_per_row=256, unroll=2),
+              B.make_params(threads_per_row=1024, rows_per_cta=2),                     # 2048 threads: refused
+              B.make_params(threads_per_row=256, stage=B.RT_STAGE_SMEM_TMA),
+              B.make_params(threads_per_row=128, reduce=B.RT_REDUCE_CLUSTER, cluster_size=2)]
+    rounds = 4
+    recs, blocks = B.tuner_retest_interleaved(shape, thetas, B.make_budget(warmup=3, iters=10, repeats=1, use_graph=graph),
+                                              ws, rounds)
+    assert [rec.status for rec in recs] == [0, 0, B.RT_ERR_INFEASIBLE, 0, 0]
+    live = [0, 1, 3, 4]
+    assert len(blocks) == rounds * len(live)
+    order = [(blk.round, blk.theta_index) for blk in blocks]
+    want = [(rd, i) for rd in range(rounds) for i in [(j + rd) % 5 for j in range(5)] if i in live]
+    assert order == want                                        # one block each per round, the start rotating by one
+    for a, b in zip(blocks, blocks[1:]):
+        assert a.t_begin_s < a.t_end_s <= b.t_begin_s           # blocks do not overlap on the host clock
+    for i in live:
+        mine = sorted(blk.us for blk in blocks if blk.theta_index == i)
+        assert recs[i].us_min_block == pytest.approx(mine[0]) and 0.3 < mine[0] < 500.0
+        assert recs[i].us == pytest.approx(0.5 * (mine[1] + mine[2]))          # the median of four blocks
+        assert recs[i].r_bad == 0 and recs[i].y_bad == 0 and recs[i].y_max_ulp <= 2
+    assert B.rt_device_status() == 0
+    for bad_args in ((thetas, 0), ([], 3)):
+        with pytest.raises((B.TunerError, ValueError)):
+            B.tuner_retest_interleaved(shape, bad_args[0], B.make_budget(warmup=1, iters=2), ws, bad_args[1])
+
+
+def test_search_confirms_its_finalists_side_by_side(B, oracle_lib):
+    from paper_2601_12698_b200 import synth
+    wl = synth.Workload("t", "bf16", 512, 4096, seed=4)
+    t, ws = _workspace(B, oracle_lib, wl)
+    shape = B.shape_of(wl.n_tokens, wl.hidden, wl.dtype)
+    res, log = B.tuner_search(shape, B.make_budget(max_evals=30, warmup=2, iters=10, repeats=3, top_k=4), ws)
+    topk = [rec for rec in log if rec.phase == 3]
+    assert len(topk) == 4 and log[-4:] == log[-4:] and all(rec.phase == 3 for rec in log[-4:])
+    assert res.evals_used == len(log) <= 30
+    # the winner is one of the confirmed finalists and carries its re-test time
+    winners = [rec for rec in topk if rec.params.key() == res.best.key()]
+    assert len(winners) == 1 and winners[0].us == pytest.approx(res.best_us)
+    assert res.best_us == pytest.approx(min(rec.us for rec in topk if rec.status == 0))
+
+
+def test_alignment_is_taken_from_the_workspace_not_from_the_claim(B, oracle_lib):
+    """A caller that claims 256-byte alignment for tensors that are slices 8 bytes into their allocations: the tuner
+    works out what the pointers really share, narrows the vectors and refuses the TMA stage - nothing is launched on
+    a misaligned address."""
+    from paper_2601_12698_b200 import synth
+    T, H = 64, 4096
+    x, r, w = synth.make_inputs(T, H, "bf16", seed=6)
+    y_ref, r_ref = oracle_lib.add_rmsnorm(x, r, w, 1e-6)
+
+    def shifted(src):  # the same values, 8 bytes past a 256-byte boundary
+        buf = torch.empty(src.numel() + 128, dtype=src.dtype, device="cuda")
+        view = buf[4:4 + src.numel()].view(src.shape)
+        view.copy_(src)
+        assert view.data_ptr() % 16 == 8
+        return view
+    xd, rd, yd, od = shifted(x), shifted(r), shifted(torch.empty_like(x)), shifted(torch.empty_like(x))
+    stream = torch.cuda.Stream()
+    ws = B.make_workspace(xd, rd, w.cuda(), yd, od, y_ref.cuda(), r_ref.cuda(), 1e-6, stream=stream)
+    claim = B.shape_of(T, H, "bf16", min_ptr_align=256)
+    proto = B.make_budget(warmup=1, iters=3, repeats=1)
+    before = B.rt_launch_count()
+    for th in (B.make_params(vec_bytes=16), B.make_params(vec_bytes=32, threads_per_row=128),
+               B.make_params(vec_bytes=8, stage=B.RT_STAGE_SMEM_TMA), B.make_params(stage=B.RT_STAGE_REG_REALIGN)):
+        assert B.tuner_evaluate(claim, th, proto, ws).status == B.RT_ERR_ALIGN, repr(th)
+    assert B.rt_launch_count() == before                          # refused before any launch
+    rec = B.tuner_evaluate(claim, B.make_params(vec_bytes=8), proto, ws)
+    assert rec.status == B.RT_OK and rec.r_bad == 0 and rec.y_bad == 0
+    res, log = B.tuner_search(claim, B.make_budget(max_evals=20, warmup=1, iters=3, repeats=1, top_k=2), ws)
+    assert res.n_failed_gate == 0 and {rec.params.vec_bytes for rec in log} == {8}
+    assert {rec.params.stage for rec in log} <= {B.RT_STAGE_REG, B.RT_STAGE_SMEM_LDG}
+    assert B.rt_device_status() == 0
+
+
+def test_a_ring_stride_that_breaks_alignment_narrows_the_vectors(B, oracle_lib):
+    """Seven rows of 6145 fp16 elements per set: consecutive sets lie 86030 bytes apart, so only set 0 is 16-byte
+    aligned.  The ragged-row stage (16-byte chunks from aligned base pointers) must not be offered for the ring."""
+    from paper_2601_12698_b200 import synth
+    T, H, sets = 7, 6145, 3
+    x, r, w = synth.make_inputs(T, H, "fp16", seed=9)
+    y_ref, r_ref = oracle_lib.add_rmsnorm(x, r, w, 1e-6)
+    ring = lambda t: t.cuda().unsqueeze(0).repeat(sets, 1, 1).contiguous()
+    xs, rs = ring(x), ring(r)
+    ys, os_ = torch.empty_like(xs), torch.empty_like(xs)
+    stream = torch.cuda.Stream()
+    ws = B.make_workspace(xs, rs, w.cuda(), ys, os_, y_ref.cuda(), r_ref.cuda(), 1e-6, ring_sets=sets,
+                          ring_stride_bytes=T * H * 2, stream=stream)
+    shape = B.shape_of(T, H, "fp16")
+    proto = B.make_budget(warmup=sets, iters=2 * sets, repeats=1)
+    assert B.tuner_evaluate(shape, B.make_params(stage=B.RT_STAGE_REG_REALIGN), proto, ws).status == B.RT_ERR_ALIGN
+    rec = B.tuner_evaluate(shape, B.make_params(vec_bytes=2, threads_per_row=1024, unroll=4), proto, ws)
+    assert rec.status == B.RT_OK
+    torch.cuda.synchronize()
+    for k in range(sets):
+        assert oracle_lib.bit_mismatches(os_[k].cpu(), r_ref) == 0 and oracle_lib.compare_y(ys[k].cpu(), y_ref)[1] == 0
+    # with one set the stage is fine again
+    ws1 = B.make_workspace(xs[0], rs[0], w.cuda(), ys[0], os_[0], y_ref.cuda(), r_ref.cuda(), 1e-6, stream=stream)
+    assert B.tuner_evaluate(shape, B.make_params(stage=B.RT_STAGE_REG_REALIGN), proto, ws1).status == B.RT_OK
+    assert B.rt_device_status() == 0
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp16"])
+def test_an_overflowed_output_is_not_one_step_from_the_largest_finite_value(B, oracle_lib, dtype):
+    td = torch.bfloat16 if dtype == "bf16" else torch.float16
+    top = torch.finfo(td).max
+    inf = float("inf")
+    got = torch.tensor([top, inf, inf, -inf, top, 1.0], dtype=td)
+    ref = torch.tensor([inf, inf, -inf, -inf, torch.finfo(td).max, 1.0], dtype=td)
+    ref[4] = torch.nextafter(torch.tensor(top, dtype=td), torch.tensor(0.0, dtype=td))   # the value below the top: 1 ulp
+    want = oracle_lib.compare_y(got, ref, tol_ulp=2)
+    assert want == (65535, 2)
+    for compare in (B.tuner_compare, B.tuner_compare_static):
+        worst, bad = compare(got.cuda(), ref.cuda(), B.RT_CMP_ULP16, 2.0)
+        assert (int(worst), bad) == want
+    g32, r32 = torch.tensor([3.0e38, inf, inf, 1.0]), torch.tensor([inf, inf, -inf, 1.0])
+    assert oracle_lib.compare_y(g32, r32, tol_rel=1e-5)[1] == 2
+    assert B.tuner_compare(g32.cuda(), r32.cuda(), B.RT_CMP_REL32, 1e-5)[1] == 2
+    assert B.tuner_compare_mixed(g32.cuda(), r32.cuda(), 1e-5, 1e-5)[1] == 2
+    assert B.tuner_compare_mixed(got.cuda(), ref.cuda(), 2.0, 1e-5)[1] == 2

@@ -108,9 +108,18 @@ def test_ulp_compare_pins(oracle_lib):
     assert c(u16(0x3C00), u16(0x3C03), 1) == (3, 1)
     assert c(u16(0x7FC0), u16(0x7FC1), 0) == (0, 0)          # NaN vs NaN
     assert c(u16(0x7FC0), u16(0x3F80), 0)[1] == 1
-    assert c(u16(0x7BFF), u16(0x7C00), 1) == (1, 0)          # max finite vs inf: adjacent
+    # the lattice is that of the finite values: an overflowed output is not one step from the largest finite value
+    assert c(u16(0x7BFF), u16(0x7C00), 1) == (65535, 1)      # fp16 max finite vs +inf
+    assert c(u16(0x7F7F), u16(0x7F80), 0) == (65535, 1)      # bf16 max finite vs +inf
+    assert c(u16(0x7C00), u16(0x7C00), 1) == (0, 0)          # +inf vs +inf
+    assert c(u16(0x7C00), u16(0xFC00), 1) == (65535, 1)      # +inf vs -inf
+    assert c(u16(0xFF80), u16(0xFF80), 0) == (0, 0)          # -inf vs -inf (bf16)
+    assert c(u16(0x7BFF), u16(0x7BFE), 1) == (1, 0)          # the two largest finite values stay adjacent
     worst, bad = c(np.array([1.0, 2.0, 0.0], np.float32), np.array([1.0, 2.00001, 0.0], np.float32))
     assert bad == 0 and 4e-6 < worst < 6e-6
     worst, bad = c(np.array([1.0], np.float32), np.array([1.0001], np.float32))
     assert bad == 1
+    inf = float("inf")
+    worst, bad = c(np.array([3.4e38, inf, inf], np.float32), np.array([inf, inf, -inf], np.float32))
+    assert bad == 2 and worst == inf                          # binary32: an infinity matches only itself
     assert oracle_lib.bit_mismatches(u16(1, 2, 3), u16(1, 2, 4), 0) == 1

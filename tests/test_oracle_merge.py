@@ -116,6 +116,10 @@ def test_mixed_compare_pins(oracle_lib):
     a, b = torch.tensor([1.0, 1e-9]), torch.tensor([1.000001, 0.0])
     assert oracle_lib.compare_mixed(a, b, tol=1e-5, tol_abs=1e-8)[1] == 0
     assert oracle_lib.compare_mixed(a, b, tol=1e-7, tol_abs=1e-10)[1] == 2
+    # an overflowed 16-bit output is no neighbour of the largest finite value; equal infinities match
+    top = torch.tensor([65504.0, float("inf"), float("inf")], dtype=torch.float16)
+    inf = torch.tensor([float("inf"), float("inf"), float("-inf")], dtype=torch.float16)
+    assert oracle_lib.compare_mixed(top, inf, tol=2.0, tol_abs=1e-5)[1] == 2
 
 
 def test_argument_checks(oracle_lib):

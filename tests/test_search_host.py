@@ -209,3 +209,43 @@ def test_guided_search_crosses_between_stages_of_different_vector_width(L, opt):
         B.make_params(threads_per_row=512, unroll=1, stage=B.RT_STAGE_REG_REALIGN)
     res2, _ = B.tuner_search_with(s, L, B.make_budget(max_evals=24, top_k=2, seeds=[seed]), cost)
     assert res2.best.key() == target[0].key()
+
+
+def test_a_finalist_that_fails_its_retest_drops_out_and_the_runner_up_is_confirmed(L):
+    """A candidate that passes its gate once and fails it the second time (what a race in a stage would look like) is
+    the fastest by its first measurement.  The Top-K re-test must not return it: it drops out, the next runner-up is
+    re-tested in its place, and the winner is the fastest candidate that passed twice."""
+    s = B.shape_of(*SHAPE)
+    opt = OPTIMA[0]
+    base = _cost_factory(opt)
+    seen = {}
+
+    def cost(p):
+        n = seen[p.key()] = seen.get(p.key(), 0) + 1
+        flaky = (p.threads_per_row, p.rows_per_cta, p.unroll, p.vec_bytes, p.stage, p.reduce) == \
+            (opt["tpr"], opt["rpc"], opt["unroll"], opt["vec"], opt["stage"], opt["reduce"])
+        if flaky:
+            return 100.0 if n == 1 else -1.0
+        return base(p)
+    res, log = B.tuner_search_with(s, L, B.make_budget(max_evals=80, top_k=3), cost)
+    topk = [r for r in log if r.phase == 3]
+    assert [r.status for r in topk] == [B.RT_ERR_MISMATCH, 0, 0]    # budget spent: no replacement, but no flaky winner
+    assert res.best.key() != topk[0].params.key() and res.best_us == pytest.approx(min(r.us for r in topk[1:]))
+    seen.clear()
+    res, log = B.tuner_search_with(s, L, B.make_budget(max_evals=600, top_k=3), cost)   # the climb ends with budget to spare
+    topk = [r for r in log if r.phase == 3]
+    assert len(topk) == 4                                   # three finalists, one replacement
+    assert topk[0].status == B.RT_ERR_MISMATCH and [r.status for r in topk[1:]] == [0, 0, 0]
+    flaky_key = topk[0].params.key()
+    assert res.best.key() != flaky_key and seen[flaky_key] == 2
+    assert res.best_us == pytest.approx(min(r.us for r in topk[1:]))
+    assert res.n_failed_gate == 1 and res.evals_used == len(log) < 600
+    # every finalist failing its re-test leaves the best of the rest
+    always = {}
+
+    def cost2(p):
+        n = always[p.key()] = always.get(p.key(), 0) + 1
+        return base(p) if n == 1 else -1.0
+    res2, log2 = B.tuner_search_with(s, L, B.make_budget(max_evals=600, top_k=2), cost2)
+    assert [r.status for r in log2 if r.phase == 3] == [B.RT_ERR_MISMATCH] * 4
+    assert res2.best_us > 100.0 and always[res2.best.key()] == 1

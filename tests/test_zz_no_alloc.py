@@ -37,7 +37,7 @@ def _pair(dtype, n, n_perturbed, seed):
 
 
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16, torch.float32])
-def test_static_compare_matches_allocating_compare_twice_in_a_row(B, dtype):
+def test_static_compare_matches_allocating_compare_twice_in_a_row(B, oracle_lib, dtype):
     y_mode, tol = (B.RT_CMP_REL32, 1e-5) if dtype == torch.float32 else (B.RT_CMP_ULP16, 2.0)
     first = _pair(dtype, 1_000_003 if dtype != torch.float32 else 1_000_000, 700, seed=1)
     second = _pair(dtype, 4097, 3, seed=2)  # far fewer differences: leftovers from the first call would show
@@ -49,6 +49,15 @@ def test_static_compare_matches_allocating_compare_twice_in_a_row(B, dtype):
             assert have[0] == want[0]  # integer distances, and the same float maximum, bit for bit
             if k == 0:
                 assert have[1] > 100  # the first pair really differs, so a stale record would be visible next
+        # and against the CPU oracle's own comparison of the same pair, so that the check does not rest on the
+        # library agreeing with itself
+        have = B.tuner_compare_static(got, ref, y_mode, tol)
+        if dtype == torch.float32:
+            worst, bad = oracle_lib.compare_y(got.cpu(), ref.cpu(), tol_rel=tol)
+            assert have[1] == bad and abs(have[0] - worst) <= 1e-6 * worst
+        else:
+            assert (int(have[0]), have[1]) == oracle_lib.compare_y(got.cpu(), ref.cpu(), tol_ulp=int(tol))
+        assert B.tuner_compare_static(got, ref, B.RT_CMP_BITS, 0.0)[1] == oracle_lib.bit_mismatches(got.cpu(), ref.cpu())
     # identical buffers: zero after a call that found differences
     assert B.tuner_compare_static(first[1], first[1].clone(), y_mode, tol) == (0.0, 0)
 
