@@ -445,18 +445,21 @@ def run_ours(args) -> None:
             raise SystemExit("--theta takes tpr,rpc,vec,unroll,stage,reduce,cluster")
         tuner = {"skipped": "theta given on the command line"}
     elif rank == 0:
-        counts = B.tuner_derive_counts(shape)
+        # --include-pipeline puts the persistent TMA pipeline stage, which the default candidate set leaves out, into
+        # both searches (and so into the per-stage table below)
+        mask = B.RT_PRUNE_DEFAULT & ~B.RT_PRUNE_PIPELINE_STAGE if args.include_pipeline else B.RT_PRUNE_DEFAULT
+        counts = B.tuner_derive_counts(shape, heuristics=mask)
         # Both searches time every candidate with the paper's protocol (20 warm-up launches, blocks of 100).
         t0 = time.perf_counter()
         sweep, sweep_log = B.tuner_search(shape, B.make_budget(max_evals=counts["feasible"], warmup=20, iters=100, repeats=2,
                                                                top_k=0, strategy=B.RT_SEARCH_EXHAUSTIVE,
-                                                               use_graph=use_graph), ws)
+                                                               use_graph=use_graph, heuristics=mask), ws)
         sweep_s = time.perf_counter() - t0
         seeds = resume_seeds(args.resume, wl.name) if args.resume else None
         t0 = time.perf_counter()
         guided, guided_log = B.tuner_search(shape, B.make_budget(max_evals=args.search_budget, warmup=20, iters=100,
                                                                  repeats=3, top_k=args.top_k, use_graph=use_graph,
-                                                                 seeds=seeds), ws)
+                                                                 seeds=seeds, heuristics=mask), ws)
         guided_s = time.perf_counter() - t0
         # Search-best against exhaustive-best, measured side by side: the sweep's fastest --retest-top points, the
         # guided winner and its runner-up are re-timed together, block by block in rotation (20 warm-up + 100 timed
@@ -516,6 +519,13 @@ def run_ours(args) -> None:
         }
         if seeds:
             tuner["resumed_seeds"] = len(seeds)
+        # the sweep's fastest point of every stage (first measurement, us): which organisation of the row wins here
+        by_stage = {}
+        for rec in sweep_log:
+            name = B.STAGE_NAMES.get(rec.params.stage, str(rec.params.stage))
+            if rec.status == 0 and (name not in by_stage or rec.us < by_stage[name][0]):
+                by_stage[name] = (rec.us, list(rec.params.key()))
+        tuner["sweep_best_per_stage"] = {name: {"us": round(us, 3), "theta": th} for name, (us, th) in sorted(by_stage.items())}
         if args.seed_thetas:
             # Cross-shape transfer: the same small budget, cold and seeded with configurations found on other
             # shapes; "evaluations to within 3%" counts evaluations until one scores within 3% of the
@@ -929,6 +939,7 @@ def main() -> None:
                     "cold-versus-seeded transfer experiment")
     ap.add_argument("--transfer-budget", type=int, default=24)
     ap.add_argument("--log", default="", help="write every evaluated theta of both searches to this JSONL file")
+    ap.add_argument("--include-pipeline", action="store_true", help="search the persistent TMA pipeline stage as well")
     ap.add_argument("--resume", default="", help="a JSONL file written by --log: its fastest thetas seed the guided search")
     ap.add_argument("--retest-top", type=int, default=8, help="points of the sweep re-timed beside the guided winner")
     ap.add_argument("--retest-rounds", type=int, default=7, help="rounds of the side-by-side re-test")

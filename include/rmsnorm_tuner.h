@@ -64,12 +64,12 @@ typedef enum {
     RT_STAGE_REG = 0,      /* ld.global vectors straight into registers, row kept as fp32 registers */
     RT_STAGE_SMEM_LDG = 1, /* ld.global vectors, sum kept as fp32 in shared memory */
     RT_STAGE_SMEM_TMA = 2, /* cp.async.bulk (TMA, one copy per row slice) into shared memory + mbarrier */
-    RT_STAGE_REG_REALIGN = 3, /* add_rmsnorm only, for rows whose byte length is not a multiple of 16 (the paper's
-                                "vectorization and alignment strategies" axis): the row is cut at the 16-byte
-                                boundaries of the tensor; the whole chunks between them move as 16-byte vectors and
-                                stay in registers, the fewer than 16 bytes before the first and after the last
-                                boundary move one element to a thread.  Takes vec_bytes = 16, the shuffle reduction,
-                                16-byte aligned base pointers and any hidden size */
+    RT_STAGE_REG_REALIGN = 3, /* add_rmsnorm only, for rows whose byte length is not a multiple of the vector width
+                                (the paper's "vectorization and alignment strategies" axis): the row is cut at the
+                                vec_bytes boundaries of the tensor; the whole chunks between them move as vectors of
+                                vec_bytes and stay in registers, the fewer than vec_bytes bytes before the first and
+                                after the last boundary move one element to a thread.  Takes vec_bytes = 16 or 32, the
+                                shuffle reduction, base pointers aligned to vec_bytes and any hidden size */
     RT_STAGE_TMA_PIPELINE = 4 /* add_rmsnorm only ("loop scheduling" in the paper's list of tuning dimensions): a
                                  persistent grid - as many CTAs as stay resident on the device, each walking over row
                                  blocks b, b + grid, ... - with a ring of `unroll` shared-memory stages per row slot
@@ -92,7 +92,7 @@ typedef struct {
     int32_t threads_per_row; /* threads cooperating on one row (blockDim.x); power of two, 32..1024 */
     int32_t rows_per_cta;    /* rows handled by one CTA (blockDim.y); 1..8 */
     int32_t vec_bytes;       /* bytes per ld/st: 32 (the 256-bit global accesses of sm_100), 16
-                                or 8 (4 and 2 exist as a narrow fall-back); 16 with
+                                or 8 (4 and 2 exist as a narrow fall-back); 16 or 32 with
                                 RT_STAGE_REG_REALIGN, whatever the row length */
     int32_t unroll;          /* independent vector loads in flight per thread and tensor: 1, 2, 4 */
     int32_t stage;           /* rt_stage */
@@ -438,6 +438,28 @@ int tuner_retest_interleaved(const rt_shape* s, const rt_params* thetas, int32_t
  * Synchronises `stream`.  (Measurement aid for "Performance Measurement"; the paper has no counterpart.)
  */
 int tuner_launch_floor(const rt_budget* b, void* stream, float* us);
+
+/*
+ * rmsnorm_template_launch through an instrumented instance of the same template, for the latency-bound shapes
+ * (measurement aid; "Performance Measurement" in the paper times whole kernels only).  The first thread of every CTA
+ * records, into RT_TRACE_WORDS 64-bit words at trace[cta * RT_TRACE_WORDS]:
+ *   [0] the global nanosecond timer at kernel entry      [6] the same timer just before the CTA exits
+ *   [1] SM cycle counter at entry                        [2] ... once the previous kernel of the stream has completed
+ *   [3] ... once the thread's share of x and r has arrived and been summed
+ *   [4] ... once the row's sum of squares is reduced     [5] ... once the thread's last store has been issued
+ *   [7] the SM the CTA ran on.
+ * Cycle counts of one CTA are comparable with each other (one SM); the nanosecond timer is comparable across CTAs and
+ * launches but ticks coarsely.  Instrumented instances exist for bf16 and fp32 with vec_bytes = 16 and unroll 1: the
+ * register stage with at most two vectors per thread (all three reductions for bf16 with one vector per thread) and,
+ * for bf16, the TMA stage; any other theta returns RT_ERR_INFEASIBLE.  trace: device, trace_words >= the value
+ * rmsnorm_trace_words returns for this theta and shape (RT_ERR_CAPACITY otherwise; -1 from rmsnorm_trace_words when
+ * theta is infeasible).  Outputs are the operator's, as from rmsnorm_template_launch.  Asynchronous, allocates nothing.
+ */
+#define RT_TRACE_WORDS 8
+int rmsnorm_template_launch_traced(const rt_params* p, const void* x, const void* r, const void* w, void* y, void* r_out,
+                                   int64_t n_tokens, int64_t hidden, float eps, int dtype, uint64_t* trace,
+                                   int64_t trace_words, void* stream);
+int64_t rmsnorm_trace_words(const rt_params* p, int64_t n_tokens, int64_t hidden, int dtype);
 
 /* ---- 4. general configuration and specialised table -------------------------------------- */
 

@@ -126,6 +126,9 @@ _SIGNATURES = {
     "rt_get_option": (c_int32, [c_int32]),
     "merge_attn_states_template_launch": (c_int, [POINTER(rt_params), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                                   c_void_p, c_int64, c_int64, c_int64, c_int, c_void_p]),
+    "rmsnorm_template_launch_traced": (c_int, [POINTER(rt_params), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                               c_int64, c_int64, c_float, c_int, c_void_p, c_int64, c_void_p]),
+    "rmsnorm_trace_words": (c_int64, [POINTER(rt_params), c_int64, c_int64, c_int]),
     "rmsnorm_template_run_host": (c_int, [POINTER(rt_params), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                           c_int64, c_int64, c_float, c_int, c_void_p, c_int64, c_int64, c_void_p]),
     "rmsnorm_host_workspace_bytes": (c_int64, [c_int64, c_int64, c_int, c_int64]),
@@ -249,6 +252,23 @@ def rmsnorm_template_launch(params: rt_params, x, r, w, y, r_out, eps: float, st
     _check(lib.rmsnorm_template_launch(byref(params), x.data_ptr(), r.data_ptr(), w.data_ptr(), y.data_ptr(),
                                        r_out.data_ptr(), n_tokens, hidden, eps, _dtype_code(x), _stream_ptr(stream)),
            "rmsnorm_template_launch")
+
+
+RT_TRACE_WORDS = 8
+
+
+def rmsnorm_template_launch_traced(params: rt_params, x, r, w, y, r_out, eps: float, trace, stream=None) -> None:
+    """rmsnorm_template_launch through an instrumented instance; `trace` is an int64 device tensor of at least
+    rmsnorm_trace_words(...) elements that receives RT_TRACE_WORDS words per CTA."""
+    n_tokens, hidden = x.shape
+    _check(lib.rmsnorm_template_launch_traced(byref(params), x.data_ptr(), r.data_ptr(), w.data_ptr(), y.data_ptr(),
+                                              r_out.data_ptr(), n_tokens, hidden, eps, _dtype_code(x), trace.data_ptr(),
+                                              trace.numel(), _stream_ptr(stream)), "rmsnorm_template_launch_traced")
+
+
+def rmsnorm_trace_words(params: rt_params, n_tokens: int, hidden: int, dtype) -> int:
+    code = DTYPE_CODES[dtype] if isinstance(dtype, str) else int(dtype)
+    return int(lib.rmsnorm_trace_words(byref(params), n_tokens, hidden, code))
 
 
 def silu_and_mul_template_launch(params: rt_params, x, out, stream=None) -> None:

@@ -28,7 +28,7 @@ LIB_PATH = os.path.join(HERE, "librmsnorm_tuner.so")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-std=c++17", "-O3", "-lineinfo",
               "-Xcompiler", "-fPIC", "-I", CSRC, "-I", INCLUDE]
-HOST_UNITS = ["launch.cu", "feasible.cu", "search.cu", "host_run.cu", "table.cu"]
+HOST_UNITS = ["launch.cu", "feasible.cu", "search.cu", "host_run.cu", "table.cu", "trace.cu"]
 ELEMENT_TYPES = {"bf16": ("__nv_bfloat16", 0), "fp16": ("__half", 1), "fp32": ("float", 2)}
 GROUPS = {"reg": 0, "smem": 1, "narrow": 2, "silu": 3, "merge": 4, "fp8out": 5, "allreduce": 6, "realign": 7}
 
@@ -50,7 +50,8 @@ def unit_flags(name: str) -> list[str]:
     return flags
 
 
-_ENTRY = re.compile(r"Compiling entry function '_ZN2rt18add_rmsnorm_kernelI(\w+?)Li(\d+)ELi(\d+)ELi(\d+)ELi(\d+)ELi(\d+)E"
+# (the plain instances: TRACE = false, mangled Lb0E; the instrumented ones of trace.cu are not part of the table)
+_ENTRY = re.compile(r"Compiling entry function '_ZN2rt18add_rmsnorm_kernelI(\w+?)Li(\d+)ELi(\d+)ELi(\d+)ELi(\d+)ELi(\d+)ELb0E"
                     r"EEvNS_10KernelArgsE'.*?(\d+) bytes spill stores.*?Used (\d+) registers.*?(\d+) bytes smem", re.S)
 _MANGLED_DTYPE = {"13__nv_bfloat16": 0, "6__half": 1, "f": 2}
 

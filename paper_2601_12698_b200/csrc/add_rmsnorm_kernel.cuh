@@ -9,7 +9,9 @@
 //
 // Compile-time axes: element type, VB, STAGE, REDUCE, U and - for the two register stages - CAP, the
 // number of row vectors one thread keeps.  Run-time axes: blockDim.x = threads per row,
-// blockDim.y = rows per CTA, cluster size.
+// blockDim.y = rows per CTA, cluster size.  In the persistent pipeline stage U is the depth of the ring of
+// shared-memory stages ("loop scheduling"): the grid is as large as the device keeps resident, and a CTA walks
+// over row blocks with the bulk copies of its next U - 1 blocks in flight.
 //
 // Per row:  s = fp32(x) + fp32(r);  r_out = rn(s);  y = rn(s * rsqrt(mean(s^2) + eps) * w).
 // The sum of squares is combined in a fixed order (no atomics): results are deterministic.
@@ -28,6 +30,8 @@ constexpr int kStageReg = 0;
 constexpr int kStageSmemLdg = 1;
 constexpr int kStageSmemTma = 2;
 constexpr int kStageRegRealign = 3;
+constexpr int kStageTmaPipeline = 4;
+constexpr int kMaxPipelineDepth = 4;
 constexpr int kReduceShfl = 0;
 constexpr int kReduceSmem = 1;
 constexpr int kReduceCluster = 2;
@@ -52,6 +56,50 @@ struct KernelArgs {
     int* status;     // device status word
     unsigned wait_polls;  // polls a bounded mbarrier wait may take (kMbarrierPollLimit unless the caller lowered it)
     int drop_copies;      // diagnostic: 1 = the TMA stages post no copy, so their waits run out and report it
+    unsigned long long* trace;  // instrumented instances only: kTraceWords words per CTA
+};
+
+// Phase stamps of the instrumented instances (TRACE = true): SM cycle counts taken by the CTA's first thread at entry,
+// after the wait for the previous kernel, when its share of x and r has arrived and been summed, after the row
+// reduction, and after its last store was issued; plus the global nanosecond timer at entry and exit and the SM
+// the CTA ran on.  Kept in registers and written once at the end, so that the stamps disturb the kernel as little
+// as a stamp can.  With TRACE = false every member is empty and compiles to nothing.
+constexpr int kTraceWords = 8;
+enum { kTraceEntry = 0, kTraceReleased = 1, kTraceLoaded = 2, kTraceReduced = 3, kTraceStored = 4 };
+template <bool TRACE>
+struct PhaseTrace {
+    long long cycles[TRACE ? 5 : 1];
+    unsigned long long ns_entry;
+    __device__ __forceinline__ void begin()
+    {
+        if constexpr (TRACE) {
+#pragma unroll
+            for (int k = 0; k < 5; ++k) cycles[k] = 0;
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns_entry));
+            cycles[kTraceEntry] = clock64();
+        }
+    }
+    __device__ __forceinline__ void mark(int phase)
+    {
+        if constexpr (TRACE) cycles[phase] = clock64();
+    }
+    __device__ __forceinline__ void flush(const KernelArgs& a)
+    {
+        if constexpr (TRACE) {
+            if (threadIdx.x == 0 && threadIdx.y == 0 && a.trace) {
+                unsigned long long ns_exit;
+                unsigned smid;
+                asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns_exit));
+                asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+                unsigned long long* out = a.trace + (size_t)blockIdx.x * kTraceWords;
+                out[0] = ns_entry;
+#pragma unroll
+                for (int k = 0; k < 5; ++k) out[1 + k] = (unsigned long long)cycles[k];
+                out[6] = ns_exit;
+                out[7] = smid;
+            }
+        }
+    }
 };
 
 // ---- vectors of VB bytes ------------------------------------------------------------------------
@@ -261,13 +309,13 @@ struct Codec {
 
 // ---- ragged rows (STAGE == kStageRegRealign) -----------------------------------------------------
 //
-// A row whose byte length is not a multiple of 16 starts at a different offset inside a 16-byte chunk from one
-// row to the next, so no vector wider than the row length's alignment divides it.  This stage cuts the row at
-// the 16-byte boundaries of the tensor instead: a head of fewer than EPV elements up to the first boundary,
-// the whole aligned chunks (moved as 16-byte vectors, kept in registers like the register stage), and a tail of
-// fewer than EPV elements.  Head and tail elements go one to a thread, so no byte outside the row is touched.
-// Only the weights are then out of step: the weights of a whole chunk start `phase` bytes past a 16-byte
-// boundary of w, the same phase for every chunk of the row.
+// A row whose byte length is not a multiple of the chunk width VB (16 or 32 bytes) starts at a different offset
+// inside a chunk from one row to the next, so no vector that wide divides it.  This stage cuts the row at the
+// VB-byte boundaries of the tensor instead: a head of fewer than EPV elements up to the first boundary, the whole
+// aligned chunks (moved as VB-byte vectors, kept in registers like the register stage), and a tail of fewer than EPV
+// elements.  Head and tail elements go one to a thread, so no byte outside the row is touched.  Only the weights are
+// then out of step: the weights of a whole chunk start `phase` bytes past a 16-byte boundary of w, the same phase
+// for every chunk of the row.
 
 template <int VB, bool EARLY>
 __device__ __forceinline__ Vec<VB> ld_weight_at(const void* p)
@@ -276,45 +324,47 @@ __device__ __forceinline__ Vec<VB> ld_weight_at(const void* p)
     else return ld_weight<VB>(p);
 }
 
-// Sixteen bytes of w from address p (a multiple of the element size; `phase` = p modulo 16, the same for every
-// chunk of a row).  phase = 0: one aligned vector.  Otherwise the two aligned vectors around p, shifted together
-// (`whole_pair`: both lie inside w), or - for the one chunk per row whose second vector would reach past the end of
-// w - element by element.  EARLY pins the loads in program order, for a fetch ahead of the row reduction.
-template <typename T, bool EARLY>
-__device__ __forceinline__ Vec<16> ld_weight_ragged(const unsigned char* p, int phase, bool whole_pair)
+// out.w[k] = the 32-bit word that starts WS words and `sh` bits into the aligned words a[].
+template <int NW, int WS>
+__device__ __forceinline__ void shift_words(const uint32_t (&a)[NW + 4], uint32_t sh, uint32_t (&out)[NW])
 {
-    if (phase == 0) return ld_weight_at<16, EARLY>(p);
-    Vec<16> v;
-    if (!whole_pair) {
+#pragma unroll
+    for (int k = 0; k < NW; ++k) out[k] = __funnelshift_r(a[k + WS], a[k + WS + 1], sh);
+}
+
+// VB bytes of w from address p (a multiple of the element size; `phase` = p modulo 16, the same for every chunk of
+// a row).  phase = 0: aligned vectors.  Otherwise the VB / 16 + 1 aligned 16-byte vectors around p, shifted together
+// (`whole_span`: all of them lie inside w), or - for the one chunk per row whose last vector would reach past the
+// end of w - element by element.  EARLY pins the loads in program order, for a fetch ahead of the row reduction.
+template <typename T, int VB, bool EARLY>
+__device__ __forceinline__ Vec<VB> ld_weight_ragged(const unsigned char* p, int phase, bool whole_span)
+{
+    if (phase == 0) return ld_weight_at<VB, EARLY>(p);
+    constexpr int NW = VB / 4;
+    Vec<VB> v;
+    if (!whole_span) {
         if constexpr (sizeof(T) == 4) {
 #pragma unroll
-            for (int k = 0; k < 4; ++k) v.w[k] = ld_weight_at<4, EARLY>(p + 4 * k).w[0];
+            for (int k = 0; k < NW; ++k) v.w[k] = ld_weight_at<4, EARLY>(p + 4 * k).w[0];
         } else {
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
+            for (int k = 0; k < NW; ++k)
                 v.w[k] = ld_weight_at<2, EARLY>(p + 4 * k).w[0] | (ld_weight_at<2, EARLY>(p + 4 * k + 2).w[0] << 16);
         }
         return v;
     }
-    const Vec<16> lo = ld_weight_at<16, EARLY>(p - phase), hi = ld_weight_at<16, EARLY>(p - phase + 16);
+    uint32_t a[NW + 4];
+#pragma unroll
+    for (int q = 0; q < NW / 4 + 1; ++q) {
+        const Vec<16> t = ld_weight_at<16, EARLY>(p - phase + 16 * q);
+        a[4 * q] = t.w[0]; a[4 * q + 1] = t.w[1]; a[4 * q + 2] = t.w[2]; a[4 * q + 3] = t.w[3];
+    }
     const uint32_t sh = (uint32_t)(phase & 3) * 8u;  // 0 or 16 bits inside a word
-    switch (phase >> 2) {
-        case 0:
-            v.w[0] = __funnelshift_r(lo.w[0], lo.w[1], sh); v.w[1] = __funnelshift_r(lo.w[1], lo.w[2], sh);
-            v.w[2] = __funnelshift_r(lo.w[2], lo.w[3], sh); v.w[3] = __funnelshift_r(lo.w[3], hi.w[0], sh);
-            break;
-        case 1:
-            v.w[0] = __funnelshift_r(lo.w[1], lo.w[2], sh); v.w[1] = __funnelshift_r(lo.w[2], lo.w[3], sh);
-            v.w[2] = __funnelshift_r(lo.w[3], hi.w[0], sh); v.w[3] = __funnelshift_r(hi.w[0], hi.w[1], sh);
-            break;
-        case 2:
-            v.w[0] = __funnelshift_r(lo.w[2], lo.w[3], sh); v.w[1] = __funnelshift_r(lo.w[3], hi.w[0], sh);
-            v.w[2] = __funnelshift_r(hi.w[0], hi.w[1], sh); v.w[3] = __funnelshift_r(hi.w[1], hi.w[2], sh);
-            break;
-        default:
-            v.w[0] = __funnelshift_r(lo.w[3], hi.w[0], sh); v.w[1] = __funnelshift_r(hi.w[0], hi.w[1], sh);
-            v.w[2] = __funnelshift_r(hi.w[1], hi.w[2], sh); v.w[3] = __funnelshift_r(hi.w[2], hi.w[3], sh);
-            break;
+    switch (phase >> 2) {  // a branch that is uniform over the row keeps every register index static
+        case 0: shift_words<NW, 0>(a, sh, v.w); break;
+        case 1: shift_words<NW, 1>(a, sh, v.w); break;
+        case 2: shift_words<NW, 2>(a, sh, v.w); break;
+        default: shift_words<NW, 3>(a, sh, v.w); break;
     }
     return v;
 }
@@ -485,9 +535,11 @@ struct SumPlanes {
     }
 };
 
-template <typename T, int VB, int STAGE, int REDUCE, int U, int CAP>
+template <typename T, int VB, int STAGE, int REDUCE, int U, int CAP, bool TRACE = false>
 __global__ void add_rmsnorm_kernel(const KernelArgs a)
 {
+    PhaseTrace<TRACE> trace;
+    trace.begin();
     using C = Codec<T, VB>;
     constexpr int EPV = C::EPV;
     static_assert((STAGE != kStageReg && STAGE != kStageRegRealign) || CAP % U == 0, "the unroll depth divides the per-thread vector count");
@@ -516,6 +568,7 @@ __global__ void add_rmsnorm_kernel(const KernelArgs a)
     unsigned char* orow = reinterpret_cast<unsigned char*>(a.r_out) + row_off;
 
     wait_for_previous_kernel();
+    trace.mark(kTraceReleased);
     float ss = 0.f;
 
     if constexpr (STAGE == kStageReg) {
@@ -569,8 +622,10 @@ __global__ void add_rmsnorm_kernel(const KernelArgs a)
                 if (v < n) wv[i] = ld_weight_early<VB>(wrow + (size_t)v * VB);
             }
         }
+        trace.mark(kTraceLoaded);
         const float total = row_reduce<REDUCE>(ss, tx, ty, tpr, crank, csize);
         const float rho = __frsqrt_rn(total / (float)a.hidden + a.eps);
+        trace.mark(kTraceReduced);
 #pragma unroll
         for (int i = 0; i < CAP; ++i) {
             const int v = tx + i * tpr;
@@ -584,12 +639,12 @@ __global__ void add_rmsnorm_kernel(const KernelArgs a)
             }
         }
     } else if constexpr (STAGE == kStageRegRealign) {
-        static_assert(VB == 16 && REDUCE != kReduceCluster, "ragged rows: 16-byte chunks, one CTA per row");
+        static_assert((VB == 16 || VB == 32) && REDUCE != kReduceCluster, "ragged rows: 16- or 32-byte chunks, one CTA per row");
         constexpr int EB = (int)sizeof(T);
         using C1 = Codec<T, EB>;  // one element
         const bool live = row < a.n_tokens;
         const size_t row_byte = (size_t)(live ? row : 0) * (size_t)a.hidden * EB;
-        int head = (int)((16u - (unsigned)(row_byte & 15u)) & 15u) / EB;  // elements before the first 16-byte boundary
+        int head = (int)(((unsigned)VB - (unsigned)(row_byte & (VB - 1))) & (VB - 1)) / EB;  // elements before the first boundary
         if (head > a.hidden) head = a.hidden;
         const int n_whole = live ? (a.hidden - head) / EPV : 0;            // aligned chunks wholly inside the row
         const int tail = a.hidden - head - n_whole * EPV;                  // elements after the last of them
@@ -603,7 +658,7 @@ __global__ void add_rmsnorm_kernel(const KernelArgs a)
         unsigned char* yc = reinterpret_cast<unsigned char*>(a.y) + chunk_off;
         unsigned char* oc = reinterpret_cast<unsigned char*>(a.r_out) + chunk_off;
         const size_t edge_off = row_byte + (size_t)edge_col * EB;
-        // the chunk whose second aligned weight vector would end past w is read element by element
+        // the chunk whose last aligned weight vector would end past w is read element by element
         const int v_unsafe = (phase != 0 && tail * EB < 16 - phase) ? n_whole - 1 : -1;
         float s[CAP][EPV];
         float s_edge = 0.f;
@@ -646,28 +701,30 @@ __global__ void add_rmsnorm_kernel(const KernelArgs a)
             ss = fmaf(s_edge, s_edge, ss);
             st_stream<EB>(reinterpret_cast<unsigned char*>(a.r_out) + edge_off, C1::pack(sf));
         }
-        // As in the register stage, a thread that owns at most two chunks fetches its weights ahead of the
+        // As in the register stage, a thread that owns at most 32 bytes of the row fetches its weights ahead of the
         // reduction; the one weight of a head or tail element always is.
-        constexpr bool kEarlyWeight = CAP <= 2;
+        constexpr bool kEarlyWeight = CAP * VB <= 32;
         Vec<VB> wv[kEarlyWeight ? CAP : 1];
         Vec<EB> w_edge;
         if constexpr (kEarlyWeight) {
 #pragma unroll
             for (int k = 0; k < CAP; ++k) {
                 const int v = tx + k * tpr;
-                if (v < n_whole) wv[k] = ld_weight_ragged<T, true>(wc + (size_t)v * VB, phase, v != v_unsafe);
+                if (v < n_whole) wv[k] = ld_weight_ragged<T, VB, true>(wc + (size_t)v * VB, phase, v != v_unsafe);
             }
         }
         if (tx < n_edge) w_edge = ld_weight_early<EB>(reinterpret_cast<const unsigned char*>(a.w) + (size_t)edge_col * EB);
+        trace.mark(kTraceLoaded);
         const float total = row_reduce<REDUCE>(ss, tx, ty, tpr, crank, csize);
         const float rho = __frsqrt_rn(total / (float)a.hidden + a.eps);
+        trace.mark(kTraceReduced);
 #pragma unroll
         for (int k = 0; k < CAP; ++k) {
             const int v = tx + k * tpr;
             if (v < n_whole) {
                 float wf[EPV], yf[EPV];
                 if constexpr (kEarlyWeight) C::unpack(wv[k], wf);
-                else C::unpack(ld_weight_ragged<T, false>(wc + (size_t)v * VB, phase, v != v_unsafe), wf);
+                else C::unpack(ld_weight_ragged<T, VB, false>(wc + (size_t)v * VB, phase, v != v_unsafe), wf);
 #pragma unroll
                 for (int e = 0; e < EPV; ++e) yf[e] = s[k][e] * rho * wf[e];
                 st_stream<VB, true>(yc + (size_t)v * VB, C::pack(yf));
@@ -713,8 +770,10 @@ __global__ void add_rmsnorm_kernel(const KernelArgs a)
                 }
             }
         }
+        trace.mark(kTraceLoaded);
         const float total = row_reduce<REDUCE>(ss, tx, ty, tpr, crank, csize);
         const float rho = __frsqrt_rn(total / (float)a.hidden + a.eps);
+        trace.mark(kTraceReduced);
         for (int v0 = tx; v0 < n; v0 += U * tpr) {
             Vec<VB> wv[U];
 #pragma unroll
@@ -735,7 +794,7 @@ __global__ void add_rmsnorm_kernel(const KernelArgs a)
                 }
             }
         }
-    } else {
+    } else if constexpr (STAGE == kStageSmemTma) {
         // TMA: one thread per row posts two bulk copies (x slice, r slice) that complete on the row's
         // mbarrier; the row's threads then work out of shared memory.
         __shared__ __align__(8) uint64_t bars[kMaxRowsPerCta];
@@ -778,8 +837,10 @@ __global__ void add_rmsnorm_kernel(const KernelArgs a)
                 }
             }
         }
+        trace.mark(kTraceLoaded);
         const float total = row_reduce<REDUCE>(ss, tx, ty, tpr, crank, csize);
         const float rho = __frsqrt_rn(total / (float)a.hidden + a.eps);
+        trace.mark(kTraceReduced);
         for (int v0 = tx; v0 < n; v0 += U * tpr) {
             Vec<VB> wv[U];
 #pragma unroll
@@ -801,7 +862,105 @@ __global__ void add_rmsnorm_kernel(const KernelArgs a)
                 }
             }
         }
+    } else {
+        // Persistent pipeline: the grid holds as many CTAs as stay resident; CTA b handles row blocks b, b + grid,
+        // b + 2 grid, ...  Every row slot of the CTA owns a ring of U shared-memory stages, each with its own
+        // mbarrier.  The slot's first thread posts the bulk copies of block i + U into a stage as soon as the slot's
+        // threads have finished with block i in it, so up to U - 1 blocks are on their way while one is reduced and
+        // stored.  Stage i % U is filled for the (i / U)-th time by block i: its mbarrier phase is (i / U) & 1.
+        static_assert(REDUCE != kReduceCluster, "the pipeline stage keeps a row inside one CTA");
+        static_assert(U <= kMaxPipelineDepth, "ring deeper than the barrier array");
+        constexpr int IU = 2;  // vectors per thread and batch in the two passes over a stage
+        __shared__ __align__(8) uint64_t bars[kMaxPipelineDepth][kMaxRowsPerCta];
+        const size_t row_bytes = (size_t)a.nvec * VB;
+        const size_t stage_bytes = (size_t)blockDim.y * 2 * row_bytes;  // one stage: x and r of every row slot
+        const long long n_blocks = (a.n_tokens + blockDim.y - 1) / blockDim.y;
+        const long long stride = gridDim.x;
+        const unsigned char* xbase = reinterpret_cast<const unsigned char*>(a.x);
+        const unsigned char* rbase = reinterpret_cast<const unsigned char*>(a.r);
+        const unsigned char* wbase = reinterpret_cast<const unsigned char*>(a.w);
+        auto post = [&](long long block, int stage) {  // called by the slot's first thread only
+            const long long rw = block * blockDim.y + ty;
+            if (block >= n_blocks || rw >= a.n_tokens || a.drop_copies) return;
+            unsigned char* xs = dyn_smem + (size_t)stage * stage_bytes + (size_t)ty * 2 * row_bytes;
+            const size_t off = (size_t)rw * row_bytes;
+            mbarrier_expect_tx(&bars[stage][ty], 2 * (uint32_t)row_bytes);
+            tma_bulk_load(xs, xbase + off, (uint32_t)row_bytes, &bars[stage][ty]);
+            tma_bulk_load(xs + row_bytes, rbase + off, (uint32_t)row_bytes, &bars[stage][ty]);
+        };
+        if (tx == 0) {
+#pragma unroll
+            for (int st = 0; st < U; ++st) mbarrier_init(&bars[st][ty], 1);
+#pragma unroll
+            for (int st = 0; st < U; ++st) post((long long)blockIdx.x + st * stride, st);
+        }
+        row_sync(ty, tpr);  // the barriers are initialised before anyone polls them
+        int it = 0;
+        for (long long block = blockIdx.x; block < n_blocks; block += stride, ++it) {
+            const int stage = it % U;
+            const uint32_t parity = (uint32_t)(it / U) & 1u;
+            const long long rw = block * blockDim.y + ty;
+            const int nv = rw < a.n_tokens ? a.nvec : 0;
+            const unsigned char* xs = dyn_smem + (size_t)stage * stage_bytes + (size_t)ty * 2 * row_bytes;
+            const unsigned char* rs = xs + row_bytes;
+            unsigned char* yr = reinterpret_cast<unsigned char*>(a.y) + (size_t)(nv ? rw : 0) * row_bytes;
+            unsigned char* orw = reinterpret_cast<unsigned char*>(a.r_out) + (size_t)(nv ? rw : 0) * row_bytes;
+            if (nv > 0) {
+                bool landed = mbarrier_wait_bounded(&bars[stage][ty], parity, a.wait_polls);
+                if (!landed) {
+                    atomicExch(a.status, kDeviceTimeoutCode);
+                    landed = mbarrier_wait_bounded(&bars[stage][ty], parity, a.wait_polls);
+                }
+            }
+            float ssb = 0.f;
+            for (int v0 = tx; v0 < nv; v0 += IU * tpr) {
+#pragma unroll
+                for (int u = 0; u < IU; ++u) {
+                    const int v = v0 + u * tpr;
+                    if (v < nv) {
+                        float xf[EPV], rf[EPV], sum[EPV];
+                        C::unpack(ld_shared<VB>(xs + (size_t)v * VB), xf);
+                        C::unpack(ld_shared<VB>(rs + (size_t)v * VB), rf);
+                        float sv = 0.f;
+#pragma unroll
+                        for (int e = 0; e < EPV; ++e) {
+                            sum[e] = xf[e] + rf[e];
+                            sv = fmaf(sum[e], sum[e], sv);
+                        }
+                        ssb += sv;
+                        st_stream<VB>(orw + (size_t)v * VB, C::pack(sum));
+                    }
+                }
+            }
+            const float total = row_reduce<REDUCE>(ssb, tx, ty, tpr, 0u, 1u);
+            const float rho = __frsqrt_rn(total / (float)a.hidden + a.eps);
+            for (int v0 = tx; v0 < nv; v0 += IU * tpr) {
+                Vec<VB> wv[IU];
+#pragma unroll
+                for (int u = 0; u < IU; ++u) {
+                    const int v = v0 + u * tpr;
+                    if (v < nv) wv[u] = ld_weight<VB>(wbase + (size_t)v * VB);
+                }
+#pragma unroll
+                for (int u = 0; u < IU; ++u) {
+                    const int v = v0 + u * tpr;
+                    if (v < nv) {
+                        float xf[EPV], rf[EPV], wf[EPV], yf[EPV];
+                        C::unpack(ld_shared<VB>(xs + (size_t)v * VB), xf);
+                        C::unpack(ld_shared<VB>(rs + (size_t)v * VB), rf);
+                        C::unpack(wv[u], wf);
+#pragma unroll
+                        for (int e = 0; e < EPV; ++e) yf[e] = (xf[e] + rf[e]) * rho * wf[e];  // same binary32 sum as pass 1
+                        st_stream<VB>(yr + (size_t)v * VB, C::pack(yf));
+                    }
+                }
+            }
+            row_sync(ty, tpr);  // every thread of the slot has read the stage for the last time
+            if (tx == 0) post(block + (long long)U * stride, stage);
+        }
     }
+    trace.mark(kTraceStored);
+    trace.flush(a);
 }
 
 }  // namespace rt

@@ -58,9 +58,12 @@ std::vector<rt_params> raw_grid(const rt_shape& s)
     // silu_and_mul and merge_attn_states have no reduction and no ld.global -> shared stage: their grid is
     // the remaining axes
     const bool is_silu = s.op == RT_OP_SILU_AND_MUL || s.op == RT_OP_MERGE_ATTN_STATES;  // no reduction axis
-    for (int stage = 0; stage < 3; ++stage)
+    const int kStages[] = {RT_STAGE_REG, RT_STAGE_SMEM_LDG, RT_STAGE_SMEM_TMA, RT_STAGE_TMA_PIPELINE};
+    for (int stage : kStages)
         for (const Mode& m : kReduceModes)
             for (int vb : vecs) {
+                // the persistent pipeline: add_rmsnorm only, a row stays inside one CTA
+                if (stage == RT_STAGE_TMA_PIPELINE && (s.op != RT_OP_ADD_RMSNORM || m.cluster != 1)) continue;
                 if (is_silu && (stage == RT_STAGE_SMEM_LDG || m.reduce != RT_REDUCE_SHFL)) continue;
                 // the fp8-output norm: 32- or 16-byte vectors, shuffle reduction, register or TMA stage
                 if (s.op == RT_OP_ADD_RMSNORM_FP8 && (stage == RT_STAGE_SMEM_LDG || m.reduce != RT_REDUCE_SHFL || vb < 16))
@@ -82,16 +85,18 @@ std::vector<rt_params> raw_grid(const rt_shape& s)
                             out.push_back(p);
                         }
             }
-    // Rows whose byte length is not a multiple of 16 also get the ragged-row register stage, which keeps 16-byte
-    // accesses on such rows; on aligned rows it would only repeat the register stage with extra bookkeeping.
-    if (s.op == RT_OP_ADD_RMSNORM && (s.hidden * elem_bytes_of(s.dtype)) % 16 != 0)
+    // Rows whose byte length is not a multiple of 32 (or of 16) also get the ragged-row register stage with 32-byte
+    // (and 16-byte) chunks, which keeps wide accesses on such rows; on rows that the chunk width divides it would only
+    // repeat the register stage with extra bookkeeping.
+    for (int chunk : {32, 16})
+        if (s.op == RT_OP_ADD_RMSNORM && (s.hidden * elem_bytes_of(s.dtype)) % chunk != 0)
         for (int tpr : kTprLevels)
             for (int rpc : kRpcLevels)
                 for (int u : kUnrollLevels) {
                     rt_params p;
                     p.threads_per_row = tpr;
                     p.rows_per_cta = rpc;
-                    p.vec_bytes = 16;
+                    p.vec_bytes = chunk;
                     p.unroll = u;
                     p.stage = RT_STAGE_REG_REALIGN;
                     p.reduce = RT_REDUCE_SHFL;
@@ -107,9 +112,14 @@ static int heuristic_reject(const rt_shape& s, const rt_limits& L, const rt_para
     // a row narrower than one warp keeps the smallest row width: something must remain feasible
     if ((mask & RT_PRUNE_IDLE_THREADS) && p.threads_per_row > std::max(plan.slice_nvec, L.warp_size))
         return RT_PRUNE_IDLE_THREADS;
+    if ((mask & RT_PRUNE_PIPELINE_STAGE) && p.stage == RT_STAGE_TMA_PIPELINE) return RT_PRUNE_PIPELINE_STAGE;
     if (mask & RT_PRUNE_DUPLICATES) {
-        // A batch deeper than the vectors a thread owns only adds predicated-off slots.
-        if (p.unroll > next_pow2(plan.vec_per_thread)) return RT_PRUNE_DUPLICATES;
+        if (p.stage == RT_STAGE_TMA_PIPELINE) {
+            // a ring deeper than the row blocks a CTA walks over never fills
+            if (p.unroll > next_pow2(plan.blocks_per_cta)) return RT_PRUNE_DUPLICATES;
+        } else if (p.unroll > next_pow2(plan.vec_per_thread)) {
+            return RT_PRUNE_DUPLICATES;  // a batch deeper than the vectors a thread owns only adds predicated-off slots
+        }
     }
     if ((mask & RT_PRUNE_CLUSTER_WAVES) && p.cluster_size > 1) {
         // Splitting rows is for shapes with too few rows to occupy the SMs: allow a split into C only

@@ -5,7 +5,8 @@
 //
 // Instance lists.  Register stage: CAP (row vectors kept per thread) in {1,2,4,8,16,32} while the row
 // stays within 128 fp32 registers per thread, unroll U in {1,2,4} with U <= CAP.  Shared-memory
-// stages: U in {1,2,4}, all three reductions.  Narrow fall-back (4- and 2-byte vectors, for rows whose
+// stages: U in {1,2,4}, all three reductions; the persistent pipeline stage (same units): ring depth U in
+// {1,2,4}, shuffle and shared-memory reductions.  Narrow fall-back (4- and 2-byte vectors, for rows whose
 // byte length is not a multiple of 8): register stage, shuffle reduction, U in {1,4}.
 // Ragged-row register stage (16-byte chunks, shuffle reduction): the register stage's (CAP, U) list.
 // silu_and_mul (one unit per element type, every vector width): stages register and TMA bulk for 32-, 16- and
@@ -115,13 +116,18 @@ rt::KernelEntry merge_entry()
     entry<ST, 0, 1, 1>(), entry<ST, 0, 2, 1>(), entry<ST, 0, 4, 1>(), entry<ST, 1, 1, 1>(), entry<ST, 1, 2, 1>(), \
     entry<ST, 1, 4, 1>(), entry<ST, 2, 1, 1>(), entry<ST, 2, 2, 1>(), entry<ST, 2, 4, 1>()
 
+// the persistent pipeline: U is the ring depth; shuffle and shared-memory reductions
+#define RT_PIPELINE_LIST                                                                                      \
+    entry<4, 0, 1, 1>(), entry<4, 0, 2, 1>(), entry<4, 0, 4, 1>(), entry<4, 1, 1, 1>(), entry<4, 1, 2, 1>(), \
+    entry<4, 1, 4, 1>()
+
 std::vector<rt::KernelEntry> build_entries()
 {
     std::vector<rt::KernelEntry> all = {
 #if RT_UNIT_GROUP == 0
         RT_REG_LIST(RT_UNIT_REDUCE)
 #elif RT_UNIT_GROUP == 1
-        RT_SMEM_LIST(1), RT_SMEM_LIST(2)
+        RT_SMEM_LIST(1), RT_SMEM_LIST(2), RT_PIPELINE_LIST
 #elif RT_UNIT_GROUP == 3
         RT_SILU_WIDE(32), RT_SILU_WIDE(16), RT_SILU_WIDE(8), silu_entry<4, 0, 1>(), silu_entry<4, 0, 4>(), silu_entry<2, 0, 1>(),
         silu_entry<2, 0, 4>()

@@ -43,6 +43,7 @@ struct DeviceCache {
     std::vector<KernelInfo> info;       // per instance
     std::vector<char> info_ready;
     std::vector<size_t> dyn_smem_set;   // largest dynamic shared memory opted in so far
+    std::unordered_map<uint64_t, int> occupancy;  // (instance, threads, dynamic shared memory) -> resident CTAs per SM
 };
 DeviceCache g_dev[kMaxDevices];
 
@@ -318,15 +319,23 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
         plan->reject_reason = kRejectArgs;
         return RT_ERR_INFEASIBLE;
     }
-    if (p->stage < 0 || p->stage > RT_STAGE_REG_REALIGN || p->reduce < 0 || p->reduce > 2) {
+    if (p->stage < 0 || p->stage > RT_STAGE_TMA_PIPELINE || p->reduce < 0 || p->reduce > 2) {
         set_error("stage=%d or reduce=%d unknown", p->stage, p->reduce);
         plan->reject_reason = kRejectArgs;
         return RT_ERR_INFEASIBLE;
     }
     const bool realign = p->stage == RT_STAGE_REG_REALIGN;
-    if (realign && (s->op != RT_OP_ADD_RMSNORM || p->vec_bytes != 16 || p->reduce != RT_REDUCE_SHFL || p->cluster_size != 1)) {
-        set_error("the ragged-row stage belongs to add_rmsnorm and takes 16-byte chunks and the shuffle reduction "
+    if (realign && (s->op != RT_OP_ADD_RMSNORM || (p->vec_bytes != 16 && p->vec_bytes != 32) || p->reduce != RT_REDUCE_SHFL ||
+                    p->cluster_size != 1)) {
+        set_error("the ragged-row stage belongs to add_rmsnorm and takes 16- or 32-byte chunks and the shuffle reduction "
                   "(op=%d vec=%d reduce=%d cluster=%d)", s->op, p->vec_bytes, p->reduce, p->cluster_size);
+        plan->reject_reason = kRejectArgs;
+        return RT_ERR_INFEASIBLE;
+    }
+    const bool pipeline = p->stage == RT_STAGE_TMA_PIPELINE;
+    if (pipeline && (s->op != RT_OP_ADD_RMSNORM || p->reduce == RT_REDUCE_CLUSTER || p->cluster_size != 1)) {
+        set_error("the pipeline stage belongs to add_rmsnorm and keeps a row inside one CTA (op=%d reduce=%d cluster=%d)",
+                  s->op, p->reduce, p->cluster_size);
         plan->reject_reason = kRejectArgs;
         return RT_ERR_INFEASIBLE;
     }
@@ -389,7 +398,7 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
         return RT_ERR_ALIGN;
     }
     // silu_and_mul: an input row is 2 * row_bytes long, so 16-byte output rows give 16-byte input rows
-    if (p->stage == RT_STAGE_SMEM_TMA && (row_bytes % 16 != 0 || s->min_ptr_align < 16)) {
+    if ((p->stage == RT_STAGE_SMEM_TMA || pipeline) && (row_bytes % 16 != 0 || s->min_ptr_align < 16)) {
         set_error("TMA bulk copies need 16-byte aligned rows and pointers (row %lld bytes, pointers %d)",
                   (long long)row_bytes, s->min_ptr_align);
         plan->reject_reason = kRejectAlign;
@@ -397,8 +406,8 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
     }
 
     plan->elem_bytes = eb;
-    // ragged rows: the most whole 16-byte chunks a row can hold (its head and tail elements go one to a thread)
-    plan->nvec = realign ? (int)std::max<int64_t>(1, row_bytes / 16) : (int)(row_bytes / vb);
+    // ragged rows: the most whole chunks a row can hold (its head and tail elements go one to a thread)
+    plan->nvec = realign ? (int)std::max<int64_t>(1, row_bytes / vb) : (int)(row_bytes / vb);
     int slice = (plan->nvec + C - 1) / C;
     const int gran = vb < 16 ? 16 / vb : 1;  // slices start on 16-byte boundaries
     slice = (slice + gran - 1) / gran * gran;
@@ -442,6 +451,8 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
         plan->dyn_smem = (size_t)rpc * slice * (vb / eb) * 4;
     else if (p->stage == RT_STAGE_SMEM_TMA)
         plan->dyn_smem = (size_t)rpc * 2 * slice * vb;
+    else if (pipeline)
+        plan->dyn_smem = (size_t)p->unroll * rpc * 2 * slice * vb;  // a ring of `unroll` stages per row slot
 
     int regs, static_smem, local_bytes = 0, max_threads = L->max_threads_per_block;
     if (L->have_device) {
@@ -484,6 +495,18 @@ int make_plan(const rt_shape* s, const rt_params* p, const rt_limits* L, Plan* p
         return RT_ERR_INFEASIBLE;
     }
     plan->grid_x = (unsigned)(row_blocks * C);
+    if (pipeline) {
+        // persistent: as many CTAs as stay resident on the device, each walking over row blocks
+        const int resident = plan_occupancy(*plan, L, nullptr);
+        if (resident < 1) {
+            set_error("the pipeline's %zu bytes of shared memory leave no CTA resident", plan->dyn_smem);
+            plan->reject_reason = kRejectSmem;
+            return RT_ERR_INFEASIBLE;
+        }
+        const int64_t most = (int64_t)resident * L->sm_count;
+        plan->grid_x = (unsigned)std::max<int64_t>(1, std::min<int64_t>(row_blocks, most));
+        plan->blocks_per_cta = (int)((row_blocks + plan->grid_x - 1) / plan->grid_x);
+    }
     return RT_OK;
 }
 
@@ -500,9 +523,25 @@ int plan_occupancy(const Plan& plan, const rt_limits* L, int* regs_per_thread)
             return 0;
         }
         int blocks = 0;
+        const uint64_t occ_key = ((uint64_t)plan.kernel_index << 40) | ((uint64_t)threads << 24) | (uint64_t)(plan.dyn_smem >> 4);
+        DeviceCache* dc = nullptr;
+        bool cached = false;
+        if (plan.cluster == 1 && current_device_cache(&dc) == RT_OK) {
+            std::lock_guard<std::mutex> lock(g_mutex);
+            auto it = dc->occupancy.find(occ_key);
+            if (it != dc->occupancy.end()) {
+                blocks = it->second;
+                cached = true;
+            }
+        }
+        if (cached) return blocks;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks, k.fn, threads, plan.dyn_smem) != cudaSuccess) {
             (void)cudaGetLastError();
             return 0;
+        }
+        if (plan.cluster == 1 && dc) {
+            std::lock_guard<std::mutex> lock(g_mutex);
+            dc->occupancy[occ_key] = blocks;
         }
         if (plan.cluster > 1 && blocks > 0) {
             cudaLaunchConfig_t cfg;
@@ -722,15 +761,30 @@ int launch_silu_plan(const Plan& plan, const void* x, void* out, int64_t n_token
 int launch_plan(const Plan& plan, const void* x, const void* r, const void* w, void* y, void* r_out,
                 int64_t n_tokens, int64_t hidden, float eps, cudaStream_t stream)
 {
+    return launch_plan_as(plan, nullptr, nullptr, x, r, w, y, r_out, n_tokens, hidden, eps, stream);
+}
+
+// The plan's launch with another compiled function of the same template coordinates in place of the registry's
+// (`fn` != NULL: an instrumented instance, which also receives `trace`).
+int launch_plan_as(const Plan& plan, const void* fn, unsigned long long* trace, const void* x, const void* r, const void* w,
+                   void* y, void* r_out, int64_t n_tokens, int64_t hidden, float eps, cudaStream_t stream)
+{
     if (n_tokens == 0) return RT_OK;
     if (plan.op != RT_OP_ADD_RMSNORM) {
         set_error("plan belongs to another kernel");
         return RT_ERR_INFEASIBLE;
     }
     const KernelEntry& k = registry()[plan.kernel_index];
-    int st = ensure_dynamic_smem(plan.kernel_index, plan.dyn_smem);
+    int st = RT_OK;
+    if (!fn) {
+        st = ensure_dynamic_smem(plan.kernel_index, plan.dyn_smem);
+    } else if (plan.dyn_smem > 48 * 1024) {
+        set_error("instrumented instances take at most 48 KB of dynamic shared memory");
+        st = RT_ERR_INFEASIBLE;
+    }
     if (st != RT_OK) return st;
     KernelArgs a;
+    a.trace = trace;
     a.x = x; a.r = r; a.w = w; a.y = y; a.r_out = r_out;
     a.n_tokens = n_tokens;
     a.hidden = (int)hidden;
@@ -751,7 +805,7 @@ int launch_plan(const Plan& plan, const void* x, const void* r, const void* w, v
     LaunchAttrs la;
     set_launch_attrs(&cfg, &la, plan.cluster);
     void* params[] = {&a};
-    cudaError_t e = cudaLaunchKernelExC(&cfg, k.fn, params);
+    cudaError_t e = cudaLaunchKernelExC(&cfg, fn ? fn : k.fn, params);
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
         set_error("kernel launch failed: %s", cudaGetErrorString(e));

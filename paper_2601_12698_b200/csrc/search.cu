@@ -869,12 +869,17 @@ struct SearchState {
             auto it = index.find(pack_params(q));
             if (it != index.end() && it->second != idx) out.push_back(it->second);
         };
+        // A step along the block-shape or vector axis can land where the current unroll depth is pruned as a
+        // duplicate (more threads per row or wider vectors leave a thread fewer vectors than the batch is deep):
+        // the neighbour is then that point with the deepest unroll that exists there.
         auto step = [&](const int* levels, int n, int rt_params::*field) {
             const int l = level_of(levels, n, p.*field);
             for (int d = -1; d <= 1; d += 2) {
                 if (l + d < 0 || l + d >= n || l < 0) continue;
                 rt_params q = p;
                 q.*field = levels[l + d];
+                if (field != &rt_params::unroll)
+                    while (q.unroll > 1 && index.find(pack_params(q)) == index.end()) q.unroll /= 2;
                 probe(q);
             }
         };
@@ -884,7 +889,7 @@ struct SearchState {
         step(kVec, 5, &rt_params::vec_bytes);
         // another stage at the same vector width; where that stage has no such point (the ragged-row stage is
         // all 16-byte chunks while the other stages of a misaligned shape are narrower), at its widest width
-        for (int stage = 0; stage <= RT_STAGE_REG_REALIGN; ++stage) {
+        for (int stage = 0; stage <= RT_STAGE_TMA_PIPELINE; ++stage) {
             rt_params q = p;
             q.stage = stage;
             if (index.find(pack_params(q)) == index.end()) {
@@ -998,7 +1003,7 @@ int run_search(const rt_shape& shape, const rt_limits& limits, const rt_budget& 
             S.time_us[idx] = t;
         }
         // 2. coarse grid, cut to half of what is left of the budget (mode by mode, nearest the middle first)
-        int widest[RT_STAGE_REG_REALIGN + 1] = {0, 0, 0, 0};  // per stage: the ragged-row stage is wider than the others
+        int widest[RT_STAGE_TMA_PIPELINE + 1] = {0, 0, 0, 0, 0};  // per stage: the ragged-row stage is wider than the others
         for (const rt_params& p : feasible) widest[p.stage] = std::max(widest[p.stage], p.vec_bytes);
         std::vector<int> coarse;
         for (int i = 0; i < (int)feasible.size(); ++i) {

@@ -30,9 +30,11 @@ int table_lookup(const rt_spec_entry* table, int32_t n, const rt_params* general
     for (int32_t i = 0; i < n; ++i) {
         const rt_spec_entry& e = table[i];
         if (e.shape.dtype != query->dtype || e.shape.op != query->op) continue;
-        // the ragged-row stage runs on any row length, but on 16-byte rows it is the register stage plus
-        // bookkeeping: an entry tuned on a misaligned shape is not a neighbour of an aligned one
-        if (e.best.stage == RT_STAGE_REG_REALIGN && (query->hidden * elem_bytes_of(query->dtype)) % 16 == 0) continue;
+        // the ragged-row stage runs on any row length, but on rows that its chunk width divides it is the register
+        // stage plus bookkeeping: an entry tuned on a misaligned shape is not a neighbour of an aligned one
+        if (e.best.stage == RT_STAGE_REG_REALIGN && e.best.vec_bytes > 0 &&
+            (query->hidden * elem_bytes_of(query->dtype)) % e.best.vec_bytes == 0)
+            continue;
         const double d = shape_distance(e.shape, *query);
         if (best >= 0 && d >= best_d) continue;
         Plan plan;

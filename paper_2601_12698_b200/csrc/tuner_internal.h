@@ -44,6 +44,7 @@ struct Plan {
     int vec_per_head; // merge_attn_states: vectors in one head
     int heads;
     int cluster;      // CTAs per row
+    int blocks_per_cta;  // pipeline stage: row blocks the busiest CTA of the persistent grid walks over (else 0)
     int block_x, block_y;
     unsigned grid_x;
     size_t dyn_smem;
@@ -73,6 +74,8 @@ int current_limits(rt_limits* out);
 
 int launch_plan(const Plan& plan, const void* x, const void* r, const void* w, void* y, void* r_out,
                 int64_t n_tokens, int64_t hidden, float eps, cudaStream_t stream);
+int launch_plan_as(const Plan& plan, const void* fn, unsigned long long* trace, const void* x, const void* r, const void* w,
+                   void* y, void* r_out, int64_t n_tokens, int64_t hidden, float eps, cudaStream_t stream);
 int launch_fp8_plan(const Plan& plan, const void* x, const void* r, const void* w, void* q, float* scale, void* r_out,
                     int64_t n_tokens, int64_t hidden, float eps, cudaStream_t stream);
 int launch_allreduce_plan(const Plan& plan, const void* const* x_parts, int n_parts, const void* r, const void* w,

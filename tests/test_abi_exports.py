@@ -27,10 +27,13 @@ def test_library_exports_every_declared_symbol():
 def test_binding_covers_the_header():
     from paper_2601_12698_b200 import binding
     assert sorted(binding.EXPORTED) == sorted(_declared_functions())
-    assert binding.lib.rt_num_kernel_instances() == 940  # 593 norm (39 of them the ragged-row stage, 144 with 32-byte vectors) + 64 silu_and_mul + 64 merge_attn_states + 54 fp8-output + 165 all-reduce-fused
+    # 677 norm (69 of them the ragged-row stage, 54 the persistent pipeline) + 64 silu_and_mul + 64 merge_attn_states
+    # + 54 fp8-output + 165 all-reduce-fused
+    assert binding.lib.rt_num_kernel_instances() == 1024
     assert binding.lib.rt_status_string(binding.RT_ERR_INFEASIBLE).decode().startswith("configuration outside")
     inst = binding.kernel_instances()
-    assert {i["dtype"] for i in inst} == {0, 1, 2} and {i["stage"] for i in inst} == {0, 1, 2, 3}
+    assert {i["dtype"] for i in inst} == {0, 1, 2} and {i["stage"] for i in inst} == {0, 1, 2, 3, 4}
+    assert sum(1 for i in inst if i["stage"] == 4) == 54 and {i["op"] for i in inst if i["stage"] == 4} == {0}
     assert sum(1 for i in inst if i["op"] == 2) == 64 and sum(1 for i in inst if i["op"] == 3) == 54
     assert sum(1 for i in inst if i["op"] == 1) == 64 and {i["stage"] for i in inst if i["op"] == 1} == {0, 2}
     fused = [i for i in inst if i["op"] == 4]
@@ -44,16 +47,16 @@ def test_struct_layouts_match_the_header_sizes():
     import subprocess
     import tempfile
     from paper_2601_12698_b200 import binding as B
-    src = ('#include <stdio.h>\n#include "rmsnorm_tuner.h"\nint main(void){printf("%zu %zu %zu %zu %zu %zu %zu\\n",'
+    src = ('#include <stdio.h>\n#include "rmsnorm_tuner.h"\nint main(void){printf("%zu %zu %zu %zu %zu %zu %zu %zu\\n",'
            "sizeof(rt_params),sizeof(rt_shape),sizeof(rt_limits),sizeof(rt_budget),sizeof(rt_workspace),"
-           "sizeof(rt_eval_record),sizeof(rt_result));return 0;}\n")
+           "sizeof(rt_eval_record),sizeof(rt_result),sizeof(rt_block_record));return 0;}\n")
     with tempfile.TemporaryDirectory() as d:
         c = os.path.join(d, "s.c")
         open(c, "w").write(src)
         exe = os.path.join(d, "s")
         subprocess.run(["gcc", "-std=c99", "-I", os.path.join(ROOT, "include"), c, "-o", exe], check=True)
         sizes = [int(v) for v in subprocess.run([exe], capture_output=True, text=True, check=True).stdout.split()]
-    mirrors = [B.rt_params, B.rt_shape, B.rt_limits, B.rt_budget, B.rt_workspace, B.rt_eval_record, B.rt_result]
+    mirrors = [B.rt_params, B.rt_shape, B.rt_limits, B.rt_budget, B.rt_workspace, B.rt_eval_record, B.rt_result, B.rt_block_record]
     assert sizes == [ctypes.sizeof(m) for m in mirrors]
 
 

@@ -124,3 +124,24 @@ def test_traffic_figures_are_tied_to_the_kernel_they_were_captured_on():
     for name, table in bench.NCU_TRAFFIC.items():
         alg = synth.workloads()[name].algorithmic_bytes
         assert all(0.85 * alg < v[0] < 1.05 * alg for v in table.values())
+
+
+def test_phase_analysis_of_synthetic_stamps():
+    """trace.analyse on stamps built by hand: 1.5 GHz, phases of 300 / 900 / 450 / 150 cycles, a launch every 2000 ns."""
+    import torch
+    from paper_2601_12698_b200 import trace
+    launches, ctas = 40, 3
+    t = torch.zeros((launches, ctas, 8), dtype=torch.int64)
+    for k in range(launches):
+        for c in range(ctas):
+            ns0 = 1_000_000 + 2000 * k + 10 * c
+            cyc0 = 5_000_000 + int(1.5 * (ns0 - 1_000_000)) + 7 * c
+            marks = [cyc0, cyc0 + 300, cyc0 + 1200, cyc0 + 1650 + 30 * c, cyc0 + 1800 + 30 * c]
+            t[k, c] = torch.tensor([ns0, *marks, ns0 + 1300, 5])
+    info = trace.analyse(t, launches, ctas, skip=4)
+    assert abs(info["sm_ghz_from_stamps"] - 1.5) < 0.01
+    assert [round(ph["cycles_median_cta"]) for ph in info["phases"]] == [300, 900, 480, 150]
+    assert [round(ph["cycles_slowest_cta"]) for ph in info["phases"]] == [300, 900, 510, 150]
+    assert info["launch_period_ns"] == 2000 and abs(info["released_to_stored_ns_slowest_cta"] - 1560 / 1.5) < 8
+    assert abs(info["outside_the_kernel_ns"] - (2000 - 1560 / 1.5)) < 8
+    assert info["next_launch_resident_before_exit_ns"] == (1300 + 20) - 2000

@@ -26,8 +26,8 @@ def test_every_emitted_theta_passes_the_hard_rules_and_counts_add_up(L, T, H, dt
     for th in feasible:
         assert B.tuner_check_params(s, th, L) == B.RT_OK
         assert th.threads_per_row * th.rows_per_cta <= 1024
-        if th.stage == B.RT_STAGE_REG_REALIGN:  # aligned 16-byte chunks over rows of any length
-            assert th.vec_bytes == 16 and th.reduce == B.RT_REDUCE_SHFL and (H * (4 if dtype == "fp32" else 2)) % 16 != 0
+        if th.stage == B.RT_STAGE_REG_REALIGN:  # aligned 16- or 32-byte chunks over rows that the chunk does not divide
+            assert th.vec_bytes in (16, 32) and th.reduce == B.RT_REDUCE_SHFL and (H * (4 if dtype == "fp32" else 2)) % th.vec_bytes != 0
         else:
             assert (H * (4 if dtype == "fp32" else 2)) % th.vec_bytes == 0
         assert (th.reduce == B.RT_REDUCE_CLUSTER) == (th.cluster_size > 1)
@@ -55,7 +55,7 @@ def test_rules_bite_where_they_should(L):
     # 6148 fp16: row bytes = 8 mod 16 -> only 8-byte row vectors, no TMA stage; the ragged-row stage keeps 16-byte chunks
     f = B.tuner_derive_feasible(B.shape_of(8192, 6148, "fp16"), L)
     assert {t.vec_bytes for t in row_vectors(f)} == {8} and {t.stage for t in f} == {0, 1, ragged}
-    assert {t.vec_bytes for t in f if t.stage == ragged} == {16}
+    assert {t.vec_bytes for t in f if t.stage == ragged} == {16, 32}
     # rows of 8192 bf16 elements: all three widths of the vector axis, for every kernel
     f = B.tuner_derive_feasible(B.shape_of(16384, 8192, "bf16"), L)
     assert {t.vec_bytes for t in f} == {8, 16, 32} and {t.stage for t in f if t.vec_bytes == 32} == {0, 1, 2}
@@ -64,9 +64,11 @@ def test_rules_bite_where_they_should(L):
     assert B.tuner_check_params(B.shape_of(64, 8192, "bf16", op=B.RT_OP_ADD_RMSNORM_FP8), B.make_params(vec_bytes=32), L) == B.RT_OK
     assert B.tuner_check_params(B.shape_of(64, 8192, "bf16", op=B.RT_OP_ADD_RMSNORM_ALLREDUCE, n_parts=2),
                                 B.make_params(vec_bytes=32), L) == B.RT_OK
-    # 6152 fp16: 769 16-byte vectors (no 32-byte ones), both widths, the three aligned stages and no ragged-row stage
+    # 6152 fp16: 769 16-byte vectors (no 32-byte row vectors): both widths in the three aligned stages, and the
+    # ragged-row stage with the 32-byte chunks that the row length does not divide into
     f = B.tuner_derive_feasible(B.shape_of(8192, 6152, "fp16"), L)
-    assert {t.vec_bytes for t in f} == {8, 16} and {t.stage for t in f} == {0, 1, 2}
+    assert {t.vec_bytes for t in row_vectors(f)} == {8, 16} and {t.stage for t in f} == {0, 1, 2, ragged}
+    assert {t.vec_bytes for t in f if t.stage == ragged} == {32}
     # rows that fit no 8-byte vector fall back to the widest narrow width, or take the ragged-row stage
     for hidden, narrow in ((6146, 4), (6145, 2)):
         f = B.tuner_derive_feasible(B.shape_of(64, hidden, "fp16"), L)
@@ -84,7 +86,7 @@ def test_rules_bite_where_they_should(L):
     assert B.tuner_check_params(s_odd, B.make_params(stage=ragged, vec_bytes=8), L) == B.RT_ERR_INFEASIBLE
     assert B.tuner_check_params(s_odd, B.make_params(stage=ragged, reduce=B.RT_REDUCE_SMEM), L) == B.RT_ERR_INFEASIBLE
     assert B.tuner_check_params(s_odd, B.make_params(stage=ragged, reduce=B.RT_REDUCE_CLUSTER, cluster_size=2), L) == B.RT_ERR_INFEASIBLE
-    assert B.tuner_check_params(s_odd, B.make_params(stage=4), L) == B.RT_ERR_INFEASIBLE
+    assert B.tuner_check_params(s_odd, B.make_params(stage=5), L) == B.RT_ERR_INFEASIBLE
     assert B.tuner_check_params(B.shape_of(64, 6145, "fp16", min_ptr_align=8), B.make_params(stage=ragged), L) == B.RT_ERR_ALIGN
     assert B.tuner_check_params(B.shape_of(128, 4096, "bf16"), B.make_params(stage=ragged), L) == B.RT_OK
     assert B.tuner_check_params(B.shape_of(64, 6145, "fp16", op=B.RT_OP_SILU_AND_MUL), B.make_params(stage=ragged), L) == B.RT_ERR_INFEASIBLE
@@ -202,3 +204,33 @@ def test_allreduce_fused_norm_grid(L):
     assert B.tuner_derive_feasible(B.shape_of(64, 6148, "fp16", op=B.RT_OP_ADD_RMSNORM_ALLREDUCE, n_parts=2), L) == []
     # fp32 rows work too
     assert B.tuner_derive_feasible(B.shape_of(64, 4096, "fp32", op=B.RT_OP_ADD_RMSNORM_ALLREDUCE, n_parts=2), L)
+
+
+def test_the_pipeline_stage_is_derived_only_on_request(L):
+    """RT_STAGE_TMA_PIPELINE is part of the raw grid and passes the hard rules, but the default mask leaves it out of
+    the feasible set (it has won on no shape measured); clearing RT_PRUNE_PIPELINE_STAGE brings it in."""
+    pipe = B.RT_STAGE_TMA_PIPELINE
+    s = B.shape_of(16384, 8192, "bf16")
+    assert pipe in {t.stage for t in B.tuner_raw_grid(s)}
+    assert pipe not in {t.stage for t in B.tuner_derive_feasible(s, L)}
+    with_pipe = B.tuner_derive_feasible(s, L, heuristics=B.RT_PRUNE_DEFAULT & ~B.RT_PRUNE_PIPELINE_STAGE)
+    mine = [t for t in with_pipe if t.stage == pipe]
+    assert mine and {t.unroll for t in mine} == {1, 2, 4} and {t.reduce for t in mine} == {0, 1}
+    assert {t.cluster_size for t in mine} == {1} and {t.vec_bytes for t in mine} == {8, 16, 32}
+    assert _keys([t for t in with_pipe if t.stage != pipe]) == _keys(B.tuner_derive_feasible(s, L))
+    c_default, c_with = B.tuner_derive_counts(s, L), B.tuner_derive_counts(s, L, B.RT_PRUNE_DEFAULT & ~B.RT_PRUNE_PIPELINE_STAGE)
+    assert c_with["feasible"] - c_default["feasible"] == len(mine) == c_default["heuristics"] - c_with["heuristics"]
+    # hard rules: one CTA per row, add_rmsnorm only, 16-byte rows and pointers, the ring must fit in shared memory
+    ok = B.make_params(stage=pipe, unroll=2)
+    assert B.tuner_check_params(s, ok, L) == B.RT_OK
+    assert B.tuner_check_params(s, B.make_params(stage=pipe, reduce=B.RT_REDUCE_CLUSTER, cluster_size=2), L) == B.RT_ERR_INFEASIBLE
+    assert B.tuner_check_params(B.shape_of(64, 8192, "bf16", op=B.RT_OP_SILU_AND_MUL), ok, L) == B.RT_ERR_INFEASIBLE
+    assert B.tuner_check_params(B.shape_of(64, 6148, "fp16"), B.make_params(stage=pipe, vec_bytes=8), L) == B.RT_ERR_ALIGN
+    assert B.tuner_check_params(B.shape_of(64, 8192, "bf16", min_ptr_align=8), B.make_params(stage=pipe, vec_bytes=8), L) == B.RT_ERR_ALIGN
+    s5 = B.shape_of(32768, 12288, "fp32")            # 96 KB per row and stage
+    assert B.tuner_check_params(s5, B.make_params(stage=pipe, unroll=2), L) == B.RT_OK
+    assert B.tuner_check_params(s5, B.make_params(stage=pipe, unroll=4), L) == B.RT_ERR_INFEASIBLE
+    assert b"shared memory" in B.lib.rt_last_error()
+    # decode shapes: a CTA walks over one row block, so a deeper ring is the same kernel again (pruned as a duplicate)
+    few = B.tuner_derive_feasible(B.shape_of(16, 4096, "bf16"), L, heuristics=B.RT_PRUNE_DEFAULT & ~B.RT_PRUNE_PIPELINE_STAGE)
+    assert {t.unroll for t in few if t.stage == pipe} == {1}

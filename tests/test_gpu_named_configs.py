@@ -97,7 +97,7 @@ def test_closed_form_rows_through_every_stage(B, oracle_lib, dtype, H):
     thetas = B.tuner_derive_feasible(B.shape_of(T, H, dtype), heuristics=0)   # hard rules only: the widest net
     per_thread = max(H // t.threads_per_row // max(1, t.cluster_size) for t in thetas)
     assert per_thread >= (384 if H == 12288 else 128)
-    assert {t.stage for t in thetas} == {0, 1, 2}
+    assert {t.stage for t in thetas} == {0, 1, 2, 4}
     n, failures, worst = _run_all(B, oracle_lib, x, r, w, dtype, thetas)
     print(f"closed-form rows {dtype} H={H}: {n} thetas, up to {per_thread} elements per thread, worst y error {worst:.3g}")
     assert not failures, f"{len(failures)} of {n} configurations differ: {failures[:5]}"

@@ -81,7 +81,7 @@ def test_every_feasible_theta_matches_oracle(B, oracle_lib, dtype, T, H):
 
 
 RAGGED_SHAPES = [(1, 1), (9, 1), (5, 3), (9, 7), (4, 9), (7, 33), (5, 1001), (3, 4097), (5, 6145), (4, 6146), (3, 6148),
-                 (2, 12289), (5, 4096)]
+                 (5, 6152), (2, 12289), (5, 4096), (6, 17), (33, 31)]
 
 
 @pytest.mark.parametrize("dtype", ["bf16", "fp16", "fp32"])
@@ -98,13 +98,14 @@ def test_ragged_row_stage_matches_oracle(B, oracle_lib, dtype, T, H):
     y, _, y_ok = _padded((T, H), TD[dtype])
     ro, _, ro_ok = _padded((T, H), TD[dtype])
     shape = B.shape_of(T, H, dtype, B._ptr_align(xd, rd, wd, y, ro))
-    thetas = [B.make_params(threads_per_row=tpr, rows_per_cta=rpc, unroll=u, stage=B.RT_STAGE_REG_REALIGN)
-              for tpr in (32, 64, 128, 256, 512, 1024) for rpc in (1, 2, 4, 8) for u in (1, 2, 4)]
+    thetas = [B.make_params(threads_per_row=tpr, rows_per_cta=rpc, unroll=u, vec_bytes=vb, stage=B.RT_STAGE_REG_REALIGN)
+              for vb in (16, 32) for tpr in (32, 64, 128, 256, 512, 1024) for rpc in (1, 2, 4, 8) for u in (1, 2, 4)]
     thetas = [th for th in thetas if B.tuner_check_params(shape, th) == B.RT_OK]
-    assert thetas
-    if (H * (4 if dtype == "fp32" else 2)) % 16 != 0:  # the deriver offers the stage exactly on such rows
-        offered = {t.key() for t in B.tuner_derive_feasible(shape, heuristics=0) if t.stage == B.RT_STAGE_REG_REALIGN}
-        assert offered == {t.key() for t in thetas}
+    assert {th.vec_bytes for th in thetas} == {16, 32}
+    # the deriver offers a chunk width exactly on the rows that width does not divide
+    offered = {t.key() for t in B.tuner_derive_feasible(shape, heuristics=0) if t.stage == B.RT_STAGE_REG_REALIGN}
+    row_bytes = H * (4 if dtype == "fp32" else 2)
+    assert offered == {t.key() for t in thetas if row_bytes % t.vec_bytes != 0}
     failures = []
     for th in thetas:
         y.fill_(float("nan")); ro.fill_(float("nan"))

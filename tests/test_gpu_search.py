@@ -112,7 +112,8 @@ def test_full_size_configs_on_sampled_rows(B, oracle_lib, name):
     for stage in (0, 1, 2, 3):  # rows that are not 16-byte multiples: no TMA stage, but the ragged-row stage
         picks += [th for th in feasible if th.stage == stage][:1]
     row_bytes = wl.hidden * (4 if wl.dtype == "fp32" else 2)
-    want = {0, 1, 2} if row_bytes % 16 == 0 else ({0, 1, 3} if row_bytes % 8 == 0 else {0, 3})  # narrow vectors: registers only
+    # narrow vectors: registers only; the ragged-row stage wherever 32-byte chunks do not divide the row
+    want = {0, 1, 2} if row_bytes % 32 == 0 else {0, 1, 2, 3} if row_bytes % 16 == 0 else {0, 1, 3} if row_bytes % 8 == 0 else {0, 3}
     assert {th.stage for th in picks[1:]} == want
     rows = sorted({0, 1, 63, 64, wl.n_tokens // 2 + 1, wl.n_tokens - 65, wl.n_tokens - 2, wl.n_tokens - 1} |
                   {int(v) for v in torch.randint(0, wl.n_tokens, (24,), generator=torch.Generator().manual_seed(5))})

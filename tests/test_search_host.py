@@ -180,30 +180,31 @@ def test_an_optimum_two_steps_from_every_leader_is_reached_with_leftover_budget(
 
 RAGGED_OPTIMA = [dict(tpr=256, rpc=1, unroll=4, vec=16, stage=3, reduce=0),   # 16-byte chunks of the ragged-row stage
                  dict(tpr=1024, rpc=1, unroll=4, vec=2, stage=0, reduce=0),   # the 2-byte row vectors of the register stage
-                 dict(tpr=128, rpc=2, unroll=1, vec=16, stage=3, reduce=0)]
+                 dict(tpr=128, rpc=2, unroll=1, vec=32, stage=3, reduce=0)]   # 32-byte chunks
 
 
 @pytest.mark.parametrize("opt", RAGGED_OPTIMA)
 def test_guided_search_crosses_between_stages_of_different_vector_width(L, opt):
-    """Rows of 6145 fp16 elements: the row-vector stage has 2-byte vectors only, the ragged-row stage 16-byte chunks.
-    The coarse grid must hold points of both (each at its own widest width) and the climb must be able to step from
-    one to the other, whichever side the optimum is on."""
+    """Rows of 6145 fp16 elements: the row-vector stage has 2-byte vectors only, the ragged-row stage 16- and 32-byte
+    chunks.  The coarse grid must hold points of both stages (each at its own widest width) and the climb must be able
+    to step from one to the other, whichever side the optimum is on."""
     s = B.shape_of(8192, 6145, "fp16")
     feasible = B.tuner_derive_feasible(s, L)
-    assert {(t.stage, t.vec_bytes) for t in feasible} == {(0, 2), (3, 16)}
+    assert {(t.stage, t.vec_bytes) for t in feasible} == {(0, 2), (3, 16), (3, 32)}
     target = [t for t in feasible if (t.threads_per_row, t.rows_per_cta, t.unroll, t.vec_bytes, t.stage, t.reduce) ==
               (opt["tpr"], opt["rpc"], opt["unroll"], opt["vec"], opt["stage"], opt["reduce"])]
     assert target, "the planted optimum must be feasible"
 
-    def cost(p):  # the bowl of _cost_factory without its vector term: the width is tied to the stage here
+    def cost(p):  # the bowl of _cost_factory with a vector term inside the ragged-row stage only (elsewhere the width is tied to the stage)
         t = 100.0 + 12.0 * abs(math.log2(p.threads_per_row) - math.log2(opt["tpr"]))
         t += 7.0 * abs(math.log2(p.rows_per_cta) - math.log2(opt["rpc"])) + 5.0 * abs(math.log2(p.unroll) - math.log2(opt["unroll"]))
+        t += 3.0 if p.stage == 3 and opt["stage"] == 3 and p.vec_bytes != opt["vec"] else 0.0
         return t + (0.0 if p.stage == opt["stage"] else 15.0)
 
     res, log = B.tuner_search_with(s, L, B.make_budget(max_evals=24, top_k=2), cost)
     assert res.best.key() == target[0].key(), (res.best, res.best_us)
     grid = [r for r in log if r.phase == 1]  # RT_PHASE_GRID
-    assert {(r.params.stage, r.params.vec_bytes) for r in grid} == {(0, 2), (3, 16)}
+    assert {(r.params.stage, r.params.vec_bytes) for r in grid} == {(0, 2), (3, 32)}   # each stage at its widest width
     # a search that starts from a seed on one side still reaches the other
     seed = B.make_params(threads_per_row=1024, vec_bytes=2, unroll=1) if opt["stage"] == 3 else \
         B.make_params(threads_per_row=512, unroll=1, stage=B.RT_STAGE_REG_REALIGN)
