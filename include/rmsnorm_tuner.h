@@ -156,7 +156,11 @@ typedef struct {
     int32_t use_graph;       /* 1: the timed block is one CUDA graph of `iters` launches */
     const rt_params* seeds;  /* host; evaluated first when given (configs found on other shapes) */
     int32_t n_seeds;
-    int32_t reserved;
+    int32_t preheat_ms;      /* 0..5000: before its first timing, and again before the Top-K re-test (and at the start
+                                of tuner_retest_interleaved), the tuner keeps the device busy for this long with
+                                launches of a candidate that has passed its gate, so that candidates are compared at
+                                the clocks of a loaded device instead of at the boost clocks of one that was waiting
+                                for the host.  0 = no pre-heating */
 } rt_budget;
 
 /* For silu_and_mul: x is the [n_tokens, 2*d] input (ring stride 2 * ring_stride_bytes), y the output,

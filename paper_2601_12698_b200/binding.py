@@ -71,7 +71,7 @@ class rt_limits(Structure):
 class rt_budget(Structure):
     _fields_ = [("max_evals", c_int32), ("warmup", c_int32), ("iters", c_int32), ("repeats", c_int32),
                 ("top_k", c_int32), ("strategy", c_int32), ("heuristics", c_int32), ("use_graph", c_int32),
-                ("seeds", POINTER(rt_params)), ("n_seeds", c_int32), ("reserved", c_int32)]
+                ("seeds", POINTER(rt_params)), ("n_seeds", c_int32), ("preheat_ms", c_int32)]
 
 
 class rt_workspace(Structure):
@@ -396,8 +396,8 @@ def tuner_check_params(shape: rt_shape, params: rt_params, limits: rt_limits | N
 # ---- 3. search ------------------------------------------------------------------------------------------------
 
 def make_budget(max_evals=64, warmup=20, iters=100, repeats=3, top_k=5, strategy=RT_SEARCH_GUIDED,
-                heuristics=RT_PRUNE_DEFAULT, use_graph=False, seeds=None) -> rt_budget:
-    b = rt_budget(max_evals, warmup, iters, repeats, top_k, strategy, heuristics, int(use_graph), None, 0, 0)
+                heuristics=RT_PRUNE_DEFAULT, use_graph=False, seeds=None, preheat_ms=0) -> rt_budget:
+    b = rt_budget(max_evals, warmup, iters, repeats, top_k, strategy, heuristics, int(use_graph), None, 0, int(preheat_ms))
     if seeds:
         arr = (rt_params * len(seeds))(*seeds)
         b._seed_storage = arr  # keep alive

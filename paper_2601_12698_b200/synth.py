@@ -107,6 +107,11 @@ def workloads() -> dict[str, Workload]:
     add(Workload("c4x_fp16_8192x6146", "fp16", 8192, 6146, seed=3))
     add(Workload("c4x_fp16_8192x6145", "fp16", 8192, 6145, seed=3))
     add(Workload("c5_fp32_32768x12288", "fp32", 32768, 12288, seed=4))
+    # mid-size batches: a few thousand rows, i.e. a few waves of CTAs with a ragged last one - between the
+    # latency-bound and the bandwidth-bound configurations (where a persistent grid would have to pay, if anywhere)
+    add(Workload("mid_bf16_2048x8192", "bf16", 2048, 8192, seed=5, dist=_PREFILL_DIST))
+    add(Workload("mid_bf16_4096x4096", "bf16", 4096, 4096, seed=5, dist=_PREFILL_DIST))
+    add(Workload("mid_bf16_3000x5120", "bf16", 3000, 5120, seed=5, dist=_PREFILL_DIST))
     # silu_and_mul: a bandwidth case (LLaMA-3-8B MLP width), and the paper's fp32 (m, n) shapes with n = d
     gate = Dist(sigma=2.5)
     add(Workload("silu_bf16_16384x14336", "bf16", 16384, 14336, seed=6, dist=gate, op="silu_and_mul"))

@@ -26,6 +26,8 @@ from . import binding as B
 from . import synth
 
 
+PREHEAT_MS = 300
+
 OPS = {"norm": B.RT_OP_ADD_RMSNORM, "silu": B.RT_OP_SILU_AND_MUL, "merge": B.RT_OP_MERGE_ATTN_STATES,
        "fp8": B.RT_OP_ADD_RMSNORM_FP8, "allreduce": B.RT_OP_ADD_RMSNORM_ALLREDUCE}
 
@@ -126,7 +128,9 @@ def tune(shapes, budget: int = 64, top_k: int = 5, finalists: int = 3, seed: int
     per_shape, candidates = [], {}  # candidates: kernel -> {theta key: theta}
     for kernel, dtype, dims in shapes:
         p = ShapeProblem(kernel, dtype, dims, seed, eps, stream)
-        res, log = B.tuner_search(p.shape, B.make_budget(max_evals=budget, top_k=top_k, use_graph=p.use_graph), p.ws)
+        # bandwidth-bound shapes are searched on a loaded device (see rt_budget.preheat_ms)
+        res, log = B.tuner_search(p.shape, B.make_budget(max_evals=budget, top_k=top_k, use_graph=p.use_graph,
+                                                         preheat_ms=0 if p.use_graph else PREHEAT_MS), p.ws)
         ranked = sorted((rec for rec in log if rec.status == B.RT_OK), key=lambda rec: rec.us)
         seen = []
         for rec in ranked:
@@ -151,7 +155,8 @@ def tune(shapes, budget: int = 64, top_k: int = 5, finalists: int = 3, seed: int
         times = [[-1.0] * len(mine) for _ in cand]
         for xi, (k, dtype, dims) in enumerate(mine):
             p = ShapeProblem(k, dtype, dims, seed, eps, stream)
-            proto = B.make_budget(warmup=20, iters=100, repeats=3, use_graph=p.use_graph)
+            proto = B.make_budget(warmup=20, iters=100, repeats=3, use_graph=p.use_graph,
+                                  preheat_ms=0 if p.use_graph else PREHEAT_MS // 4)
             for ci, th in enumerate(cand):
                 if B.tuner_check_params(p.shape, th) != B.RT_OK:
                     continue
@@ -178,6 +183,19 @@ def tune(shapes, budget: int = 64, top_k: int = 5, finalists: int = 3, seed: int
     return table, report
 
 
+def merge_tables(old: "B.SpecTable", new: "B.SpecTable", keep_general: bool = False) -> "B.SpecTable":
+    """The entries of `old` with those of `new` laid over them (same kernel, dtype, shape, head size and part count:
+    the new entry wins), old entries first in their order; general configurations of `new` win unless keep_general."""
+    key = lambda s: (int(s.op), int(s.dtype), int(s.n_tokens), int(s.hidden), int(s.head_dim), int(s.n_parts))
+    fresh = {key(s): (s, th, us) for s, th, us in new.entries}
+    entries = [fresh.pop(key(s), (s, th, us)) for s, th, us in old.entries] + list(fresh.values())
+    generals = dict(old.generals)
+    for op, th in new.generals.items():
+        if not (keep_general and op in generals):
+            generals[op] = th
+    return B.SpecTable(entries, None, new.device_name or old.device_name, generals)
+
+
 def main() -> None:
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
     ap.add_argument("--shapes", required=True, help="comma-separated [kernel/]dtype:dims, e.g. bf16:128x4096,"
@@ -185,10 +203,18 @@ def main() -> None:
     ap.add_argument("--budget", type=int, default=64, help="kernel evaluations per shape")
     ap.add_argument("--out", default="", help="write the table as JSON here")
     ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--merge", default="", help="an existing table (JSON): its entries are kept, except where this run "
+                    "tuned the same kernel and shape again; its general configurations are kept for the kernels this run "
+                    "did not tune")
+    ap.add_argument("--keep-general", action="store_true", help="with --merge: keep the existing general configurations "
+                    "of the kernels tuned in this run as well (for a run over shapes only some stages can serve)")
     args = ap.parse_args()
     if not torch.cuda.is_available():
         raise SystemExit("tuning needs a CUDA device")
     table, report = tune(parse_shapes(args.shapes), budget=args.budget, seed=args.seed, verbose=True)
+    if args.merge:
+        with open(args.merge) as f:
+            table = merge_tables(B.SpecTable.from_json(json.load(f)), table, args.keep_general)
     if args.out:
         with open(args.out, "w") as f:
             json.dump(table.to_json(), f, indent=1)

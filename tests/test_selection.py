@@ -121,3 +121,23 @@ def test_shipped_table_loads_and_every_entry_is_feasible_for_its_shape():
     # (rows that are not 16-byte multiples are served by their own entries: the general 16-byte vectors do not divide them)
     assert all(B.tuner_check_params(s, table.generals[int(s.op)], L) == B.RT_OK for s, _, _ in table.entries
                if (s.hidden * (4 if s.dtype == B.RT_FP32 else 2)) % 16 == 0)
+
+
+def test_merging_tables_keeps_what_was_not_tuned_again():
+    from paper_2601_12698_b200 import binding as B
+    from paper_2601_12698_b200 import tune
+    th = lambda tpr: B.make_params(threads_per_row=tpr)
+    old = B.SpecTable([(B.shape_of(16, 4096, "bf16"), th(512), 1.6), (B.shape_of(8192, 5120, "fp16"), th(256), 52.0),
+                       (B.shape_of(64, 11008, "bf16", op=B.RT_OP_SILU_AND_MUL), th(1024), 2.3)],
+                      generals={B.RT_OP_ADD_RMSNORM: th(512), B.RT_OP_SILU_AND_MUL: th(1024)}, device_name="old device")
+    new = B.SpecTable([(B.shape_of(8192, 5120, "fp16"), th(128), 51.0), (B.shape_of(8192, 6145, "fp16"), th(64), 63.0)],
+                      generals={B.RT_OP_ADD_RMSNORM: th(128)}, device_name="new device")
+    merged = tune.merge_tables(old, new)
+    got = [(int(s.op), int(s.n_tokens), int(s.hidden), t.threads_per_row, round(us, 1)) for s, t, us in merged.entries]
+    assert got == [(0, 16, 4096, 512, 1.6), (0, 8192, 5120, 128, 51.0), (1, 64, 11008, 1024, 2.3), (0, 8192, 6145, 64, 63.0)]
+    assert merged.generals[B.RT_OP_ADD_RMSNORM].threads_per_row == 128 and merged.generals[B.RT_OP_SILU_AND_MUL].threads_per_row == 1024
+    assert tune.merge_tables(old, new, keep_general=True).generals[B.RT_OP_ADD_RMSNORM].threads_per_row == 512
+    assert merged.device_name == "new device"
+    # the merged table round-trips through its JSON form
+    again = B.SpecTable.from_json(merged.to_json())
+    assert [(t.key(), round(us, 1)) for _, t, us in again.entries] == [(t.key(), round(us, 1)) for _, t, us in merged.entries]
