@@ -221,7 +221,7 @@ def run_reference(args) -> None:
     if rank != 0:
         return  # rank 0 alone runs the oracle
     import oracle
-    wl = synth.workloads()[args.workload]
+    wl = workload_of(args.workload)
     cores = os.cpu_count() or 1
     is_silu = wl.op == "silu_and_mul"
 
@@ -289,6 +289,23 @@ def run_reference(args) -> None:
     print(json.dumps(line), flush=True)
 
 
+def workload_of(name: str):
+    """A named workload of synth.workloads(), or an ad-hoc shape of the norm written dtype:TOKENSxHIDDEN (N(0, 1) inputs,
+    seed 9) - e.g. bf16:5000x6144, for timing shapes the shipped table has no entry for."""
+    from paper_2601_12698_b200 import synth
+    table = synth.workloads()
+    if name in table:
+        return table[name]
+    try:
+        dtype, dims = name.split(":")
+        tokens, hidden = (int(v) for v in dims.lower().split("x"))
+        if dtype not in synth.DTYPE_BYTES or tokens < 1 or hidden < 1:
+            raise ValueError(name)
+    except ValueError:
+        raise SystemExit(f"unknown workload {name!r}: one of {', '.join(table)} or dtype:TOKENSxHIDDEN")
+    return synth.Workload(f"adhoc_{dtype}_{tokens}x{hidden}", dtype, tokens, hidden, seed=9)
+
+
 def fastest_of(log, k: int) -> list:
     """The k fastest distinct thetas of a search log that passed their gate (a theta's last record counts)."""
     last = {}
@@ -333,7 +350,7 @@ def run_ours(args) -> None:
     device = torch.device("cuda", local_rank)
     torch.cuda.set_device(device)
     dp.init(device=device)
-    wl = synth.workloads()[args.workload]
+    wl = workload_of(args.workload)
     if wl.op == "add_rmsnorm_allreduce" and world > 1:
         return run_tensor_parallel(args, wl, rank, world, device)
     shard = dp.weak_shard(wl.n_tokens, rank, world)
@@ -472,6 +489,18 @@ def run_ours(args) -> None:
         for th in (fastest_of(sweep_log, args.retest_top) + [guided.best] + fastest_of(guided_log, 2)):
             if th.key() not in [f.key() for f in finalists]:
                 finalists.append(th)
+        # what the shipped table would launch on this shape without any search (its entry for the shape, else the
+        # nearest entry's theta, else the general configuration), and the general configuration itself: timed in the
+        # same re-test, so that the cost of a table miss and of the one-size-fits-all choice is on record
+        shipped = B.SpecTable.default()
+        table_theta, table_source = shipped.lookup(shape)
+        general_theta = shipped.generals.get(op_code)
+        extras = {"table": table_theta}
+        if general_theta is not None and B.tuner_check_params(shape, general_theta) == B.RT_OK:
+            extras["general"] = general_theta
+        for th in extras.values():
+            if th.key() not in [f.key() for f in finalists]:
+                finalists.append(th)
         proto = B.make_budget(warmup=20, iters=100, repeats=1, use_graph=use_graph, preheat_ms=heat)
         recs, blocks = B.tuner_retest_interleaved(shape, finalists, proto, ws, args.retest_rounds)
         i_guided = [f.key() for f in finalists].index(guided.best.key())
@@ -511,7 +540,9 @@ def run_ours(args) -> None:
                                 "spread": round((max(blk.us for blk in per[i]) - recs[i].us_min_block) / recs[i].us, 4),
                                 "sm_mhz": sorted(m for m in mhz[i] if m)[len([m for m in mhz[i] if m]) // 2] if any(mhz[i]) else None,
                                 "us_x_mhz": round(normalised(i), 1) if normalised(i) else None,
-                                "from": ("guided" if i == i_guided else "sweep" if i < args.retest_top else "guided runner-up")}
+                                "from": ("guided" if i == i_guided else "sweep" if i < args.retest_top else
+                                         "shipped table / general" if finalists[i].key() in [e.key() for e in extras.values()]
+                                         else "guided runner-up")}
                                for i in ok],
             },
             "timing": ("CUDA graph of 100 launches, same buffers (L2-warm)" if use_graph else
@@ -522,6 +553,11 @@ def run_ours(args) -> None:
         }
         if seeds:
             tuner["resumed_seeds"] = len(seeds)
+        for name, th in extras.items():
+            i = [f.key() for f in finalists].index(th.key())
+            tuner["shipped_" + name] = {"theta": list(th.key()), "us": round(recs[i].us, 3) if recs[i].status == 0 else None,
+                                        "vs_exhaustive": round(recs[i].us / t_sweep.us, 4) if recs[i].status == 0 else None}
+        tuner["shipped_table"]["source"] = table_source
         # the sweep's fastest point of every stage (first measurement, us): which organisation of the row wins here
         by_stage = {}
         for rec in sweep_log:

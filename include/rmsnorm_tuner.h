@@ -226,7 +226,14 @@ typedef enum {
     RT_ERR_SHAPE = 3,          /* n_tokens < 0, hidden <= 0, hidden too large */
     RT_ERR_ALIGN = 4,          /* a pointer or the row length is not a multiple of vec_bytes (or of 16 for TMA);
                                   RT_STAGE_REG_REALIGN constrains the pointers only */
-    RT_ERR_INFEASIBLE = 5,     /* theta violates a hard limit; nothing was launched */
+    RT_ERR_INFEASIBLE = 5,     /* theta violates a hard limit; nothing was launched.  Also the answer for rows longer
+                                  than any theta can serve: a row is reduced in one pass by one CTA or one cluster,
+                                  so it must fit on chip.  The longest rows are served by RT_STAGE_SMEM_LDG, which
+                                  keeps the row as fp32 in up to 227 KB of shared memory: 57 856 elements in one CTA
+                                  and 462 336 split over a cluster of 8, for every dtype (the register stages hold
+                                  at most 128 elements per thread within 64 K registers per CTA, i.e. 32 768).
+                                  There is no multi-pass fall-back for longer rows (hidden sizes of language models
+                                  are an order of magnitude and more below the limit) */
     RT_ERR_CUDA = 6,           /* a CUDA runtime call failed; see rt_last_error() */
     RT_ERR_MISMATCH = 7,       /* correctness gate failed (search: for every candidate) */
     RT_ERR_BUDGET = 8,         /* the budget allows no evaluation */

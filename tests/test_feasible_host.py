@@ -234,3 +234,18 @@ def test_the_pipeline_stage_is_derived_only_on_request(L):
     # decode shapes: a CTA walks over one row block, so a deeper ring is the same kernel again (pruned as a duplicate)
     few = B.tuner_derive_feasible(B.shape_of(16, 4096, "bf16"), L, heuristics=B.RT_PRUNE_DEFAULT & ~B.RT_PRUNE_PIPELINE_STAGE)
     assert {t.unroll for t in few if t.stage == pipe} == {1}
+
+
+def test_the_longest_row_the_template_serves(L):
+    """The header states the limit: 57 856 elements in one CTA, 462 336 over a cluster of 8 (shared-memory stage)."""
+    for dtype in ("bf16", "fp32"):
+        f = B.tuner_derive_feasible(B.shape_of(4, 57856, dtype), L, heuristics=0)
+        assert {(t.stage, t.cluster_size) for t in f if t.cluster_size == 1} == {(B.RT_STAGE_SMEM_LDG, 1)}
+        assert not [t for t in B.tuner_derive_feasible(B.shape_of(4, 57856 + 64, dtype), L, heuristics=0) if t.cluster_size == 1]
+        assert B.tuner_derive_feasible(B.shape_of(4, 462336, dtype), L, heuristics=0)
+        assert B.tuner_derive_feasible(B.shape_of(4, 462336 + 64, dtype), L, heuristics=0) == []
+    # the register stages end at 128 elements per thread within the CTA's 64 K registers
+    f = B.tuner_derive_feasible(B.shape_of(4, 32768, "bf16"), L, heuristics=0)
+    assert any(t.stage == B.RT_STAGE_REG and t.cluster_size == 1 for t in f)
+    f = B.tuner_derive_feasible(B.shape_of(4, 32768 + 64, "bf16"), L, heuristics=0)
+    assert not any(t.stage == B.RT_STAGE_REG and t.cluster_size == 1 for t in f)

@@ -62,5 +62,29 @@ def test_searched_line_on_ragged_rows_reports_the_tuner():
     t = d["tuner"]
     assert t["feasible"] > 0 and t["raw_grid"] >= t["feasible"] and t["search_evals_used"] <= 24 and t["failed_gate"] == 0
     assert t["search_best"] == d["config"]["theta"] and t["search_best"]["stage"] == 3
-    assert 0.9 < t["search_vs_exhaustive"] < 1.1
+    assert 1.0 <= t["search_vs_exhaustive"] < 1.1          # the guided winner is a member of the re-tested set
     assert d["roofline"]["frac"] > 0.75
+    # the side-by-side re-test: every candidate with its spread and clock, the per-round ratios, the shipped table's pick
+    rt = t["retest"]
+    assert len(rt["per_round_ratio_min_median_max"]) == 3 and rt["per_round_ratio_min_median_max"][0] >= 1.0
+    assert any(c["from"] == "guided" for c in rt["candidates"]) and all(c["us"] > 0 and c["spread"] >= 0 for c in rt["candidates"])
+    assert t["shipped_table"]["source"] == "table_exact" and t["shipped_table"]["vs_exhaustive"] >= 1.0
+    assert set(t["sweep_best_per_stage"]) == {"reg", "reg_realign"}
+    assert d["cpu_baseline"]["single_thread"]["cores"] == 1 and d["cpu_baseline"]["single_thread"]["value"] > 0
+    assert d["clocks"]["samples"] >= 1 and d["roofline"]["traffic_capture"] is None or "kernel_sha256_16_now" in d["roofline"]["traffic_capture"]
+
+
+def test_a_search_resumes_from_its_log_and_ad_hoc_shapes_run(tmp_path):
+    """--log writes the search log, --resume seeds the next search with its fastest thetas (evaluated first, phase
+    'seed'); the workload is an ad-hoc shape the shipped table has no entry for, so the table's answer is a neighbour's."""
+    log = str(tmp_path / "search.jsonl")
+    d = _run("--workload", "bf16:700x4096", "--steps", "20", "--warmup", "3", "--e2e-steps", "2", "--search-budget", "20",
+             "--retest-rounds", "3", "--log", log)
+    assert d["config"]["workload"] == "adhoc_bf16_700x4096" and d["tuner"]["shipped_table"]["source"] == "table_nearest"
+    first = d["tuner"]["search_best"]
+    d2 = _run("--workload", "bf16:700x4096", "--steps", "20", "--warmup", "3", "--e2e-steps", "2", "--search-budget", "20",
+              "--retest-rounds", "3", "--resume", log, "--log", log + ".2")
+    assert d2["tuner"]["resumed_seeds"] >= 8
+    phases = [json.loads(line)["phase"] for line in open(log + ".2") if '"guided"' in line]
+    assert phases[0] == "seed" and phases.count("seed") >= 4
+    assert d2["tuner"]["search_best_us"] <= 1.1 * d["tuner"]["search_best_us"] and first

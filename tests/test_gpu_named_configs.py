@@ -122,3 +122,19 @@ def test_closed_forms_hold_on_the_device(B):
         assert float(y[row].abs().sum() - y[row, k].abs()) == 0.0
         assert abs(float(y[row, k]) - float(w64[k] * 7.0 / (49.0 / H + 1e-6) ** 0.5)) <= 2e-6 * abs(float(y[row, k]))
     assert torch.allclose(y[13], s[13] * w64 / (1.0 + 1e-6) ** 0.5, rtol=2e-6, atol=0)
+
+
+@pytest.mark.parametrize("dtype,T,H", [("fp32", 3, 57856), ("bf16", 3, 57856), ("bf16", 2, 462336), ("fp32", 2, 200000)])
+def test_the_longest_rows_the_template_serves(B, oracle_lib, dtype, T, H):
+    """Maximum sizes: the longest row one CTA serves (57 856 elements, shared-memory stage), the longest a cluster of 8
+    serves (462 336), and a length in between - every theta the deriver offers."""
+    from paper_2601_12698_b200 import synth
+    x, r, w = synth.make_inputs(T, H, dtype, seed=50)
+    thetas = B.tuner_derive_feasible(B.shape_of(T, H, dtype), heuristics=0)
+    assert thetas and (H <= 57856 or {t.cluster_size for t in thetas} <= {4, 8})
+    n, failures, worst = _run_all(B, oracle_lib, x, r, w, dtype, thetas)
+    assert not failures, f"{len(failures)} of {n} configurations differ: {failures[:5]}"
+    # one element more than the chip holds is refused, and nothing is launched
+    before = B.rt_launch_count()
+    assert B.tuner_derive_feasible(B.shape_of(T, 462336 + 64, dtype), heuristics=0) == []
+    assert B.rt_launch_count() == before
