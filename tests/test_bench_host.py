@@ -113,17 +113,18 @@ def test_clock_windows_pick_the_samples_of_an_interval():
 
 def test_traffic_figures_are_tied_to_the_kernel_they_were_captured_on():
     bench = _bench()
-    wl, theta = "c3_prefill_bf16_16384x8192", (256, 1, 32, 2, 0, 0, 1)
+    wl, theta = "c3_prefill_bf16_16384x8192", (512, 1, 32, 1, 0, 0, 1)
     nbytes, captured_on = bench.NCU_TRAFFIC[wl][theta]
     traffic, info = bench.ncu_traffic(wl, theta)
     assert info["bytes_per_launch"] == nbytes and info["kernel_sha256_16_now"] == bench.kernel_source_hash()
     assert (traffic == nbytes) == (captured_on == bench.kernel_source_hash())  # null once the kernel has changed
     assert bench.ncu_traffic(wl, (32, 8, 8, 1, 1, 1, 1)) == (None, None)
-    # every stored figure is within a few percent of the workload's algorithmic bytes: no re-reads
+    # every stored figure is at most the workload's algorithmic bytes plus a few percent (no re-reads), and short of
+    # them by no more than the share of the outputs that can still be dirty in L2 when the kernel ends
     from paper_2601_12698_b200 import synth
     for name, table in bench.NCU_TRAFFIC.items():
         alg = synth.workloads()[name].algorithmic_bytes
-        assert all(0.85 * alg < v[0] < 1.05 * alg for v in table.values())
+        assert all(alg - 60e6 < v[0] < 1.02 * alg for v in table.values())
 
 
 def test_phase_analysis_of_synthetic_stamps():
