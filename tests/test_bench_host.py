@@ -146,3 +146,30 @@ def test_phase_analysis_of_synthetic_stamps():
     assert info["launch_period_ns"] == 2000 and abs(info["released_to_stored_ns_slowest_cta"] - 1560 / 1.5) < 8
     assert abs(info["outside_the_kernel_ns"] - (2000 - 1560 / 1.5)) < 8
     assert info["next_launch_resident_before_exit_ns"] == (1300 + 20) - 2000
+
+
+def test_replay_of_a_recorded_sweep(tmp_path):
+    """replay.py: the guided search over a sweep log's times; a budget that covers the set finds the optimum exactly."""
+    import math
+    from paper_2601_12698_b200 import binding as B
+    from paper_2601_12698_b200 import replay, synth
+    wl = synth.workloads()["c2_decode_bf16_16x4096"]
+    shape = replay.shape_of_workload(wl)
+    feasible = B.tuner_derive_feasible(shape, B.sm100_nominal_limits())
+    names = [name for name, _ in B.rt_params._fields_]
+    cost = lambda t: 2.0 + 0.3 * abs(math.log2(t.threads_per_row) - 9) + 0.1 * (t.unroll - 1) + 0.2 * t.stage + 0.05 * t.reduce
+    log = tmp_path / "sweep.jsonl"
+    with open(log, "w") as f:
+        for t in feasible:
+            f.write(json.dumps({"search": "exhaustive", "workload": wl.name, "status": 0, "us": cost(t),
+                                "params": dict(zip(names, t.key()))}) + "\n")
+        f.write(json.dumps({"search": "guided", "workload": wl.name, "status": 0, "us": 0.1,
+                            "params": dict(zip(names, feasible[0].key()))}) + "\n")      # not part of the sweep: ignored
+        f.write(json.dumps({"search": "exhaustive", "workload": wl.name, "status": 7, "us": 0.1,
+                            "params": dict(zip(names, feasible[1].key()))}) + "\n")      # failed its gate: ignored
+    times = replay.load_sweep(str(log))[wl.name]
+    assert len(times) == len(feasible) and min(times.values()) >= 2.0
+    rows = replay.replay(times, shape, [4, 64, 4 * len(feasible)])
+    assert [b for b, _, _ in rows] == [4, 64, 4 * len(feasible)]
+    assert all(ratio >= 1.0 for _, ratio, _ in rows) and rows[0][2] <= 4 and rows[1][2] <= 64
+    assert rows[1][1] < 1.1 and rows[2][1] == 1.0
