@@ -88,8 +88,8 @@ std::vector<rt_params> raw_grid(const rt_shape& s)
     // Rows whose byte length is not a multiple of 32 (or of 16) also get the ragged-row register stage with 32-byte
     // (and 16-byte) chunks, which keeps wide accesses on such rows; on rows that the chunk width divides it would only
     // repeat the register stage with extra bookkeeping.
-    for (int chunk : {32, 16})
-        if (s.op == RT_OP_ADD_RMSNORM && (s.hidden * elem_bytes_of(s.dtype)) % chunk != 0)
+    for (int chunk : {32, 16}) {
+        if (s.op != RT_OP_ADD_RMSNORM || (s.hidden * elem_bytes_of(s.dtype)) % chunk == 0) continue;
         for (int tpr : kTprLevels)
             for (int rpc : kRpcLevels)
                 for (int u : kUnrollLevels) {
@@ -103,6 +103,7 @@ std::vector<rt_params> raw_grid(const rt_shape& s)
                     p.cluster_size = 1;
                     out.push_back(p);
                 }
+    }
     return out;
 }
 
