@@ -501,9 +501,9 @@ int tuner_select_general(const float* times_us, int32_t n_candidates, int32_t n_
 
 /*
  * BuildSpecialized's table put to use: theta for a query shape.  Host only (limits == NULL asks the
- * current device).  Order of preference: the table entry of the same dtype nearest to the query (distance
+ * current device).  Order of preference: the table entry of the same element size nearest to the query (distance
  * = 4 x octaves of hidden size + octaves of token count + 2 x octaves of head size where the kernel has
- * heads; distance 0 is an exact hit) whose theta passes the
+ * heads, + 0.25 for a bf16 entry serving an fp16 query or the reverse; distance 0 is an exact hit) whose theta passes the
  * hard feasibility rules for the query; else `general` (may be NULL) if feasible; else the first point
  * of the derived feasible set.  *source (may be NULL) receives an rt_theta_source.
  */

@@ -916,6 +916,30 @@ struct SearchState {
         step(kRpc, 4, &rt_params::rows_per_cta);
         step(kUnr, 3, &rt_params::unroll);
         step(kVec, 5, &rt_params::vec_bytes);
+        // Two diagonal steps that keep what a thread does unchanged: half the vector width with twice the unroll (the
+        // same bytes in flight per thread, in narrower instructions), and half the vector width with twice the threads per
+        // row (the same vectors per thread), and their reverses.  Along a single axis both halves of such a move are
+        // usually worse than the point they start from, so a climb over single steps does not cross them.
+        {
+            const int lv = level_of(kVec, 5, p.vec_bytes), lu = level_of(kUnr, 3, p.unroll),
+                      lt = level_of(kTpr, 6, p.threads_per_row);
+            for (int d = -1; d <= 1; d += 2) {
+                if (lv < 0 || lv + d < 0 || lv + d >= 5) continue;
+                if (lu >= 0 && lu - d >= 0 && lu - d < 3) {
+                    rt_params q = p;
+                    q.vec_bytes = kVec[lv + d];
+                    q.unroll = kUnr[lu - d];
+                    probe(q);
+                }
+                if (lt >= 0 && lt - d >= 0 && lt - d < 6) {
+                    rt_params q = p;
+                    q.vec_bytes = kVec[lv + d];
+                    q.threads_per_row = kTpr[lt - d];
+                    while (q.unroll > 1 && index.find(pack_params(q)) == index.end()) q.unroll /= 2;
+                    probe(q);
+                }
+            }
+        }
         // another stage at the same vector width; where that stage has no such point (the ragged-row stage is
         // all 16-byte chunks while the other stages of a misaligned shape are narrower), at its widest width
         for (int stage = 0; stage <= RT_STAGE_TMA_PIPELINE; ++stage) {

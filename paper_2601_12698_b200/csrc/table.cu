@@ -8,9 +8,11 @@
 
 namespace rt {
 
-// Distance between two shapes of one dtype: octaves of hidden size and of token count.  Hidden size
+// Distance between two shapes of one element size: octaves of hidden size and of token count.  Hidden size
 // weighs more: it fixes vector counts, register and shared-memory footprints; the token count only
-// decides how full the machine is.
+// decides how full the machine is.  bf16 and fp16 entries are neighbours of each other (the same bytes move through
+// the same instances; only the conversions differ), a quarter of an octave further away than an entry of the query's own
+// type: a table tuned on bf16 decode shapes then serves fp16 ones, instead of the nearest fp16 entry however far.
 static double shape_distance(const rt_shape& a, const rt_shape& b)
 {
     const double dh = fabs(log2((double)a.hidden) - log2((double)b.hidden));
@@ -19,7 +21,7 @@ static double shape_distance(const rt_shape& a, const rt_shape& b)
     if (a.head_dim > 0 && b.head_dim > 0) dd = fabs(log2((double)a.head_dim) - log2((double)b.head_dim));
     // all-reduce-fused norm: the part count multiplies the loads in flight per thread
     if (a.n_parts > 0 && b.n_parts > 0) dd += fabs(log2((double)a.n_parts) - log2((double)b.n_parts));
-    return 4.0 * dh + dt + 2.0 * dd;
+    return 4.0 * dh + dt + 2.0 * dd + (a.dtype != b.dtype ? 0.25 : 0.0);
 }
 
 int table_lookup(const rt_spec_entry* table, int32_t n, const rt_params* general, const rt_shape* query,
@@ -29,7 +31,7 @@ int table_lookup(const rt_spec_entry* table, int32_t n, const rt_params* general
     double best_d = 0.0;
     for (int32_t i = 0; i < n; ++i) {
         const rt_spec_entry& e = table[i];
-        if (e.shape.dtype != query->dtype || e.shape.op != query->op) continue;
+        if (elem_bytes_of(e.shape.dtype) != elem_bytes_of(query->dtype) || e.shape.op != query->op) continue;
         // the ragged-row stage runs on any row length, but on rows that its chunk width divides it is the register
         // stage plus bookkeeping: an entry tuned on a misaligned shape is not a neighbour of an aligned one
         if (e.best.stage == RT_STAGE_REG_REALIGN && e.best.vec_bytes > 0 &&

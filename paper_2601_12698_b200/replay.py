@@ -43,6 +43,18 @@ def shape_of_workload(wl) -> B.rt_shape:
     return B.shape_of(wl.n_tokens, wl.hidden, wl.dtype, op=op, head_dim=wl.head_dim, n_parts=wl.n_parts)
 
 
+def workload_named(name: str):
+    """A workload of synth.workloads(), or the ad-hoc norm shapes bench.py names adhoc_<dtype>_<tokens>x<hidden>."""
+    table = synth.workloads()
+    if name in table:
+        return table[name]
+    parts = name.split("_")
+    if len(parts) == 3 and parts[0] == "adhoc" and parts[1] in synth.DTYPE_BYTES and "x" in parts[2]:
+        tokens, hidden = (int(v) for v in parts[2].split("x"))
+        return synth.Workload(name, parts[1], tokens, hidden, seed=9)
+    return None
+
+
 def replay(times: dict, shape: B.rt_shape, budgets, top_k: int = 5) -> list:
     """[(budget, ratio of the returned theta's time to the sweep's optimum, evaluations used)]."""
     limits = B.sm100_nominal_limits()
@@ -62,14 +74,14 @@ def main(argv=None) -> None:
     ap.add_argument("--top-k", type=int, default=5)
     args = ap.parse_args(argv)
     budgets = [int(v) for v in args.budgets.split(",")]
-    table = synth.workloads()
     print("workload | swept | " + " | ".join(f"budget {b}" for b in budgets))
     for path in args.logs:
         for name, times in load_sweep(path).items():
-            if name not in table:
-                print(f"{name}: not a named workload, skipped", file=sys.stderr)
+            wl = workload_named(name)
+            if wl is None:
+                print(f"{name}: not a workload this tool knows, skipped", file=sys.stderr)
                 continue
-            rows = replay(times, shape_of_workload(table[name]), budgets, args.top_k)
+            rows = replay(times, shape_of_workload(wl), budgets, args.top_k)
             print(f"{name} | {len(times)} | " + " | ".join(f"{ratio:.3f} ({used})" for _, ratio, used in rows))
 
 

@@ -76,8 +76,17 @@ def test_table_lookup_prefers_exact_then_nearest_then_general():
     assert (theta.key(), src) == (th_big.key(), "table_nearest")
     theta, src = table.lookup(B.shape_of(300, 5120, "bf16"), L)     # 4*0.32+1.23 vs 4*0.68+5.77
     assert (theta.key(), src) == (th_small.key(), "table_nearest")
-    # a dtype the table lacks falls back to the general configuration
+    # bf16 and fp16 entries serve each other (same element size, a quarter of an octave further away than an entry of
+    # the query's own type); an element size the table lacks falls back to the general configuration
     theta, src = table.lookup(B.shape_of(8192, 5120, "fp16"), L)
+    assert (theta.key(), src) == (th_big.key(), "table_nearest")
+    theta, src = table.lookup(B.shape_of(128, 4096, "fp16"), L)           # same shape, other 16-bit type: nearest, not exact
+    assert (theta.key(), src) == (th_small.key(), "table_nearest")
+    both = B.SpecTable([(B.shape_of(128, 4096, "bf16"), th_small, 2.0), (B.shape_of(160, 4096, "fp16"), th_big, 2.1)], general)
+    assert both.lookup(B.shape_of(128, 4096, "fp16"), L)[0].key() == th_small.key()   # 0.25 for the type < 0.32 for the rows
+    assert both.lookup(B.shape_of(150, 4096, "fp16"), L)[0].key() == th_big.key()     # 0.09 for the rows < 0.23 + 0.25
+    only32 = B.SpecTable([(B.shape_of(32768, 12288, "fp32"), th_fp32, 950.0)], general)
+    theta, src = only32.lookup(B.shape_of(8192, 5120, "fp16"), L)
     assert (theta.key(), src) == (general.key(), "general")
     # an entry whose theta is not launchable for the query is skipped: rows of 6148 fp16 take no 16-byte vectors
     t16 = B.SpecTable([(B.shape_of(8192, 6152, "fp16"), B.make_params(vec_bytes=16), 66.0)],
