@@ -167,6 +167,24 @@ def tune(shapes, budget: int = 64, top_k: int = 5, finalists: int = 3, seed: int
             torch.cuda.empty_cache()
         entry = {"specialised_us": [round(min((times[c][x] for c in range(len(cand)) if times[c][x] > 0), default=-1.0), 3)
                                     for x in range(len(mine))]}
+        # BuildSpecialized: a shape's entry is its own search's winner, unless another shape's finalist beat it by more
+        # than half a percent when every finalist was timed on every shape (less than that is timing noise, and often
+        # the very same kernel under another name: an unroll deeper than the vectors a thread owns)
+        labels = [f"{k}/{d}:" + "x".join(str(v) for v in dims) for k, d, dims in mine]
+        keys = [c.key() for c in cand]
+        for i, (shape_i, th_i, us_i, n_i, label_i) in enumerate(per_shape):
+            if label_i not in labels:
+                continue
+            x = labels.index(label_i)
+            timed = [(times[c][x], c) for c in range(len(cand)) if times[c][x] > 0]
+            if not timed:
+                continue
+            us_best, c_best = min(timed)
+            us_own = times[keys.index(th_i.key())][x]
+            if us_own > 0 and us_best >= 0.995 * us_own:
+                per_shape[i] = (shape_i, th_i, us_own, n_i, label_i)
+            else:
+                per_shape[i] = (shape_i, cand[c_best], us_best, n_i, label_i)
         try:
             gi, score, _ = B.tuner_select_general(times)
             generals[OPS[kernel]] = cand[gi]
