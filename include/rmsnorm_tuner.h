@@ -385,7 +385,8 @@ int tuner_derive_counts(const rt_shape* s, const rt_limits* limits, int32_t heur
 /*
  * Search(S~, x, Theta_feasible) for one input shape (Algorithm 1): seeds first, then a coarse
  * grid over the feasible set, then best-first hill-climbing over one-step neighbours on
- * measured time (around the three fastest points, then, while budget remains, around up to the
+ * measured time (around the fastest point, then once around the fastest point of every other stage
+ * that is within 3 % of it, then around the three fastest and, while budget remains, up to the
  * twelve fastest), then a re-test of the top_k finalists ("Tuning agent": Top-K re-testing): they are
  * re-timed side by side as tuner_retest_interleaved does, each counts as one evaluation, the winner is the
  * fastest finalist that passes again, and a finalist that fails its re-test is replaced by the next runner-up

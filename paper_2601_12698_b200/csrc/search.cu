@@ -846,6 +846,7 @@ const int kRpc[] = {1, 2, 4, 8};
 const int kUnr[] = {1, 2, 4};
 const int kVec[] = {2, 4, 8, 16, 32};
 const int kClu[] = {1, 2, 4, 8};
+constexpr float kStageLeaderMargin = 1.03f;  // a stage's fastest point is climbed from while it is this close to the leader
 
 struct SearchState {
     std::vector<rt_params> cand;
@@ -1079,7 +1080,7 @@ int run_search(const rt_shape& shape, const rt_limits& limits, const rt_budget& 
             S.time_us[idx] = t;
         }
         // 3. best-first hill-climb: expand the neighbours of the fastest point not yet expanded, among
-        //    the three fastest found so far.  When those are all expanded and budget is left, the frontier
+        //    the three fastest found so far (and the stage leaders, below).  When those are all expanded and budget is left, the frontier
         //    widens by three at a time (up to the twelve fastest): an optimum two steps away from every
         //    leader - a narrower vector that only pays with a deeper unroll, say - is reached through a
         //    runner-up.  Stops when the widest frontier is expanded or the budget is spent.
@@ -1089,12 +1090,20 @@ int run_search(const rt_shape& shape, const rt_limits& limits, const rt_budget& 
             for (int i = 0; i < (int)S.cand.size(); ++i)
                 if (S.time_us[i] >= 0.f && isfinite(S.time_us[i])) order.push_back(i);
             std::sort(order.begin(), order.end(), [&](int a, int c) { return S.time_us[a] < S.time_us[c]; });
+            // the stages are separate basins, and the coarse grid may have met one of them only two levels away from
+            // its optimum: after the leader itself, the fastest point of every stage is climbed from once while it is
+            // within 3 % of the leader; then the rest of the `frontier` fastest points
             int pick = -1;
-            for (int k = 0; k < (int)order.size() && k < frontier; ++k)
-                if (!S.expanded[order[k]]) {
-                    pick = order[k];
-                    break;
-                }
+            if (!order.empty() && !S.expanded[order[0]]) pick = order[0];
+            bool seen[RT_STAGE_TMA_PIPELINE + 1] = {false, false, false, false, false};
+            for (int k = 0; k < (int)order.size() && pick < 0; ++k) {
+                if (S.time_us[order[k]] > kStageLeaderMargin * S.time_us[order[0]]) break;
+                const int s = S.cand[order[k]].stage;
+                if (!seen[s] && !S.expanded[order[k]]) pick = order[k];
+                seen[s] = true;
+            }
+            for (int k = 0; k < (int)order.size() && k < frontier && pick < 0; ++k)
+                if (!S.expanded[order[k]]) pick = order[k];
             if (pick < 0) {
                 if (frontier >= 12 || frontier >= (int)order.size()) break;
                 frontier += 3;

@@ -178,6 +178,31 @@ def test_an_optimum_two_steps_from_every_leader_is_reached_with_leftover_budget(
     assert small.evals_used <= 20
 
 
+def test_the_fastest_point_of_another_stage_is_climbed_from_while_the_leaders_keep_improving(L):
+    """The shape of a sweep recorded on fp32 32768 x 12288: the shared-memory stage is a wide shallow bowl whose
+    points keep the three leaders busy for the whole budget, the register stage is a narrow one whose optimum
+    (512 threads per row) lies between two levels of the coarse grid and 2 % under the other stage's best.  The
+    register stage's fastest grid point is within 3 % of the leader, so it gets an expansion of its own."""
+    s = B.shape_of(32768, 12288, "fp32")
+
+    def cost(p):
+        lt, lr, lu = math.log2(p.threads_per_row), math.log2(p.rows_per_cta), math.log2(p.unroll)
+        wide = 0.0 if p.vec_bytes == 32 else 6.0
+        tree = 0.0 if p.reduce == 0 else 9.0
+        if p.stage == 1:      # shallow: 0.4 % per level around 256 x 2, unroll 2
+            return 100.0 + 0.4 * (abs(lt - 8) + abs(lr - 1) + abs(lu - 1)) + wide + tree
+        if p.stage == 0:      # narrow: 98 at 512 x 1, unroll 2; 2.5 per level of threads per row
+            return 98.0 + 4.0 * abs(lt - 9) + 6.0 * lr + 1.0 * abs(lu - 1) + wide + tree
+        return 112.0 + wide + tree
+
+    feasible = B.tuner_derive_feasible(s, L)
+    assert any(t.key() == (512, 1, 32, 2, 0, 0, 1) for t in feasible)
+    res, log = B.tuner_search_with(s, L, B.make_budget(max_evals=64, top_k=5), cost)
+    grid = [r.params for r in log if r.phase == 1]  # 1: the coarse grid
+    assert not any(p.stage == 0 and p.threads_per_row == 512 for p in grid)      # the grid itself does not see it
+    assert res.best.key() == (512, 1, 32, 2, 0, 0, 1) and res.best_us == pytest.approx(98.0)
+
+
 RAGGED_OPTIMA = [dict(tpr=256, rpc=1, unroll=4, vec=16, stage=3, reduce=0),   # 16-byte chunks of the ragged-row stage
                  dict(tpr=1024, rpc=1, unroll=4, vec=2, stage=0, reduce=0),   # the 2-byte row vectors of the register stage
                  dict(tpr=128, rpc=2, unroll=1, vec=32, stage=3, reduce=0)]   # 32-byte chunks
