@@ -125,7 +125,7 @@ typedef struct {
     int32_t max_cluster_size;
     int32_t have_device;            /* 1: per-kernel registers/spills and occupancy come from the CUDA
                                        runtime; 0: registers, spills and shared memory come from the
-                                       compiler's report for this build, occupancy from arithmetic on r(h) */
+                                       compiler's report for the library as compiled, occupancy from arithmetic on r(h) */
     int64_t smem_per_block_optin;   /* largest dynamic + static shared memory one CTA may ask for */
     int64_t smem_per_sm;
     int64_t smem_reserved_per_block;

@@ -228,7 +228,7 @@ int min_pointer_alignment(const void* a, const void* b, const void* c, const voi
 }
 
 // Registers per thread, static shared memory and spill size of every instance as ptxas reported them for
-// this build (table generated by the build script).  Used when no device can be asked; with a device the
+// this compilation of the library (table generated by the build script).  Used when no device can be asked; with a device the
 // runtime's own figures are used instead.
 struct InstanceResources {
     int op, dtype, vec_bytes, stage, reduce, unroll, cap, regs, static_smem, spill_bytes, parts;

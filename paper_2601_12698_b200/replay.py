@@ -7,7 +7,7 @@ guided search, which is ignored here).  The sweep's measured times become the co
 (a lookup: a theta the sweep did not time counts as failing its gate), and the guided search is run over it once per
 budget.  Printed per budget: the time of the theta the search returns divided by the sweep's optimum, and the
 evaluations it used - how much of the optimum a budget buys, free of re-timing noise.  The feasible set is derived
-from the documented sm_100 limits and this build's compiler report, so the replay runs on any machine.
+from the documented sm_100 limits and the compiler's report on the library as compiled, so the replay runs on any machine.
 """
 from __future__ import annotations
 
