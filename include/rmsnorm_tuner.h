@@ -140,7 +140,15 @@ enum {
     RT_PRUNE_IDLE_ROWS = 8,     /* more rows per CTA than the batch has rows */
     RT_PRUNE_PIPELINE_STAGE = 16, /* RT_STAGE_TMA_PIPELINE: measured on B200 it wins on no shape tried, so the
                                      default search does not pay for its points; clear the bit to include them */
-    RT_PRUNE_DEFAULT = 31
+    RT_PRUNE_BYTES_IN_FLIGHT = 32, /* Little's law on the loads.  On a batch of two waves of CTAs or more: theta keeps
+                                      fewer than 32 KB of input in flight per SM (resident CTAs x what one CTA requests
+                                      before it consumes anything: a row slice per input in the bulk-copy stages, one
+                                      batch of `unroll` vectors per thread and input otherwise) while some other theta
+                                      of the shape reaches that.  B200 needs 16-22 KB per SM (3.3 TB/s of reads x
+                                      0.7-1 us); of 7579 such points timed in 59 exhaustive sweeps none came within
+                                      21 % of its shape's optimum.  Not applied to the fall-back vector widths (4, 2
+                                      bytes) nor to merge_attn_states */
+    RT_PRUNE_DEFAULT = 63
 };
 
 typedef enum { RT_SEARCH_GUIDED = 0, RT_SEARCH_EXHAUSTIVE = 1 } rt_strategy;

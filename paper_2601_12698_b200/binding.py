@@ -23,7 +23,8 @@ RT_STAGE_REG, RT_STAGE_SMEM_LDG, RT_STAGE_SMEM_TMA, RT_STAGE_REG_REALIGN, RT_STA
 RT_REDUCE_SHFL, RT_REDUCE_SMEM, RT_REDUCE_CLUSTER = 0, 1, 2
 RT_PRUNE_IDLE_THREADS, RT_PRUNE_DUPLICATES, RT_PRUNE_CLUSTER_WAVES, RT_PRUNE_IDLE_ROWS = 1, 2, 4, 8
 RT_PRUNE_PIPELINE_STAGE = 16
-RT_PRUNE_DEFAULT = 31
+RT_PRUNE_BYTES_IN_FLIGHT = 32
+RT_PRUNE_DEFAULT = 63
 RT_SEARCH_GUIDED, RT_SEARCH_EXHAUSTIVE = 0, 1
 RT_CMP_BITS, RT_CMP_ULP16, RT_CMP_REL32 = 0, 1, 2
 (RT_OK, RT_ERR_NULL, RT_ERR_DTYPE, RT_ERR_SHAPE, RT_ERR_ALIGN, RT_ERR_INFEASIBLE, RT_ERR_CUDA, RT_ERR_MISMATCH,

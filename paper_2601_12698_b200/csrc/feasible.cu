@@ -107,6 +107,32 @@ std::vector<rt_params> raw_grid(const rt_shape& s)
     return out;
 }
 
+// Bytes of input an SM has in flight at once under theta: resident CTAs x what one CTA asks for before it
+// consumes anything (a whole row slice per input for the bulk-copy stages, one batch of `unroll` vectors per
+// thread and input otherwise).  0 when the rule below does not apply: fewer than two waves of CTAs (the batch, not
+// theta, bounds what is in flight), the fall-back vector widths (nothing wider exists for the shape), and
+// merge_attn_states (rows of one head: its CTAs are bound by their count, not by what each one loads).
+static int64_t load_bytes_in_flight_per_sm(const rt_shape& s, const rt_limits& L, const rt_params& p, const Plan& plan,
+                                           int occupancy)
+{
+    if (s.op == RT_OP_MERGE_ATTN_STATES || p.vec_bytes < 8 || occupancy < 1) return 0;
+    if ((int64_t)plan.grid_x < 2 * (int64_t)L.sm_count * occupancy) return 0;
+    const int64_t slice_bytes = (int64_t)plan.slice_nvec * p.vec_bytes * p.rows_per_cta;
+    const int inputs = s.op == RT_OP_ADD_RMSNORM_ALLREDUCE ? s.n_parts + 1 : 2;  // x and r; gate and up; the parts and r
+    int64_t per_cta = slice_bytes;
+    if (p.stage == RT_STAGE_TMA_PIPELINE)
+        per_cta = slice_bytes * p.unroll;
+    else if (p.stage != RT_STAGE_SMEM_TMA)
+        per_cta = std::min<int64_t>(slice_bytes, (int64_t)p.threads_per_row * p.rows_per_cta * p.vec_bytes * p.unroll);
+    return per_cta * inputs * occupancy;
+}
+
+// Little's law on the loads: DRAM read bandwidth x latency under load is what the whole GPU must have in flight
+// (about 3.3 TB/s of reads x 0.7-1 us = 2.3-3.3 MB on B200, 16-22 KB per SM) before bandwidth, not latency, bounds the
+// kernel.  Measured on 59 exhaustive sweeps of bandwidth-bound shapes (bf16, fp16, fp32; 1024 to 32768 rows of 4096 to
+// 14336 elements): of the 7579 points below 32 KB per SM none came within 21 % of its shape's optimum.
+constexpr int64_t kMinLoadBytesInFlightPerSm = 32 * 1024;
+
 // The heuristic rules.  Returns the RT_PRUNE_* bit of the first rule that removes theta, or 0.
 static int heuristic_reject(const rt_shape& s, const rt_limits& L, const rt_params& p, const Plan& plan, int mask)
 {
@@ -146,6 +172,9 @@ int derive_feasible(const rt_shape& s, const rt_limits& L, int heuristics, std::
     }
     const std::vector<rt_params> raw = raw_grid(s);
     local[kRejectReasons + 2] = (int32_t)raw.size();
+    std::vector<rt_params> kept;
+    std::vector<int64_t> in_flight;  // per kept theta; 0: the bytes-in-flight rule does not apply to it
+    int64_t most_in_flight = 0;
     for (const rt_params& p : raw) {
         Plan plan;
         const int st = make_plan(&s, &p, &L, &plan);
@@ -154,7 +183,8 @@ int derive_feasible(const rt_shape& s, const rt_limits& L, int heuristics, std::
             local[plan.reject_reason < kRejectReasons ? plan.reject_reason : kRejectArgs]++;
             continue;
         }
-        if (plan_occupancy(plan, &L, nullptr) < 1) {
+        const int occupancy = plan_occupancy(plan, &L, nullptr);
+        if (occupancy < 1) {
             local[plan.dyn_smem > 0 ? kRejectSmem : kRejectRegisters]++;
             continue;
         }
@@ -162,8 +192,20 @@ int derive_feasible(const rt_shape& s, const rt_limits& L, int heuristics, std::
             local[kRejectReasons]++;
             continue;
         }
+        kept.push_back(p);
+        in_flight.push_back(load_bytes_in_flight_per_sm(s, L, p, plan, occupancy));
+        most_in_flight = std::max(most_in_flight, in_flight.back());
+    }
+    // RT_PRUNE_BYTES_IN_FLIGHT: a theta that keeps too few bytes of loads in flight to cover DRAM latency, on a
+    // shape where some other theta does (narrow rows may allow none: then the rule is void and all stay)
+    const bool rule_applies = (heuristics & RT_PRUNE_BYTES_IN_FLIGHT) && most_in_flight >= kMinLoadBytesInFlightPerSm;
+    for (size_t i = 0; i < kept.size(); ++i) {
+        if (rule_applies && in_flight[i] > 0 && in_flight[i] < kMinLoadBytesInFlightPerSm) {
+            local[kRejectReasons]++;
+            continue;
+        }
         local[kRejectReasons + 1]++;
-        if (out) out->push_back(p);
+        if (out) out->push_back(kept[i]);
     }
     if (counts) memcpy(counts, local, sizeof(local));
     return RT_OK;

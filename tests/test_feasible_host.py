@@ -40,10 +40,42 @@ def test_heuristics_only_remove_points(L):
     s = B.shape_of(128, 4096, "bf16")
     wide = _keys(B.tuner_derive_feasible(s, L, heuristics=0))
     for mask in (B.RT_PRUNE_IDLE_THREADS, B.RT_PRUNE_DUPLICATES, B.RT_PRUNE_CLUSTER_WAVES, B.RT_PRUNE_IDLE_ROWS,
-                 B.RT_PRUNE_DEFAULT):
+                 B.RT_PRUNE_BYTES_IN_FLIGHT, B.RT_PRUNE_DEFAULT):
         narrow = _keys(B.tuner_derive_feasible(s, L, heuristics=mask))
         assert narrow <= wide
     assert len(_keys(B.tuner_derive_feasible(s, L))) < len(wide)
+
+
+def test_the_bytes_in_flight_rule_follows_littles_law_and_only_where_it_can(L):
+    """On a batch of two waves or more, a theta that keeps less than 32 KB of input in flight per SM goes; the figure
+    is recomputed here from the 48 KB rows, the block shape and the resident CTAs that the registers allow."""
+    without = B.RT_PRUNE_DEFAULT & ~B.RT_PRUNE_BYTES_IN_FLIGHT
+    s = B.shape_of(32768, 12288, "fp32")
+    wide, narrow = _keys(B.tuner_derive_feasible(s, L, heuristics=without)), _keys(B.tuner_derive_feasible(s, L))
+    assert narrow < wide and len(wide) - len(narrow) > 100
+    gone = wide - narrow
+    # register stage, 128 threads x 1 row, 32-byte vectors, unroll 1: 128 x 32 B x 2 inputs = 8 KB per CTA; three such
+    # CTAs per SM (12 vectors of fp32 per thread cost registers) stay under 32 KB - the closest any pruned point came
+    # to an optimum in the recorded sweeps (1.22 of it)
+    assert (128, 1, 32, 1, 0, 0, 1) in gone and (512, 1, 32, 2, 0, 0, 1) in narrow and (256, 2, 32, 2, 1, 0, 1) in narrow
+    # the bulk-copy stage requests whole rows: 2 x 48 KB per CTA, never pruned by this rule
+    assert not any(k[4] == B.RT_STAGE_SMEM_TMA for k in gone)
+    # a pruned point's CTA itself asks for less than 32 KB (threads x vector x unroll x 2 inputs)
+    assert all(k[0] * k[1] * k[2] * k[3] * 2 < 32 * 1024 for k in gone)
+    # fewer than two waves: the batch bounds what is in flight, the rule is void (decode and the small configuration)
+    for shape in (B.shape_of(128, 4096, "bf16"), B.shape_of(256, 4096, "bf16"), B.shape_of(64, 8192, "bf16", op=B.RT_OP_SILU_AND_MUL)):
+        assert _keys(B.tuner_derive_feasible(shape, L, heuristics=without)) == _keys(B.tuner_derive_feasible(shape, L))
+    # rows so narrow that no theta reaches the threshold: all stay
+    s = B.shape_of(1 << 20, 64, "bf16")
+    assert _keys(B.tuner_derive_feasible(s, L, heuristics=without)) == _keys(B.tuner_derive_feasible(s, L)) != set()
+    # the fall-back vector widths are exempt (nothing wider exists for the row), the ragged-row stage is not
+    s = B.shape_of(8192, 6145, "fp16")
+    wide, narrow = B.tuner_derive_feasible(s, L, heuristics=without), B.tuner_derive_feasible(s, L)
+    assert {t.key() for t in wide if t.vec_bytes == 2} == {t.key() for t in narrow if t.vec_bytes == 2} != set()
+    assert len([t for t in narrow if t.stage == B.RT_STAGE_REG_REALIGN]) < len([t for t in wide if t.stage == B.RT_STAGE_REG_REALIGN])
+    # merge_attn_states is left alone
+    s = B.shape_of(32768, 4096, "bf16", op=B.RT_OP_MERGE_ATTN_STATES, head_dim=128)
+    assert _keys(B.tuner_derive_feasible(s, L, heuristics=without)) == _keys(B.tuner_derive_feasible(s, L))
 
 
 def test_rules_bite_where_they_should(L):

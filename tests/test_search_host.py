@@ -36,7 +36,7 @@ def _cost_factory(opt, noise=None, counter=None):
 OPTIMA = [dict(tpr=256, rpc=1, unroll=1, vec=16, stage=2, reduce=0),
           dict(tpr=128, rpc=2, unroll=2, vec=16, stage=0, reduce=1),
           dict(tpr=512, rpc=1, unroll=4, vec=8, stage=1, reduce=0),
-          dict(tpr=64, rpc=4, unroll=2, vec=16, stage=1, reduce=0)]
+          dict(tpr=128, rpc=4, unroll=4, vec=16, stage=1, reduce=0)]
 
 
 @pytest.mark.parametrize("opt", OPTIMA)
