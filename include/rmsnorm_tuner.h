@@ -134,7 +134,7 @@ typedef struct {
 
 /* Heuristic ("obvious inefficiency") pruning rules; hard rules are always applied. */
 enum {
-    RT_PRUNE_IDLE_THREADS = 1,  /* a thread of the row would never own a vector */
+    RT_PRUNE_IDLE_THREADS = 1,  /* half the threads of the row or more would never own a vector */
     RT_PRUNE_DUPLICATES = 2,    /* unroll deeper than the per-thread vector count: same kernel again */
     RT_PRUNE_CLUSTER_WAVES = 4, /* split rows over a cluster only while whole rows cannot fill the SMs */
     RT_PRUNE_IDLE_ROWS = 8,     /* more rows per CTA than the batch has rows */

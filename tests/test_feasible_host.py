@@ -78,6 +78,17 @@ def test_the_bytes_in_flight_rule_follows_littles_law_and_only_where_it_can(L):
     assert _keys(B.tuner_derive_feasible(s, L, heuristics=without)) == _keys(B.tuner_derive_feasible(s, L))
 
 
+def test_idle_threads_are_pruned_from_half_the_row_on(L):
+    """5120 bf16 elements are 320 32-byte vectors: 512 threads per row (one vector per thread, 192 idle) stay - measured
+    the fastest on 32 x 5120 -, 1024 (more than half idle) go; on a power-of-two vector count nothing is in between."""
+    f = _keys(B.tuner_derive_feasible(B.shape_of(32, 5120, "bf16"), L))
+    assert (512, 1, 32, 1, 0, 0, 1) in f and (1024, 1, 32, 1, 0, 0, 1) not in f and (1024, 1, 16, 1, 0, 0, 1) in f
+    wide = _keys(B.tuner_derive_feasible(B.shape_of(32, 5120, "bf16"), L, heuristics=B.RT_PRUNE_DEFAULT & ~B.RT_PRUNE_IDLE_THREADS))
+    assert (1024, 1, 32, 1, 0, 0, 1) in wide
+    f = _keys(B.tuner_derive_feasible(B.shape_of(128, 4096, "bf16"), L))     # 256 vectors of 32 bytes
+    assert (256, 1, 32, 1, 0, 0, 1) in f and (512, 1, 32, 1, 0, 0, 1) not in f
+
+
 def test_rules_bite_where_they_should(L):
     ragged = B.RT_STAGE_REG_REALIGN
 
