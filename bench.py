@@ -477,14 +477,18 @@ def run_ours(args) -> None:
         # both searches (and so into the per-stage table below)
         mask = B.RT_PRUNE_DEFAULT & ~B.RT_PRUNE_PIPELINE_STAGE if args.include_pipeline else B.RT_PRUNE_DEFAULT
         counts = B.tuner_derive_counts(shape, heuristics=mask)
+        # --sweep-heuristics widens (or narrows) the exhaustive sweep alone: with 0 it covers every hard-feasible theta,
+        # and the re-test below then shows what the heuristic rules cost on this shape, if anything
+        sweep_mask = mask if args.sweep_heuristics < 0 else args.sweep_heuristics
+        sweep_evals = B.tuner_derive_counts(shape, heuristics=sweep_mask)["feasible"]
         # bandwidth-bound workloads are compared on a loaded device: the tuner keeps the GPU busy this long before its
         # first timing and before every side-by-side re-test (the latency-bound ones never reach the power limit)
         heat = 0 if small else args.preheat_ms
         # Both searches time every candidate with the paper's protocol (20 warm-up launches, blocks of 100).
         t0 = time.perf_counter()
-        sweep, sweep_log = B.tuner_search(shape, B.make_budget(max_evals=counts["feasible"], warmup=20, iters=100, repeats=2,
+        sweep, sweep_log = B.tuner_search(shape, B.make_budget(max_evals=sweep_evals, warmup=20, iters=100, repeats=2,
                                                                top_k=0, strategy=B.RT_SEARCH_EXHAUSTIVE,
-                                                               use_graph=use_graph, heuristics=mask, preheat_ms=heat), ws_tune)
+                                                               use_graph=use_graph, heuristics=sweep_mask, preheat_ms=heat), ws_tune)
         sweep_s = time.perf_counter() - t0
         seeds = resume_seeds(args.resume, wl.name) if args.resume else None
         t0 = time.perf_counter()
@@ -537,7 +541,7 @@ def run_ours(args) -> None:
             "search_budget_evals": args.search_budget, "search_evals_used": guided.evals_used,
             "search_best": theta_dict(guided.best), "search_best_us": round(t_guided.us, 3),
             "exhaustive_best": theta_dict(finalists[i_best]), "exhaustive_best_us": round(t_sweep.us, 3),
-            "exhaustive_evals": sweep.evals_used, "failed_gate": guided.n_failed_gate + sweep.n_failed_gate,
+            "exhaustive_evals": sweep.evals_used, "sweep_heuristics": sweep_mask, "failed_gate": guided.n_failed_gate + sweep.n_failed_gate,
             "search_vs_exhaustive": round(t_guided.us / t_sweep.us, 4),
             "search_vs_exhaustive_clock_normalised": (round(norm_guided / norm_best, 4) if norm_guided and norm_best else None),
             "retest": {
@@ -992,6 +996,8 @@ def main() -> None:
     ap.add_argument("--transfer-budget", type=int, default=24)
     ap.add_argument("--log", default="", help="write every evaluated theta of both searches to this JSONL file")
     ap.add_argument("--include-pipeline", action="store_true", help="search the persistent TMA pipeline stage as well")
+    ap.add_argument("--sweep-heuristics", type=int, default=-1, help="RT_PRUNE_* mask of the exhaustive sweep alone "
+                    "(0: every hard-feasible theta; default: the mask of the guided search)")
     ap.add_argument("--resume", default="", help="a JSONL file written by --log: its fastest thetas seed the guided search")
     ap.add_argument("--preheat-ms", type=int, default=300, help="how long the tuner loads the device before it compares "
                     "candidates of a bandwidth-bound workload")
