@@ -69,7 +69,8 @@ NCU_TRAFFIC = {
         (256, 1, 32, 1, 2, 0, 1): (1022521600, "b88197c58880f0a9"),
     },
     "c4_fp16_8192x5120": {(256, 1, 32, 2, 0, 0, 1): (283748096, "b88197c58880f0a9")},
-    "c4_fp16_8192x7168": {(256, 1, 32, 2, 0, 0, 1): (416248320, "b88197c58880f0a9")},
+    "c4_fp16_8192x7168": {(256, 1, 32, 2, 0, 0, 1): (416248320, "b88197c58880f0a9"),
+                          (512, 1, 32, 1, 0, 0, 1): (416799744, "b88197c58880f0a9")},
     "c4_fp16_8192x6152": {(256, 1, 16, 4, 0, 0, 1): (350612992, "b88197c58880f0a9")},
     # the ragged-row stage with 32-byte chunks; 6145: 201.58 MB read + 152.15 MB written (--set full)
     "c4x_fp16_8192x6145": {(256, 1, 32, 2, 3, 0, 1): (353729280, "b88197c58880f0a9")},
