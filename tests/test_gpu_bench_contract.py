@@ -76,15 +76,19 @@ def test_searched_line_on_ragged_rows_reports_the_tuner():
 
 def test_a_search_resumes_from_its_log_and_ad_hoc_shapes_run(tmp_path):
     """--log writes the search log, --resume seeds the next search with its fastest thetas (evaluated first, phase
-    'seed'); the workload is an ad-hoc shape the shipped table has no entry for, so the table's answer is a neighbour's."""
+    'seed'); the workload is an ad-hoc shape the shipped table has no entry for, so the table's answer is a neighbour's;
+    --sweep-heuristics widens the exhaustive sweep alone."""
     log = str(tmp_path / "search.jsonl")
     d = _run("--workload", "bf16:700x4096", "--steps", "20", "--warmup", "3", "--e2e-steps", "2", "--search-budget", "20",
              "--retest-rounds", "3", "--log", log)
     assert d["config"]["workload"] == "adhoc_bf16_700x4096" and d["tuner"]["shipped_table"]["source"] == "table_nearest"
     first = d["tuner"]["search_best"]
     d2 = _run("--workload", "bf16:700x4096", "--steps", "20", "--warmup", "3", "--e2e-steps", "2", "--search-budget", "20",
-              "--retest-rounds", "3", "--resume", log, "--log", log + ".2")
+              "--retest-rounds", "3", "--resume", log, "--log", log + ".2", "--sweep-heuristics", "18")
     assert d2["tuner"]["resumed_seeds"] >= 8
+    # the sweep alone ran over the hard-feasible set (duplicates and the pipeline stage aside), the search over the default one
+    assert d2["tuner"]["sweep_heuristics"] == 18 and d2["tuner"]["exhaustive_evals"] > d2["tuner"]["feasible"] == d["tuner"]["feasible"]
+    assert d["tuner"]["sweep_heuristics"] == 63 and d["tuner"]["exhaustive_evals"] == d["tuner"]["feasible"]
     phases = [json.loads(line)["phase"] for line in open(log + ".2") if '"guided"' in line]
     assert phases[0] == "seed" and phases.count("seed") >= 4
     assert d2["tuner"]["search_best_us"] <= 1.1 * d["tuner"]["search_best_us"] and first
