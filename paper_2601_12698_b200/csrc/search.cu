@@ -846,7 +846,8 @@ const int kRpc[] = {1, 2, 4, 8};
 const int kUnr[] = {1, 2, 4};
 const int kVec[] = {2, 4, 8, 16, 32};
 const int kClu[] = {1, 2, 4, 8};
-constexpr float kStageLeaderMargin = 1.03f;  // a stage's fastest point is climbed from while it is this close to the leader
+constexpr float kStageLeaderMargin = 1.03f;
+constexpr int kCentreVectorsPerThread = 1;  // vectors a thread owns at the centre level of the threads-per-row axis  // a stage's fastest point is climbed from while it is this close to the leader
 
 struct SearchState {
     std::vector<rt_params> cand;
@@ -967,29 +968,43 @@ struct SearchState {
     }
 };
 
-// The coarse grid: every other level of the ordered axes (threads per row 64/256/1024, rows per CTA
-// 1/4, unroll 1 and the deepest feasible), the widest vector of the point's stage, every stage and reduction mode.
-bool on_coarse_grid(const rt_params& p, int widest_vec, bool deepest_unroll)
+// The centre of the threads-per-row axis for a point's mode: the level at which a thread owns about one vector of its
+// CTA's slice of the row at the stage's widest vector (8192 bf16 elements in 32-byte vectors: 512 threads; the same
+// row split over a cluster of 8: 64).  The optima of the recorded sweeps sit at that level or next to it, so the grid
+// and the small-budget order are laid out from there instead of from a fixed 256.
+int centre_level(const rt_shape& s, const rt_params& p, int vec_bytes)
 {
-    const int lt = level_of(kTpr, 6, p.threads_per_row), lr = level_of(kRpc, 4, p.rows_per_cta),
-              lu = level_of(kUnr, 3, p.unroll);
+    const int64_t slice_vectors =
+        std::max<int64_t>(1, s.hidden * (s.dtype == RT_FP32 ? 4 : 2) / vec_bytes / std::max(1, p.cluster_size));
+    int level = 0;
+    while (level < 5 && kTpr[level] * kCentreVectorsPerThread < slice_vectors) ++level;
+    return level;
+}
+
+// The coarse grid: every other level of the ordered axes (threads per row: the centre level and every second level
+// from it; rows per CTA 1/4; unroll 1 and the deepest feasible), the widest vector of the point's stage, every stage
+// and reduction mode.
+bool on_coarse_grid(const rt_shape& s, const rt_params& p, int widest_vec, bool deepest_unroll)
+{
+    const int lt = level_of(kTpr, 6, p.threads_per_row) - centre_level(s, p, widest_vec);
+    const int lr = level_of(kRpc, 4, p.rows_per_cta), lu = level_of(kUnr, 3, p.unroll);
     // the two ends of the unroll axis: 1, and the deepest unroll that is feasible beside these other parameters
     // (4 where a thread owns that many vectors; with wide vectors and many threads per row it is 2, and the
     // step from 1 to 2 can be the steepest of the whole space)
-    return (lt % 2 == 1) && (lr % 2 == 0) && (lu == 0 || deepest_unroll) && p.vec_bytes == widest_vec;
+    return (lt % 2 == 0) && (lr % 2 == 0) && (lu == 0 || deepest_unroll) && p.vec_bytes == widest_vec;
 }
 
 // When the budget cannot cover the whole coarse grid, the part that is evaluated must still touch every
 // stage x reduction mode: the grid points are ordered mode by mode in rounds - first every mode's point
-// nearest the middle of the ordered axes (256 threads per row, one row per CTA, unroll 1), then every mode's
+// nearest its centre (the centre level of threads per row, one row per CTA, unroll 1), then every mode's
 // second nearest, and so on - and the first `keep` of that order are taken.
-std::vector<int> stratified(const std::vector<int>& coarse, const std::vector<rt_params>& cand, int keep)
+std::vector<int> stratified(const rt_shape& s, const std::vector<int>& coarse, const std::vector<rt_params>& cand, int keep)
 {
     if (keep <= 0) return {};
     if ((int)coarse.size() <= keep) return coarse;
     auto mode_of = [](const rt_params& p) { return (p.reduce * 16 + p.cluster_size) * 4 + p.stage; };
-    auto off_centre = [](const rt_params& p) {
-        return 2 * abs(level_of(kTpr, 6, p.threads_per_row) - 3) + level_of(kRpc, 4, p.rows_per_cta) +
+    auto off_centre = [&](const rt_params& p) {
+        return 2 * abs(level_of(kTpr, 6, p.threads_per_row) - centre_level(s, p, p.vec_bytes)) + level_of(kRpc, 4, p.rows_per_cta) +
                level_of(kUnr, 3, p.unroll);
     };
     std::vector<int> order = coarse;
@@ -1056,7 +1071,7 @@ int run_search(const rt_shape& shape, const rt_limits& limits, const rt_budget& 
             if (st != RT_OK) return st;
             S.time_us[idx] = t;
         }
-        // 2. coarse grid, cut to half of what is left of the budget (mode by mode, nearest the middle first)
+        // 2. coarse grid, cut to half of what is left of the budget (mode by mode, nearest each mode's centre first)
         int widest[RT_STAGE_TMA_PIPELINE + 1] = {0, 0, 0, 0, 0};  // per stage: the ragged-row stage is wider than the others
         for (const rt_params& p : feasible) widest[p.stage] = std::max(widest[p.stage], p.vec_bytes);
         std::vector<int> coarse;
@@ -1067,12 +1082,12 @@ int run_search(const rt_shape& shape, const rt_limits& limits, const rt_budget& 
                 q.unroll = u;
                 if (S.index.find(pack_params(q)) != S.index.end()) deepest = false;
             }
-            if (on_coarse_grid(S.cand[i], widest[S.cand[i].stage], deepest)) coarse.push_back(i);
+            if (on_coarse_grid(shape, S.cand[i], widest[S.cand[i].stage], deepest)) coarse.push_back(i);
         }
         if (coarse.empty())
             for (int i = 0; i < (int)feasible.size(); ++i) coarse.push_back(i);
         const int grid_budget = std::max(1, (S.max_evals - top_k - S.used) / 2);
-        for (int idx : stratified(coarse, S.cand, grid_budget)) {
+        for (int idx : stratified(shape, coarse, S.cand, grid_budget)) {
             if (!S.budget_left(top_k)) break;
             if (S.time_us[idx] >= 0.f) continue;
             st = S.run(idx, RT_PHASE_GRID, &t);

@@ -153,8 +153,19 @@ def test_a_small_budget_still_touches_every_stage_and_reduction_mode(L):
     modes = [(r.params.stage, r.params.reduce) for r in grid]
     assert set(modes[:6]) == {(st, rd) for st in (0, 1, 2) for rd in (0, 1)}
     assert all(modes.count(m) == 2 for m in set(modes))
-    # the first point of every mode is the one nearest the middle of the ordered axes
-    assert all(r.params.threads_per_row == 256 and r.params.rows_per_cta == 1 and r.params.unroll == 1 for r in grid[:6])
+    # the first point of every mode is the one where a thread owns one vector of the row (8192 bf16 elements are 512
+    # vectors of 32 bytes), one row per CTA, unroll 1
+    assert all(r.params.threads_per_row == 512 and r.params.rows_per_cta == 1 and r.params.unroll == 1 for r in grid[:6])
+    # and the grid's levels of threads per row are every other one counted from there
+    assert {r.params.threads_per_row for r in grid} <= {128, 512}
+    # a row split over a cluster of 8 moves the centre with the slice: 768 vectors / 8 = 96 -> 128 threads; whole rows: 1024
+    s2 = B.shape_of(16, 12288, "bf16")
+    _, log2 = B.tuner_search_with(s2, L, B.make_budget(max_evals=60, top_k=5), _cost_factory(OPTIMA[0]))
+    first = {}
+    for r in log2:
+        if r.phase == 1:
+            first.setdefault((r.params.stage, r.params.reduce, r.params.cluster_size), r.params.threads_per_row)
+    assert first[(0, 2, 8)] == 128 and first[(0, 0, 1)] == 1024
 
 
 def test_an_optimum_two_steps_from_every_leader_is_reached_with_leftover_budget(L):
