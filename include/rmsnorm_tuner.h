@@ -397,7 +397,8 @@ int tuner_derive_counts(const rt_shape* s, const rt_limits* limits, int32_t heur
  * that is within 3 % of it, then around the three fastest and, while budget remains, up to the
  * twelve fastest), then a re-test of the top_k finalists ("Tuning agent": Top-K re-testing): they are
  * re-timed side by side as tuner_retest_interleaved does, each counts as one evaluation, the winner is the
- * fastest finalist that passes again, and a finalist that fails its re-test is replaced by the next runner-up
+ * fastest finalist that passes again (re-test times within 0.5 % of the fastest are a tie, which goes to the finalist
+ * that was faster when the search first timed it), and a finalist that fails its re-test is replaced by the next runner-up
  * while budget remains.
  * Every candidate passes the correctness gate (r_out bit-exact, y within 2 ulp for 16-bit types or
  * 1e-5 relative for fp32, against the uploaded references) before it is timed; candidates that

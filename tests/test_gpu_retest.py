@@ -70,7 +70,13 @@ def test_search_confirms_its_finalists_side_by_side(B, oracle_lib):
     # the winner is one of the confirmed finalists and carries its re-test time
     winners = [rec for rec in topk if rec.params.key() == res.best.key()]
     assert len(winners) == 1 and winners[0].us == pytest.approx(res.best_us)
-    assert res.best_us == pytest.approx(min(rec.us for rec in topk if rec.status == 0))
+    # it is the fastest of them, or within the 0.5 % that counts as a tie (which goes to the leader of the first ranking)
+    fastest = min(rec.us for rec in topk if rec.status == 0)
+    assert fastest <= res.best_us <= 1.005 * fastest * (1 + 1e-6)
+    if res.best_us > fastest * (1 + 1e-6):
+        first = {rec.params.key(): rec.us for rec in log if rec.phase != 3}
+        quickest = min((rec for rec in topk if rec.status == 0), key=lambda rec: rec.us)
+        assert first[res.best.key()] < first[quickest.params.key()]
 
 
 def test_alignment_is_taken_from_the_workspace_not_from_the_claim(B, oracle_lib):

@@ -286,3 +286,28 @@ def test_a_finalist_that_fails_its_retest_drops_out_and_the_runner_up_is_confirm
     res2, log2 = B.tuner_search_with(s, L, B.make_budget(max_evals=600, top_k=2), cost2)
     assert [r.status for r in log2 if r.phase == 3] == [B.RT_ERR_MISMATCH] * 4
     assert res2.best_us > 100.0 and always[res2.best.key()] == 1
+
+
+def test_a_photo_finish_in_the_retest_does_not_overturn_the_first_ranking(L):
+    """The optimum reads 4 % slow for the length of the re-test (the callback's evaluator scores a finalist by the mean
+    of its two times: 104.1 against the runner-up's 104.0).  Re-test times within 0.5 % are a tie, and a tie goes to the
+    finalist that led by the first measurement; a finalist that loses its re-test by more than that loses."""
+    s = B.shape_of(*SHAPE)
+    opt = OPTIMA[0]
+    base = _cost_factory(opt)
+
+    def is_opt(p):
+        return (p.threads_per_row, p.rows_per_cta, p.unroll, p.vec_bytes, p.stage, p.reduce) == \
+            (opt["tpr"], opt["rpc"], opt["unroll"], opt["vec"], opt["stage"], opt["reduce"])
+
+    for second, opt_wins in ((108.2, True), (112.0, False)):
+        seen = {}
+
+        def cost(p):
+            n = seen[p.key()] = seen.get(p.key(), 0) + 1
+            return second if is_opt(p) and n == 2 else base(p)
+        res, log = B.tuner_search_with(s, L, B.make_budget(max_evals=80, top_k=3), cost)
+        topk = [r for r in log if r.phase == 3]
+        assert is_opt(topk[0].params) and topk[0].us == pytest.approx(second) and topk[1].us == pytest.approx(104.0)
+        assert is_opt(res.best) == opt_wins, (second, res.best, res.best_us)
+        assert res.best_us == pytest.approx(0.5 * (100.0 + second) if opt_wins else 104.0)
